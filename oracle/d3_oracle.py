@@ -1,0 +1,392 @@
+"""CPU oracle for threshold-based masked-block diffusion decoding.
+
+TEST INFRASTRUCTURE ONLY.  Plain NumPy, written from the paper's description
+of the decoding loop; it shares no code with the CUDA path and must never be
+imported by the product package.  Only tests, the smoke check and the
+benchmark's CPU-baseline leg use it.
+
+What the paper fixes (cited per function) and what it leaves open
+-----------------------------------------------------------------
+* A diffusion LLM predicts every masked position of a block at once with a
+  bidirectional (non-causal) transformer (Sec. 1; Appendix "Combined with
+  SGLang", item (i)).
+* Generation proceeds block by block with a fixed block size (Appendix "More
+  Implementation Details", inference settings).
+* Each forward pass is followed by a decision: tokens whose confidence clears
+  a threshold are decoded in parallel (Sec. 2, the threshold paragraph), or,
+  in the entropy variant, tokens whose predictive entropy is below the
+  threshold, lower entropy first (Sec. 3.2, first paragraph).
+* At least one token is decoded per forward pass regardless of the threshold
+  (Sec. 3.2, the Fully-Activated state).
+* A finished block's key/value states enter the cache only after a further
+  forward pass over its final tokens (Sec. 3.2, "Completed but Stabilizing";
+  KV-cache paragraph: a short delay before caching).
+* Unmasking exactly one token per step is the teacher-trajectory mode
+  (Sec. 3.1; Appendix, pseudo-trajectory extraction).
+
+Readings taken where the paper is silent are listed in the repository's
+design notes; in short: block-causal visibility between segments (prompt =
+segment 0, generation block j = segment j), which makes the prefix cache
+exact; confidence = softmax probability of the arg-max token with the mask
+token excluded; strict comparisons (conf > tau, entropy < tau, nats); forced
+commit = most confident masked position, lowest index on ties; one finalize
+forward per block; rotate-half RoPE; RMSNorm with eps inside the root.
+
+Parity status: the decoding loop, decision rule, cache and every layer
+primitive are pinned by tests/test_oracle_*.py (closed forms, library
+routines, brute force).  The numeric values of the logits for the synthetic
+configurations are "parity unpinned" by the paper, which prints no per-step
+values; they are pinned only through those invariants and an independent
+torch-CPU forward.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+MODE_CONFIDENCE = 0  # commit if max-prob > tau
+MODE_ENTROPY = 1     # commit if entropy (nats) < tau
+
+
+# ----------------------------------------------------------------------------- number formats
+def bf16_bits_to_float(bits: np.ndarray, dtype=np.float32) -> np.ndarray:
+    """uint16 bf16 bit patterns -> floating point (exact)."""
+    return (bits.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(dtype, copy=False)
+
+
+def round_to_bf16(x: np.ndarray) -> np.ndarray:
+    """Round to the nearest bf16 value (ties to even), result in x's dtype."""
+    f = np.ascontiguousarray(x, dtype=np.float32)
+    u = f.view(np.uint32)
+    r = (u + np.uint32(0x7FFF) + ((u >> np.uint32(16)) & np.uint32(1))) & np.uint32(0xFFFF0000)
+    return r.view(np.float32).astype(x.dtype, copy=False)
+
+
+# ----------------------------------------------------------------------------- layer primitives
+def rms_norm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
+    """x / sqrt(mean(x^2) + eps) * gain over the last axis."""
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return x / np.sqrt(ms + eps) * gain
+
+
+def rope_tables(positions: np.ndarray, d_head: int, theta: float) -> Tuple[np.ndarray, np.ndarray]:
+    """cos/sin of position * theta^(-2k/d_head), k = 0..d_head/2-1, in float64: [n, d_head/2]."""
+    k = np.arange(d_head // 2, dtype=np.float64)
+    inv_freq = np.power(np.float64(theta), -2.0 * k / d_head)
+    ang = np.asarray(positions, dtype=np.float64)[:, None] * inv_freq[None, :]
+    return np.cos(ang), np.sin(ang)
+
+
+def apply_rope(x: np.ndarray, cos: np.ndarray, sin: np.ndarray) -> np.ndarray:
+    """Rotate-half RoPE.  x: [n, heads, d_head]; pairs are (k, k + d_head/2)."""
+    half = x.shape[-1] // 2
+    x1, x2 = x[..., :half], x[..., half:]
+    c, s = cos[:, None, :].astype(x.dtype), sin[:, None, :].astype(x.dtype)
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
+def silu(x: np.ndarray) -> np.ndarray:
+    return x / (1.0 + np.exp(-x))
+
+
+def softmax_rows(s: np.ndarray) -> np.ndarray:
+    m = np.max(s, axis=-1, keepdims=True)
+    e = np.exp(s - m)
+    return e / np.sum(e, axis=-1, keepdims=True)
+
+
+def attention(q: np.ndarray, k: np.ndarray, v: np.ndarray,
+              visible: Optional[np.ndarray] = None, round_probs_bf16: bool = False) -> np.ndarray:
+    """softmax(q k^T / sqrt(d_head)) v per head, no causal mask.
+
+    q: [n, hq, dh]; k, v: [L, hkv, dh]; query head h reads kv head h // (hq/hkv).
+    visible: optional bool [n, L]; False entries get probability 0."""
+    n, hq, dh = q.shape
+    hkv = k.shape[1]
+    group = hq // hkv
+    out = np.empty_like(q)
+    scale = 1.0 / np.sqrt(np.float64(dh))
+    for h in range(hq):
+        g = h // group
+        s = (q[:, h, :] @ k[:, g, :].T) * q.dtype.type(scale)
+        if visible is not None:
+            s = np.where(visible, s, -np.inf)
+        p = softmax_rows(s)
+        if round_probs_bf16:
+            p = round_to_bf16(p)
+        out[:, h, :] = p @ v[:, g, :]
+    return out
+
+
+def softmax_stats(logits: np.ndarray, mask_id: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Per row: probabilities with the mask token excluded, confidence = max prob,
+    token = arg max (lowest index on ties), entropy in nats.  Computed in float64."""
+    l = np.array(logits, dtype=np.float64, copy=True)
+    l[:, mask_id] = -np.inf
+    p = softmax_rows(l)
+    tok = np.argmax(l, axis=-1).astype(np.int32)  # first occurrence = lowest index
+    conf = p[np.arange(p.shape[0]), tok]
+    with np.errstate(divide="ignore", invalid="ignore"):
+        plogp = np.where(p > 0.0, p * np.log(p), 0.0)
+    ent = -np.sum(plogp, axis=-1)
+    return p, conf, tok, ent
+
+
+def decide(conf: np.ndarray, ent: np.ndarray, mask: np.ndarray, tau: float, mode: int = MODE_CONFIDENCE
+           ) -> np.ndarray:
+    """Which masked positions of one block are committed this step (bool [B]).
+
+    Every masked position clearing the threshold, plus always the single most confident
+    masked position (highest max-prob, or lowest entropy in entropy mode; lowest index on
+    ties).  A block without masked positions commits nothing."""
+    mask = np.asarray(mask, dtype=bool)
+    commit = np.zeros(mask.shape, dtype=bool)
+    if not mask.any():
+        return commit
+    if mode == MODE_CONFIDENCE:
+        commit = mask & (conf > tau)
+        score = np.where(mask, conf, -np.inf)
+        forced = int(np.argmax(score))
+    else:
+        commit = mask & (ent < tau)
+        score = np.where(mask, ent, np.inf)
+        forced = int(np.argmin(score))
+    commit[forced] = True
+    return commit
+
+
+# ----------------------------------------------------------------------------- model
+@dataclass
+class SeqState:
+    """Per-sequence cache: post-RoPE K and V of the committed prefix, per layer [L, hkv, dh]."""
+    k: List[np.ndarray]
+    v: List[np.ndarray]
+
+    @property
+    def prefix_len(self) -> int:
+        return int(self.k[0].shape[0])
+
+    def copy(self) -> "SeqState":
+        return SeqState([a.copy() for a in self.k], [a.copy() for a in self.v])
+
+
+class OracleModel:
+    """Pre-norm transformer without causal mask: RMSNorm, RoPE attention (MHA/GQA), SwiGLU FFN,
+    untied LM head, logits multiplied by ``logit_scale``.  No biases; norm gains default to 1.
+
+    ``weights``: {"tok_emb": [V,d], "lm_head": [V,d], "layers": {l: {"wq","wk","wv","wo",
+    "w_gate","w_up","w_down"}}}, each matrix [out, in], floating point or bf16 bits (uint16).
+    ``dtype`` is the arithmetic type.  ``mirror_bf16`` additionally rounds activations to bf16
+    where a bf16 pipeline stores them (normed input, q/k/v after RoPE, attention output, FFN
+    hidden) so that rounding can be told from errors; the residual stream is never rounded.
+    """
+
+    def __init__(self, *, n_layers: int, d_model: int, n_q_heads: int, n_kv_heads: int, d_head: int,
+                 d_ffn: int, vocab: int, mask_id: int, weights: Dict[str, object],
+                 rope_theta: float = 1.0e4, rms_eps: float = 1.0e-5, logit_scale: float = 20.0,
+                 dtype=np.float64, mirror_bf16: bool = False, gains: Optional[Dict[str, object]] = None):
+        self.n_layers, self.d_model = n_layers, d_model
+        self.n_q_heads, self.n_kv_heads, self.d_head = n_q_heads, n_kv_heads, d_head
+        self.d_ffn, self.vocab, self.mask_id = d_ffn, vocab, mask_id
+        self.rope_theta, self.rms_eps, self.logit_scale = rope_theta, rms_eps, logit_scale
+        self.dtype = np.dtype(dtype)
+        self.mirror = mirror_bf16
+        self.w = weights
+        self.gains = gains or {}
+
+    # -- helpers
+    def _mat(self, a: np.ndarray) -> np.ndarray:
+        if a.dtype == np.uint16:
+            return bf16_bits_to_float(a, self.dtype)
+        return a.astype(self.dtype, copy=False)
+
+    def _gain(self, name: str, layer: Optional[int] = None) -> np.ndarray:
+        g = self.gains.get((name, layer)) if layer is not None else self.gains.get(name)
+        if g is None:
+            return np.ones(self.d_model, dtype=self.dtype)
+        return np.asarray(g, dtype=self.dtype)
+
+    def _r(self, x: np.ndarray) -> np.ndarray:
+        return round_to_bf16(x) if self.mirror else x
+
+    def embed(self, ids: np.ndarray) -> np.ndarray:
+        return self._mat(np.asarray(self.w["tok_emb"])[np.asarray(ids, dtype=np.int64)])
+
+    # -- one layer
+    def layer_forward(self, layer: int, x: np.ndarray, positions: np.ndarray,
+                      k_prefix: Optional[np.ndarray], v_prefix: Optional[np.ndarray],
+                      visible: Optional[np.ndarray] = None
+                      ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+        """x: [n, d] rows at absolute ``positions``; keys/values = prefix cache followed by
+        these rows' own K/V.  Returns (x_out, k_rows, v_rows) with k_rows post-RoPE."""
+        W = self.w["layers"][layer]
+        n = x.shape[0]
+        hq, hkv, dh = self.n_q_heads, self.n_kv_heads, self.d_head
+        xn = self._r(rms_norm(x, self._gain("attn_norm", layer), self.rms_eps))
+        q = (xn @ self._mat(W["wq"]).T).reshape(n, hq, dh)
+        k = (xn @ self._mat(W["wk"]).T).reshape(n, hkv, dh)
+        v = (xn @ self._mat(W["wv"]).T).reshape(n, hkv, dh)
+        cos, sin = rope_tables(positions, dh, self.rope_theta)
+        q = self._r(apply_rope(q, cos, sin))
+        k = self._r(apply_rope(k, cos, sin))
+        v = self._r(v)
+        if k_prefix is not None and k_prefix.shape[0] > 0:
+            k_all = np.concatenate([k_prefix.astype(self.dtype, copy=False), k], axis=0)
+            v_all = np.concatenate([v_prefix.astype(self.dtype, copy=False), v], axis=0)
+        else:
+            k_all, v_all = k, v
+        o = self._r(attention(q, k_all, v_all, visible, round_probs_bf16=False))
+        x = x + o.reshape(n, hq * dh) @ self._mat(W["wo"]).T
+        xn = self._r(rms_norm(x, self._gain("ffn_norm", layer), self.rms_eps))
+        gate = xn @ self._mat(W["w_gate"]).T
+        up = xn @ self._mat(W["w_up"]).T
+        h = self._r(silu(gate) * up)
+        x = x + h @ self._mat(W["w_down"]).T
+        return x, k, v
+
+    def forward_rows(self, ids: np.ndarray, positions: np.ndarray, state: Optional[SeqState],
+                     visible: Optional[np.ndarray] = None
+                     ) -> Tuple[np.ndarray, List[np.ndarray], List[np.ndarray]]:
+        """All layers over the given rows against ``state``'s cache.  Returns the residual
+        stream after the last layer and the rows' per-layer K/V."""
+        x = self.embed(ids)
+        ks, vs = [], []
+        for l in range(self.n_layers):
+            kp = state.k[l] if state is not None else None
+            vp = state.v[l] if state is not None else None
+            x, k, v = self.layer_forward(l, x, positions, kp, vp, visible)
+            ks.append(k)
+            vs.append(v)
+        return x, ks, vs
+
+    def logits(self, x: np.ndarray) -> np.ndarray:
+        xn = self._r(rms_norm(x, self._gain("final_norm"), self.rms_eps))
+        return (xn @ self._mat(np.asarray(self.w["lm_head"])).T) * self.dtype.type(self.logit_scale)
+
+    # -- decoding path
+    def empty_state(self) -> SeqState:
+        z = lambda: np.zeros((0, self.n_kv_heads, self.d_head), dtype=self.dtype)
+        return SeqState([z() for _ in range(self.n_layers)], [z() for _ in range(self.n_layers)])
+
+    def prefill(self, prompt: np.ndarray) -> SeqState:
+        """Forward over the prompt alone (bidirectional within it); keep post-RoPE K and V."""
+        prompt = np.asarray(prompt)
+        if prompt.shape[0] == 0:
+            return self.empty_state()
+        _, ks, vs = self.forward_rows(prompt, np.arange(prompt.shape[0]), None)
+        return SeqState(ks, vs)
+
+    def denoise_forward(self, state: SeqState, block_ids: np.ndarray):
+        """One forward of the block's rows (masked rows hold mask_id) against the prefix cache.
+        Returns (logits [B, V], conf, tok, entropy)."""
+        B = len(block_ids)
+        pos = state.prefix_len + np.arange(B)
+        x, _, _ = self.forward_rows(np.asarray(block_ids), pos, state)
+        lg = self.logits(x)
+        _, conf, tok, ent = softmax_stats(lg, self.mask_id)
+        return lg, conf, tok, ent
+
+    def denoise_step(self, state: SeqState, block_ids: np.ndarray, mask: np.ndarray, tau: float,
+                     mode: int = MODE_CONFIDENCE):
+        """Forward + decision.  Returns (new_ids, new_mask, commit[bool B], conf, tok, entropy)."""
+        block_ids = np.array(block_ids, dtype=np.int32, copy=True)
+        mask = np.array(mask, dtype=bool, copy=True)
+        _, conf, tok, ent = self.denoise_forward(state, block_ids)
+        commit = decide(conf, ent, mask, tau, mode)
+        block_ids[commit] = tok[commit]
+        mask[commit] = False
+        return block_ids, mask, commit, conf, tok, ent
+
+    def finalize_block(self, state: SeqState, block_ids: np.ndarray) -> SeqState:
+        """Forward of the fully unmasked block; its K/V are appended to the cache."""
+        B = len(block_ids)
+        pos = state.prefix_len + np.arange(B)
+        _, ks, vs = self.forward_rows(np.asarray(block_ids), pos, state)
+        return SeqState([np.concatenate([a, b], axis=0) for a, b in zip(state.k, ks)],
+                        [np.concatenate([a, b], axis=0) for a, b in zip(state.v, vs)])
+
+    def generate(self, prompt: np.ndarray, gen_len: int, block: int, tau: float,
+                 mode: int = MODE_CONFIDENCE, record: bool = False) -> Dict[str, object]:
+        """Block-by-block threshold decoding of one sequence.
+
+        Returns tokens [gen_len], the step index (within its block, from 1) at which each
+        position was committed, forward counts, and optionally a per-step trace."""
+        assert gen_len % block == 0
+        state = self.prefill(prompt)
+        out = np.full(gen_len, self.mask_id, dtype=np.int32)
+        commit_step = np.zeros(gen_len, dtype=np.int32)
+        n_denoise = n_finalize = 0
+        trace: List[Dict[str, object]] = []
+        for j in range(gen_len // block):
+            ids = np.full(block, self.mask_id, dtype=np.int32)
+            mask = np.ones(block, dtype=bool)
+            step = 0
+            while mask.any():
+                step += 1
+                assert step <= block, "each step must remove at least one mask"
+                ids_in, mask_in = ids.copy(), mask.copy()
+                ids, mask, commit, conf, tok, ent = self.denoise_step(state, ids, mask, tau, mode)
+                n_denoise += 1
+                commit_step[j * block:(j + 1) * block][commit] = step
+                if record:
+                    trace.append(dict(block=j, step=step, prefix_len=state.prefix_len, ids_in=ids_in,
+                                      mask_in=mask_in, conf=conf, tok=tok, ent=ent, commit=commit,
+                                      ids_out=ids.copy(), mask_out=mask.copy()))
+            state = self.finalize_block(state, ids)
+            n_finalize += 1
+            out[j * block:(j + 1) * block] = ids
+        res = dict(tokens=out, commit_step=commit_step, n_denoise=n_denoise, n_finalize=n_finalize,
+                   tpf_denoise=gen_len / max(n_denoise, 1),
+                   tpf_all=gen_len / max(n_denoise + n_finalize, 1), state=state)
+        if record:
+            res["trace"] = trace
+        return res
+
+    # -- independent references used to pin the path above
+    def brute_force_block(self, prompt: np.ndarray, done_blocks: Sequence[np.ndarray],
+                          cur_block: np.ndarray):
+        """The same block forward with no cache: the whole sequence (prompt, finished blocks,
+        current block) goes through the stack under segment visibility seg(key) <= seg(query).
+        Returns (logits of the current block's rows, conf, tok, entropy)."""
+        segs = [np.asarray(prompt)] + [np.asarray(b) for b in done_blocks] + [np.asarray(cur_block)]
+        ids = np.concatenate(segs)
+        seg_id = np.concatenate([np.full(len(s), i) for i, s in enumerate(segs)])
+        visible = seg_id[None, :] <= seg_id[:, None]
+        x, _, _ = self.forward_rows(ids, np.arange(len(ids)), None, visible)
+        lg = self.logits(x[-len(cur_block):])
+        _, conf, tok, ent = softmax_stats(lg, self.mask_id)
+        return lg, conf, tok, ent
+
+    def sequential_decode(self, prompt: np.ndarray, gen_len: int, block: int) -> Tuple[np.ndarray, np.ndarray]:
+        """One token per forward pass: in each block, repeatedly run the block forward and unmask
+        only the masked position whose prediction is most probable.  Written separately from
+        ``generate``/``decide``.  Returns (tokens, order) where order[t] is the global position
+        unmasked at step t."""
+        state = self.prefill(prompt)
+        tokens = np.full(gen_len, self.mask_id, dtype=np.int32)
+        order = []
+        for j in range(gen_len // block):
+            ids = np.full(block, self.mask_id, dtype=np.int32)
+            for _ in range(block):
+                _, conf, tok, _ = self.denoise_forward(state, ids)
+                best, best_r = -1.0, -1
+                for r in range(block):
+                    if ids[r] == self.mask_id and conf[r] > best:
+                        best, best_r = conf[r], r
+                ids[best_r] = tok[best_r]
+                order.append(j * block + best_r)
+            state = self.finalize_block(state, ids)
+            tokens[j * block:(j + 1) * block] = ids
+        return tokens, np.asarray(order, dtype=np.int32)
+
+
+def model_from_shape(shape, weights: Dict[str, object], dtype=np.float64, mirror_bf16: bool = False
+                     ) -> OracleModel:
+    """Build an OracleModel from any object with the usual shape attributes."""
+    return OracleModel(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
+                       n_kv_heads=shape.n_kv_heads, d_head=shape.d_head, d_ffn=shape.d_ffn,
+                       vocab=shape.vocab, mask_id=shape.mask_id, weights=weights,
+                       rope_theta=shape.rope_theta, rms_eps=shape.rms_eps,
+                       logit_scale=shape.logit_scale, dtype=dtype, mirror_bf16=mirror_bf16)

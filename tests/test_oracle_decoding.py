@@ -1,0 +1,286 @@
+"""Pins for the oracle's decoding path: brute force, special cases, an independent torch forward."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+from oracle import d3_oracle as o
+from paper_2601_07568_b200 import synth_inputs as si
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+
+
+def paper_facts():
+    facts = {}
+    for line in open(os.path.join(HERE, "golden", "paper_facts.txt")):
+        line = line.split("#")[0].strip()
+        if line:
+            k, v = line.split("=")
+            facts[k.strip()] = float(v)
+    return facts
+
+
+def micro_model(seed=3, n_layers=2, d=32, hq=4, hkv=2, dh=8, f=48, V=40, scale=4.0, std=0.3):
+    """A tiny GQA model with larger weights so that confidences spread over (0,1)."""
+    rng = np.random.default_rng(seed)
+    lay = {}
+    for l in range(n_layers):
+        lay[l] = dict(wq=rng.normal(0, std, (hq * dh, d)), wk=rng.normal(0, std, (hkv * dh, d)),
+                      wv=rng.normal(0, std, (hkv * dh, d)), wo=rng.normal(0, std, (d, hq * dh)),
+                      w_gate=rng.normal(0, std, (f, d)), w_up=rng.normal(0, std, (f, d)),
+                      w_down=rng.normal(0, std, (d, f)))
+    W = dict(tok_emb=rng.normal(0, 1.0, (V, d)), lm_head=rng.normal(0, std / 4, (V, d)), layers=lay)
+    return o.OracleModel(n_layers=n_layers, d_model=d, n_q_heads=hq, n_kv_heads=hkv, d_head=dh, d_ffn=f,
+                         vocab=V, mask_id=V - 1, weights=W, logit_scale=scale, dtype=np.float64)
+
+
+@pytest.fixture(scope="module")
+def c1():
+    w = si.WORKLOADS["c1"]
+    W = si.gen_weights(w.model)
+    ids, lens = si.gen_prompts(w)
+    return w, o.model_from_shape(w.model, W, np.float64), ids[0, :lens[0]]
+
+
+# ----------------------------------------------------------------------------- independent forward
+def torch_forward(m: o.OracleModel, ids, visible=None):
+    """The same architecture written with torch CPU ops (float64), whole sequence, no cache."""
+    t = lambda a: torch.tensor(np.asarray(a, dtype=np.float64))
+    n = len(ids)
+    x = t(m.w["tok_emb"])[torch.tensor(np.asarray(ids), dtype=torch.long)]
+    half = m.d_head // 2
+    inv = torch.pow(torch.tensor(m.rope_theta, dtype=torch.float64),
+                    -torch.arange(0, m.d_head, 2, dtype=torch.float64) / m.d_head)
+    ang = torch.arange(n, dtype=torch.float64)[:, None] * inv[None, :]
+    rot = torch.polar(torch.ones_like(ang), ang)  # e^{i angle}
+
+    def rope(z):  # z: [n, h, dh]
+        zc = torch.complex(z[..., :half], z[..., half:]) * rot[:, None, :]
+        return torch.cat([zc.real, zc.imag], -1)
+
+    am = None if visible is None else torch.tensor(visible)
+    for l in range(m.n_layers):
+        W = m.w["layers"][l]
+        xn = F.rms_norm(x, (m.d_model,), None, m.rms_eps)
+        q = rope(F.linear(xn, t(W["wq"])).view(n, m.n_q_heads, m.d_head)).transpose(0, 1)
+        k = rope(F.linear(xn, t(W["wk"])).view(n, m.n_kv_heads, m.d_head)).transpose(0, 1)
+        v = F.linear(xn, t(W["wv"])).view(n, m.n_kv_heads, m.d_head).transpose(0, 1)
+        a = F.scaled_dot_product_attention(q[None], k[None], v[None], attn_mask=am, enable_gqa=True)[0]
+        x = x + F.linear(a.transpose(0, 1).reshape(n, -1), t(W["wo"]))
+        xn = F.rms_norm(x, (m.d_model,), None, m.rms_eps)
+        x = x + F.linear(F.silu(F.linear(xn, t(W["w_gate"]))) * F.linear(xn, t(W["w_up"])), t(W["w_down"]))
+    xn = F.rms_norm(x, (m.d_model,), None, m.rms_eps)
+    return (F.linear(xn, t(m.w["lm_head"])) * m.logit_scale).numpy()
+
+
+def test_forward_matches_independent_torch_model_c1(c1):
+    w, m, prompt = c1
+    ids = np.concatenate([prompt, np.full(w.block, m.mask_id)])
+    x, _, _ = m.forward_rows(ids, np.arange(len(ids)), None)
+    assert np.allclose(m.logits(x), torch_forward(m, ids), rtol=1e-9, atol=1e-9)
+
+
+def test_forward_matches_independent_torch_model_gqa_with_segments():
+    m = micro_model()
+    rng = np.random.default_rng(0)
+    ids = rng.integers(0, 38, size=14)
+    seg = np.array([0] * 6 + [1] * 4 + [2] * 4)
+    vis = seg[None, :] <= seg[:, None]
+    x, _, _ = m.forward_rows(ids, np.arange(14), None, vis)
+    assert np.allclose(m.logits(x), torch_forward(m, ids, vis), rtol=1e-9, atol=1e-9)
+
+
+# ----------------------------------------------------------------------------- cache == brute force
+@pytest.mark.parametrize("P", [0, 1, 5])
+def test_cached_prefix_equals_full_recompute(P):
+    m = micro_model()
+    rng = np.random.default_rng(P)
+    B = 4
+    prompt = rng.integers(0, 38, size=P)
+    state = m.prefill(prompt)
+    done = []
+    for j in range(3):
+        cur = np.full(B, m.mask_id)
+        cur[rng.integers(0, B)] = rng.integers(0, 38)  # a partly unmasked block
+        lg_c, conf_c, tok_c, ent_c = m.denoise_forward(state, cur)
+        lg_b, conf_b, tok_b, ent_b = m.brute_force_block(prompt, done, cur)
+        assert np.allclose(lg_c, lg_b, rtol=1e-11, atol=1e-11)
+        assert np.allclose(conf_c, conf_b, atol=1e-12) and np.array_equal(tok_c, tok_b)
+        final = rng.integers(0, 38, size=B)
+        state = m.finalize_block(state, final)
+        done.append(final)
+    assert state.prefix_len == P + 3 * B
+
+
+def test_cache_must_hold_final_tokens_not_masked_ones():
+    # If the cached K/V came from the last denoise forward (which still saw mask tokens), the next
+    # block would differ from the full recompute: the finalize forward is what makes the cache exact.
+    m = micro_model()
+    prompt = np.array([1, 2, 3])
+    state = m.prefill(prompt)
+    final = np.array([4, 5, 6, 7])
+    good = m.finalize_block(state, final)
+    stale = m.finalize_block(state, np.array([4, 5, m.mask_id, 7]))
+    cur = np.full(4, m.mask_id)
+    ref = m.brute_force_block(prompt, [final], cur)[0]
+    assert np.allclose(m.denoise_forward(good, cur)[0], ref, atol=1e-11)
+    assert not np.allclose(m.denoise_forward(stale, cur)[0], ref, atol=1e-3)
+
+
+def test_fully_unmasked_block_is_dense_bidirectional_attention():
+    # one segment only (no prompt): every row sees every row -> identical to the plain torch model
+    m = micro_model()
+    ids = np.array([3, 9, 1, 30, 22, 17])
+    lg = m.denoise_forward(m.empty_state(), ids)[0]
+    assert np.allclose(lg, torch_forward(m, ids), rtol=1e-9, atol=1e-9)
+    # and bidirectional: changing the LAST token changes the FIRST row's logits
+    ids2 = ids.copy()
+    ids2[-1] = 5
+    assert not np.allclose(m.denoise_forward(m.empty_state(), ids2)[0][0], lg[0], atol=1e-6)
+
+
+def test_later_segments_do_not_influence_earlier_ones():
+    m = micro_model()
+    prompt = np.array([1, 2, 3, 4])
+    a = m.brute_force_block(prompt, [], np.array([5, 6, 7]))[0]
+    x, _, _ = m.forward_rows(np.concatenate([prompt, [5, 6, 7], [8, 9, 10]]), np.arange(10), None,
+                             (np.array([0] * 4 + [1] * 3 + [2] * 3)[None, :]
+                              <= np.array([0] * 4 + [1] * 3 + [2] * 3)[:, None]))
+    assert np.allclose(m.logits(x[4:7]), a, atol=1e-11)
+
+
+# ----------------------------------------------------------------------------- decision rule
+def brute_decide(conf, ent, mask, tau, mode):
+    B = len(mask)
+    out = [False] * B
+    best = None
+    for r in range(B):
+        if not mask[r]:
+            continue
+        s = conf[r] if mode == 0 else -ent[r]
+        if (mode == 0 and conf[r] > tau) or (mode == 1 and ent[r] < tau):
+            out[r] = True
+        if best is None or s > best[0]:
+            best = (s, r)
+    if best is not None:
+        out[best[1]] = True
+    return np.array(out)
+
+
+def test_decide_matches_brute_force_on_all_small_cases():
+    rng = np.random.default_rng(1)
+    grid = [0.1, 0.5, 0.5, 0.9]  # repeated value -> ties
+    for mask in itertools.product([False, True], repeat=4):
+        for _ in range(8):
+            conf = rng.choice(grid, size=4)
+            ent = rng.choice(grid, size=4)
+            for tau in (0.05, 0.5, 0.7, 1.0):
+                for mode in (0, 1):
+                    got = o.decide(conf, ent, np.array(mask), tau, mode)
+                    assert np.array_equal(got, brute_decide(conf, ent, mask, tau, mode))
+                    assert not np.any(got & ~np.array(mask))
+                    assert got.any() == any(mask)
+
+
+def test_decide_strict_threshold_and_forced_commit():
+    conf = np.array([0.9, 0.95, 0.2, 0.9])
+    ent = np.zeros(4)
+    m = np.ones(4, bool)
+    assert list(o.decide(conf, ent, m, 0.9, 0)) == [False, True, False, False]  # 0.9 is not > 0.9
+    assert list(o.decide(conf, ent, m, 0.99, 0)) == [False, True, False, False]  # forced top-1
+    assert list(o.decide(conf, ent, np.array([1, 0, 1, 1], bool), 0.99, 0)) == [True, False, False, False]
+    assert list(o.decide(conf, ent, m, 0.1, 0)) == [True] * 4
+
+
+def test_commit_set_shrinks_as_threshold_rises(c1):
+    w, m, prompt = c1
+    mm = micro_model()
+    state = mm.prefill(np.array([1, 2, 3]))
+    ids = np.full(8, mm.mask_id)
+    _, conf, tok, ent = mm.denoise_forward(state, ids)
+    prev = None
+    for tau in np.linspace(0.0, 1.0, 21):
+        c = o.decide(conf, ent, np.ones(8, bool), tau, 0)
+        assert c.sum() >= 1
+        if prev is not None:
+            assert not np.any(c & ~prev)
+        prev = c
+
+
+# ----------------------------------------------------------------------------- whole loop
+def test_threshold_one_is_sequential_most_confident_first():
+    facts = paper_facts()
+    m = micro_model()
+    prompt = np.array([7, 8, 9, 10, 11])
+    r = m.generate(prompt, 16, 4, 1.0, record=True)
+    tok, order = m.sequential_decode(prompt, 16, 4)
+    assert np.array_equal(r["tokens"], tok)
+    assert all(t["commit"].sum() == facts["min_tokens_per_forward"] for t in r["trace"])
+    assert r["n_denoise"] == 16 and r["tpf_denoise"] == facts["tpf_one_token_per_step"]
+    got_order = [t["block"] * 4 + int(np.argmax(t["commit"])) for t in r["trace"]]
+    assert got_order == list(order)
+
+
+def test_threshold_one_c1_equals_sequential(c1):
+    w, m, prompt = c1
+    r = m.generate(prompt, w.gen_len, w.block, 1.0)
+    tok, _ = m.sequential_decode(prompt, w.gen_len, w.block)
+    assert np.array_equal(r["tokens"], tok)
+
+
+def test_tiny_threshold_commits_whole_block_in_one_step():
+    m = micro_model()
+    r = m.generate(np.array([1, 2, 3]), 12, 4, 1.0 / m.vocab - 1e-9)
+    assert r["n_denoise"] == 3 and r["tpf_denoise"] == 4.0 and r["n_finalize"] == 3
+
+
+def test_progress_and_step_bounds():
+    m = micro_model(seed=5)
+    for tau in (0.2, 0.5, 0.9):
+        r = m.generate(np.array([4, 4, 4, 4]), 24, 8, tau, record=True)
+        for t in r["trace"]:
+            assert t["mask_out"].sum() < t["mask_in"].sum()
+            assert t["step"] <= 8
+            assert np.array_equal(t["ids_out"][~t["mask_in"]], t["ids_in"][~t["mask_in"]])
+        assert np.all(r["tokens"] != m.mask_id) and np.all(r["commit_step"] >= 1)
+        assert r["n_finalize"] == 3
+
+
+def test_entropy_mode_runs_and_orders_by_entropy():
+    m = micro_model(seed=6)
+    r = m.generate(np.array([1, 2]), 8, 4, 0.45, mode=o.MODE_ENTROPY, record=True)
+    for t in r["trace"]:
+        masked = np.flatnonzero(t["mask_in"])
+        best = masked[np.argmin(t["ent"][masked])]
+        assert t["commit"][best]
+        assert np.array_equal(t["commit"][masked] & (masked != best), (t["ent"][masked] < 0.45) & (masked != best))
+
+
+def test_paper_block_arithmetic():
+    f = paper_facts()
+    assert f["max_generation_length"] / f["block_size"] == f["blocks_per_generation"]
+    w = si.WORKLOADS["c2"]
+    assert w.block == f["block_size"] and w.gen_len == f["max_generation_length"]
+
+
+def test_batch_elements_are_independent_and_deterministic(c1):
+    w, m, prompt = c1
+    a = m.generate(prompt, 32, 16, 0.3)
+    b = m.generate(prompt, 32, 16, 0.3)
+    assert np.array_equal(a["tokens"], b["tokens"]) and a["n_denoise"] == b["n_denoise"]
+
+
+def test_mirror_mode_stays_close_to_exact():
+    w = si.WORKLOADS["c1"]
+    shape = si.scaled_shape(si.LLADA8B, name="s", n_layers=2, d_model=128, n_q_heads=2, n_kv_heads=2,
+                            d_ffn=256, vocab=300, d_head=64)
+    W = si.gen_weights(shape)
+    ids = np.arange(20) % 290
+    a = o.model_from_shape(shape, W, np.float64)
+    b = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
+    la = a.denoise_forward(a.prefill(ids[:12]), ids[12:])[0]
+    lb = b.denoise_forward(b.prefill(ids[:12]), ids[12:])[0]
+    assert np.max(np.abs(la - lb)) < 3e-2 * np.max(np.abs(la))
