@@ -1,0 +1,201 @@
+/*
+ * d3.h -- C ABI of the masked-block denoising path of threshold-based
+ * diffusion-LLM decoding on one NVIDIA B200 (sm_100a).
+ *
+ * The operations follow the paper's statement of the decoding problem:
+ *   - a bidirectional transformer predicts every masked position of the
+ *     current block at once (Sec. 1; Appendix "Combined with SGLang" (i));
+ *   - generation runs block by block, block size fixed (Appendix "More
+ *     Implementation Details", inference settings);
+ *   - after each forward, tokens whose confidence clears a threshold are
+ *     unmasked in parallel (Sec. 2, threshold paragraph) or, in the entropy
+ *     variant, tokens whose entropy is below it (Sec. 3.2, first paragraph);
+ *   - at least one token is unmasked per forward (Sec. 3.2, Fully-Activated);
+ *   - a finished block is cached only after one more forward over its final
+ *     tokens (Sec. 3.2, "Completed but Stabilizing"; KV-cache paragraph).
+ *
+ * Conventions
+ *   - C linkage, no exceptions cross the boundary.  Every function returns
+ *     D3_OK (0) or a negative D3_ERR_* code; d3_strerror() names it and
+ *     d3_last_error() gives a longer per-context message.
+ *   - Pointers are marked [host] or [device].  A buffer passed in belongs to
+ *     the caller and must stay valid until the context's stream has finished
+ *     the call's work; everything the context allocates it frees in
+ *     d3_destroy().
+ *   - Calls enqueue work on the stream given to d3_create() and return
+ *     without waiting, except where stated (d3_generate, d3_load_weights,
+ *     d3_get_error_word).
+ *   - One context per host thread.  No global state.
+ *   - Matrices are row-major [out_features, in_features]; activations are
+ *     row-major [rows, features].  Token ids are int32.  Element type is
+ *     float (D3_DTYPE_F32) or bfloat16 (D3_DTYPE_BF16) as the config says.
+ *   - Visibility: the prompt is segment 0, generation block j is segment j;
+ *     a position attends to every position of its own and earlier segments
+ *     (no causal mask inside a segment).
+ */
+#ifndef D3_H_
+#define D3_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct d3_ctx d3_ctx;
+
+enum {
+  D3_OK = 0,
+  D3_ERR_INVALID_ARG = -1,    /* null pointer, non-finite threshold, negative size, ... */
+  D3_ERR_SHAPE = -2,          /* sizes exceed the configured maxima or break a divisibility rule */
+  D3_ERR_OOM = -3,            /* device allocation failed */
+  D3_ERR_CUDA = -4,           /* a CUDA runtime / driver call failed */
+  D3_ERR_DEVICE_TIMEOUT = -5, /* a bounded device-side wait gave up (see d3_get_error_word) */
+  D3_ERR_STATE = -6,          /* call out of order (e.g. step before prefill / load) */
+  D3_ERR_UNSUPPORTED = -7     /* configuration outside what the kernels handle */
+};
+
+enum { D3_DTYPE_F32 = 0, D3_DTYPE_BF16 = 1 };
+enum { D3_DECIDE_CONFIDENCE = 0, /* commit where max softmax probability > threshold */
+       D3_DECIDE_ENTROPY = 1 /* commit where entropy (nats) < threshold */ };
+enum { D3_GEMM_AUTO = 0,  /* bf16: tcgen05 tensor-core kernel; f32: SIMT kernel */
+       D3_GEMM_SIMT = 1 /* debugging: plain SIMT kernel for every matmul */ };
+
+typedef struct d3_config {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, d_head, d_ffn, vocab;
+  int32_t mask_id;      /* excluded from softmax/argmax; fills undecided positions */
+  float rope_theta;     /* rotate-half RoPE, angle = position * theta^(-2k/d_head) */
+  float rms_eps;        /* RMSNorm: x * rsqrt(mean(x^2) + eps) * gain */
+  float logit_scale;    /* logits = scale * (norm(x) . lm_head^T), applied in fp32 */
+  int32_t dtype;        /* D3_DTYPE_* : storage type of weights, activations and KV cache */
+  int32_t block;        /* block size B (1..128) */
+  int32_t max_batch;    /* largest batch any call will use */
+  int32_t max_seq;      /* cache slots per sequence: >= longest prompt + generated tokens */
+  int32_t max_prefill_rows; /* largest batch * padded prompt length passed to d3_prefill (0: max_batch*max_seq) */
+  int32_t decide_mode;  /* D3_DECIDE_* */
+  int32_t gemm_impl;    /* D3_GEMM_* */
+} d3_config;
+
+/* All pointers [host] or all [device] (see d3_load_weights).  Per-layer arrays have n_layers
+ * entries.  Norm gains may be NULL (= all ones).  Shapes: tok_emb, lm_head [vocab, d_model];
+ * wq [n_q_heads*d_head, d_model]; wk, wv [n_kv_heads*d_head, d_model]; wo [d_model,
+ * n_q_heads*d_head]; w_gate, w_up [d_ffn, d_model]; w_down [d_model, d_ffn]; gains [d_model]. */
+typedef struct d3_weights {
+  const void *tok_emb, *lm_head, *final_norm;
+  const void *const *attn_norm, *const *wq, *const *wk, *const *wv, *const *wo;
+  const void *const *ffn_norm, *const *w_gate, *const *w_up, *const *w_down;
+} d3_weights;
+
+typedef struct d3_stats {
+  int64_t denoise_forwards;  /* per-sequence denoise forwards, summed over the batch */
+  int64_t finalize_forwards; /* per-sequence finalize forwards, summed over the batch */
+  int64_t tokens_committed;
+  int64_t forced_commits;    /* commits that did not clear the threshold (the >=1 rule) */
+  int64_t steps;             /* batched forward passes launched by d3_generate */
+  int64_t kernel_launches;   /* kernels of this library launched by the call */
+  float prefill_ms, decode_ms; /* not filled by the library unless timing was requested */
+} d3_stats;
+
+/* Create a context on the current CUDA device.  cuda_stream is a cudaStream_t (NULL = default
+ * stream).  Allocates the KV cache [n_layers][2][max_batch][n_kv_heads][max_seq][d_head] and the
+ * activation workspaces.  Errors: INVALID_ARG, UNSUPPORTED (d_head not in {32,64,128}, odd sizes),
+ * OOM, CUDA. */
+int d3_create(const d3_config *cfg, void *cuda_stream, d3_ctx **out);
+void d3_destroy(d3_ctx *ctx);
+
+/* Copy the weights into context-owned device memory, repacked for the kernels (q,k,v rows
+ * concatenated; gate/up rows interleaved in groups of 64).  src_is_device: 0 = host pointers,
+ * 1 = device pointers.  Synchronises the stream before returning. */
+int d3_load_weights(d3_ctx *ctx, const d3_weights *w, int src_is_device);
+
+/* Prefill (KV-cache paragraph of Sec. 3.2): forward over each sequence's prompt alone and store the
+ * post-RoPE keys and the values of every layer in cache slots [0, len_i).  prompt_ids: [device]
+ * [bs, p_max] right-padded (pad value arbitrary but a valid id); prompt_lens: [device] [bs],
+ * 0 <= len_i <= p_max.  Resets the per-sequence prefix length to len_i.  Errors: SHAPE when
+ * bs > max_batch or p_max > max_seq or bs*p_max > max_prefill_rows; STATE before d3_load_weights. */
+int d3_prefill(d3_ctx *ctx, const int32_t *prompt_ids, const int32_t *prompt_lens, int32_t bs, int32_t p_max);
+
+/* One denoising step (Sec. 2 threshold decoding; Sec. 3.2 at-least-one rule): forward of the bs
+ * current blocks against the cached prefixes, softmax statistics over the vocabulary at every row
+ * (mask_id excluded), then per sequence commit every masked position with confidence > threshold
+ * (or entropy < threshold) and always the most confident masked position (lowest index on ties).
+ *   block_ids [device][bs, B] in/out: current ids, masked positions hold mask_id on entry;
+ *   mask      [device][bs, B] in/out: 1 = masked;
+ *   out_pos, out_ids [device][bs, B]: committed positions (ascending) and their ids, first
+ *   out_count[b] entries valid; out_count [device][bs].
+ * A block with no masked position commits nothing (count 0) and is left unchanged.  The cache is
+ * not modified beyond the scratch slots [prefix, prefix+B).  Errors: INVALID_ARG (NaN threshold,
+ * null pointers), SHAPE, STATE (before prefill). */
+int d3_denoise_step(d3_ctx *ctx, int32_t *block_ids, uint8_t *mask, float threshold, int32_t bs,
+                    int32_t *out_pos, int32_t *out_ids, int32_t *out_count);
+
+/* Finalize (Sec. 3.2 "Completed but Stabilizing", then "store its KV cache"): forward of the fully
+ * unmasked blocks without the LM head; their K/V stay in the cache and each prefix length grows
+ * by B.  block_ids [device][bs, B].  Errors: SHAPE when a prefix would exceed max_seq. */
+int d3_commit_block(d3_ctx *ctx, const int32_t *block_ids, int32_t bs);
+
+/* Whole decoding loop after d3_prefill: gen_len/B blocks per sequence, each starting fully masked;
+ * sequences advance independently (a sequence whose block is complete runs its finalize forward
+ * while others still denoise).  out_ids [device][bs, gen_len]; commit_step (may be NULL)
+ * [device][bs, gen_len]: 1-based step within its block at which each position was committed;
+ * host_stats [host] may be NULL.  Waits for the stream.  Errors: SHAPE when gen_len is not a
+ * multiple of B or prefix + gen_len > max_seq. */
+int d3_generate(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32_t *out_ids,
+                int32_t *commit_step, d3_stats *host_stats);
+
+/* Statistics of the latest denoise forward: conf, entropy [device][bs*B] float, argmax
+ * [device][bs*B] int32 (any may be NULL). */
+int d3_get_step_stats(d3_ctx *ctx, float *conf, float *entropy, int32_t *argmax, int32_t bs);
+
+/* Parity hooks.  d3_forward_logits runs the same forward as a denoise step but writes the scaled
+ * fp32 logits [device][bs*B, vocab] instead of reducing them (mask_id column left as computed).
+ * d3_set_tap selects a layer whose residual-stream input and output rows of the next forwards are
+ * kept (layer < 0: none); d3_read_tap copies them out as fp32 [rows, d_model].  d3_read_kv copies
+ * cache slots [pos0, pos0+n) of one layer and sequence as fp32 [n_kv_heads, n, d_head]. */
+int d3_forward_logits(d3_ctx *ctx, const int32_t *block_ids, int32_t bs, float *logits);
+int d3_set_tap(d3_ctx *ctx, int32_t layer);
+int d3_read_tap(d3_ctx *ctx, float *resid_in, float *resid_out, int32_t rows);
+int d3_read_kv(d3_ctx *ctx, int32_t layer, int32_t seq, int32_t pos0, int32_t n, float *k_out, float *v_out);
+
+/* Per-sequence prefix lengths ([device][bs]).  Setting them rewinds or advances the cache
+ * cursor; cache contents are untouched. */
+int d3_get_state(d3_ctx *ctx, int32_t *prefix_len, int32_t bs);
+int d3_set_state(d3_ctx *ctx, const int32_t *prefix_len, int32_t bs);
+
+/* Single operators through the same kernels the path uses (per-kernel parity tests).
+ * d3_op_linear: y = x . w^T.  x [device][m, k], w [device][n, k] in the context dtype;
+ *   epilogue 0: y fp32 [m, n];  1: y in context dtype [m, n];  2: y fp32 [m, n] += product
+ *   (residual);  3: w holds gate/up rows interleaved in groups of 64 (n = 2*f), y in context dtype
+ *   [m, f] = silu(gate) * up.   splits: split-K factor for the tensor-core kernel (0 = auto).
+ * d3_op_lm_head_stats: conf/entropy/argmax [device][m] of scale * x . w^T with mask_id excluded.
+ * d3_op_attention: q [device][bs*rows, n_q_heads*d_head]; keys/values are the context's cache of
+ *   `layer`; sequence b attends to its slots [0, kv_len[b]); out like q.  kv_len [device][bs].
+ * d3_op_unmask: the decision alone on caller-provided statistics. */
+int d3_op_linear(d3_ctx *ctx, const void *x, const void *w, void *y, int32_t m, int32_t n, int32_t k,
+                 int32_t epilogue, int32_t splits);
+int d3_op_lm_head_stats(d3_ctx *ctx, const void *x, const void *w, int32_t m, int32_t vocab, int32_t k,
+                        float scale, int32_t mask_id, float *conf, float *entropy, int32_t *argmax);
+int d3_op_attention(d3_ctx *ctx, const void *q, int32_t layer, int32_t bs, int32_t rows,
+                    const int32_t *kv_len, void *out);
+int d3_op_write_kv(d3_ctx *ctx, int32_t layer, int32_t seq, int32_t pos0, int32_t n, const float *k, const float *v);
+int d3_op_unmask(d3_ctx *ctx, const float *conf, const float *entropy, const int32_t *argmax,
+                 int32_t *block_ids, uint8_t *mask, float threshold, int32_t bs, int32_t *out_pos,
+                 int32_t *out_ids, int32_t *out_count);
+
+/* Device error word: 0 when no bounded wait has given up and no kernel saw an invalid index.
+ * Synchronises the stream.  Returns D3_OK and writes the word, or D3_ERR_CUDA. */
+int d3_get_error_word(d3_ctx *ctx, uint32_t *word);
+/* Number of this library's kernels launched on the context since creation. */
+int64_t d3_launch_count(d3_ctx *ctx);
+/* Bytes of device memory the context holds. */
+int64_t d3_device_bytes(d3_ctx *ctx);
+
+const char *d3_strerror(int code);
+const char *d3_last_error(d3_ctx *ctx);
+const char *d3_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* D3_H_ */

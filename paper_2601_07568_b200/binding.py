@@ -1,0 +1,298 @@
+"""ctypes binding of libd3.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (see include/d3.h) and does nothing
+but turn torch tensors into raw pointers and check the returned status.  All arithmetic of the
+decoding path runs in the CUDA kernels of the library; there is no CPU fallback: if the library
+cannot be loaded, or no CUDA device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libd3.so")
+
+D3_OK = 0
+D3_ERR_INVALID_ARG, D3_ERR_SHAPE, D3_ERR_OOM, D3_ERR_CUDA = -1, -2, -3, -4
+D3_ERR_DEVICE_TIMEOUT, D3_ERR_STATE, D3_ERR_UNSUPPORTED = -5, -6, -7
+D3_DTYPE_F32, D3_DTYPE_BF16 = 0, 1
+D3_DECIDE_CONFIDENCE, D3_DECIDE_ENTROPY = 0, 1
+D3_GEMM_AUTO, D3_GEMM_SIMT = 0, 1
+
+EXPORTS = [
+    "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
+    "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
+    "d3_get_state", "d3_set_state", "d3_op_linear", "d3_op_lm_head_stats", "d3_op_attention",
+    "d3_op_write_kv", "d3_op_unmask", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
+    "d3_strerror", "d3_last_error", "d3_version",
+]
+
+
+class d3_config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "d_head", "d_ffn",
+                                          "vocab", "mask_id")] + \
+               [(n, C.c_float) for n in ("rope_theta", "rms_eps", "logit_scale")] + \
+               [(n, C.c_int32) for n in ("dtype", "block", "max_batch", "max_seq", "max_prefill_rows",
+                                          "decide_mode", "gemm_impl")]
+
+
+class d3_weights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in ("tok_emb", "lm_head", "final_norm")] + \
+               [(n, C.POINTER(C.c_void_p)) for n in ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate",
+                                                     "w_up", "w_down")]
+
+
+class d3_stats(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in ("denoise_forwards", "finalize_forwards", "tokens_committed",
+                                          "forced_commits", "steps", "kernel_launches")] + \
+               [("prefill_ms", C.c_float), ("decode_ms", C.c_float)]
+
+
+class D3Error(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"d3 error {code}: {msg}")
+        self.code = code
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Load libd3.so (built in-tree by build.py).  Raises if it is missing."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2601_07568_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(LIB_PATH)
+        L.d3_strerror.restype = C.c_char_p
+        L.d3_last_error.restype = C.c_char_p
+        L.d3_last_error.argtypes = [C.c_void_p]
+        L.d3_version.restype = C.c_char_p
+        L.d3_launch_count.restype = C.c_int64
+        L.d3_launch_count.argtypes = [C.c_void_p]
+        L.d3_device_bytes.restype = C.c_int64
+        L.d3_device_bytes.argtypes = [C.c_void_p]
+        L.d3_destroy.restype = None
+        L.d3_destroy.argtypes = [C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _ptr(t: Optional[torch.Tensor]) -> C.c_void_p:
+    if t is None:
+        return C.c_void_p(0)
+    if not t.is_contiguous():
+        raise ValueError("tensor must be contiguous")
+    return C.c_void_p(t.data_ptr())
+
+
+def _dev(t: torch.Tensor, dtype=None) -> torch.Tensor:
+    if not t.is_cuda:
+        raise ValueError("expected a CUDA tensor")
+    if dtype is not None and t.dtype != dtype:
+        raise ValueError(f"expected dtype {dtype}, got {t.dtype}")
+    return t
+
+
+def _check(ctx, rc: int) -> None:
+    if rc != D3_OK:
+        L = lib()
+        detail = L.d3_last_error(ctx).decode() if ctx else ""
+        raise D3Error(rc, f"{L.d3_strerror(rc).decode()}: {detail}")
+
+
+# ----------------------------------------------------------------------------- C entry points
+def d3_create(cfg: d3_config, stream: Optional[torch.cuda.Stream] = None) -> C.c_void_p:
+    if not torch.cuda.is_available():
+        raise RuntimeError("d3 needs a CUDA device (no CPU fallback)")
+    ctx = C.c_void_p(0)
+    s = C.c_void_p(stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream)
+    rc = lib().d3_create(C.byref(cfg), s, C.byref(ctx))
+    if rc != D3_OK:
+        raise D3Error(rc, lib().d3_strerror(rc).decode())
+    return ctx
+
+
+def d3_destroy(ctx) -> None:
+    lib().d3_destroy(ctx)
+
+
+def d3_load_weights(ctx, tensors: Dict[str, object], n_layers: int) -> None:
+    """tensors: {"tok_emb", "lm_head", optional "final_norm", "layers": [ {wq, wk, wv, wo, w_gate, w_up,
+    w_down, optional attn_norm, ffn_norm} ]}; all on the host or all on the device."""
+    first = tensors["tok_emb"]
+    on_dev = bool(first.is_cuda)
+    keep = []
+
+    def p(t):
+        if t is None:
+            return None
+        if bool(t.is_cuda) != on_dev:
+            raise ValueError("all weights must live on the same side (host or device)")
+        t = t.contiguous()
+        keep.append(t)
+        return t.data_ptr()
+
+    w = d3_weights()
+    w.tok_emb, w.lm_head, w.final_norm = p(tensors["tok_emb"]), p(tensors["lm_head"]), p(tensors.get("final_norm"))
+    layers = tensors["layers"]
+    arrays = {}
+    for name in ("attn_norm", "wq", "wk", "wv", "wo", "ffn_norm", "w_gate", "w_up", "w_down"):
+        arr = (C.c_void_p * n_layers)()
+        for l in range(n_layers):
+            arr[l] = p(layers[l].get(name))
+        arrays[name] = arr
+        setattr(w, name, C.cast(arr, C.POINTER(C.c_void_p)))
+    _check(ctx, lib().d3_load_weights(ctx, C.byref(w), C.c_int(1 if on_dev else 0)))
+
+
+def d3_prefill(ctx, prompt_ids: torch.Tensor, prompt_lens: torch.Tensor) -> None:
+    bs, p_max = prompt_ids.shape
+    _check(ctx, lib().d3_prefill(ctx, _ptr(_dev(prompt_ids, torch.int32)), _ptr(_dev(prompt_lens, torch.int32)),
+                                 C.c_int32(bs), C.c_int32(p_max)))
+
+
+def d3_denoise_step(ctx, block_ids: torch.Tensor, mask: torch.Tensor, threshold: float, out_pos: torch.Tensor,
+                    out_ids: torch.Tensor, out_count: torch.Tensor) -> None:
+    bs = block_ids.shape[0]
+    _check(ctx, lib().d3_denoise_step(ctx, _ptr(_dev(block_ids, torch.int32)), _ptr(_dev(mask, torch.uint8)),
+                                      C.c_float(threshold), C.c_int32(bs), _ptr(_dev(out_pos, torch.int32)),
+                                      _ptr(_dev(out_ids, torch.int32)), _ptr(_dev(out_count, torch.int32))))
+
+
+def d3_commit_block(ctx, block_ids: torch.Tensor) -> None:
+    _check(ctx, lib().d3_commit_block(ctx, _ptr(_dev(block_ids, torch.int32)), C.c_int32(block_ids.shape[0])))
+
+
+def d3_generate(ctx, gen_len: int, threshold: float, out_ids: torch.Tensor,
+                commit_step: Optional[torch.Tensor] = None) -> d3_stats:
+    st = d3_stats()
+    bs = out_ids.shape[0]
+    _check(ctx, lib().d3_generate(ctx, C.c_int32(gen_len), C.c_float(threshold), C.c_int32(bs),
+                                  _ptr(_dev(out_ids, torch.int32)),
+                                  _ptr(_dev(commit_step, torch.int32)) if commit_step is not None else C.c_void_p(0),
+                                  C.byref(st)))
+    return st
+
+
+def d3_get_step_stats(ctx, conf: torch.Tensor, entropy: torch.Tensor, argmax: torch.Tensor, bs: int) -> None:
+    _check(ctx, lib().d3_get_step_stats(ctx, _ptr(_dev(conf, torch.float32)), _ptr(_dev(entropy, torch.float32)),
+                                        _ptr(_dev(argmax, torch.int32)), C.c_int32(bs)))
+
+
+def d3_forward_logits(ctx, block_ids: torch.Tensor, logits: torch.Tensor) -> None:
+    _check(ctx, lib().d3_forward_logits(ctx, _ptr(_dev(block_ids, torch.int32)), C.c_int32(block_ids.shape[0]),
+                                        _ptr(_dev(logits, torch.float32))))
+
+
+def d3_set_tap(ctx, layer: int) -> None:
+    _check(ctx, lib().d3_set_tap(ctx, C.c_int32(layer)))
+
+
+def d3_read_tap(ctx, resid_in: torch.Tensor, resid_out: torch.Tensor, rows: int) -> None:
+    _check(ctx, lib().d3_read_tap(ctx, _ptr(_dev(resid_in, torch.float32)), _ptr(_dev(resid_out, torch.float32)),
+                                  C.c_int32(rows)))
+
+
+def d3_read_kv(ctx, layer: int, seq: int, pos0: int, n: int, k_out: torch.Tensor, v_out: torch.Tensor) -> None:
+    _check(ctx, lib().d3_read_kv(ctx, C.c_int32(layer), C.c_int32(seq), C.c_int32(pos0), C.c_int32(n),
+                                 _ptr(_dev(k_out, torch.float32)), _ptr(_dev(v_out, torch.float32))))
+
+
+def d3_get_state(ctx, prefix_len: torch.Tensor) -> None:
+    _check(ctx, lib().d3_get_state(ctx, _ptr(_dev(prefix_len, torch.int32)), C.c_int32(prefix_len.numel())))
+
+
+def d3_set_state(ctx, prefix_len: torch.Tensor) -> None:
+    _check(ctx, lib().d3_set_state(ctx, _ptr(_dev(prefix_len, torch.int32)), C.c_int32(prefix_len.numel())))
+
+
+def d3_op_linear(ctx, x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, epilogue: int, splits: int = 0) -> None:
+    m, k = x.shape
+    n = w.shape[0]
+    _check(ctx, lib().d3_op_linear(ctx, _ptr(_dev(x)), _ptr(_dev(w)), _ptr(_dev(y)), C.c_int32(m), C.c_int32(n),
+                                   C.c_int32(k), C.c_int32(epilogue), C.c_int32(splits)))
+
+
+def d3_op_lm_head_stats(ctx, x: torch.Tensor, w: torch.Tensor, scale: float, mask_id: int, conf: torch.Tensor,
+                        entropy: torch.Tensor, argmax: torch.Tensor) -> None:
+    m, k = x.shape
+    _check(ctx, lib().d3_op_lm_head_stats(ctx, _ptr(_dev(x)), _ptr(_dev(w)), C.c_int32(m), C.c_int32(w.shape[0]),
+                                          C.c_int32(k), C.c_float(scale), C.c_int32(mask_id),
+                                          _ptr(_dev(conf, torch.float32)), _ptr(_dev(entropy, torch.float32)),
+                                          _ptr(_dev(argmax, torch.int32))))
+
+
+def d3_op_attention(ctx, q: torch.Tensor, layer: int, bs: int, rows: int, kv_len: torch.Tensor,
+                    out: torch.Tensor) -> None:
+    _check(ctx, lib().d3_op_attention(ctx, _ptr(_dev(q)), C.c_int32(layer), C.c_int32(bs), C.c_int32(rows),
+                                      _ptr(_dev(kv_len, torch.int32)), _ptr(_dev(out))))
+
+
+def d3_op_write_kv(ctx, layer: int, seq: int, pos0: int, k: torch.Tensor, v: torch.Tensor) -> None:
+    n = k.shape[1]
+    _check(ctx, lib().d3_op_write_kv(ctx, C.c_int32(layer), C.c_int32(seq), C.c_int32(pos0), C.c_int32(n),
+                                     _ptr(_dev(k, torch.float32)), _ptr(_dev(v, torch.float32))))
+
+
+def d3_op_unmask(ctx, conf: torch.Tensor, entropy: torch.Tensor, argmax: torch.Tensor, block_ids: torch.Tensor,
+                 mask: torch.Tensor, threshold: float, out_pos: torch.Tensor, out_ids: torch.Tensor,
+                 out_count: torch.Tensor) -> None:
+    _check(ctx, lib().d3_op_unmask(ctx, _ptr(_dev(conf, torch.float32)), _ptr(_dev(entropy, torch.float32)),
+                                   _ptr(_dev(argmax, torch.int32)), _ptr(_dev(block_ids, torch.int32)),
+                                   _ptr(_dev(mask, torch.uint8)), C.c_float(threshold),
+                                   C.c_int32(block_ids.shape[0]), _ptr(_dev(out_pos, torch.int32)),
+                                   _ptr(_dev(out_ids, torch.int32)), _ptr(_dev(out_count, torch.int32))))
+
+
+def d3_get_error_word(ctx) -> int:
+    w = C.c_uint32(0)
+    _check(ctx, lib().d3_get_error_word(ctx, C.byref(w)))
+    return int(w.value)
+
+
+def d3_launch_count(ctx) -> int:
+    return int(lib().d3_launch_count(ctx))
+
+
+def d3_device_bytes(ctx) -> int:
+    return int(lib().d3_device_bytes(ctx))
+
+
+def d3_version() -> str:
+    return lib().d3_version().decode()
+
+
+# ----------------------------------------------------------------------------- convenience
+def make_config(shape, *, block: int, max_batch: int, max_seq: int, max_prefill_rows: int = 0,
+                decide_mode: int = D3_DECIDE_CONFIDENCE, gemm_impl: int = D3_GEMM_AUTO) -> d3_config:
+    """d3_config from any object with the usual model-shape attributes."""
+    cfg = d3_config()
+    cfg.n_layers, cfg.d_model = shape.n_layers, shape.d_model
+    cfg.n_q_heads, cfg.n_kv_heads, cfg.d_head = shape.n_q_heads, shape.n_kv_heads, shape.d_head
+    cfg.d_ffn, cfg.vocab, cfg.mask_id = shape.d_ffn, shape.vocab, shape.mask_id
+    cfg.rope_theta, cfg.rms_eps, cfg.logit_scale = shape.rope_theta, shape.rms_eps, shape.logit_scale
+    cfg.dtype = D3_DTYPE_BF16 if shape.dtype == "bf16" else D3_DTYPE_F32
+    cfg.block, cfg.max_batch, cfg.max_seq = block, max_batch, max_seq
+    cfg.max_prefill_rows = max_prefill_rows
+    cfg.decide_mode, cfg.gemm_impl = decide_mode, gemm_impl
+    return cfg
+
+
+def weights_from_numpy(shape, weights: Dict[str, object], pin: bool = False) -> Dict[str, object]:
+    """Wrap generator output (fp32 arrays or bf16 bit patterns) as host torch tensors, without copies."""
+    import numpy as np
+
+    def t(a):
+        a = np.ascontiguousarray(a)
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
+        return torch.from_numpy(a)
+
+    return {"tok_emb": t(weights["tok_emb"]), "lm_head": t(weights["lm_head"]),
+            "layers": [{k: t(v) for k, v in weights["layers"][l].items()} for l in range(shape.n_layers)]}

@@ -1,0 +1,85 @@
+// Shared declarations of the d3 CUDA library: element types, epilogue codes, device error word.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace d3 {
+
+// ---- device error word bits (read back through d3_get_error_word)
+enum : uint32_t {
+  ERRW_MBAR_TIMEOUT = 1u << 0,   // a bounded mbarrier wait gave up
+  ERRW_BAD_TOKEN_ID = 1u << 1,   // a token id outside [0, vocab)
+  ERRW_BAD_POSITION = 1u << 2,   // a cache slot outside [0, max_seq)
+  ERRW_TMEM_ALLOC = 1u << 3,     // tensor-memory allocation returned an unexpected address
+};
+
+// ---- matmul epilogues
+enum : int {
+  EPI_F32 = 0,     // y fp32 [m, n] = acc * scale
+  EPI_T = 1,       // y T [m, n] = acc
+  EPI_RESID = 2,   // y fp32 [m, n] += acc
+  EPI_SWIGLU = 3,  // y T [m, n/2]: columns come in groups of 128 = 64 gate then 64 up
+  EPI_STATS = 4,   // per (row, 128-column tile): (max, sum exp, sum exp*(l-max), argmax) of scale*acc
+  EPI_QKV = 5,     // RoPE on q and k heads (d_head = 128 = one tile), q -> y T, k/v -> cache
+};
+
+struct EpiParams {
+  void* y = nullptr;          // output (meaning depends on the epilogue)
+  int ldy = 0;                // leading dimension of y in elements
+  float scale = 1.0f;         // EPI_F32 / EPI_STATS
+  int mask_id = -1;           // EPI_STATS: excluded column
+  float4* stat_part = nullptr;  // EPI_STATS: [m][n_tiles]
+  int n_tiles = 0;
+};
+
+template <typename T> struct TypeOps;
+template <> struct TypeOps<float> {
+  static __device__ __forceinline__ float to_f(float v) { return v; }
+  static __device__ __forceinline__ float from_f(float v) { return v; }
+};
+template <> struct TypeOps<__nv_bfloat16> {
+  static __device__ __forceinline__ float to_f(__nv_bfloat16 v) { return __bfloat162float(v); }
+  static __device__ __forceinline__ __nv_bfloat16 from_f(float v) { return __float2bfloat16_rn(v); }
+};
+
+__device__ __forceinline__ float silu_f(float g) { return g / (1.0f + __expf(-g)); }
+
+// Running softmax statistics of a set of logits: m = max, z = sum e^(l-m), s = sum e^(l-m)(l-m),
+// a = lowest index attaining m.  Empty set: m = -inf, z = s = 0, a = INT_MAX.
+struct SoftStat {
+  float m, z, s;
+  int a;
+};
+__device__ __forceinline__ SoftStat stat_empty() { return SoftStat{-INFINITY, 0.f, 0.f, 0x7fffffff}; }
+// Merge b into a.  Associative up to rounding; ties on the maximum keep the lower index.
+__device__ __forceinline__ SoftStat stat_merge(const SoftStat& a, const SoftStat& b) {
+  if (b.z == 0.f) return a;
+  if (a.z == 0.f) return b;
+  SoftStat r;
+  r.m = fmaxf(a.m, b.m);
+  float da = a.m - r.m, db = b.m - r.m;  // <= 0
+  float ea = __expf(da), eb = __expf(db);
+  r.z = ea * a.z + eb * b.z;
+  r.s = ea * (a.s + da * a.z) + eb * (b.s + db * b.z);
+  r.a = (a.m > b.m) ? a.a : (b.m > a.m) ? b.a : min(a.a, b.a);
+  return r;
+}
+__device__ __forceinline__ void stat_add(SoftStat& st, float l, int idx) {
+  if (l > st.m) {
+    float d = st.m - l;  // < 0 (or -inf when empty)
+    float e = (st.z == 0.f) ? 0.f : __expf(d);
+    st.s = (st.z == 0.f) ? 0.f : e * (st.s + d * st.z);
+    st.z = e * st.z + 1.0f;
+    st.m = l;
+    st.a = idx;
+  } else {
+    float d = l - st.m;  // <= 0
+    float e = __expf(d);
+    st.z += e;
+    st.s += e * d;
+    // equal maxima: indices are visited in ascending order, so the first one stays
+  }
+}
+
+}  // namespace d3

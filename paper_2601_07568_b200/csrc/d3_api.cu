@@ -1,0 +1,871 @@
+// C ABI of the d3 library (see include/d3.h): context, weight repacking, the forward pass as a
+// sequence of kernel launches on one stream, the decision kernels and the generate loop.
+#include "../../include/d3.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+#include "small_kernels.cuh"
+
+using namespace d3;
+typedef __nv_bfloat16 bf16;
+
+// ----------------------------------------------------------------------------- context
+struct d3_ctx {
+  d3_config cfg{};
+  cudaStream_t stream = nullptr;
+  bool is_bf16 = false;
+  bool use_tc = false;
+  bool fuse_qkv = false;
+  size_t esz = 4;
+  int n_sms = 148;
+  // weights (context dtype), repacked
+  void* tok_emb = nullptr;
+  void* lm_head = nullptr;
+  float* final_norm = nullptr;
+  std::vector<void*> wqkv, wo, wgu, wd;
+  std::vector<float*> attn_norm, ffn_norm;
+  bool weights_loaded = false, prefilled = false;
+  // cache and tables
+  void* kv = nullptr;
+  size_t kv_layer_elems = 0;  // elements of one K (or V) plane of one layer
+  float *rope_cos = nullptr, *rope_sin = nullptr;
+  // workspaces
+  int max_rows = 0;
+  float* x = nullptr;
+  void* xn = nullptr;
+  float* qkv_f32 = nullptr;
+  void* q = nullptr;
+  void* o = nullptr;
+  void* h = nullptr;
+  float4* stat_part = nullptr;
+  float *conf = nullptr, *ent = nullptr;
+  int* argmax = nullptr;
+  int *prefix_len = nullptr, *pos_base = nullptr, *n_valid = nullptr, *kv_len = nullptr;
+  uint32_t* error_word = nullptr;
+  float* partial = nullptr;
+  size_t partial_slots = 0;  // capacity in (tile, split) slots of 128*128 floats
+  int* tile_count = nullptr;
+  int n_tile_count = 0;
+  // generate state
+  GenState gen{};
+  long long* host_counters = nullptr;  // pinned
+  // taps
+  int tap_layer = -1;
+  float *tap_in = nullptr, *tap_out = nullptr;
+  int tap_rows = 0;
+  int last_rows = 0;
+  int64_t launches = 0;
+  int64_t dev_bytes = 0;
+  std::string last_error;
+  std::vector<void*> allocs;
+  std::map<std::tuple<const void*, int, int, int>, CUtensorMap> tmaps;
+};
+
+namespace {
+
+const char* kVersion = "d3-b200 0.1";
+
+int fail(d3_ctx* c, int code, const std::string& msg) {
+  if (c) c->last_error = msg;
+  return code;
+}
+#define CUDA_TRY(c, expr)                                                                         \
+  do {                                                                                            \
+    cudaError_t e_ = (expr);                                                                      \
+    if (e_ != cudaSuccess)                                                                        \
+      return fail((c), e_ == cudaErrorMemoryAllocation ? D3_ERR_OOM : D3_ERR_CUDA,                \
+                  std::string(#expr) + ": " + cudaGetErrorString(e_));                            \
+  } while (0)
+
+int dev_alloc(d3_ctx* c, void** p, size_t bytes, bool zero = true) {
+  if (bytes == 0) bytes = 16;
+  cudaError_t e = cudaMalloc(p, bytes);
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return fail(c, D3_ERR_OOM, "cudaMalloc of " + std::to_string(bytes) + " bytes: " + cudaGetErrorString(e));
+  }
+  c->allocs.push_back(*p);
+  c->dev_bytes += static_cast<int64_t>(bytes);
+  if (zero) {
+    e = cudaMemsetAsync(*p, 0, bytes, c->stream);
+    if (e != cudaSuccess) return fail(c, D3_ERR_CUDA, std::string("cudaMemsetAsync: ") + cudaGetErrorString(e));
+  }
+  return D3_OK;
+}
+#define ALLOC(c, ptr, bytes)                                                     \
+  do {                                                                           \
+    int rc_ = dev_alloc((c), reinterpret_cast<void**>(&(ptr)), (bytes));         \
+    if (rc_ != D3_OK) return rc_;                                                \
+  } while (0)
+
+int check_launch(d3_ctx* c, const char* what) {
+  c->launches++;
+  cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) {
+    (void)cudaGetLastError();
+    return fail(c, D3_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+  }
+  return D3_OK;
+}
+#define LAUNCHED(c, what)                    \
+  do {                                       \
+    int rc_ = check_launch((c), (what));     \
+    if (rc_ != D3_OK) return rc_;            \
+  } while (0)
+#define TRY(expr)                  \
+  do {                             \
+    int rc_ = (expr);              \
+    if (rc_ != D3_OK) return rc_;  \
+  } while (0)
+
+// ---- tensor maps (driver entry point fetched through the runtime: no link against libcuda)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  }
+  return fn;
+}
+
+// bf16 row-major [rows, cols] matrix, box = [box_rows, 64 columns], 128-byte swizzle, zero fill.
+int get_tmap(d3_ctx* c, const void* ptr, int rows, int cols, int box_rows, const CUtensorMap** out) {
+  auto key = std::make_tuple(ptr, rows, cols, box_rows);
+  auto it = c->tmaps.find(key);
+  if (it != c->tmaps.end()) {
+    *out = &it->second;
+    return D3_OK;
+  }
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return fail(c, D3_ERR_CUDA, "cuTensorMapEncodeTiled entry point not found");
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) != 0 || (cols % 8) != 0)
+    return fail(c, D3_ERR_UNSUPPORTED, "tensor-core matmul needs 16-byte aligned operands and K % 8 == 0");
+  CUtensorMap m;
+  cuuint64_t gdim[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  cuuint64_t gstr[1] = {static_cast<cuuint64_t>(cols) * 2};
+  cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstr, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) return fail(c, D3_ERR_CUDA, "cuTensorMapEncodeTiled failed with " + std::to_string(r));
+  if (c->tmaps.size() > 4096) c->tmaps.clear();
+  auto ins = c->tmaps.emplace(key, m);
+  *out = &ins.first->second;
+  return D3_OK;
+}
+
+// ---- matmul dispatch
+struct QkvExtra {
+  RowMap rm;
+  void* k_cache;
+  void* v_cache;
+};
+
+template <int EPI>
+int launch_tc(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, dim3 grid,
+              size_t smem) {
+  auto kern = tc::gemm_tc_kernel<EPI, 128>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    attr_set = true;
+  }
+  kern<<<grid, tc::NUM_THREADS, smem, c->stream>>>(*tx, *tw, p);
+  LAUNCHED(c, "gemm_tc_kernel");
+  return D3_OK;
+}
+
+int pick_splits(const d3_ctx* c, int m_tiles, int n_tiles, int k_chunks, int epi, int hint) {
+  if (epi == EPI_STATS) return 1;
+  int tiles = m_tiles * n_tiles;
+  int s = hint;
+  if (s <= 0) {
+    s = 1;
+    const int target = 2 * c->n_sms;
+    if (tiles < target) s = (target + tiles - 1) / tiles;
+    int cap = k_chunks / 4;  // keep at least four 64-wide K slabs per split
+    if (cap < 1) cap = 1;
+    if (s > cap) s = cap;
+    if (s > 16) s = 16;
+  }
+  if (s > k_chunks) s = k_chunks;
+  if (s < 1) s = 1;
+  while (s > 1 && static_cast<size_t>(tiles) * s > c->partial_slots) --s;
+  if (tiles > c->n_tile_count) s = 1;
+  return s;
+}
+
+int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
+                  int splits_hint, const QkvExtra* qx) {
+  const int BLOCK_N = 128;
+  const int m_tiles = (M + 127) / 128, n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
+  const int k_chunks = (K + 63) / 64;
+  int a_rows = M >= 128 ? 128 : ((M + 31) / 32) * 32;
+  tc::GemmParams p{};
+  p.M = M; p.N = N; p.K = K;
+  p.a_rows = a_rows;
+  p.splits = pick_splits(c, m_tiles, n_tiles, k_chunks, epi, splits_hint);
+  const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + BLOCK_N * 128;
+  int stages = static_cast<int>((100 * 1024) / stage_bytes);
+  if (stages > 8) stages = 8;
+  if (stages < 2) stages = 2;
+  p.stages = stages;
+  p.partial = c->partial;
+  p.tile_count = c->tile_count;
+  p.error_word = c->error_word;
+  p.ep = ep;
+  if (qx) {
+    p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
+    p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
+    p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
+    p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
+  }
+  const CUtensorMap *tx, *tw;
+  TRY(get_tmap(c, X, M, K, a_rows, &tx));
+  TRY(get_tmap(c, W, N, K, BLOCK_N, &tw));
+  dim3 grid(m_tiles, n_tiles, p.splits);
+  size_t smem = tc::gemm_tc_smem_bytes(a_rows, BLOCK_N, stages);
+  switch (epi) {
+    case EPI_F32: return launch_tc<EPI_F32>(c, tx, tw, p, grid, smem);
+    case EPI_T: return launch_tc<EPI_T>(c, tx, tw, p, grid, smem);
+    case EPI_RESID: return launch_tc<EPI_RESID>(c, tx, tw, p, grid, smem);
+    case EPI_SWIGLU: return launch_tc<EPI_SWIGLU>(c, tx, tw, p, grid, smem);
+    case EPI_STATS: return launch_tc<EPI_STATS>(c, tx, tw, p, grid, smem);
+    case EPI_QKV: return launch_tc<EPI_QKV>(c, tx, tw, p, grid, smem);
+  }
+  return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
+}
+
+template <typename T>
+int run_linear_simt(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep) {
+  dim3 grid((N + simt::BN - 1) / simt::BN, (M + simt::BM - 1) / simt::BM);
+  const T* x = static_cast<const T*>(X);
+  const T* w = static_cast<const T*>(W);
+  switch (epi) {
+    case EPI_F32: simt::gemm_simt_kernel<T, EPI_F32><<<grid, simt::THREADS, 0, c->stream>>>(x, w, M, N, K, ep); break;
+    case EPI_T: simt::gemm_simt_kernel<T, EPI_T><<<grid, simt::THREADS, 0, c->stream>>>(x, w, M, N, K, ep); break;
+    case EPI_RESID: simt::gemm_simt_kernel<T, EPI_RESID><<<grid, simt::THREADS, 0, c->stream>>>(x, w, M, N, K, ep); break;
+    case EPI_SWIGLU: simt::gemm_simt_kernel<T, EPI_SWIGLU><<<grid, simt::THREADS, 0, c->stream>>>(x, w, M, N, K, ep); break;
+    case EPI_STATS: simt::gemm_simt_kernel<T, EPI_STATS><<<grid, simt::THREADS, 0, c->stream>>>(x, w, M, N, K, ep); break;
+    default: return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
+  }
+  LAUNCHED(c, "gemm_simt_kernel");
+  return D3_OK;
+}
+
+int run_linear(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
+               int splits_hint = 0, const QkvExtra* qx = nullptr) {
+  if (M <= 0 || N <= 0 || K <= 0) return D3_OK;
+  if (c->use_tc) return run_linear_tc(c, X, W, M, N, K, epi, ep, splits_hint, qx);
+  if (c->is_bf16) return run_linear_simt<bf16>(c, X, W, M, N, K, epi, ep);
+  return run_linear_simt<float>(c, X, W, M, N, K, epi, ep);
+}
+
+// ---- typed launch helpers
+template <typename T>
+int launch_attention(d3_ctx* c, const void* q, const void* kc, const void* vc, void* out, const RowMap& rm) {
+  const d3_config& g = c->cfg;
+  dim3 grid((rm.rows_per_seq + attn::QT - 1) / attn::QT, g.n_q_heads, rm.bs);
+  const float scale = 1.0f / std::sqrt(static_cast<float>(g.d_head));
+  const T* qq = static_cast<const T*>(q);
+  const T* kk = static_cast<const T*>(kc);
+  const T* vv = static_cast<const T*>(vc);
+  T* oo = static_cast<T*>(out);
+  switch (g.d_head) {
+    case 32: attn::attn_simt_kernel<T, 32><<<grid, attn::THREADS, 0, c->stream>>>(qq, kk, vv, oo, rm, g.n_q_heads, g.n_kv_heads, g.max_seq, scale); break;
+    case 64: attn::attn_simt_kernel<T, 64><<<grid, attn::THREADS, 0, c->stream>>>(qq, kk, vv, oo, rm, g.n_q_heads, g.n_kv_heads, g.max_seq, scale); break;
+    case 128: attn::attn_simt_kernel<T, 128><<<grid, attn::THREADS, 0, c->stream>>>(qq, kk, vv, oo, rm, g.n_q_heads, g.n_kv_heads, g.max_seq, scale); break;
+    default: return fail(c, D3_ERR_UNSUPPORTED, "d_head must be 32, 64 or 128");
+  }
+  LAUNCHED(c, "attn_simt_kernel");
+  return D3_OK;
+}
+
+int run_attention(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
+  const char* base = static_cast<const char*>(c->kv);
+  const void* kc = base + (static_cast<size_t>(layer) * 2 + 0) * c->kv_layer_elems * c->esz;
+  const void* vc = base + (static_cast<size_t>(layer) * 2 + 1) * c->kv_layer_elems * c->esz;
+  if (c->is_bf16) return launch_attention<bf16>(c, q, kc, vc, out, rm);
+  return launch_attention<float>(c, q, kc, vc, out, rm);
+}
+
+void* k_plane(d3_ctx* c, int layer) {
+  return static_cast<char*>(c->kv) + (static_cast<size_t>(layer) * 2 + 0) * c->kv_layer_elems * c->esz;
+}
+void* v_plane(d3_ctx* c, int layer) {
+  return static_cast<char*>(c->kv) + (static_cast<size_t>(layer) * 2 + 1) * c->kv_layer_elems * c->esz;
+}
+
+int run_rmsnorm(d3_ctx* c, const float* x, const float* gain, void* xn, int M) {
+  const int d = c->cfg.d_model;
+  const int threads = d >= 1024 ? 256 : 128;
+  if (c->is_bf16) rmsnorm_kernel<bf16><<<M, threads, 0, c->stream>>>(x, gain, static_cast<bf16*>(xn), d, c->cfg.rms_eps);
+  else rmsnorm_kernel<float><<<M, threads, 0, c->stream>>>(x, gain, static_cast<float*>(xn), d, c->cfg.rms_eps);
+  LAUNCHED(c, "rmsnorm_kernel");
+  return D3_OK;
+}
+
+int run_stats_merge(d3_ctx* c, int M, int n_tiles, float* conf, float* ent, int* argmax) {
+  stats_merge_kernel<<<(M + 3) / 4, 128, 0, c->stream>>>(c->stat_part, n_tiles, M, conf, ent, argmax);
+  LAUNCHED(c, "stats_merge_kernel");
+  return D3_OK;
+}
+
+// The transformer stack over M rows laid out as bs x rows_per_seq (row map already on the device).
+//   head: 0 = none, 1 = fused statistics into ctx conf/ent/argmax, 2 = fp32 logits into `logits`.
+int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float* logits) {
+  const d3_config& g = c->cfg;
+  const int M = bs * rows_per_seq;
+  if (M == 0) return D3_OK;
+  if (M > c->max_rows) return fail(c, D3_ERR_SHAPE, "forward over more rows than the workspaces hold");
+  const int d = g.d_model, nq = g.n_q_heads * g.d_head, nkv = g.n_kv_heads * g.d_head, f = g.d_ffn;
+  RowMap rm{c->pos_base, c->n_valid, c->kv_len, rows_per_seq, bs};
+  c->last_rows = M;
+
+  if (c->is_bf16) embed_kernel<bf16><<<M, 128, 0, c->stream>>>(ids, static_cast<const bf16*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
+  else embed_kernel<float><<<M, 128, 0, c->stream>>>(ids, static_cast<const float*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
+  LAUNCHED(c, "embed_kernel");
+
+  for (int l = 0; l < g.n_layers; ++l) {
+    if (l == c->tap_layer && M <= c->tap_rows)
+      CUDA_TRY(c, cudaMemcpyAsync(c->tap_in, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
+    TRY(run_rmsnorm(c, c->x, c->attn_norm[l], c->xn, M));
+    if (c->fuse_qkv) {
+      EpiParams ep;
+      ep.y = c->q; ep.ldy = nq;
+      QkvExtra qx{rm, k_plane(c, l), v_plane(c, l)};
+      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_QKV, ep, 0, &qx));
+    } else {
+      EpiParams ep;
+      ep.y = c->qkv_f32; ep.ldy = nq + 2 * nkv;
+      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_F32, ep));
+      if (c->is_bf16)
+        rope_kv_kernel<bf16><<<M, 256, 0, c->stream>>>(c->qkv_f32, static_cast<bf16*>(c->q), static_cast<bf16*>(k_plane(c, l)), static_cast<bf16*>(v_plane(c, l)), c->rope_cos, c->rope_sin, rm, g.n_q_heads, g.n_kv_heads, g.d_head, g.max_seq, c->error_word);
+      else
+        rope_kv_kernel<float><<<M, 256, 0, c->stream>>>(c->qkv_f32, static_cast<float*>(c->q), static_cast<float*>(k_plane(c, l)), static_cast<float*>(v_plane(c, l)), c->rope_cos, c->rope_sin, rm, g.n_q_heads, g.n_kv_heads, g.d_head, g.max_seq, c->error_word);
+      LAUNCHED(c, "rope_kv_kernel");
+    }
+    TRY(run_attention(c, c->q, l, c->o, rm));
+    {
+      EpiParams ep;
+      ep.y = c->x; ep.ldy = d;
+      TRY(run_linear(c, c->o, c->wo[l], M, d, nq, EPI_RESID, ep));
+    }
+    TRY(run_rmsnorm(c, c->x, c->ffn_norm[l], c->xn, M));
+    {
+      EpiParams ep;
+      ep.y = c->h; ep.ldy = f;
+      TRY(run_linear(c, c->xn, c->wgu[l], M, 2 * f, d, EPI_SWIGLU, ep));
+    }
+    {
+      EpiParams ep;
+      ep.y = c->x; ep.ldy = d;
+      TRY(run_linear(c, c->h, c->wd[l], M, d, f, EPI_RESID, ep));
+    }
+    if (l == c->tap_layer && M <= c->tap_rows)
+      CUDA_TRY(c, cudaMemcpyAsync(c->tap_out, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
+  }
+  if (head == 0) return D3_OK;
+  TRY(run_rmsnorm(c, c->x, c->final_norm, c->xn, M));
+  if (head == 1) {
+    const int n_tiles = (g.vocab + 127) / 128;
+    EpiParams ep;
+    ep.scale = g.logit_scale; ep.mask_id = g.mask_id; ep.stat_part = c->stat_part; ep.n_tiles = n_tiles;
+    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_STATS, ep));
+    TRY(run_stats_merge(c, M, n_tiles, c->conf, c->ent, c->argmax));
+  } else {
+    EpiParams ep;
+    ep.y = logits; ep.ldy = g.vocab; ep.scale = g.logit_scale;
+    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_F32, ep));
+  }
+  return D3_OK;
+}
+
+int check_device_error(d3_ctx* c) {
+  uint32_t w = 0;
+  CUDA_TRY(c, cudaMemcpyAsync(&w, c->error_word, sizeof(w), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  if (w & ERRW_MBAR_TIMEOUT) return fail(c, D3_ERR_DEVICE_TIMEOUT, "a bounded device-side wait gave up");
+  if (w) return fail(c, D3_ERR_INVALID_ARG, "device error word " + std::to_string(w) + " (bad token id or position)");
+  return D3_OK;
+}
+
+template <typename T>
+void cast_to_f32(d3_ctx* c, const void* src, float* dst, size_t n) {
+  cast_to_f32_kernel<T><<<static_cast<unsigned>((n + 255) / 256), 256, 0, c->stream>>>(static_cast<const T*>(src), dst, n);
+  c->launches++;
+}
+
+}  // namespace
+
+// ----------------------------------------------------------------------------- create / destroy
+extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) {
+  if (!cfg || !out) return D3_ERR_INVALID_ARG;
+  *out = nullptr;
+  const d3_config& g = *cfg;
+  if (g.n_layers <= 0 || g.d_model <= 0 || g.n_q_heads <= 0 || g.n_kv_heads <= 0 || g.d_ffn <= 0 || g.vocab <= 1 ||
+      g.block <= 0 || g.max_batch <= 0 || g.max_seq <= 0 || g.mask_id < 0 || g.mask_id >= g.vocab)
+    return D3_ERR_INVALID_ARG;
+  if (g.dtype != D3_DTYPE_F32 && g.dtype != D3_DTYPE_BF16) return D3_ERR_INVALID_ARG;
+  if (g.decide_mode != D3_DECIDE_CONFIDENCE && g.decide_mode != D3_DECIDE_ENTROPY) return D3_ERR_INVALID_ARG;
+  if (!(g.rms_eps >= 0.f) || !(g.rope_theta > 0.f) || !std::isfinite(g.logit_scale)) return D3_ERR_INVALID_ARG;
+  if (g.d_head != 32 && g.d_head != 64 && g.d_head != 128) return D3_ERR_UNSUPPORTED;
+  if (g.n_q_heads % g.n_kv_heads != 0 || g.d_ffn % 64 != 0 || g.d_model % 8 != 0 || g.block > 128 ||
+      g.block > g.max_seq)
+    return D3_ERR_UNSUPPORTED;
+  d3_ctx* c = new (std::nothrow) d3_ctx();
+  if (!c) return D3_ERR_OOM;
+  c->cfg = g;
+  c->stream = static_cast<cudaStream_t>(cuda_stream);
+  c->is_bf16 = g.dtype == D3_DTYPE_BF16;
+  c->esz = c->is_bf16 ? 2 : 4;
+  c->use_tc = c->is_bf16 && g.gemm_impl == D3_GEMM_AUTO;
+  c->fuse_qkv = c->use_tc && g.d_head == 128;
+  auto bail = [&](int rc) {
+    d3_destroy(c);
+    return rc;
+  };
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return bail(D3_ERR_CUDA);
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return bail(D3_ERR_CUDA);
+  c->n_sms = prop.multiProcessorCount;
+  if (c->use_tc && prop.major != 10) return bail(D3_ERR_UNSUPPORTED);
+
+  const size_t d = g.d_model, nq = static_cast<size_t>(g.n_q_heads) * g.d_head,
+               nkv = static_cast<size_t>(g.n_kv_heads) * g.d_head, f = g.d_ffn;
+  long long pre_rows = g.max_prefill_rows > 0 ? g.max_prefill_rows : static_cast<long long>(g.max_batch) * g.max_seq;
+  long long dec_rows = static_cast<long long>(g.max_batch) * g.block;
+  c->max_rows = static_cast<int>(std::max(pre_rows, dec_rows));
+  const size_t R = c->max_rows;
+#define A_(ptr, bytes)                                                         \
+  do {                                                                         \
+    int rc_ = dev_alloc(c, reinterpret_cast<void**>(&(ptr)), (bytes));         \
+    if (rc_ != D3_OK) return bail(rc_);                                        \
+  } while (0)
+  c->kv_layer_elems = static_cast<size_t>(g.max_batch) * g.n_kv_heads * g.max_seq * g.d_head;
+  A_(c->kv, c->kv_layer_elems * 2 * g.n_layers * c->esz);
+  A_(c->rope_cos, sizeof(float) * g.max_seq * (g.d_head / 2));
+  A_(c->rope_sin, sizeof(float) * g.max_seq * (g.d_head / 2));
+  A_(c->x, sizeof(float) * R * d);
+  A_(c->xn, c->esz * R * std::max(d, nq));
+  if (!c->fuse_qkv) A_(c->qkv_f32, sizeof(float) * R * (nq + 2 * nkv));
+  A_(c->q, c->esz * R * nq);
+  A_(c->o, c->esz * R * nq);
+  A_(c->h, c->esz * R * f);
+  const size_t n_tiles = (g.vocab + 127) / 128;
+  A_(c->stat_part, sizeof(float4) * static_cast<size_t>(dec_rows) * n_tiles);
+  A_(c->conf, sizeof(float) * dec_rows);
+  A_(c->ent, sizeof(float) * dec_rows);
+  A_(c->argmax, sizeof(int) * dec_rows);
+  A_(c->prefix_len, sizeof(int) * g.max_batch);
+  A_(c->pos_base, sizeof(int) * g.max_batch);
+  A_(c->n_valid, sizeof(int) * g.max_batch);
+  A_(c->kv_len, sizeof(int) * g.max_batch);
+  A_(c->error_word, sizeof(uint32_t));
+  if (c->use_tc) {
+    c->partial_slots = 2048;
+    A_(c->partial, c->partial_slots * 128 * 128 * sizeof(float));
+    c->n_tile_count = 1 << 16;
+    A_(c->tile_count, sizeof(int) * c->n_tile_count);
+  }
+  A_(c->gen.mode, sizeof(int) * g.max_batch);
+  A_(c->gen.block_idx, sizeof(int) * g.max_batch);
+  A_(c->gen.step, sizeof(int) * g.max_batch);
+  c->gen.prefix_len = c->prefix_len;
+  A_(c->gen.ids, sizeof(int) * dec_rows);
+  A_(c->gen.mask, sizeof(uint8_t) * dec_rows);
+  A_(c->gen.counters, sizeof(long long) * 8);
+  if (cudaMallocHost(reinterpret_cast<void**>(&c->host_counters), sizeof(long long) * 8) != cudaSuccess)
+    return bail(D3_ERR_OOM);
+  c->tap_rows = static_cast<int>(dec_rows);
+  A_(c->tap_in, sizeof(float) * dec_rows * d);
+  A_(c->tap_out, sizeof(float) * dec_rows * d);
+#undef A_
+  // RoPE table in double precision on the host
+  {
+    const int half = g.d_head / 2;
+    std::vector<float> cs(static_cast<size_t>(g.max_seq) * half), sn(cs.size());
+    for (int k = 0; k < half; ++k) {
+      const double inv = std::pow(static_cast<double>(g.rope_theta), -2.0 * k / g.d_head);
+      for (int p = 0; p < g.max_seq; ++p) {
+        const double a = p * inv;
+        cs[static_cast<size_t>(p) * half + k] = static_cast<float>(std::cos(a));
+        sn[static_cast<size_t>(p) * half + k] = static_cast<float>(std::sin(a));
+      }
+    }
+    if (cudaMemcpyAsync(c->rope_cos, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+        cudaMemcpyAsync(c->rope_sin, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess)
+      return bail(D3_ERR_CUDA);
+  }
+  *out = c;
+  return D3_OK;
+}
+
+extern "C" void d3_destroy(d3_ctx* c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->stream);
+  for (void* p : c->allocs) cudaFree(p);
+  if (c->host_counters) cudaFreeHost(c->host_counters);
+  delete c;
+}
+
+// ----------------------------------------------------------------------------- weights
+namespace {
+int upload(d3_ctx* c, void* dst, const void* src, size_t bytes, int src_is_device) {
+  CUDA_TRY(c, cudaMemcpyAsync(dst, src, bytes, src_is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
+  return D3_OK;
+}
+int load_gain(d3_ctx* c, float** dst, const void* src, int src_is_device, void* tmp) {
+  const size_t d = c->cfg.d_model;
+  if (!*dst) ALLOC(c, *dst, sizeof(float) * d);
+  if (!src) {
+    std::vector<float> ones(d, 1.0f);
+    CUDA_TRY(c, cudaMemcpyAsync(*dst, ones.data(), sizeof(float) * d, cudaMemcpyHostToDevice, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    return D3_OK;
+  }
+  TRY(upload(c, tmp, src, c->esz * d, src_is_device));
+  if (c->is_bf16) cast_to_f32<bf16>(c, tmp, *dst, d);
+  else cast_to_f32<float>(c, tmp, *dst, d);
+  return D3_OK;
+}
+}  // namespace
+
+extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!w || !w->tok_emb || !w->lm_head || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up || !w->w_down)
+    return fail(c, D3_ERR_INVALID_ARG, "null weight pointer");
+  const d3_config& g = c->cfg;
+  const size_t d = g.d_model, nq = static_cast<size_t>(g.n_q_heads) * g.d_head,
+               nkv = static_cast<size_t>(g.n_kv_heads) * g.d_head, f = g.d_ffn, V = g.vocab, e = c->esz;
+  for (int l = 0; l < g.n_layers; ++l)
+    if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l])
+      return fail(c, D3_ERR_INVALID_ARG, "null per-layer weight pointer");
+  if (!c->tok_emb) {
+    ALLOC(c, c->tok_emb, V * d * e);
+    ALLOC(c, c->lm_head, V * d * e);
+    c->wqkv.assign(g.n_layers, nullptr); c->wo.assign(g.n_layers, nullptr);
+    c->wgu.assign(g.n_layers, nullptr); c->wd.assign(g.n_layers, nullptr);
+    c->attn_norm.assign(g.n_layers, nullptr); c->ffn_norm.assign(g.n_layers, nullptr);
+    for (int l = 0; l < g.n_layers; ++l) {
+      ALLOC(c, c->wqkv[l], (nq + 2 * nkv) * d * e);
+      ALLOC(c, c->wo[l], d * nq * e);
+      ALLOC(c, c->wgu[l], 2 * f * d * e);
+      ALLOC(c, c->wd[l], d * f * e);
+    }
+  }
+  // staging for gate / up (interleaved on the device) and gains
+  void *tg = nullptr, *tu = nullptr, *tgain = nullptr;
+  CUDA_TRY(c, cudaMalloc(&tg, f * d * e));
+  CUDA_TRY(c, cudaMalloc(&tu, f * d * e));
+  CUDA_TRY(c, cudaMalloc(&tgain, d * e));
+  int rc = D3_OK;
+  auto step = [&](int r) { if (rc == D3_OK) rc = r; };
+  step(upload(c, c->tok_emb, w->tok_emb, V * d * e, src_is_device));
+  step(upload(c, c->lm_head, w->lm_head, V * d * e, src_is_device));
+  step(load_gain(c, &c->final_norm, w->final_norm, src_is_device, tgain));
+  for (int l = 0; l < g.n_layers && rc == D3_OK; ++l) {
+    char* qkv = static_cast<char*>(c->wqkv[l]);
+    step(upload(c, qkv, w->wq[l], nq * d * e, src_is_device));
+    step(upload(c, qkv + nq * d * e, w->wk[l], nkv * d * e, src_is_device));
+    step(upload(c, qkv + (nq + nkv) * d * e, w->wv[l], nkv * d * e, src_is_device));
+    step(upload(c, c->wo[l], w->wo[l], d * nq * e, src_is_device));
+    step(upload(c, c->wd[l], w->w_down[l], d * f * e, src_is_device));
+    step(upload(c, tg, w->w_gate[l], f * d * e, src_is_device));
+    step(upload(c, tu, w->w_up[l], f * d * e, src_is_device));
+    if (rc == D3_OK) {
+      if (c->is_bf16)
+        interleave_gate_up_kernel<bf16><<<static_cast<unsigned>(2 * f), 128, 0, c->stream>>>(static_cast<const bf16*>(tg), static_cast<const bf16*>(tu), static_cast<bf16*>(c->wgu[l]), g.d_ffn, g.d_model);
+      else
+        interleave_gate_up_kernel<float><<<static_cast<unsigned>(2 * f), 128, 0, c->stream>>>(static_cast<const float*>(tg), static_cast<const float*>(tu), static_cast<float*>(c->wgu[l]), g.d_ffn, g.d_model);
+      step(check_launch(c, "interleave_gate_up_kernel"));
+    }
+    step(load_gain(c, &c->attn_norm[l], w->attn_norm ? w->attn_norm[l] : nullptr, src_is_device, tgain));
+    step(load_gain(c, &c->ffn_norm[l], w->ffn_norm ? w->ffn_norm[l] : nullptr, src_is_device, tgain));
+    // the staging buffers are reused by the next layer: the copies above are stream-ordered
+  }
+  cudaError_t es = cudaStreamSynchronize(c->stream);
+  cudaFree(tg); cudaFree(tu); cudaFree(tgain);
+  if (rc != D3_OK) return rc;
+  if (es != cudaSuccess) return fail(c, D3_ERR_CUDA, std::string("sync after weight load: ") + cudaGetErrorString(es));
+  c->weights_loaded = true;
+  return D3_OK;
+}
+
+// ----------------------------------------------------------------------------- decoding path
+extern "C" int d3_prefill(d3_ctx* c, const int32_t* prompt_ids, const int32_t* prompt_lens, int32_t bs, int32_t p_max) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!prompt_lens || (!prompt_ids && p_max > 0) || bs <= 0 || p_max < 0) return fail(c, D3_ERR_INVALID_ARG, "bad prefill arguments");
+  if (!c->weights_loaded) return fail(c, D3_ERR_STATE, "d3_prefill before d3_load_weights");
+  if (bs > c->cfg.max_batch || p_max > c->cfg.max_seq || static_cast<long long>(bs) * p_max > c->max_rows)
+    return fail(c, D3_ERR_SHAPE, "prefill larger than max_batch / max_seq / max_prefill_rows");
+  prefill_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(prompt_lens, bs, p_max, c->prefix_len, c->pos_base, c->n_valid, c->kv_len);
+  LAUNCHED(c, "prefill_rowmap_kernel");
+  TRY(forward(c, prompt_ids, bs, p_max, 0, nullptr));
+  c->prefilled = true;
+  return D3_OK;
+}
+
+extern "C" int d3_denoise_step(d3_ctx* c, int32_t* block_ids, uint8_t* mask, float threshold, int32_t bs,
+                               int32_t* out_pos, int32_t* out_ids, int32_t* out_count) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!block_ids || !mask || !out_pos || !out_ids || !out_count || bs <= 0 || std::isnan(threshold))
+    return fail(c, D3_ERR_INVALID_ARG, "bad denoise_step arguments");
+  if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_denoise_step before d3_prefill");
+  if (bs > c->cfg.max_batch) return fail(c, D3_ERR_SHAPE, "bs > max_batch");
+  const int B = c->cfg.block;
+  decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B, c->pos_base, c->n_valid, c->kv_len);
+  LAUNCHED(c, "decode_rowmap_kernel");
+  TRY(forward(c, block_ids, bs, B, 1, nullptr));
+  unmask_kernel<<<bs, 32, 0, c->stream>>>(c->conf, c->ent, c->argmax, block_ids, mask, B, threshold, c->cfg.decide_mode, out_pos, out_ids, out_count);
+  LAUNCHED(c, "unmask_kernel");
+  return D3_OK;
+}
+
+extern "C" int d3_commit_block(d3_ctx* c, const int32_t* block_ids, int32_t bs) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!block_ids || bs <= 0) return fail(c, D3_ERR_INVALID_ARG, "bad commit_block arguments");
+  if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_commit_block before d3_prefill");
+  if (bs > c->cfg.max_batch) return fail(c, D3_ERR_SHAPE, "bs > max_batch");
+  const int B = c->cfg.block;
+  decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B, c->pos_base, c->n_valid, c->kv_len);
+  LAUNCHED(c, "decode_rowmap_kernel");
+  TRY(forward(c, block_ids, bs, B, 0, nullptr));
+  add_prefix_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B);
+  LAUNCHED(c, "add_prefix_kernel");
+  return D3_OK;
+}
+
+extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t bs, int32_t* out_ids,
+                           int32_t* commit_step, d3_stats* host_stats) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!out_ids || bs <= 0 || gen_len <= 0 || std::isnan(threshold)) return fail(c, D3_ERR_INVALID_ARG, "bad generate arguments");
+  if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_generate before d3_prefill");
+  const int B = c->cfg.block;
+  if (bs > c->cfg.max_batch || gen_len % B != 0) return fail(c, D3_ERR_SHAPE, "bs > max_batch or gen_len not a multiple of the block size");
+  {  // prefix + gen_len must fit the cache
+    std::vector<int> pl(bs);
+    CUDA_TRY(c, cudaMemcpyAsync(pl.data(), c->prefix_len, sizeof(int) * bs, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (int b = 0; b < bs; ++b)
+      if (pl[b] + gen_len > c->cfg.max_seq) return fail(c, D3_ERR_SHAPE, "prefix + gen_len exceeds max_seq");
+  }
+  const int n_blocks = gen_len / B;
+  const int64_t launches0 = c->launches;
+  GenState g = c->gen;
+  g.out_ids = out_ids;
+  g.commit_step = commit_step;
+  gen_init_kernel<<<bs, 32, 0, c->stream>>>(g, bs, B, c->cfg.mask_id);
+  LAUNCHED(c, "gen_init_kernel");
+  const long long max_iter = static_cast<long long>(n_blocks) * (B + 1) + 1;
+  long long steps = 0;
+  for (long long it = 0; it < max_iter; ++it) {
+    gen_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(g, bs, B, c->pos_base, c->n_valid, c->kv_len);
+    LAUNCHED(c, "gen_rowmap_kernel");
+    TRY(forward(c, g.ids, bs, B, 1, nullptr));
+    gen_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, n_blocks, gen_len, threshold, c->cfg.decide_mode, c->cfg.mask_id);
+    LAUNCHED(c, "gen_advance_kernel");
+    ++steps;
+    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 5, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (c->host_counters[4] <= 0) break;
+  }
+  if (host_stats) {
+    std::memset(host_stats, 0, sizeof(*host_stats));
+    host_stats->denoise_forwards = c->host_counters[0];
+    host_stats->finalize_forwards = c->host_counters[1];
+    host_stats->tokens_committed = c->host_counters[2];
+    host_stats->forced_commits = c->host_counters[3];
+    host_stats->steps = steps;
+    host_stats->kernel_launches = c->launches - launches0;
+  }
+  if (c->host_counters[4] > 0) return fail(c, D3_ERR_STATE, "generate loop did not finish within its step bound");
+  return check_device_error(c);
+}
+
+extern "C" int d3_get_step_stats(d3_ctx* c, float* conf, float* entropy, int32_t* argmax, int32_t bs) {
+  if (!c || bs <= 0 || bs > c->cfg.max_batch) return D3_ERR_INVALID_ARG;
+  const size_t n = static_cast<size_t>(bs) * c->cfg.block;
+  if (conf) CUDA_TRY(c, cudaMemcpyAsync(conf, c->conf, n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if (entropy) CUDA_TRY(c, cudaMemcpyAsync(entropy, c->ent, n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if (argmax) CUDA_TRY(c, cudaMemcpyAsync(argmax, c->argmax, n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  return D3_OK;
+}
+
+extern "C" int d3_forward_logits(d3_ctx* c, const int32_t* block_ids, int32_t bs, float* logits) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!block_ids || !logits || bs <= 0) return fail(c, D3_ERR_INVALID_ARG, "bad forward_logits arguments");
+  if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_forward_logits before d3_prefill");
+  if (bs > c->cfg.max_batch) return fail(c, D3_ERR_SHAPE, "bs > max_batch");
+  const int B = c->cfg.block;
+  decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B, c->pos_base, c->n_valid, c->kv_len);
+  LAUNCHED(c, "decode_rowmap_kernel");
+  return forward(c, block_ids, bs, B, 2, logits);
+}
+
+extern "C" int d3_set_tap(d3_ctx* c, int32_t layer) {
+  if (!c || layer >= c->cfg.n_layers) return D3_ERR_INVALID_ARG;
+  c->tap_layer = layer < 0 ? -1 : layer;
+  return D3_OK;
+}
+
+extern "C" int d3_read_tap(d3_ctx* c, float* resid_in, float* resid_out, int32_t rows) {
+  if (!c || rows <= 0 || rows > c->tap_rows) return D3_ERR_INVALID_ARG;
+  const size_t n = static_cast<size_t>(rows) * c->cfg.d_model * sizeof(float);
+  if (resid_in) CUDA_TRY(c, cudaMemcpyAsync(resid_in, c->tap_in, n, cudaMemcpyDeviceToDevice, c->stream));
+  if (resid_out) CUDA_TRY(c, cudaMemcpyAsync(resid_out, c->tap_out, n, cudaMemcpyDeviceToDevice, c->stream));
+  return D3_OK;
+}
+
+extern "C" int d3_read_kv(d3_ctx* c, int32_t layer, int32_t seq, int32_t pos0, int32_t n, float* k_out, float* v_out) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  const d3_config& g = c->cfg;
+  if (layer < 0 || layer >= g.n_layers || seq < 0 || seq >= g.max_batch || pos0 < 0 || n <= 0 || pos0 + n > g.max_seq)
+    return fail(c, D3_ERR_INVALID_ARG, "bad read_kv range");
+  for (int hh = 0; hh < g.n_kv_heads; ++hh) {
+    const size_t off = ((static_cast<size_t>(seq) * g.n_kv_heads + hh) * g.max_seq + pos0) * g.d_head;
+    const size_t cnt = static_cast<size_t>(n) * g.d_head;
+    for (int which = 0; which < 2; ++which) {
+      float* dst = which == 0 ? k_out : v_out;
+      if (!dst) continue;
+      const char* src = static_cast<const char*>(which == 0 ? k_plane(c, layer) : v_plane(c, layer)) + off * c->esz;
+      if (c->is_bf16) cast_to_f32<bf16>(c, src, dst + static_cast<size_t>(hh) * cnt, cnt);
+      else cast_to_f32<float>(c, src, dst + static_cast<size_t>(hh) * cnt, cnt);
+    }
+  }
+  cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) return fail(c, D3_ERR_CUDA, std::string("cast_to_f32_kernel: ") + cudaGetErrorString(e));
+  return D3_OK;
+}
+
+extern "C" int d3_get_state(d3_ctx* c, int32_t* prefix_len, int32_t bs) {
+  if (!c || !prefix_len || bs <= 0 || bs > c->cfg.max_batch) return D3_ERR_INVALID_ARG;
+  CUDA_TRY(c, cudaMemcpyAsync(prefix_len, c->prefix_len, sizeof(int) * bs, cudaMemcpyDeviceToDevice, c->stream));
+  return D3_OK;
+}
+extern "C" int d3_set_state(d3_ctx* c, const int32_t* prefix_len, int32_t bs) {
+  if (!c || !prefix_len || bs <= 0 || bs > c->cfg.max_batch) return D3_ERR_INVALID_ARG;
+  CUDA_TRY(c, cudaMemcpyAsync(c->prefix_len, prefix_len, sizeof(int) * bs, cudaMemcpyDeviceToDevice, c->stream));
+  c->prefilled = true;
+  return D3_OK;
+}
+
+// ----------------------------------------------------------------------------- single operators
+extern "C" int d3_op_linear(d3_ctx* c, const void* x, const void* w, void* y, int32_t m, int32_t n, int32_t k,
+                            int32_t epilogue, int32_t splits) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!x || !w || !y || m <= 0 || n <= 0 || k <= 0 || epilogue < 0 || epilogue > 3)
+    return fail(c, D3_ERR_INVALID_ARG, "bad op_linear arguments");
+  if (epilogue == EPI_SWIGLU && n % 128 != 0) return fail(c, D3_ERR_SHAPE, "SwiGLU epilogue needs n % 128 == 0");
+  EpiParams ep;
+  ep.y = y;
+  ep.ldy = epilogue == EPI_SWIGLU ? n / 2 : n;
+  return run_linear(c, x, w, m, n, k, epilogue, ep, splits);
+}
+
+extern "C" int d3_op_lm_head_stats(d3_ctx* c, const void* x, const void* w, int32_t m, int32_t vocab, int32_t k,
+                                   float scale, int32_t mask_id, float* conf, float* entropy, int32_t* argmax) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!x || !w || !conf || !entropy || !argmax || m <= 0 || vocab <= 0 || k <= 0)
+    return fail(c, D3_ERR_INVALID_ARG, "bad op_lm_head_stats arguments");
+  const int n_tiles = (vocab + 127) / 128;
+  const size_t cap = static_cast<size_t>(c->cfg.max_batch) * c->cfg.block * ((c->cfg.vocab + 127) / 128);
+  if (static_cast<size_t>(m) * n_tiles > cap) return fail(c, D3_ERR_SHAPE, "m * vocab tiles exceed the statistics workspace");
+  EpiParams ep;
+  ep.scale = scale; ep.mask_id = mask_id; ep.stat_part = c->stat_part; ep.n_tiles = n_tiles;
+  TRY(run_linear(c, x, w, m, vocab, k, EPI_STATS, ep));
+  return run_stats_merge(c, m, n_tiles, conf, entropy, argmax);
+}
+
+extern "C" int d3_op_attention(d3_ctx* c, const void* q, int32_t layer, int32_t bs, int32_t rows,
+                               const int32_t* kv_len, void* out) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!q || !out || !kv_len || layer < 0 || layer >= c->cfg.n_layers || bs <= 0 || bs > c->cfg.max_batch || rows <= 0)
+    return fail(c, D3_ERR_INVALID_ARG, "bad op_attention arguments");
+  // all rows live, positions irrelevant here
+  decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(kv_len, bs, rows, c->pos_base, c->n_valid, c->kv_len);
+  LAUNCHED(c, "decode_rowmap_kernel");
+  RowMap rm{c->pos_base, c->n_valid, kv_len, rows, bs};
+  return run_attention(c, q, layer, out, rm);
+}
+
+extern "C" int d3_op_write_kv(d3_ctx* c, int32_t layer, int32_t seq, int32_t pos0, int32_t n, const float* k, const float* v) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  const d3_config& g = c->cfg;
+  if (!k || !v || layer < 0 || layer >= g.n_layers || seq < 0 || seq >= g.max_batch || pos0 < 0 || n <= 0 || pos0 + n > g.max_seq)
+    return fail(c, D3_ERR_INVALID_ARG, "bad op_write_kv range");
+  for (int hh = 0; hh < g.n_kv_heads; ++hh) {
+    const size_t off = ((static_cast<size_t>(seq) * g.n_kv_heads + hh) * g.max_seq + pos0) * g.d_head;
+    const size_t cnt = static_cast<size_t>(n) * g.d_head;
+    for (int which = 0; which < 2; ++which) {
+      const float* src = (which == 0 ? k : v) + static_cast<size_t>(hh) * cnt;
+      char* dst = static_cast<char*>(which == 0 ? k_plane(c, layer) : v_plane(c, layer)) + off * c->esz;
+      const unsigned blocks = static_cast<unsigned>((cnt + 255) / 256);
+      if (c->is_bf16) cast_from_f32_kernel<bf16><<<blocks, 256, 0, c->stream>>>(src, reinterpret_cast<bf16*>(dst), cnt);
+      else cast_from_f32_kernel<float><<<blocks, 256, 0, c->stream>>>(src, reinterpret_cast<float*>(dst), cnt);
+      LAUNCHED(c, "cast_from_f32_kernel");
+    }
+  }
+  return D3_OK;
+}
+
+extern "C" int d3_op_unmask(d3_ctx* c, const float* conf, const float* entropy, const int32_t* argmax,
+                            int32_t* block_ids, uint8_t* mask, float threshold, int32_t bs, int32_t* out_pos,
+                            int32_t* out_ids, int32_t* out_count) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!conf || !entropy || !argmax || !block_ids || !mask || !out_pos || !out_ids || !out_count || bs <= 0 ||
+      std::isnan(threshold))
+    return fail(c, D3_ERR_INVALID_ARG, "bad op_unmask arguments");
+  unmask_kernel<<<bs, 32, 0, c->stream>>>(conf, entropy, argmax, block_ids, mask, c->cfg.block, threshold, c->cfg.decide_mode, out_pos, out_ids, out_count);
+  LAUNCHED(c, "unmask_kernel");
+  return D3_OK;
+}
+
+// ----------------------------------------------------------------------------- misc
+extern "C" int d3_get_error_word(d3_ctx* c, uint32_t* word) {
+  if (!c || !word) return D3_ERR_INVALID_ARG;
+  CUDA_TRY(c, cudaMemcpyAsync(word, c->error_word, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return D3_OK;
+}
+extern "C" int64_t d3_launch_count(d3_ctx* c) { return c ? c->launches : 0; }
+extern "C" int64_t d3_device_bytes(d3_ctx* c) { return c ? c->dev_bytes : 0; }
+
+extern "C" const char* d3_strerror(int code) {
+  switch (code) {
+    case D3_OK: return "ok";
+    case D3_ERR_INVALID_ARG: return "invalid argument";
+    case D3_ERR_SHAPE: return "shape outside the configured limits";
+    case D3_ERR_OOM: return "out of device memory";
+    case D3_ERR_CUDA: return "CUDA call failed";
+    case D3_ERR_DEVICE_TIMEOUT: return "bounded device-side wait gave up";
+    case D3_ERR_STATE: return "call out of order";
+    case D3_ERR_UNSUPPORTED: return "unsupported configuration";
+  }
+  return "unknown error";
+}
+extern "C" const char* d3_last_error(d3_ctx* c) { return c ? c->last_error.c_str() : ""; }
+extern "C" const char* d3_version(void) { return kVersion; }

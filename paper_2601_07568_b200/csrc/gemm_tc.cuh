@@ -1,0 +1,531 @@
+// bf16 matmul Y[M,N] = X[M,K] . W[N,K]^T on the sm_100a tensor cores.
+//
+//   * operands are staged in shared memory by TMA (128-byte swizzle, 64-element K slabs),
+//   * one elected thread issues tcgen05.mma (128 x BLOCK_N x 16) into a TMEM accumulator,
+//   * four epilogue warps read the accumulator back with tcgen05.ld; TMEM lane = row of X, so every
+//     epilogue (residual add, SwiGLU, RoPE + cache write, softmax statistics) is thread-local,
+//   * split-K: each split writes an fp32 partial tile; the last split to arrive (an atomic counter
+//     per tile, nobody spins) sums the partials in split order, which keeps results deterministic.
+//
+// Skinny case (M <= 64 rows, the batch-1 denoise step): the X box is only a_rows high, and the
+// stage stride of X in shared memory shrinks with it, so that almost all of shared memory holds
+// weight slabs in flight; rows a_rows..127 of the MMA's A operand then alias neighbouring stages
+// and produce garbage in TMEM lanes that no one reads.
+#pragma once
+#include <cuda.h>
+
+#include "common.cuh"
+
+namespace d3 {
+namespace tc {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;  // 64 bf16 = 128 bytes = one swizzle row
+constexpr int UMMA_K = 16;
+constexpr int NUM_THREADS = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr uint64_t WAIT_LIMIT_NS = 4000000000ull;
+
+struct GemmParams {
+  int M, N, K;
+  int a_rows;       // rows of the X box: 32, 64 or 128
+  int stages;       // pipeline depth
+  int splits;       // split-K factor (grid.z)
+  float* partial;   // split-K workspace [tile][split][BLOCK_N][128] fp32 (splits > 1)
+  int* tile_count;  // split-K arrival counters [tiles], zero on entry and on exit
+  uint32_t* error_word;
+  EpiParams ep;
+  // EPI_QKV only
+  const float* rope_cos;  // [max_seq][64]
+  const float* rope_sin;
+  const int* pos_base;    // [bs]
+  const int* n_valid;     // [bs]
+  int rows_per_seq;
+  int n_q_heads, n_kv_heads, max_seq;
+  __nv_bfloat16* k_cache;  // this layer: [bs][n_kv_heads][max_seq][128]
+  __nv_bfloat16* v_cache;
+};
+
+// ----------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait.  Returns false (and raises the error word and the CTA's abort flag) when the
+// phase did not complete within WAIT_LIMIT_NS or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          uint32_t* error_word) {
+  if (mbar_try_wait(bar, parity)) return true;
+  uint64_t t0 = global_ns();
+  uint32_t it = 0;
+  while (!mbar_try_wait(bar, parity)) {
+    if ((++it & 0x3ff) == 0) {
+      if (*abort_flag) return false;
+      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicOr(error_word, ERRW_MBAR_TIMEOUT);
+        return false;
+      }
+    }
+  }
+  return true;
+}
+__device__ __forceinline__ void fence_barrier_init() {
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* smem_dst, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(smem_dst)),
+               "r"(ncols)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrive on an mbarrier once all MMAs issued so far by this thread have completed.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread t of the warp gets lane (base + t).
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, float (&v)[32]) {
+  uint32_t* r = reinterpret_cast<uint32_t*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major operand tile in shared memory, 128-byte swizzle: rows of 128 bytes, 8-row groups 1024 bytes
+// apart.  Field layout of the 64-bit matrix descriptor: start address >> 4 in bits [0,14), leading
+// byte offset >> 4 in [16,30) (1 for swizzled K-major), stride byte offset >> 4 in [32,46) (1024 >> 4),
+// descriptor version 1 in [46,48), swizzle mode in [61,64) (2 = 128 bytes).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t smem_addr) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4);
+  d |= static_cast<uint64_t>(1) << 16;
+  d |= static_cast<uint64_t>(1024 >> 4) << 32;
+  d |= static_cast<uint64_t>(1) << 46;
+  d |= static_cast<uint64_t>(2) << 61;
+  return d;
+}
+// Instruction descriptor for kind::f16: D fp32 (bits [4,6) = 1), A and B bf16 ([7,10) = [10,13) = 1),
+// both K-major (bits 15, 16 = 0), N >> 3 in [17,23), M >> 4 in [24,29).
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// ----------------------------------------------------------------------------- epilogue helpers
+// Source of one 32-column chunk of this thread's accumulator row: TMEM, or the sum of split-K partials.
+struct TmemSource {
+  uint32_t taddr_row;  // tmem base + (lane group << 16)
+  __device__ __forceinline__ void load(int c, float (&v)[32]) const {
+    tmem_ld_32x32(taddr_row + static_cast<uint32_t>(c), v);
+    tmem_ld_wait();
+  }
+};
+template <int BLOCK_N>
+struct PartialSource {
+  const float* base;  // this tile's partials: [split][BLOCK_N][128]
+  int splits, row;
+  __device__ __forceinline__ void load(int c, float (&v)[32]) const {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = 0.f;
+    for (int s = 0; s < splits; ++s) {
+      const float* p = base + (static_cast<size_t>(s) * BLOCK_N + c) * 128 + row;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += __ldcg(p + j * 128);
+    }
+  }
+};
+
+// All 32 threads of a warp must call this together (the TMEM loads are warp-wide); `live` only
+// predicates this thread's stores.
+template <int EPI, int BLOCK_N, typename Source>
+__device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams& p, int m, int n0, bool live) {
+  const int N = p.N;
+  if constexpr (EPI == EPI_F32 || EPI == EPI_RESID) {
+    float* y = static_cast<float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
+    for (int c = 0; c < BLOCK_N; c += 32) {
+      if (n0 + c >= N) break;
+      float v[32];
+      src.load(c, v);
+      const bool vec = (n0 + c + 32 <= N) && ((p.ep.ldy & 3) == 0);
+      if (!live) continue;
+      if (vec) {
+        float4* y4 = reinterpret_cast<float4*>(y + n0 + c);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          float4 o;
+          if constexpr (EPI == EPI_RESID) {
+            o = y4[j];
+            o.x += v[4 * j]; o.y += v[4 * j + 1]; o.z += v[4 * j + 2]; o.w += v[4 * j + 3];
+          } else {
+            o = make_float4(v[4 * j] * p.ep.scale, v[4 * j + 1] * p.ep.scale, v[4 * j + 2] * p.ep.scale,
+                            v[4 * j + 3] * p.ep.scale);
+          }
+          y4[j] = o;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          int n = n0 + c + j;
+          if (n < N) {
+            if constexpr (EPI == EPI_RESID) y[n] += v[j];
+            else y[n] = v[j] * p.ep.scale;
+          }
+        }
+      }
+    }
+  } else if constexpr (EPI == EPI_T) {
+    __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
+    for (int c = 0; c < BLOCK_N; c += 32) {
+      if (n0 + c >= N) break;
+      float v[32];
+      src.load(c, v);
+      if (!live) continue;
+      if ((n0 + c + 32 <= N) && ((p.ep.ldy & 7) == 0)) {
+        uint4* y4 = reinterpret_cast<uint4*>(y + n0 + c);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          __nv_bfloat162 a = __floats2bfloat162_rn(v[8 * j], v[8 * j + 1]);
+          __nv_bfloat162 b = __floats2bfloat162_rn(v[8 * j + 2], v[8 * j + 3]);
+          __nv_bfloat162 cc = __floats2bfloat162_rn(v[8 * j + 4], v[8 * j + 5]);
+          __nv_bfloat162 d = __floats2bfloat162_rn(v[8 * j + 6], v[8 * j + 7]);
+          uint4 o;
+          o.x = *reinterpret_cast<uint32_t*>(&a); o.y = *reinterpret_cast<uint32_t*>(&b);
+          o.z = *reinterpret_cast<uint32_t*>(&cc); o.w = *reinterpret_cast<uint32_t*>(&d);
+          y4[j] = o;
+        }
+      } else {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+          if (n0 + c + j < N) y[n0 + c + j] = __float2bfloat16_rn(v[j]);
+      }
+    }
+  } else if constexpr (EPI == EPI_SWIGLU) {
+    // columns [g*128, g*128+64) are gate rows of hidden units [g*64, g*64+64), the next 64 the up rows
+    __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
+    for (int g = 0; g < BLOCK_N; g += 128) {
+      if (n0 + g >= N) break;
+      for (int c = 0; c < 64; c += 32) {
+        float gate[32], up[32];
+        src.load(g + c, gate);
+        src.load(g + c + 64, up);
+        const int h0 = (n0 + g) / 2 + c;
+        const int F = N / 2;
+        if (!live) continue;
+        if (h0 + 32 <= F && (p.ep.ldy & 7) == 0) {
+          uint4* y4 = reinterpret_cast<uint4*>(y + h0);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            uint32_t w[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              __nv_bfloat162 t = __floats2bfloat162_rn(silu_f(gate[8 * j + 2 * q]) * up[8 * j + 2 * q],
+                                                       silu_f(gate[8 * j + 2 * q + 1]) * up[8 * j + 2 * q + 1]);
+              w[q] = *reinterpret_cast<uint32_t*>(&t);
+            }
+            y4[j] = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (h0 + j < F) y[h0 + j] = __float2bfloat16_rn(silu_f(gate[j]) * up[j]);
+        }
+      }
+    }
+  } else if constexpr (EPI == EPI_STATS) {
+    // one partial per 128-column tile so that the merge kernel sees the same tiling for any BLOCK_N
+    for (int g = 0; g < BLOCK_N; g += 128) {
+      SoftStat st = stat_empty();
+      for (int c = 0; c < 128; c += 32) {
+        if (n0 + g + c >= N) break;
+        float v[32];
+        src.load(g + c, v);
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          int n = n0 + g + c + j;
+          if (n < N && n != p.ep.mask_id) stat_add(st, v[j] * p.ep.scale, n);
+        }
+      }
+      int t = (n0 + g) / 128;
+      if (live && t < p.ep.n_tiles)
+        p.ep.stat_part[static_cast<size_t>(m) * p.ep.n_tiles + t] = make_float4(st.m, st.z, st.s, __int_as_float(st.a));
+    }
+  } else if constexpr (EPI == EPI_QKV) {
+    // one 128-column group = one head (d_head = 128): q heads, then k heads, then v heads
+    int pos = 0, b = 0;
+    if (live) {
+      b = m / p.rows_per_seq;
+      const int r = m % p.rows_per_seq;
+      pos = p.pos_base[b] + r;
+      if (r >= p.n_valid[b]) live = false;
+      else if (pos < 0 || pos >= p.max_seq) {
+        atomicOr(p.error_word, ERRW_BAD_POSITION);
+        live = false;
+      }
+      if (!live) pos = 0;
+    }
+    for (int g = 0; g < BLOCK_N; g += 128) {
+      const int head = (n0 + g) / 128;
+      if (head >= p.n_q_heads + 2 * p.n_kv_heads) break;
+      __nv_bfloat16* dst;
+      bool rotate = true;
+      if (head < p.n_q_heads) {
+        dst = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy + head * 128;
+      } else if (head < p.n_q_heads + p.n_kv_heads) {
+        int kh = head - p.n_q_heads;
+        dst = p.k_cache + ((static_cast<size_t>(b) * p.n_kv_heads + kh) * p.max_seq + pos) * 128;
+      } else {
+        int vh = head - p.n_q_heads - p.n_kv_heads;
+        dst = p.v_cache + ((static_cast<size_t>(b) * p.n_kv_heads + vh) * p.max_seq + pos) * 128;
+        rotate = false;
+      }
+      const float* cs = p.rope_cos + static_cast<size_t>(pos) * 64;
+      const float* sn = p.rope_sin + static_cast<size_t>(pos) * 64;
+      for (int c = 0; c < 64; c += 32) {
+        float lo[32], hi[32];
+        src.load(g + c, lo);
+        src.load(g + c + 64, hi);
+        if (!live) continue;
+        if (rotate) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            float co = cs[c + j], si = sn[c + j];
+            float a = lo[j], bb = hi[j];
+            lo[j] = a * co - bb * si;
+            hi[j] = bb * co + a * si;
+          }
+        }
+        uint4* d_lo = reinterpret_cast<uint4*>(dst + c);
+        uint4* d_hi = reinterpret_cast<uint4*>(dst + c + 64);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          uint32_t w[4], x[4];
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(lo[8 * j + 2 * q], lo[8 * j + 2 * q + 1]);
+            __nv_bfloat162 u = __floats2bfloat162_rn(hi[8 * j + 2 * q], hi[8 * j + 2 * q + 1]);
+            w[q] = *reinterpret_cast<uint32_t*>(&t);
+            x[q] = *reinterpret_cast<uint32_t*>(&u);
+          }
+          d_lo[j] = make_uint4(w[0], w[1], w[2], w[3]);
+          d_hi[j] = make_uint4(x[0], x[1], x[2], x[3]);
+        }
+      }
+    }
+  }
+}
+
+// ----------------------------------------------------------------------------- kernel
+// grid = (m_tiles, n_tiles, splits); dynamic shared memory (1024-byte aligned inside the kernel):
+//   [stages x a_rows x 128 B]  X slabs      (stage stride a_rows*128)
+//   [stages x BLOCK_N x 128 B] W slabs
+//   barriers: full[stages], empty[stages], accum; tmem address; flags
+template <int EPI, int BLOCK_N>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+               const GemmParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int stages = p.stages;
+  const uint32_t a_stage_bytes = static_cast<uint32_t>(p.a_rows) * 128u;
+  constexpr uint32_t b_stage_bytes = BLOCK_N * 128u;
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + static_cast<size_t>(stages) * a_stage_bytes;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_b + static_cast<size_t>(stages) * b_stage_bytes);
+  uint64_t* empty_bar = full_bar + stages;
+  uint64_t* accum_bar = empty_bar + stages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_bar + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  int* last_flag = const_cast<int*>(abort_flag) + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tile = blockIdx.x, n_tile = blockIdx.y, split = blockIdx.z;
+  const int k_chunks = (p.K + BLOCK_K - 1) / BLOCK_K;
+  const int kc0 = static_cast<int>(static_cast<long long>(k_chunks) * split / p.splits);
+  const int kc1 = static_cast<int>(static_cast<long long>(k_chunks) * (split + 1) / p.splits);
+  const int n_k = kc1 - kc0;
+  constexpr uint32_t TMEM_COLS = BLOCK_N < 32 ? 32 : BLOCK_N;
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_x);
+    prefetch_tensormap(&tmap_w);
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(accum_bar, 1);
+    *abort_flag = 0;
+    *last_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, TMEM_COLS);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer
+    if (lane == 0) {
+      const uint32_t tx = a_stage_bytes + b_stage_bytes;
+      for (int i = 0; i < n_k; ++i) {
+        const int s = i % stages;
+        const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+        if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.error_word)) break;
+        mbar_arrive_expect_tx(&full_bar[s], tx);
+        const int kx = (kc0 + i) * BLOCK_K;
+        tma_load_2d(smem_b + static_cast<size_t>(s) * b_stage_bytes, &tmap_w, &full_bar[s], kx, n_tile * BLOCK_N);
+        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kx, m_tile * BLOCK_M);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
+      for (int i = 0; i < n_k; ++i) {
+        const int s = i % stages;
+        const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+        if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) break;
+        tc_fence_after();
+        const uint64_t adesc = make_smem_desc(smem_u32(smem_a + static_cast<size_t>(s) * a_stage_bytes));
+        const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + static_cast<size_t>(s) * b_stage_bytes));
+#pragma unroll
+        for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
+          // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in the (>>4) address field
+          umma_bf16(tmem_base, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
+                    (i > 0 || kk > 0) ? 1u : 0u);
+        }
+        umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+      }
+      umma_commit(accum_bar);  // accumulator complete
+    }
+  } else {
+    // ---------------- epilogue warps: TMEM lane group = warp % 4
+    const int lg = warp & 3;
+    const int row = lg * 32 + lane;
+    const int m = m_tile * BLOCK_M + row;
+    const int n0 = n_tile * BLOCK_N;
+    bool ok = (n_k == 0) || mbar_wait(accum_bar, 0, abort_flag, p.error_word);
+    ok = __all_sync(0xffffffffu, ok);
+    tc_fence_after();
+    // warp-uniform: does this lane group hold any row of X at all?
+    const bool warp_live = ok && (lg * 32 < p.a_rows) && (m_tile * BLOCK_M + lg * 32 < p.M);
+    const bool live = warp_live && m < p.M;
+    TmemSource tsrc{tmem_base + (static_cast<uint32_t>(lg * 32) << 16)};
+    if (p.splits == 1) {
+      if (warp_live && n_k > 0) run_epilogue<EPI, BLOCK_N>(tsrc, p, m, n0, live);
+    } else {
+      const int tile_id = n_tile * gridDim.x + m_tile;
+      float* part = p.partial + static_cast<size_t>(tile_id) * p.splits * BLOCK_N * 128;
+      if (warp_live) {
+        float* mine = part + static_cast<size_t>(split) * BLOCK_N * 128 + row;
+        for (int c = 0; c < BLOCK_N; c += 32) {
+          float v[32];
+          if (n_k > 0) tsrc.load(c, v);
+          else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = 0.f;
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) mine[static_cast<size_t>(c + j) * 128] = v[j];
+        }
+      }
+      __threadfence();
+      epi_bar_sync();
+      if (threadIdx.x == 64) {
+        int old = atomicAdd(&p.tile_count[tile_id], 1);
+        int last = (old == p.splits - 1) ? 1 : 0;
+        if (last) p.tile_count[tile_id] = 0;  // ready for the next launch
+        *last_flag = last;
+        __threadfence();
+      }
+      epi_bar_sync();
+      if (*last_flag && warp_live) {
+        PartialSource<BLOCK_N> psrc{part, p.splits, row};
+        run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, live);
+      }
+    }
+    tc_fence_before();
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+inline size_t gemm_tc_smem_bytes(int a_rows, int block_n, int stages) {
+  return 1024 + static_cast<size_t>(stages) * (a_rows * 128 + block_n * 128) + (2 * stages + 1) * 8 + 64 +
+         // slack so that the MMA's 128-row read of the last X stage stays inside the allocation
+         (a_rows < 128 ? 0 : 0);
+}
+
+}  // namespace tc
+}  // namespace d3

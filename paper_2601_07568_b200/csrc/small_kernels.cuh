@@ -1,0 +1,389 @@
+// Row-wise and per-sequence kernels around the matmuls: embedding gather, RMSNorm, RoPE + cache
+// write, softmax-statistics merge, the threshold unmask decision and the generate-loop bookkeeping.
+#pragma once
+#include "common.cuh"
+
+namespace d3 {
+
+// Per-sequence row map of one forward: row m belongs to sequence b = m / rows_per_seq at offset
+// r = m % rows_per_seq; it is live when r < n_valid[b] and sits at absolute position pos_base[b] + r;
+// its attention reads cache slots [0, kv_len[b]).
+struct RowMap {
+  const int* pos_base;
+  const int* n_valid;
+  const int* kv_len;
+  int rows_per_seq;
+  int bs;
+};
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ----------------------------------------------------------------------------- embedding
+template <typename T>
+__global__ void embed_kernel(const int* __restrict__ ids, const T* __restrict__ emb, float* __restrict__ x, int d,
+                             int vocab, uint32_t* error_word) {
+  const int m = blockIdx.x;
+  int id = ids[m];
+  if (id < 0 || id >= vocab) {
+    if (threadIdx.x == 0) atomicOr(error_word, ERRW_BAD_TOKEN_ID);
+    id = 0;
+  }
+  const T* src = emb + static_cast<size_t>(id) * d;
+  float* dst = x + static_cast<size_t>(m) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = TypeOps<T>::to_f(src[i]);
+}
+
+// ----------------------------------------------------------------------------- RMSNorm
+// xn[m, :] = T(x[m, :] * rsqrt(mean(x^2) + eps) * gain); fp32 arithmetic, fixed reduction order.
+template <typename T>
+__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain, T* __restrict__ xn, int d,
+                               float eps) {
+  const int m = blockIdx.x;
+  const float* row = x + static_cast<size_t>(m) * d;
+  float ss = 0.f;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) {
+    float v = row[i];
+    ss += v * v;
+  }
+  __shared__ float red[32];
+  ss = warp_sum(ss);
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float v = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
+    v = warp_sum(v);
+    if (threadIdx.x == 0) red[0] = v;
+  }
+  __syncthreads();
+  const float rstd = rsqrtf(red[0] / static_cast<float>(d) + eps);
+  T* out = xn + static_cast<size_t>(m) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) out[i] = TypeOps<T>::from_f(row[i] * rstd * gain[i]);
+}
+
+// ----------------------------------------------------------------------------- RoPE + cache write
+// qkv: fp32 [M, (hq + 2 hkv) * dh] straight from the projection.  q heads are rotated and stored as
+// T [M, hq*dh]; k heads are rotated and stored in the cache, v heads stored as they are.
+template <typename T>
+__global__ void rope_kv_kernel(const float* __restrict__ qkv, T* __restrict__ q_out, T* __restrict__ k_cache,
+                               T* __restrict__ v_cache, const float* __restrict__ rope_cos,
+                               const float* __restrict__ rope_sin, RowMap rm, int hq, int hkv, int dh, int max_seq,
+                               uint32_t* error_word) {
+  const int m = blockIdx.x;
+  const int b = m / rm.rows_per_seq, r = m % rm.rows_per_seq;
+  if (r >= rm.n_valid[b]) return;
+  const int pos = rm.pos_base[b] + r;
+  if (pos < 0 || pos >= max_seq) {
+    if (threadIdx.x == 0) atomicOr(error_word, ERRW_BAD_POSITION);
+    return;
+  }
+  const int half = dh / 2;
+  const int nq = hq * dh, nkv = hkv * dh;
+  const float* row = qkv + static_cast<size_t>(m) * (nq + 2 * nkv);
+  const float* cs = rope_cos + static_cast<size_t>(pos) * half;
+  const float* sn = rope_sin + static_cast<size_t>(pos) * half;
+  // rotated pairs of q and k
+  const int n_pairs = (hq + hkv) * half;
+  for (int i = threadIdx.x; i < n_pairs; i += blockDim.x) {
+    const int head = i / half, k = i % half;
+    const float a = row[head * dh + k], bb = row[head * dh + k + half];
+    const float lo = a * cs[k] - bb * sn[k];
+    const float hi = bb * cs[k] + a * sn[k];
+    if (head < hq) {
+      T* dst = q_out + static_cast<size_t>(m) * nq + head * dh;
+      dst[k] = TypeOps<T>::from_f(lo);
+      dst[k + half] = TypeOps<T>::from_f(hi);
+    } else {
+      T* dst = k_cache + ((static_cast<size_t>(b) * hkv + (head - hq)) * max_seq + pos) * dh;
+      dst[k] = TypeOps<T>::from_f(lo);
+      dst[k + half] = TypeOps<T>::from_f(hi);
+    }
+  }
+  for (int i = threadIdx.x; i < nkv; i += blockDim.x) {
+    const int head = i / dh, k = i % dh;
+    v_cache[((static_cast<size_t>(b) * hkv + head) * max_seq + pos) * dh + k] =
+        TypeOps<T>::from_f(row[nq + nkv + i]);
+  }
+}
+
+// ----------------------------------------------------------------------------- statistics merge
+// One warp per row merges the per-tile partial statistics in ascending tile order (fixed tree) and
+// writes confidence = 1/Z, entropy = ln Z - S/Z (nats) and the arg max.
+__global__ void stats_merge_kernel(const float4* __restrict__ part, int n_tiles, int M, float* __restrict__ conf,
+                                   float* __restrict__ entropy, int* __restrict__ argmax) {
+  const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (m >= M) return;
+  SoftStat st = stat_empty();
+  for (int t = lane; t < n_tiles; t += 32) {
+    float4 v = part[static_cast<size_t>(m) * n_tiles + t];
+    SoftStat o{v.x, v.y, v.z, __float_as_int(v.w)};
+    st = stat_merge(st, o);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    SoftStat other;
+    other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+    other.z = __shfl_xor_sync(0xffffffffu, st.z, o);
+    other.s = __shfl_xor_sync(0xffffffffu, st.s, o);
+    other.a = __shfl_xor_sync(0xffffffffu, st.a, o);
+    // keep the operand order fixed (lower lane first) so every lane computes the same bits
+    st = (lane & o) ? stat_merge(other, st) : stat_merge(st, other);
+  }
+  if (lane == 0) {
+    if (st.z > 0.f) {
+      conf[m] = 1.0f / st.z;
+      entropy[m] = fmaxf(logf(st.z) - st.s / st.z, 0.f);
+      argmax[m] = st.a;
+    } else {
+      conf[m] = 0.f;
+      entropy[m] = 0.f;
+      argmax[m] = 0;
+    }
+  }
+}
+
+// Statistics straight from fp32 logits rows (SIMT path and tests): one block per row.
+__global__ void stats_from_logits_kernel(const float* __restrict__ logits, int V, int mask_id, float4* __restrict__ part,
+                                         int n_tiles) {
+  // one warp per (row, 128-column tile); lanes stride the tile, then a fixed shuffle tree
+  const int m = blockIdx.y;
+  const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (t >= n_tiles) return;
+  const float* row = logits + static_cast<size_t>(m) * V;
+  SoftStat st = stat_empty();
+  for (int j = lane; j < 128; j += 32) {
+    int n = t * 128 + j;
+    if (n < V && n != mask_id) stat_add(st, row[n], n);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    SoftStat other;
+    other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+    other.z = __shfl_xor_sync(0xffffffffu, st.z, o);
+    other.s = __shfl_xor_sync(0xffffffffu, st.s, o);
+    other.a = __shfl_xor_sync(0xffffffffu, st.a, o);
+    st = (lane & o) ? stat_merge(other, st) : stat_merge(st, other);
+  }
+  if (lane == 0) part[static_cast<size_t>(m) * n_tiles + t] = make_float4(st.m, st.z, st.s, __int_as_float(st.a));
+}
+
+// ----------------------------------------------------------------------------- decision
+// One warp per sequence.  Commits every masked position clearing the threshold and always the most
+// confident masked one (lowest index on ties); writes ids, clears mask bytes, emits (pos, id) in
+// ascending position order.  Returns through the out arrays; `remaining` (optional) gets the number of
+// masks left.  B <= 128.
+struct UnmaskOut {
+  int committed;
+  int forced;     // 1 when the forced position did not clear the threshold
+  int remaining;
+};
+__device__ __forceinline__ UnmaskOut unmask_block(const float* conf, const float* ent, const int* argmax, int* ids,
+                                                  uint8_t* mask, int B, float tau, int mode, int* out_pos,
+                                                  int* out_ids, int* commit_step, int step) {
+  const int lane = threadIdx.x & 31;
+  // pass 1: best masked position
+  float best = -INFINITY;
+  int best_r = 0x7fffffff;
+  for (int r = lane; r < B; r += 32) {
+    if (mask[r]) {
+      float s = (mode == 0) ? conf[r] : -ent[r];
+      if (s > best || (s == best && r < best_r)) {
+        best = s;
+        best_r = r;
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    float ob = __shfl_xor_sync(0xffffffffu, best, o);
+    int orr = __shfl_xor_sync(0xffffffffu, best_r, o);
+    if (orr != 0x7fffffff && (best_r == 0x7fffffff || ob > best || (ob == best && orr < best_r))) {
+      best = ob;
+      best_r = orr;
+    }
+  }
+  UnmaskOut res{0, 0, 0};
+  if (best_r == 0x7fffffff) return res;  // nothing masked
+  int base = 0;
+  for (int r0 = 0; r0 < B; r0 += 32) {
+    const int r = r0 + lane;
+    bool masked = (r < B) && mask[r];
+    bool clears = masked && ((mode == 0) ? (conf[r] > tau) : (ent[r] < tau));
+    bool commit = clears || (masked && r == best_r);
+    if (masked && r == best_r && !clears) res.forced = 1;
+    unsigned bal = __ballot_sync(0xffffffffu, commit);
+    if (commit) {
+      int slot = base + __popc(bal & ((1u << lane) - 1u));
+      int tok = argmax[r];
+      ids[r] = tok;
+      mask[r] = 0;
+      if (out_pos) out_pos[slot] = r;
+      if (out_ids) out_ids[slot] = tok;
+      if (commit_step) commit_step[r] = step;
+    }
+    base += __popc(bal);
+    res.remaining += __popc(__ballot_sync(0xffffffffu, masked && !commit));
+  }
+  res.forced = __any_sync(0xffffffffu, res.forced) ? 1 : 0;
+  res.committed = base;
+  return res;
+}
+
+__global__ void unmask_kernel(const float* __restrict__ conf, const float* __restrict__ ent,
+                              const int* __restrict__ argmax, int* ids, uint8_t* mask, int B, float tau, int mode,
+                              int* out_pos, int* out_ids, int* out_count) {
+  const int b = blockIdx.x;
+  UnmaskOut r = unmask_block(conf + b * B, ent + b * B, argmax + b * B, ids + b * B, mask + b * B, B, tau, mode,
+                             out_pos ? out_pos + b * B : nullptr, out_ids ? out_ids + b * B : nullptr, nullptr, 0);
+  if (threadIdx.x == 0 && out_count) out_count[b] = r.committed;
+}
+
+// ----------------------------------------------------------------------------- generate bookkeeping
+enum : int { SEQ_DENOISE = 0, SEQ_FINALIZE = 1, SEQ_DONE = 2 };
+struct GenState {
+  int* mode;        // [bs] SEQ_*
+  int* block_idx;   // [bs]
+  int* step;        // [bs] denoise steps taken in the current block
+  int* prefix_len;  // [bs]
+  int* ids;         // [bs, B] current block
+  uint8_t* mask;    // [bs, B]
+  int* out_ids;     // [bs, gen_len]
+  int* commit_step; // [bs, gen_len] or null
+  long long* counters;  // [0] denoise fwd, [1] finalize fwd, [2] tokens, [3] forced, [4] seqs not done
+};
+
+// Row map of the next decode forward from the generate state (one thread per sequence).
+__global__ void gen_rowmap_kernel(GenState g, int bs, int B, int* pos_base, int* n_valid, int* kv_len) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= bs) return;
+  const bool live = g.mode[b] != SEQ_DONE;
+  pos_base[b] = g.prefix_len[b];
+  n_valid[b] = live ? B : 0;
+  kv_len[b] = live ? g.prefix_len[b] + B : 0;
+}
+
+// After a forward: sequences that ran a finalize forward append their block and start the next one;
+// sequences that ran a denoise forward take the unmask decision.  One warp per sequence.
+__global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, const float* __restrict__ ent,
+                                   const int* __restrict__ argmax, int bs, int B, int n_blocks, int gen_len, float tau,
+                                   int decide_mode, int mask_id) {
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31;
+  const int mode = g.mode[b];
+  if (mode == SEQ_DONE) return;
+  int* ids = g.ids + b * B;
+  uint8_t* mask = g.mask + b * B;
+  if (mode == SEQ_FINALIZE) {
+    const int j = g.block_idx[b];
+    for (int r = lane; r < B; r += 32) {
+      g.out_ids[static_cast<size_t>(b) * gen_len + j * B + r] = ids[r];
+      ids[r] = mask_id;
+      mask[r] = 1;
+    }
+    __syncwarp();
+    if (lane == 0) {
+      g.prefix_len[b] += B;
+      g.block_idx[b] = j + 1;
+      g.step[b] = 0;
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[1]), 1ull);
+      if (j + 1 >= n_blocks) {
+        g.mode[b] = SEQ_DONE;
+        atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[4]), static_cast<unsigned long long>(-1ll));
+      } else {
+        g.mode[b] = SEQ_DENOISE;
+      }
+    }
+    return;
+  }
+  const int step = g.step[b] + 1;
+  int* cs = g.commit_step ? g.commit_step + static_cast<size_t>(b) * gen_len + g.block_idx[b] * B : nullptr;
+  UnmaskOut r = unmask_block(conf + b * B, ent + b * B, argmax + b * B, ids, mask, B, tau, decide_mode, nullptr,
+                             nullptr, cs, step);
+  if (lane == 0) {
+    g.step[b] = step;
+    atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[0]), 1ull);
+    atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[2]), static_cast<unsigned long long>(r.committed));
+    atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[3]), static_cast<unsigned long long>(r.forced));
+    if (r.remaining == 0) g.mode[b] = SEQ_FINALIZE;
+  }
+}
+
+__global__ void gen_init_kernel(GenState g, int bs, int B, int mask_id) {
+  const int b = blockIdx.x;
+  for (int r = threadIdx.x; r < B; r += blockDim.x) {
+    g.ids[b * B + r] = mask_id;
+    g.mask[b * B + r] = 1;
+  }
+  if (threadIdx.x == 0) {
+    g.mode[b] = SEQ_DENOISE;
+    g.block_idx[b] = 0;
+    g.step[b] = 0;
+    if (b == 0) {
+      g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = 0;
+      g.counters[4] = bs;
+    }
+  }
+}
+
+// Row maps for the explicit API.
+__global__ void decode_rowmap_kernel(const int* prefix_len, int bs, int B, int* pos_base, int* n_valid, int* kv_len) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= bs) return;
+  pos_base[b] = prefix_len[b];
+  n_valid[b] = B;
+  kv_len[b] = prefix_len[b] + B;
+}
+__global__ void prefill_rowmap_kernel(const int* prompt_lens, int bs, int p_max, int* prefix_len, int* pos_base,
+                                      int* n_valid, int* kv_len) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= bs) return;
+  int len = prompt_lens[b];
+  len = len < 0 ? 0 : (len > p_max ? p_max : len);
+  prefix_len[b] = len;
+  pos_base[b] = 0;
+  n_valid[b] = len;
+  kv_len[b] = len;
+}
+__global__ void add_prefix_kernel(int* prefix_len, int bs, int B) {
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b < bs) prefix_len[b] += B;
+}
+
+template <typename T>
+__global__ void cast_to_f32_kernel(const T* __restrict__ src, float* __restrict__ dst, size_t n) {
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = TypeOps<T>::to_f(src[i]);
+}
+template <typename T>
+__global__ void cast_from_f32_kernel(const float* __restrict__ src, T* __restrict__ dst, size_t n) {
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = TypeOps<T>::from_f(src[i]);
+}
+
+// Weight repacking on the device: dst rows [r0, r0+rows) <- src rows; and gate/up interleave.
+template <typename T>
+__global__ void copy_rows_kernel(const T* __restrict__ src, T* __restrict__ dst, size_t n) {
+  size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = src[i];
+}
+// dst [2f, d]: group g of 128 rows = gate rows [64g, 64g+64) then up rows [64g, 64g+64).
+template <typename T>
+__global__ void interleave_gate_up_kernel(const T* __restrict__ gate, const T* __restrict__ up, T* __restrict__ dst,
+                                          int f, int d) {
+  const int row = blockIdx.x;  // 0 .. 2f-1 in dst
+  const int g = row / 128, w = row % 128;
+  const int h = g * 64 + (w % 64);
+  if (h >= f) {  // padding rows of a ragged last group
+    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[static_cast<size_t>(row) * d + i] = TypeOps<T>::from_f(0.f);
+    return;
+  }
+  const T* src = (w < 64 ? gate : up) + static_cast<size_t>(h) * d;
+  for (int i = threadIdx.x; i < d; i += blockDim.x) dst[static_cast<size_t>(row) * d + i] = src[i];
+}
+
+}  // namespace d3

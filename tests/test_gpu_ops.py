@@ -1,0 +1,255 @@
+"""Per-kernel parity: each operator called through the C ABI against the oracle's definition."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import d3_oracle as o
+from paper_2601_07568_b200 import binding as d3
+from paper_2601_07568_b200 import synth_inputs as si
+from gpu_utils import DEV, Ctx
+
+pytestmark = pytest.mark.gpu
+
+BF16_SHAPE = si.scaled_shape(si.LLADA8B, name="ops-bf16", n_layers=1, d_model=256, n_q_heads=4, n_kv_heads=2,
+                             d_ffn=512, vocab=1000, d_head=64)
+F32_SHAPE = si.scaled_shape(si.TINY, name="ops-f32", n_layers=1, d_model=128, n_q_heads=4, n_kv_heads=2,
+                            d_ffn=256, vocab=1000, d_head=32)
+
+
+@pytest.fixture(scope="module")
+def ctx_bf16():
+    with Ctx(BF16_SHAPE, None, block=32, max_batch=32, max_seq=640) as c:
+        yield c
+
+
+@pytest.fixture(scope="module")
+def ctx_f32():
+    with Ctx(F32_SHAPE, None, block=16, max_batch=8, max_seq=256) as c:
+        yield c
+
+
+def rand_bf16(rng, shape, scale=1.0):
+    x = (rng.standard_normal(shape) * scale).astype(np.float32)
+    t = torch.from_numpy(x).to(torch.bfloat16)
+    return t, t.float().numpy().astype(np.float64)
+
+
+def swiglu_ref(y, n):
+    # columns in groups of 128: 64 gate then 64 up
+    g = y.reshape(y.shape[0], n // 128, 2, 64)
+    return (o.silu(g[:, :, 0]) * g[:, :, 1]).reshape(y.shape[0], n // 2)
+
+
+LINEAR_SHAPES = [(32, 256, 128), (16, 128, 64), (48, 200, 192), (130, 384, 256), (1, 128, 4096), (32, 4096, 4096),
+                 (256, 640, 1024), (1024, 256, 512)]
+
+
+@pytest.mark.parametrize("m,n,k", LINEAR_SHAPES)
+@pytest.mark.parametrize("splits", [0, 1, 3])
+def test_linear_bf16_tensor_core(ctx_bf16, m, n, k, splits):
+    rng = np.random.default_rng(m * 7 + n + k)
+    xt, x = rand_bf16(rng, (m, k))
+    wt, w = rand_bf16(rng, (n, k), 0.05)
+    ref = x @ w.T
+    tol = 2e-5 * np.sqrt(k) * np.abs(ref).max() + 1e-6
+    xd, wd = xt.to(DEV), wt.to(DEV)
+    # fp32 out
+    y = torch.full((m, n), 7.0, dtype=torch.float32, device=DEV)
+    d3.d3_op_linear(ctx_bf16.ctx, xd, wd, y, 0, splits)
+    assert np.max(np.abs(y.cpu().numpy() - ref)) <= tol
+    # residual: y += x w^T
+    y0 = rng.standard_normal((m, n)).astype(np.float32)
+    y = torch.from_numpy(y0).to(DEV)
+    d3.d3_op_linear(ctx_bf16.ctx, xd, wd, y, 2, splits)
+    assert np.max(np.abs(y.cpu().numpy() - (ref + y0))) <= tol + 1e-6
+    # bf16 out
+    y = torch.zeros((m, n), dtype=torch.bfloat16, device=DEV)
+    d3.d3_op_linear(ctx_bf16.ctx, xd, wd, y, 1, splits)
+    assert np.max(np.abs(y.float().cpu().numpy() - ref)) <= tol + 2 ** -8 * np.abs(ref).max()
+    # SwiGLU
+    if n % 128 == 0:
+        y = torch.zeros((m, n // 2), dtype=torch.bfloat16, device=DEV)
+        d3.d3_op_linear(ctx_bf16.ctx, xd, wd, y, 3, splits)
+        sref = swiglu_ref(ref, n)
+        assert np.max(np.abs(y.float().cpu().numpy() - sref)) <= 2 ** -7 * np.abs(sref).max() + 4 * tol
+    assert ctx_bf16.error_word() == 0
+
+
+def test_linear_bf16_repeated_launches_keep_split_counters_clean(ctx_bf16):
+    rng = np.random.default_rng(3)
+    xt, x = rand_bf16(rng, (32, 1024))
+    wt, w = rand_bf16(rng, (256, 1024), 0.05)
+    ref = x @ w.T
+    xd, wd = xt.to(DEV), wt.to(DEV)
+    outs = []
+    for _ in range(4):
+        y = torch.zeros((32, 256), dtype=torch.float32, device=DEV)
+        d3.d3_op_linear(ctx_bf16.ctx, xd, wd, y, 0, 4)
+        outs.append(y.cpu().numpy())
+    assert all(np.array_equal(outs[0], a) for a in outs[1:])  # deterministic split-K
+    assert np.max(np.abs(outs[0] - ref)) <= 1e-3 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("m,n,k", [(16, 128, 128), (5, 100, 100), (33, 256, 72), (64, 512, 128)])
+def test_linear_fp32_simt(ctx_f32, m, n, k):
+    rng = np.random.default_rng(m + n + k)
+    x = rng.standard_normal((m, k)).astype(np.float32)
+    w = (rng.standard_normal((n, k)) * 0.05).astype(np.float32)
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    tol = 2e-6 * np.sqrt(k) * np.abs(ref).max()
+    xd, wd = torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV)
+    y = torch.zeros((m, n), dtype=torch.float32, device=DEV)
+    d3.d3_op_linear(ctx_f32.ctx, xd, wd, y, 0)
+    assert np.max(np.abs(y.cpu().numpy() - ref)) <= tol
+    y2 = torch.zeros((m, n), dtype=torch.float32, device=DEV)
+    d3.d3_op_linear(ctx_f32.ctx, xd, wd, y2, 1)
+    assert torch.equal(y, y2)
+    d3.d3_op_linear(ctx_f32.ctx, xd, wd, y2, 2)
+    assert np.max(np.abs(y2.cpu().numpy() - 2 * ref)) <= 2 * tol
+    if n % 128 == 0:
+        y3 = torch.zeros((m, n // 2), dtype=torch.float32, device=DEV)
+        d3.d3_op_linear(ctx_f32.ctx, xd, wd, y3, 3)
+        sref = swiglu_ref(ref, n)
+        assert np.max(np.abs(y3.cpu().numpy() - sref)) <= 1e-5 * np.abs(sref).max() + 4 * tol
+
+
+def _stats_case(ctx, bf16, m, V, k, mask_id, scale, seed):
+    rng = np.random.default_rng(seed)
+    if bf16:
+        xt, x = rand_bf16(rng, (m, k))
+        wt, w = rand_bf16(rng, (V, k), 0.05)
+    else:
+        x32 = rng.standard_normal((m, k)).astype(np.float32)
+        w32 = (rng.standard_normal((V, k)) * 0.05).astype(np.float32)
+        xt, wt, x, w = torch.from_numpy(x32), torch.from_numpy(w32), x32.astype(np.float64), w32.astype(np.float64)
+    lg = scale * (x @ w.T)
+    p, conf, tok, ent = o.softmax_stats(lg, mask_id)
+    part = np.partition(p, -2, axis=-1)
+    gap = part[:, -1] - part[:, -2]
+    c = torch.zeros(m, dtype=torch.float32, device=DEV)
+    e = torch.zeros(m, dtype=torch.float32, device=DEV)
+    a = torch.zeros(m, dtype=torch.int32, device=DEV)
+    d3.d3_op_lm_head_stats(ctx.ctx, xt.to(DEV), wt.to(DEV), scale, mask_id, c, e, a)
+    c, e, a = c.cpu().numpy(), e.cpu().numpy(), a.cpu().numpy()
+    tol = 3e-3 if bf16 else 2e-4
+    assert np.max(np.abs(c - conf)) <= tol
+    assert np.max(np.abs(e - ent)) <= 3 * tol
+    bad = (a != tok) & (gap >= 1e-3)
+    assert not bad.any()
+    assert np.all(a != mask_id)
+
+
+@pytest.mark.parametrize("V,mask_id", [(1000, 999), (1000, 500), (512, 511), (128, 0), (300, 130)])
+def test_lm_head_stats_bf16(ctx_bf16, V, mask_id):
+    _stats_case(ctx_bf16, True, 32, V, 256, mask_id, 20.0, V + mask_id)
+    _stats_case(ctx_bf16, True, 17, V, 128, mask_id, 3.0, V + mask_id + 1)
+
+
+@pytest.mark.parametrize("V,mask_id", [(1000, 999), (512, 511), (77, 3)])
+def test_lm_head_stats_fp32(ctx_f32, V, mask_id):
+    _stats_case(ctx_f32, False, 16, V, 128, mask_id, 20.0, V)
+    _stats_case(ctx_f32, False, 7, V, 100, mask_id, 2.0, V + 1)
+
+
+def test_lm_head_stats_special_rows(ctx_f32):
+    # all-equal logits -> conf = 1/(V-1), H = ln(V-1), token 0; one dominant column -> conf ~ 1, H ~ 0
+    V, k = 300, 64
+    x = np.zeros((2, k), dtype=np.float32)
+    x[1, 0] = 1.0
+    w = np.zeros((V, k), dtype=np.float32)
+    w[123, 0] = 5.0
+    c = torch.zeros(2, dtype=torch.float32, device=DEV)
+    e = torch.zeros(2, dtype=torch.float32, device=DEV)
+    a = torch.zeros(2, dtype=torch.int32, device=DEV)
+    d3.d3_op_lm_head_stats(ctx_f32.ctx, torch.from_numpy(x).to(DEV), torch.from_numpy(w).to(DEV), 20.0, V - 1, c, e, a)
+    c, e, a = c.cpu().numpy(), e.cpu().numpy(), a.cpu().numpy()
+    assert abs(c[0] - 1.0 / (V - 1)) < 1e-7 and abs(e[0] - np.log(V - 1)) < 1e-5 and a[0] == 0
+    assert c[1] > 1 - 1e-6 and e[1] < 1e-5 and a[1] == 123
+
+
+def _attention_case(ctx, shape, bf16, bs, rows, kv_lens, seed):
+    rng = np.random.default_rng(seed)
+    hq, hkv, dh = shape.n_q_heads, shape.n_kv_heads, shape.d_head
+    rnd = (lambda s: rand_bf16(rng, s)) if bf16 else (
+        lambda s: (lambda a: (torch.from_numpy(a), a.astype(np.float64)))(rng.standard_normal(s).astype(np.float32)))
+    qt, q = rnd((bs * rows, hq * dh))
+    refs = []
+    for b in range(bs):
+        L = kv_lens[b]
+        kt, k = rnd((hkv, L, dh))
+        vt, v = rnd((hkv, L, dh))
+        d3.d3_op_write_kv(ctx.ctx, 0, b, 0, kt.float().to(DEV).contiguous(), vt.float().to(DEV).contiguous())
+        qb = q[b * rows:(b + 1) * rows].reshape(rows, hq, dh)
+        refs.append(o.attention(qb, k.transpose(1, 0, 2), v.transpose(1, 0, 2)).reshape(rows, hq * dh))
+    ref = np.concatenate(refs)
+    out = torch.zeros_like(qt, device=DEV)
+    d3.d3_op_attention(ctx.ctx, qt.to(DEV), 0, bs, rows, torch.tensor(kv_lens, dtype=torch.int32, device=DEV), out)
+    got = out.float().cpu().numpy()
+    tol = (2 ** -7 if bf16 else 2e-5) * np.abs(ref).max()
+    assert np.max(np.abs(got - ref)) <= tol
+    assert ctx.error_word() == 0
+
+
+@pytest.mark.parametrize("rows,kv_lens", [(32, [64, 33, 1]), (7, [40, 300, 5]), (32, [600, 32, 257])])
+def test_attention_bf16(ctx_bf16, rows, kv_lens):
+    _attention_case(ctx_bf16, BF16_SHAPE, True, 3, rows, kv_lens, rows + sum(kv_lens))
+
+
+@pytest.mark.parametrize("rows,kv_lens", [(16, [48, 17]), (5, [5, 200])])
+def test_attention_fp32(ctx_f32, rows, kv_lens):
+    _attention_case(ctx_f32, F32_SHAPE, False, 2, rows, kv_lens, rows)
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_unmask_matches_oracle_decision(mode):
+    shape = F32_SHAPE
+    with Ctx(shape, None, block=32, max_batch=64, max_seq=64, decide_mode=mode) as c:
+        rng = np.random.default_rng(mode)
+        bs, B = 64, 32
+        grid = np.array([0.05, 0.3, 0.3, 0.6, 0.9, 0.9, 0.95], dtype=np.float32)
+        conf = rng.choice(grid, size=(bs, B)).astype(np.float32)
+        ent = rng.choice(grid, size=(bs, B)).astype(np.float32)
+        tok = rng.integers(0, 900, size=(bs, B)).astype(np.int32)
+        mask = rng.random((bs, B)) < 0.6
+        mask[0] = False
+        mask[1] = True
+        ids = np.where(mask, shape.mask_id, 5).astype(np.int32)
+        for tau in (0.3, 0.6, 1.0, 0.0):
+            t = lambda a, dt: torch.tensor(a, dtype=dt, device=DEV)
+            idt, mt = t(ids, torch.int32), t(mask.astype(np.uint8), torch.uint8)
+            pos = torch.full((bs, B), -1, dtype=torch.int32, device=DEV)
+            oid = torch.full((bs, B), -1, dtype=torch.int32, device=DEV)
+            cnt = torch.zeros(bs, dtype=torch.int32, device=DEV)
+            d3.d3_op_unmask(c.ctx, t(conf.reshape(-1), torch.float32), t(ent.reshape(-1), torch.float32),
+                            t(tok.reshape(-1), torch.int32), idt, mt, tau, pos, oid, cnt)
+            idn, mn, pos, oid, cnt = (a.cpu().numpy() for a in (idt, mt, pos, oid, cnt))
+            for b in range(bs):
+                commit = o.decide(conf[b], ent[b], mask[b], np.float32(tau), mode)
+                assert cnt[b] == commit.sum()
+                assert np.array_equal(pos[b, :cnt[b]], np.flatnonzero(commit))
+                assert np.array_equal(oid[b, :cnt[b]], tok[b][commit])
+                assert np.array_equal(mn[b].astype(bool), mask[b] & ~commit)
+                assert np.array_equal(idn[b], np.where(commit, tok[b], ids[b]))
+
+
+def test_argument_errors(ctx_f32):
+    L = d3.lib()
+    import ctypes as C
+    assert L.d3_create(None, None, None) == d3.D3_ERR_INVALID_ARG
+    bad = d3.make_config(F32_SHAPE, block=16, max_batch=1, max_seq=64)
+    bad.d_head = 48
+    out = C.c_void_p(0)
+    assert L.d3_create(C.byref(bad), None, C.byref(out)) == d3.D3_ERR_UNSUPPORTED
+    ids = torch.zeros((1, 16), dtype=torch.int32, device=DEV)
+    m = torch.ones((1, 16), dtype=torch.uint8, device=DEV)
+    cnt = torch.zeros(1, dtype=torch.int32, device=DEV)
+    with pytest.raises(d3.D3Error) as ei:
+        d3.d3_denoise_step(ctx_f32.ctx, ids, m, 0.9, ids.clone(), ids.clone(), cnt)
+    assert ei.value.code == d3.D3_ERR_STATE  # no weights / prefill yet
+    with pytest.raises(d3.D3Error) as ei:
+        d3.d3_denoise_step(ctx_f32.ctx, ids, m, float("nan"), ids.clone(), ids.clone(), cnt)
+    assert ei.value.code == d3.D3_ERR_INVALID_ARG
+    with pytest.raises(d3.D3Error) as ei:
+        d3.d3_prefill(ctx_f32.ctx, ids, cnt)
+    assert ei.value.code == d3.D3_ERR_STATE
+    assert d3.lib().d3_strerror(-5).decode().startswith("bounded")
