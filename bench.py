@@ -1,0 +1,376 @@
+#!/usr/bin/env python
+"""Benchmark of the masked-block denoising path on B200.
+
+One "step" is one whole request of the workload through the hot path: prefill of the prompt, then
+block-by-block threshold decoding (denoise forwards + decisions + one finalize forward per block)
+until gen_len tokens are committed.  The metric is decoded tokens per second.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+N > 1 (launched under torchrun) runs independent replicas, one per GPU, with no collective on the
+data path; value = tokens of all replicas / max-over-ranks time ("weak" scaling).
+`--impl reference` times the CPU oracle (oracle/) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "decoded tokens/s"
+UNIT = "tokens/s"
+
+
+def host_cores() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------- clocks
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- oracle sample
+_SAMPLE_WEIGHTS = {}
+
+
+def oracle_sample(workload, n_denoise: int, n_finalize: int, layers=(0, 1)):
+    """Time the CPU oracle, as it stands, on a bounded sample of the workload: the given layers of one
+    block forward (M = block rows against a prompt-length prefix) and of one prompt forward, and the
+    LM head with its statistics on one block; extrapolate to a whole request."""
+    from oracle import d3_oracle as o
+    from paper_2601_07568_b200 import synth_inputs as si
+    shape = workload.model
+    dtype = np.float64 if shape.dtype == "fp32" else np.float32
+    key = (shape.name, tuple(layers))
+    if key not in _SAMPLE_WEIGHTS:  # input generation is not part of the timed work
+        _SAMPLE_WEIGHTS[key] = {"layers": {l: si.gen_layer(shape, l) for l in layers},
+                                "lm_head": si.gen_tensor(shape, "lm_head"),
+                                "tok_emb": si.gen_tensor(shape, "tok_emb", rows=(0, 8))}
+    W = _SAMPLE_WEIGHTS[key]
+    model = o.model_from_shape(shape, W, dtype)
+    rng = np.random.default_rng(0)
+    B, P = workload.block, workload.prompt_max
+    kp = rng.standard_normal((P, shape.n_kv_heads, shape.d_head)).astype(dtype)
+    x = rng.standard_normal((B, shape.d_model)).astype(dtype)
+    xp = rng.standard_normal((P, shape.d_model)).astype(dtype)
+    t0 = time.perf_counter()
+    for l in layers:
+        model.layer_forward(l, x, P + np.arange(B), kp, kp)
+    t_layer = (time.perf_counter() - t0) / len(layers)
+    t0 = time.perf_counter()
+    for l in layers:
+        model.layer_forward(l, xp, np.arange(P), None, None)
+    t_layer_prefill = (time.perf_counter() - t0) / len(layers)
+    t0 = time.perf_counter()
+    lg = model.logits(x)
+    o.softmax_stats(lg, shape.mask_id)
+    t_head = time.perf_counter() - t0
+    L = shape.n_layers
+    per_seq = (n_denoise * (L * t_layer + t_head) + n_finalize * L * t_layer + L * t_layer_prefill)
+    tokens_per_s = workload.gen_len / per_seq  # sequences are independent: same rate for any batch on one host
+    sample = (f"layers {list(layers)} of one {B}-row block forward at prefix {P} ({t_layer * 1e3:.0f} ms/layer), of one "
+              f"{P}-row prompt forward ({t_layer_prefill * 1e3:.0f} ms/layer) and the LM head + statistics on one block "
+              f"({t_head * 1e3:.0f} ms); extrapolated to {L} layers and {n_denoise} denoise + {n_finalize} finalize forwards per sequence")
+    return tokens_per_s, sample, dict(ms_layer=t_layer * 1e3, ms_layer_prefill=t_layer_prefill * 1e3, ms_head=t_head * 1e3)
+
+
+def default_forward_counts(workload):
+    """Forward counts for the reference arm when no GPU run supplies them: one token per forward (the
+    behaviour of these random-init models at the configured threshold) plus one finalize per block."""
+    return workload.gen_len, workload.gen_len // workload.block
+
+
+def run_reference(args):
+    from paper_2601_07568_b200 import synth_inputs as si
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    w = si.WORKLOADS[args.workload]
+    nd, nf = default_forward_counts(w)
+    vals, sample = [], ""
+    for i in range(args.warmup + args.steps):
+        v, sample, _ = oracle_sample(w, nd, nf, layers=(0,))
+        if i >= args.warmup:
+            vals.append(v)
+    value = float(np.mean(vals))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * w.batch * w.gen_len / value,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64" if w.model.dtype == "fp32" else "f32", "data": "synthetic",
+            "config": workload_config(w),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(w):
+    return {"workload": f"{w.name}: {w.model.name}, batch {w.batch}, prompt {w.prompt_min}-{w.prompt_max}, "
+                        f"generate {w.gen_len}, block {w.block}, threshold {w.threshold}",
+            "l2": "inputs larger than L2 (weights read once per forward)", "replicas": "independent per GPU"}
+
+
+# ----------------------------------------------------------------------------- our arm
+def gemm_bytes(shape, M):
+    """Algorithmic bytes of each matmul launch of one M-row forward: weights + inputs + outputs."""
+    d, f, V = shape.d_model, shape.d_ffn, shape.vocab
+    nq, nkv = shape.n_q_heads * shape.d_head, shape.n_kv_heads * shape.d_head
+    return {
+        "gemm_qkv": (nq + 2 * nkv) * d * 2 + M * d * 2 + M * (nq + 2 * nkv) * 2,
+        "gemm_o": d * nq * 2 + M * nq * 2 + 2 * M * d * 4,
+        "gemm_gate_up": 2 * f * d * 2 + M * d * 2 + M * f * 2,
+        "gemm_down": d * f * 2 + M * f * 2 + 2 * M * d * 4,
+        "gemm_head": V * d * 2 + M * d * 2 + M * ((V + 127) // 128) * 16,
+    }
+
+
+def gemm_flops(shape, M):
+    d, f, V = shape.d_model, shape.d_ffn, shape.vocab
+    nq, nkv = shape.n_q_heads * shape.d_head, shape.n_kv_heads * shape.d_head
+    return {"gemm_qkv": 2 * M * (nq + 2 * nkv) * d, "gemm_o": 2 * M * d * nq, "gemm_gate_up": 2 * M * 2 * f * d,
+            "gemm_down": 2 * M * d * f, "gemm_head": 2 * M * V * d}
+
+
+def run_ours(args):
+    import torch
+    from paper_2601_07568_b200 import binding as d3
+    from paper_2601_07568_b200 import build as d3build
+    from paper_2601_07568_b200 import synth_inputs as si
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    d3build.build()
+    w = si.WORKLOADS[args.workload]
+    shape = w.model
+    t0 = time.time()
+    W = si.gen_weights(shape)
+    t_gen = time.time() - t0
+    cfg = d3.make_config(shape, block=w.block, max_batch=w.batch, max_seq=w.max_seq,
+                         max_prefill_rows=w.batch * w.prompt_max)
+    ctx = d3.d3_create(cfg)
+    d3.d3_load_weights(ctx, d3.weights_from_numpy(shape, W), shape.n_layers)
+    del W
+    ids_np, lens_np = si.gen_prompts(w)
+    ids_pin = torch.from_numpy(ids_np).pin_memory()
+    lens_pin = torch.from_numpy(lens_np).pin_memory()
+    ids_dev, lens_dev = ids_pin.to(dev), lens_pin.to(dev)
+    out_dev = torch.zeros((w.batch, w.gen_len), dtype=torch.int32, device=dev)
+    out_pin = torch.zeros((w.batch, w.gen_len), dtype=torch.int32).pin_memory()
+
+    def step_resident():
+        d3.d3_prefill(ctx, ids_dev, lens_dev)
+        return d3.d3_generate(ctx, w.gen_len, w.threshold, out_dev)
+
+    def step_e2e():
+        a = ids_pin.to(dev, non_blocking=True)
+        b = lens_pin.to(dev, non_blocking=True)
+        d3.d3_prefill(ctx, a, b)
+        st = d3.d3_generate(ctx, w.gen_len, w.threshold, out_dev)
+        out_pin.copy_(out_dev, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        return st
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(fn, k):
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        st = None
+        for _ in range(k):
+            st = fn()
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
+        return ms, st
+
+    for _ in range(args.warmup):
+        step_resident()
+    clocks = ClockSampler(local)
+    clocks.start()
+    launches0 = d3.d3_launch_count(ctx)
+    ms_total, st = timed(step_resident, args.steps)
+    launches = d3.d3_launch_count(ctx) - launches0
+    clock_info = clocks.stop()
+    ms_e2e, _ = timed(step_e2e, args.steps)
+
+    # per-class kernel times of the decode loop (one request, events around every launch)
+    d3.d3_prefill(ctx, ids_dev, lens_dev)
+    torch.cuda.synchronize()
+    d3.d3_profile_enable(ctx, True)
+    st_prof = d3.d3_generate(ctx, w.gen_len, w.threshold, out_dev)
+    prof = d3.d3_profile_read(ctx)
+    d3.d3_profile_enable(ctx, False)
+    # prefill alone
+    ms_prefill, _ = timed(lambda: d3.d3_prefill(ctx, ids_dev, lens_dev), 3)
+    ms_prefill /= 3
+    err_word = d3.d3_get_error_word(ctx)
+    tokens = w.batch * w.gen_len
+    value = world * tokens * args.steps / (ms_total / 1e3)
+    e2e_value = world * tokens * args.steps / (ms_e2e / 1e3)
+    ms_step = ms_total / args.steps
+
+    peaks = measured_peaks()
+    M = w.batch * w.block
+    gb = gemm_bytes(shape, M)
+    gf = gemm_flops(shape, M)
+    tot_bytes = sum(gb[k] * prof[k]["launches"] for k in gb)
+    tot_flops = sum(gf[k] * prof[k]["launches"] for k in gf)
+    tot_ms = sum(prof[k]["ms"] for k in gb)
+    n_gemm = sum(prof[k]["launches"] for k in gb)
+    hbm_bound = tot_flops / max(tot_bytes, 1) < peaks["bf16_tflops_sustained"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if hbm_bound:
+        achieved = tot_bytes / (tot_ms / 1e3) / 1e9 if tot_ms > 0 else 0.0
+        roofline = {"bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "frac_of_8TBs_nominal": achieved / 8000.0}
+    else:
+        achieved = tot_flops / (tot_ms / 1e3) / 1e12 if tot_ms > 0 else 0.0
+        roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None}
+    roofline.update({"kernel": "gemm_tc_kernel (all matmul launches of the decode loop)", "peak_source": f"of {peaks['source']}",
+                     "launches": n_gemm, "avg_launch_us": 1e3 * tot_ms / max(n_gemm, 1),
+                     "algorithmic_bytes_per_launch": tot_bytes / max(n_gemm, 1)})
+    per_class = {}
+    for k, v in prof.items():
+        if v["launches"] == 0:
+            continue
+        e = {"ms": round(v["ms"], 3), "launches": v["launches"], "us_per_launch": round(1e3 * v["ms"] / v["launches"], 2)}
+        if k in gb and v["ms"] > 0:
+            e["GB/s"] = round(gb[k] * v["launches"] / (v["ms"] / 1e3) / 1e9, 1)
+            e["TFLOP/s"] = round(gf[k] * v["launches"] / (v["ms"] / 1e3) / 1e12, 1)
+        per_class[k] = e
+    forwards = st.steps
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32",
+        "data": "synthetic", "config": workload_config(w),
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(ids_pin.numel() * 4 + lens_pin.numel() * 4),
+                "d2h_bytes_per_step": int(out_pin.numel() * 4)},
+        "gpu_launches": int(launches), "clocks": clock_info, "roofline": roofline,
+        "decode": {"forwards_per_request": int(forwards), "denoise_forwards": int(st.denoise_forwards),
+                   "finalize_forwards": int(st.finalize_forwards), "tokens_per_denoise_forward": tokens / max(st.denoise_forwards, 1),
+                   "tokens_per_forward_incl_finalize": tokens / max(st.denoise_forwards + st.finalize_forwards, 1),
+                   "ms_per_forward": (ms_step - ms_prefill) / max(forwards, 1), "prefill_ms": ms_prefill,
+                   "forced_commits": int(st.forced_commits)},
+        "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
+        "device_bytes": d3.d3_device_bytes(ctx),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        nd = int(st.denoise_forwards // w.batch)
+        nf = int(st.finalize_forwards // w.batch)
+        v, sample, _ = oracle_sample(w, nd, nf)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": sample}
+    d3.d3_destroy(ctx)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="c2", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -105,7 +105,7 @@ int d3_create(const d3_config *cfg, void *cuda_stream, d3_ctx **out);
 void d3_destroy(d3_ctx *ctx);
 
 /* Copy the weights into context-owned device memory, repacked for the kernels (q,k,v rows
- * concatenated; gate/up rows interleaved in groups of 64).  src_is_device: 0 = host pointers,
+ * concatenated with each RoPE pair of a head adjacent; gate/up rows interleaved).  src_is_device: 0 = host pointers,
  * 1 = device pointers.  Synchronises the stream before returning. */
 int d3_load_weights(d3_ctx *ctx, const d3_weights *w, int src_is_device);
 
@@ -166,8 +166,8 @@ int d3_set_state(d3_ctx *ctx, const int32_t *prefix_len, int32_t bs);
 /* Single operators through the same kernels the path uses (per-kernel parity tests).
  * d3_op_linear: y = x . w^T.  x [device][m, k], w [device][n, k] in the context dtype;
  *   epilogue 0: y fp32 [m, n];  1: y in context dtype [m, n];  2: y fp32 [m, n] += product
- *   (residual);  3: w holds gate/up rows interleaved in groups of 64 (n = 2*f), y in context dtype
- *   [m, f] = silu(gate) * up.   splits: split-K factor for the tensor-core kernel (0 = auto).
+ *   (residual);  3: w holds gate/up rows interleaved (row 2j = gate j, row 2j+1 = up j; n = 2*f), y in
+ *   context dtype [m, f] = silu(gate) * up.   splits: split-K factor for the tensor-core kernel (0 = auto).
  * d3_op_lm_head_stats: conf/entropy/argmax [device][m] of scale * x . w^T with mask_id excluded.
  * d3_op_attention: q [device][bs*rows, n_q_heads*d_head]; keys/values are the context's cache of
  *   `layer`; sequence b attends to its slots [0, kv_len[b]); out like q.  kv_len [device][bs].
@@ -182,6 +182,17 @@ int d3_op_write_kv(d3_ctx *ctx, int32_t layer, int32_t seq, int32_t pos0, int32_
 int d3_op_unmask(d3_ctx *ctx, const float *conf, const float *entropy, const int32_t *argmax,
                  int32_t *block_ids, uint8_t *mask, float threshold, int32_t bs, int32_t *out_pos,
                  int32_t *out_ids, int32_t *out_count);
+
+/* Per-class kernel timing for measurement runs.  While enabled, every launch of the forward pass is
+ * bracketed by a CUDA event pair on the context's stream; d3_profile_read waits for the stream and
+ * returns, per class, the summed elapsed milliseconds and the number of launches since enabling.
+ * ms, launches: [host] arrays of D3_PROF_CLASSES entries.  Off by default (it costs two event
+ * records per launch). */
+enum { D3_PROF_GEMM_QKV = 0, D3_PROF_GEMM_O = 1, D3_PROF_GEMM_GATE_UP = 2, D3_PROF_GEMM_DOWN = 3,
+       D3_PROF_GEMM_HEAD = 4, D3_PROF_GEMM_OTHER = 5, D3_PROF_ATTENTION = 6, D3_PROF_RMSNORM = 7,
+       D3_PROF_OTHER = 8, D3_PROF_CLASSES = 9 };
+int d3_profile_enable(d3_ctx *ctx, int on);
+int d3_profile_read(d3_ctx *ctx, double *ms, int64_t *launches);
 
 /* Device error word: 0 when no bounded wait has given up and no kernel saw an invalid index.
  * Synchronises the stream.  Returns D3_OK and writes the word, or D3_ERR_CUDA. */

@@ -27,7 +27,7 @@ EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
     "d3_get_state", "d3_set_state", "d3_op_linear", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
+    "d3_op_write_kv", "d3_op_unmask", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
 
@@ -248,6 +248,22 @@ def d3_op_unmask(ctx, conf: torch.Tensor, entropy: torch.Tensor, argmax: torch.T
                                    _ptr(_dev(mask, torch.uint8)), C.c_float(threshold),
                                    C.c_int32(block_ids.shape[0]), _ptr(_dev(out_pos, torch.int32)),
                                    _ptr(_dev(out_ids, torch.int32)), _ptr(_dev(out_count, torch.int32))))
+
+
+PROF_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_head", "gemm_other", "attention",
+                "rmsnorm", "other")
+
+
+def d3_profile_enable(ctx, on: bool) -> None:
+    _check(ctx, lib().d3_profile_enable(ctx, C.c_int(1 if on else 0)))
+
+
+def d3_profile_read(ctx) -> Dict[str, Dict[str, float]]:
+    n = len(PROF_CLASSES)
+    ms = (C.c_double * n)()
+    cnt = (C.c_int64 * n)()
+    _check(ctx, lib().d3_profile_read(ctx, ms, cnt))
+    return {name: {"ms": float(ms[i]), "launches": int(cnt[i])} for i, name in enumerate(PROF_CLASSES)}
 
 
 def d3_get_error_word(ctx) -> int:

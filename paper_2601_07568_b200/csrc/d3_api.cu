@@ -70,6 +70,13 @@ struct d3_ctx {
   int last_rows = 0;
   int64_t launches = 0;
   int64_t dev_bytes = 0;
+  // per-class kernel timing (off by default)
+  bool prof_on = false;
+  struct ProfPair { cudaEvent_t a, b; int cls; };
+  std::vector<ProfPair> prof_pool;
+  size_t prof_used = 0;
+  double prof_ms[D3_PROF_CLASSES] = {};
+  int64_t prof_n[D3_PROF_CLASSES] = {};
   std::string last_error;
   std::vector<void*> allocs;
   std::map<std::tuple<const void*, int, int, int>, CUtensorMap> tmaps;
@@ -132,6 +139,42 @@ int check_launch(d3_ctx* c, const char* what) {
     if (rc_ != D3_OK) return rc_;  \
   } while (0)
 
+// ---- optional per-class timing: an event pair around every launch of the class
+void prof_flush(d3_ctx* c) {
+  if (c->prof_used == 0) return;
+  cudaStreamSynchronize(c->stream);
+  for (size_t i = 0; i < c->prof_used; ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_pool[i].a, c->prof_pool[i].b) == cudaSuccess) {
+      c->prof_ms[c->prof_pool[i].cls] += ms;
+      c->prof_n[c->prof_pool[i].cls] += 1;
+    }
+  }
+  c->prof_used = 0;
+}
+struct ProfScope {
+  d3_ctx* c;
+  long idx = -1;
+  ProfScope(d3_ctx* ctx, int cls) : c(ctx) {
+    if (!c->prof_on) return;
+    if (c->prof_used == c->prof_pool.size()) {
+      if (c->prof_pool.size() < 8192) {
+        d3_ctx::ProfPair pp{};
+        if (cudaEventCreate(&pp.a) != cudaSuccess || cudaEventCreate(&pp.b) != cudaSuccess) return;
+        c->prof_pool.push_back(pp);
+      } else {
+        prof_flush(c);
+      }
+    }
+    idx = static_cast<long>(c->prof_used++);
+    c->prof_pool[idx].cls = cls;
+    cudaEventRecord(c->prof_pool[idx].a, c->stream);
+  }
+  ~ProfScope() {
+    if (idx >= 0) cudaEventRecord(c->prof_pool[idx].b, c->stream);
+  }
+};
+
 // ---- tensor maps (driver entry point fetched through the runtime: no link against libcuda)
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -182,10 +225,10 @@ struct QkvExtra {
   void* v_cache;
 };
 
-template <int EPI>
+template <int EPI, int BLOCK_N>
 int launch_tc(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, dim3 grid,
               size_t smem) {
-  auto kern = tc::gemm_tc_kernel<EPI, 128>;
+  auto kern = tc::gemm_tc_kernel<EPI, BLOCK_N>;
   static bool attr_set = false;
   if (!attr_set) {
     CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
@@ -201,13 +244,15 @@ int pick_splits(const d3_ctx* c, int m_tiles, int n_tiles, int k_chunks, int epi
   int tiles = m_tiles * n_tiles;
   int s = hint;
   if (s <= 0) {
+    // split K only when even 32-wide column tiles leave most SMs idle
     s = 1;
-    const int target = 2 * c->n_sms;
-    if (tiles < target) s = (target + tiles - 1) / tiles;
-    int cap = k_chunks / 4;  // keep at least four 64-wide K slabs per split
-    if (cap < 1) cap = 1;
-    if (s > cap) s = cap;
-    if (s > 16) s = 16;
+    if (tiles * 2 <= c->n_sms) {
+      s = c->n_sms / tiles;
+      int cap = k_chunks / 8;  // keep at least eight 64-wide K slabs per split
+      if (cap < 1) cap = 1;
+      if (s > cap) s = cap;
+      if (s > 8) s = 8;
+    }
   }
   if (s > k_chunks) s = k_chunks;
   if (s < 1) s = 1;
@@ -216,9 +261,36 @@ int pick_splits(const d3_ctx* c, int m_tiles, int n_tiles, int k_chunks, int epi
   return s;
 }
 
+template <int BLOCK_N>
+int dispatch_tc(d3_ctx* c, int epi, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, dim3 grid,
+                size_t smem) {
+  switch (epi) {
+    case EPI_F32: return launch_tc<EPI_F32, BLOCK_N>(c, tx, tw, p, grid, smem);
+    case EPI_T: return launch_tc<EPI_T, BLOCK_N>(c, tx, tw, p, grid, smem);
+    case EPI_RESID: return launch_tc<EPI_RESID, BLOCK_N>(c, tx, tw, p, grid, smem);
+    case EPI_SWIGLU: return launch_tc<EPI_SWIGLU, BLOCK_N>(c, tx, tw, p, grid, smem);
+    case EPI_QKV: return launch_tc<EPI_QKV, BLOCK_N>(c, tx, tw, p, grid, smem);
+    case EPI_STATS:
+      if constexpr (BLOCK_N % 128 == 0) return launch_tc<EPI_STATS, BLOCK_N>(c, tx, tw, p, grid, smem);
+      break;
+  }
+  return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
+}
+
+// Column-tile width.  Skinny matmuls (one row tile) stream every weight byte exactly once, so the
+// tile is chosen to give about one CTA per SM or more with no split-K; wide row counts use 128.
+int pick_block_n(const d3_ctx* c, int M, int N, int epi) {
+  if (epi == EPI_STATS) return 128;
+  if (M > 128) return 128;
+  for (int bn : {128, 64, 32}) {
+    if ((N + bn - 1) / bn >= c->n_sms - 20) return bn;
+  }
+  return 32;
+}
+
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
                   int splits_hint, const QkvExtra* qx) {
-  const int BLOCK_N = 128;
+  const int BLOCK_N = pick_block_n(c, M, N, epi);
   const int m_tiles = (M + 127) / 128, n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_chunks = (K + 63) / 64;
   int a_rows = M >= 128 ? 128 : ((M + 31) / 32) * 32;
@@ -227,8 +299,10 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   p.a_rows = a_rows;
   p.splits = pick_splits(c, m_tiles, n_tiles, k_chunks, epi, splits_hint);
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + BLOCK_N * 128;
-  int stages = static_cast<int>((100 * 1024) / stage_bytes);
-  if (stages > 8) stages = 8;
+  // two CTAs per SM when there are more tiles than SMs, otherwise one CTA with a deeper pipeline
+  const bool two_per_sm = static_cast<long long>(m_tiles) * n_tiles * p.splits > c->n_sms;
+  int stages = static_cast<int>(((two_per_sm ? 100 : 190) * 1024) / stage_bytes);
+  if (stages > 24) stages = 24;
   if (stages < 2) stages = 2;
   p.stages = stages;
   p.partial = c->partial;
@@ -246,15 +320,11 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   TRY(get_tmap(c, W, N, K, BLOCK_N, &tw));
   dim3 grid(m_tiles, n_tiles, p.splits);
   size_t smem = tc::gemm_tc_smem_bytes(a_rows, BLOCK_N, stages);
-  switch (epi) {
-    case EPI_F32: return launch_tc<EPI_F32>(c, tx, tw, p, grid, smem);
-    case EPI_T: return launch_tc<EPI_T>(c, tx, tw, p, grid, smem);
-    case EPI_RESID: return launch_tc<EPI_RESID>(c, tx, tw, p, grid, smem);
-    case EPI_SWIGLU: return launch_tc<EPI_SWIGLU>(c, tx, tw, p, grid, smem);
-    case EPI_STATS: return launch_tc<EPI_STATS>(c, tx, tw, p, grid, smem);
-    case EPI_QKV: return launch_tc<EPI_QKV>(c, tx, tw, p, grid, smem);
+  switch (BLOCK_N) {
+    case 32: return dispatch_tc<32>(c, epi, tx, tw, p, grid, smem);
+    case 64: return dispatch_tc<64>(c, epi, tx, tw, p, grid, smem);
+    default: return dispatch_tc<128>(c, epi, tx, tw, p, grid, smem);
   }
-  return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
 template <typename T>
@@ -275,8 +345,9 @@ int run_linear_simt(d3_ctx* c, const void* X, const void* W, int M, int N, int K
 }
 
 int run_linear(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
-               int splits_hint = 0, const QkvExtra* qx = nullptr) {
+               int splits_hint = 0, const QkvExtra* qx = nullptr, int cls = D3_PROF_GEMM_OTHER) {
   if (M <= 0 || N <= 0 || K <= 0) return D3_OK;
+  ProfScope ps(c, cls);
   if (c->use_tc) return run_linear_tc(c, X, W, M, N, K, epi, ep, splits_hint, qx);
   if (c->is_bf16) return run_linear_simt<bf16>(c, X, W, M, N, K, epi, ep);
   return run_linear_simt<float>(c, X, W, M, N, K, epi, ep);
@@ -303,6 +374,7 @@ int launch_attention(d3_ctx* c, const void* q, const void* kc, const void* vc, v
 }
 
 int run_attention(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
+  ProfScope ps(c, D3_PROF_ATTENTION);
   const char* base = static_cast<const char*>(c->kv);
   const void* kc = base + (static_cast<size_t>(layer) * 2 + 0) * c->kv_layer_elems * c->esz;
   const void* vc = base + (static_cast<size_t>(layer) * 2 + 1) * c->kv_layer_elems * c->esz;
@@ -318,6 +390,7 @@ void* v_plane(d3_ctx* c, int layer) {
 }
 
 int run_rmsnorm(d3_ctx* c, const float* x, const float* gain, void* xn, int M) {
+  ProfScope ps(c, D3_PROF_RMSNORM);
   const int d = c->cfg.d_model;
   const int threads = d >= 1024 ? 256 : 128;
   if (c->is_bf16) rmsnorm_kernel<bf16><<<M, threads, 0, c->stream>>>(x, gain, static_cast<bf16*>(xn), d, c->cfg.rms_eps);
@@ -327,6 +400,7 @@ int run_rmsnorm(d3_ctx* c, const float* x, const float* gain, void* xn, int M) {
 }
 
 int run_stats_merge(d3_ctx* c, int M, int n_tiles, float* conf, float* ent, int* argmax) {
+  ProfScope ps(c, D3_PROF_OTHER);
   stats_merge_kernel<<<(M + 3) / 4, 128, 0, c->stream>>>(c->stat_part, n_tiles, M, conf, ent, argmax);
   LAUNCHED(c, "stats_merge_kernel");
   return D3_OK;
@@ -343,9 +417,12 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
   RowMap rm{c->pos_base, c->n_valid, c->kv_len, rows_per_seq, bs};
   c->last_rows = M;
 
-  if (c->is_bf16) embed_kernel<bf16><<<M, 128, 0, c->stream>>>(ids, static_cast<const bf16*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
-  else embed_kernel<float><<<M, 128, 0, c->stream>>>(ids, static_cast<const float*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
-  LAUNCHED(c, "embed_kernel");
+  {
+    ProfScope ps(c, D3_PROF_OTHER);
+    if (c->is_bf16) embed_kernel<bf16><<<M, 128, 0, c->stream>>>(ids, static_cast<const bf16*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
+    else embed_kernel<float><<<M, 128, 0, c->stream>>>(ids, static_cast<const float*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
+    LAUNCHED(c, "embed_kernel");
+  }
 
   for (int l = 0; l < g.n_layers; ++l) {
     if (l == c->tap_layer && M <= c->tap_rows)
@@ -355,11 +432,12 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
       EpiParams ep;
       ep.y = c->q; ep.ldy = nq;
       QkvExtra qx{rm, k_plane(c, l), v_plane(c, l)};
-      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_QKV, ep, 0, &qx));
+      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_QKV, ep, 0, &qx, D3_PROF_GEMM_QKV));
     } else {
       EpiParams ep;
       ep.y = c->qkv_f32; ep.ldy = nq + 2 * nkv;
-      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_F32, ep));
+      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_QKV));
+      ProfScope ps(c, D3_PROF_OTHER);
       if (c->is_bf16)
         rope_kv_kernel<bf16><<<M, 256, 0, c->stream>>>(c->qkv_f32, static_cast<bf16*>(c->q), static_cast<bf16*>(k_plane(c, l)), static_cast<bf16*>(v_plane(c, l)), c->rope_cos, c->rope_sin, rm, g.n_q_heads, g.n_kv_heads, g.d_head, g.max_seq, c->error_word);
       else
@@ -370,18 +448,18 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     {
       EpiParams ep;
       ep.y = c->x; ep.ldy = d;
-      TRY(run_linear(c, c->o, c->wo[l], M, d, nq, EPI_RESID, ep));
+      TRY(run_linear(c, c->o, c->wo[l], M, d, nq, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_O));
     }
     TRY(run_rmsnorm(c, c->x, c->ffn_norm[l], c->xn, M));
     {
       EpiParams ep;
       ep.y = c->h; ep.ldy = f;
-      TRY(run_linear(c, c->xn, c->wgu[l], M, 2 * f, d, EPI_SWIGLU, ep));
+      TRY(run_linear(c, c->xn, c->wgu[l], M, 2 * f, d, EPI_SWIGLU, ep, 0, nullptr, D3_PROF_GEMM_GATE_UP));
     }
     {
       EpiParams ep;
       ep.y = c->x; ep.ldy = d;
-      TRY(run_linear(c, c->h, c->wd[l], M, d, f, EPI_RESID, ep));
+      TRY(run_linear(c, c->h, c->wd[l], M, d, f, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_DOWN));
     }
     if (l == c->tap_layer && M <= c->tap_rows)
       CUDA_TRY(c, cudaMemcpyAsync(c->tap_out, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
@@ -392,12 +470,12 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     const int n_tiles = (g.vocab + 127) / 128;
     EpiParams ep;
     ep.scale = g.logit_scale; ep.mask_id = g.mask_id; ep.stat_part = c->stat_part; ep.n_tiles = n_tiles;
-    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_STATS, ep));
+    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_STATS, ep, 0, nullptr, D3_PROF_GEMM_HEAD));
     TRY(run_stats_merge(c, M, n_tiles, c->conf, c->ent, c->argmax));
   } else {
     EpiParams ep;
     ep.y = logits; ep.ldy = g.vocab; ep.scale = g.logit_scale;
-    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_F32, ep));
+    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_HEAD));
   }
   return D3_OK;
 }
@@ -527,6 +605,10 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
 extern "C" void d3_destroy(d3_ctx* c) {
   if (!c) return;
   cudaStreamSynchronize(c->stream);
+  for (auto& pp : c->prof_pool) {
+    cudaEventDestroy(pp.a);
+    cudaEventDestroy(pp.b);
+  }
   for (void* p : c->allocs) cudaFree(p);
   if (c->host_counters) cudaFreeHost(c->host_counters);
   delete c;
@@ -579,7 +661,7 @@ extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device
   }
   // staging for gate / up (interleaved on the device) and gains
   void *tg = nullptr, *tu = nullptr, *tgain = nullptr;
-  CUDA_TRY(c, cudaMalloc(&tg, f * d * e));
+  CUDA_TRY(c, cudaMalloc(&tg, std::max(f, nq) * d * e));
   CUDA_TRY(c, cudaMalloc(&tu, f * d * e));
   CUDA_TRY(c, cudaMalloc(&tgain, d * e));
   int rc = D3_OK;
@@ -589,8 +671,18 @@ extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device
   step(load_gain(c, &c->final_norm, w->final_norm, src_is_device, tgain));
   for (int l = 0; l < g.n_layers && rc == D3_OK; ++l) {
     char* qkv = static_cast<char*>(c->wqkv[l]);
-    step(upload(c, qkv, w->wq[l], nq * d * e, src_is_device));
-    step(upload(c, qkv + nq * d * e, w->wk[l], nkv * d * e, src_is_device));
+    // q and k rows go through the staging buffer and are packed as RoPE pairs
+    for (int which = 0; which < 2 && rc == D3_OK; ++which) {
+      const size_t rows = which == 0 ? nq : nkv;
+      char* dst = qkv + (which == 0 ? 0 : nq * d * e);
+      step(upload(c, tg, which == 0 ? w->wq[l] : w->wk[l], rows * d * e, src_is_device));
+      if (rc != D3_OK) break;
+      if (c->is_bf16)
+        pack_rope_rows_kernel<bf16><<<static_cast<unsigned>(rows), 128, 0, c->stream>>>(static_cast<const bf16*>(tg), reinterpret_cast<bf16*>(dst), g.d_head, g.d_model);
+      else
+        pack_rope_rows_kernel<float><<<static_cast<unsigned>(rows), 128, 0, c->stream>>>(static_cast<const float*>(tg), reinterpret_cast<float*>(dst), g.d_head, g.d_model);
+      step(check_launch(c, "pack_rope_rows_kernel"));
+    }
     step(upload(c, qkv + (nq + nkv) * d * e, w->wv[l], nkv * d * e, src_is_device));
     step(upload(c, c->wo[l], w->wo[l], d * nq * e, src_is_device));
     step(upload(c, c->wd[l], w->w_down[l], d * f * e, src_is_device));
@@ -779,7 +871,7 @@ extern "C" int d3_op_linear(d3_ctx* c, const void* x, const void* w, void* y, in
   if (!c) return D3_ERR_INVALID_ARG;
   if (!x || !w || !y || m <= 0 || n <= 0 || k <= 0 || epilogue < 0 || epilogue > 3)
     return fail(c, D3_ERR_INVALID_ARG, "bad op_linear arguments");
-  if (epilogue == EPI_SWIGLU && n % 128 != 0) return fail(c, D3_ERR_SHAPE, "SwiGLU epilogue needs n % 128 == 0");
+  if (epilogue == EPI_SWIGLU && n % 2 != 0) return fail(c, D3_ERR_SHAPE, "SwiGLU epilogue needs an even n");
   EpiParams ep;
   ep.y = y;
   ep.ldy = epilogue == EPI_SWIGLU ? n / 2 : n;
@@ -849,6 +941,27 @@ extern "C" int d3_get_error_word(d3_ctx* c, uint32_t* word) {
   if (!c || !word) return D3_ERR_INVALID_ARG;
   CUDA_TRY(c, cudaMemcpyAsync(word, c->error_word, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return D3_OK;
+}
+extern "C" int d3_profile_enable(d3_ctx* c, int on) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  prof_flush(c);
+  if (on) {
+    for (int i = 0; i < D3_PROF_CLASSES; ++i) {
+      c->prof_ms[i] = 0.0;
+      c->prof_n[i] = 0;
+    }
+  }
+  c->prof_on = on != 0;
+  return D3_OK;
+}
+extern "C" int d3_profile_read(d3_ctx* c, double* ms, int64_t* launches) {
+  if (!c || !ms || !launches) return D3_ERR_INVALID_ARG;
+  prof_flush(c);
+  for (int i = 0; i < D3_PROF_CLASSES; ++i) {
+    ms[i] = c->prof_ms[i];
+    launches[i] = c->prof_n[i];
+  }
   return D3_OK;
 }
 extern "C" int64_t d3_launch_count(d3_ctx* c) { return c ? c->launches : 0; }

@@ -67,14 +67,14 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const T* __restrict_
       }
     }
   } else if constexpr (EPI == EPI_SWIGLU) {
-    // tile = one group: 64 gate columns then 64 up columns of hidden units [n0/2, n0/2 + 64)
+    // packed rows of W: 2j = gate row of hidden unit j, 2j+1 = its up row
     const int F = N / 2;
     for (int e = t; e < BM * 64; e += THREADS) {
       int r = e / 64, c = e % 64;
       int m = m0 + r, h = n0 / 2 + c;
       if (m < M && h < F)
         static_cast<T*>(ep.y)[static_cast<size_t>(m) * ep.ldy + h] =
-            TypeOps<T>::from_f(silu_f(Cs[r][c]) * Cs[r][c + 64]);
+            TypeOps<T>::from_f(silu_f(Cs[r][2 * c]) * Cs[r][2 * c + 1]);
     }
   } else if constexpr (EPI == EPI_STATS) {
     // one warp per row (8 warps, 4 rows each): lanes stride the 128 columns, fixed shuffle tree

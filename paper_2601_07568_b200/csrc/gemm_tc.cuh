@@ -265,39 +265,34 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       }
     }
   } else if constexpr (EPI == EPI_SWIGLU) {
-    // columns [g*128, g*128+64) are gate rows of hidden units [g*64, g*64+64), the next 64 the up rows
+    // packed rows of W: 2j = gate row of hidden unit j, 2j+1 = its up row; a 32-column chunk gives 16 outputs
     __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
-    for (int g = 0; g < BLOCK_N; g += 128) {
-      if (n0 + g >= N) break;
-      for (int c = 0; c < 64; c += 32) {
-        float gate[32], up[32];
-        src.load(g + c, gate);
-        src.load(g + c + 64, up);
-        const int h0 = (n0 + g) / 2 + c;
-        const int F = N / 2;
-        if (!live) continue;
-        if (h0 + 32 <= F && (p.ep.ldy & 7) == 0) {
-          uint4* y4 = reinterpret_cast<uint4*>(y + h0);
+    const int F = N / 2;
+    for (int c = 0; c < BLOCK_N; c += 32) {
+      if (n0 + c >= N) break;
+      float v[32];
+      src.load(c, v);
+      if (!live) continue;
+      const int h0 = (n0 + c) / 2;
+      if (h0 + 16 <= F && (p.ep.ldy & 7) == 0) {
+        uint32_t w[8];
 #pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            uint32_t w[4];
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              __nv_bfloat162 t = __floats2bfloat162_rn(silu_f(gate[8 * j + 2 * q]) * up[8 * j + 2 * q],
-                                                       silu_f(gate[8 * j + 2 * q + 1]) * up[8 * j + 2 * q + 1]);
-              w[q] = *reinterpret_cast<uint32_t*>(&t);
-            }
-            y4[j] = make_uint4(w[0], w[1], w[2], w[3]);
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (h0 + j < F) y[h0 + j] = __float2bfloat16_rn(silu_f(gate[j]) * up[j]);
+        for (int q = 0; q < 8; ++q) {
+          __nv_bfloat162 t = __floats2bfloat162_rn(silu_f(v[4 * q]) * v[4 * q + 1], silu_f(v[4 * q + 2]) * v[4 * q + 3]);
+          w[q] = *reinterpret_cast<uint32_t*>(&t);
         }
+        uint4* y4 = reinterpret_cast<uint4*>(y + h0);
+        y4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+        y4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (h0 + j < F) y[h0 + j] = __float2bfloat16_rn(silu_f(v[2 * j]) * v[2 * j + 1]);
       }
     }
   } else if constexpr (EPI == EPI_STATS) {
     // one partial per 128-column tile so that the merge kernel sees the same tiling for any BLOCK_N
+    static_assert(BLOCK_N % 128 == 0, "statistics epilogue works on 128-column tiles");
     for (int g = 0; g < BLOCK_N; g += 128) {
       SoftStat st = stat_empty();
       for (int c = 0; c < 128; c += 32) {
@@ -315,7 +310,8 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
         p.ep.stat_part[static_cast<size_t>(m) * p.ep.n_tiles + t] = make_float4(st.m, st.z, st.s, __int_as_float(st.a));
     }
   } else if constexpr (EPI == EPI_QKV) {
-    // one 128-column group = one head (d_head = 128): q heads, then k heads, then v heads
+    // d_head = 128.  Packed rows of W inside a q or k head: 2i = dim i, 2i+1 = dim i+64 (a RoPE pair);
+    // v heads keep their order.  q heads first, then k heads, then v heads.
     int pos = 0, b = 0;
     if (live) {
       b = m / p.rows_per_seq;
@@ -328,52 +324,58 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       }
       if (!live) pos = 0;
     }
-    for (int g = 0; g < BLOCK_N; g += 128) {
-      const int head = (n0 + g) / 128;
-      if (head >= p.n_q_heads + 2 * p.n_kv_heads) break;
-      __nv_bfloat16* dst;
-      bool rotate = true;
-      if (head < p.n_q_heads) {
-        dst = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy + head * 128;
-      } else if (head < p.n_q_heads + p.n_kv_heads) {
-        int kh = head - p.n_q_heads;
-        dst = p.k_cache + ((static_cast<size_t>(b) * p.n_kv_heads + kh) * p.max_seq + pos) * 128;
-      } else {
-        int vh = head - p.n_q_heads - p.n_kv_heads;
-        dst = p.v_cache + ((static_cast<size_t>(b) * p.n_kv_heads + vh) * p.max_seq + pos) * 128;
-        rotate = false;
-      }
-      const float* cs = p.rope_cos + static_cast<size_t>(pos) * 64;
-      const float* sn = p.rope_sin + static_cast<size_t>(pos) * 64;
-      for (int c = 0; c < 64; c += 32) {
-        float lo[32], hi[32];
-        src.load(g + c, lo);
-        src.load(g + c + 64, hi);
-        if (!live) continue;
-        if (rotate) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            float co = cs[c + j], si = sn[c + j];
-            float a = lo[j], bb = hi[j];
-            lo[j] = a * co - bb * si;
-            hi[j] = bb * co + a * si;
-          }
+    const float* cs = p.rope_cos + static_cast<size_t>(pos) * 64;
+    const float* sn = p.rope_sin + static_cast<size_t>(pos) * 64;
+    for (int c = 0; c < BLOCK_N; c += 32) {
+      const int n = n0 + c;
+      if (n >= N) break;
+      float v[32];
+      src.load(c, v);
+      if (!live) continue;
+      const int head = n / 128, off = n % 128;
+      if (head < p.n_q_heads + p.n_kv_heads) {
+        __nv_bfloat16* dst;
+        if (head < p.n_q_heads) {
+          dst = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy + head * 128;
+        } else {
+          dst = p.k_cache + ((static_cast<size_t>(b) * p.n_kv_heads + (head - p.n_q_heads)) * p.max_seq + pos) * 128;
         }
-        uint4* d_lo = reinterpret_cast<uint4*>(dst + c);
-        uint4* d_hi = reinterpret_cast<uint4*>(dst + c + 64);
+        const int i0 = off / 2;  // pair index of column 0 of this chunk: 16 pairs, dims i0.. and 64+i0..
+        uint32_t lo[8], hi[8];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          uint32_t w[4], x[4];
+        for (int q = 0; q < 8; ++q) {
+          float l2[2], h2[2];
 #pragma unroll
-          for (int q = 0; q < 4; ++q) {
-            __nv_bfloat162 t = __floats2bfloat162_rn(lo[8 * j + 2 * q], lo[8 * j + 2 * q + 1]);
-            __nv_bfloat162 u = __floats2bfloat162_rn(hi[8 * j + 2 * q], hi[8 * j + 2 * q + 1]);
-            w[q] = *reinterpret_cast<uint32_t*>(&t);
-            x[q] = *reinterpret_cast<uint32_t*>(&u);
+          for (int e = 0; e < 2; ++e) {
+            const int j = 2 * q + e;
+            const float co = cs[i0 + j], si = sn[i0 + j];
+            const float a = v[2 * j], bb = v[2 * j + 1];
+            l2[e] = a * co - bb * si;
+            h2[e] = bb * co + a * si;
           }
-          d_lo[j] = make_uint4(w[0], w[1], w[2], w[3]);
-          d_hi[j] = make_uint4(x[0], x[1], x[2], x[3]);
+          __nv_bfloat162 tl = __floats2bfloat162_rn(l2[0], l2[1]);
+          __nv_bfloat162 th = __floats2bfloat162_rn(h2[0], h2[1]);
+          lo[q] = *reinterpret_cast<uint32_t*>(&tl);
+          hi[q] = *reinterpret_cast<uint32_t*>(&th);
         }
+        uint4* d_lo = reinterpret_cast<uint4*>(dst + i0);
+        uint4* d_hi = reinterpret_cast<uint4*>(dst + 64 + i0);
+        d_lo[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        d_lo[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+        d_hi[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        d_hi[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
+      } else if (head < p.n_q_heads + 2 * p.n_kv_heads) {
+        __nv_bfloat16* dst = p.v_cache +
+            ((static_cast<size_t>(b) * p.n_kv_heads + (head - p.n_q_heads - p.n_kv_heads)) * p.max_seq + pos) * 128 + off;
+        uint32_t w[16];
+#pragma unroll
+        for (int q = 0; q < 16; ++q) {
+          __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
+          w[q] = *reinterpret_cast<uint32_t*>(&t);
+        }
+        uint4* d4 = reinterpret_cast<uint4*>(dst);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) d4[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
       }
     }
   }
@@ -522,9 +524,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 }
 
 inline size_t gemm_tc_smem_bytes(int a_rows, int block_n, int stages) {
-  return 1024 + static_cast<size_t>(stages) * (a_rows * 128 + block_n * 128) + (2 * stages + 1) * 8 + 64 +
-         // slack so that the MMA's 128-row read of the last X stage stays inside the allocation
-         (a_rows < 128 ? 0 : 0);
+  // The MMA reads 128 rows of the X operand whatever a_rows is: the last X stage must be followed by
+  // at least (128 - a_rows) * 128 bytes of allocated shared memory (the W stages, plus padding).
+  size_t body = static_cast<size_t>(stages) * (a_rows * 128 + block_n * 128);
+  size_t need = static_cast<size_t>(stages) * a_rows * 128 + static_cast<size_t>(128 - a_rows) * 128 + 128 * 128;
+  if (body < need) body = need;
+  return 1024 + body + (2 * stages + 1) * 8 + 64;
 }
 
 }  // namespace tc

@@ -65,8 +65,10 @@ __global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restr
 }
 
 // ----------------------------------------------------------------------------- RoPE + cache write
-// qkv: fp32 [M, (hq + 2 hkv) * dh] straight from the projection.  q heads are rotated and stored as
-// T [M, hq*dh]; k heads are rotated and stored in the cache, v heads stored as they are.
+// qkv: fp32 [M, (hq + 2 hkv) * dh] straight from the projection, whose q and k rows are packed so
+// that columns (2k, 2k+1) of a head hold dims (k, k + dh/2).  q heads are rotated and stored as
+// T [M, hq*dh] in natural dim order; k heads are rotated and stored in the cache, v heads stored as
+// they are.
 template <typename T>
 __global__ void rope_kv_kernel(const float* __restrict__ qkv, T* __restrict__ q_out, T* __restrict__ k_cache,
                                T* __restrict__ v_cache, const float* __restrict__ rope_cos,
@@ -89,7 +91,7 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, T* __restrict__ q_
   const int n_pairs = (hq + hkv) * half;
   for (int i = threadIdx.x; i < n_pairs; i += blockDim.x) {
     const int head = i / half, k = i % half;
-    const float a = row[head * dh + k], bb = row[head * dh + k + half];
+    const float a = row[head * dh + 2 * k], bb = row[head * dh + 2 * k + 1];
     const float lo = a * cs[k] - bb * sn[k];
     const float hi = bb * cs[k] + a * sn[k];
     if (head < hq) {
@@ -371,19 +373,23 @@ __global__ void copy_rows_kernel(const T* __restrict__ src, T* __restrict__ dst,
   size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = src[i];
 }
-// dst [2f, d]: group g of 128 rows = gate rows [64g, 64g+64) then up rows [64g, 64g+64).
+// dst [2f, d]: row 2j = gate row j, row 2j+1 = up row j.
 template <typename T>
 __global__ void interleave_gate_up_kernel(const T* __restrict__ gate, const T* __restrict__ up, T* __restrict__ dst,
                                           int f, int d) {
   const int row = blockIdx.x;  // 0 .. 2f-1 in dst
-  const int g = row / 128, w = row % 128;
-  const int h = g * 64 + (w % 64);
-  if (h >= f) {  // padding rows of a ragged last group
-    for (int i = threadIdx.x; i < d; i += blockDim.x) dst[static_cast<size_t>(row) * d + i] = TypeOps<T>::from_f(0.f);
-    return;
-  }
-  const T* src = (w < 64 ? gate : up) + static_cast<size_t>(h) * d;
+  const T* src = ((row & 1) ? up : gate) + static_cast<size_t>(row >> 1) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[static_cast<size_t>(row) * d + i] = src[i];
+}
+// RoPE-pair packing of q / k projection rows: inside each head, dst row 2i = src row i and dst row
+// 2i+1 = src row i + dh/2.
+template <typename T>
+__global__ void pack_rope_rows_kernel(const T* __restrict__ src, T* __restrict__ dst, int dh, int d) {
+  const int row = blockIdx.x;  // dst row
+  const int head = row / dh, w = row % dh;
+  const int s = head * dh + (w >> 1) + (w & 1) * (dh / 2);
+  for (int i = threadIdx.x; i < d; i += blockDim.x)
+    dst[static_cast<size_t>(row) * d + i] = src[static_cast<size_t>(s) * d + i];
 }
 
 }  // namespace d3
