@@ -284,6 +284,14 @@ def d3_version() -> str:
     return lib().d3_version().decode()
 
 
+def d3_strerror(code: int) -> str:
+    return lib().d3_strerror(C.c_int(code)).decode()
+
+
+def d3_last_error(ctx) -> str:
+    return lib().d3_last_error(ctx).decode()
+
+
 # ----------------------------------------------------------------------------- convenience
 def make_config(shape, *, block: int, max_batch: int, max_seq: int, max_prefill_rows: int = 0,
                 decide_mode: int = D3_DECIDE_CONFIDENCE, gemm_impl: int = D3_GEMM_AUTO) -> d3_config:

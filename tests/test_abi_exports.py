@@ -1,0 +1,47 @@
+"""The C-ABI library builds without a GPU, loads, and exports every function include/d3.h declares.
+No compute call is made here."""
+import ctypes
+import os
+import re
+
+from paper_2601_07568_b200 import binding
+from paper_2601_07568_b200 import build as d3build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    src = open(os.path.join(ROOT, "include", "d3.h")).read()
+    src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
+    return sorted(set(re.findall(r"\b(d3_[a-z0-9_]+)\s*\(", src)))
+
+
+def test_header_functions_are_exported_and_bound():
+    lib_path = d3build.build()
+    L = ctypes.CDLL(lib_path)
+    names = declared_functions()
+    assert len(names) >= 20
+    missing = [n for n in names if not hasattr(L, n)]
+    assert not missing, missing
+    assert sorted(binding.EXPORTS) == names
+    unbound = [n for n in names if not hasattr(binding, n)]
+    assert not unbound, unbound
+
+
+def test_host_only_entry_points():
+    L = binding.lib()
+    assert binding.d3_version().startswith("d3-b200")
+    assert L.d3_strerror(0) == b"ok"
+    assert L.d3_strerror(binding.D3_ERR_DEVICE_TIMEOUT) == b"bounded device-side wait gave up"
+    assert L.d3_strerror(-99) == b"unknown error"
+    # null arguments are rejected before any CUDA call
+    assert L.d3_create(None, None, None) == binding.D3_ERR_INVALID_ARG
+    assert L.d3_prefill(None, None, None, 1, 1) == binding.D3_ERR_INVALID_ARG
+    assert L.d3_generate(None, 32, ctypes.c_float(0.9), 1, None, None, None) == binding.D3_ERR_INVALID_ARG
+
+
+def test_struct_layouts_match_header():
+    # 8 int32 + 3 float + 7 int32 = 18 four-byte fields; 12 pointers; 6 int64 + 2 float
+    assert ctypes.sizeof(binding.d3_config) == 18 * 4
+    assert ctypes.sizeof(binding.d3_weights) == 12 * ctypes.sizeof(ctypes.c_void_p)
+    assert ctypes.sizeof(binding.d3_stats) == 6 * 8 + 2 * 4
