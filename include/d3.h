@@ -183,6 +183,43 @@ int d3_op_unmask(d3_ctx *ctx, const float *conf, const float *entropy, const int
                  int32_t *block_ids, uint8_t *mask, float threshold, int32_t bs, int32_t *out_pos,
                  int32_t *out_ids, int32_t *out_count);
 
+/* LM-head statistics without any allocation.  (The paper has no counterpart: this entry point exists
+ * for the sake of callers, not of the method.)
+ *
+ * Some callers of this library may not create device memory at the moment they need the
+ * statistics: code running between the begin and end of a region in which the allocator is frozen,
+ * a plug-in that was handed a fixed memory budget by its host process, or a real-time loop in which
+ * a cudaMalloc (which may synchronise the device) is not acceptable.  Those callers cannot use
+ * d3_create(), which allocates the cache and the workspaces.  This function needs no context: it
+ * computes, for every row of x, the same three numbers as d3_op_lm_head_stats -- confidence = largest
+ * softmax probability of scale * (x . w^T) with column mask_id left out, entropy in nats, and the
+ * arg max (lowest index on ties) -- and keeps its only intermediate, one partial statistic per
+ * (row, 128-column tile of the vocabulary), in an array that is part of the loaded library image.
+ *
+ *   x [device][m, k], w [device][vocab, k], both of `dtype` (D3_DTYPE_*), row-major;
+ *   conf, entropy [device][m] float, argmax [device][m] int32: written by the call;
+ *   cuda_stream: a cudaStream_t (NULL = default stream) of the current device; work is enqueued
+ *   there and the call returns without waiting.
+ *
+ * Limits and rules
+ *   - m * ceil(vocab / 128) must not exceed D3_STATIC_MAX_PARTIALS (65536 entries, 1 MiB, held by
+ *     every GPU that loads the library until the process exits); larger problems return
+ *     D3_ERR_SHAPE and nothing is launched.
+ *   - The function calls no cudaMalloc / cudaFree and no library routine that allocates.  The first
+ *     call on each device looks up the device address of the array (a symbol query, with that
+ *     device current); make that first call outside any stream capture.
+ *   - All calls on one device share the array.  Two calls whose kernels may overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them on one stream or with
+ *     events.  The array keeps what the previous call left; every entry that a call reads it has
+ *     written itself first, so nothing needs clearing between calls.
+ *   - The matmul inside runs on the plain SIMT kernel of this library for both element types (it is
+ *     meant for operator-sized problems, not for streaming a full vocabulary at speed).
+ * Errors: INVALID_ARG (null pointer, non-positive size, unknown dtype), SHAPE, CUDA. */
+#define D3_STATIC_MAX_PARTIALS 65536
+int d3_lm_head_stats_static(const void *x, const void *w, int32_t dtype, int32_t m, int32_t vocab, int32_t k,
+                            float scale, int32_t mask_id, float *conf, float *entropy, int32_t *argmax,
+                            void *cuda_stream);
+
 /* Per-class kernel timing for measurement runs.  While enabled, every launch of the forward pass is
  * bracketed by a CUDA event pair on the context's stream; d3_profile_read waits for the stream and
  * returns, per class, the summed elapsed milliseconds and the number of launches since enabling.

@@ -27,7 +27,7 @@ EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
     "d3_get_state", "d3_set_state", "d3_op_linear", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
+    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
 
@@ -248,6 +248,30 @@ def d3_op_unmask(ctx, conf: torch.Tensor, entropy: torch.Tensor, argmax: torch.T
                                    _ptr(_dev(mask, torch.uint8)), C.c_float(threshold),
                                    C.c_int32(block_ids.shape[0]), _ptr(_dev(out_pos, torch.int32)),
                                    _ptr(_dev(out_ids, torch.int32)), _ptr(_dev(out_count, torch.int32))))
+
+
+D3_STATIC_MAX_PARTIALS = 65536
+
+
+def d3_lm_head_stats_static(x: torch.Tensor, w: torch.Tensor, scale: float, mask_id: int, conf: torch.Tensor,
+                            entropy: torch.Tensor, argmax: torch.Tensor,
+                            stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Context-free LM-head statistics that allocate nothing on the device (for callers that may not
+    allocate: frozen-allocator regions, fixed memory budgets, real-time loops).  x [m, k] and w [vocab, k]
+    are float32 or bfloat16 CUDA tensors of the same type; the outputs are written on ``stream`` (default:
+    torch's current stream).  Raises D3Error(D3_ERR_SHAPE) when m * ceil(vocab/128) exceeds
+    D3_STATIC_MAX_PARTIALS.  Calls that may overlap on the GPU race on the shared scratch array."""
+    _dev(x), _dev(w, x.dtype)
+    if x.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("x and w must be float32 or bfloat16")
+    m, k = x.shape
+    s = C.c_void_p(stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream)
+    rc = lib().d3_lm_head_stats_static(_ptr(x), _ptr(w), C.c_int32(D3_DTYPE_BF16 if x.dtype == torch.bfloat16 else D3_DTYPE_F32),
+                                       C.c_int32(m), C.c_int32(w.shape[0]), C.c_int32(k), C.c_float(scale),
+                                       C.c_int32(mask_id), _ptr(_dev(conf, torch.float32)),
+                                       _ptr(_dev(entropy, torch.float32)), _ptr(_dev(argmax, torch.int32)), s)
+    if rc != D3_OK:
+        raise D3Error(rc, lib().d3_strerror(rc).decode())
 
 
 PROF_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_head", "gemm_other", "attention",

@@ -982,3 +982,69 @@ extern "C" const char* d3_strerror(int code) {
 }
 extern "C" const char* d3_last_error(d3_ctx* c) { return c ? c->last_error.c_str() : ""; }
 extern "C" const char* d3_version(void) { return kVersion; }
+
+// ----------------------------------------------------------------------------- allocation-free variant
+// LM-head statistics for callers that must not allocate device memory (see include/d3.h).  The
+// per-tile partial statistics, which the context-based entry point keeps in a buffer from cudaMalloc,
+// live here in a fixed array inside the loaded module.
+static __device__ __align__(256) float4 g_static_stat_part[D3_STATIC_MAX_PARTIALS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+float4* g_static_stat_ptr[kMaxDevices] = {};  // device address of the array, per device ordinal
+
+// `g_static_stat_part` names a host-side handle in host code, not a device address: resolve it once
+// per device, with that device current, and cache the result.
+int static_scratch(float4** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return D3_ERR_CUDA;
+  if (!g_static_stat_ptr[dev]) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_stat_part) != cudaSuccess || !p) {
+      (void)cudaGetLastError();
+      return D3_ERR_CUDA;
+    }
+    g_static_stat_ptr[dev] = static_cast<float4*>(p);
+  }
+  *out = g_static_stat_ptr[dev];
+  return D3_OK;
+}
+
+template <typename T>
+int lm_head_stats_static(const void* x, const void* w, int m, int vocab, int k, float scale, int mask_id, float* conf,
+                         float* entropy, int* argmax, float4* part, cudaStream_t stream) {
+  const int n_tiles = (vocab + simt::BN - 1) / simt::BN;
+  EpiParams ep;
+  ep.scale = scale; ep.mask_id = mask_id; ep.stat_part = part; ep.n_tiles = n_tiles;
+  dim3 grid(n_tiles, (m + simt::BM - 1) / simt::BM);
+  simt::gemm_simt_kernel<T, EPI_STATS><<<grid, simt::THREADS, 0, stream>>>(static_cast<const T*>(x), static_cast<const T*>(w), m, vocab, k, ep);
+  if (cudaPeekAtLastError() != cudaSuccess) {
+    (void)cudaGetLastError();
+    return D3_ERR_CUDA;
+  }
+  stats_merge_kernel<<<(m + 3) / 4, 128, 0, stream>>>(part, n_tiles, m, conf, entropy, argmax);
+  if (cudaPeekAtLastError() != cudaSuccess) {
+    (void)cudaGetLastError();
+    return D3_ERR_CUDA;
+  }
+  return D3_OK;
+}
+}  // namespace
+
+extern "C" int d3_lm_head_stats_static(const void* x, const void* w, int32_t dtype, int32_t m, int32_t vocab, int32_t k,
+                                       float scale, int32_t mask_id, float* conf, float* entropy, int32_t* argmax,
+                                       void* cuda_stream) {
+  if (!x || !w || !conf || !entropy || !argmax || m <= 0 || vocab <= 0 || k <= 0) return D3_ERR_INVALID_ARG;
+  if (dtype != D3_DTYPE_F32 && dtype != D3_DTYPE_BF16) return D3_ERR_INVALID_ARG;
+  const long long n_tiles = (static_cast<long long>(vocab) + simt::BN - 1) / simt::BN;
+  if (static_cast<long long>(m) * n_tiles > D3_STATIC_MAX_PARTIALS) return D3_ERR_SHAPE;
+  float4* part = nullptr;
+  int rc = static_scratch(&part);
+  if (rc != D3_OK) return rc;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  // Every partial that the merge reads is written by the matmul launch before it, so nothing in
+  // the shared array has to start at zero and stale contents of earlier calls are never read.
+  if (dtype == D3_DTYPE_BF16)
+    return lm_head_stats_static<bf16>(x, w, m, vocab, k, scale, mask_id, conf, entropy, argmax, part, stream);
+  return lm_head_stats_static<float>(x, w, m, vocab, k, scale, mask_id, conf, entropy, argmax, part, stream);
+}
