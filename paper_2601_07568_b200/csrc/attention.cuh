@@ -93,3 +93,320 @@ __global__ void __launch_bounds__(THREADS) attn_simt_kernel(const T* __restrict_
 
 }  // namespace attn
 }  // namespace d3
+
+// ----------------------------------------------------------------------------- tensor-core kernel
+// bf16, d_head = 128.  The work is bound by reading K and V once from HBM (at 32 query rows per
+// kv head the arithmetic intensity is 32 flop/byte), so the design goal is bytes in flight, not
+// tensor throughput: K/V tiles of 64 keys are staged by TMA (128-byte swizzle) in a 3-deep ring,
+// the two small products per tile run on mma.sync m16n8k16 with fragments read by ldmatrix, and the
+// softmax stays in registers.  One CTA = one (sequence, kv head, query tile, key split); a query
+// tile packs the rows of all query heads that share the kv head (GQA): packed row pr = head_in_group
+// * rows_per_seq + r.  With several key splits every CTA writes an unnormalised partial (O, m, l)
+// and the last one to arrive (atomic counter, nobody waits) merges them in split order.
+#include "ptx_sm100.cuh"
+
+namespace d3 {
+namespace attn {
+
+constexpr int KT = 64;        // keys per tile
+constexpr int TC_STAGES = 3;  // ring depth: 3 x 32 KB
+constexpr int PART_LD = 132;  // floats per partial row: 128 outputs, m, l, 2 pad
+constexpr uint32_t STAGE_BYTES = 4u * KT * 128u;  // K lo, K hi, V lo, V hi slabs of [KT][64] bf16
+
+struct AttnTcParams {
+  const __nv_bfloat16* q;  // [bs * rows_per_seq, hq * 128]
+  __nv_bfloat16* out;      // same shape
+  RowMap rm;
+  int hq, hkv, max_seq;
+  long long k_row0, v_row0;  // first row of this layer's K / V plane in the cache tensor map
+  int n_splits;
+  float scale_log2;  // 1/sqrt(d_head) * log2(e)
+  float* partial;    // [(pair * q_tiles + qt) * n_splits + split][BM][PART_LD]
+  int* counters;     // [(pair * q_tiles + qt)], zero on entry and on exit
+  uint32_t* error_word;
+};
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+  __nv_bfloat162 t = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&t);
+}
+// Byte offset of 16-byte chunk `c` (0..7) of row `r` inside a [rows][64] bf16 slab written by TMA
+// with the 128-byte swizzle (slab base 1024-byte aligned).
+__device__ __forceinline__ uint32_t swz(int r, int c) { return static_cast<uint32_t>(r * 128 + ((c ^ (r & 7)) << 4)); }
+
+// grid (q_tiles, bs * hkv, n_splits); NW warps of 16 packed rows each.
+template <int NW>
+__global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_kv,
+                                                          const AttnTcParams p) {
+  constexpr int BM = NW * 16;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + TC_STAGES * STAGE_BYTES);
+  uint64_t* empty_bar = full_bar + TC_STAGES;
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + TC_STAGES);
+  int* last_flag = const_cast<int*>(abort_flag) + 1;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g4 = lane >> 2, t4 = lane & 3;
+  const int qt = blockIdx.x, pair = blockIdx.y, split = blockIdx.z;
+  const int b = pair / p.hkv, g = pair % p.hkv;
+  const int group = p.hq / p.hkv;
+  const int rps = p.rm.rows_per_seq;
+
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmap_kv);
+    for (int s = 0; s < TC_STAGES; ++s) {
+      ptx::mbar_init(&full_bar[s], 1);
+      ptx::mbar_init(&empty_bar[s], NW);
+    }
+    *abort_flag = 0;
+    *last_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  __syncthreads();
+  ptx::grid_dep_wait();  // everything below reads what earlier kernels of the stream wrote
+  ptx::grid_dep_launch();
+
+  const int n_valid = p.rm.n_valid[b];
+  const int kv_len = p.rm.kv_len[b];
+  const int R = group * rps;
+  // rows of this tile that exist at all (uniform over the CTA)
+  if (qt * BM >= R || n_valid <= 0 || kv_len <= 0) return;
+  // a tile whose rows are all beyond n_valid has nothing to do (rows of one head are contiguous)
+  {
+    bool any = false;
+    for (int pr = qt * BM; pr < min(R, (qt + 1) * BM) && !any; pr += 1) any = (pr % rps) < n_valid;
+    if (!any) return;
+  }
+  const int n_tiles = (kv_len + KT - 1) / KT;
+  const int tps = (n_tiles + p.n_splits - 1) / p.n_splits;
+  const int t0 = split * tps, t1 = min(n_tiles, t0 + tps);
+  const int n_my = max(t1 - t0, 0);
+
+  const long long krow = p.k_row0 + (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
+  const long long vrow = p.v_row0 + (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
+  auto issue = [&](int i) {  // tile t0 + i into stage i % TC_STAGES
+    const int s = i % TC_STAGES;
+    uint8_t* st = smem + s * STAGE_BYTES;
+    const int j0 = (t0 + i) * KT;
+    ptx::mbar_arrive_expect_tx(&full_bar[s], STAGE_BYTES);
+    ptx::tma_load_2d(st, &tmap_kv, &full_bar[s], 0, static_cast<int>(krow + j0));
+    ptx::tma_load_2d(st + KT * 128, &tmap_kv, &full_bar[s], 64, static_cast<int>(krow + j0));
+    ptx::tma_load_2d(st + 2 * KT * 128, &tmap_kv, &full_bar[s], 0, static_cast<int>(vrow + j0));
+    ptx::tma_load_2d(st + 3 * KT * 128, &tmap_kv, &full_bar[s], 64, static_cast<int>(vrow + j0));
+  };
+  if (threadIdx.x == 0)
+    for (int i = 0; i < min(n_my, TC_STAGES); ++i) issue(i);
+
+  // ---- Q fragments of this warp's 16 packed rows (rows g4 and g4 + 8), straight from global memory
+  const int pr_lo = qt * BM + warp * 16 + g4, pr_hi = pr_lo + 8;
+  auto row_ptr = [&](int pr, bool& ok) -> const __nv_bfloat16* {
+    const int hg = pr / rps, r = pr % rps;
+    ok = pr < R && r < n_valid;
+    return p.q + (static_cast<size_t>(b) * rps + r) * p.hq * 128 + (g * group + hg) * 128;
+  };
+  bool ok_lo, ok_hi;
+  const __nv_bfloat16* q_lo = row_ptr(pr_lo, ok_lo);
+  const __nv_bfloat16* q_hi = row_ptr(pr_hi, ok_hi);
+  uint32_t qa[8][4];
+#pragma unroll
+  for (int kk = 0; kk < 8; ++kk) {
+    const int c = kk * 16 + t4 * 2;
+    qa[kk][0] = ok_lo ? *reinterpret_cast<const uint32_t*>(q_lo + c) : 0u;
+    qa[kk][1] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + c) : 0u;
+    qa[kk][2] = ok_lo ? *reinterpret_cast<const uint32_t*>(q_lo + c + 8) : 0u;
+    qa[kk][3] = ok_hi ? *reinterpret_cast<const uint32_t*>(q_hi + c + 8) : 0u;
+  }
+
+  float o_acc[16][4];
+#pragma unroll
+  for (int n = 0; n < 16; ++n)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o_acc[n][e] = 0.f;
+  float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
+
+  // ldmatrix lane roles: lanes 0-7 address matrix 0, 8-15 matrix 1, 16-23 matrix 2, 24-31 matrix 3
+  const int lm_row = lane & 7, lm_mat = lane >> 3;
+  bool alive = true;
+  for (int i = 0; i < n_my && alive; ++i) {
+    const int s = i % TC_STAGES;
+    const uint32_t ph = static_cast<uint32_t>(i / TC_STAGES) & 1u;
+    alive = ptx::mbar_wait(&full_bar[s], ph, abort_flag, p.error_word);
+    alive = __all_sync(0xffffffffu, alive);
+    if (!alive) break;
+    const uint32_t sb = ptx::smem_u32(smem + s * STAGE_BYTES);
+    const int j0 = (t0 + i) * KT;
+
+    // ---- S = Q K^T for 64 keys: 8 key groups of 8, 8 k-steps of 16 over d_head
+    float sc[8][4];
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
+      const int key = n * 8 + lm_row;
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {      // K lo slab (dims 0-63), K hi slab (dims 64-127)
+#pragma unroll
+        for (int k2 = 0; k2 < 2; ++k2) {          // 32 dims per ldmatrix.x4 = two k-steps
+          uint32_t b0, b1, b2, b3;
+          ldmatrix_x4(sb + half * (KT * 128) + swz(key, k2 * 4 + lm_mat), b0, b1, b2, b3);
+          const int kk = half * 4 + k2 * 2;
+          mma_bf16_16816(sc[n], qa[kk], b0, b1);
+          mma_bf16_16816(sc[n], qa[kk + 1], b2, b3);
+        }
+      }
+    }
+    // ---- scale, mask keys beyond kv_len, online softmax (rows g4 and g4 + 8)
+    float mx_lo = -INFINITY, mx_hi = -INFINITY;
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const int key = j0 + n * 8 + t4 * 2;
+      const bool v0 = key < kv_len, v1 = key + 1 < kv_len;
+      sc[n][0] = v0 ? sc[n][0] * p.scale_log2 : -INFINITY;
+      sc[n][1] = v1 ? sc[n][1] * p.scale_log2 : -INFINITY;
+      sc[n][2] = v0 ? sc[n][2] * p.scale_log2 : -INFINITY;
+      sc[n][3] = v1 ? sc[n][3] * p.scale_log2 : -INFINITY;
+      mx_lo = fmaxf(mx_lo, fmaxf(sc[n][0], sc[n][1]));
+      mx_hi = fmaxf(mx_hi, fmaxf(sc[n][2], sc[n][3]));
+    }
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 1));
+    mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
+    mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
+    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);  // finite: every tile holds a valid key
+    const float c_lo = exp2f(m_lo - mn_lo), c_hi = exp2f(m_hi - mn_hi);
+    m_lo = mn_lo;
+    m_hi = mn_hi;
+    float s_lo = 0.f, s_hi = 0.f;
+    uint32_t pa[4][4];  // P as A fragments: 4 k-steps of 16 keys
+#pragma unroll
+    for (int n = 0; n < 8; ++n) {
+      const float p0 = exp2f(sc[n][0] - mn_lo), p1 = exp2f(sc[n][1] - mn_lo);
+      const float p2 = exp2f(sc[n][2] - mn_hi), p3 = exp2f(sc[n][3] - mn_hi);
+      s_lo += p0 + p1;
+      s_hi += p2 + p3;
+      pa[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
+      pa[n >> 1][(n & 1) * 2 + 1] = pack_bf16(p2, p3);
+    }
+    l_lo = l_lo * c_lo + s_lo;
+    l_hi = l_hi * c_hi + s_hi;
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      o_acc[n][0] *= c_lo; o_acc[n][1] *= c_lo;
+      o_acc[n][2] *= c_hi; o_acc[n][3] *= c_hi;
+    }
+    // ---- O += P V: 4 k-steps of 16 keys, 16 output groups of 8 dims
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      // matrices of one ldmatrix.x4.trans: (keys 0-7, dims d..d+7), (keys 8-15, same dims),
+      // (keys 0-7, dims d+8..), (keys 8-15, dims d+8..)
+      const int key = kk * 16 + (lm_mat & 1) * 8 + lm_row;
+#pragma unroll
+      for (int n2 = 0; n2 < 8; ++n2) {  // 16 dims per ldmatrix
+        const int chunk = n2 * 2 + (lm_mat >> 1);  // 16-byte chunk 0..15 over 128 dims
+        uint32_t b0, b1, b2, b3;
+        ldmatrix_x4_trans(sb + (2 + (chunk >> 3)) * (KT * 128) + swz(key, chunk & 7), b0, b1, b2, b3);
+        mma_bf16_16816(o_acc[n2 * 2], pa[kk], b0, b1);
+        mma_bf16_16816(o_acc[n2 * 2 + 1], pa[kk], b2, b3);
+      }
+    }
+    // ---- release the stage; the producer thread refills it with tile i + TC_STAGES
+    __syncwarp();
+    if (lane == 0) ptx::mbar_arrive(&empty_bar[s]);
+    if (threadIdx.x == 0 && i + TC_STAGES < n_my) {
+      if (ptx::mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) issue(i + TC_STAGES);
+    }
+  }
+  // row sums over the quad
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1);
+  l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1);
+  l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
+
+  auto out_ptr = [&](int pr) -> __nv_bfloat16* {
+    const int hg = pr / rps, r = pr % rps;
+    return p.out + (static_cast<size_t>(b) * rps + r) * p.hq * 128 + (g * group + hg) * 128;
+  };
+  if (p.n_splits == 1) {
+    if (!alive) return;
+    const float i_lo = 1.0f / l_lo, i_hi = 1.0f / l_hi;
+    if (ok_lo) {
+      __nv_bfloat16* o = out_ptr(pr_lo);
+#pragma unroll
+      for (int n = 0; n < 16; ++n)
+        *reinterpret_cast<uint32_t*>(o + n * 8 + t4 * 2) = pack_bf16(o_acc[n][0] * i_lo, o_acc[n][1] * i_lo);
+    }
+    if (ok_hi) {
+      __nv_bfloat16* o = out_ptr(pr_hi);
+#pragma unroll
+      for (int n = 0; n < 16; ++n)
+        *reinterpret_cast<uint32_t*>(o + n * 8 + t4 * 2) = pack_bf16(o_acc[n][2] * i_hi, o_acc[n][3] * i_hi);
+    }
+    return;
+  }
+  // ---- several key splits: write the partial, the last CTA to arrive merges
+  const int tile_id = pair * gridDim.x + qt;
+  float* part = p.partial + (static_cast<size_t>(tile_id) * p.n_splits + split) * BM * PART_LD;
+  {
+    float* r_lo = part + static_cast<size_t>(warp * 16 + g4) * PART_LD;
+    float* r_hi = r_lo + 8 * PART_LD;
+#pragma unroll
+    for (int n = 0; n < 16; ++n) {
+      *reinterpret_cast<float2*>(r_lo + n * 8 + t4 * 2) = make_float2(o_acc[n][0], o_acc[n][1]);
+      *reinterpret_cast<float2*>(r_hi + n * 8 + t4 * 2) = make_float2(o_acc[n][2], o_acc[n][3]);
+    }
+    if (t4 == 0) {
+      r_lo[128] = m_lo; r_lo[129] = l_lo;  // a split without tiles leaves m = -inf, l = 0
+      r_hi[128] = m_hi; r_hi[129] = l_hi;
+    }
+  }
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int old = atomicAdd(&p.counters[tile_id], 1);
+    const int last = (old == p.n_splits - 1) ? 1 : 0;
+    if (last) p.counters[tile_id] = 0;
+    *last_flag = last;
+    __threadfence();
+  }
+  __syncthreads();
+  if (!*last_flag) return;
+  const float* base = p.partial + static_cast<size_t>(tile_id) * p.n_splits * BM * PART_LD;
+  for (int e = threadIdx.x; e < BM * 32; e += NW * 32) {  // one thread per (row, 4 output dims)
+    const int row = e >> 5, c4 = (e & 31) * 4;
+    const int pr = qt * BM + row;
+    if (pr >= R || (pr % rps) >= n_valid) continue;
+    float M = -INFINITY;
+    for (int s2 = 0; s2 < p.n_splits; ++s2) M = fmaxf(M, __ldcg(base + (static_cast<size_t>(s2) * BM + row) * PART_LD + 128));
+    float L = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int s2 = 0; s2 < p.n_splits; ++s2) {
+      const float* pr_s = base + (static_cast<size_t>(s2) * BM + row) * PART_LD;
+      const float ls = __ldcg(pr_s + 129);
+      if (ls == 0.f) continue;
+      const float w = exp2f(__ldcg(pr_s + 128) - M);
+      const float4 v = __ldcg(reinterpret_cast<const float4*>(pr_s + c4));
+      L += w * ls;
+      a0 += w * v.x; a1 += w * v.y; a2 += w * v.z; a3 += w * v.w;
+    }
+    const float inv = 1.0f / L;
+    uint2 o2 = make_uint2(pack_bf16(a0 * inv, a1 * inv), pack_bf16(a2 * inv, a3 * inv));
+    *reinterpret_cast<uint2*>(out_ptr(pr) + c4) = o2;
+  }
+}
+
+inline size_t attn_tc_smem_bytes() { return 1024 + TC_STAGES * STAGE_BYTES + 2 * TC_STAGES * 8 + 64; }
+
+}  // namespace attn
+}  // namespace d3

@@ -56,6 +56,13 @@ struct d3_ctx {
   int* argmax = nullptr;
   int *prefix_len = nullptr, *pos_base = nullptr, *n_valid = nullptr, *kv_len = nullptr;
   uint32_t* error_word = nullptr;
+  // tensor-core attention (bf16, d_head 128)
+  bool attn_tc = false;
+  CUtensorMap kv_tmap{};
+  float* attn_partial = nullptr;
+  size_t attn_partial_floats = 0;
+  int* attn_counters = nullptr;
+  int n_attn_counters = 0;
   float* partial = nullptr;
   size_t partial_slots = 0;  // capacity in (tile, split) slots of 128*128 floats
   int* tile_count = nullptr;
@@ -373,8 +380,62 @@ int launch_attention(d3_ctx* c, const void* q, const void* kc, const void* vc, v
   return D3_OK;
 }
 
+// Tensor-core attention launch: warps per CTA from the packed rows per kv head, key splits so that
+// about two CTAs per SM exist even at batch 1 (decode only; prefill has enough query tiles).
+template <int NW>
+int launch_attn_tc(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
+  auto kern = attn::attn_tc_kernel<NW>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::attn_tc_smem_bytes())));
+    attr_set = true;
+  }
+  kern<<<grid, NW * 32, attn::attn_tc_smem_bytes(), c->stream>>>(c->kv_tmap, p);
+  LAUNCHED(c, "attn_tc_kernel");
+  return D3_OK;
+}
+
+int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
+  const d3_config& g = c->cfg;
+  const int group = g.n_q_heads / g.n_kv_heads;
+  const int R = group * rm.rows_per_seq;
+  const int nw = R <= 32 ? 2 : (R <= 64 ? 4 : 8);
+  const int bm = nw * 16;
+  const int q_tiles = (R + bm - 1) / bm;
+  const int pairs = rm.bs * g.n_kv_heads;
+  int splits = 1;
+  if (q_tiles <= 2) {  // decode-sized: split the keys when (sequence, kv head) pairs alone leave SMs idle
+    const int max_tiles = (g.max_seq + attn::KT - 1) / attn::KT;
+    splits = (2 * c->n_sms + pairs * q_tiles - 1) / (pairs * q_tiles);
+    splits = std::min(splits, std::max(1, max_tiles / 2));
+    splits = std::max(1, std::min(splits, 16));
+    const size_t need = static_cast<size_t>(pairs) * q_tiles * splits * bm * attn::PART_LD;
+    if (need > c->attn_partial_floats || pairs * q_tiles > c->n_attn_counters) splits = 1;
+  }
+  attn::AttnTcParams p{};
+  p.q = static_cast<const bf16*>(q);
+  p.out = static_cast<bf16*>(out);
+  p.rm = rm;
+  p.hq = g.n_q_heads; p.hkv = g.n_kv_heads; p.max_seq = g.max_seq;
+  const long long plane_rows = static_cast<long long>(g.max_batch) * g.n_kv_heads * g.max_seq;
+  p.k_row0 = (static_cast<long long>(layer) * 2 + 0) * plane_rows;
+  p.v_row0 = (static_cast<long long>(layer) * 2 + 1) * plane_rows;
+  p.n_splits = splits;
+  p.scale_log2 = 1.4426950408889634f / std::sqrt(static_cast<float>(g.d_head));
+  p.partial = c->attn_partial;
+  p.counters = c->attn_counters;
+  p.error_word = c->error_word;
+  dim3 grid(q_tiles, pairs, splits);
+  switch (nw) {
+    case 2: return launch_attn_tc<2>(c, p, grid);
+    case 4: return launch_attn_tc<4>(c, p, grid);
+    default: return launch_attn_tc<8>(c, p, grid);
+  }
+}
+
 int run_attention(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
   ProfScope ps(c, D3_PROF_ATTENTION);
+  if (c->attn_tc) return run_attention_tc(c, q, layer, out, rm);
   const char* base = static_cast<const char*>(c->kv);
   const void* kc = base + (static_cast<size_t>(layer) * 2 + 0) * c->kv_layer_elems * c->esz;
   const void* vc = base + (static_cast<size_t>(layer) * 2 + 1) * c->kv_layer_elems * c->esz;
@@ -567,6 +628,25 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
     A_(c->partial, c->partial_slots * 128 * 128 * sizeof(float));
     c->n_tile_count = 1 << 16;
     A_(c->tile_count, sizeof(int) * c->n_tile_count);
+  }
+  if (c->use_tc && g.d_head == 128) {
+    const long long kv_rows = static_cast<long long>(g.n_layers) * 2 * g.max_batch * g.n_kv_heads * g.max_seq;
+    if (kv_rows < (1ll << 31)) {
+      const CUtensorMap* tm = nullptr;
+      int rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, attn::KT, &tm);
+      if (rc_ != D3_OK) return bail(rc_);
+      c->kv_tmap = *tm;
+      // partial (O, m, l) of every (sequence, kv head, query tile, key split) of a decode forward
+      const int group = g.n_q_heads / g.n_kv_heads;
+      const int R = group * g.block;
+      const int bm = R <= 32 ? 32 : (R <= 64 ? 64 : 128);
+      const size_t tiles = static_cast<size_t>(g.max_batch) * g.n_kv_heads * ((R + bm - 1) / bm);
+      c->attn_partial_floats = (tiles + 4 * static_cast<size_t>(c->n_sms)) * bm * attn::PART_LD;
+      A_(c->attn_partial, c->attn_partial_floats * sizeof(float));
+      c->n_attn_counters = static_cast<int>(tiles);
+      A_(c->attn_counters, sizeof(int) * tiles);
+      c->attn_tc = true;
+    }
   }
   A_(c->gen.mode, sizeof(int) * g.max_batch);
   A_(c->gen.block_idx, sizeof(int) * g.max_batch);

@@ -194,6 +194,25 @@ def test_attention_bf16(ctx_bf16, rows, kv_lens):
     _attention_case(ctx_bf16, BF16_SHAPE, True, 3, rows, kv_lens, rows + sum(kv_lens))
 
 
+ATT_GQA = si.scaled_shape(si.QWEN7B, name="att-gqa7", n_layers=1, d_model=256, n_q_heads=14, n_kv_heads=2,
+                          d_ffn=256, vocab=1000, d_head=128)
+ATT_MHA = si.scaled_shape(si.LLADA8B, name="att-mha", n_layers=1, d_model=256, n_q_heads=3, n_kv_heads=3,
+                          d_ffn=256, vocab=1000, d_head=128)
+
+
+@pytest.mark.parametrize("shape", [ATT_GQA, ATT_MHA], ids=["gqa7", "mha"])
+@pytest.mark.parametrize("rows,kv_lens", [(32, [64, 33, 1]), (32, [600, 65, 257]), (64, [640, 63, 128]),
+                                          (7, [40, 300, 5]), (100, [100, 37, 129]), (300, [300, 5, 64])])
+def test_attention_bf16_tensor_core(shape, rows, kv_lens):
+    """d_head 128 runs the TMA-staged tensor-core kernel: decode-sized row counts take several key
+    splits (partials merged by the last CTA), prefill-sized ones several query tiles; group 7 packs
+    the query heads of one kv head into shared tiles."""
+    with Ctx(shape, None, block=32, max_batch=3, max_seq=640, max_prefill_rows=3 * 300) as ctx:
+        _attention_case(ctx, shape, True, 3, rows, kv_lens, rows + sum(kv_lens))
+        # same inputs again: split counters must have been left clean
+        _attention_case(ctx, shape, True, 3, rows, kv_lens, rows + sum(kv_lens))
+
+
 @pytest.mark.parametrize("rows,kv_lens", [(16, [48, 17]), (5, [5, 200])])
 def test_attention_fp32(ctx_f32, rows, kv_lens):
     _attention_case(ctx_f32, F32_SHAPE, False, 2, rows, kv_lens, rows)
