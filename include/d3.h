@@ -167,7 +167,9 @@ int d3_set_state(d3_ctx *ctx, const int32_t *prefix_len, int32_t bs);
  * d3_op_linear: y = x . w^T.  x [device][m, k], w [device][n, k] in the context dtype;
  *   epilogue 0: y fp32 [m, n];  1: y in context dtype [m, n];  2: y fp32 [m, n] += product
  *   (residual);  3: w holds gate/up rows interleaved (row 2j = gate j, row 2j+1 = up j; n = 2*f), y in
- *   context dtype [m, f] = silu(gate) * up.   splits: split-K factor for the tensor-core kernel (0 = auto).
+ *   context dtype [m, f] = silu(gate) * up.   splits: number of CTAs the tensor-core kernel deals its
+ *   (output tile, K slab) units to (0 = auto: one per SM); any value gives the same result up to the
+ *   order of fp32 partial sums.
  * d3_op_lm_head_stats: conf/entropy/argmax [device][m] of scale * x . w^T with mask_id excluded.
  * d3_op_attention: q [device][bs*rows, n_q_heads*d_head]; keys/values are the context's cache of
  *   `layer`; sequence b attends to its slots [0, kv_len[b]); out like q.  kv_len [device][bs].
@@ -219,6 +221,13 @@ int d3_op_unmask(d3_ctx *ctx, const float *conf, const float *entropy, const int
 int d3_lm_head_stats_static(const void *x, const void *w, int32_t dtype, int32_t m, int32_t vocab, int32_t k,
                             float scale, int32_t mask_id, float *conf, float *entropy, int32_t *argmax,
                             void *cuda_stream);
+
+/* Kernel overlap.  By default consecutive kernels of a forward are launched with programmatic stream
+ * serialization: a kernel may become resident and prefetch its weights while its predecessor drains,
+ * and waits (griddepcontrol.wait) before it touches anything the predecessor wrote.  on = 0 launches
+ * every kernel fully serialized (for timing kernels in isolation and for debugging); results are
+ * identical either way. */
+int d3_set_overlap(d3_ctx *ctx, int on);
 
 /* Per-class kernel timing for measurement runs.  While enabled, every launch of the forward pass is
  * bracketed by a CUDA event pair on the context's stream; d3_profile_read waits for the stream and

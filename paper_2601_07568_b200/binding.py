@@ -27,7 +27,7 @@ EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
     "d3_get_state", "d3_set_state", "d3_op_linear", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
+    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
 
@@ -276,6 +276,10 @@ def d3_lm_head_stats_static(x: torch.Tensor, w: torch.Tensor, scale: float, mask
 
 PROF_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_head", "gemm_other", "attention",
                 "rmsnorm", "other")
+
+
+def d3_set_overlap(ctx, on: bool) -> None:
+    _check(ctx, lib().d3_set_overlap(ctx, C.c_int(1 if on else 0)))
 
 
 def d3_profile_enable(ctx, on: bool) -> None:

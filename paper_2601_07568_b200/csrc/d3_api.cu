@@ -12,6 +12,7 @@
 #include <map>
 #include <string>
 #include <tuple>
+#include <utility>
 #include <vector>
 
 #include "attention.cuh"
@@ -79,6 +80,8 @@ struct d3_ctx {
   int64_t dev_bytes = 0;
   // per-class kernel timing (off by default)
   bool prof_on = false;
+  bool pdl = true;           // programmatic dependent launch between the kernels of a forward
+  int* skip_flag = nullptr;  // device flag: non-zero turns the forward's kernels into no-ops
   struct ProfPair { cudaEvent_t a, b; int cls; };
   std::vector<ProfPair> prof_pool;
   size_t prof_used = 0;
@@ -232,89 +235,82 @@ struct QkvExtra {
   void* v_cache;
 };
 
+// Launch with programmatic stream serialization: the kernel may become resident while the previous
+// kernel of the stream is still running; everything it does before griddepcontrol.wait must be
+// independent of that kernel.  Off while per-class timing is on, so that event pairs bracket one kernel.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(d3_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  at[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = (c->pdl && !c->prof_on) ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+
 template <int EPI, int BLOCK_N>
-int launch_tc(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, dim3 grid,
+int launch_tc(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, int n_ctas,
               size_t smem) {
   auto kern = tc::gemm_tc_kernel<EPI, BLOCK_N>;
   static bool attr_set = false;
   if (!attr_set) {
-    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
     attr_set = true;
   }
-  kern<<<grid, tc::NUM_THREADS, smem, c->stream>>>(*tx, *tw, p);
+  CUDA_TRY(c, launch_pdl(c, kern, dim3(n_ctas), dim3(tc::NUM_THREADS), smem, *tx, *tw, p));
   LAUNCHED(c, "gemm_tc_kernel");
   return D3_OK;
 }
 
-int pick_splits(const d3_ctx* c, int m_tiles, int n_tiles, int k_chunks, int epi, int hint) {
-  if (epi == EPI_STATS) return 1;
-  int tiles = m_tiles * n_tiles;
-  int s = hint;
-  if (s <= 0) {
-    // split K only when even 32-wide column tiles leave most SMs idle
-    s = 1;
-    if (tiles * 2 <= c->n_sms) {
-      s = c->n_sms / tiles;
-      int cap = k_chunks / 8;  // keep at least eight 64-wide K slabs per split
-      if (cap < 1) cap = 1;
-      if (s > cap) s = cap;
-      if (s > 8) s = 8;
-    }
-  }
-  if (s > k_chunks) s = k_chunks;
-  if (s < 1) s = 1;
-  while (s > 1 && static_cast<size_t>(tiles) * s > c->partial_slots) --s;
-  if (tiles > c->n_tile_count) s = 1;
-  return s;
-}
-
 template <int BLOCK_N>
-int dispatch_tc(d3_ctx* c, int epi, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, dim3 grid,
+int dispatch_tc(d3_ctx* c, int epi, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, int n_ctas,
                 size_t smem) {
   switch (epi) {
-    case EPI_F32: return launch_tc<EPI_F32, BLOCK_N>(c, tx, tw, p, grid, smem);
-    case EPI_T: return launch_tc<EPI_T, BLOCK_N>(c, tx, tw, p, grid, smem);
-    case EPI_RESID: return launch_tc<EPI_RESID, BLOCK_N>(c, tx, tw, p, grid, smem);
-    case EPI_SWIGLU: return launch_tc<EPI_SWIGLU, BLOCK_N>(c, tx, tw, p, grid, smem);
-    case EPI_QKV: return launch_tc<EPI_QKV, BLOCK_N>(c, tx, tw, p, grid, smem);
-    case EPI_STATS:
-      if constexpr (BLOCK_N % 128 == 0) return launch_tc<EPI_STATS, BLOCK_N>(c, tx, tw, p, grid, smem);
-      break;
+    case EPI_F32: return launch_tc<EPI_F32, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
+    case EPI_T: return launch_tc<EPI_T, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
+    case EPI_RESID: return launch_tc<EPI_RESID, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
+    case EPI_SWIGLU: return launch_tc<EPI_SWIGLU, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
+    case EPI_QKV: return launch_tc<EPI_QKV, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
+    case EPI_STATS: return launch_tc<EPI_STATS, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
   }
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
-// Column-tile width.  Skinny matmuls (one row tile) stream every weight byte exactly once, so the
-// tile is chosen to give about one CTA per SM or more with no split-K; wide row counts use 128.
-int pick_block_n(const d3_ctx* c, int M, int N, int epi) {
-  if (epi == EPI_STATS) return 128;
-  if (M > 128) return 128;
-  for (int bn : {128, 64, 32}) {
-    if ((N + bn - 1) / bn >= c->n_sms - 20) return bn;
-  }
-  return 32;
-}
-
+// One persistent CTA per SM; the (tile, K slab) units are dealt out evenly (see gemm_tc.cuh).
+// `ctas_hint` > 0 forces the grid size (tests use it to move the segment borders around).
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
-                  int splits_hint, const QkvExtra* qx) {
-  const int BLOCK_N = pick_block_n(c, M, N, epi);
+                  int ctas_hint, const QkvExtra* qx) {
+  constexpr int BLOCK_N = 128;
   const int m_tiles = (M + 127) / 128, n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_chunks = (K + 63) / 64;
-  int a_rows = M >= 128 ? 128 : ((M + 31) / 32) * 32;
+  const long long tiles = static_cast<long long>(m_tiles) * n_tiles;
+  if (tiles > c->n_tile_count) return fail(c, D3_ERR_SHAPE, "matmul has more output tiles than arrival counters");
+  const int a_rows = M >= 128 ? 128 : ((M + 31) / 32) * 32;
   tc::GemmParams p{};
   p.M = M; p.N = N; p.K = K;
   p.a_rows = a_rows;
-  p.splits = pick_splits(c, m_tiles, n_tiles, k_chunks, epi, splits_hint);
+  p.m_tiles = m_tiles; p.n_tiles = n_tiles; p.k_chunks = k_chunks;
+  p.total_units = tiles * k_chunks;
+  // at least eight K slabs per CTA: shorter ranges only add partial tiles
+  long long n_ctas = std::min<long long>(c->n_sms, std::max<long long>(1, p.total_units / 8));
+  if (ctas_hint > 0) n_ctas = std::min<long long>(ctas_hint, p.total_units);
+  n_ctas = std::min<long long>(n_ctas, std::min<long long>(tc::MAX_CTAS, static_cast<long long>(c->partial_slots / 2)));
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + BLOCK_N * 128;
-  // two CTAs per SM when there are more tiles than SMs, otherwise one CTA with a deeper pipeline
-  const bool two_per_sm = static_cast<long long>(m_tiles) * n_tiles * p.splits > c->n_sms;
-  int stages = static_cast<int>(((two_per_sm ? 100 : 190) * 1024) / stage_bytes);
-  if (stages > 24) stages = 24;
-  if (stages < 2) stages = 2;
+  // skinny matmuls are bound by HBM: keep the ring near 100 KB so that the next kernel's CTAs fit
+  // beside this one's and start streaming their weights; wide ones get all of shared memory
+  const size_t ring = (M <= 128 ? 100 : 200) * 1024;
+  int stages = static_cast<int>(ring / stage_bytes);
+  stages = std::max(2, std::min(stages, 16));
   p.stages = stages;
   p.partial = c->partial;
   p.tile_count = c->tile_count;
   p.error_word = c->error_word;
+  p.skip_flag = c->skip_flag;
   p.ep = ep;
   if (qx) {
     p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
@@ -325,13 +321,8 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   const CUtensorMap *tx, *tw;
   TRY(get_tmap(c, X, M, K, a_rows, &tx));
   TRY(get_tmap(c, W, N, K, BLOCK_N, &tw));
-  dim3 grid(m_tiles, n_tiles, p.splits);
-  size_t smem = tc::gemm_tc_smem_bytes(a_rows, BLOCK_N, stages);
-  switch (BLOCK_N) {
-    case 32: return dispatch_tc<32>(c, epi, tx, tw, p, grid, smem);
-    case 64: return dispatch_tc<64>(c, epi, tx, tw, p, grid, smem);
-    default: return dispatch_tc<128>(c, epi, tx, tw, p, grid, smem);
-  }
+  const size_t smem = tc::gemm_tc_smem_bytes(a_rows, BLOCK_N, stages);
+  return dispatch_tc<BLOCK_N>(c, epi, tx, tw, p, static_cast<int>(n_ctas), smem);
 }
 
 template <typename T>
@@ -390,7 +381,7 @@ int launch_attn_tc(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
     CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::attn_tc_smem_bytes())));
     attr_set = true;
   }
-  kern<<<grid, NW * 32, attn::attn_tc_smem_bytes(), c->stream>>>(c->kv_tmap, p);
+  CUDA_TRY(c, launch_pdl(c, kern, grid, dim3(NW * 32), attn::attn_tc_smem_bytes(), c->kv_tmap, p));
   LAUNCHED(c, "attn_tc_kernel");
   return D3_OK;
 }
@@ -453,16 +444,15 @@ void* v_plane(d3_ctx* c, int layer) {
 int run_rmsnorm(d3_ctx* c, const float* x, const float* gain, void* xn, int M) {
   ProfScope ps(c, D3_PROF_RMSNORM);
   const int d = c->cfg.d_model;
-  const int threads = d >= 1024 ? 256 : 128;
-  if (c->is_bf16) rmsnorm_kernel<bf16><<<M, threads, 0, c->stream>>>(x, gain, static_cast<bf16*>(xn), d, c->cfg.rms_eps);
-  else rmsnorm_kernel<float><<<M, threads, 0, c->stream>>>(x, gain, static_cast<float*>(xn), d, c->cfg.rms_eps);
+  if (c->is_bf16) CUDA_TRY(c, launch_pdl(c, rmsnorm_kernel<bf16>, dim3(M), dim3(256), 0, x, gain, static_cast<bf16*>(xn), d, c->cfg.rms_eps));
+  else CUDA_TRY(c, launch_pdl(c, rmsnorm_kernel<float>, dim3(M), dim3(256), 0, x, gain, static_cast<float*>(xn), d, c->cfg.rms_eps));
   LAUNCHED(c, "rmsnorm_kernel");
   return D3_OK;
 }
 
 int run_stats_merge(d3_ctx* c, int M, int n_tiles, float* conf, float* ent, int* argmax) {
   ProfScope ps(c, D3_PROF_OTHER);
-  stats_merge_kernel<<<(M + 3) / 4, 128, 0, c->stream>>>(c->stat_part, n_tiles, M, conf, ent, argmax);
+  CUDA_TRY(c, launch_pdl(c, stats_merge_kernel, dim3((M + 3) / 4), dim3(128), 0, static_cast<const float4*>(c->stat_part), n_tiles, M, conf, ent, argmax));
   LAUNCHED(c, "stats_merge_kernel");
   return D3_OK;
 }
@@ -480,8 +470,8 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
 
   {
     ProfScope ps(c, D3_PROF_OTHER);
-    if (c->is_bf16) embed_kernel<bf16><<<M, 128, 0, c->stream>>>(ids, static_cast<const bf16*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
-    else embed_kernel<float><<<M, 128, 0, c->stream>>>(ids, static_cast<const float*>(c->tok_emb), c->x, d, g.vocab, c->error_word);
+    if (c->is_bf16) CUDA_TRY(c, launch_pdl(c, embed_kernel<bf16>, dim3(M), dim3(128), 0, ids, static_cast<const bf16*>(c->tok_emb), c->x, d, g.vocab, c->error_word));
+    else CUDA_TRY(c, launch_pdl(c, embed_kernel<float>, dim3(M), dim3(128), 0, ids, static_cast<const float*>(c->tok_emb), c->x, d, g.vocab, c->error_word));
     LAUNCHED(c, "embed_kernel");
   }
 
@@ -1021,6 +1011,11 @@ extern "C" int d3_get_error_word(d3_ctx* c, uint32_t* word) {
   if (!c || !word) return D3_ERR_INVALID_ARG;
   CUDA_TRY(c, cudaMemcpyAsync(word, c->error_word, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return D3_OK;
+}
+extern "C" int d3_set_overlap(d3_ctx* c, int on) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  c->pdl = on != 0;
   return D3_OK;
 }
 extern "C" int d3_profile_enable(d3_ctx* c, int on) {

@@ -3,9 +3,21 @@
 //   * operands are staged in shared memory by TMA (128-byte swizzle, 64-element K slabs),
 //   * one elected thread issues tcgen05.mma (128 x BLOCK_N x 16) into a TMEM accumulator,
 //   * four epilogue warps read the accumulator back with tcgen05.ld; TMEM lane = row of X, so every
-//     epilogue (residual add, SwiGLU, RoPE + cache write, softmax statistics) is thread-local,
-//   * split-K: each split writes an fp32 partial tile; the last split to arrive (an atomic counter
-//     per tile, nobody spins) sums the partials in split order, which keeps results deterministic.
+//     epilogue (residual add, SwiGLU, RoPE + cache write, softmax statistics) is thread-local.
+//
+// Scheduling.  The work is the list of units (output tile, 64-wide K slab), tile-major.  The grid is
+// at most one CTA per SM and CTA i owns the contiguous unit range [U*i/n, U*(i+1)/n): every SM
+// streams the same number of weight bytes whatever the shape.  A range is cut into segments at tile
+// borders.  A segment that spans a whole tile goes straight from TMEM to its epilogue; otherwise the
+// CTA writes an fp32 partial tile and bumps the tile's arrival counter, and the CTA that arrives last
+// (nobody waits) sums the partials in K order and runs the epilogue, so results do not depend on
+// timing.  Two TMEM accumulators alternate between segments: the epilogue of one segment overlaps the
+// MMAs of the next.
+//
+// Dependent launch.  Weights do not depend on the previous kernel of the stream, so the producer
+// fills the whole shared-memory ring with weight slabs before it executes griddepcontrol.wait, and
+// only then loads the matching activation slabs; with at most ~100 KB of shared memory per CTA the
+// next matmul's CTAs become resident and stream weights while the current kernel drains.
 //
 // Skinny case (M <= 64 rows, the batch-1 denoise step): the X box is only a_rows high, and the
 // stage stride of X in shared memory shrinks with it, so that almost all of shared memory holds
@@ -24,15 +36,18 @@ constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
 constexpr int NUM_THREADS = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int MAX_CTAS = 512;     // upper bound of the grid (segment list of a tile lives in shared memory)
 
 struct GemmParams {
   int M, N, K;
   int a_rows;       // rows of the X box: 32, 64 or 128
   int stages;       // pipeline depth
-  int splits;       // split-K factor (grid.z)
-  float* partial;   // split-K workspace [tile][split][BLOCK_N][128] fp32 (splits > 1)
-  int* tile_count;  // split-K arrival counters [tiles], zero on entry and on exit
+  int m_tiles, n_tiles, k_chunks;
+  long long total_units;  // m_tiles * n_tiles * k_chunks
+  float* partial;   // partial tiles [2 * grid][BLOCK_N][128] fp32: slot 2i = CTA i's first segment, 2i+1 = its last
+  int* tile_count;  // arrival counters [tiles], zero on entry and on exit
   uint32_t* error_word;
+  const int* skip_flag;  // optional: non-zero -> the whole launch is a no-op
   EpiParams ep;
   // EPI_QKV only
   const float* rope_cos;  // [max_seq][64]
@@ -80,13 +95,14 @@ struct TmemSource {
 };
 template <int BLOCK_N>
 struct PartialSource {
-  const float* base;  // this tile's partials: [split][BLOCK_N][128]
-  int splits, row;
+  const float* partial;   // workspace base
+  const int* slots;       // shared memory: partial slots of this tile's segments in K order
+  int n_seg, row;
   __device__ __forceinline__ void load(int c, float (&v)[32]) const {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = 0.f;
-    for (int s = 0; s < splits; ++s) {
-      const float* p = base + (static_cast<size_t>(s) * BLOCK_N + c) * 128 + row;
+    for (int s = 0; s < n_seg; ++s) {
+      const float* p = partial + (static_cast<size_t>(slots[s]) * BLOCK_N + c) * 128 + row;
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] += __ldcg(p + j * 128);
     }
@@ -275,14 +291,26 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
 }
 
 // ----------------------------------------------------------------------------- kernel
-// grid = (m_tiles, n_tiles, splits); dynamic shared memory (1024-byte aligned inside the kernel):
+__device__ __forceinline__ long long unit_begin(long long U, int i, int n) { return U * i / n; }
+// The CTA whose unit range contains unit x (ranges of CTAs without units are skipped by construction).
+__device__ __forceinline__ int cta_of_unit(long long x, long long U, int n) {
+  int i = static_cast<int>(x * n / U);
+  if (i > n - 1) i = n - 1;
+  while (i + 1 < n && unit_begin(U, i + 1, n) <= x) ++i;
+  while (i > 0 && unit_begin(U, i, n) > x) --i;
+  return i;
+}
+
+// grid = (n_ctas); dynamic shared memory (1024-byte aligned inside the kernel):
 //   [stages x a_rows x 128 B]  X slabs      (stage stride a_rows*128)
 //   [stages x BLOCK_N x 128 B] W slabs
-//   barriers: full[stages], empty[stages], accum; tmem address; flags
+//   barriers: full[stages], empty[stages], acc_full[2], acc_empty[2]; tmem address; flags; segment list
 template <int EPI, int BLOCK_N>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                const GemmParams p) {
+  if (p.skip_flag != nullptr && *p.skip_flag != 0) return;  // written at least one whole graph launch earlier
+  grid_dep_launch();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int stages = p.stages;
@@ -292,18 +320,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   uint8_t* smem_b = smem + static_cast<size_t>(stages) * a_stage_bytes;
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem_b + static_cast<size_t>(stages) * b_stage_bytes);
   uint64_t* empty_bar = full_bar + stages;
-  uint64_t* accum_bar = empty_bar + stages;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(accum_bar + 1);
+  uint64_t* acc_full = empty_bar + stages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  int* last_flag = const_cast<int*>(abort_flag) + 1;
+  int* last_flag = const_cast<int*>(abort_flag) + 1;  // 0: not last, else number of segments of the tile
+  int* seg_slots = last_flag + 1;                      // [MAX_CTAS]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tile = blockIdx.x, n_tile = blockIdx.y, split = blockIdx.z;
-  const int k_chunks = (p.K + BLOCK_K - 1) / BLOCK_K;
-  const int kc0 = static_cast<int>(static_cast<long long>(k_chunks) * split / p.splits);
-  const int kc1 = static_cast<int>(static_cast<long long>(k_chunks) * (split + 1) / p.splits);
-  const int n_k = kc1 - kc0;
-  constexpr uint32_t TMEM_COLS = BLOCK_N < 32 ? 32 : BLOCK_N;
+  const int cta = blockIdx.x, n_cta = gridDim.x;
+  const long long U = p.total_units;
+  const long long u0 = unit_begin(U, cta, n_cta), u1 = unit_begin(U, cta + 1, n_cta);
+  const int KC = p.k_chunks;
+  constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;  // 256 or 512: a power of two >= 32
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmap_x);
@@ -312,7 +341,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(accum_bar, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 128);
+    }
     *abort_flag = 0;
     *last_flag = 0;
     fence_barrier_init();
@@ -330,82 +362,141 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     // ---------------- TMA producer
     if (lane == 0) {
       const uint32_t tx = a_stage_bytes + b_stage_bytes;
-      for (int i = 0; i < n_k; ++i) {
-        const int s = i % stages;
+      const long long n_total = u1 - u0;
+      const int pre = static_cast<int>(n_total < stages ? n_total : stages);
+      // weights first: they do not depend on the kernels before this one
+      for (int i = 0; i < pre; ++i) {
+        const long long u = u0 + i;
+        const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
+        mbar_arrive_expect_tx(&full_bar[i], tx);
+        tma_load_2d(smem_b + static_cast<size_t>(i) * b_stage_bytes, &tmap_w, &full_bar[i], kc * BLOCK_K,
+                    (tile / p.m_tiles) * BLOCK_N);
+      }
+      grid_dep_wait();
+      for (int i = 0; i < pre; ++i) {
+        const long long u = u0 + i;
+        const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
+        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], kc * BLOCK_K,
+                    (tile % p.m_tiles) * BLOCK_M);
+      }
+      for (long long i = pre; i < n_total; ++i) {
+        const int s = static_cast<int>(i % stages);
         const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
         if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.error_word)) break;
+        const long long u = u0 + i;
+        const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
         mbar_arrive_expect_tx(&full_bar[s], tx);
-        const int kx = (kc0 + i) * BLOCK_K;
-        tma_load_2d(smem_b + static_cast<size_t>(s) * b_stage_bytes, &tmap_w, &full_bar[s], kx, n_tile * BLOCK_N);
-        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kx, m_tile * BLOCK_M);
+        tma_load_2d(smem_b + static_cast<size_t>(s) * b_stage_bytes, &tmap_w, &full_bar[s], kc * BLOCK_K,
+                    (tile / p.m_tiles) * BLOCK_N);
+        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K,
+                    (tile % p.m_tiles) * BLOCK_M);
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
-      for (int i = 0; i < n_k; ++i) {
-        const int s = i % stages;
-        const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
-        if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) break;
+      long long i = 0;
+      int seg = 0;
+      bool ok = true;
+      for (long long u = u0; u < u1 && ok; ++seg) {
+        const int tile = static_cast<int>(u / KC);
+        const int kc0 = static_cast<int>(u - static_cast<long long>(tile) * KC);
+        const long long left = u1 - u;
+        const int n_k = static_cast<int>(left < KC - kc0 ? left : KC - kc0);
+        const int buf = seg & 1;
+        // the epilogue must have drained this accumulator (two segments ago)
+        if (!mbar_wait(&acc_empty[buf], (static_cast<uint32_t>(seg >> 1) & 1u) ^ 1u, abort_flag, p.error_word)) break;
         tc_fence_after();
-        const uint64_t adesc = make_smem_desc(smem_u32(smem_a + static_cast<size_t>(s) * a_stage_bytes));
-        const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + static_cast<size_t>(s) * b_stage_bytes));
+        const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * BLOCK_N);
+        for (int j = 0; j < n_k; ++j, ++i) {
+          const int s = static_cast<int>(i % stages);
+          const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+          if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t adesc = make_smem_desc(smem_u32(smem_a + static_cast<size_t>(s) * a_stage_bytes));
+          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + static_cast<size_t>(s) * b_stage_bytes));
 #pragma unroll
-        for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
-          // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in the (>>4) address field
-          umma_bf16(tmem_base, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
-                    (i > 0 || kk > 0) ? 1u : 0u);
+          for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
+            // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in the (>>4) address field
+            umma_bf16(tmem_d, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
+                      (j > 0 || kk > 0) ? 1u : 0u);
+          }
+          umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
         }
-        umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+        if (ok) umma_commit(&acc_full[buf]);  // this segment's accumulator is complete
+        u += n_k;
       }
-      umma_commit(accum_bar);  // accumulator complete
     }
   } else {
     // ---------------- epilogue warps: TMEM lane group = warp % 4
+    grid_dep_wait();  // residual rows, positions and counters come from earlier kernels
     const int lg = warp & 3;
     const int row = lg * 32 + lane;
-    const int m = m_tile * BLOCK_M + row;
-    const int n0 = n_tile * BLOCK_N;
-    bool ok = (n_k == 0) || mbar_wait(accum_bar, 0, abort_flag, p.error_word);
-    ok = __all_sync(0xffffffffu, ok);
-    tc_fence_after();
-    // warp-uniform: does this lane group hold any row of X at all?
-    const bool warp_live = ok && (lg * 32 < p.a_rows) && (m_tile * BLOCK_M + lg * 32 < p.M);
-    const bool live = warp_live && m < p.M;
-    TmemSource tsrc{tmem_base + (static_cast<uint32_t>(lg * 32) << 16)};
-    if (p.splits == 1) {
-      if (warp_live && n_k > 0) run_epilogue<EPI, BLOCK_N>(tsrc, p, m, n0, live);
-    } else {
-      const int tile_id = n_tile * gridDim.x + m_tile;
-      float* part = p.partial + static_cast<size_t>(tile_id) * p.splits * BLOCK_N * 128;
+    const int et = threadIdx.x - 64;  // 0..127
+    int seg = 0;
+    for (long long u = u0; u < u1; ++seg) {
+      const int tile = static_cast<int>(u / KC);
+      const int kc0 = static_cast<int>(u - static_cast<long long>(tile) * KC);
+      const long long left = u1 - u;
+      const int n_k = static_cast<int>(left < KC - kc0 ? left : KC - kc0);
+      u += n_k;
+      const int buf = seg & 1;
+      const int m_tile = tile % p.m_tiles, n_tile = tile / p.m_tiles;
+      const int m = m_tile * BLOCK_M + row;
+      const int n0 = n_tile * BLOCK_N;
+      bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      // warp-uniform: does this lane group hold any row of X at all?
+      const bool warp_live = (lg * 32 < p.a_rows) && (m_tile * BLOCK_M + lg * 32 < p.M);
+      const bool live = warp_live && m < p.M;
+      TmemSource tsrc{tmem_base + static_cast<uint32_t>(buf * BLOCK_N) + (static_cast<uint32_t>(lg * 32) << 16)};
+      if (n_k == KC) {
+        if (warp_live) run_epilogue<EPI, BLOCK_N>(tsrc, p, m, n0, live);
+        tc_fence_before();
+        mbar_arrive(&acc_empty[buf]);
+        continue;
+      }
+      // partial tile: park it, then let the last arrival finish the tile
+      const int my_slot = 2 * cta + (kc0 == 0 ? 1 : 0);  // a segment starting at K = 0 is this CTA's last one
       if (warp_live) {
-        float* mine = part + static_cast<size_t>(split) * BLOCK_N * 128 + row;
+        float* mine = p.partial + static_cast<size_t>(my_slot) * BLOCK_N * 128 + row;
         for (int c = 0; c < BLOCK_N; c += 32) {
           float v[32];
-          if (n_k > 0) tsrc.load(c, v);
-          else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = 0.f;
-          }
+          tsrc.load(c, v);
 #pragma unroll
           for (int j = 0; j < 32; ++j) mine[static_cast<size_t>(c + j) * 128] = v[j];
         }
       }
+      tc_fence_before();
+      mbar_arrive(&acc_empty[buf]);
       __threadfence();
       epi_bar_sync();
-      if (threadIdx.x == 64) {
-        int old = atomicAdd(&p.tile_count[tile_id], 1);
-        int last = (old == p.splits - 1) ? 1 : 0;
-        if (last) p.tile_count[tile_id] = 0;  // ready for the next launch
+      if (et == 0) {
+        // segments of this tile, in K order: the CTAs whose ranges meet [tile*KC, (tile+1)*KC)
+        const long long t_lo = static_cast<long long>(tile) * KC, t_hi = t_lo + KC;
+        const int i_lo = cta_of_unit(t_lo, U, n_cta), i_hi = cta_of_unit(t_hi - 1, U, n_cta);
+        int n_seg = 0;
+        for (int i = i_lo; i <= i_hi; ++i) {
+          const long long a = unit_begin(U, i, n_cta), b = unit_begin(U, i + 1, n_cta);
+          const long long lo = a > t_lo ? a : t_lo, hi = b < t_hi ? b : t_hi;
+          if (lo < hi) seg_slots[n_seg++] = 2 * i + (lo == t_lo ? 1 : 0);
+        }
+        const int old = atomicAdd(&p.tile_count[tile], 1);
+        const int last = (old == n_seg - 1) ? n_seg : 0;
+        if (last) p.tile_count[tile] = 0;  // ready for the next launch
         *last_flag = last;
         __threadfence();
       }
       epi_bar_sync();
-      if (*last_flag && warp_live) {
-        PartialSource<BLOCK_N> psrc{part, p.splits, row};
+      const int n_seg = *last_flag;
+      if (n_seg > 0 && warp_live) {
+        PartialSource<BLOCK_N> psrc{p.partial, seg_slots, n_seg, row};
         run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, live);
       }
+      epi_bar_sync();  // seg_slots and last_flag are reused by the next segment
     }
     tc_fence_before();
   }
@@ -422,7 +513,7 @@ inline size_t gemm_tc_smem_bytes(int a_rows, int block_n, int stages) {
   size_t body = static_cast<size_t>(stages) * (a_rows * 128 + block_n * 128);
   size_t need = static_cast<size_t>(stages) * a_rows * 128 + static_cast<size_t>(128 - a_rows) * 128 + 128 * 128;
   if (body < need) body = need;
-  return 1024 + body + (2 * stages + 1) * 8 + 64;
+  return 1024 + body + (2 * stages + 4) * 8 + 64 + MAX_CTAS * 4;
 }
 
 }  // namespace tc

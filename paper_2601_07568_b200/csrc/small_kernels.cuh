@@ -2,6 +2,7 @@
 // write, softmax-statistics merge, the threshold unmask decision and the generate-loop bookkeeping.
 #pragma once
 #include "common.cuh"
+#include "ptx_sm100.cuh"
 
 namespace d3 {
 
@@ -26,6 +27,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 template <typename T>
 __global__ void embed_kernel(const int* __restrict__ ids, const T* __restrict__ emb, float* __restrict__ x, int d,
                              int vocab, uint32_t* error_word) {
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
   const int m = blockIdx.x;
   int id = ids[m];
   if (id < 0 || id >= vocab) {
@@ -39,29 +42,57 @@ __global__ void embed_kernel(const int* __restrict__ ids, const T* __restrict__ 
 
 // ----------------------------------------------------------------------------- RMSNorm
 // xn[m, :] = T(x[m, :] * rsqrt(mean(x^2) + eps) * gain); fp32 arithmetic, fixed reduction order.
+// One 256-thread block per row; d % 4 == 0.  The row is read once as float4 and the first 4096
+// elements stay in registers between the two passes.
+__device__ __forceinline__ void store4(float* dst, float a, float b, float c, float d) {
+  *reinterpret_cast<float4*>(dst) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store4(__nv_bfloat16* dst, float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  *reinterpret_cast<uint2*>(dst) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+}
 template <typename T>
-__global__ void rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain, T* __restrict__ xn, int d,
-                               float eps) {
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+                                                      T* __restrict__ xn, int d, float eps) {
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
   const int m = blockIdx.x;
-  const float* row = x + static_cast<size_t>(m) * d;
+  const float4* row = reinterpret_cast<const float4*>(x + static_cast<size_t>(m) * d);
+  const float4* g4 = reinterpret_cast<const float4*>(gain);
+  const int n4 = d >> 2;
+  float4 v[4];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) {
-    float v = row[i];
-    ss += v * v;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int idx = threadIdx.x + i * 256;
+    v[i] = idx < n4 ? row[idx] : make_float4(0.f, 0.f, 0.f, 0.f);
+    ss += v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w;
   }
-  __shared__ float red[32];
+  for (int idx = threadIdx.x + 1024; idx < n4; idx += 256) {
+    const float4 t = row[idx];
+    ss += t.x * t.x + t.y * t.y + t.z * t.z + t.w * t.w;
+  }
+  __shared__ float red[8];
   ss = warp_sum(ss);
   if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = (threadIdx.x < (blockDim.x >> 5)) ? red[threadIdx.x] : 0.f;
-    v = warp_sum(v);
-    if (threadIdx.x == 0) red[0] = v;
-  }
-  __syncthreads();
-  const float rstd = rsqrtf(red[0] / static_cast<float>(d) + eps);
+  float tot = 0.f;
+#pragma unroll
+  for (int w = 0; w < 8; ++w) tot += red[w];  // same order in every thread
+  const float rstd = rsqrtf(tot / static_cast<float>(d) + eps);
   T* out = xn + static_cast<size_t>(m) * d;
-  for (int i = threadIdx.x; i < d; i += blockDim.x) out[i] = TypeOps<T>::from_f(row[i] * rstd * gain[i]);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int idx = threadIdx.x + i * 256;
+    if (idx < n4) {
+      const float4 g = g4[idx];
+      store4(out + 4 * idx, v[i].x * rstd * g.x, v[i].y * rstd * g.y, v[i].z * rstd * g.z, v[i].w * rstd * g.w);
+    }
+  }
+  for (int idx = threadIdx.x + 1024; idx < n4; idx += 256) {
+    const float4 t = row[idx], g = g4[idx];
+    store4(out + 4 * idx, t.x * rstd * g.x, t.y * rstd * g.y, t.z * rstd * g.z, t.w * rstd * g.w);
+  }
 }
 
 // ----------------------------------------------------------------------------- RoPE + cache write
@@ -116,6 +147,8 @@ __global__ void rope_kv_kernel(const float* __restrict__ qkv, T* __restrict__ q_
 // writes confidence = 1/Z, entropy = ln Z - S/Z (nats) and the arg max.
 __global__ void stats_merge_kernel(const float4* __restrict__ part, int n_tiles, int M, float* __restrict__ conf,
                                    float* __restrict__ entropy, int* __restrict__ argmax) {
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
   const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (m >= M) return;

@@ -44,7 +44,7 @@ LINEAR_SHAPES = [(32, 9000, 128), (32, 256, 128), (16, 128, 64), (48, 200, 192),
 
 
 @pytest.mark.parametrize("m,n,k", LINEAR_SHAPES)
-@pytest.mark.parametrize("splits", [0, 1, 3])
+@pytest.mark.parametrize("splits", [0, 1, 3, 7, 148])
 def test_linear_bf16_tensor_core(ctx_bf16, m, n, k, splits):
     rng = np.random.default_rng(m * 7 + n + k)
     xt, x = rand_bf16(rng, (m, k))
