@@ -176,6 +176,16 @@ int d3_set_state(d3_ctx *ctx, const int32_t *prefix_len, int32_t bs);
  * d3_op_unmask: the decision alone on caller-provided statistics. */
 int d3_op_linear(d3_ctx *ctx, const void *x, const void *w, void *y, int32_t m, int32_t n, int32_t k,
                  int32_t epilogue, int32_t splits);
+/* Tiled weight layout (bfloat16, tensor-core path).  The model's matrices are stored, and streamed by
+ * the matmul, as contiguous blocks of 128 rows x 64 columns (16 KB), in the order (row tile, column
+ * slab), zero-padded to whole blocks, so that a CTA walking along K reads one contiguous stretch of
+ * HBM.  d3_packed_weight_elems: elements of the packed form of an [n, k] matrix (0 on bad sizes).
+ * d3_pack_weight: w [device][n, k] row-major -> packed [device][d3_packed_weight_elems(n, k)].
+ * d3_op_linear_packed: d3_op_linear with the weights in that form. */
+int64_t d3_packed_weight_elems(int32_t n, int32_t k);
+int d3_pack_weight(d3_ctx *ctx, const void *w, int32_t n, int32_t k, void *packed);
+int d3_op_linear_packed(d3_ctx *ctx, const void *x, const void *w_packed, void *y, int32_t m, int32_t n, int32_t k,
+                        int32_t epilogue, int32_t splits);
 int d3_op_lm_head_stats(d3_ctx *ctx, const void *x, const void *w, int32_t m, int32_t vocab, int32_t k,
                         float scale, int32_t mask_id, float *conf, float *entropy, int32_t *argmax);
 int d3_op_attention(d3_ctx *ctx, const void *q, int32_t layer, int32_t bs, int32_t rows,
@@ -228,6 +238,12 @@ int d3_lm_head_stats_static(const void *x, const void *w, int32_t dtype, int32_t
  * every kernel fully serialized (for timing kernels in isolation and for debugging); results are
  * identical either way. */
 int d3_set_overlap(d3_ctx *ctx, int on);
+
+/* Matmul tuning overrides for measurement sweeps: shared-memory ring per CTA in KB (0 = default:
+ * about 100 KB for matmuls of up to 128 rows, 200 KB otherwise; at most 200) and CTAs per SM that the
+ * (tile, K slab) units are dealt to (0 = default 1; at most 3).  Results do not change beyond the
+ * order of fp32 partial sums. */
+int d3_set_matmul_tuning(d3_ctx *ctx, int32_t ring_kb, int32_t ctas_per_sm);
 
 /* Per-class kernel timing for measurement runs.  While enabled, every launch of the forward pass is
  * bracketed by a CUDA event pair on the context's stream; d3_profile_read waits for the stream and

@@ -26,8 +26,8 @@ D3_GEMM_AUTO, D3_GEMM_SIMT = 0, 1
 EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
-    "d3_get_state", "d3_set_state", "d3_op_linear", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
+    "d3_get_state", "d3_set_state", "d3_op_linear", "d3_packed_weight_elems", "d3_pack_weight", "d3_op_linear_packed", "d3_op_lm_head_stats", "d3_op_attention",
+    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_device_bytes",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
 
@@ -219,6 +219,27 @@ def d3_op_linear(ctx, x: torch.Tensor, w: torch.Tensor, y: torch.Tensor, epilogu
                                    C.c_int32(k), C.c_int32(epilogue), C.c_int32(splits)))
 
 
+def d3_packed_weight_elems(n: int, k: int) -> int:
+    f = lib().d3_packed_weight_elems
+    f.restype = C.c_int64
+    return int(f(C.c_int32(n), C.c_int32(k)))
+
+
+def d3_pack_weight(ctx, w: torch.Tensor, packed: torch.Tensor) -> None:
+    n, k = w.shape
+    if packed.numel() < d3_packed_weight_elems(n, k):
+        raise ValueError("packed buffer too small")
+    _check(ctx, lib().d3_pack_weight(ctx, _ptr(_dev(w, torch.bfloat16)), C.c_int32(n), C.c_int32(k),
+                                     _ptr(_dev(packed, torch.bfloat16))))
+
+
+def d3_op_linear_packed(ctx, x: torch.Tensor, w_packed: torch.Tensor, y: torch.Tensor, n: int, epilogue: int,
+                        splits: int = 0) -> None:
+    m, k = x.shape
+    _check(ctx, lib().d3_op_linear_packed(ctx, _ptr(_dev(x)), _ptr(_dev(w_packed)), _ptr(_dev(y)), C.c_int32(m),
+                                          C.c_int32(n), C.c_int32(k), C.c_int32(epilogue), C.c_int32(splits)))
+
+
 def d3_op_lm_head_stats(ctx, x: torch.Tensor, w: torch.Tensor, scale: float, mask_id: int, conf: torch.Tensor,
                         entropy: torch.Tensor, argmax: torch.Tensor) -> None:
     m, k = x.shape
@@ -280,6 +301,10 @@ PROF_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_head", 
 
 def d3_set_overlap(ctx, on: bool) -> None:
     _check(ctx, lib().d3_set_overlap(ctx, C.c_int(1 if on else 0)))
+
+
+def d3_set_matmul_tuning(ctx, ring_kb: int = 0, ctas_per_sm: int = 0) -> None:
+    _check(ctx, lib().d3_set_matmul_tuning(ctx, C.c_int32(ring_kb), C.c_int32(ctas_per_sm)))
 
 
 def d3_profile_enable(ctx, on: bool) -> None:

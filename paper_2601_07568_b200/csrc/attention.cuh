@@ -101,8 +101,10 @@ __global__ void __launch_bounds__(THREADS) attn_simt_kernel(const T* __restrict_
 // the two small products per tile run on mma.sync m16n8k16 with fragments read by ldmatrix, and the
 // softmax stays in registers.  One CTA = one (sequence, kv head, query tile, key split); a query
 // tile packs the rows of all query heads that share the kv head (GQA): packed row pr = head_in_group
-// * rows_per_seq + r.  With several key splits every CTA writes an unnormalised partial (O, m, l)
-// and the last one to arrive (atomic counter, nobody waits) merges them in split order.
+// * rows_per_seq + r.  With several key splits (at most 8) the CTAs of one query tile form a
+// thread-block cluster: each leaves its unnormalised partial (O, m, l) in its own shared memory,
+// and after a cluster barrier every CTA merges a slice of the rows, reading its peers' partials
+// through distributed shared memory in split order; nothing goes through global memory.
 #include "ptx_sm100.cuh"
 
 namespace d3 {
@@ -119,10 +121,8 @@ struct AttnTcParams {
   RowMap rm;
   int hq, hkv, max_seq;
   long long k_row0, v_row0;  // first row of this layer's K / V plane in the cache tensor map
-  int n_splits;
+  int n_splits;      // = gridDim.z = cluster size along z (1..8)
   float scale_log2;  // 1/sqrt(d_head) * log2(e)
-  float* partial;    // [(pair * q_tiles + qt) * n_splits + split][BM][PART_LD]
-  int* counters;     // [(pair * q_tiles + qt)], zero on entry and on exit
   uint32_t* error_word;
 };
 
@@ -157,7 +157,6 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + TC_STAGES * STAGE_BYTES);
   uint64_t* empty_bar = full_bar + TC_STAGES;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + TC_STAGES);
-  int* last_flag = const_cast<int*>(abort_flag) + 1;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g4 = lane >> 2, t4 = lane & 3;
@@ -173,7 +172,6 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
       ptx::mbar_init(&empty_bar[s], NW);
     }
     *abort_flag = 0;
-    *last_flag = 0;
     ptx::fence_barrier_init();
   }
   __syncthreads();
@@ -356,11 +354,11 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     }
     return;
   }
-  // ---- several key splits: write the partial, the last CTA to arrive merges
-  const int tile_id = pair * gridDim.x + qt;
-  float* part = p.partial + (static_cast<size_t>(tile_id) * p.n_splits + split) * BM * PART_LD;
+  // ---- several key splits: partials stay in shared memory, merged across the cluster
+  __syncthreads();  // every warp is done with the K/V stages: their memory now holds the partial
+  float* red = reinterpret_cast<float*>(smem);  // [BM][PART_LD]
   {
-    float* r_lo = part + static_cast<size_t>(warp * 16 + g4) * PART_LD;
+    float* r_lo = red + static_cast<size_t>(warp * 16 + g4) * PART_LD;
     float* r_hi = r_lo + 8 * PART_LD;
 #pragma unroll
     for (int n = 0; n < 16; ++n) {
@@ -372,38 +370,46 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
       r_hi[128] = m_hi; r_hi[129] = l_hi;
     }
   }
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const int old = atomicAdd(&p.counters[tile_id], 1);
-    const int last = (old == p.n_splits - 1) ? 1 : 0;
-    if (last) p.counters[tile_id] = 0;
-    *last_flag = last;
-    __threadfence();
-  }
-  __syncthreads();
-  if (!*last_flag) return;
-  const float* base = p.partial + static_cast<size_t>(tile_id) * p.n_splits * BM * PART_LD;
-  for (int e = threadIdx.x; e < BM * 32; e += NW * 32) {  // one thread per (row, 4 output dims)
-    const int row = e >> 5, c4 = (e & 31) * 4;
-    const int pr = qt * BM + row;
-    if (pr >= R || (pr % rps) >= n_valid) continue;
-    float M = -INFINITY;
-    for (int s2 = 0; s2 < p.n_splits; ++s2) M = fmaxf(M, __ldcg(base + (static_cast<size_t>(s2) * BM + row) * PART_LD + 128));
-    float L = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int s2 = 0; s2 < p.n_splits; ++s2) {
-      const float* pr_s = base + (static_cast<size_t>(s2) * BM + row) * PART_LD;
-      const float ls = __ldcg(pr_s + 129);
-      if (ls == 0.f) continue;
-      const float w = exp2f(__ldcg(pr_s + 128) - M);
-      const float4 v = __ldcg(reinterpret_cast<const float4*>(pr_s + c4));
-      L += w * ls;
-      a0 += w * v.x; a1 += w * v.y; a2 += w * v.z; a3 += w * v.w;
+  ptx::cluster_sync_all();
+  {
+    const int S = p.n_splits;
+    const int rank = static_cast<int>(ptx::cluster_ctarank());
+    const int rpr = (BM + S - 1) / S;  // rows per CTA of the cluster
+    const int row0 = rank * rpr, row1 = min(BM, row0 + rpr);
+    const uint32_t red_addr = ptx::smem_u32(red);
+    for (int e = threadIdx.x; e < (row1 - row0) * 32; e += NW * 32) {  // one thread per (row, 4 output dims)
+      const int row = row0 + (e >> 5), c4 = (e & 31) * 4;
+      const int pr = qt * BM + row;
+      if (pr >= R || (pr % rps) >= n_valid) continue;
+      const uint32_t off = static_cast<uint32_t>(row * PART_LD) * 4u;
+      float ms[8], ls[8];
+      float4 vs[8];
+      float M = -INFINITY;
+#pragma unroll
+      for (int s2 = 0; s2 < 8; ++s2) {
+        if (s2 < S) {
+          const uint32_t a = ptx::map_to_cta(red_addr + off, static_cast<uint32_t>(s2));
+          ms[s2] = ptx::ld_cluster_f(a + 128 * 4);
+          ls[s2] = ptx::ld_cluster_f(a + 129 * 4);
+          vs[s2] = ptx::ld_cluster_f4(a + c4 * 4);
+          M = fmaxf(M, ms[s2]);
+        }
+      }
+      float L = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+      for (int s2 = 0; s2 < 8; ++s2) {
+        if (s2 < S && ls[s2] != 0.f) {
+          const float w = exp2f(ms[s2] - M);
+          L += w * ls[s2];
+          a0 += w * vs[s2].x; a1 += w * vs[s2].y; a2 += w * vs[s2].z; a3 += w * vs[s2].w;
+        }
+      }
+      const float inv = 1.0f / L;
+      uint2 o2 = make_uint2(pack_bf16(a0 * inv, a1 * inv), pack_bf16(a2 * inv, a3 * inv));
+      *reinterpret_cast<uint2*>(out_ptr(pr) + c4) = o2;
     }
-    const float inv = 1.0f / L;
-    uint2 o2 = make_uint2(pack_bf16(a0 * inv, a1 * inv), pack_bf16(a2 * inv, a3 * inv));
-    *reinterpret_cast<uint2*>(out_ptr(pr) + c4) = o2;
   }
+  ptx::cluster_sync_all();  // no CTA may leave while a peer still reads its partial
 }
 
 inline size_t attn_tc_smem_bytes() { return 1024 + TC_STAGES * STAGE_BYTES + 2 * TC_STAGES * 8 + 64; }

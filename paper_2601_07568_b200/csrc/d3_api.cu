@@ -31,6 +31,7 @@ struct d3_ctx {
   bool is_bf16 = false;
   bool use_tc = false;
   bool fuse_qkv = false;
+  bool w_tiled = false;  // model matrices stored as contiguous 128 x 64 blocks (tensor-core path)
   size_t esz = 4;
   int n_sms = 148;
   // weights (context dtype), repacked
@@ -60,10 +61,6 @@ struct d3_ctx {
   // tensor-core attention (bf16, d_head 128)
   bool attn_tc = false;
   CUtensorMap kv_tmap{};
-  float* attn_partial = nullptr;
-  size_t attn_partial_floats = 0;
-  int* attn_counters = nullptr;
-  int n_attn_counters = 0;
   float* partial = nullptr;
   size_t partial_slots = 0;  // capacity in (tile, split) slots of 128*128 floats
   int* tile_count = nullptr;
@@ -82,6 +79,8 @@ struct d3_ctx {
   bool prof_on = false;
   bool pdl = true;           // programmatic dependent launch between the kernels of a forward
   int* skip_flag = nullptr;  // device flag: non-zero turns the forward's kernels into no-ops
+  int tune_producers = 0;
+  int tune_ring_kb = 0, tune_ctas_per_sm = 0;  // matmul tuning overrides (0 = default)
   struct ProfPair { cudaEvent_t a, b; int cls; };
   std::vector<ProfPair> prof_pool;
   size_t prof_used = 0;
@@ -284,7 +283,7 @@ int dispatch_tc(d3_ctx* c, int epi, const CUtensorMap* tx, const CUtensorMap* tw
 // One persistent CTA per SM; the (tile, K slab) units are dealt out evenly (see gemm_tc.cuh).
 // `ctas_hint` > 0 forces the grid size (tests use it to move the segment borders around).
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
-                  int ctas_hint, const QkvExtra* qx) {
+                  int ctas_hint, const QkvExtra* qx, int w_tiled) {
   constexpr int BLOCK_N = 128;
   const int m_tiles = (M + 127) / 128, n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_chunks = (K + 63) / 64;
@@ -297,13 +296,15 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   p.m_tiles = m_tiles; p.n_tiles = n_tiles; p.k_chunks = k_chunks;
   p.total_units = tiles * k_chunks;
   // at least eight K slabs per CTA: shorter ranges only add partial tiles
-  long long n_ctas = std::min<long long>(c->n_sms, std::max<long long>(1, p.total_units / 8));
+  // skinny matmuls: two CTAs per SM (two sets of TMA-issuing threads keep more loads in flight)
+  const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : (M <= 128 ? 2 : 1);
+  long long n_ctas = std::min<long long>(static_cast<long long>(c->n_sms) * per_sm, std::max<long long>(1, p.total_units / 8));
   if (ctas_hint > 0) n_ctas = std::min<long long>(ctas_hint, p.total_units);
   n_ctas = std::min<long long>(n_ctas, std::min<long long>(tc::MAX_CTAS, static_cast<long long>(c->partial_slots / 2)));
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + BLOCK_N * 128;
   // skinny matmuls are bound by HBM: keep the ring near 100 KB so that the next kernel's CTAs fit
   // beside this one's and start streaming their weights; wide ones get all of shared memory
-  const size_t ring = (M <= 128 ? 100 : 200) * 1024;
+  const size_t ring = (c->tune_ring_kb > 0 ? c->tune_ring_kb : (M <= 128 ? 100 : 200)) * 1024;
   int stages = static_cast<int>(ring / stage_bytes);
   stages = std::max(2, std::min(stages, 16));
   p.stages = stages;
@@ -311,6 +312,8 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   p.tile_count = c->tile_count;
   p.error_word = c->error_word;
   p.skip_flag = c->skip_flag;
+  p.w_tiled = w_tiled;
+  p.n_producers = c->tune_producers > 0 ? c->tune_producers : 2;
   p.ep = ep;
   if (qx) {
     p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
@@ -320,7 +323,14 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   }
   const CUtensorMap *tx, *tw;
   TRY(get_tmap(c, X, M, K, a_rows, &tx));
-  TRY(get_tmap(c, W, N, K, BLOCK_N, &tw));
+  if (w_tiled) {
+    if ((reinterpret_cast<uintptr_t>(W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
+    p.w_packed = static_cast<const bf16*>(W);
+    p.w_blocks = static_cast<long long>((N + 127) / 128) * k_chunks;
+    tw = tx;  // unused by the kernel in this mode
+  } else {
+    TRY(get_tmap(c, W, N, K, BLOCK_N, &tw));
+  }
   const size_t smem = tc::gemm_tc_smem_bytes(a_rows, BLOCK_N, stages);
   return dispatch_tc<BLOCK_N>(c, epi, tx, tw, p, static_cast<int>(n_ctas), smem);
 }
@@ -343,10 +353,10 @@ int run_linear_simt(d3_ctx* c, const void* X, const void* W, int M, int N, int K
 }
 
 int run_linear(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
-               int splits_hint = 0, const QkvExtra* qx = nullptr, int cls = D3_PROF_GEMM_OTHER) {
+               int splits_hint = 0, const QkvExtra* qx = nullptr, int cls = D3_PROF_GEMM_OTHER, int w_tiled = 0) {
   if (M <= 0 || N <= 0 || K <= 0) return D3_OK;
   ProfScope ps(c, cls);
-  if (c->use_tc) return run_linear_tc(c, X, W, M, N, K, epi, ep, splits_hint, qx);
+  if (c->use_tc) return run_linear_tc(c, X, W, M, N, K, epi, ep, splits_hint, qx, w_tiled);
   if (c->is_bf16) return run_linear_simt<bf16>(c, X, W, M, N, K, epi, ep);
   return run_linear_simt<float>(c, X, W, M, N, K, epi, ep);
 }
@@ -381,7 +391,28 @@ int launch_attn_tc(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
     CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::attn_tc_smem_bytes())));
     attr_set = true;
   }
-  CUDA_TRY(c, launch_pdl(c, kern, grid, dim3(NW * 32), attn::attn_tc_smem_bytes(), c->kv_tmap, p));
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(NW * 32);
+  cfg.dynamicSmemBytes = attn::attn_tc_smem_bytes();
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (grid.z > 1) {  // the key splits of one query tile form a cluster
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 1;
+    at[na].val.clusterDim.y = 1;
+    at[na].val.clusterDim.z = grid.z;
+    ++na;
+  }
+  if (c->pdl && !c->prof_on) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = na;
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, c->kv_tmap, p));
   LAUNCHED(c, "attn_tc_kernel");
   return D3_OK;
 }
@@ -391,17 +422,14 @@ int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMa
   const int group = g.n_q_heads / g.n_kv_heads;
   const int R = group * rm.rows_per_seq;
   const int nw = R <= 32 ? 2 : (R <= 64 ? 4 : 8);
-  const int bm = nw * 16;
-  const int q_tiles = (R + bm - 1) / bm;
+  const int q_tiles = (R + nw * 16 - 1) / (nw * 16);
   const int pairs = rm.bs * g.n_kv_heads;
   int splits = 1;
   if (q_tiles <= 2) {  // decode-sized: split the keys when (sequence, kv head) pairs alone leave SMs idle
     const int max_tiles = (g.max_seq + attn::KT - 1) / attn::KT;
     splits = (2 * c->n_sms + pairs * q_tiles - 1) / (pairs * q_tiles);
     splits = std::min(splits, std::max(1, max_tiles / 2));
-    splits = std::max(1, std::min(splits, 16));
-    const size_t need = static_cast<size_t>(pairs) * q_tiles * splits * bm * attn::PART_LD;
-    if (need > c->attn_partial_floats || pairs * q_tiles > c->n_attn_counters) splits = 1;
+    splits = std::max(1, std::min(splits, 8));  // one cluster per query tile: at most 8 CTAs
   }
   attn::AttnTcParams p{};
   p.q = static_cast<const bf16*>(q);
@@ -413,8 +441,6 @@ int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMa
   p.v_row0 = (static_cast<long long>(layer) * 2 + 1) * plane_rows;
   p.n_splits = splits;
   p.scale_log2 = 1.4426950408889634f / std::sqrt(static_cast<float>(g.d_head));
-  p.partial = c->attn_partial;
-  p.counters = c->attn_counters;
   p.error_word = c->error_word;
   dim3 grid(q_tiles, pairs, splits);
   switch (nw) {
@@ -483,11 +509,11 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
       EpiParams ep;
       ep.y = c->q; ep.ldy = nq;
       QkvExtra qx{rm, k_plane(c, l), v_plane(c, l)};
-      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_QKV, ep, 0, &qx, D3_PROF_GEMM_QKV));
+      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_QKV, ep, 0, &qx, D3_PROF_GEMM_QKV, c->w_tiled));
     } else {
       EpiParams ep;
       ep.y = c->qkv_f32; ep.ldy = nq + 2 * nkv;
-      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_QKV));
+      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_QKV, c->w_tiled));
       ProfScope ps(c, D3_PROF_OTHER);
       if (c->is_bf16)
         rope_kv_kernel<bf16><<<M, 256, 0, c->stream>>>(c->qkv_f32, static_cast<bf16*>(c->q), static_cast<bf16*>(k_plane(c, l)), static_cast<bf16*>(v_plane(c, l)), c->rope_cos, c->rope_sin, rm, g.n_q_heads, g.n_kv_heads, g.d_head, g.max_seq, c->error_word);
@@ -499,18 +525,18 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     {
       EpiParams ep;
       ep.y = c->x; ep.ldy = d;
-      TRY(run_linear(c, c->o, c->wo[l], M, d, nq, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_O));
+      TRY(run_linear(c, c->o, c->wo[l], M, d, nq, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_O, c->w_tiled));
     }
     TRY(run_rmsnorm(c, c->x, c->ffn_norm[l], c->xn, M));
     {
       EpiParams ep;
       ep.y = c->h; ep.ldy = f;
-      TRY(run_linear(c, c->xn, c->wgu[l], M, 2 * f, d, EPI_SWIGLU, ep, 0, nullptr, D3_PROF_GEMM_GATE_UP));
+      TRY(run_linear(c, c->xn, c->wgu[l], M, 2 * f, d, EPI_SWIGLU, ep, 0, nullptr, D3_PROF_GEMM_GATE_UP, c->w_tiled));
     }
     {
       EpiParams ep;
       ep.y = c->x; ep.ldy = d;
-      TRY(run_linear(c, c->h, c->wd[l], M, d, f, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_DOWN));
+      TRY(run_linear(c, c->h, c->wd[l], M, d, f, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_DOWN, c->w_tiled));
     }
     if (l == c->tap_layer && M <= c->tap_rows)
       CUDA_TRY(c, cudaMemcpyAsync(c->tap_out, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
@@ -521,12 +547,12 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     const int n_tiles = (g.vocab + 127) / 128;
     EpiParams ep;
     ep.scale = g.logit_scale; ep.mask_id = g.mask_id; ep.stat_part = c->stat_part; ep.n_tiles = n_tiles;
-    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_STATS, ep, 0, nullptr, D3_PROF_GEMM_HEAD));
+    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_STATS, ep, 0, nullptr, D3_PROF_GEMM_HEAD, c->w_tiled));
     TRY(run_stats_merge(c, M, n_tiles, c->conf, c->ent, c->argmax));
   } else {
     EpiParams ep;
     ep.y = logits; ep.ldy = g.vocab; ep.scale = g.logit_scale;
-    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_HEAD));
+    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_HEAD, c->w_tiled));
   }
   return D3_OK;
 }
@@ -571,6 +597,7 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   c->esz = c->is_bf16 ? 2 : 4;
   c->use_tc = c->is_bf16 && g.gemm_impl == D3_GEMM_AUTO;
   c->fuse_qkv = c->use_tc && g.d_head == 128;
+  c->w_tiled = c->use_tc;
   auto bail = [&](int rc) {
     d3_destroy(c);
     return rc;
@@ -626,15 +653,6 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
       int rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, attn::KT, &tm);
       if (rc_ != D3_OK) return bail(rc_);
       c->kv_tmap = *tm;
-      // partial (O, m, l) of every (sequence, kv head, query tile, key split) of a decode forward
-      const int group = g.n_q_heads / g.n_kv_heads;
-      const int R = group * g.block;
-      const int bm = R <= 32 ? 32 : (R <= 64 ? 64 : 128);
-      const size_t tiles = static_cast<size_t>(g.max_batch) * g.n_kv_heads * ((R + bm - 1) / bm);
-      c->attn_partial_floats = (tiles + 4 * static_cast<size_t>(c->n_sms)) * bm * attn::PART_LD;
-      A_(c->attn_partial, c->attn_partial_floats * sizeof(float));
-      c->n_attn_counters = static_cast<int>(tiles);
-      A_(c->attn_counters, sizeof(int) * tiles);
       c->attn_tc = true;
     }
   }
@@ -706,6 +724,25 @@ int load_gain(d3_ctx* c, float** dst, const void* src, int src_is_device, void* 
 }
 }  // namespace
 
+// Elements of the stored form of an [n, k] matrix: row-major as given, or padded to whole
+// 128 x 64 blocks for the tiled layout.
+static size_t stored_elems(const d3_ctx* c, size_t n, size_t k) {
+  if (!c->w_tiled) return n * k;
+  return ((n + 127) / 128) * ((k + 63) / 64) * 128 * 64;
+}
+
+namespace {
+// Final store of one assembled row-major matrix `rm` [n, k]: tiled blocks on the tensor-core path,
+// a plain copy otherwise (then `rm` already is the final buffer and nothing is done).
+int finish_matrix(d3_ctx* c, const void* rm, void* dst, size_t n, size_t k) {
+  if (!c->w_tiled) return D3_OK;
+  dim3 grid(static_cast<unsigned>((k + 63) / 64), static_cast<unsigned>((n + 127) / 128));
+  pack_tiled_kernel<<<grid, 256, 0, c->stream>>>(static_cast<const bf16*>(rm), static_cast<bf16*>(dst), static_cast<int>(n),
+                                                 static_cast<int>(k));
+  return check_launch(c, "pack_tiled_kernel");
+}
+}  // namespace
+
 extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device) {
   if (!c) return D3_ERR_INVALID_ARG;
   if (!w || !w->tok_emb || !w->lm_head || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up || !w->w_down)
@@ -718,30 +755,41 @@ extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device
       return fail(c, D3_ERR_INVALID_ARG, "null per-layer weight pointer");
   if (!c->tok_emb) {
     ALLOC(c, c->tok_emb, V * d * e);
-    ALLOC(c, c->lm_head, V * d * e);
+    ALLOC(c, c->lm_head, stored_elems(c, V, d) * e);
     c->wqkv.assign(g.n_layers, nullptr); c->wo.assign(g.n_layers, nullptr);
     c->wgu.assign(g.n_layers, nullptr); c->wd.assign(g.n_layers, nullptr);
     c->attn_norm.assign(g.n_layers, nullptr); c->ffn_norm.assign(g.n_layers, nullptr);
     for (int l = 0; l < g.n_layers; ++l) {
-      ALLOC(c, c->wqkv[l], (nq + 2 * nkv) * d * e);
-      ALLOC(c, c->wo[l], d * nq * e);
-      ALLOC(c, c->wgu[l], 2 * f * d * e);
-      ALLOC(c, c->wd[l], d * f * e);
+      ALLOC(c, c->wqkv[l], stored_elems(c, nq + 2 * nkv, d) * e);
+      ALLOC(c, c->wo[l], stored_elems(c, d, nq) * e);
+      ALLOC(c, c->wgu[l], stored_elems(c, 2 * f, d) * e);
+      ALLOC(c, c->wd[l], stored_elems(c, d, f) * e);
     }
   }
-  // staging for gate / up (interleaved on the device) and gains
-  void *tg = nullptr, *tu = nullptr, *tgain = nullptr;
-  CUDA_TRY(c, cudaMalloc(&tg, std::max(f, nq) * d * e));
-  CUDA_TRY(c, cudaMalloc(&tu, f * d * e));
-  CUDA_TRY(c, cudaMalloc(&tgain, d * e));
+  // Staging: tg / tu take one uploaded source matrix each; on the tiled path `rm` holds the
+  // assembled row-major matrix (RoPE-pair permuted q/k rows + v, interleaved gate/up, or a matrix as
+  // given) before it is cut into blocks; otherwise matrices are assembled in place.
+  void *tg = nullptr, *tu = nullptr, *tgain = nullptr, *rm = nullptr;
+  const size_t rm_elems = std::max(std::max(V * d, 2 * f * d), std::max((nq + 2 * nkv) * d, d * nq));
+  cudaError_t ea = cudaMalloc(&tg, std::max(f, nq) * d * e);
+  if (ea == cudaSuccess) ea = cudaMalloc(&tu, f * d * e);
+  if (ea == cudaSuccess) ea = cudaMalloc(&tgain, d * e);
+  if (ea == cudaSuccess && c->w_tiled) ea = cudaMalloc(&rm, rm_elems * e);
+  if (ea != cudaSuccess) {
+    (void)cudaGetLastError();
+    cudaFree(tg); cudaFree(tu); cudaFree(tgain); cudaFree(rm);
+    return fail(c, D3_ERR_OOM, std::string("staging buffers for the weight load: ") + cudaGetErrorString(ea));
+  }
   int rc = D3_OK;
   auto step = [&](int r) { if (rc == D3_OK) rc = r; };
+  auto target = [&](void* final_buf) { return c->w_tiled ? rm : final_buf; };
   step(upload(c, c->tok_emb, w->tok_emb, V * d * e, src_is_device));
-  step(upload(c, c->lm_head, w->lm_head, V * d * e, src_is_device));
+  step(upload(c, target(c->lm_head), w->lm_head, V * d * e, src_is_device));
+  step(finish_matrix(c, rm, c->lm_head, V, d));
   step(load_gain(c, &c->final_norm, w->final_norm, src_is_device, tgain));
   for (int l = 0; l < g.n_layers && rc == D3_OK; ++l) {
-    char* qkv = static_cast<char*>(c->wqkv[l]);
-    // q and k rows go through the staging buffer and are packed as RoPE pairs
+    // ---- q, k (rows permuted so that each RoPE pair of a head is adjacent) and v
+    char* qkv = static_cast<char*>(target(c->wqkv[l]));
     for (int which = 0; which < 2 && rc == D3_OK; ++which) {
       const size_t rows = which == 0 ? nq : nkv;
       char* dst = qkv + (which == 0 ? 0 : nq * d * e);
@@ -754,23 +802,30 @@ extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device
       step(check_launch(c, "pack_rope_rows_kernel"));
     }
     step(upload(c, qkv + (nq + nkv) * d * e, w->wv[l], nkv * d * e, src_is_device));
-    step(upload(c, c->wo[l], w->wo[l], d * nq * e, src_is_device));
-    step(upload(c, c->wd[l], w->w_down[l], d * f * e, src_is_device));
+    step(finish_matrix(c, rm, c->wqkv[l], nq + 2 * nkv, d));
+    // ---- o, down: as given
+    step(upload(c, target(c->wo[l]), w->wo[l], d * nq * e, src_is_device));
+    step(finish_matrix(c, rm, c->wo[l], d, nq));
+    step(upload(c, target(c->wd[l]), w->w_down[l], d * f * e, src_is_device));
+    step(finish_matrix(c, rm, c->wd[l], d, f));
+    // ---- gate / up: rows interleaved
     step(upload(c, tg, w->w_gate[l], f * d * e, src_is_device));
     step(upload(c, tu, w->w_up[l], f * d * e, src_is_device));
     if (rc == D3_OK) {
+      void* gu = target(c->wgu[l]);
       if (c->is_bf16)
-        interleave_gate_up_kernel<bf16><<<static_cast<unsigned>(2 * f), 128, 0, c->stream>>>(static_cast<const bf16*>(tg), static_cast<const bf16*>(tu), static_cast<bf16*>(c->wgu[l]), g.d_ffn, g.d_model);
+        interleave_gate_up_kernel<bf16><<<static_cast<unsigned>(2 * f), 128, 0, c->stream>>>(static_cast<const bf16*>(tg), static_cast<const bf16*>(tu), static_cast<bf16*>(gu), g.d_ffn, g.d_model);
       else
-        interleave_gate_up_kernel<float><<<static_cast<unsigned>(2 * f), 128, 0, c->stream>>>(static_cast<const float*>(tg), static_cast<const float*>(tu), static_cast<float*>(c->wgu[l]), g.d_ffn, g.d_model);
+        interleave_gate_up_kernel<float><<<static_cast<unsigned>(2 * f), 128, 0, c->stream>>>(static_cast<const float*>(tg), static_cast<const float*>(tu), static_cast<float*>(gu), g.d_ffn, g.d_model);
       step(check_launch(c, "interleave_gate_up_kernel"));
     }
+    step(finish_matrix(c, rm, c->wgu[l], 2 * f, d));
     step(load_gain(c, &c->attn_norm[l], w->attn_norm ? w->attn_norm[l] : nullptr, src_is_device, tgain));
     step(load_gain(c, &c->ffn_norm[l], w->ffn_norm ? w->ffn_norm[l] : nullptr, src_is_device, tgain));
-    // the staging buffers are reused by the next layer: the copies above are stream-ordered
+    // the staging buffers are reused by the next matrix: everything above is stream-ordered
   }
   cudaError_t es = cudaStreamSynchronize(c->stream);
-  cudaFree(tg); cudaFree(tu); cudaFree(tgain);
+  cudaFree(tg); cudaFree(tu); cudaFree(tgain); cudaFree(rm);
   if (rc != D3_OK) return rc;
   if (es != cudaSuccess) return fail(c, D3_ERR_CUDA, std::string("sync after weight load: ") + cudaGetErrorString(es));
   c->weights_loaded = true;
@@ -948,6 +1003,34 @@ extern "C" int d3_op_linear(d3_ctx* c, const void* x, const void* w, void* y, in
   return run_linear(c, x, w, m, n, k, epilogue, ep, splits);
 }
 
+extern "C" int64_t d3_packed_weight_elems(int32_t n, int32_t k) {
+  if (n <= 0 || k <= 0) return 0;
+  return static_cast<int64_t>((n + 127) / 128) * ((k + 63) / 64) * 128 * 64;
+}
+
+extern "C" int d3_pack_weight(d3_ctx* c, const void* w, int32_t n, int32_t k, void* packed) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!w || !packed || n <= 0 || k <= 0) return fail(c, D3_ERR_INVALID_ARG, "bad pack_weight arguments");
+  if (!c->is_bf16) return fail(c, D3_ERR_UNSUPPORTED, "the tiled layout exists for bfloat16 only");
+  dim3 grid(static_cast<unsigned>((k + 63) / 64), static_cast<unsigned>((n + 127) / 128));
+  pack_tiled_kernel<<<grid, 256, 0, c->stream>>>(static_cast<const bf16*>(w), static_cast<bf16*>(packed), n, k);
+  LAUNCHED(c, "pack_tiled_kernel");
+  return D3_OK;
+}
+
+extern "C" int d3_op_linear_packed(d3_ctx* c, const void* x, const void* w_packed, void* y, int32_t m, int32_t n,
+                                   int32_t k, int32_t epilogue, int32_t splits) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!x || !w_packed || !y || m <= 0 || n <= 0 || k <= 0 || epilogue < 0 || epilogue > 3)
+    return fail(c, D3_ERR_INVALID_ARG, "bad op_linear_packed arguments");
+  if (!c->use_tc) return fail(c, D3_ERR_UNSUPPORTED, "the tiled layout is read by the tensor-core matmul only");
+  if (epilogue == EPI_SWIGLU && n % 2 != 0) return fail(c, D3_ERR_SHAPE, "SwiGLU epilogue needs an even n");
+  EpiParams ep;
+  ep.y = y;
+  ep.ldy = epilogue == EPI_SWIGLU ? n / 2 : n;
+  return run_linear(c, x, w_packed, m, n, k, epilogue, ep, splits, nullptr, D3_PROF_GEMM_OTHER, 1);
+}
+
 extern "C" int d3_op_lm_head_stats(d3_ctx* c, const void* x, const void* w, int32_t m, int32_t vocab, int32_t k,
                                    float scale, int32_t mask_id, float* conf, float* entropy, int32_t* argmax) {
   if (!c) return D3_ERR_INVALID_ARG;
@@ -1011,6 +1094,13 @@ extern "C" int d3_get_error_word(d3_ctx* c, uint32_t* word) {
   if (!c || !word) return D3_ERR_INVALID_ARG;
   CUDA_TRY(c, cudaMemcpyAsync(word, c->error_word, sizeof(uint32_t), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  return D3_OK;
+}
+extern "C" int d3_set_matmul_tuning(d3_ctx* c, int32_t ring_kb, int32_t ctas_per_sm) {
+  if (!c || ring_kb < 0 || (ring_kb & 0xffff) > 200 || ctas_per_sm < 0 || ctas_per_sm > 3) return D3_ERR_INVALID_ARG;
+  c->tune_producers = ring_kb >> 16;  // experiment: bits 16.. of ring_kb select the number of producer warps
+  c->tune_ring_kb = ring_kb & 0xffff;
+  c->tune_ctas_per_sm = ctas_per_sm;
   return D3_OK;
 }
 extern "C" int d3_set_overlap(d3_ctx* c, int on) {

@@ -35,7 +35,7 @@ namespace tc {
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;  // 64 bf16 = 128 bytes = one swizzle row
 constexpr int UMMA_K = 16;
-constexpr int NUM_THREADS = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr int NUM_THREADS = 224;  // warps 0 and 6: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr int MAX_CTAS = 512;     // upper bound of the grid (segment list of a tile lives in shared memory)
 
 struct GemmParams {
@@ -48,6 +48,11 @@ struct GemmParams {
   int* tile_count;  // arrival counters [tiles], zero on entry and on exit
   uint32_t* error_word;
   const int* skip_flag;  // optional: non-zero -> the whole launch is a no-op
+  int n_producers;       // 1 or 2 TMA-issuing warps
+  const __nv_bfloat16* w_packed;  // tiled weights (w_tiled = 1)
+  long long w_blocks;             // number of 128 x 64 blocks in w_packed
+  int w_tiled;           // 0: W row-major [N, K]; 1: W stored as contiguous [128 x 64] blocks, block (n_tile, kc) at
+                         // row (n_tile * k_chunks + kc) * 128 of a [rows, 64] array (see pack_tiled_kernel)
   EpiParams ep;
   // EPI_QKV only
   const float* rope_cos;  // [max_seq][64]
@@ -101,22 +106,37 @@ struct PartialSource {
   __device__ __forceinline__ void load(int c, float (&v)[32]) const {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = 0.f;
-    for (int s = 0; s < n_seg; ++s) {
-      const float* p = partial + (static_cast<size_t>(slots[s]) * BLOCK_N + c) * 128 + row;
+    int s = 0;
+    for (; s + 1 < n_seg; s += 2) {  // two segments' loads in flight; the sums stay in K order
+      const float* p0 = partial + (static_cast<size_t>(slots[s]) * BLOCK_N + c) * 128 + row;
+      const float* p1 = partial + (static_cast<size_t>(slots[s + 1]) * BLOCK_N + c) * 128 + row;
+      float t0[32], t1[32];
 #pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] += __ldcg(p + j * 128);
+      for (int j = 0; j < 32; ++j) t0[j] = __ldcg(p0 + j * 128);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) t1[j] = __ldcg(p1 + j * 128);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = (v[j] + t0[j]) + t1[j];
+    }
+    if (s < n_seg) {
+      const float* p0 = partial + (static_cast<size_t>(slots[s]) * BLOCK_N + c) * 128 + row;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += __ldcg(p0 + j * 128);
     }
   }
 };
 
 // All 32 threads of a warp must call this together (the TMEM loads are warp-wide); `live` only
 // predicates this thread's stores.
+// Chunks (32 columns each) c_first, c_first + c_stride, ... of the tile are handled; the TMEM path
+// takes them all (0, 1), the partial-sum path spreads them over the threads that share a row.
 template <int EPI, int BLOCK_N, typename Source>
-__device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams& p, int m, int n0, bool live) {
+__device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams& p, int m, int n0, bool live,
+                                             int c_first = 0, int c_stride = 1) {
   const int N = p.N;
   if constexpr (EPI == EPI_F32 || EPI == EPI_RESID) {
     float* y = static_cast<float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
-    for (int c = 0; c < BLOCK_N; c += 32) {
+    for (int c = 32 * c_first; c < BLOCK_N; c += 32 * c_stride) {
       if (n0 + c >= N) break;
       float v[32];
       src.load(c, v);
@@ -149,7 +169,7 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
     }
   } else if constexpr (EPI == EPI_T) {
     __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
-    for (int c = 0; c < BLOCK_N; c += 32) {
+    for (int c = 32 * c_first; c < BLOCK_N; c += 32 * c_stride) {
       if (n0 + c >= N) break;
       float v[32];
       src.load(c, v);
@@ -177,7 +197,7 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
     // packed rows of W: 2j = gate row of hidden unit j, 2j+1 = its up row; a 32-column chunk gives 16 outputs
     __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
     const int F = N / 2;
-    for (int c = 0; c < BLOCK_N; c += 32) {
+    for (int c = 32 * c_first; c < BLOCK_N; c += 32 * c_stride) {
       if (n0 + c >= N) break;
       float v[32];
       src.load(c, v);
@@ -235,7 +255,7 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
     }
     const float* cs = p.rope_cos + static_cast<size_t>(pos) * 64;
     const float* sn = p.rope_sin + static_cast<size_t>(pos) * 64;
-    for (int c = 0; c < BLOCK_N; c += 32) {
+    for (int c = 32 * c_first; c < BLOCK_N; c += 32 * c_stride) {
       const int n = n0 + c;
       if (n >= N) break;
       float v[32];
@@ -306,7 +326,7 @@ __device__ __forceinline__ int cta_of_unit(long long x, long long U, int n) {
 //   [stages x BLOCK_N x 128 B] W slabs
 //   barriers: full[stages], empty[stages], acc_full[2], acc_empty[2]; tmem address; flags; segment list
 template <int EPI, int BLOCK_N>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(NUM_THREADS, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                const GemmParams p) {
   if (p.skip_flag != nullptr && *p.skip_flag != 0) return;  // written at least one whole graph launch earlier
@@ -358,39 +378,56 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp == 0) {
-    // ---------------- TMA producer
-    if (lane == 0) {
+  if (warp == 0 || warp == 6) {
+    // ---------------- TMA producers: warp 0 alone, or warps 0 and 6 taking alternate units
+    const int n_prod = p.n_producers, pi = warp == 0 ? 0 : 1;
+    if (lane == 0 && pi < n_prod) {
       const uint32_t tx = a_stage_bytes + b_stage_bytes;
       const long long n_total = u1 - u0;
+      auto load_w = [&](int s, int tile, int kc) {
+        const int n_tile = tile / p.m_tiles;
+        uint8_t* dst = smem_b + static_cast<size_t>(s) * b_stage_bytes;
+        if (p.w_tiled) {
+#pragma unroll
+          for (int h = 0; h < BLOCK_N / 128; ++h) {  // one contiguous, pre-swizzled 16 KB block per 128 weight rows
+            const long long blk = static_cast<long long>(n_tile * (BLOCK_N / 128) + h) * KC + kc;
+            if (blk < p.w_blocks)
+              bulk_load_1d(dst + h * 128 * 128, p.w_packed + blk * (128 * 64), 128 * 128, &full_bar[s]);
+          }
+        } else {
+          tma_load_2d(dst, &tmap_w, &full_bar[s], kc * BLOCK_K, n_tile * BLOCK_N);
+        }
+      };
       const int pre = static_cast<int>(n_total < stages ? n_total : stages);
       // weights first: they do not depend on the kernels before this one
-      for (int i = 0; i < pre; ++i) {
+      for (int i = pi; i < pre; i += n_prod) {
         const long long u = u0 + i;
         const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
         mbar_arrive_expect_tx(&full_bar[i], tx);
-        tma_load_2d(smem_b + static_cast<size_t>(i) * b_stage_bytes, &tmap_w, &full_bar[i], kc * BLOCK_K,
-                    (tile / p.m_tiles) * BLOCK_N);
+        load_w(i, tile, kc);
       }
       grid_dep_wait();
-      for (int i = 0; i < pre; ++i) {
+      for (int i = pi; i < pre; i += n_prod) {
         const long long u = u0 + i;
         const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
         tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], kc * BLOCK_K,
                     (tile % p.m_tiles) * BLOCK_M);
       }
-      for (long long i = pre; i < n_total; ++i) {
+      long long i = pre;
+      while (i % n_prod != pi) ++i;
+      for (; i < n_total; i += n_prod) {
         const int s = static_cast<int>(i % stages);
         const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
         if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.error_word)) break;
         const long long u = u0 + i;
         const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
         mbar_arrive_expect_tx(&full_bar[s], tx);
-        tma_load_2d(smem_b + static_cast<size_t>(s) * b_stage_bytes, &tmap_w, &full_bar[s], kc * BLOCK_K,
-                    (tile / p.m_tiles) * BLOCK_N);
+        load_w(s, tile, kc);
         tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K,
                     (tile % p.m_tiles) * BLOCK_M);
       }
+    } else if (lane == 0) {
+      grid_dep_wait();
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer
@@ -492,9 +529,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       }
       epi_bar_sync();
       const int n_seg = *last_flag;
-      if (n_seg > 0 && warp_live) {
-        PartialSource<BLOCK_N> psrc{p.partial, seg_slots, n_seg, row};
-        run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, live);
+      if (n_seg > 0) {
+        if constexpr (EPI == EPI_STATS) {  // one statistic per (row, 128 columns): a row stays with one thread
+          if (warp_live) {
+            PartialSource<BLOCK_N> psrc{p.partial, seg_slots, n_seg, row};
+            run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, live);
+          }
+        } else {
+          // the sums come from memory, not from TMEM lanes: spread (row, 32-column chunk) pairs over
+          // all 128 threads so that a 32-row matmul does not leave the reduction to one warp
+          const int tpr = 128 / p.a_rows;  // threads per row: 4, 2, 1, 1 for 32, 64, 96, 128 rows
+          const int prow = et % p.a_rows, part = et / p.a_rows;
+          if (part < tpr) {
+            const int m2 = m_tile * BLOCK_M + prow;
+            PartialSource<BLOCK_N> psrc{p.partial, seg_slots, n_seg, prow};
+            run_epilogue<EPI, BLOCK_N>(psrc, p, m2, n0, m2 < p.M, part, tpr);
+          }
+        }
       }
       epi_bar_sync();  // seg_slots and last_flag are reused by the next segment
     }

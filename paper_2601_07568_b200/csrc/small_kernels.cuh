@@ -414,6 +414,35 @@ __global__ void interleave_gate_up_kernel(const T* __restrict__ gate, const T* _
   const T* src = ((row & 1) ? up : gate) + static_cast<size_t>(row >> 1) * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[static_cast<size_t>(row) * d + i] = src[i];
 }
+// Tiled weight layout for the tensor-core matmul: the [n, k] row-major matrix is cut into blocks of
+// 128 rows x 64 columns, each stored contiguously (16 KB, rows of 128 bytes) in the order
+// (row tile, column slab); rows and columns beyond n, k are zero.  Inside a block the eight 16-byte
+// chunks of row r are stored at positions chunk ^ (r & 7): the 128-byte shared-memory swizzle that
+// the MMA descriptors expect, applied once here, so that a plain bulk copy of the block is a ready
+// operand tile.  A CTA that walks along K of one row tile reads one contiguous stretch of memory.
+// grid (k_chunks, n_tiles), 256 threads.
+__global__ void pack_tiled_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int n, int k) {
+  const int kc = blockIdx.x, nt = blockIdx.y, k_chunks = gridDim.x;
+  uint4* out = reinterpret_cast<uint4*>(dst + (static_cast<size_t>(nt) * k_chunks + kc) * 128 * 64);
+  for (int e = threadIdx.x; e < 128 * 8; e += blockDim.x) {  // 8 chunks of 8 elements per row
+    const int r = e >> 3, ch = e & 7;
+    const int row = nt * 128 + r, col = kc * 64 + ch * 8;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (row < n) {
+      const __nv_bfloat16* s = src + static_cast<size_t>(row) * k + col;
+      if (col + 8 <= k && (k & 7) == 0) {
+        v = *reinterpret_cast<const uint4*>(s);
+      } else {
+        __nv_bfloat16 t[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) t[j] = (col + j < k) ? s[j] : __float2bfloat16_rn(0.f);
+        v = *reinterpret_cast<uint4*>(t);
+      }
+    }
+    out[r * 8 + (ch ^ (r & 7))] = v;
+  }
+}
+
 // RoPE-pair packing of q / k projection rows: inside each head, dst row 2i = src row i and dst row
 // 2i+1 = src row i + dh/2.
 template <typename T>

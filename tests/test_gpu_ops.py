@@ -74,6 +74,34 @@ def test_linear_bf16_tensor_core(ctx_bf16, m, n, k, splits):
     assert ctx_bf16.error_word() == 0
 
 
+@pytest.mark.parametrize("m,n,k", [(32, 9000, 128), (48, 200, 192), (130, 384, 256), (1, 128, 4096), (32, 4096, 4096),
+                                   (7, 100, 72), (256, 640, 1024)])
+@pytest.mark.parametrize("splits", [0, 1, 5])
+def test_linear_bf16_packed_weights(ctx_bf16, m, n, k, splits):
+    """Weights in the tiled layout (contiguous 128 x 64 blocks, zero-padded) give the same products as
+    the row-major form, ragged edges included."""
+    rng = np.random.default_rng(m * 11 + n + k)
+    xt, x = rand_bf16(rng, (m, k))
+    wt, w = rand_bf16(rng, (n, k), 0.05)
+    ref = x @ w.T
+    tol = 2e-5 * np.sqrt(k) * np.abs(ref).max() + 1e-6
+    xd, wd = xt.to(DEV), wt.to(DEV)
+    packed = torch.full((d3.d3_packed_weight_elems(n, k),), 3.0, dtype=torch.bfloat16, device=DEV)
+    d3.d3_pack_weight(ctx_bf16.ctx, wd, packed)
+    y = torch.full((m, n), 7.0, dtype=torch.float32, device=DEV)
+    d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, y, n, 0, splits)
+    assert np.max(np.abs(y.cpu().numpy() - ref)) <= tol
+    y2 = torch.full((m, n), 7.0, dtype=torch.float32, device=DEV)
+    d3.d3_op_linear(ctx_bf16.ctx, xd, wd, y2, 0, splits)
+    assert torch.equal(y, y2)  # same units, same order of sums: identical bits
+    if n % 2 == 0:
+        h = torch.zeros((m, n // 2), dtype=torch.bfloat16, device=DEV)
+        d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, h, n, 3, splits)
+        want = swiglu_ref(ref, n)
+        assert np.max(np.abs(h.float().cpu().numpy() - want)) <= 2 ** -7 * np.abs(want).max() + tol
+    assert ctx_bf16.error_word() == 0
+
+
 def test_linear_bf16_repeated_launches_keep_split_counters_clean(ctx_bf16):
     rng = np.random.default_rng(3)
     xt, x = rand_bf16(rng, (32, 1024))
