@@ -80,6 +80,7 @@ struct d3_ctx {
   bool pdl = true;           // programmatic dependent launch between the kernels of a forward
   int* skip_flag = nullptr;  // device flag: non-zero turns the forward's kernels into no-ops
   int tune_producers = 0;
+  int tune_wide_tiles = -1;  // -1: by row count; 0 / 1: force 128- / 256-column tiles
   int tune_ring_kb = 0, tune_ctas_per_sm = 0;  // matmul tuning overrides (0 = default)
   struct ProfPair { cudaEvent_t a, b; int cls; };
   std::vector<ProfPair> prof_pool;
@@ -280,11 +281,11 @@ int dispatch_tc(d3_ctx* c, int epi, const CUtensorMap* tx, const CUtensorMap* tw
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
-// One persistent CTA per SM; the (tile, K slab) units are dealt out evenly (see gemm_tc.cuh).
+// Persistent CTAs; the (tile, K slab) units are dealt out evenly (see gemm_tc.cuh).
 // `ctas_hint` > 0 forces the grid size (tests use it to move the segment borders around).
-int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
-                  int ctas_hint, const QkvExtra* qx, int w_tiled) {
-  constexpr int BLOCK_N = 128;
+template <int BLOCK_N>
+int run_linear_tc_bn(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
+                     int ctas_hint, const QkvExtra* qx, int w_tiled) {
   const int m_tiles = (M + 127) / 128, n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_chunks = (K + 63) / 64;
   const long long tiles = static_cast<long long>(m_tiles) * n_tiles;
@@ -295,15 +296,15 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   p.a_rows = a_rows;
   p.m_tiles = m_tiles; p.n_tiles = n_tiles; p.k_chunks = k_chunks;
   p.total_units = tiles * k_chunks;
-  // at least eight K slabs per CTA: shorter ranges only add partial tiles
   // skinny matmuls: two CTAs per SM (two sets of TMA-issuing threads keep more loads in flight)
   const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : (M <= 128 ? 2 : 1);
+  // at least eight K slabs per CTA: shorter ranges only add partial tiles
   long long n_ctas = std::min<long long>(static_cast<long long>(c->n_sms) * per_sm, std::max<long long>(1, p.total_units / 8));
   if (ctas_hint > 0) n_ctas = std::min<long long>(ctas_hint, p.total_units);
-  n_ctas = std::min<long long>(n_ctas, std::min<long long>(tc::MAX_CTAS, static_cast<long long>(c->partial_slots / 2)));
+  n_ctas = std::min<long long>(n_ctas, std::min<long long>(tc::MAX_CTAS, static_cast<long long>(c->partial_slots / (2 * (BLOCK_N / 128)))));
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + BLOCK_N * 128;
-  // skinny matmuls are bound by HBM: keep the ring near 100 KB so that the next kernel's CTAs fit
-  // beside this one's and start streaming their weights; wide ones get all of shared memory
+  // skinny matmuls are bound by HBM: keep the ring near 100 KB so that two CTAs (of this kernel, or
+  // of this one and the next) share an SM; wide ones get all of shared memory
   const size_t ring = (c->tune_ring_kb > 0 ? c->tune_ring_kb : (M <= 128 ? 100 : 200)) * 1024;
   int stages = static_cast<int>(ring / stage_bytes);
   stages = std::max(2, std::min(stages, 16));
@@ -333,6 +334,15 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   }
   const size_t smem = tc::gemm_tc_smem_bytes(a_rows, BLOCK_N, stages);
   return dispatch_tc<BLOCK_N>(c, epi, tx, tw, p, static_cast<int>(n_ctas), smem);
+}
+
+// Tile width: 128 columns while weight streaming dominates, 256 when
+// it is bound by the tensor pipe (from 512 rows on: a third less operand traffic per flop).
+int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
+                  int ctas_hint, const QkvExtra* qx, int w_tiled) {
+  const bool wide = c->tune_wide_tiles >= 0 ? c->tune_wide_tiles != 0 : M >= 512;
+  if (wide && N >= 256) return run_linear_tc_bn<256>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
+  return run_linear_tc_bn<128>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
 }
 
 template <typename T>
@@ -1098,7 +1108,8 @@ extern "C" int d3_get_error_word(d3_ctx* c, uint32_t* word) {
 }
 extern "C" int d3_set_matmul_tuning(d3_ctx* c, int32_t ring_kb, int32_t ctas_per_sm) {
   if (!c || ring_kb < 0 || (ring_kb & 0xffff) > 200 || ctas_per_sm < 0 || ctas_per_sm > 3) return D3_ERR_INVALID_ARG;
-  c->tune_producers = ring_kb >> 16;  // experiment: bits 16.. of ring_kb select the number of producer warps
+  c->tune_producers = (ring_kb >> 16) & 0xf;  // experiments: bits 16-19 of ring_kb = producer warps, 20-21 = tile width + 1
+  c->tune_wide_tiles = ((ring_kb >> 20) & 3) - 1;
   c->tune_ring_kb = ring_kb & 0xffff;
   c->tune_ctas_per_sm = ctas_per_sm;
   return D3_OK;

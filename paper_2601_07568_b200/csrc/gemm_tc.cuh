@@ -384,17 +384,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     if (lane == 0 && pi < n_prod) {
       const uint32_t tx = a_stage_bytes + b_stage_bytes;
       const long long n_total = u1 - u0;
+      // Arms the stage's barrier with the bytes that will arrive and issues the weight loads.
       auto load_w = [&](int s, int tile, int kc) {
         const int n_tile = tile / p.m_tiles;
         uint8_t* dst = smem_b + static_cast<size_t>(s) * b_stage_bytes;
         if (p.w_tiled) {
+          // one contiguous, pre-swizzled 16 KB block per 128 weight rows; a 256-wide tile at the
+          // ragged end of N may have only its first block (the other half of the stage keeps stale
+          // data, which lands in output columns >= N that nobody stores)
+          const long long blk0 = static_cast<long long>(n_tile * (BLOCK_N / 128)) * KC + kc;
+          int nb = 0;
 #pragma unroll
-          for (int h = 0; h < BLOCK_N / 128; ++h) {  // one contiguous, pre-swizzled 16 KB block per 128 weight rows
-            const long long blk = static_cast<long long>(n_tile * (BLOCK_N / 128) + h) * KC + kc;
-            if (blk < p.w_blocks)
-              bulk_load_1d(dst + h * 128 * 128, p.w_packed + blk * (128 * 64), 128 * 128, &full_bar[s]);
-          }
+          for (int h = 0; h < BLOCK_N / 128; ++h)
+            if (blk0 + static_cast<long long>(h) * KC < p.w_blocks) ++nb;
+          mbar_arrive_expect_tx(&full_bar[s], a_stage_bytes + static_cast<uint32_t>(nb) * 128u * 128u);
+#pragma unroll
+          for (int h = 0; h < BLOCK_N / 128; ++h)
+            if (h < nb)
+              bulk_load_1d(dst + h * 128 * 128, p.w_packed + (blk0 + static_cast<long long>(h) * KC) * (128 * 64),
+                           128 * 128, &full_bar[s]);
         } else {
+          mbar_arrive_expect_tx(&full_bar[s], tx);
           tma_load_2d(dst, &tmap_w, &full_bar[s], kc * BLOCK_K, n_tile * BLOCK_N);
         }
       };
@@ -403,7 +413,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       for (int i = pi; i < pre; i += n_prod) {
         const long long u = u0 + i;
         const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
-        mbar_arrive_expect_tx(&full_bar[i], tx);
         load_w(i, tile, kc);
       }
       grid_dep_wait();
@@ -421,7 +430,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.error_word)) break;
         const long long u = u0 + i;
         const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
-        mbar_arrive_expect_tx(&full_bar[s], tx);
         load_w(s, tile, kc);
         tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K,
                     (tile % p.m_tiles) * BLOCK_M);
