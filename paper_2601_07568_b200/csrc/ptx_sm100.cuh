@@ -42,13 +42,16 @@ __device__ __forceinline__ uint64_t global_ns() {
 // phase did not complete within WAIT_LIMIT_NS or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
                                           uint32_t* error_word) {
-  if (mbar_try_wait(bar, parity)) return true;
-  uint64_t t0 = global_ns();
+  // The common case must stay a bare try_wait loop: the clock is only read after 1024 failed
+  // polls (reading %globaltimer on every blocking wait costs more than the wait itself).
+  uint64_t t0 = 0;
   uint32_t it = 0;
   while (!mbar_try_wait(bar, parity)) {
     if ((++it & 0x3ff) == 0) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > WAIT_LIMIT_NS) {
+      const uint64_t now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > WAIT_LIMIT_NS) {
         *abort_flag = 1;
         atomicOr(error_word, ERRW_MBAR_TIMEOUT);
         return false;
@@ -61,6 +64,9 @@ __device__ __forceinline__ void fence_barrier_init() {
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Orders this thread's earlier (acquired) view of memory written through ordinary stores before its
+// later asynchronous-proxy operations (TMA loads) on any state space.
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* map, uint64_t* bar, int c0, int c1) {
   asm volatile(
