@@ -181,6 +181,23 @@ def workload_config(w):
             "l2": "inputs larger than L2 (weights read once per forward)", "replicas": "independent per GPU"}
 
 
+# ----------------------------------------------------------------------------- replicas
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The job's time is the slowest replica's: MAX all-reduce of the locally measured milliseconds
+    (the only collective of a multi-GPU run; `dist` is None for one process)."""
+    if dist is None:
+        return float(ms)
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(world: int, tokens_per_replica: int, steps: int, ms_max: float) -> float:
+    """Independent replicas, one per GPU: every rank decodes its own copy of the workload."""
+    return world * tokens_per_replica * steps / (ms_max / 1e3)
+
+
 # ----------------------------------------------------------------------------- our arm
 def gemm_bytes(shape, M):
     """Algorithmic bytes of each matmul launch of one M-row forward: weights + inputs + outputs."""
@@ -264,12 +281,7 @@ def run_ours(args):
             st = fn()
         e1.record()
         barrier()
-        ms = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ms], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ms = float(t.item())
-        return ms, st
+        return max_over_ranks(e0.elapsed_time(e1), dist, dev), st
 
     for _ in range(args.warmup):
         step_resident()
@@ -293,8 +305,8 @@ def run_ours(args):
     ms_prefill /= 3
     err_word = d3.d3_get_error_word(ctx)
     tokens = w.batch * w.gen_len
-    value = world * tokens * args.steps / (ms_total / 1e3)
-    e2e_value = world * tokens * args.steps / (ms_e2e / 1e3)
+    value = whole_job_tokens_per_s(world, tokens, args.steps, ms_total)
+    e2e_value = whole_job_tokens_per_s(world, tokens, args.steps, ms_e2e)
     ms_step = ms_total / args.steps
 
     peaks = measured_peaks()
@@ -315,6 +327,16 @@ def run_ours(args):
         achieved = tot_flops / (tot_ms / 1e3) / 1e12 if tot_ms > 0 else 0.0
         roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                     "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None}
+    # whole forward as one unit: weights + KV of one forward over its share of the timed region
+    ms_fwd = (ms_step - ms_prefill) / max(st.steps, 1)
+    kv_mid = 2 * shape.n_layers * shape.n_kv_heads * shape.d_head * 2 * sum(int(l) + w.gen_len // 2 for l in lens_np)
+    fwd_bytes = sum(gb[k] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) * shape.n_layers + gb["gemm_head"] + kv_mid
+    fwd_flops = sum(gf[k] for k in ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down")) * shape.n_layers + gf["gemm_head"]
+    roofline["step_effective"] = {"GB/s": fwd_bytes / (ms_fwd / 1e3) / 1e9, "TFLOP/s": fwd_flops / (ms_fwd / 1e3) / 1e12,
+                                  "frac_of_measured_hbm": fwd_bytes / (ms_fwd / 1e3) / 1e9 / peaks["hbm_gbs"],
+                                  "frac_of_8TBs_nominal": fwd_bytes / (ms_fwd / 1e3) / 1e9 / 8000.0,
+                                  "frac_of_measured_tensor": fwd_flops / (ms_fwd / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
+                                  "ms_per_forward": ms_fwd, "bytes_per_forward": fwd_bytes}
     roofline.update({"kernel": "gemm_tc_kernel (all matmul launches of the decode loop)", "peak_source": f"of {peaks['source']}",
                      "launches": n_gemm, "avg_launch_us": 1e3 * tot_ms / max(n_gemm, 1),
                      "algorithmic_bytes_per_launch": tot_bytes / max(n_gemm, 1)})
