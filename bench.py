@@ -27,6 +27,23 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
+# DRAM traffic (dram bytes read + written) per launch of the matmul kernel at 32 rows on the c2 shapes,
+# from the ncu capture summarised in profiles/gemm_tc_kernel_c2_rows32.md.  It is reported only while the
+# kernel sources still hash to the value below; after any change to them it reads null until re-captured.
+NCU_GEMM_TRAFFIC_MB = {"gemm_qkv": 104.7, "gemm_o": 34.4, "gemm_gate_up": 208.2, "gemm_down": 105.8, "gemm_head": 1050.2}
+NCU_GEMM_SOURCE_HASH = "3d0bc32e5d2d2b9a"
+NCU_GEMM_WORKLOAD = "c2"
+
+
+def gemm_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in ("gemm_tc.cuh", "ptx_sm100.cuh"):
+        with open(os.path.join(ROOT, "paper_2601_07568_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
 METRIC = "decoded tokens/s"
 UNIT = "tokens/s"
 
@@ -337,6 +354,9 @@ def run_ours(args):
                                   "frac_of_8TBs_nominal": fwd_bytes / (ms_fwd / 1e3) / 1e9 / 8000.0,
                                   "frac_of_measured_tensor": fwd_flops / (ms_fwd / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
                                   "ms_per_forward": ms_fwd, "bytes_per_forward": fwd_bytes}
+    if hbm_bound and w.name == NCU_GEMM_WORKLOAD and gemm_source_hash() == NCU_GEMM_SOURCE_HASH and n_gemm > 0:
+        roofline["traffic"] = 1e6 * sum(NCU_GEMM_TRAFFIC_MB[k] * prof[k]["launches"] for k in NCU_GEMM_TRAFFIC_MB) / n_gemm
+        roofline["traffic_source"] = "ncu, profiles/gemm_tc_kernel_c2_rows32.md (bytes per launch, averaged over the launch mix)"
     roofline.update({"kernel": "gemm_tc_kernel (all matmul launches of the decode loop)", "peak_source": f"of {peaks['source']}",
                      "launches": n_gemm, "avg_launch_us": 1e3 * tot_ms / max(n_gemm, 1),
                      "algorithmic_bytes_per_launch": tot_bytes / max(n_gemm, 1)})
