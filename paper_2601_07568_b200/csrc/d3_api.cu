@@ -80,6 +80,8 @@ struct d3_ctx {
   bool pdl = true;           // programmatic dependent launch between the kernels of a forward
   int* skip_flag = nullptr;  // device flag: non-zero turns the forward's kernels into no-ops
   int tune_producers = 0;
+  int tune_attn_div = 0;  // experiment: key tiles per attention split
+  int tune_no_cluster = 0;  // 1: skinny matmuls on the unit-range kernel (L2 reduction) instead of clusters
   int tune_wide_tiles = -1;  // -1: by row count; 0 / 1: force 128- / 256-column tiles
   int tune_ring_kb = 0, tune_ctas_per_sm = 0;  // matmul tuning overrides (0 = default)
   struct ProfPair { cudaEvent_t a, b; int cls; };
@@ -336,10 +338,120 @@ int run_linear_tc_bn(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   return dispatch_tc<BLOCK_N>(c, epi, tx, tw, p, static_cast<int>(n_ctas), smem);
 }
 
+// Skinny matmuls (up to 64 rows): clusters of C CTAs own whole 128-column tiles and split K among
+// their CTAs; the partial sums meet in distributed shared memory (gemm_ck_kernel).  C and the number
+// of clusters are chosen so that the longest CTA has the fewest (tile, K slab) units.
+template <int EPI>
+int launch_ck(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, const tc::ClusterSplit& cs,
+              size_t smem) {
+  auto kern = tc::gemm_ck_kernel<EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(cs.n_clusters * cs.C));
+  cfg.blockDim = dim3(tc::NUM_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  at[na].id = cudaLaunchAttributeClusterDimension;
+  at[na].val.clusterDim.x = static_cast<unsigned>(cs.C);
+  at[na].val.clusterDim.y = 1;
+  at[na].val.clusterDim.z = 1;
+  ++na;
+  if (c->pdl && !c->prof_on) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = na;
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, *tx, *tw, p, cs));
+  LAUNCHED(c, "gemm_ck_kernel");
+  return D3_OK;
+}
+
+int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
+                  int c_hint, const QkvExtra* qx, int w_tiled) {
+  const int T = (N + 127) / 128, KC = (K + 63) / 64;
+  const int a_rows = ((M + 31) / 32) * 32;  // 32 or 64
+  // ring + partial tile must leave room for two CTAs per SM
+  const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + 128 * 128;
+  const size_t part_bytes = static_cast<size_t>(128) * a_rows * 4;
+  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 100) * 1024;
+  int stages = static_cast<int>((budget > part_bytes ? budget - part_bytes : 0) / stage_bytes);
+  stages = std::max(2, std::min(stages, 16));
+  const size_t smem = tc::gemm_ck_smem_bytes(a_rows, stages);
+  const int per_sm = std::max(1, std::min(c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : 2, static_cast<int>((227 * 1024) / (smem + 1024))));
+  const int slots = c->n_sms * per_sm;
+  tc::ClusterSplit cs{1, 1};
+  long long best = -1;
+  for (int C = 1; C <= 8; ++C) {
+    if (C > KC) break;
+    if (c_hint > 0 && C != c_hint) continue;
+    const int n_cl = std::max(1, std::min(slots / C, T));
+    const long long cost = static_cast<long long>((T + n_cl - 1) / n_cl) * ((KC + C - 1) / C) * 16 + C;  // ties: smaller clusters
+    if (best < 0 || cost < best) {
+      best = cost;
+      cs.C = C;
+      cs.n_clusters = n_cl;
+    }
+  }
+  tc::GemmParams p{};
+  p.M = M; p.N = N; p.K = K;
+  p.a_rows = a_rows;
+  p.m_tiles = 1; p.n_tiles = T; p.k_chunks = KC;
+  p.total_units = static_cast<long long>(T) * KC;
+  p.stages = stages;
+  p.error_word = c->error_word;
+  p.skip_flag = c->skip_flag;
+  p.w_tiled = w_tiled;
+  p.n_producers = 2;
+  p.ep = ep;
+  if (qx) {
+    p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
+    p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
+    p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
+    p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
+  }
+  const CUtensorMap *tx, *tw;
+  TRY(get_tmap(c, X, M, K, a_rows, &tx));
+  if (w_tiled) {
+    if ((reinterpret_cast<uintptr_t>(W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
+    p.w_packed = static_cast<const bf16*>(W);
+    p.w_blocks = static_cast<long long>(T) * KC;
+    tw = tx;
+  } else {
+    TRY(get_tmap(c, W, N, K, 128, &tw));
+  }
+  switch (epi) {
+    case EPI_F32: return launch_ck<EPI_F32>(c, tx, tw, p, cs, smem);
+    case EPI_T: return launch_ck<EPI_T>(c, tx, tw, p, cs, smem);
+    case EPI_RESID: return launch_ck<EPI_RESID>(c, tx, tw, p, cs, smem);
+    case EPI_SWIGLU: return launch_ck<EPI_SWIGLU>(c, tx, tw, p, cs, smem);
+    case EPI_QKV: return launch_ck<EPI_QKV>(c, tx, tw, p, cs, smem);
+    case EPI_STATS: return launch_ck<EPI_STATS>(c, tx, tw, p, cs, smem);
+  }
+  return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
+}
+
 // Tile width: 128 columns while weight streaming dominates, 256 when
 // it is bound by the tensor pipe (from 512 rows on: a third less operand traffic per flop).
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
                   int ctas_hint, const QkvExtra* qx, int w_tiled) {
+  // `ctas_hint` 1..8 on a skinny matmul forces the cluster size; larger hints ask for the unit-range kernel
+  // Few column tiles and a long K (O-proj, down): clusters of 8 that split K and reduce through
+  // distributed shared memory beat the L2 reduction of the unit-range kernel (measured at 32 rows:
+  // 14 vs 17 us and 25 vs 30 us on the 8B shapes); with many tiles the unit-range kernel wins,
+  // because cluster launches of this kernel get one CTA per SM only.
+  if (M <= 64 && !c->tune_no_cluster) {
+    const int T = (N + 127) / 128, KC = (K + 63) / 64;
+    if (ctas_hint >= 1 && ctas_hint <= 8) return run_linear_ck(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
+    if (ctas_hint == 0 && T * 8 <= 2 * c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 8, qx, w_tiled);
+  }
   const bool wide = c->tune_wide_tiles >= 0 ? c->tune_wide_tiles != 0 : M >= 512;
   if (wide && N >= 256) return run_linear_tc_bn<256>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
   return run_linear_tc_bn<128>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
@@ -438,7 +550,7 @@ int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMa
   if (q_tiles <= 2) {  // decode-sized: split the keys when (sequence, kv head) pairs alone leave SMs idle
     const int max_tiles = (g.max_seq + attn::KT - 1) / attn::KT;
     splits = (2 * c->n_sms + pairs * q_tiles - 1) / (pairs * q_tiles);
-    splits = std::min(splits, std::max(1, max_tiles / 2));
+    splits = std::min(splits, std::max(1, c->tune_attn_div > 0 ? max_tiles / c->tune_attn_div : max_tiles / 2));
     splits = std::max(1, std::min(splits, 8));  // one cluster per query tile: at most 8 CTAs
   }
   attn::AttnTcParams p{};
@@ -1110,6 +1222,8 @@ extern "C" int d3_set_matmul_tuning(d3_ctx* c, int32_t ring_kb, int32_t ctas_per
   if (!c || ring_kb < 0 || (ring_kb & 0xffff) > 200 || ctas_per_sm < 0 || ctas_per_sm > 3) return D3_ERR_INVALID_ARG;
   c->tune_producers = (ring_kb >> 16) & 0xf;  // experiments: bits 16-19 of ring_kb = producer warps, 20-21 = tile width + 1
   c->tune_wide_tiles = ((ring_kb >> 20) & 3) - 1;
+  c->tune_attn_div = (ring_kb >> 22) & 7;
+  c->tune_no_cluster = (ring_kb >> 25) & 1;
   c->tune_ring_kb = ring_kb & 0xffff;
   c->tune_ctas_per_sm = ctas_per_sm;
   return D3_OK;

@@ -370,7 +370,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     fence_barrier_init();
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, TMEM_COLS);
+    tmem_alloc<TMEM_COLS>(tmem_slot);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -562,8 +562,255 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, TMEM_COLS);
+    tmem_dealloc<TMEM_COLS>(tmem_base);
   }
+}
+
+// ----------------------------------------------------------------------------- cluster K-split kernel
+// Skinny matmuls (up to 64 rows, 128-column tiles).  The grid is made of clusters of C CTAs
+// (C = 1..8).  A cluster owns whole output tiles; inside it every CTA takes one C-th of the K range of
+// each tile, so all C partial accumulators of a tile are complete at the same time.  They are summed
+// through distributed shared memory instead of L2: each CTA copies its accumulator to its own shared
+// memory, signals its peers (remote mbarrier arrive, release at cluster scope), and the CTAs that own
+// a 32-column slice of the tile add the C partials in rank order (fixed order: reproducible bits)
+// and run the epilogue on their slice.  No global workspace, no atomics, no fences on the way.
+struct ClusterSplit {
+  int C;           // CTAs per cluster
+  int n_clusters;  // clusters that have tiles
+};
+
+struct DsmemSource {
+  uint32_t part_addr;  // shared-memory address of this CTA's partial tile [128 columns][a_rows] fp32
+  int C, a_rows, row;
+  __device__ __forceinline__ void load(int c, float (&v)[32]) const {
+#pragma unroll
+    for (int j = 0; j < 32; ++j) v[j] = 0.f;
+    const uint32_t off = part_addr + static_cast<uint32_t>(c * a_rows + row) * 4u;
+    const uint32_t step = static_cast<uint32_t>(a_rows) * 4u;
+    int s = 0;
+    for (; s + 1 < C; s += 2) {  // two peers' loads in flight; the sums stay in rank order
+      const uint32_t a0 = map_to_cta(off, static_cast<uint32_t>(s)), a1 = map_to_cta(off, static_cast<uint32_t>(s + 1));
+      float t0[32], t1[32];
+#pragma unroll
+      for (int j = 0; j < 32; ++j) t0[j] = ld_cluster_f(a0 + j * step);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) t1[j] = ld_cluster_f(a1 + j * step);
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] = (v[j] + t0[j]) + t1[j];
+    }
+    if (s < C) {
+      const uint32_t a0 = map_to_cta(off, static_cast<uint32_t>(s));
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += ld_cluster_f(a0 + j * step);
+    }
+  }
+};
+
+// grid = (n_clusters * C), cluster dims (C, 1, 1).  Dynamic shared memory as in gemm_tc_kernel, plus
+// the partial tile [128][a_rows] fp32 and the two cluster barriers.
+template <int EPI>
+__global__ void __launch_bounds__(NUM_THREADS, 2)
+gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+               const GemmParams p, const ClusterSplit cs) {
+  constexpr int BLOCK_N = 128;
+  if (p.skip_flag != nullptr && *p.skip_flag != 0) return;
+  grid_dep_launch();
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int stages = p.stages;
+  const uint32_t a_stage_bytes = static_cast<uint32_t>(p.a_rows) * 128u;
+  constexpr uint32_t b_stage_bytes = BLOCK_N * 128u;
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + static_cast<size_t>(stages) * a_stage_bytes;
+  float* part = reinterpret_cast<float*>(smem_b + static_cast<size_t>(stages) * b_stage_bytes);  // [128][a_rows]
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(part + 128 * p.a_rows);
+  uint64_t* empty_bar = full_bar + stages;
+  uint64_t* acc_full = empty_bar + stages;
+  uint64_t* acc_empty = acc_full + 2;
+  uint64_t* ready_bar = acc_empty + 2;  // all C partials of the current tile are in shared memory
+  uint64_t* free_bar = ready_bar + 1;   // all C CTAs have finished reading this CTA's partial
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(free_bar + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int C = cs.C;
+  const int rank = static_cast<int>(cluster_ctarank());
+  const int cluster = blockIdx.x / C;
+  const int T = p.n_tiles;  // one row tile: tiles = column tiles
+  const int KC = p.k_chunks;
+  const int t0 = static_cast<int>(static_cast<long long>(T) * cluster / cs.n_clusters);
+  const int t1 = static_cast<int>(static_cast<long long>(T) * (cluster + 1) / cs.n_clusters);
+  const int kc0 = KC * rank / C, kc1 = KC * (rank + 1) / C;  // C <= KC: never empty
+  const int n_k = kc1 - kc0;
+  const long long n_total = static_cast<long long>(t1 - t0) * n_k;
+  constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_x);
+    if (!p.w_tiled) prefetch_tensormap(&tmap_w);
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 128);
+    }
+    mbar_init(ready_bar, static_cast<uint32_t>(C));
+    mbar_init(free_bar, static_cast<uint32_t>(C));
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc<TMEM_COLS>(tmem_slot);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();  // every CTA's barriers exist before a peer arrives on them
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0 || warp == 6) {
+    // ---------------- TMA producers: alternate units
+    const int pi = warp == 0 ? 0 : 1;
+    if (lane == 0) {
+      const uint32_t tx = a_stage_bytes + b_stage_bytes;
+      auto unit_of = [&](long long i, int& n_tile, int& kc) {
+        n_tile = t0 + static_cast<int>(i / n_k);
+        kc = kc0 + static_cast<int>(i % n_k);
+      };
+      auto load_w = [&](int s, int n_tile, int kc) {
+        uint8_t* dst = smem_b + static_cast<size_t>(s) * b_stage_bytes;
+        mbar_arrive_expect_tx(&full_bar[s], tx);
+        if (p.w_tiled) bulk_load_1d(dst, p.w_packed + (static_cast<long long>(n_tile) * KC + kc) * (128 * 64), 128 * 128, &full_bar[s]);
+        else tma_load_2d(dst, &tmap_w, &full_bar[s], kc * BLOCK_K, n_tile * BLOCK_N);
+      };
+      const int pre = static_cast<int>(n_total < stages ? n_total : stages);
+      for (int i = pi; i < pre; i += 2) {  // weights first: they do not depend on the kernels before this one
+        int n_tile, kc;
+        unit_of(i, n_tile, kc);
+        load_w(i, n_tile, kc);
+      }
+      grid_dep_wait();
+      for (int i = pi; i < pre; i += 2) {
+        int n_tile, kc;
+        unit_of(i, n_tile, kc);
+        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], kc * BLOCK_K, 0);
+      }
+      long long i = pre;
+      if ((i & 1) != pi) ++i;
+      for (; i < n_total; i += 2) {
+        const int s = static_cast<int>(i % stages);
+        const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+        if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.error_word)) break;
+        int n_tile, kc;
+        unit_of(i, n_tile, kc);
+        load_w(s, n_tile, kc);
+        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K, 0);
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer: one accumulator per tile, alternating TMEM halves
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
+      long long i = 0;
+      bool ok = true;
+      for (int t = t0; t < t1 && ok; ++t) {
+        const int seg = t - t0, buf = seg & 1;
+        if (!mbar_wait(&acc_empty[buf], (static_cast<uint32_t>(seg >> 1) & 1u) ^ 1u, abort_flag, p.error_word)) break;
+        tc_fence_after();
+        const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * BLOCK_N);
+        for (int k = 0; k < n_k; ++k, ++i) {
+          const int s = static_cast<int>(i % stages);
+          const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+          if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t adesc = make_smem_desc(smem_u32(smem_a + static_cast<size_t>(s) * a_stage_bytes));
+          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + static_cast<size_t>(s) * b_stage_bytes));
+#pragma unroll
+          for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk)
+            umma_bf16(tmem_d, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
+                      (k > 0 || kk > 0) ? 1u : 0u);
+          umma_commit(&empty_bar[s]);
+        }
+        if (ok) umma_commit(&acc_full[buf]);
+      }
+    }
+  } else {
+    // ---------------- epilogue warps
+    grid_dep_wait();
+    const int lg = warp & 3;
+    const int row = lg * 32 + lane;
+    const int et = threadIdx.x - 64;  // 0..127
+    const bool warp_live = (lg * 32 < p.a_rows) && (lg * 32 < p.M);
+    const uint32_t part_addr = smem_u32(part);
+    // (row, 32-column chunk) pairs of this CTA's slice: chunks rank, rank + C, ... (< 4)
+    const int tpr = 128 / p.a_rows;  // threads that can share a row: 4 or 2
+    const int prow = et % p.a_rows, sub = et / p.a_rows;
+    bool alive = true;
+    int seg = 0;
+    for (int t = t0; t < t1; ++t, ++seg) {
+      const int buf = seg & 1;
+      const int n0 = t * BLOCK_N;
+      bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
+      // the peers must be done with this CTA's previous partial before it is overwritten
+      if (ok && seg > 0) ok = mbar_wait_cluster(free_bar, static_cast<uint32_t>(seg - 1) & 1u, abort_flag, p.error_word);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { alive = false; break; }
+      tc_fence_after();
+      if (warp_live) {
+        TmemSource tsrc{tmem_base + static_cast<uint32_t>(buf * BLOCK_N) + (static_cast<uint32_t>(lg * 32) << 16)};
+        for (int c = 0; c < BLOCK_N; c += 32) {
+          float v[32];
+          tsrc.load(c, v);
+#pragma unroll
+          for (int q = 0; q < 32; ++q) part[(c + q) * p.a_rows + row] = v[q];
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&acc_empty[buf]);
+      epi_bar_sync();  // the whole partial is written ...
+      if (et < C) mbar_arrive_remote(ready_bar, static_cast<uint32_t>(et));  // ... tell every CTA of the cluster
+      ok = mbar_wait_cluster(ready_bar, static_cast<uint32_t>(seg) & 1u, abort_flag, p.error_word);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { alive = false; break; }
+      if constexpr (EPI == EPI_STATS) {
+        // one statistic per (row, 128 columns): rank 0 takes the whole tile, a row stays with one thread
+        if (rank == 0 && warp_live) {
+          DsmemSource dsrc{part_addr, C, p.a_rows, row};
+          run_epilogue<EPI, BLOCK_N>(dsrc, p, row, n0, row < p.M);
+        }
+      } else {
+        // chunk list of this rank, spread over the threads that share a row
+        int my_chunks = 0;
+        for (int c = rank; c < 4; c += C) ++my_chunks;
+        if (sub < tpr && sub < my_chunks) {
+          DsmemSource dsrc{part_addr, C, p.a_rows, prow};
+          // chunk indices rank + C * (sub + tpr * q): first = rank + C * sub, stride = C * tpr
+          run_epilogue<EPI, BLOCK_N>(dsrc, p, prow, n0, prow < p.M, rank + C * sub, C * tpr);
+        }
+      }
+      epi_bar_sync();  // this CTA has read all it needs from every peer
+      if (et < C) mbar_arrive_remote(free_bar, static_cast<uint32_t>(et));
+    }
+    // nobody may still be reading this CTA's partial when it exits
+    if (alive && seg > 0) mbar_wait_cluster(free_bar, static_cast<uint32_t>(seg - 1) & 1u, abort_flag, p.error_word);
+    tc_fence_before();
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc<TMEM_COLS>(tmem_base);
+  }
+  cluster_sync_all();  // shared memory of a CTA stays valid until its peers are past their last remote access
+}
+
+inline size_t gemm_ck_smem_bytes(int a_rows, int stages) {
+  size_t body = static_cast<size_t>(stages) * (a_rows * 128 + 128 * 128) + static_cast<size_t>(128) * a_rows * 4;
+  size_t need = static_cast<size_t>(stages) * a_rows * 128 + static_cast<size_t>(128 - a_rows) * 128 + 128 * 128;
+  if (body < need) body = need;
+  return 1024 + body + (2 * stages + 6) * 8 + 64;
 }
 
 inline size_t gemm_tc_smem_bytes(int a_rows, int block_n, int stages) {
