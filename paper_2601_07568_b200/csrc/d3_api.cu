@@ -81,6 +81,8 @@ struct d3_ctx {
   int* skip_flag = nullptr;  // device flag: non-zero turns the forward's kernels into no-ops
   int tune_producers = 0;
   int tune_attn_div = 0;  // experiment: key tiles per attention split
+  int tune_pair = -1;     // -1: by row count; 0 / 1: one / two row tiles per matmul unit
+  int tune_no_rr = 0;     // 1: wide matmuls on contiguous unit ranges
   int tune_no_cluster = 0;  // 1: skinny matmuls on the unit-range kernel (L2 reduction) instead of clusters
   int tune_wide_tiles = -1;  // -1: by row count; 0 / 1: force 128- / 256-column tiles
   int tune_ring_kb = 0, tune_ctas_per_sm = 0;  // matmul tuning overrides (0 = default)
@@ -255,10 +257,10 @@ cudaError_t launch_pdl(d3_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block,
   return cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
 }
 
-template <int EPI, int BLOCK_N>
+template <int EPI, int BLOCK_N, int MT>
 int launch_tc(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, int n_ctas,
               size_t smem) {
-  auto kern = tc::gemm_tc_kernel<EPI, BLOCK_N>;
+  auto kern = tc::gemm_tc_kernel<EPI, BLOCK_N, MT>;
   static bool attr_set = false;
   if (!attr_set) {
     CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
@@ -269,30 +271,31 @@ int launch_tc(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc:
   return D3_OK;
 }
 
-template <int BLOCK_N>
+template <int BLOCK_N, int MT>
 int dispatch_tc(d3_ctx* c, int epi, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, int n_ctas,
                 size_t smem) {
   switch (epi) {
-    case EPI_F32: return launch_tc<EPI_F32, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
-    case EPI_T: return launch_tc<EPI_T, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
-    case EPI_RESID: return launch_tc<EPI_RESID, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
-    case EPI_SWIGLU: return launch_tc<EPI_SWIGLU, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
-    case EPI_QKV: return launch_tc<EPI_QKV, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
-    case EPI_STATS: return launch_tc<EPI_STATS, BLOCK_N>(c, tx, tw, p, n_ctas, smem);
+    case EPI_F32: return launch_tc<EPI_F32, BLOCK_N, MT>(c, tx, tw, p, n_ctas, smem);
+    case EPI_T: return launch_tc<EPI_T, BLOCK_N, MT>(c, tx, tw, p, n_ctas, smem);
+    case EPI_RESID: return launch_tc<EPI_RESID, BLOCK_N, MT>(c, tx, tw, p, n_ctas, smem);
+    case EPI_SWIGLU: return launch_tc<EPI_SWIGLU, BLOCK_N, MT>(c, tx, tw, p, n_ctas, smem);
+    case EPI_QKV: return launch_tc<EPI_QKV, BLOCK_N, MT>(c, tx, tw, p, n_ctas, smem);
+    case EPI_STATS: return launch_tc<EPI_STATS, BLOCK_N, MT>(c, tx, tw, p, n_ctas, smem);
   }
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
 // Persistent CTAs; the (tile, K slab) units are dealt out evenly (see gemm_tc.cuh).
 // `ctas_hint` > 0 forces the grid size (tests use it to move the segment borders around).
-template <int BLOCK_N>
+template <int BLOCK_N, int MT>
 int run_linear_tc_bn(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
                      int ctas_hint, const QkvExtra* qx, int w_tiled) {
-  const int m_tiles = (M + 127) / 128, n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
+  // m_tiles counts the row groups a unit covers: 128 rows, or 256 when two row tiles share a weight slab
+  const int m_tiles = (M + 128 * MT - 1) / (128 * MT), n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_chunks = (K + 63) / 64;
   const long long tiles = static_cast<long long>(m_tiles) * n_tiles;
   if (tiles > c->n_tile_count) return fail(c, D3_ERR_SHAPE, "matmul has more output tiles than arrival counters");
-  const int a_rows = M >= 128 ? 128 : ((M + 31) / 32) * 32;
+  const int a_rows = MT == 2 ? 256 : (M >= 128 ? 128 : ((M + 31) / 32) * 32);
   tc::GemmParams p{};
   p.M = M; p.N = N; p.K = K;
   p.a_rows = a_rows;
@@ -303,7 +306,15 @@ int run_linear_tc_bn(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   // at least eight K slabs per CTA: shorter ranges only add partial tiles
   long long n_ctas = std::min<long long>(static_cast<long long>(c->n_sms) * per_sm, std::max<long long>(1, p.total_units / 8));
   if (ctas_hint > 0) n_ctas = std::min<long long>(ctas_hint, p.total_units);
-  n_ctas = std::min<long long>(n_ctas, std::min<long long>(tc::MAX_CTAS, static_cast<long long>(c->partial_slots / (2 * (BLOCK_N / 128)))));
+  // From 512 rows on the matmul is bound by the tensor pipe and by L2 reuse, not by balance: whole
+  // tiles dealt round-robin in a banded order keep the CTAs of a moment on neighbouring tiles, so
+  // weights are read from HBM once instead of once per row tile.
+  if (BLOCK_N == 256 && MT == 1 && ctas_hint == 0 && !c->tune_no_rr) {
+    p.rr = 1;
+    p.gm = std::min(m_tiles, 16);
+    n_ctas = std::min<long long>(c->n_sms, tiles);
+  }
+  n_ctas = std::min<long long>(n_ctas, std::min<long long>(tc::MAX_CTAS, static_cast<long long>(c->partial_slots / (2 * MT * (BLOCK_N / 128)))));
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + BLOCK_N * 128;
   // skinny matmuls are bound by HBM: keep the ring near 100 KB so that two CTAs (of this kernel, or
   // of this one and the next) share an SM; wide ones get all of shared memory
@@ -335,7 +346,7 @@ int run_linear_tc_bn(d3_ctx* c, const void* X, const void* W, int M, int N, int 
     TRY(get_tmap(c, W, N, K, BLOCK_N, &tw));
   }
   const size_t smem = tc::gemm_tc_smem_bytes(a_rows, BLOCK_N, stages);
-  return dispatch_tc<BLOCK_N>(c, epi, tx, tw, p, static_cast<int>(n_ctas), smem);
+  return dispatch_tc<BLOCK_N, MT>(c, epi, tx, tw, p, static_cast<int>(n_ctas), smem);
 }
 
 // Skinny matmuls (up to 64 rows): clusters of C CTAs own whole 128-column tiles and split K among
@@ -453,8 +464,13 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
     if (ctas_hint == 0 && T * 8 <= 2 * c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 8, qx, w_tiled);
   }
   const bool wide = c->tune_wide_tiles >= 0 ? c->tune_wide_tiles != 0 : M >= 512;
-  if (wide && N >= 256) return run_linear_tc_bn<256>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
-  return run_linear_tc_bn<128>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
+  if (wide && N >= 256) return run_linear_tc_bn<256, 1>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
+  // 129..511 rows: two row tiles per unit share each weight slab
+  // (worth it when there are enough column tiles to give every SM whole tiles: with few tiles the
+  // doubled partial tiles of split outputs cost more than the saved weight traffic)
+  const bool pair = c->tune_pair >= 0 ? c->tune_pair != 0 : (M > 128 && (N + 127) / 128 >= c->n_sms);
+  if (pair && M > 128) return run_linear_tc_bn<128, 2>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
+  return run_linear_tc_bn<128, 1>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
 }
 
 template <typename T>
@@ -1224,6 +1240,8 @@ extern "C" int d3_set_matmul_tuning(d3_ctx* c, int32_t ring_kb, int32_t ctas_per
   c->tune_wide_tiles = ((ring_kb >> 20) & 3) - 1;
   c->tune_attn_div = (ring_kb >> 22) & 7;
   c->tune_no_cluster = (ring_kb >> 25) & 1;
+  c->tune_pair = ((ring_kb >> 26) & 3) - 1;
+  c->tune_no_rr = (ring_kb >> 28) & 1;
   c->tune_ring_kb = ring_kb & 0xffff;
   c->tune_ctas_per_sm = ctas_per_sm;
   return D3_OK;

@@ -40,15 +40,17 @@ constexpr int MAX_CTAS = 512;     // upper bound of the grid (segment list of a 
 
 struct GemmParams {
   int M, N, K;
-  int a_rows;       // rows of the X box: 32, 64 or 128
+  int a_rows;       // rows of the X box: 32, 64, 96 or 128 (one row tile per unit), 256 (two)
   int stages;       // pipeline depth
   int m_tiles, n_tiles, k_chunks;
   long long total_units;  // m_tiles * n_tiles * k_chunks
-  float* partial;   // partial tiles [2 * grid][BLOCK_N][128] fp32: slot 2i = CTA i's first segment, 2i+1 = its last
+  float* partial;   // partial tiles [2 * grid][row tiles per unit][BLOCK_N][128] fp32: slot 2i = CTA i's first segment, 2i+1 = its last
   int* tile_count;  // arrival counters [tiles], zero on entry and on exit
   uint32_t* error_word;
   const int* skip_flag;  // optional: non-zero -> the whole launch is a no-op
   int n_producers;       // 1 or 2 TMA-issuing warps
+  int rr;                // 1: whole tiles dealt round-robin in a rasterised order (wide matmuls), 0: contiguous unit ranges
+  int gm;                // round-robin mode: row tiles per band
   const __nv_bfloat16* w_packed;  // tiled weights (w_tiled = 1)
   long long w_blocks;             // number of 128 x 64 blocks in w_packed
   int w_tiled;           // 0: W row-major [N, K]; 1: W stored as contiguous [128 x 64] blocks, block (n_tile, kc) at
@@ -98,18 +100,19 @@ struct TmemSource {
     tmem_ld_wait();
   }
 };
-template <int BLOCK_N>
+template <int SLOT_COLS>
 struct PartialSource {
-  const float* partial;   // workspace base
+  const float* partial;   // workspace base; one slot = SLOT_COLS columns x 128 rows
   const int* slots;       // shared memory: partial slots of this tile's segments in K order
   int n_seg, row;
+  int col0;               // first column of this row tile inside the slot
   __device__ __forceinline__ void load(int c, float (&v)[32]) const {
 #pragma unroll
     for (int j = 0; j < 32; ++j) v[j] = 0.f;
     int s = 0;
     for (; s + 1 < n_seg; s += 2) {  // two segments' loads in flight; the sums stay in K order
-      const float* p0 = partial + (static_cast<size_t>(slots[s]) * BLOCK_N + c) * 128 + row;
-      const float* p1 = partial + (static_cast<size_t>(slots[s + 1]) * BLOCK_N + c) * 128 + row;
+      const float* p0 = partial + (static_cast<size_t>(slots[s]) * SLOT_COLS + col0 + c) * 128 + row;
+      const float* p1 = partial + (static_cast<size_t>(slots[s + 1]) * SLOT_COLS + col0 + c) * 128 + row;
       float t0[32], t1[32];
 #pragma unroll
       for (int j = 0; j < 32; ++j) t0[j] = __ldcg(p0 + j * 128);
@@ -119,7 +122,7 @@ struct PartialSource {
       for (int j = 0; j < 32; ++j) v[j] = (v[j] + t0[j]) + t1[j];
     }
     if (s < n_seg) {
-      const float* p0 = partial + (static_cast<size_t>(slots[s]) * BLOCK_N + c) * 128 + row;
+      const float* p0 = partial + (static_cast<size_t>(slots[s]) * SLOT_COLS + col0 + c) * 128 + row;
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] += __ldcg(p0 + j * 128);
     }
@@ -325,7 +328,10 @@ __device__ __forceinline__ int cta_of_unit(long long x, long long U, int n) {
 //   [stages x a_rows x 128 B]  X slabs      (stage stride a_rows*128)
 //   [stages x BLOCK_N x 128 B] W slabs
 //   barriers: full[stages], empty[stages], acc_full[2], acc_empty[2]; tmem address; flags; segment list
-template <int EPI, int BLOCK_N>
+// MT = 1: one 128-row tile per unit.  MT = 2 (129..511 rows): a unit covers two row tiles that share
+// the weight slab (X box of 256 rows, two MMAs per K step into two accumulators), so weights cross
+// L2 and shared memory once for both; p.m_tiles then counts groups of 256 rows and p.a_rows is 256.
+template <int EPI, int BLOCK_N, int MT>
 __global__ void __launch_bounds__(NUM_THREADS, 2)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                const GemmParams p) {
@@ -350,9 +356,32 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, n_cta = gridDim.x;
   const long long U = p.total_units;
-  const long long u0 = unit_begin(U, cta, n_cta), u1 = unit_begin(U, cta + 1, n_cta);
   const int KC = p.k_chunks;
-  constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;  // 256 or 512: a power of two >= 32
+  // Unit range of this CTA.  Round-robin mode (wide matmuls): the CTA owns whole tiles cta, cta + n,
+  // cta + 2n, ... of a rasterised tile order, numbered here 0, 1, 2, ... (see tile_mn below).
+  const int n_tiles_all = p.m_tiles * p.n_tiles;
+  const int my_tiles = p.rr ? (cta < n_tiles_all ? (n_tiles_all - cta + n_cta - 1) / n_cta : 0) : 0;
+  const long long u0 = p.rr ? 0 : unit_begin(U, cta, n_cta);
+  const long long u1 = p.rr ? static_cast<long long>(my_tiles) * KC : unit_begin(U, cta + 1, n_cta);
+  // Row tile (group) and column tile of a tile index.  Contiguous mode: row tiles fastest.  Round-robin
+  // mode: the CTAs running at the same time work on neighbouring tiles of bands of p.gm row tiles, so
+  // a weight tile is fetched from HBM once and shared through L2 by the CTAs of its band column, and
+  // an activation tile by the CTAs of its band row.
+  auto tile_mn = [&](int t, int& m_t, int& n_t) {
+    if (p.rr) {
+      const int q = cta + t * n_cta;
+      const int band_sz = p.gm * p.n_tiles;
+      const int band = q / band_sz, r = q - band * band_sz;
+      const int rows_here = (p.m_tiles - band * p.gm) < p.gm ? (p.m_tiles - band * p.gm) : p.gm;
+      n_t = r / rows_here;
+      m_t = band * p.gm + r % rows_here;
+    } else {
+      m_t = t % p.m_tiles;
+      n_t = t / p.m_tiles;
+    }
+  };
+  constexpr uint32_t TMEM_COLS = 2 * MT * BLOCK_N;  // 256 or 512: a power of two >= 32
+  static_assert(TMEM_COLS <= 512, "two accumulators of MT row tiles must fit tensor memory");
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmap_x);
@@ -386,7 +415,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       const long long n_total = u1 - u0;
       // Arms the stage's barrier with the bytes that will arrive and issues the weight loads.
       auto load_w = [&](int s, int tile, int kc) {
-        const int n_tile = tile / p.m_tiles;
+        int m_unused, n_tile;
+        tile_mn(tile, m_unused, n_tile);
         uint8_t* dst = smem_b + static_cast<size_t>(s) * b_stage_bytes;
         if (p.w_tiled) {
           // one contiguous, pre-swizzled 16 KB block per 128 weight rows; a 256-wide tile at the
@@ -419,8 +449,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       for (int i = pi; i < pre; i += n_prod) {
         const long long u = u0 + i;
         const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
-        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], kc * BLOCK_K,
-                    (tile % p.m_tiles) * BLOCK_M);
+        int m_t, n_unused;
+        tile_mn(tile, m_t, n_unused);
+        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], kc * BLOCK_K, m_t * (MT * BLOCK_M));
       }
       long long i = pre;
       while (i % n_prod != pi) ++i;
@@ -431,8 +462,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         const long long u = u0 + i;
         const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
         load_w(s, tile, kc);
-        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K,
-                    (tile % p.m_tiles) * BLOCK_M);
+        int m_t, n_unused;
+        tile_mn(tile, m_t, n_unused);
+        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K, m_t * (MT * BLOCK_M));
       }
     } else if (lane == 0) {
       grid_dep_wait();
@@ -453,7 +485,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         // the epilogue must have drained this accumulator (two segments ago)
         if (!mbar_wait(&acc_empty[buf], (static_cast<uint32_t>(seg >> 1) & 1u) ^ 1u, abort_flag, p.error_word)) break;
         tc_fence_after();
-        const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * BLOCK_N);
+        const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * MT * BLOCK_N);
         for (int j = 0; j < n_k; ++j, ++i) {
           const int s = static_cast<int>(i % stages);
           const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
@@ -464,8 +496,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 #pragma unroll
           for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
             // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in the (>>4) address field
-            umma_bf16(tmem_d, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
-                      (j > 0 || kk > 0) ? 1u : 0u);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)  // row tile mt: 128 rows = 16 KB further down the X stage
+              umma_bf16(tmem_d + static_cast<uint32_t>(mt * BLOCK_N), adesc + static_cast<uint64_t>(2 * kk + mt * 1024),
+                        bdesc + static_cast<uint64_t>(2 * kk), idesc, (j > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
         }
@@ -487,32 +521,44 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       const int n_k = static_cast<int>(left < KC - kc0 ? left : KC - kc0);
       u += n_k;
       const int buf = seg & 1;
-      const int m_tile = tile % p.m_tiles, n_tile = tile / p.m_tiles;
-      const int m = m_tile * BLOCK_M + row;
+      int m_group, n_tile;
+      tile_mn(tile, m_group, n_tile);
       const int n0 = n_tile * BLOCK_N;
       bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      // warp-uniform: does this lane group hold any row of X at all?
-      const bool warp_live = (lg * 32 < p.a_rows) && (m_tile * BLOCK_M + lg * 32 < p.M);
-      const bool live = warp_live && m < p.M;
-      TmemSource tsrc{tmem_base + static_cast<uint32_t>(buf * BLOCK_N) + (static_cast<uint32_t>(lg * 32) << 16)};
+      const int rows_pad = p.a_rows < 128 ? p.a_rows : 128;  // rows of one row tile that can be live
+      const uint32_t tmem_seg = tmem_base + static_cast<uint32_t>(buf * MT * BLOCK_N) + (static_cast<uint32_t>(lg * 32) << 16);
       if (n_k == KC) {
-        if (warp_live) run_epilogue<EPI, BLOCK_N>(tsrc, p, m, n0, live);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const int m_tile = m_group * MT + mt;
+          const int m = m_tile * BLOCK_M + row;
+          // warp-uniform: does this lane group hold any row of X at all?
+          const bool warp_live = (lg * 32 < rows_pad) && (m_tile * BLOCK_M + lg * 32 < p.M);
+          TmemSource tsrc{tmem_seg + static_cast<uint32_t>(mt * BLOCK_N)};
+          if (warp_live) run_epilogue<EPI, BLOCK_N>(tsrc, p, m, n0, m < p.M);
+        }
         tc_fence_before();
         mbar_arrive(&acc_empty[buf]);
         continue;
       }
       // partial tile: park it, then let the last arrival finish the tile
       const int my_slot = 2 * cta + (kc0 == 0 ? 1 : 0);  // a segment starting at K = 0 is this CTA's last one
-      if (warp_live) {
-        float* mine = p.partial + static_cast<size_t>(my_slot) * BLOCK_N * 128 + row;
-        for (int c = 0; c < BLOCK_N; c += 32) {
-          float v[32];
-          tsrc.load(c, v);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mine[static_cast<size_t>(c + j) * 128] = v[j];
+      for (int mt = 0; mt < MT; ++mt) {
+        const int m_tile = m_group * MT + mt;
+        const bool warp_live = (lg * 32 < rows_pad) && (m_tile * BLOCK_M + lg * 32 < p.M);
+        if (warp_live) {
+          TmemSource tsrc{tmem_seg + static_cast<uint32_t>(mt * BLOCK_N)};
+          float* mine = p.partial + (static_cast<size_t>(my_slot) * MT + mt) * BLOCK_N * 128 + row;
+          for (int c = 0; c < BLOCK_N; c += 32) {
+            float v[32];
+            tsrc.load(c, v);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) mine[static_cast<size_t>(c + j) * 128] = v[j];
+          }
         }
       }
       tc_fence_before();
@@ -538,20 +584,27 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       epi_bar_sync();
       const int n_seg = *last_flag;
       if (n_seg > 0) {
-        if constexpr (EPI == EPI_STATS) {  // one statistic per (row, 128 columns): a row stays with one thread
-          if (warp_live) {
-            PartialSource<BLOCK_N> psrc{p.partial, seg_slots, n_seg, row};
-            run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, live);
-          }
-        } else {
-          // the sums come from memory, not from TMEM lanes: spread (row, 32-column chunk) pairs over
-          // all 128 threads so that a 32-row matmul does not leave the reduction to one warp
-          const int tpr = 128 / p.a_rows;  // threads per row: 4, 2, 1, 1 for 32, 64, 96, 128 rows
-          const int prow = et % p.a_rows, part = et / p.a_rows;
-          if (part < tpr) {
-            const int m2 = m_tile * BLOCK_M + prow;
-            PartialSource<BLOCK_N> psrc{p.partial, seg_slots, n_seg, prow};
-            run_epilogue<EPI, BLOCK_N>(psrc, p, m2, n0, m2 < p.M, part, tpr);
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+          const int m_tile = m_group * MT + mt;
+          if (m_tile * BLOCK_M >= p.M) break;
+          if constexpr (EPI == EPI_STATS) {  // one statistic per (row, 128 columns): a row stays with one thread
+            const bool warp_live = (lg * 32 < rows_pad) && (m_tile * BLOCK_M + lg * 32 < p.M);
+            if (warp_live) {
+              const int m = m_tile * BLOCK_M + row;
+              PartialSource<MT * BLOCK_N> psrc{p.partial, seg_slots, n_seg, row, mt * BLOCK_N};
+              run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, m < p.M);
+            }
+          } else {
+            // the sums come from memory, not from TMEM lanes: spread (row, 32-column chunk) pairs over
+            // all 128 threads so that a 32-row matmul does not leave the reduction to one warp
+            const int tpr = 128 / rows_pad;  // threads per row: 4, 2, 1, 1 for 32, 64, 96, 128 rows
+            const int prow = et % rows_pad, part = et / rows_pad;
+            if (part < tpr) {
+              const int m2 = m_tile * BLOCK_M + prow;
+              PartialSource<MT * BLOCK_N> psrc{p.partial, seg_slots, n_seg, prow, mt * BLOCK_N};
+              run_epilogue<EPI, BLOCK_N>(psrc, p, m2, n0, m2 < p.M, part, tpr);
+            }
           }
         }
       }
@@ -817,7 +870,7 @@ inline size_t gemm_tc_smem_bytes(int a_rows, int block_n, int stages) {
   // The MMA reads 128 rows of the X operand whatever a_rows is: the last X stage must be followed by
   // at least (128 - a_rows) * 128 bytes of allocated shared memory (the W stages, plus padding).
   size_t body = static_cast<size_t>(stages) * (a_rows * 128 + block_n * 128);
-  size_t need = static_cast<size_t>(stages) * a_rows * 128 + static_cast<size_t>(128 - a_rows) * 128 + 128 * 128;
+  size_t need = static_cast<size_t>(stages) * a_rows * 128 + static_cast<size_t>(a_rows < 128 ? 128 - a_rows : 0) * 128 + 128 * 128;
   if (body < need) body = need;
   return 1024 + body + (2 * stages + 4) * 8 + 64 + MAX_CTAS * 4;
 }
