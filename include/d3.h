@@ -181,7 +181,9 @@ int d3_op_linear(d3_ctx *ctx, const void *x, const void *w, void *y, int32_t m, 
  * slab), zero-padded to whole blocks, so that a CTA walking along K reads one contiguous stretch of
  * HBM.  d3_packed_weight_elems: elements of the packed form of an [n, k] matrix (0 on bad sizes).
  * d3_pack_weight: w [device][n, k] row-major -> packed [device][d3_packed_weight_elems(n, k)].
- * d3_op_linear_packed: d3_op_linear with the weights in that form. */
+ * d3_op_linear_packed: d3_op_linear with the weights in that form.  Here splits may also be -S: run
+ *   the column-strip kernel with strips of S columns (S a multiple of 16, at most 256, dividing n;
+ *   m <= 64), D3_ERR_UNSUPPORTED otherwise. */
 int64_t d3_packed_weight_elems(int32_t n, int32_t k);
 int d3_pack_weight(d3_ctx *ctx, const void *w, int32_t n, int32_t k, void *packed);
 int d3_op_linear_packed(d3_ctx *ctx, const void *x, const void *w_packed, void *y, int32_t m, int32_t n, int32_t k,
@@ -241,8 +243,11 @@ int d3_set_overlap(d3_ctx *ctx, int on);
 
 /* Matmul tuning overrides for measurement sweeps: shared-memory ring per CTA in KB (0 = default:
  * about 100 KB for matmuls of up to 128 rows, 200 KB otherwise; at most 200) and CTAs per SM that the
- * (tile, K slab) units are dealt to (0 = default 1; at most 3).  Results do not change beyond the
- * order of fp32 partial sums. */
+ * (tile, K slab) units are dealt to (0 = default 1; at most 3).  Bits 16 and up of ring_kb select
+ * scheduling variants for sweeps and tests: 16-19 producer warps, 20-21 tile width + 1, 22-24 divisor
+ * of the attention key splits, 25 no cluster K-split, 26-27 row-tile pairs + 1, 28 no round-robin
+ * tiles, 29-30 column strips for skinny matmuls (0 when they pay, 1 never, 2 with one CTA per SM,
+ * 3 wherever the shape allows).  Results do not change beyond the order of fp32 partial sums. */
 int d3_set_matmul_tuning(d3_ctx *ctx, int32_t ring_kb, int32_t ctas_per_sm);
 
 /* Per-class kernel timing for measurement runs.  While enabled, every launch of the forward pass is
@@ -261,6 +266,8 @@ int d3_profile_read(d3_ctx *ctx, double *ms, int64_t *launches);
 int d3_get_error_word(d3_ctx *ctx, uint32_t *word);
 /* Number of this library's kernels launched on the context since creation. */
 int64_t d3_launch_count(d3_ctx *ctx);
+/* The same for one kernel, by its name in the source (e.g. "gemm_strip_kernel"); 0 for unknown names. */
+int64_t d3_launch_count_of(d3_ctx *ctx, const char *kernel);
 /* Bytes of device memory the context holds. */
 int64_t d3_device_bytes(d3_ctx *ctx);
 

@@ -74,6 +74,7 @@ struct d3_ctx {
   int tap_rows = 0;
   int last_rows = 0;
   int64_t launches = 0;
+  std::map<std::string, int64_t> launches_by_kernel;  // the same, per kernel name
   int64_t dev_bytes = 0;
   // per-class kernel timing (off by default)
   bool prof_on = false;
@@ -83,6 +84,7 @@ struct d3_ctx {
   int tune_attn_div = 0;  // experiment: key tiles per attention split
   int tune_pair = -1;     // -1: by row count; 0 / 1: one / two row tiles per matmul unit
   int tune_no_rr = 0;     // 1: wide matmuls on contiguous unit ranges
+  int tune_strip = 0;     // skinny matmuls as column strips: 0 when it pays, 1 never, 2 with one CTA per SM, 3 whenever possible
   int tune_no_cluster = 0;  // 1: skinny matmuls on the unit-range kernel (L2 reduction) instead of clusters
   int tune_wide_tiles = -1;  // -1: by row count; 0 / 1: force 128- / 256-column tiles
   int tune_ring_kb = 0, tune_ctas_per_sm = 0;  // matmul tuning overrides (0 = default)
@@ -135,6 +137,7 @@ int dev_alloc(d3_ctx* c, void** p, size_t bytes, bool zero = true) {
 
 int check_launch(d3_ctx* c, const char* what) {
   c->launches++;
+  c->launches_by_kernel[what]++;
   cudaError_t e = cudaPeekAtLastError();
   if (e != cudaSuccess) {
     (void)cudaGetLastError();
@@ -449,6 +452,81 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
+// Skinny matmuls with many columns as column strips over the whole K range (gemm_strip_kernel): the
+// narrowest strip (a multiple of 16 columns that divides N) whose CTAs are all resident at once.
+// Returns 0 when no strip width qualifies.
+int strip_width(const d3_ctx* c, int M, int N, int w_tiled) {
+  if (!w_tiled || M > 64 || c->tune_strip == 1) return 0;
+  const int a_rows = ((M + 31) / 32) * 32;
+  const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : (c->tune_strip == 2 ? 1 : 2);
+  const int slots = c->n_sms * per_sm;
+  if (c->tune_strip == 3) {  // tests: the narrowest strip the shape allows, whatever it costs
+    for (int S = 16; S <= 256; S += 16)
+      if (N % S == 0) return S;
+    return 0;
+  }
+  for (int S = 16; S <= 256; S += 16) {
+    // every CTA reads all of X: worth it while that is no more than its share of the weights
+    if (N % S != 0 || N / S > slots || S < a_rows) continue;
+    return N / S >= c->n_sms / 2 ? S : 0;  // most SMs must get a strip
+  }
+  return 0;
+}
+
+template <int EPI>
+int launch_strip(d3_ctx* c, const CUtensorMap* tx, const tc::GemmParams& p, int S, int n_ctas, size_t smem) {
+  static bool attr_set[2] = {false, false};
+  const int wide = S > 128 ? 1 : 0;
+  auto kern = wide ? tc::gemm_strip_kernel<EPI, 256> : tc::gemm_strip_kernel<EPI, 128>;
+  if (!attr_set[wide]) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+    attr_set[wide] = true;
+  }
+  CUDA_TRY(c, launch_pdl(c, kern, dim3(n_ctas), dim3(tc::NUM_THREADS), smem, *tx, p, S));
+  LAUNCHED(c, "gemm_strip_kernel");
+  return D3_OK;
+}
+
+int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep, int S,
+                     const QkvExtra* qx) {
+  if ((reinterpret_cast<uintptr_t>(W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
+  const int a_rows = ((M + 31) / 32) * 32;
+  const int KC = (K + 63) / 64;
+  tc::GemmParams p{};
+  p.M = M; p.N = N; p.K = K;
+  p.a_rows = a_rows;
+  p.m_tiles = 1; p.n_tiles = N / S; p.k_chunks = KC;
+  p.total_units = static_cast<long long>(p.n_tiles) * KC;
+  const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : (c->tune_strip == 2 ? 1 : 2);
+  const size_t ring = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 200 / per_sm) * 1024;
+  const size_t stage_bytes = static_cast<size_t>(a_rows + S) * 128;
+  p.stages = std::max(2, std::min<int>(std::min<int>(static_cast<int>(ring / stage_bytes), KC), 32));
+  p.error_word = c->error_word;
+  p.skip_flag = c->skip_flag;
+  p.w_tiled = 1;
+  p.w_packed = static_cast<const bf16*>(W);
+  p.w_blocks = static_cast<long long>((N + 127) / 128) * KC;
+  p.gm = 1;  // K walk of CTA b starts at slab b mod KC
+  p.ep = ep;
+  if (qx) {
+    p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
+    p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
+    p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
+    p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
+  }
+  const CUtensorMap* tx;
+  TRY(get_tmap(c, X, M, K, a_rows, &tx));
+  const size_t smem = tc::gemm_strip_smem_bytes(a_rows, S, p.stages);
+  switch (epi) {
+    case EPI_F32: return launch_strip<EPI_F32>(c, tx, p, S, p.n_tiles, smem);
+    case EPI_T: return launch_strip<EPI_T>(c, tx, p, S, p.n_tiles, smem);
+    case EPI_RESID: return launch_strip<EPI_RESID>(c, tx, p, S, p.n_tiles, smem);
+    case EPI_SWIGLU: return launch_strip<EPI_SWIGLU>(c, tx, p, S, p.n_tiles, smem);
+    case EPI_QKV: return launch_strip<EPI_QKV>(c, tx, p, S, p.n_tiles, smem);
+  }
+  return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
+}
+
 // Tile width: 128 columns while weight streaming dominates, 256 when
 // it is bound by the tensor pipe (from 512 rows on: a third less operand traffic per flop).
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
@@ -462,6 +540,16 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
     const int T = (N + 127) / 128, KC = (K + 63) / 64;
     if (ctas_hint >= 1 && ctas_hint <= 8) return run_linear_ck(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
     if (ctas_hint == 0 && T * 8 <= 2 * c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 8, qx, w_tiled);
+  }
+  if (ctas_hint < 0) {  // a strip width asked for by name
+    const int S = -ctas_hint;
+    if (!w_tiled || M > 64 || epi == EPI_STATS || S % 16 != 0 || S > 256 || N % S != 0)
+      return fail(c, D3_ERR_UNSUPPORTED, "column strips need tiled weights, at most 64 rows and a width that is a multiple of 16, at most 256, and divides n");
+    return run_linear_strip(c, X, W, M, N, K, epi, ep, S, qx);
+  }
+  if (ctas_hint == 0 && epi != EPI_STATS) {
+    const int S = strip_width(c, M, N, w_tiled);
+    if (S > 0) return run_linear_strip(c, X, W, M, N, K, epi, ep, S, qx);
   }
   const bool wide = c->tune_wide_tiles >= 0 ? c->tune_wide_tiles != 0 : M >= 512;
   if (wide && N >= 256) return run_linear_tc_bn<256, 1>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
@@ -1242,6 +1330,7 @@ extern "C" int d3_set_matmul_tuning(d3_ctx* c, int32_t ring_kb, int32_t ctas_per
   c->tune_no_cluster = (ring_kb >> 25) & 1;
   c->tune_pair = ((ring_kb >> 26) & 3) - 1;
   c->tune_no_rr = (ring_kb >> 28) & 1;
+  c->tune_strip = (ring_kb >> 29) & 3;
   c->tune_ring_kb = ring_kb & 0xffff;
   c->tune_ctas_per_sm = ctas_per_sm;
   return D3_OK;
@@ -1273,6 +1362,11 @@ extern "C" int d3_profile_read(d3_ctx* c, double* ms, int64_t* launches) {
   return D3_OK;
 }
 extern "C" int64_t d3_launch_count(d3_ctx* c) { return c ? c->launches : 0; }
+extern "C" int64_t d3_launch_count_of(d3_ctx* c, const char* kernel) {
+  if (!c || !kernel) return 0;
+  auto it = c->launches_by_kernel.find(kernel);
+  return it == c->launches_by_kernel.end() ? 0 : it->second;
+}
 extern "C" int64_t d3_device_bytes(d3_ctx* c) { return c ? c->dev_bytes : 0; }
 
 extern "C" const char* d3_strerror(int code) {

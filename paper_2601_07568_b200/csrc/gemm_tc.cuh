@@ -133,10 +133,12 @@ struct PartialSource {
 // predicates this thread's stores.
 // Chunks (32 columns each) c_first, c_first + c_stride, ... of the tile are handled; the TMEM path
 // takes them all (0, 1), the partial-sum path spreads them over the threads that share a row.
+// `n_end` >= 0 ends the tile before column n_end (a column strip narrower than BLOCK_N; a multiple of
+// 16, so the last chunk may be half a chunk); otherwise the tile ends with the matrix.
 template <int EPI, int BLOCK_N, typename Source>
 __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams& p, int m, int n0, bool live,
-                                             int c_first = 0, int c_stride = 1) {
-  const int N = p.N;
+                                             int c_first = 0, int c_stride = 1, int n_end = -1) {
+  const int N = n_end >= 0 ? n_end : p.N;
   if constexpr (EPI == EPI_F32 || EPI == EPI_RESID) {
     float* y = static_cast<float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
     for (int c = 32 * c_first; c < BLOCK_N; c += 32 * c_stride) {
@@ -216,6 +218,14 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
         uint4* y4 = reinterpret_cast<uint4*>(y + h0);
         y4[0] = make_uint4(w[0], w[1], w[2], w[3]);
         y4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      } else if (h0 + 8 == F && (p.ep.ldy & 7) == 0) {  // half a chunk: 8 outputs
+        uint32_t w[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          __nv_bfloat162 t = __floats2bfloat162_rn(silu_f(v[4 * q]) * v[4 * q + 1], silu_f(v[4 * q + 2]) * v[4 * q + 3]);
+          w[q] = *reinterpret_cast<uint32_t*>(&t);
+        }
+        *reinterpret_cast<uint4*>(y + h0) = make_uint4(w[0], w[1], w[2], w[3]);
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j)
@@ -264,60 +274,67 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       float v[32];
       src.load(c, v);
       if (!live) continue;
-      const int head = n / 128, off = n % 128;
-      if (head < p.n_q_heads + p.n_kv_heads) {
-        __nv_bfloat16* dst;
-        if (head < p.n_q_heads) {
-          dst = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy + head * 128;
-        } else {
-          dst = p.k_cache + ((static_cast<size_t>(b) * p.n_kv_heads + (head - p.n_q_heads)) * p.max_seq + pos) * 128;
-        }
-        const int i0 = off / 2;  // pair index of column 0 of this chunk: 16 pairs, dims i0.. and 64+i0..
-        uint32_t lo[8], hi[8];
+      // two halves of 16 columns: a chunk that starts 16 columns before a head border spans two heads
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          float l2[2], h2[2];
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int j = 2 * q + e;
-            const float co = cs[i0 + j], si = sn[i0 + j];
-            const float a = v[2 * j], bb = v[2 * j + 1];
-            l2[e] = a * co - bb * si;
-            h2[e] = bb * co + a * si;
+      for (int h = 0; h < 2; ++h) {
+        const int nh = n + 16 * h;
+        if (nh >= N) break;
+        const int head = nh / 128, off = nh % 128;
+        if (head < p.n_q_heads + p.n_kv_heads) {
+          __nv_bfloat16* dst;
+          if (head < p.n_q_heads) {
+            dst = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy + head * 128;
+          } else {
+            dst = p.k_cache + ((static_cast<size_t>(b) * p.n_kv_heads + (head - p.n_q_heads)) * p.max_seq + pos) * 128;
           }
-          __nv_bfloat162 tl = __floats2bfloat162_rn(l2[0], l2[1]);
-          __nv_bfloat162 th = __floats2bfloat162_rn(h2[0], h2[1]);
-          lo[q] = *reinterpret_cast<uint32_t*>(&tl);
-          hi[q] = *reinterpret_cast<uint32_t*>(&th);
-        }
-        uint4* d_lo = reinterpret_cast<uint4*>(dst + i0);
-        uint4* d_hi = reinterpret_cast<uint4*>(dst + 64 + i0);
-        d_lo[0] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        d_lo[1] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
-        d_hi[0] = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-        d_hi[1] = make_uint4(hi[4], hi[5], hi[6], hi[7]);
-      } else if (head < p.n_q_heads + 2 * p.n_kv_heads) {
-        __nv_bfloat16* dst = p.v_cache +
-            ((static_cast<size_t>(b) * p.n_kv_heads + (head - p.n_q_heads - p.n_kv_heads)) * p.max_seq + pos) * 128 + off;
-        uint32_t w[16];
+          const int i0 = off / 2;  // pair index of column 0 of this half: 8 pairs, dims i0.. and 64+i0..
+          uint32_t lo[4], hi[4];
 #pragma unroll
-        for (int q = 0; q < 16; ++q) {
-          __nv_bfloat162 t = __floats2bfloat162_rn(v[2 * q], v[2 * q + 1]);
-          w[q] = *reinterpret_cast<uint32_t*>(&t);
-        }
-        uint4* d4 = reinterpret_cast<uint4*>(dst);
+          for (int q = 0; q < 4; ++q) {
+            float l2[2], h2[2];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) d4[q] = make_uint4(w[4 * q], w[4 * q + 1], w[4 * q + 2], w[4 * q + 3]);
+            for (int e = 0; e < 2; ++e) {
+              const int j = 2 * q + e;
+              const float co = cs[i0 + j], si = sn[i0 + j];
+              const float a = v[16 * h + 2 * j], bb = v[16 * h + 2 * j + 1];
+              l2[e] = a * co - bb * si;
+              h2[e] = bb * co + a * si;
+            }
+            __nv_bfloat162 tl = __floats2bfloat162_rn(l2[0], l2[1]);
+            __nv_bfloat162 th = __floats2bfloat162_rn(h2[0], h2[1]);
+            lo[q] = *reinterpret_cast<uint32_t*>(&tl);
+            hi[q] = *reinterpret_cast<uint32_t*>(&th);
+          }
+          *reinterpret_cast<uint4*>(dst + i0) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+          *reinterpret_cast<uint4*>(dst + 64 + i0) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        } else if (head < p.n_q_heads + 2 * p.n_kv_heads) {
+          __nv_bfloat16* dst = p.v_cache +
+              ((static_cast<size_t>(b) * p.n_kv_heads + (head - p.n_q_heads - p.n_kv_heads)) * p.max_seq + pos) * 128 + off;
+          uint32_t w[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            __nv_bfloat162 t = __floats2bfloat162_rn(v[16 * h + 2 * q], v[16 * h + 2 * q + 1]);
+            w[q] = *reinterpret_cast<uint32_t*>(&t);
+          }
+          uint4* d4 = reinterpret_cast<uint4*>(dst);
+          d4[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          d4[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
       }
     }
   }
 }
 
 // ----------------------------------------------------------------------------- kernel
-__device__ __forceinline__ long long unit_begin(long long U, int i, int n) { return U * i / n; }
+__device__ __forceinline__ long long unit_begin(long long U, int i, int n) {
+  // 64-bit division is emulated (hundreds of cycles) and sits on the critical tail of split tiles
+  if (U * n < 0x7fffffffll) return static_cast<long long>(static_cast<unsigned int>(U) * static_cast<unsigned int>(i) / static_cast<unsigned int>(n));
+  return U * i / n;
+}
 // The CTA whose unit range contains unit x (ranges of CTAs without units are skipped by construction).
 __device__ __forceinline__ int cta_of_unit(long long x, long long U, int n) {
-  int i = static_cast<int>(x * n / U);
+  int i = (U * n < 0x7fffffffll) ? static_cast<int>(static_cast<unsigned int>(x) * static_cast<unsigned int>(n) / static_cast<unsigned int>(U))
+                                 : static_cast<int>(x * n / U);
   if (i > n - 1) i = n - 1;
   while (i + 1 < n && unit_begin(U, i + 1, n) <= x) ++i;
   while (i > 0 && unit_begin(U, i, n) > x) --i;
@@ -351,7 +368,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   int* last_flag = const_cast<int*>(abort_flag) + 1;  // 0: not last, else number of segments of the tile
-  int* seg_slots = last_flag + 1;                      // [MAX_CTAS]
+  int* list_len = last_flag + 1;                       // number of segments of the tile being finished
+  int* seg_slots = last_flag + 2;                      // [MAX_CTAS]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, n_cta = gridDim.x;
@@ -414,9 +432,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       const uint32_t tx = a_stage_bytes + b_stage_bytes;
       const long long n_total = u1 - u0;
       // Arms the stage's barrier with the bytes that will arrive and issues the weight loads.
-      auto load_w = [&](int s, int tile, int kc) {
-        int m_unused, n_tile;
-        tile_mn(tile, m_unused, n_tile);
+      auto load_w = [&](int s, int n_tile, int kc) {
         uint8_t* dst = smem_b + static_cast<size_t>(s) * b_stage_bytes;
         if (p.w_tiled) {
           // one contiguous, pre-swizzled 16 KB block per 128 weight rows; a 256-wide tile at the
@@ -439,32 +455,45 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         }
       };
       const int pre = static_cast<int>(n_total < stages ? n_total : stages);
+      // These loops run once per K slab in a single thread and pace the CTA: (tile, K slab) and
+      // (stage, parity) are running counters, no division per slab.
+      const int tile0 = static_cast<int>(u0 / KC);
+      const int kc_first = static_cast<int>(u0 - static_cast<long long>(tile0) * KC);
       // weights first: they do not depend on the kernels before this one
-      for (int i = pi; i < pre; i += n_prod) {
-        const long long u = u0 + i;
-        const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
-        load_w(i, tile, kc);
+      int m_t = 0, n_t = 0, mn_of = -1;  // row and column tile of tile `mn_of`
+      {
+        int tile = tile0, kc = kc_first + pi;
+        while (kc >= KC) { kc -= KC; ++tile; }
+        for (int i = pi; i < pre; i += n_prod) {
+          if (tile != mn_of) { tile_mn(tile, m_t, n_t); mn_of = tile; }
+          load_w(i, n_t, kc);
+          kc += n_prod;
+          while (kc >= KC) { kc -= KC; ++tile; }
+        }
       }
       grid_dep_wait();
+      int tile = tile0, kc = kc_first + pi;
+      while (kc >= KC) { kc -= KC; ++tile; }
       for (int i = pi; i < pre; i += n_prod) {
-        const long long u = u0 + i;
-        const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
-        int m_t, n_unused;
-        tile_mn(tile, m_t, n_unused);
+        if (tile != mn_of) { tile_mn(tile, m_t, n_t); mn_of = tile; }
         tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], kc * BLOCK_K, m_t * (MT * BLOCK_M));
+        kc += n_prod;
+        while (kc >= KC) { kc -= KC; ++tile; }
       }
+      // (tile, kc) now name unit `first`, the first one past the prefetched ring that is this producer's
       long long i = pre;
       while (i % n_prod != pi) ++i;
+      int s = static_cast<int>(i % stages);
+      uint32_t ph = (static_cast<uint32_t>(i / stages) & 1u) ^ 1u;  // parity to wait for on the empty barrier
       for (; i < n_total; i += n_prod) {
-        const int s = static_cast<int>(i % stages);
-        const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.error_word)) break;
-        const long long u = u0 + i;
-        const int tile = static_cast<int>(u / KC), kc = static_cast<int>(u - static_cast<long long>(tile) * KC);
-        load_w(s, tile, kc);
-        int m_t, n_unused;
-        tile_mn(tile, m_t, n_unused);
+        if (!mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
+        if (tile != mn_of) { tile_mn(tile, m_t, n_t); mn_of = tile; }
+        load_w(s, n_t, kc);
         tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K, m_t * (MT * BLOCK_M));
+        kc += n_prod;
+        while (kc >= KC) { kc -= KC; ++tile; }
+        s += n_prod;
+        if (s >= stages) { s -= stages; ph ^= 1u; }
       }
     } else if (lane == 0) {
       grid_dep_wait();
@@ -473,12 +502,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     // ---------------- MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
-      long long i = 0;
+      const uint64_t adesc0 = make_smem_desc(smem_u32(smem_a)), bdesc0 = make_smem_desc(smem_u32(smem_b));
+      const uint64_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;  // stage strides in descriptor units
+      uint64_t adesc = adesc0, bdesc = bdesc0;
+      int s = 0;
+      uint32_t ph = 0;
       int seg = 0;
       bool ok = true;
+      int tile = static_cast<int>(u0 / KC);
+      int kc0 = static_cast<int>(u0 - static_cast<long long>(tile) * KC);
       for (long long u = u0; u < u1 && ok; ++seg) {
-        const int tile = static_cast<int>(u / KC);
-        const int kc0 = static_cast<int>(u - static_cast<long long>(tile) * KC);
         const long long left = u1 - u;
         const int n_k = static_cast<int>(left < KC - kc0 ? left : KC - kc0);
         const int buf = seg & 1;
@@ -486,13 +519,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         if (!mbar_wait(&acc_empty[buf], (static_cast<uint32_t>(seg >> 1) & 1u) ^ 1u, abort_flag, p.error_word)) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * MT * BLOCK_N);
-        for (int j = 0; j < n_k; ++j, ++i) {
-          const int s = static_cast<int>(i % stages);
-          const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+        for (int j = 0; j < n_k; ++j) {
           if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t adesc = make_smem_desc(smem_u32(smem_a + static_cast<size_t>(s) * a_stage_bytes));
-          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + static_cast<size_t>(s) * b_stage_bytes));
 #pragma unroll
           for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
             // advancing K by 16 bf16 = 32 bytes inside the swizzled row: +2 in the (>>4) address field
@@ -502,9 +531,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
                         bdesc + static_cast<uint64_t>(2 * kk), idesc, (j > 0 || kk > 0) ? 1u : 0u);
           }
           umma_commit(&empty_bar[s]);  // frees the stage once these MMAs have read it
+          adesc += a_step;
+          bdesc += b_step;
+          if (++s == stages) { s = 0; ph ^= 1u; adesc = adesc0; bdesc = bdesc0; }
         }
         if (ok) umma_commit(&acc_full[buf]);  // this segment's accumulator is complete
         u += n_k;
+        ++tile;  // a segment ends at a tile border or at the end of the range
+        kc0 = 0;
       }
     }
   } else {
@@ -524,6 +558,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       int m_group, n_tile;
       tile_mn(tile, m_group, n_tile);
       const int n0 = n_tile * BLOCK_N;
+      if (n_k != KC && et == 0) {
+        // split tile: its segments in K order (the CTAs whose ranges meet [tile*KC, (tile+1)*KC)),
+        // worked out while the MMAs of this segment still run
+        const long long t_lo = static_cast<long long>(tile) * KC, t_hi = t_lo + KC;
+        const int i_lo = cta_of_unit(t_lo, U, n_cta), i_hi = cta_of_unit(t_hi - 1, U, n_cta);
+        int n_list = 0;
+        for (int i = i_lo; i <= i_hi; ++i) {
+          const long long a = unit_begin(U, i, n_cta), b = unit_begin(U, i + 1, n_cta);
+          const long long lo = a > t_lo ? a : t_lo, hi = b < t_hi ? b : t_hi;
+          if (lo < hi) seg_slots[n_list++] = 2 * i + (lo == t_lo ? 1 : 0);
+        }
+        *list_len = n_list;
+      }
       bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -563,23 +610,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       }
       tc_fence_before();
       mbar_arrive(&acc_empty[buf]);
-      __threadfence();
-      epi_bar_sync();
+      epi_bar_sync();  // every thread's partial stores are ordered before thread 0's release below
       if (et == 0) {
-        // segments of this tile, in K order: the CTAs whose ranges meet [tile*KC, (tile+1)*KC)
-        const long long t_lo = static_cast<long long>(tile) * KC, t_hi = t_lo + KC;
-        const int i_lo = cta_of_unit(t_lo, U, n_cta), i_hi = cta_of_unit(t_hi - 1, U, n_cta);
-        int n_seg = 0;
-        for (int i = i_lo; i <= i_hi; ++i) {
-          const long long a = unit_begin(U, i, n_cta), b = unit_begin(U, i + 1, n_cta);
-          const long long lo = a > t_lo ? a : t_lo, hi = b < t_hi ? b : t_hi;
-          if (lo < hi) seg_slots[n_seg++] = 2 * i + (lo == t_lo ? 1 : 0);
-        }
-        const int old = atomicAdd(&p.tile_count[tile], 1);
-        const int last = (old == n_seg - 1) ? n_seg : 0;
+        const int n_list = *list_len;
+        int old;  // release: the partial is visible to whoever sees the count; acquire: so are the others'
+        asm volatile("atom.add.acq_rel.gpu.global.s32 %0, [%1], 1;" : "=r"(old) : "l"(&p.tile_count[tile]) : "memory");
+        const int last = (old == n_list - 1) ? n_list : 0;
         if (last) p.tile_count[tile] = 0;  // ready for the next launch
         *last_flag = last;
-        __threadfence();
       }
       epi_bar_sync();
       const int n_seg = *last_flag;
@@ -729,9 +767,11 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     const int pi = warp == 0 ? 0 : 1;
     if (lane == 0) {
       const uint32_t tx = a_stage_bytes + b_stage_bytes;
-      auto unit_of = [&](long long i, int& n_tile, int& kc) {
-        n_tile = t0 + static_cast<int>(i / n_k);
-        kc = kc0 + static_cast<int>(i % n_k);
+      // unit i of this CTA = (tile t0 + i / n_k, slab kc0 + i % n_k), kept as running counters (no
+      // division per slab: these single-thread loops pace the CTA)
+      auto advance = [&](int& n_tile, int& k, int by) {
+        k += by;
+        while (k >= n_k) { k -= n_k; ++n_tile; }
       };
       auto load_w = [&](int s, int n_tile, int kc) {
         uint8_t* dst = smem_b + static_cast<size_t>(s) * b_stage_bytes;
@@ -740,52 +780,60 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         else tma_load_2d(dst, &tmap_w, &full_bar[s], kc * BLOCK_K, n_tile * BLOCK_N);
       };
       const int pre = static_cast<int>(n_total < stages ? n_total : stages);
-      for (int i = pi; i < pre; i += 2) {  // weights first: they do not depend on the kernels before this one
-        int n_tile, kc;
-        unit_of(i, n_tile, kc);
-        load_w(i, n_tile, kc);
+      {
+        int n_tile = t0, k = 0;
+        advance(n_tile, k, pi);
+        for (int i = pi; i < pre; i += 2) {  // weights first: they do not depend on the kernels before this one
+          load_w(i, n_tile, kc0 + k);
+          advance(n_tile, k, 2);
+        }
       }
       grid_dep_wait();
+      int n_tile = t0, k = 0;
+      advance(n_tile, k, pi);
       for (int i = pi; i < pre; i += 2) {
-        int n_tile, kc;
-        unit_of(i, n_tile, kc);
-        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], kc * BLOCK_K, 0);
+        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], (kc0 + k) * BLOCK_K, 0);
+        advance(n_tile, k, 2);
       }
       long long i = pre;
       if ((i & 1) != pi) ++i;
+      int s = static_cast<int>(i % stages);
+      uint32_t ph = (static_cast<uint32_t>(i / stages) & 1u) ^ 1u;  // parity to wait for on the empty barrier
       for (; i < n_total; i += 2) {
-        const int s = static_cast<int>(i % stages);
-        const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
-        if (!mbar_wait(&empty_bar[s], ph ^ 1u, abort_flag, p.error_word)) break;
-        int n_tile, kc;
-        unit_of(i, n_tile, kc);
-        load_w(s, n_tile, kc);
-        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K, 0);
+        if (!mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
+        load_w(s, n_tile, kc0 + k);
+        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], (kc0 + k) * BLOCK_K, 0);
+        advance(n_tile, k, 2);
+        s += 2;
+        if (s >= stages) { s -= stages; ph ^= 1u; }
       }
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer: one accumulator per tile, alternating TMEM halves
     if (lane == 0) {
       constexpr uint32_t idesc = make_idesc(BLOCK_M, BLOCK_N);
-      long long i = 0;
+      const uint64_t adesc0 = make_smem_desc(smem_u32(smem_a)), bdesc0 = make_smem_desc(smem_u32(smem_b));
+      const uint64_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;
+      uint64_t adesc = adesc0, bdesc = bdesc0;
+      int s = 0;
+      uint32_t ph = 0;
       bool ok = true;
       for (int t = t0; t < t1 && ok; ++t) {
         const int seg = t - t0, buf = seg & 1;
         if (!mbar_wait(&acc_empty[buf], (static_cast<uint32_t>(seg >> 1) & 1u) ^ 1u, abort_flag, p.error_word)) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * BLOCK_N);
-        for (int k = 0; k < n_k; ++k, ++i) {
-          const int s = static_cast<int>(i % stages);
-          const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+        for (int k = 0; k < n_k; ++k) {
           if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) { ok = false; break; }
           tc_fence_after();
-          const uint64_t adesc = make_smem_desc(smem_u32(smem_a + static_cast<size_t>(s) * a_stage_bytes));
-          const uint64_t bdesc = make_smem_desc(smem_u32(smem_b + static_cast<size_t>(s) * b_stage_bytes));
 #pragma unroll
           for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk)
             umma_bf16(tmem_d, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
                       (k > 0 || kk > 0) ? 1u : 0u);
           umma_commit(&empty_bar[s]);
+          adesc += a_step;
+          bdesc += b_step;
+          if (++s == stages) { s = 0; ph ^= 1u; adesc = adesc0; bdesc = bdesc0; }
         }
         if (ok) umma_commit(&acc_full[buf]);
       }
@@ -864,6 +912,171 @@ inline size_t gemm_ck_smem_bytes(int a_rows, int stages) {
   size_t need = static_cast<size_t>(stages) * a_rows * 128 + static_cast<size_t>(128 - a_rows) * 128 + 128 * 128;
   if (body < need) body = need;
   return 1024 + body + (2 * stages + 6) * 8 + 64;
+}
+
+// ----------------------------------------------------------------------------- column-strip kernel
+// Skinny matmuls with many output columns (QKV, gate/up at up to 64 rows).  CTA b owns the column
+// strip [b*S, (b+1)*S) over the whole K range (S a multiple of 16 that divides N, S <= 256): every
+// output is produced by one CTA, so there are no partial tiles, no arrival counters and no fix-up
+// after the last weight byte has arrived; all CTAs stream the same number of weight bytes.  The price
+// is that every CTA reads all of X (from L2), which the host accepts while S >= rows of X.
+// Weights must be in the tiled form: strip rows are a run of whole 8-row swizzle groups inside the
+// 128-row blocks, copied with one bulk copy per block touched.
+// Warp 0 streams weights (never waits for the previous kernel), warp 6 waits for the previous kernel
+// and streams X slabs, warp 1 issues the MMAs (128 x S x 16) into one accumulator, warps 2-5 run the
+// epilogue.  Shared memory: [stages x a_rows x 128 B] X, [stages x S x 128 B] W, barriers.
+template <int EPI, int TCOLS>
+__global__ void __launch_bounds__(NUM_THREADS, 2)
+gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p, const int S) {
+  if (p.skip_flag != nullptr && *p.skip_flag != 0) return;
+  grid_dep_launch();
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int stages = p.stages;
+  const uint32_t a_stage_bytes = static_cast<uint32_t>(p.a_rows) * 128u;
+  const uint32_t b_stage_bytes = static_cast<uint32_t>(S) * 128u;
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + static_cast<size_t>(stages) * a_stage_bytes;
+  // the MMA reads 128 rows of X whatever a_rows is: the barriers start after that reach
+  size_t body = static_cast<size_t>(stages) * (a_stage_bytes + b_stage_bytes);
+  const size_t reach = static_cast<size_t>(stages - 1) * a_stage_bytes + 128 * 128;
+  if (body < reach) body = reach;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + ((body + 7) & ~size_t(7)));
+  uint64_t* empty_bar = full_bar + stages;
+  uint64_t* acc_full = empty_bar + stages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_full + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KC = p.k_chunks;
+  const int c0 = static_cast<int>(blockIdx.x) * S;  // first column of the strip
+  // CTA b walks K from slab (b * p.gm) mod KC and wraps around, so that the CTAs of a moment do not
+  // all read the same X slab (the same few L2 lines); the order of a strip's fp32 sums is fixed by b.
+  const int k_off = static_cast<int>((static_cast<long long>(blockIdx.x) * p.gm) % KC);
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_x);
+    for (int s = 0; s < stages; ++s) {
+      mbar_init(&full_bar[s], 2);  // the weight producer and the X producer each arm it once
+      mbar_init(&empty_bar[s], 1);
+    }
+    mbar_init(acc_full, 1);
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc<TCOLS>(tmem_slot);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // The three single-thread loops below run once per K slab and pace the whole kernel (a CTA moves a
+  // slab every few hundred cycles), so they carry running counters instead of dividing by `stages`
+  // or KC, and all address arithmetic that does not change with the slab is done up front.
+  if (warp == 0) {
+    // ---------------- weight producer
+    if (lane == 0) {
+      // the strip's rows inside the 128-row blocks it touches: up to three runs of whole 8-row groups
+      const __nv_bfloat16* piece_src[3];
+      uint32_t piece_bytes[3], piece_dst[3];
+      {
+        int row = c0, left = S;
+        uint32_t off = 0;
+#pragma unroll
+        for (int j = 0; j < 3; ++j) {  // S <= 256: at most three blocks
+          const int blk = row >> 7, r0 = row & 127;
+          const int n = left < 128 - r0 ? left : 128 - r0;  // 0 once the strip is covered
+          piece_src[j] = p.w_packed + (static_cast<long long>(blk) * KC * 128 + r0) * 64;
+          piece_bytes[j] = static_cast<uint32_t>(n) * 128u;
+          piece_dst[j] = off;
+          off += static_cast<uint32_t>(n) * 128u;
+          row += n;
+          left -= n;
+        }
+      }
+      int s = 0, kc = k_off;
+      uint32_t ph = 1;  // parity to wait for on the stage's empty barrier (first lap: passes at once)
+      for (int i = 0; i < KC; ++i) {
+        if (i >= stages && !mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
+        mbar_arrive_expect_tx(&full_bar[s], b_stage_bytes);
+        uint8_t* dst = smem_b + static_cast<uint32_t>(s) * b_stage_bytes;
+        const size_t slab = static_cast<size_t>(kc) * (128 * 64);
+#pragma unroll
+        for (int j = 0; j < 3; ++j)
+          if (piece_bytes[j] != 0) bulk_load_1d(dst + piece_dst[j], piece_src[j] + slab, piece_bytes[j], &full_bar[s]);
+        if (++s == stages) { s = 0; ph ^= 1u; }
+        if (++kc == KC) kc = 0;
+      }
+    }
+  } else if (warp == 6) {
+    // ---------------- X producer
+    if (lane == 0) {
+      grid_dep_wait();
+      int s = 0, kc = k_off;
+      uint32_t ph = 1;
+      for (int i = 0; i < KC; ++i) {
+        if (i >= stages && !mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
+        mbar_arrive_expect_tx(&full_bar[s], a_stage_bytes);
+        tma_load_2d(smem_a + static_cast<uint32_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K, 0);
+        if (++s == stages) { s = 0; ph ^= 1u; }
+        if (++kc == KC) kc = 0;
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc(BLOCK_M, S);
+      const uint64_t adesc0 = make_smem_desc(smem_u32(smem_a)), bdesc0 = make_smem_desc(smem_u32(smem_b));
+      const uint64_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;  // stage strides in descriptor units
+      uint64_t adesc = adesc0, bdesc = bdesc0;
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int i = 0; i < KC; ++i) {
+        if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) { ok = false; break; }
+        tc_fence_after();
+#pragma unroll
+        for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk)
+          umma_bf16(tmem_base, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
+                    (i > 0 || kk > 0) ? 1u : 0u);
+        umma_commit(&empty_bar[s]);
+        adesc += a_step;
+        bdesc += b_step;
+        if (++s == stages) { s = 0; ph ^= 1u; adesc = adesc0; bdesc = bdesc0; }
+      }
+      if (ok) umma_commit(acc_full);
+    }
+  } else {
+    // ---------------- epilogue warps: TMEM lane group = warp % 4
+    grid_dep_wait();
+    const int lg = warp & 3;
+    const int row = lg * 32 + lane;
+    bool ok = mbar_wait(acc_full, 0u, abort_flag, p.error_word);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      if (lg * 32 < p.a_rows && lg * 32 < p.M) {
+        TmemSource tsrc{tmem_base + (static_cast<uint32_t>(lg * 32) << 16)};
+        run_epilogue<EPI, 256>(tsrc, p, row, c0, row < p.M, 0, 1, c0 + S);
+      }
+    }
+    tc_fence_before();
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc<TCOLS>(tmem_base);
+  }
+}
+
+inline size_t gemm_strip_smem_bytes(int a_rows, int S, int stages) {
+  size_t body = static_cast<size_t>(stages) * (a_rows * 128 + S * 128);
+  const size_t reach = static_cast<size_t>(stages - 1) * a_rows * 128 + 128 * 128;
+  if (body < reach) body = reach;
+  return 1024 + body + 8 + (2 * stages + 1) * 8 + 64;
 }
 
 inline size_t gemm_tc_smem_bytes(int a_rows, int block_n, int stages) {

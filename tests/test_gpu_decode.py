@@ -241,6 +241,29 @@ def test_padded_batch_equals_single_sequences():
             assert np.max(np.abs(single - batch[b])) <= tol * np.max(np.abs(batch[b]))
 
 
+def test_column_strip_schedule_in_the_forward():
+    """One 32-row block with every skinny matmul forced onto the column-strip kernel (QKV with RoPE and
+    cache writes, gate/up with SwiGLU, the residual matmuls): logits, cache rows and commits agree with
+    the default schedule within the padded-batch bound, and with the oracle within the bf16 bar."""
+    shape = small_bf16(128, 4, 2, "strips")
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("strips", shape, 1, [45], 32, 32, 0.5, 17)
+    model = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
+    blk = np.full((1, 32), shape.mask_id, dtype=np.int32)
+    with Ctx(shape, W, block=32, max_batch=1, max_seq=wl.max_seq) as ctx:
+        ctx.prefill(ids, lens)
+        base = ctx.logits(blk)
+        n0 = d3.d3_launch_count_of(ctx.ctx, "gemm_strip_kernel")
+        d3.d3_set_matmul_tuning(ctx.ctx, 3 << 29, 0)
+        ctx.prefill(ids, lens)
+        forced = ctx.logits(blk)
+        assert d3.d3_launch_count_of(ctx.ctx, "gemm_strip_kernel") >= n0 + 4 * shape.n_layers
+        assert np.max(np.abs(forced - base)) <= 1e-2 * np.max(np.abs(base))
+        rep, _ = step_locked(ctx, model, ids, lens, 32, 32, 0.5, logit_tol=3e-2)
+        assert rep["max_logit_err"] <= 3e-2 and rep["self_diff"] == 0 and rep["unexplained"] == 0
+        assert ctx.error_word() == 0
+
+
 def test_empty_prompt_and_state_errors():
     shape = small_bf16(128, 4, 2, "empty")
     W = si.gen_weights(shape)

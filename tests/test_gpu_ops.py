@@ -102,6 +102,43 @@ def test_linear_bf16_packed_weights(ctx_bf16, m, n, k, splits):
     assert ctx_bf16.error_word() == 0
 
 
+@pytest.mark.parametrize("m,n,k,widths", [(32, 2400, 256, [16, 48, 80, 96, 240]), (64, 2400, 200, [48, 160]),
+                                          (7, 4736, 1024, [32, 128]), (1, 512, 4096, [16, 256])])
+def test_linear_bf16_column_strips(ctx_bf16, m, n, k, widths):
+    """The column-strip kernel (one CTA per strip of S columns, whole K range) against the fp64 product:
+    strips that start and end inside the 128-row weight blocks, span three blocks, end in half a
+    32-column chunk; ragged K; all four epilogues."""
+    rng = np.random.default_rng(m * 13 + n + k)
+    xt, x = rand_bf16(rng, (m, k))
+    wt, w = rand_bf16(rng, (n, k), 0.05)
+    ref = x @ w.T
+    tol = 2e-5 * np.sqrt(k) * np.abs(ref).max() + 1e-6
+    xd, wd = xt.to(DEV), wt.to(DEV)
+    packed = torch.full((d3.d3_packed_weight_elems(n, k),), 3.0, dtype=torch.bfloat16, device=DEV)
+    d3.d3_pack_weight(ctx_bf16.ctx, wd, packed)
+    y0 = rng.standard_normal((m, n)).astype(np.float32)
+    sref = swiglu_ref(ref, n)
+    for S in widths:
+        y = torch.full((m, n), 7.0, dtype=torch.float32, device=DEV)
+        d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, y, n, 0, -S)
+        assert np.max(np.abs(y.cpu().numpy() - ref)) <= tol, S
+        y = torch.from_numpy(y0).to(DEV)
+        d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, y, n, 2, -S)
+        assert np.max(np.abs(y.cpu().numpy() - (ref + y0))) <= tol + 1e-6, S
+        y = torch.zeros((m, n), dtype=torch.bfloat16, device=DEV)
+        d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, y, n, 1, -S)
+        assert np.max(np.abs(y.float().cpu().numpy() - ref)) <= tol + 2 ** -8 * np.abs(ref).max(), S
+        h = torch.zeros((m, n // 2), dtype=torch.bfloat16, device=DEV)
+        d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, h, n, 3, -S)
+        assert np.max(np.abs(h.float().cpu().numpy() - sref)) <= 2 ** -7 * np.abs(sref).max() + 4 * tol, S
+    # widths the kernel cannot take are refused, not rounded
+    y = torch.zeros((m, n), dtype=torch.float32, device=DEV)
+    for bad in (-24, -272, -(n + 16)):
+        with pytest.raises(d3.D3Error):
+            d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, y, n, 0, bad)
+    assert ctx_bf16.error_word() == 0
+
+
 def test_linear_bf16_repeated_launches_keep_split_counters_clean(ctx_bf16):
     rng = np.random.default_rng(3)
     xt, x = rand_bf16(rng, (32, 1024))
