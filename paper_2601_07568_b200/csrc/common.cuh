@@ -31,7 +31,36 @@ struct EpiParams {
   int mask_id = -1;           // EPI_STATS: excluded column
   float4* stat_part = nullptr;  // EPI_STATS: [m][n_tiles]
   int n_tiles = 0;
+  // RMSNorm folded into the tensor-core matmuls.  A residual epilogue also leaves a bf16 copy of the
+  // updated rows (the next matmul's operand) and the sum of squares of every 32-column chunk of them;
+  // a matmul fed with that un-normalised copy multiplies accumulator row m by
+  // rsqrt(sum(ssq_in[m][0 .. ssq_chunks)) * inv_k + rms_eps) (the norm's gains sit in the weight columns).
+  __nv_bfloat16* yb = nullptr;   // EPI_RESID: [m][ldy] bf16 copy of y after the update
+  float* ssq_out = nullptr;      // EPI_RESID: [m][ceil(n / 32)]
+  const float* ssq_in = nullptr; // any epilogue but EPI_RESID: chunk sums of the operand rows
+  int ssq_chunks = 0;
+  float inv_k = 0.f, rms_eps = 0.f;
 };
+
+// Row factor of a matmul whose operand rows were left un-normalised; chunk sums added in index
+// order (the same bits whichever thread or kernel asks).
+__device__ __forceinline__ float row_rstd(const EpiParams& ep, int m) {
+  const float* r = ep.ssq_in + static_cast<size_t>(m) * ep.ssq_chunks;
+  float tot = 0.f;
+  int i = 0;
+  if ((ep.ssq_chunks & 3) == 0) {
+    const float4* r4 = reinterpret_cast<const float4*>(r);
+    for (; i + 16 <= ep.ssq_chunks; i += 16) {  // four independent 16-byte loads in flight
+      const float4 a = __ldcg(r4 + i / 4), b = __ldcg(r4 + i / 4 + 1), c = __ldcg(r4 + i / 4 + 2), d = __ldcg(r4 + i / 4 + 3);
+      tot += a.x; tot += a.y; tot += a.z; tot += a.w;
+      tot += b.x; tot += b.y; tot += b.z; tot += b.w;
+      tot += c.x; tot += c.y; tot += c.z; tot += c.w;
+      tot += d.x; tot += d.y; tot += d.z; tot += d.w;
+    }
+  }
+  for (; i < ep.ssq_chunks; ++i) tot += __ldcg(r + i);
+  return rsqrtf(tot * ep.inv_k + ep.rms_eps);
+}
 
 template <typename T> struct TypeOps;
 template <> struct TypeOps<float> {

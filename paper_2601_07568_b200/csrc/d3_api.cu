@@ -31,6 +31,9 @@ struct d3_ctx {
   bool is_bf16 = false;
   bool use_tc = false;
   bool fuse_qkv = false;
+  bool fold_norm = false;  // tensor-core path: RMSNorm lives inside the matmuls (gains in the weight columns, row factors in the epilogues)
+  void* xb = nullptr;      // bf16 copy of the residual stream (fold_norm)
+  float* ssq = nullptr;    // [rows][ceil(d_model / 32)] chunk sums of squares of x (fold_norm)
   bool w_tiled = false;  // model matrices stored as contiguous 128 x 64 blocks (tensor-core path)
   size_t esz = 4;
   int n_sms = 148;
@@ -399,8 +402,8 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   int stages = static_cast<int>((budget > part_bytes ? budget - part_bytes : 0) / stage_bytes);
   stages = std::max(2, std::min(stages, 16));
   const size_t smem = tc::gemm_ck_smem_bytes(a_rows, stages);
-  const int per_sm = std::max(1, std::min(c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : 2, static_cast<int>((227 * 1024) / (smem + 1024))));
-  const int slots = c->n_sms * per_sm;
+  // cluster launches of this kernel get one CTA per SM, whatever its shared memory
+  const int slots = c->n_sms;
   tc::ClusterSplit cs{1, 1};
   long long best = -1;
   for (int C = 1; C <= 8; ++C) {
@@ -532,14 +535,15 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
                   int ctas_hint, const QkvExtra* qx, int w_tiled) {
   // `ctas_hint` 1..8 on a skinny matmul forces the cluster size; larger hints ask for the unit-range kernel
-  // Few column tiles and a long K (O-proj, down): clusters of 8 that split K and reduce through
-  // distributed shared memory beat the L2 reduction of the unit-range kernel (measured at 32 rows:
-  // 14 vs 17 us and 25 vs 30 us on the 8B shapes); with many tiles the unit-range kernel wins,
-  // because cluster launches of this kernel get one CTA per SM only.
+  // Few column tiles and a long K (O-proj, down): clusters that split K and reduce through
+  // distributed shared memory beat the L2 reduction of the unit-range kernel (measured at 32 rows on
+  // the 8B shapes: 13 vs 16 us and 23 vs 25 us); cluster launches of this kernel get one CTA per SM
+  // only, so the cluster size is chosen for a single wave (run_linear_ck).
   if (M <= 64 && !c->tune_no_cluster) {
     const int T = (N + 127) / 128, KC = (K + 63) / 64;
     if (ctas_hint >= 1 && ctas_hint <= 8) return run_linear_ck(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
-    if (ctas_hint == 0 && T * 8 <= 2 * c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 8, qx, w_tiled);
+    // few enough tiles that every tile gets a cluster of at least two resident CTAs
+    if (ctas_hint == 0 && T * 2 <= c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 0, qx, w_tiled);
   }
   if (ctas_hint < 0) {  // a strip width asked for by name
     const int S = -ctas_hint;
@@ -549,7 +553,8 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   }
   if (ctas_hint == 0 && epi != EPI_STATS) {
     const int S = strip_width(c, M, N, w_tiled);
-    if (S > 0) return run_linear_strip(c, X, W, M, N, K, epi, ep, S, qx);
+    // a residual epilogue that also writes chunk sums of squares needs whole 32-column chunks
+    if (S > 0 && !(ep.ssq_out != nullptr && S % 32 != 0)) return run_linear_strip(c, X, W, M, N, K, epi, ep, S, qx);
   }
   const bool wide = c->tune_wide_tiles >= 0 ? c->tune_wide_tiles != 0 : M >= 512;
   if (wide && N >= 256) return run_linear_tc_bn<256, 1>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
@@ -725,21 +730,39 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     if (c->is_bf16) CUDA_TRY(c, launch_pdl(c, embed_kernel<bf16>, dim3(M), dim3(128), 0, ids, static_cast<const bf16*>(c->tok_emb), c->x, d, g.vocab, c->error_word));
     else CUDA_TRY(c, launch_pdl(c, embed_kernel<float>, dim3(M), dim3(128), 0, ids, static_cast<const float*>(c->tok_emb), c->x, d, g.vocab, c->error_word));
     LAUNCHED(c, "embed_kernel");
+    if (c->fold_norm) {
+      CUDA_TRY(c, launch_pdl(c, row_prep_kernel, dim3(M), dim3(128), 0, static_cast<const float*>(c->x), static_cast<bf16*>(c->xb), c->ssq, d));
+      LAUNCHED(c, "row_prep_kernel");
+    }
   }
+  // Folded RMSNorm: the matmuls after a norm read the bf16 copy of the residual stream and scale
+  // their accumulator rows; the matmuls that update the residual stream refresh the copy and the
+  // chunk sums of squares.
+  const void* normed = c->fold_norm ? c->xb : c->xn;
+  auto after_norm = [&](EpiParams& ep) {
+    if (!c->fold_norm) return;
+    ep.ssq_in = c->ssq; ep.ssq_chunks = (d + 31) / 32; ep.inv_k = 1.0f / static_cast<float>(d); ep.rms_eps = g.rms_eps;
+  };
+  auto updates_resid = [&](EpiParams& ep) {
+    if (!c->fold_norm) return;
+    ep.yb = static_cast<bf16*>(c->xb); ep.ssq_out = c->ssq;
+  };
 
   for (int l = 0; l < g.n_layers; ++l) {
     if (l == c->tap_layer && M <= c->tap_rows)
       CUDA_TRY(c, cudaMemcpyAsync(c->tap_in, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
-    TRY(run_rmsnorm(c, c->x, c->attn_norm[l], c->xn, M));
+    if (!c->fold_norm) TRY(run_rmsnorm(c, c->x, c->attn_norm[l], c->xn, M));
     if (c->fuse_qkv) {
       EpiParams ep;
       ep.y = c->q; ep.ldy = nq;
+      after_norm(ep);
       QkvExtra qx{rm, k_plane(c, l), v_plane(c, l)};
-      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_QKV, ep, 0, &qx, D3_PROF_GEMM_QKV, c->w_tiled));
+      TRY(run_linear(c, normed, c->wqkv[l], M, nq + 2 * nkv, d, EPI_QKV, ep, 0, &qx, D3_PROF_GEMM_QKV, c->w_tiled));
     } else {
       EpiParams ep;
       ep.y = c->qkv_f32; ep.ldy = nq + 2 * nkv;
-      TRY(run_linear(c, c->xn, c->wqkv[l], M, nq + 2 * nkv, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_QKV, c->w_tiled));
+      after_norm(ep);
+      TRY(run_linear(c, normed, c->wqkv[l], M, nq + 2 * nkv, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_QKV, c->w_tiled));
       ProfScope ps(c, D3_PROF_OTHER);
       if (c->is_bf16)
         rope_kv_kernel<bf16><<<M, 256, 0, c->stream>>>(c->qkv_f32, static_cast<bf16*>(c->q), static_cast<bf16*>(k_plane(c, l)), static_cast<bf16*>(v_plane(c, l)), c->rope_cos, c->rope_sin, rm, g.n_q_heads, g.n_kv_heads, g.d_head, g.max_seq, c->error_word);
@@ -751,34 +774,39 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     {
       EpiParams ep;
       ep.y = c->x; ep.ldy = d;
+      updates_resid(ep);
       TRY(run_linear(c, c->o, c->wo[l], M, d, nq, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_O, c->w_tiled));
     }
-    TRY(run_rmsnorm(c, c->x, c->ffn_norm[l], c->xn, M));
+    if (!c->fold_norm) TRY(run_rmsnorm(c, c->x, c->ffn_norm[l], c->xn, M));
     {
       EpiParams ep;
       ep.y = c->h; ep.ldy = f;
-      TRY(run_linear(c, c->xn, c->wgu[l], M, 2 * f, d, EPI_SWIGLU, ep, 0, nullptr, D3_PROF_GEMM_GATE_UP, c->w_tiled));
+      after_norm(ep);
+      TRY(run_linear(c, normed, c->wgu[l], M, 2 * f, d, EPI_SWIGLU, ep, 0, nullptr, D3_PROF_GEMM_GATE_UP, c->w_tiled));
     }
     {
       EpiParams ep;
       ep.y = c->x; ep.ldy = d;
+      updates_resid(ep);
       TRY(run_linear(c, c->h, c->wd[l], M, d, f, EPI_RESID, ep, 0, nullptr, D3_PROF_GEMM_DOWN, c->w_tiled));
     }
     if (l == c->tap_layer && M <= c->tap_rows)
       CUDA_TRY(c, cudaMemcpyAsync(c->tap_out, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
   }
   if (head == 0) return D3_OK;
-  TRY(run_rmsnorm(c, c->x, c->final_norm, c->xn, M));
+  if (!c->fold_norm) TRY(run_rmsnorm(c, c->x, c->final_norm, c->xn, M));
   if (head == 1) {
     const int n_tiles = (g.vocab + 127) / 128;
     EpiParams ep;
     ep.scale = g.logit_scale; ep.mask_id = g.mask_id; ep.stat_part = c->stat_part; ep.n_tiles = n_tiles;
-    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_STATS, ep, 0, nullptr, D3_PROF_GEMM_HEAD, c->w_tiled));
+    after_norm(ep);
+    TRY(run_linear(c, normed, c->lm_head, M, g.vocab, d, EPI_STATS, ep, 0, nullptr, D3_PROF_GEMM_HEAD, c->w_tiled));
     TRY(run_stats_merge(c, M, n_tiles, c->conf, c->ent, c->argmax));
   } else {
     EpiParams ep;
     ep.y = logits; ep.ldy = g.vocab; ep.scale = g.logit_scale;
-    TRY(run_linear(c, c->xn, c->lm_head, M, g.vocab, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_HEAD, c->w_tiled));
+    after_norm(ep);
+    TRY(run_linear(c, normed, c->lm_head, M, g.vocab, d, EPI_F32, ep, 0, nullptr, D3_PROF_GEMM_HEAD, c->w_tiled));
   }
   return D3_OK;
 }
@@ -824,6 +852,7 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   c->use_tc = c->is_bf16 && g.gemm_impl == D3_GEMM_AUTO;
   c->fuse_qkv = c->use_tc && g.d_head == 128;
   c->w_tiled = c->use_tc;
+  c->fold_norm = c->use_tc;
   auto bail = [&](int rc) {
     d3_destroy(c);
     return rc;
@@ -852,6 +881,10 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   A_(c->rope_sin, sizeof(float) * g.max_seq * (g.d_head / 2));
   A_(c->x, sizeof(float) * R * d);
   A_(c->xn, c->esz * R * std::max(d, nq));
+  if (c->fold_norm) {
+    A_(c->xb, sizeof(bf16) * R * d);
+    A_(c->ssq, sizeof(float) * R * ((d + 31) / 32));
+  }
   if (!c->fuse_qkv) A_(c->qkv_f32, sizeof(float) * R * (nq + 2 * nkv));
   A_(c->q, c->esz * R * nq);
   A_(c->o, c->esz * R * nq);
@@ -960,8 +993,13 @@ static size_t stored_elems(const d3_ctx* c, size_t n, size_t k) {
 namespace {
 // Final store of one assembled row-major matrix `rm` [n, k]: tiled blocks on the tensor-core path,
 // a plain copy otherwise (then `rm` already is the final buffer and nothing is done).
-int finish_matrix(d3_ctx* c, const void* rm, void* dst, size_t n, size_t k) {
+int finish_matrix(d3_ctx* c, void* rm, void* dst, size_t n, size_t k, const float* fold_gain = nullptr) {
   if (!c->w_tiled) return D3_OK;
+  if (fold_gain != nullptr && c->fold_norm) {  // the norm in front of this matmul becomes a row factor: its gains go into the columns
+    const size_t total = n * k;
+    scale_columns_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, c->stream>>>(static_cast<bf16*>(rm), fold_gain, total, static_cast<int>(k));
+    TRY(check_launch(c, "scale_columns_kernel"));
+  }
   dim3 grid(static_cast<unsigned>((k + 63) / 64), static_cast<unsigned>((n + 127) / 128));
   pack_tiled_kernel<<<grid, 256, 0, c->stream>>>(static_cast<const bf16*>(rm), static_cast<bf16*>(dst), static_cast<int>(n),
                                                  static_cast<int>(k));
@@ -1010,10 +1048,12 @@ extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device
   auto step = [&](int r) { if (rc == D3_OK) rc = r; };
   auto target = [&](void* final_buf) { return c->w_tiled ? rm : final_buf; };
   step(upload(c, c->tok_emb, w->tok_emb, V * d * e, src_is_device));
-  step(upload(c, target(c->lm_head), w->lm_head, V * d * e, src_is_device));
-  step(finish_matrix(c, rm, c->lm_head, V, d));
   step(load_gain(c, &c->final_norm, w->final_norm, src_is_device, tgain));
+  step(upload(c, target(c->lm_head), w->lm_head, V * d * e, src_is_device));
+  step(finish_matrix(c, rm, c->lm_head, V, d, c->final_norm));
   for (int l = 0; l < g.n_layers && rc == D3_OK; ++l) {
+    step(load_gain(c, &c->attn_norm[l], w->attn_norm ? w->attn_norm[l] : nullptr, src_is_device, tgain));
+    step(load_gain(c, &c->ffn_norm[l], w->ffn_norm ? w->ffn_norm[l] : nullptr, src_is_device, tgain));
     // ---- q, k (rows permuted so that each RoPE pair of a head is adjacent) and v
     char* qkv = static_cast<char*>(target(c->wqkv[l]));
     for (int which = 0; which < 2 && rc == D3_OK; ++which) {
@@ -1028,7 +1068,7 @@ extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device
       step(check_launch(c, "pack_rope_rows_kernel"));
     }
     step(upload(c, qkv + (nq + nkv) * d * e, w->wv[l], nkv * d * e, src_is_device));
-    step(finish_matrix(c, rm, c->wqkv[l], nq + 2 * nkv, d));
+    step(finish_matrix(c, rm, c->wqkv[l], nq + 2 * nkv, d, c->attn_norm[l]));
     // ---- o, down: as given
     step(upload(c, target(c->wo[l]), w->wo[l], d * nq * e, src_is_device));
     step(finish_matrix(c, rm, c->wo[l], d, nq));
@@ -1045,9 +1085,7 @@ extern "C" int d3_load_weights(d3_ctx* c, const d3_weights* w, int src_is_device
         interleave_gate_up_kernel<float><<<static_cast<unsigned>(2 * f), 128, 0, c->stream>>>(static_cast<const float*>(tg), static_cast<const float*>(tu), static_cast<float*>(gu), g.d_ffn, g.d_model);
       step(check_launch(c, "interleave_gate_up_kernel"));
     }
-    step(finish_matrix(c, rm, c->wgu[l], 2 * f, d));
-    step(load_gain(c, &c->attn_norm[l], w->attn_norm ? w->attn_norm[l] : nullptr, src_is_device, tgain));
-    step(load_gain(c, &c->ffn_norm[l], w->ffn_norm ? w->ffn_norm[l] : nullptr, src_is_device, tgain));
+    step(finish_matrix(c, rm, c->wgu[l], 2 * f, d, c->ffn_norm[l]));
     // the staging buffers are reused by the next matrix: everything above is stream-ordered
   }
   cudaError_t es = cudaStreamSynchronize(c->stream);

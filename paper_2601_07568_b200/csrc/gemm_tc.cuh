@@ -135,9 +135,11 @@ struct PartialSource {
 // takes them all (0, 1), the partial-sum path spreads them over the threads that share a row.
 // `n_end` >= 0 ends the tile before column n_end (a column strip narrower than BLOCK_N; a multiple of
 // 16, so the last chunk may be half a chunk); otherwise the tile ends with the matrix.
+// `rs` multiplies the accumulator row first (the RMSNorm factor of row m when the operand was the
+// un-normalised residual copy, see EpiParams; 1 otherwise).
 template <int EPI, int BLOCK_N, typename Source>
 __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams& p, int m, int n0, bool live,
-                                             int c_first = 0, int c_stride = 1, int n_end = -1) {
+                                             int c_first = 0, int c_stride = 1, int n_end = -1, float rs = 1.f) {
   const int N = n_end >= 0 ? n_end : p.N;
   if constexpr (EPI == EPI_F32 || EPI == EPI_RESID) {
     float* y = static_cast<float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
@@ -145,31 +147,55 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       if (n0 + c >= N) break;
       float v[32];
       src.load(c, v);
-      const bool vec = (n0 + c + 32 <= N) && ((p.ep.ldy & 3) == 0);
+      const bool vec = (n0 + c + 32 <= N) && ((p.ep.ldy & 7) == 0);
       if (!live) continue;
+      const float sc = p.ep.scale * rs;
+      float sq = 0.f;  // EPI_RESID: sum of squares of this chunk of the updated row
       if (vec) {
         float4* y4 = reinterpret_cast<float4*>(y + n0 + c);
+        if constexpr (EPI == EPI_RESID) {
+          float4 o[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          float4 o;
-          if constexpr (EPI == EPI_RESID) {
-            o = y4[j];
-            o.x += v[4 * j]; o.y += v[4 * j + 1]; o.z += v[4 * j + 2]; o.w += v[4 * j + 3];
-          } else {
-            o = make_float4(v[4 * j] * p.ep.scale, v[4 * j + 1] * p.ep.scale, v[4 * j + 2] * p.ep.scale,
-                            v[4 * j + 3] * p.ep.scale);
+          for (int j = 0; j < 8; ++j) o[j] = y4[j];  // all eight loads in flight
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            o[j].x += v[4 * j]; o[j].y += v[4 * j + 1]; o[j].z += v[4 * j + 2]; o[j].w += v[4 * j + 3];
+            y4[j] = o[j];
+            sq += o[j].x * o[j].x; sq += o[j].y * o[j].y; sq += o[j].z * o[j].z; sq += o[j].w * o[j].w;
           }
-          y4[j] = o;
+          if (p.ep.yb != nullptr) {
+            uint4* b4 = reinterpret_cast<uint4*>(p.ep.yb + static_cast<size_t>(m) * p.ep.ldy + n0 + c);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              __nv_bfloat162 a = __floats2bfloat162_rn(o[2 * j].x, o[2 * j].y), b = __floats2bfloat162_rn(o[2 * j].z, o[2 * j].w);
+              __nv_bfloat162 cc = __floats2bfloat162_rn(o[2 * j + 1].x, o[2 * j + 1].y), d = __floats2bfloat162_rn(o[2 * j + 1].z, o[2 * j + 1].w);
+              b4[j] = make_uint4(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b),
+                                 *reinterpret_cast<uint32_t*>(&cc), *reinterpret_cast<uint32_t*>(&d));
+            }
+          }
+        } else {
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            y4[j] = make_float4(v[4 * j] * sc, v[4 * j + 1] * sc, v[4 * j + 2] * sc, v[4 * j + 3] * sc);
         }
       } else {
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           int n = n0 + c + j;
           if (n < N) {
-            if constexpr (EPI == EPI_RESID) y[n] += v[j];
-            else y[n] = v[j] * p.ep.scale;
+            if constexpr (EPI == EPI_RESID) {
+              const float o = y[n] + v[j];
+              y[n] = o;
+              sq += o * o;
+              if (p.ep.yb != nullptr) p.ep.yb[static_cast<size_t>(m) * p.ep.ldy + n] = __float2bfloat16_rn(o);
+            } else {
+              y[n] = v[j] * sc;
+            }
           }
         }
+      }
+      if constexpr (EPI == EPI_RESID) {
+        if (p.ep.ssq_out != nullptr) p.ep.ssq_out[static_cast<size_t>(m) * ((p.N + 31) / 32) + (n0 + c) / 32] = sq;
       }
     }
   } else if constexpr (EPI == EPI_T) {
@@ -179,6 +205,8 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       float v[32];
       src.load(c, v);
       if (!live) continue;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] *= rs;
       if ((n0 + c + 32 <= N) && ((p.ep.ldy & 7) == 0)) {
         uint4* y4 = reinterpret_cast<uint4*>(y + n0 + c);
 #pragma unroll
@@ -207,6 +235,8 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       float v[32];
       src.load(c, v);
       if (!live) continue;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] *= rs;
       const int h0 = (n0 + c) / 2;
       if (h0 + 16 <= F && (p.ep.ldy & 7) == 0) {
         uint32_t w[8];
@@ -244,7 +274,7 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
           int n = n0 + g + c + j;
-          if (n < N && n != p.ep.mask_id) stat_add(st, v[j] * p.ep.scale, n);
+          if (n < N && n != p.ep.mask_id) stat_add(st, v[j] * (p.ep.scale * rs), n);
         }
       }
       int t = (n0 + g) / 128;
@@ -274,6 +304,8 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       float v[32];
       src.load(c, v);
       if (!live) continue;
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] *= rs;
       // two halves of 16 columns: a chunk that starts 16 columns before a head border spans two heads
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
@@ -571,11 +603,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         }
         *list_len = n_list;
       }
+      const int rows_pad = p.a_rows < 128 ? p.a_rows : 128;  // rows of one row tile that can be live
+      // Row factors (folded RMSNorm) of the rows this thread may finish, fetched while the MMAs of the
+      // segment still run: its TMEM lane's row for a whole tile, row et % rows_pad when the partial
+      // sums of a split tile are spread over the threads.
+      float rs_tmem[MT], rs_part[MT];
+#pragma unroll
+      for (int mt = 0; mt < MT; ++mt) {
+        rs_tmem[mt] = 1.f;
+        rs_part[mt] = 1.f;
+        if (p.ep.ssq_in != nullptr) {
+          const int m_tile = m_group * MT + mt;
+          if (n_k == KC || EPI == EPI_STATS) {
+            const int m = m_tile * BLOCK_M + row;
+            if (lg * 32 < rows_pad && m < p.M) rs_tmem[mt] = row_rstd(p.ep, m);
+          } else {
+            const int m2 = m_tile * BLOCK_M + et % rows_pad;
+            if (et / rows_pad < 128 / rows_pad && m2 < p.M) rs_part[mt] = row_rstd(p.ep, m2);
+          }
+        }
+      }
       bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
-      const int rows_pad = p.a_rows < 128 ? p.a_rows : 128;  // rows of one row tile that can be live
       const uint32_t tmem_seg = tmem_base + static_cast<uint32_t>(buf * MT * BLOCK_N) + (static_cast<uint32_t>(lg * 32) << 16);
       if (n_k == KC) {
 #pragma unroll
@@ -585,7 +636,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
           // warp-uniform: does this lane group hold any row of X at all?
           const bool warp_live = (lg * 32 < rows_pad) && (m_tile * BLOCK_M + lg * 32 < p.M);
           TmemSource tsrc{tmem_seg + static_cast<uint32_t>(mt * BLOCK_N)};
-          if (warp_live) run_epilogue<EPI, BLOCK_N>(tsrc, p, m, n0, m < p.M);
+          if (warp_live) run_epilogue<EPI, BLOCK_N>(tsrc, p, m, n0, m < p.M, 0, 1, -1, rs_tmem[mt]);
         }
         tc_fence_before();
         mbar_arrive(&acc_empty[buf]);
@@ -631,7 +682,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
             if (warp_live) {
               const int m = m_tile * BLOCK_M + row;
               PartialSource<MT * BLOCK_N> psrc{p.partial, seg_slots, n_seg, row, mt * BLOCK_N};
-              run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, m < p.M);
+              run_epilogue<EPI, BLOCK_N>(psrc, p, m, n0, m < p.M, 0, 1, -1, rs_tmem[mt]);
             }
           } else {
             // the sums come from memory, not from TMEM lanes: spread (row, 32-column chunk) pairs over
@@ -641,7 +692,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
             if (part < tpr) {
               const int m2 = m_tile * BLOCK_M + prow;
               PartialSource<MT * BLOCK_N> psrc{p.partial, seg_slots, n_seg, prow, mt * BLOCK_N};
-              run_epilogue<EPI, BLOCK_N>(psrc, p, m2, n0, m2 < p.M, part, tpr);
+              run_epilogue<EPI, BLOCK_N>(psrc, p, m2, n0, m2 < p.M, part, tpr, -1, rs_part[mt]);
             }
           }
         }
@@ -849,6 +900,15 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     // (row, 32-column chunk) pairs of this CTA's slice: chunks rank, rank + C, ... (< 4)
     const int tpr = 128 / p.a_rows;  // threads that can share a row: 4 or 2
     const int prow = et % p.a_rows, sub = et / p.a_rows;
+    // row factors (folded RMSNorm): fetched now, while the first accumulator is still being built
+    float rs_row = 1.f, rs_prow = 1.f;
+    if (p.ep.ssq_in != nullptr) {
+      if constexpr (EPI == EPI_STATS) {
+        if (rank == 0 && warp_live && row < p.M) rs_row = row_rstd(p.ep, row);
+      } else {
+        if (sub < tpr && prow < p.M) rs_prow = row_rstd(p.ep, prow);
+      }
+    }
     bool alive = true;
     int seg = 0;
     for (int t = t0; t < t1; ++t, ++seg) {
@@ -880,7 +940,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         // one statistic per (row, 128 columns): rank 0 takes the whole tile, a row stays with one thread
         if (rank == 0 && warp_live) {
           DsmemSource dsrc{part_addr, C, p.a_rows, row};
-          run_epilogue<EPI, BLOCK_N>(dsrc, p, row, n0, row < p.M);
+          run_epilogue<EPI, BLOCK_N>(dsrc, p, row, n0, row < p.M, 0, 1, -1, rs_row);
         }
       } else {
         // chunk list of this rank, spread over the threads that share a row
@@ -889,7 +949,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         if (sub < tpr && sub < my_chunks) {
           DsmemSource dsrc{part_addr, C, p.a_rows, prow};
           // chunk indices rank + C * (sub + tpr * q): first = rank + C * sub, stride = C * tpr
-          run_epilogue<EPI, BLOCK_N>(dsrc, p, prow, n0, prow < p.M, rank + C * sub, C * tpr);
+          run_epilogue<EPI, BLOCK_N>(dsrc, p, prow, n0, prow < p.M, rank + C * sub, C * tpr, -1, rs_prow);
         }
       }
       epi_bar_sync();  // this CTA has read all it needs from every peer
@@ -1054,13 +1114,16 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p
     grid_dep_wait();
     const int lg = warp & 3;
     const int row = lg * 32 + lane;
+    const bool warp_live = lg * 32 < p.a_rows && lg * 32 < p.M;
+    // row factor (folded RMSNorm): fetched while the accumulator is still being built
+    const float rs = (warp_live && row < p.M && p.ep.ssq_in != nullptr) ? row_rstd(p.ep, row) : 1.f;
     bool ok = mbar_wait(acc_full, 0u, abort_flag, p.error_word);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after();
-      if (lg * 32 < p.a_rows && lg * 32 < p.M) {
+      if (warp_live) {
         TmemSource tsrc{tmem_base + (static_cast<uint32_t>(lg * 32) << 16)};
-        run_epilogue<EPI, 256>(tsrc, p, row, c0, row < p.M, 0, 1, c0 + S);
+        run_epilogue<EPI, 256>(tsrc, p, row, c0, row < p.M, 0, 1, c0 + S, rs);
       }
     }
     tc_fence_before();

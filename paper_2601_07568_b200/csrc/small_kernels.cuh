@@ -40,6 +40,36 @@ __global__ void embed_kernel(const int* __restrict__ ids, const T* __restrict__ 
   for (int i = threadIdx.x; i < d; i += blockDim.x) dst[i] = TypeOps<T>::to_f(src[i]);
 }
 
+// ----------------------------------------------------------------------------- folded RMSNorm helpers
+// What a residual epilogue leaves behind for the next matmul (see EpiParams), for rows that no matmul
+// has written yet (the embeddings): bf16 copy of x and the sum of squares of every 32-column chunk.
+// One block per row; thread t takes chunks t, t + blockDim.x, ...
+__global__ void row_prep_kernel(const float* __restrict__ x, __nv_bfloat16* __restrict__ xb, float* __restrict__ ssq, int d) {
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
+  const int m = blockIdx.x;
+  const int n_chunks = (d + 31) / 32;
+  const float* row = x + static_cast<size_t>(m) * d;
+  __nv_bfloat16* out = xb + static_cast<size_t>(m) * d;
+  for (int ch = threadIdx.x; ch < n_chunks; ch += blockDim.x) {
+    float sq = 0.f;
+    const int e1 = min(d, ch * 32 + 32);
+    for (int e = ch * 32; e < e1; ++e) {  // same element order as the matmul epilogue's chunk sum
+      const float v = row[e];
+      sq += v * v;
+      out[e] = __float2bfloat16_rn(v);
+    }
+    ssq[static_cast<size_t>(m) * n_chunks + ch] = sq;
+  }
+}
+
+// w[n, k] *= gain[k] (rounded to bf16 once): the gains of the RMSNorm in front of a matmul, moved
+// into its weight columns when the weights are loaded.
+__global__ void scale_columns_kernel(__nv_bfloat16* __restrict__ w, const float* __restrict__ gain, size_t total, int k) {
+  const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i < total) w[i] = __float2bfloat16_rn(__bfloat162float(w[i]) * gain[i % k]);
+}
+
 // ----------------------------------------------------------------------------- RMSNorm
 // xn[m, :] = T(x[m, :] * rsqrt(mean(x^2) + eps) * gain); fp32 arithmetic, fixed reduction order.
 // One 256-thread block per row; d % 4 == 0.  The row is read once as float4 and the first 4096
