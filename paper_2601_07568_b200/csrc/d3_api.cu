@@ -402,19 +402,28 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   int stages = static_cast<int>((budget > part_bytes ? budget - part_bytes : 0) / stage_bytes);
   stages = std::max(2, std::min(stages, 16));
   const size_t smem = tc::gemm_ck_smem_bytes(a_rows, stages);
-  // cluster launches of this kernel get one CTA per SM, whatever its shared memory
+  // Cluster launches of this kernel get one CTA per SM, whatever its shared memory.  The kernel is
+  // paced by its single-thread pipeline loops (a fixed time per K slab), so what counts is the number
+  // of slabs a CTA walks through.  Either the clusters are all resident and loop over their tiles, or
+  // every tile gets its own cluster and the grid runs in waves; a later wave overlaps the tail of the
+  // one before it (measured: about three quarters of its length is added).
   const int slots = c->n_sms;
   tc::ClusterSplit cs{1, 1};
   long long best = -1;
   for (int C = 1; C <= 8; ++C) {
     if (C > KC) break;
     if (c_hint > 0 && C != c_hint) continue;
-    const int n_cl = std::max(1, std::min(slots / C, T));
-    const long long cost = static_cast<long long>((T + n_cl - 1) / n_cl) * ((KC + C - 1) / C) * 16 + C;  // ties: smaller clusters
+    const long long slabs = (KC + C - 1) / C;
+    const int n_res = std::max(1, std::min(slots / C, T));
+    const long long cost_res = static_cast<long long>((T + n_res - 1) / n_res) * slabs * 16;
+    const long long waves = (static_cast<long long>(T) * C + slots - 1) / slots;
+    const long long cost_waves = slabs * (4 + 3 * (waves - 1)) * 4;  // slabs * (1 + 0.75 (waves - 1)) * 16
+    const bool by_waves = cost_waves < cost_res;
+    const long long cost = (by_waves ? cost_waves : cost_res) + C;  // ties: smaller clusters
     if (best < 0 || cost < best) {
       best = cost;
       cs.C = C;
-      cs.n_clusters = n_cl;
+      cs.n_clusters = by_waves ? T : n_res;
     }
   }
   tc::GemmParams p{};
@@ -479,13 +488,14 @@ int strip_width(const d3_ctx* c, int M, int N, int w_tiled) {
 template <int EPI>
 int launch_strip(d3_ctx* c, const CUtensorMap* tx, const tc::GemmParams& p, int S, int n_ctas, size_t smem) {
   static bool attr_set[2] = {false, false};
-  const int wide = S > 128 ? 1 : 0;
+  // tensor memory: one accumulator of S columns per pipeline, the second one half way up
+  const int wide = S * p.n_producers > 128 ? 1 : 0;
   auto kern = wide ? tc::gemm_strip_kernel<EPI, 256> : tc::gemm_strip_kernel<EPI, 128>;
   if (!attr_set[wide]) {
     CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
     attr_set[wide] = true;
   }
-  CUDA_TRY(c, launch_pdl(c, kern, dim3(n_ctas), dim3(tc::NUM_THREADS), smem, *tx, p, S));
+  CUDA_TRY(c, launch_pdl(c, kern, dim3(n_ctas), dim3(tc::STRIP_THREADS), smem, *tx, p, S));
   LAUNCHED(c, "gemm_strip_kernel");
   return D3_OK;
 }
@@ -510,6 +520,8 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   p.w_packed = static_cast<const bf16*>(W);
   p.w_blocks = static_cast<long long>((N + 127) / 128) * KC;
   p.gm = 1;  // K walk of CTA b starts at slab b mod KC
+  // two issue pipelines per CTA while both accumulators fit 256 tensor-memory columns
+  p.n_producers = (S <= 128 && KC >= 4 && c->tune_producers != 1) ? 2 : 1;
   p.ep = ep;
   if (qx) {
     p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;

@@ -982,11 +982,36 @@ inline size_t gemm_ck_smem_bytes(int a_rows, int stages) {
 // is that every CTA reads all of X (from L2), which the host accepts while S >= rows of X.
 // Weights must be in the tiled form: strip rows are a run of whole 8-row swizzle groups inside the
 // 128-row blocks, copied with one bulk copy per block touched.
-// Warp 0 streams weights (never waits for the previous kernel), warp 6 waits for the previous kernel
-// and streams X slabs, warp 1 issues the MMAs (128 x S x 16) into one accumulator, warps 2-5 run the
-// epilogue.  Shared memory: [stages x a_rows x 128 B] X, [stages x S x 128 B] W, barriers.
+//
+// A CTA moves a K slab every few hundred cycles, and what paces it is the latency of the dependent
+// instructions one thread executes per slab (barrier wait, copy or MMA issue, commit), not bandwidth.
+// So the slabs are dealt to p.n_producers (1 or 2) independent pipelines, slab i to pipeline
+// i mod n: each has a producer thread (weights, then after the dependency wait X slabs), an
+// MMA-issuing thread and its own TMEM accumulator; they share the stage ring, and the epilogue
+// adds the accumulators (pipeline 0 first: fixed order).  Producer / MMA warps: 0 / 1 and 6 / 7;
+// warps 2-5 run the epilogue.  Shared memory: [stages x a_rows x 128 B] X, [stages x S x 128 B] W,
+// barriers.
+constexpr int STRIP_THREADS = 256;
+
+// The sum of two accumulators, pipeline 0 first.
+struct TmemPairSource {
+  uint32_t taddr_row0, taddr_row1;
+  bool two;
+  __device__ __forceinline__ void load(int c, float (&v)[32]) const {
+    tmem_ld_32x32(taddr_row0 + static_cast<uint32_t>(c), v);
+    tmem_ld_wait();
+    if (two) {
+      float w[32];
+      tmem_ld_32x32(taddr_row1 + static_cast<uint32_t>(c), w);
+      tmem_ld_wait();
+#pragma unroll
+      for (int j = 0; j < 32; ++j) v[j] += w[j];
+    }
+  }
+};
+
 template <int EPI, int TCOLS>
-__global__ void __launch_bounds__(NUM_THREADS, 2)
+__global__ void __launch_bounds__(STRIP_THREADS, 2)
 gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p, const int S) {
   if (p.skip_flag != nullptr && *p.skip_flag != 0) return;
   grid_dep_launch();
@@ -1009,6 +1034,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int KC = p.k_chunks;
+  const int n_pipe = p.n_producers;                  // 1 or 2; the host gives 2 only when 2 * S <= TCOLS and KC >= 2
   const int c0 = static_cast<int>(blockIdx.x) * S;  // first column of the strip
   // CTA b walks K from slab (b * p.gm) mod KC and wraps around, so that the CTAs of a moment do not
   // all read the same X slab (the same few L2 lines); the order of a strip's fp32 sums is fixed by b.
@@ -1017,10 +1043,10 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmap_x);
     for (int s = 0; s < stages; ++s) {
-      mbar_init(&full_bar[s], 2);  // the weight producer and the X producer each arm it once
+      mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
     }
-    mbar_init(acc_full, 1);
+    mbar_init(acc_full, static_cast<uint32_t>(n_pipe));  // one commit per pipeline
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -1033,11 +1059,11 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  // The three single-thread loops below run once per K slab and pace the whole kernel (a CTA moves a
-  // slab every few hundred cycles), so they carry running counters instead of dividing by `stages`
-  // or KC, and all address arithmetic that does not change with the slab is done up front.
-  if (warp == 0) {
-    // ---------------- weight producer
+  // The single-thread loops below carry running counters instead of dividing by `stages` or KC, and
+  // all address arithmetic that does not change with the slab is done up front.
+  const int pipe = (warp == 0 || warp == 1) ? 0 : 1;
+  if ((warp == 0 || warp == 6) && pipe < n_pipe) {
+    // ---------------- producer of pipeline `pipe`: slabs pipe, pipe + n_pipe, ...
     if (lane == 0) {
       // the strip's rows inside the 128-row blocks it touches: up to three runs of whole 8-row groups
       const __nv_bfloat16* piece_src[3];
@@ -1057,72 +1083,82 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p
           left -= n;
         }
       }
-      int s = 0, kc = k_off;
-      uint32_t ph = 1;  // parity to wait for on the stage's empty barrier (first lap: passes at once)
-      for (int i = 0; i < KC; ++i) {
-        if (i >= stages && !mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
-        mbar_arrive_expect_tx(&full_bar[s], b_stage_bytes);
+      auto load_w = [&](int s, int kc) {  // arms the stage with all the bytes that will arrive, then the weights
+        mbar_arrive_expect_tx(&full_bar[s], a_stage_bytes + b_stage_bytes);
         uint8_t* dst = smem_b + static_cast<uint32_t>(s) * b_stage_bytes;
         const size_t slab = static_cast<size_t>(kc) * (128 * 64);
 #pragma unroll
         for (int j = 0; j < 3; ++j)
           if (piece_bytes[j] != 0) bulk_load_1d(dst + piece_dst[j], piece_src[j] + slab, piece_bytes[j], &full_bar[s]);
-        if (++s == stages) { s = 0; ph ^= 1u; }
-        if (++kc == KC) kc = 0;
-      }
-    }
-  } else if (warp == 6) {
-    // ---------------- X producer
-    if (lane == 0) {
-      grid_dep_wait();
-      int s = 0, kc = k_off;
-      uint32_t ph = 1;
-      for (int i = 0; i < KC; ++i) {
-        if (i >= stages && !mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
-        mbar_arrive_expect_tx(&full_bar[s], a_stage_bytes);
+      };
+      auto load_x = [&](int s, int kc) {
         tma_load_2d(smem_a + static_cast<uint32_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K, 0);
-        if (++s == stages) { s = 0; ph ^= 1u; }
-        if (++kc == KC) kc = 0;
+      };
+      auto wrap_kc = [&](int kc) { return kc >= KC ? kc - KC : kc; };
+      const int pre = KC < stages ? KC : stages;  // slabs of the first lap: their stages are free
+      // weights of the first lap: they do not depend on the kernels before this one
+      int kc = wrap_kc(k_off + pipe);
+      for (int i = pipe; i < pre; i += n_pipe) {
+        load_w(i, kc);
+        kc = wrap_kc(kc + n_pipe);
+      }
+      grid_dep_wait();
+      kc = wrap_kc(k_off + pipe);
+      int i = pipe;
+      for (; i < pre; i += n_pipe) {
+        load_x(i, kc);
+        kc = wrap_kc(kc + n_pipe);
+      }
+      int s = i - stages;          // slab i >= stages lives in stage i mod stages (i < stages + n_pipe here)
+      uint32_t ph = 0;             // parity of the empty barrier's completed phase to wait for
+      for (; i < KC; i += n_pipe) {
+        if (!mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
+        load_w(s, kc);
+        load_x(s, kc);
+        kc = wrap_kc(kc + n_pipe);
+        s += n_pipe;
+        if (s >= stages) { s -= stages; ph ^= 1u; }
       }
     }
-  } else if (warp == 1) {
-    // ---------------- MMA issuer
+  } else if ((warp == 1 || warp == 7) && pipe < n_pipe) {
+    // ---------------- MMA issuer of pipeline `pipe`
     if (lane == 0) {
       const uint32_t idesc = make_idesc(BLOCK_M, S);
       const uint64_t adesc0 = make_smem_desc(smem_u32(smem_a)), bdesc0 = make_smem_desc(smem_u32(smem_b));
       const uint64_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;  // stage strides in descriptor units
-      uint64_t adesc = adesc0, bdesc = bdesc0;
-      int s = 0;
+      const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(pipe * (TCOLS / 2));
+      int s = pipe;
       uint32_t ph = 0;
       bool ok = true;
-      for (int i = 0; i < KC; ++i) {
+      for (int i = pipe; i < KC; i += n_pipe) {
         if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) { ok = false; break; }
         tc_fence_after();
+        const uint64_t adesc = adesc0 + a_step * static_cast<uint64_t>(s), bdesc = bdesc0 + b_step * static_cast<uint64_t>(s);
 #pragma unroll
         for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk)
-          umma_bf16(tmem_base, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
-                    (i > 0 || kk > 0) ? 1u : 0u);
+          umma_bf16(tmem_d, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), idesc,
+                    (i > pipe || kk > 0) ? 1u : 0u);
         umma_commit(&empty_bar[s]);
-        adesc += a_step;
-        bdesc += b_step;
-        if (++s == stages) { s = 0; ph ^= 1u; adesc = adesc0; bdesc = bdesc0; }
+        s += n_pipe;
+        if (s >= stages) { s -= stages; ph ^= 1u; }
       }
       if (ok) umma_commit(acc_full);
     }
-  } else {
+  } else if (warp >= 2 && warp <= 5) {
     // ---------------- epilogue warps: TMEM lane group = warp % 4
     grid_dep_wait();
     const int lg = warp & 3;
     const int row = lg * 32 + lane;
     const bool warp_live = lg * 32 < p.a_rows && lg * 32 < p.M;
-    // row factor (folded RMSNorm): fetched while the accumulator is still being built
+    // row factor (folded RMSNorm): fetched while the accumulators are still being built
     const float rs = (warp_live && row < p.M && p.ep.ssq_in != nullptr) ? row_rstd(p.ep, row) : 1.f;
     bool ok = mbar_wait(acc_full, 0u, abort_flag, p.error_word);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after();
       if (warp_live) {
-        TmemSource tsrc{tmem_base + (static_cast<uint32_t>(lg * 32) << 16)};
+        const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16);
+        TmemPairSource tsrc{lane_addr, lane_addr + static_cast<uint32_t>(TCOLS / 2), n_pipe == 2};
         run_epilogue<EPI, 256>(tsrc, p, row, c0, row < p.M, 0, 1, c0 + S, rs);
       }
     }
