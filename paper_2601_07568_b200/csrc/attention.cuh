@@ -147,18 +147,27 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // with the 128-byte swizzle (slab base 1024-byte aligned).
 __device__ __forceinline__ uint32_t swz(int r, int c) { return static_cast<uint32_t>(r * 128 + ((c ^ (r & 7)) << 4)); }
 
-// grid (q_tiles, bs * hkv, n_splits); NW warps of 16 packed rows each.
-template <int NW>
-__global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_kv,
-                                                          const AttnTcParams p) {
+// grid (q_tiles, bs * hkv, n_splits); NW groups of 16 packed rows, each worked on by KQ warps that
+// take KT / KQ keys of every tile (a decode-sized CTA would otherwise keep two of the SM's four
+// tensor-core partitions idle and walk through its tiles four times as long).  Warp w: row group
+// w % NW, key part w / NW.  Every warp keeps its own running softmax state; the key parts are
+// merged through shared memory after the last tile, then the key splits across the cluster.
+template <int NW, int KQ>
+__global__ void __launch_bounds__(NW * KQ * 32) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_kv,
+                                                               const AttnTcParams p) {
   constexpr int BM = NW * 16;
+  constexpr int KPW = KT / KQ;  // keys per warp and tile: 64, 32 or 16
+  constexpr int NTHREADS = NW * KQ * 32;
+  static_assert(KPW % 16 == 0, "a warp takes whole 16-key MMA steps");
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + TC_STAGES * STAGE_BYTES);
   uint64_t* empty_bar = full_bar + TC_STAGES;
   volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + TC_STAGES);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp_id = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = warp_id % NW;  // row group
+  const int kq = warp_id / NW;    // key part
   const int g4 = lane >> 2, t4 = lane & 3;
   const int qt = blockIdx.x, pair = blockIdx.y, split = blockIdx.z;
   const int b = pair / p.hkv, g = pair % p.hkv;
@@ -169,7 +178,7 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     ptx::prefetch_tensormap(&tmap_kv);
     for (int s = 0; s < TC_STAGES; ++s) {
       ptx::mbar_init(&full_bar[s], 1);
-      ptx::mbar_init(&empty_bar[s], NW);
+      ptx::mbar_init(&empty_bar[s], NW * KQ);
     }
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -249,11 +258,11 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     const int j0 = (t0 + i) * KT;
 
     // ---- S = Q K^T for 64 keys: 8 key groups of 8, 8 k-steps of 16 over d_head
-    float sc[8][4];
+    float sc[KPW / 8][4];
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
+    for (int n = 0; n < KPW / 8; ++n) {
       sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
-      const int key = n * 8 + lm_row;
+      const int key = kq * KPW + n * 8 + lm_row;
 #pragma unroll
       for (int half = 0; half < 2; ++half) {      // K lo slab (dims 0-63), K hi slab (dims 64-127)
 #pragma unroll
@@ -269,8 +278,8 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     // ---- scale, mask keys beyond kv_len, online softmax (rows g4 and g4 + 8)
     float mx_lo = -INFINITY, mx_hi = -INFINITY;
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      const int key = j0 + n * 8 + t4 * 2;
+    for (int n = 0; n < KPW / 8; ++n) {
+      const int key = j0 + kq * KPW + n * 8 + t4 * 2;
       const bool v0 = key < kv_len, v1 = key + 1 < kv_len;
       sc[n][0] = v0 ? sc[n][0] * p.scale_log2 : -INFINITY;
       sc[n][1] = v1 ? sc[n][1] * p.scale_log2 : -INFINITY;
@@ -283,16 +292,19 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     mx_lo = fmaxf(mx_lo, __shfl_xor_sync(0xffffffffu, mx_lo, 2));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 1));
     mx_hi = fmaxf(mx_hi, __shfl_xor_sync(0xffffffffu, mx_hi, 2));
-    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);  // finite: every tile holds a valid key
-    const float c_lo = exp2f(m_lo - mn_lo), c_hi = exp2f(m_hi - mn_hi);
+    // a key part of the last tile may lie wholly beyond kv_len: the maximum then stays -inf, and the
+    // exponentials are taken against 0 so that they come out as 0 instead of NaN
+    const float mn_lo = fmaxf(m_lo, mx_lo), mn_hi = fmaxf(m_hi, mx_hi);
+    const float b_lo = mn_lo == -INFINITY ? 0.f : mn_lo, b_hi = mn_hi == -INFINITY ? 0.f : mn_hi;
+    const float c_lo = exp2f(m_lo - b_lo), c_hi = exp2f(m_hi - b_hi);
     m_lo = mn_lo;
     m_hi = mn_hi;
     float s_lo = 0.f, s_hi = 0.f;
-    uint32_t pa[4][4];  // P as A fragments: 4 k-steps of 16 keys
+    uint32_t pa[KPW / 16][4];  // P as A fragments: k-steps of 16 keys
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
-      const float p0 = exp2f(sc[n][0] - mn_lo), p1 = exp2f(sc[n][1] - mn_lo);
-      const float p2 = exp2f(sc[n][2] - mn_hi), p3 = exp2f(sc[n][3] - mn_hi);
+    for (int n = 0; n < KPW / 8; ++n) {
+      const float p0 = exp2f(sc[n][0] - b_lo), p1 = exp2f(sc[n][1] - b_lo);
+      const float p2 = exp2f(sc[n][2] - b_hi), p3 = exp2f(sc[n][3] - b_hi);
       s_lo += p0 + p1;
       s_hi += p2 + p3;
       pa[n >> 1][(n & 1) * 2 + 0] = pack_bf16(p0, p1);
@@ -307,10 +319,10 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     }
     // ---- O += P V: 4 k-steps of 16 keys, 16 output groups of 8 dims
 #pragma unroll
-    for (int kk = 0; kk < 4; ++kk) {
+    for (int kk = 0; kk < KPW / 16; ++kk) {
       // matrices of one ldmatrix.x4.trans: (keys 0-7, dims d..d+7), (keys 8-15, same dims),
       // (keys 0-7, dims d+8..), (keys 8-15, dims d+8..)
-      const int key = kk * 16 + (lm_mat & 1) * 8 + lm_row;
+      const int key = kq * KPW + kk * 16 + (lm_mat & 1) * 8 + lm_row;
 #pragma unroll
       for (int n2 = 0; n2 < 8; ++n2) {  // 16 dims per ldmatrix
         const int chunk = n2 * 2 + (lm_mat >> 1);  // 16-byte chunk 0..15 over 128 dims
@@ -337,28 +349,30 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     const int hg = pr / rps, r = pr % rps;
     return p.out + (static_cast<size_t>(b) * rps + r) * p.hq * 128 + (g * group + hg) * 128;
   };
-  if (p.n_splits == 1) {
-    if (!alive) return;
-    const float i_lo = 1.0f / l_lo, i_hi = 1.0f / l_hi;
-    if (ok_lo) {
-      __nv_bfloat16* o = out_ptr(pr_lo);
+  float* red = reinterpret_cast<float*>(smem);  // [KQ][BM][PART_LD]: partial of every key part; part 0 becomes the CTA's
+  if constexpr (KQ == 1) {
+    if (p.n_splits == 1) {
+      if (!alive) return;
+      const float i_lo = 1.0f / l_lo, i_hi = 1.0f / l_hi;
+      if (ok_lo) {
+        __nv_bfloat16* o = out_ptr(pr_lo);
 #pragma unroll
-      for (int n = 0; n < 16; ++n)
-        *reinterpret_cast<uint32_t*>(o + n * 8 + t4 * 2) = pack_bf16(o_acc[n][0] * i_lo, o_acc[n][1] * i_lo);
-    }
-    if (ok_hi) {
-      __nv_bfloat16* o = out_ptr(pr_hi);
+        for (int n = 0; n < 16; ++n)
+          *reinterpret_cast<uint32_t*>(o + n * 8 + t4 * 2) = pack_bf16(o_acc[n][0] * i_lo, o_acc[n][1] * i_lo);
+      }
+      if (ok_hi) {
+        __nv_bfloat16* o = out_ptr(pr_hi);
 #pragma unroll
-      for (int n = 0; n < 16; ++n)
-        *reinterpret_cast<uint32_t*>(o + n * 8 + t4 * 2) = pack_bf16(o_acc[n][2] * i_hi, o_acc[n][3] * i_hi);
+        for (int n = 0; n < 16; ++n)
+          *reinterpret_cast<uint32_t*>(o + n * 8 + t4 * 2) = pack_bf16(o_acc[n][2] * i_hi, o_acc[n][3] * i_hi);
+      }
+      return;
     }
-    return;
   }
-  // ---- several key splits: partials stay in shared memory, merged across the cluster
-  __syncthreads();  // every warp is done with the K/V stages: their memory now holds the partial
-  float* red = reinterpret_cast<float*>(smem);  // [BM][PART_LD]
+  // ---- partials go to shared memory: merged over the key parts here, over the key splits across the cluster
+  __syncthreads();  // every warp is done with the K/V stages: their memory now holds the partials
   {
-    float* r_lo = red + static_cast<size_t>(warp * 16 + g4) * PART_LD;
+    float* r_lo = red + (static_cast<size_t>(kq) * BM + warp * 16 + g4) * PART_LD;
     float* r_hi = r_lo + 8 * PART_LD;
 #pragma unroll
     for (int n = 0; n < 16; ++n) {
@@ -366,8 +380,67 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
       *reinterpret_cast<float2*>(r_hi + n * 8 + t4 * 2) = make_float2(o_acc[n][2], o_acc[n][3]);
     }
     if (t4 == 0) {
-      r_lo[128] = m_lo; r_lo[129] = l_lo;  // a split without tiles leaves m = -inf, l = 0
+      r_lo[128] = m_lo; r_lo[129] = l_lo;  // a part or split without keys leaves m = -inf, l = 0
       r_hi[128] = m_hi; r_hi[129] = l_hi;
+    }
+  }
+  if constexpr (KQ > 1) {
+    __syncthreads();
+    // one thread per (row, 4 output dims); everything is read before anything of part 0 is overwritten
+    constexpr int EPT = (BM * 32 + NTHREADS - 1) / NTHREADS;
+    float4 acc[EPT];
+    float Ms[EPT], Ls[EPT];
+#pragma unroll
+    for (int j = 0; j < EPT; ++j) {
+      const int e = threadIdx.x + j * NTHREADS;
+      acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      Ms[j] = -INFINITY;
+      Ls[j] = 0.f;
+      if (e < BM * 32) {
+        const int row = e >> 5, c4 = (e & 31) * 4;
+        float mq[KQ], lq[KQ];
+#pragma unroll
+        for (int q2 = 0; q2 < KQ; ++q2) {
+          const float* r = red + (static_cast<size_t>(q2) * BM + row) * PART_LD;
+          mq[q2] = r[128];
+          lq[q2] = r[129];
+          Ms[j] = fmaxf(Ms[j], mq[q2]);
+        }
+#pragma unroll
+        for (int q2 = 0; q2 < KQ; ++q2) {  // key parts in index order: fixed order of the sums
+          if (lq[q2] != 0.f) {
+            const float w = exp2f(mq[q2] - Ms[j]);
+            const float4 v = *reinterpret_cast<const float4*>(red + (static_cast<size_t>(q2) * BM + row) * PART_LD + c4);
+            Ls[j] += w * lq[q2];
+            acc[j].x += w * v.x; acc[j].y += w * v.y; acc[j].z += w * v.z; acc[j].w += w * v.w;
+          }
+        }
+      }
+    }
+    if (p.n_splits == 1) {
+      if (!alive) return;
+#pragma unroll
+      for (int j = 0; j < EPT; ++j) {
+        const int e = threadIdx.x + j * NTHREADS;
+        if (e >= BM * 32) continue;
+        const int row = e >> 5, c4 = (e & 31) * 4;
+        const int pr = qt * BM + row;
+        if (pr >= R || (pr % rps) >= n_valid) continue;
+        const float inv = 1.0f / Ls[j];
+        *reinterpret_cast<uint2*>(out_ptr(pr) + c4) =
+            make_uint2(pack_bf16(acc[j].x * inv, acc[j].y * inv), pack_bf16(acc[j].z * inv, acc[j].w * inv));
+      }
+      return;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < EPT; ++j) {
+      const int e = threadIdx.x + j * NTHREADS;
+      if (e >= BM * 32) continue;
+      const int row = e >> 5, c4 = (e & 31) * 4;
+      float* r = red + static_cast<size_t>(row) * PART_LD;
+      *reinterpret_cast<float4*>(r + c4) = acc[j];
+      if (c4 == 0) { r[128] = Ms[j]; r[129] = Ls[j]; }
     }
   }
   ptx::cluster_sync_all();
@@ -377,7 +450,7 @@ __global__ void __launch_bounds__(NW * 32) attn_tc_kernel(const __grid_constant_
     const int rpr = (BM + S - 1) / S;  // rows per CTA of the cluster
     const int row0 = rank * rpr, row1 = min(BM, row0 + rpr);
     const uint32_t red_addr = ptx::smem_u32(red);
-    for (int e = threadIdx.x; e < (row1 - row0) * 32; e += NW * 32) {  // one thread per (row, 4 output dims)
+    for (int e = threadIdx.x; e < (row1 - row0) * 32; e += NTHREADS) {  // one thread per (row, 4 output dims)
       const int row = row0 + (e >> 5), c4 = (e & 31) * 4;
       const int pr = qt * BM + row;
       if (pr >= R || (pr % rps) >= n_valid) continue;

@@ -626,9 +626,9 @@ int launch_attention(d3_ctx* c, const void* q, const void* kc, const void* vc, v
 
 // Tensor-core attention launch: warps per CTA from the packed rows per kv head, key splits so that
 // about two CTAs per SM exist even at batch 1 (decode only; prefill has enough query tiles).
-template <int NW>
+template <int NW, int KQ>
 int launch_attn_tc(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
-  auto kern = attn::attn_tc_kernel<NW>;
+  auto kern = attn::attn_tc_kernel<NW, KQ>;
   static bool attr_set = false;
   if (!attr_set) {
     CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::attn_tc_smem_bytes())));
@@ -636,7 +636,7 @@ int launch_attn_tc(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(NW * 32);
+  cfg.blockDim = dim3(NW * KQ * 32);
   cfg.dynamicSmemBytes = attn::attn_tc_smem_bytes();
   cfg.stream = c->stream;
   cudaLaunchAttribute at[2];
@@ -687,9 +687,10 @@ int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMa
   p.error_word = c->error_word;
   dim3 grid(q_tiles, pairs, splits);
   switch (nw) {
-    case 2: return launch_attn_tc<2>(c, p, grid);
-    case 4: return launch_attn_tc<4>(c, p, grid);
-    default: return launch_attn_tc<8>(c, p, grid);
+    // eight warps per CTA whatever the rows: few row groups leave warps to split the keys of a tile
+    case 2: return launch_attn_tc<2, 4>(c, p, grid);
+    case 4: return launch_attn_tc<4, 2>(c, p, grid);
+    default: return launch_attn_tc<8, 1>(c, p, grid);
   }
 }
 
