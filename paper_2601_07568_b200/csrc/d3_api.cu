@@ -395,13 +395,7 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
                   int c_hint, const QkvExtra* qx, int w_tiled) {
   const int T = (N + 127) / 128, KC = (K + 63) / 64;
   const int a_rows = ((M + 31) / 32) * 32;  // 32 or 64
-  // ring + partial tile must leave room for two CTAs per SM
-  const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + 128 * 128;
-  const size_t part_bytes = static_cast<size_t>(128) * a_rows * 4;
-  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 100) * 1024;
-  int stages = static_cast<int>((budget > part_bytes ? budget - part_bytes : 0) / stage_bytes);
-  stages = std::max(2, std::min(stages, 16));
-  const size_t smem = tc::gemm_ck_smem_bytes(a_rows, stages);
+  if (epi != EPI_F32 && epi != EPI_T && epi != EPI_RESID) return fail(c, D3_ERR_UNSUPPORTED, "the cluster K-split kernel has elementwise epilogues only");
   // Cluster launches of this kernel get one CTA per SM, whatever its shared memory.  The kernel is
   // paced by its single-thread pipeline loops (a fixed time per K slab), so what counts is the number
   // of slabs a CTA walks through.  Either the clusters are all resident and loop over their tiles, or
@@ -426,6 +420,13 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
       cs.n_clusters = by_waves ? T : n_res;
     }
   }
+  // ring + receive buffer stay near 100 KB, so that a CTA of the next kernel fits beside this one
+  const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + 128 * 128;
+  const size_t recv_bytes = tc::gemm_ck_recv_bytes(a_rows, cs.C);
+  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 100) * 1024;
+  int stages = static_cast<int>((budget > recv_bytes ? budget - recv_bytes : 0) / stage_bytes);
+  stages = std::max(2, std::min(stages, 16));
+  const size_t smem = tc::gemm_ck_smem_bytes(a_rows, stages, cs.C);
   tc::GemmParams p{};
   p.M = M; p.N = N; p.K = K;
   p.a_rows = a_rows;
@@ -457,9 +458,6 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
     case EPI_F32: return launch_ck<EPI_F32>(c, tx, tw, p, cs, smem);
     case EPI_T: return launch_ck<EPI_T>(c, tx, tw, p, cs, smem);
     case EPI_RESID: return launch_ck<EPI_RESID>(c, tx, tw, p, cs, smem);
-    case EPI_SWIGLU: return launch_ck<EPI_SWIGLU>(c, tx, tw, p, cs, smem);
-    case EPI_QKV: return launch_ck<EPI_QKV>(c, tx, tw, p, cs, smem);
-    case EPI_STATS: return launch_ck<EPI_STATS>(c, tx, tw, p, cs, smem);
   }
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
@@ -553,9 +551,10 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   // only, so the cluster size is chosen for a single wave (run_linear_ck).
   if (M <= 64 && !c->tune_no_cluster) {
     const int T = (N + 127) / 128, KC = (K + 63) / 64;
-    if (ctas_hint >= 1 && ctas_hint <= 8) return run_linear_ck(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
+    const bool elementwise = epi == EPI_F32 || epi == EPI_T || epi == EPI_RESID;
+    if (elementwise && ctas_hint >= 1 && ctas_hint <= 8) return run_linear_ck(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
     // few enough tiles that every tile gets a cluster of at least two resident CTAs
-    if (ctas_hint == 0 && T * 2 <= c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 0, qx, w_tiled);
+    if (elementwise && ctas_hint == 0 && T * 2 <= c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 0, qx, w_tiled);
   }
   if (ctas_hint < 0) {  // a strip width asked for by name
     const int S = -ctas_hint;

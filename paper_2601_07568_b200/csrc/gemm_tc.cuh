@@ -709,47 +709,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 }
 
 // ----------------------------------------------------------------------------- cluster K-split kernel
-// Skinny matmuls (up to 64 rows, 128-column tiles).  The grid is made of clusters of C CTAs
-// (C = 1..8).  A cluster owns whole output tiles; inside it every CTA takes one C-th of the K range of
-// each tile, so all C partial accumulators of a tile are complete at the same time.  They are summed
-// through distributed shared memory instead of L2: each CTA copies its accumulator to its own shared
-// memory, signals its peers (remote mbarrier arrive, release at cluster scope), and the CTAs that own
-// a 32-column slice of the tile add the C partials in rank order (fixed order: reproducible bits)
-// and run the epilogue on their slice.  No global workspace, no atomics, no fences on the way.
+// Skinny matmuls (up to 64 rows, 128-column tiles) with an elementwise epilogue (fp32, bf16 or
+// residual output).  The grid is made of clusters of C CTAs (C = 1..8).  A cluster owns whole output
+// tiles; inside it every CTA takes one C-th of the K range of each tile, so all C partial
+// accumulators of a tile are complete at about the same time.  They meet in distributed shared
+// memory: a tile is cut into units of 16 rows x 32 columns, unit u belongs to CTA u mod C, and every
+// CTA pushes its partial of each unit into the owner's shared memory (remote stores), then arrives
+// on the owner's barrier (release at cluster scope).  An owner waits for its C arrivals, adds the
+// partials in rank order (fixed order: reproducible bits) with one (row, 4 columns) element per
+// thread, and runs the epilogue.  Nobody reads another CTA's memory, so a CTA leaves as soon as it
+// has pushed its partials and finished its own units; no global workspace, no atomics.
 struct ClusterSplit {
   int C;           // CTAs per cluster
   int n_clusters;  // clusters that have tiles
 };
 
-struct DsmemSource {
-  uint32_t part_addr;  // shared-memory address of this CTA's partial tile [128 columns][a_rows] fp32
-  int C, a_rows, row;
-  __device__ __forceinline__ void load(int c, float (&v)[32]) const {
-#pragma unroll
-    for (int j = 0; j < 32; ++j) v[j] = 0.f;
-    const uint32_t off = part_addr + static_cast<uint32_t>(c * a_rows + row) * 4u;
-    const uint32_t step = static_cast<uint32_t>(a_rows) * 4u;
-    int s = 0;
-    for (; s + 1 < C; s += 2) {  // two peers' loads in flight; the sums stay in rank order
-      const uint32_t a0 = map_to_cta(off, static_cast<uint32_t>(s)), a1 = map_to_cta(off, static_cast<uint32_t>(s + 1));
-      float t0[32], t1[32];
-#pragma unroll
-      for (int j = 0; j < 32; ++j) t0[j] = ld_cluster_f(a0 + j * step);
-#pragma unroll
-      for (int j = 0; j < 32; ++j) t1[j] = ld_cluster_f(a1 + j * step);
-#pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] = (v[j] + t0[j]) + t1[j];
-    }
-    if (s < C) {
-      const uint32_t a0 = map_to_cta(off, static_cast<uint32_t>(s));
-#pragma unroll
-      for (int j = 0; j < 32; ++j) v[j] += ld_cluster_f(a0 + j * step);
-    }
-  }
-};
-
 // grid = (n_clusters * C), cluster dims (C, 1, 1).  Dynamic shared memory as in gemm_tc_kernel, plus
-// the partial tile [128][a_rows] fp32 and the two cluster barriers.
+// the receive buffer [units per owner][C sources][16 rows][32 columns] fp32 and the two cluster barriers.
 template <int EPI>
 __global__ void __launch_bounds__(NUM_THREADS, 2)
 gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -764,13 +740,15 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   constexpr uint32_t b_stage_bytes = BLOCK_N * 128u;
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + static_cast<size_t>(stages) * a_stage_bytes;
-  float* part = reinterpret_cast<float*>(smem_b + static_cast<size_t>(stages) * b_stage_bytes);  // [128][a_rows]
-  uint64_t* full_bar = reinterpret_cast<uint64_t*>(part + 128 * p.a_rows);
+  float* recv = reinterpret_cast<float*>(smem_b + static_cast<size_t>(stages) * b_stage_bytes);
+  const int n_units = 4 * (p.a_rows / 16);             // 16-row x 32-column units of a tile
+  const int units_per_owner = (n_units + cs.C - 1) / cs.C;
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(recv + static_cast<size_t>(units_per_owner) * cs.C * 512);
   uint64_t* empty_bar = full_bar + stages;
   uint64_t* acc_full = empty_bar + stages;
   uint64_t* acc_empty = acc_full + 2;
-  uint64_t* ready_bar = acc_empty + 2;  // all C partials of the current tile are in shared memory
-  uint64_t* free_bar = ready_bar + 1;   // all C CTAs have finished reading this CTA's partial
+  uint64_t* ready_bar = acc_empty + 2;  // all C partials of this CTA's units of the current tile have arrived
+  uint64_t* free_bar = ready_bar + 1;   // every owner has added up the previous tile: its buffers may be overwritten
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(free_bar + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -799,7 +777,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       mbar_init(&acc_empty[b], 128);
     }
     mbar_init(ready_bar, static_cast<uint32_t>(C));
-    mbar_init(free_bar, static_cast<uint32_t>(C));
+    mbar_init(free_bar, static_cast<uint32_t>(n_units < C ? n_units : C));  // one arrival per owner
     *abort_flag = 0;
     fence_barrier_init();
   }
@@ -895,68 +873,140 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     const int lg = warp & 3;
     const int row = lg * 32 + lane;
     const int et = threadIdx.x - 64;  // 0..127
-    const bool warp_live = (lg * 32 < p.a_rows) && (lg * 32 < p.M);
-    const uint32_t part_addr = smem_u32(part);
-    // (row, 32-column chunk) pairs of this CTA's slice: chunks rank, rank + C, ... (< 4)
-    const int tpr = 128 / p.a_rows;  // threads that can share a row: 4 or 2
-    const int prow = et % p.a_rows, sub = et / p.a_rows;
-    // row factors (folded RMSNorm): fetched now, while the first accumulator is still being built
-    float rs_row = 1.f, rs_prow = 1.f;
-    if (p.ep.ssq_in != nullptr) {
-      if constexpr (EPI == EPI_STATS) {
-        if (rank == 0 && warp_live && row < p.M) rs_row = row_rstd(p.ep, row);
-      } else {
-        if (sub < tpr && prow < p.M) rs_prow = row_rstd(p.ep, prow);
-      }
-    }
+    const bool warp_live = lg * 32 < p.a_rows;  // this warp's TMEM lanes hold rows of X (zero rows beyond M)
+    const uint32_t recv_addr = smem_u32(recv);
+    const int RS = p.a_rows / 16;     // row slices of a tile
+    const int n_owners = n_units < C ? n_units : C;
+    const int n_tiles_mine = t1 - t0;
+    // as an owner: element (row e_row of the unit, columns 4 * e_j ..) of every unit of this CTA
+    const int e_j = et & 7, e_row = et >> 3;
     bool alive = true;
     int seg = 0;
     for (int t = t0; t < t1; ++t, ++seg) {
       const int buf = seg & 1;
       const int n0 = t * BLOCK_N;
+      // the residual values this thread will update (first unit): in flight while the MMAs still run
+      float4 y_pre = make_float4(0.f, 0.f, 0.f, 0.f);
+      bool y_pre_ok = false;
+      if constexpr (EPI == EPI_RESID) {
+        if (rank < n_units) {
+          const int c = rank / RS, m = (rank % RS) * 16 + e_row, n = n0 + c * 32 + e_j * 4;
+          if (m < p.M && n + 4 <= p.N && (p.ep.ldy & 3) == 0) {
+            y_pre = *reinterpret_cast<const float4*>(static_cast<const float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy + n);
+            y_pre_ok = true;
+          }
+        }
+      }
+      float rs = 1.f;  // row factor (folded RMSNorm) of this thread's row of its first unit; others are fetched later
+      if (EPI != EPI_RESID && p.ep.ssq_in != nullptr && rank < n_units) {
+        const int m = (rank % RS) * 16 + e_row;
+        if (m < p.M) rs = row_rstd(p.ep, m);
+      }
       bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
-      // the peers must be done with this CTA's previous partial before it is overwritten
+      // the owners must have added up the previous tile before their buffers are overwritten
       if (ok && seg > 0) ok = mbar_wait_cluster(free_bar, static_cast<uint32_t>(seg - 1) & 1u, abort_flag, p.error_word);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) { alive = false; break; }
       tc_fence_after();
       if (warp_live) {
+        // push this lane's row of every 32-column chunk to the chunk's owner:
+        // receive buffer [slot][source rank][16 rows][8 groups of 4 columns]
         TmemSource tsrc{tmem_base + static_cast<uint32_t>(buf * BLOCK_N) + (static_cast<uint32_t>(lg * 32) << 16)};
-        for (int c = 0; c < BLOCK_N; c += 32) {
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
           float v[32];
-          tsrc.load(c, v);
+          tsrc.load(c * 32, v);
+          const int u = c * RS + (row >> 4);
+          const int owner = u % C, slot = u / C;
+          const uint32_t dst = map_to_cta(recv_addr + static_cast<uint32_t>(((slot * C + rank) * 16 + (row & 15)) * 128), static_cast<uint32_t>(owner));
 #pragma unroll
-          for (int q = 0; q < 32; ++q) part[(c + q) * p.a_rows + row] = v[q];
+          for (int j = 0; j < 8; ++j) st_cluster_f4(dst + j * 16, v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
         }
       }
       tc_fence_before();
       mbar_arrive(&acc_empty[buf]);
-      epi_bar_sync();  // the whole partial is written ...
-      if (et < C) mbar_arrive_remote(ready_bar, static_cast<uint32_t>(et));  // ... tell every CTA of the cluster
-      ok = mbar_wait_cluster(ready_bar, static_cast<uint32_t>(seg) & 1u, abort_flag, p.error_word);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) { alive = false; break; }
-      if constexpr (EPI == EPI_STATS) {
-        // one statistic per (row, 128 columns): rank 0 takes the whole tile, a row stays with one thread
-        if (rank == 0 && warp_live) {
-          DsmemSource dsrc{part_addr, C, p.a_rows, row};
-          run_epilogue<EPI, BLOCK_N>(dsrc, p, row, n0, row < p.M, 0, 1, -1, rs_row);
+      epi_bar_sync();  // every pushing thread's stores are ordered before the arrivals below
+      if (et < n_owners) mbar_arrive_remote(ready_bar, static_cast<uint32_t>(et));
+      if (rank < n_units) {
+        // ---- owner: wait for the C partials of its units, add them in rank order, epilogue
+        ok = mbar_wait_cluster(ready_bar, static_cast<uint32_t>(seg) & 1u, abort_flag, p.error_word);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { alive = false; break; }
+        for (int slot = 0, u = rank; u < n_units; ++slot, u += C) {
+          const int c = u / RS;
+          const int m = (u % RS) * 16 + e_row, n = n0 + c * 32 + e_j * 4;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4* src = reinterpret_cast<const float4*>(recv) + (static_cast<size_t>(slot) * C * 16 + e_row) * 8 + e_j;
+          for (int s2 = 0; s2 < C; ++s2) {
+            const float4 w = src[static_cast<size_t>(s2) * 128];
+            acc.x += w.x; acc.y += w.y; acc.z += w.z; acc.w += w.w;
+          }
+          const bool live = m < p.M;
+          const bool vec = n + 4 <= p.N && (p.ep.ldy & 3) == 0;
+          if constexpr (EPI == EPI_RESID) {
+            float* y = static_cast<float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
+            float sq = 0.f;
+            if (live) {
+              if (vec) {
+                const float4 o0 = (slot == 0 && y_pre_ok) ? y_pre : *reinterpret_cast<const float4*>(y + n);
+                const float4 o = make_float4(o0.x + acc.x, o0.y + acc.y, o0.z + acc.z, o0.w + acc.w);
+                *reinterpret_cast<float4*>(y + n) = o;
+                sq = ((o.x * o.x + o.y * o.y) + o.z * o.z) + o.w * o.w;
+                if (p.ep.yb != nullptr) {
+                  __nv_bfloat162 lo = __floats2bfloat162_rn(o.x, o.y), hi = __floats2bfloat162_rn(o.z, o.w);
+                  *reinterpret_cast<uint2*>(p.ep.yb + static_cast<size_t>(m) * p.ep.ldy + n) =
+                      make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                }
+              } else {
+                const float a4[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                  if (n + q < p.N) {
+                    const float o = y[n + q] + a4[q];
+                    y[n + q] = o;
+                    sq += o * o;
+                    if (p.ep.yb != nullptr) p.ep.yb[static_cast<size_t>(m) * p.ep.ldy + n + q] = __float2bfloat16_rn(o);
+                  }
+                }
+              }
+            }
+            // the 8 threads of a row are 8 neighbouring lanes: chunk sum of squares in a fixed tree
+            sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+            sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+            sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+            if (live && e_j == 0 && p.ep.ssq_out != nullptr && n0 + c * 32 < p.N)
+              p.ep.ssq_out[static_cast<size_t>(m) * ((p.N + 31) / 32) + (n0 + c * 32) / 32] = sq;
+          } else {
+            if (slot > 0 && p.ep.ssq_in != nullptr && live) rs = row_rstd(p.ep, m);
+            const float sc = (EPI == EPI_F32 ? p.ep.scale : 1.f) * rs;
+            const float a4[4] = {acc.x * sc, acc.y * sc, acc.z * sc, acc.w * sc};
+            if (live) {
+              if constexpr (EPI == EPI_F32) {
+                float* y = static_cast<float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
+                if (vec) *reinterpret_cast<float4*>(y + n) = make_float4(a4[0], a4[1], a4[2], a4[3]);
+                else
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) if (n + q < p.N) y[n + q] = a4[q];
+              } else {
+                __nv_bfloat16* y = static_cast<__nv_bfloat16*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy;
+                if (vec) {
+                  __nv_bfloat162 lo = __floats2bfloat162_rn(a4[0], a4[1]), hi = __floats2bfloat162_rn(a4[2], a4[3]);
+                  *reinterpret_cast<uint2*>(y + n) = make_uint2(*reinterpret_cast<uint32_t*>(&lo), *reinterpret_cast<uint32_t*>(&hi));
+                } else {
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) if (n + q < p.N) y[n + q] = __float2bfloat16_rn(a4[q]);
+                }
+              }
+            }
+          }
         }
-      } else {
-        // chunk list of this rank, spread over the threads that share a row
-        int my_chunks = 0;
-        for (int c = rank; c < 4; c += C) ++my_chunks;
-        if (sub < tpr && sub < my_chunks) {
-          DsmemSource dsrc{part_addr, C, p.a_rows, prow};
-          // chunk indices rank + C * (sub + tpr * q): first = rank + C * sub, stride = C * tpr
-          run_epilogue<EPI, BLOCK_N>(dsrc, p, prow, n0, prow < p.M, rank + C * sub, C * tpr, -1, rs_prow);
+        if (seg + 1 < n_tiles_mine) {  // more tiles: tell every CTA of the cluster that this owner's buffers are free
+          epi_bar_sync();
+          if (et < C) mbar_arrive_remote(free_bar, static_cast<uint32_t>(et));
         }
       }
-      epi_bar_sync();  // this CTA has read all it needs from every peer
-      if (et < C) mbar_arrive_remote(free_bar, static_cast<uint32_t>(et));
     }
-    // nobody may still be reading this CTA's partial when it exits
-    if (alive && seg > 0) mbar_wait_cluster(free_bar, static_cast<uint32_t>(seg - 1) & 1u, abort_flag, p.error_word);
+    (void)alive;
     tc_fence_before();
   }
   __syncthreads();
@@ -964,11 +1014,14 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     tc_fence_after();
     tmem_dealloc<TMEM_COLS>(tmem_base);
   }
-  cluster_sync_all();  // shared memory of a CTA stays valid until its peers are past their last remote access
 }
 
-inline size_t gemm_ck_smem_bytes(int a_rows, int stages) {
-  size_t body = static_cast<size_t>(stages) * (a_rows * 128 + 128 * 128) + static_cast<size_t>(128) * a_rows * 4;
+inline size_t gemm_ck_recv_bytes(int a_rows, int C) {
+  const int n_units = 4 * (a_rows / 16);
+  return static_cast<size_t>((n_units + C - 1) / C) * C * 2048;
+}
+inline size_t gemm_ck_smem_bytes(int a_rows, int stages, int C) {
+  size_t body = static_cast<size_t>(stages) * (a_rows * 128 + 128 * 128) + gemm_ck_recv_bytes(a_rows, C);
   size_t need = static_cast<size_t>(stages) * a_rows * 128 + static_cast<size_t>(128 - a_rows) * 128 + 128 * 128;
   if (body < need) body = need;
   return 1024 + body + (2 * stages + 6) * 8 + 64;
