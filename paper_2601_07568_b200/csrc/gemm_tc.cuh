@@ -129,6 +129,10 @@ struct PartialSource {
   }
 };
 
+// SiLU with the approximate division (the exact one is a long dependent sequence, and a skinny
+// matmul's epilogue is one warp deep): error of a few ulp, far below the bf16 rounding of the output.
+__device__ __forceinline__ float silu_fast(float g) { return __fdividef(g, 1.0f + __expf(-g)); }
+
 // All 32 threads of a warp must call this together (the TMEM loads are warp-wide); `live` only
 // predicates this thread's stores.
 // Chunks (32 columns each) c_first, c_first + c_stride, ... of the tile are handled; the TMEM path
@@ -242,7 +246,7 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
         uint32_t w[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) {
-          __nv_bfloat162 t = __floats2bfloat162_rn(silu_f(v[4 * q]) * v[4 * q + 1], silu_f(v[4 * q + 2]) * v[4 * q + 3]);
+          __nv_bfloat162 t = __floats2bfloat162_rn(silu_fast(v[4 * q]) * v[4 * q + 1], silu_fast(v[4 * q + 2]) * v[4 * q + 3]);
           w[q] = *reinterpret_cast<uint32_t*>(&t);
         }
         uint4* y4 = reinterpret_cast<uint4*>(y + h0);
@@ -252,14 +256,14 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
         uint32_t w[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          __nv_bfloat162 t = __floats2bfloat162_rn(silu_f(v[4 * q]) * v[4 * q + 1], silu_f(v[4 * q + 2]) * v[4 * q + 3]);
+          __nv_bfloat162 t = __floats2bfloat162_rn(silu_fast(v[4 * q]) * v[4 * q + 1], silu_fast(v[4 * q + 2]) * v[4 * q + 3]);
           w[q] = *reinterpret_cast<uint32_t*>(&t);
         }
         *reinterpret_cast<uint4*>(y + h0) = make_uint4(w[0], w[1], w[2], w[3]);
       } else {
 #pragma unroll
         for (int j = 0; j < 16; ++j)
-          if (h0 + j < F) y[h0 + j] = __float2bfloat16_rn(silu_f(v[2 * j]) * v[2 * j + 1]);
+          if (h0 + j < F) y[h0 + j] = __float2bfloat16_rn(silu_fast(v[2 * j]) * v[2 * j + 1]);
       }
     }
   } else if constexpr (EPI == EPI_STATS) {
@@ -320,6 +324,12 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
             dst = p.k_cache + ((static_cast<size_t>(b) * p.n_kv_heads + (head - p.n_q_heads)) * p.max_seq + pos) * 128;
           }
           const int i0 = off / 2;  // pair index of column 0 of this half: 8 pairs, dims i0.. and 64+i0..
+          // the 8 cosines and sines of this row and half in four 16-byte loads (a lane reads its own
+          // table row: scalar loads would cost a cache line each)
+          const float4 ca = *reinterpret_cast<const float4*>(cs + i0), cb = *reinterpret_cast<const float4*>(cs + i0 + 4);
+          const float4 sa = *reinterpret_cast<const float4*>(sn + i0), sb = *reinterpret_cast<const float4*>(sn + i0 + 4);
+          const float cs8[8] = {ca.x, ca.y, ca.z, ca.w, cb.x, cb.y, cb.z, cb.w};
+          const float sn8[8] = {sa.x, sa.y, sa.z, sa.w, sb.x, sb.y, sb.z, sb.w};
           uint32_t lo[4], hi[4];
 #pragma unroll
           for (int q = 0; q < 4; ++q) {
@@ -327,7 +337,7 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
               const int j = 2 * q + e;
-              const float co = cs[i0 + j], si = sn[i0 + j];
+              const float co = cs8[j], si = sn8[j];
               const float a = v[16 * h + 2 * j], bb = v[16 * h + 2 * j + 1];
               l2[e] = a * co - bb * si;
               h2[e] = bb * co + a * si;
@@ -1052,13 +1062,14 @@ struct TmemPairSource {
   bool two;
   __device__ __forceinline__ void load(int c, float (&v)[32]) const {
     tmem_ld_32x32(taddr_row0 + static_cast<uint32_t>(c), v);
-    tmem_ld_wait();
     if (two) {
       float w[32];
-      tmem_ld_32x32(taddr_row1 + static_cast<uint32_t>(c), w);
+      tmem_ld_32x32(taddr_row1 + static_cast<uint32_t>(c), w);  // both loads in flight
       tmem_ld_wait();
 #pragma unroll
       for (int j = 0; j < 32; ++j) v[j] += w[j];
+    } else {
+      tmem_ld_wait();
     }
   }
 };
@@ -1197,12 +1208,19 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p
       }
       if (ok) umma_commit(acc_full);
     }
-  } else if (warp >= 2 && warp <= 5) {
-    // ---------------- epilogue warps: TMEM lane group = warp % 4
+  }
+  // ---------------- epilogue: warps 2-5, TMEM lane group = warp % 4.  With at most 32 rows only lane
+  // group 0 holds anything, and one warp alone would take microseconds over a wide strip: warp 0
+  // (same lane group; its producer thread is done by then) takes every other 32-column chunk.
+  const bool helper = warp == 0 && p.a_rows <= 32 && S > 32;
+  if (warp == 0) __syncwarp();  // lanes 1-31 wait here for the producer thread instead of polling beside it
+  if ((warp >= 2 && warp <= 5) || helper) {
     grid_dep_wait();
     const int lg = warp & 3;
     const int row = lg * 32 + lane;
     const bool warp_live = lg * 32 < p.a_rows && lg * 32 < p.M;
+    const bool shared_chunks = p.a_rows <= 32 && S > 32;  // lane group 0 is worked on by warps 4 and 0
+    const int c_first = helper ? 1 : 0, c_stride = shared_chunks ? 2 : 1;
     // row factor (folded RMSNorm): fetched while the accumulators are still being built
     const float rs = (warp_live && row < p.M && p.ep.ssq_in != nullptr) ? row_rstd(p.ep, row) : 1.f;
     bool ok = mbar_wait(acc_full, 0u, abort_flag, p.error_word);
@@ -1212,7 +1230,7 @@ gemm_strip_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p
       if (warp_live) {
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(lg * 32) << 16);
         TmemPairSource tsrc{lane_addr, lane_addr + static_cast<uint32_t>(TCOLS / 2), n_pipe == 2};
-        run_epilogue<EPI, 256>(tsrc, p, row, c0, row < p.M, 0, 1, c0 + S, rs);
+        run_epilogue<EPI, 256>(tsrc, p, row, c0, row < p.M, c_first, c_stride, c0 + S, rs);
       }
     }
     tc_fence_before();
