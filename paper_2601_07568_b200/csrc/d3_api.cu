@@ -518,8 +518,10 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   p.w_packed = static_cast<const bf16*>(W);
   p.w_blocks = static_cast<long long>((N + 127) / 128) * KC;
   p.gm = 1;  // K walk of CTA b starts at slab b mod KC
-  // two issue pipelines per CTA while both accumulators fit 256 tensor-memory columns
+  // two issue pipelines per CTA while both accumulators fit 256 tensor-memory columns; each then owns
+  // the stages of its parity, so the ring has an even number of them
   p.n_producers = (S <= 128 && KC >= 4 && c->tune_producers != 1) ? 2 : 1;
+  if (p.n_producers == 2) p.stages &= ~1;
   p.ep = ep;
   if (qx) {
     p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
