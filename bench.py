@@ -27,11 +27,11 @@ if ROOT not in sys.path:
 
 import numpy as np  # noqa: E402
 
-# DRAM traffic (dram bytes read + written) per launch of the matmul kernel at 32 rows on the c2 shapes,
-# from the ncu capture summarised in profiles/gemm_tc_kernel_c2_rows32.md.  It is reported only while the
+# DRAM traffic (dram bytes read + written) per launch of the matmul kernels at 32 rows on the c2 shapes,
+# from the ncu capture summarised in profiles/matmul_kernels_c2_rows32.md.  It is reported only while the
 # kernel sources still hash to the value below; after any change to them it reads null until re-captured.
-NCU_GEMM_TRAFFIC_MB = {"gemm_qkv": 104.7, "gemm_o": 34.4, "gemm_gate_up": 208.2, "gemm_down": 105.8, "gemm_head": 1050.2}
-NCU_GEMM_SOURCE_HASH = "3d0bc32e5d2d2b9a"
+NCU_GEMM_TRAFFIC_MB = {"gemm_qkv": 104.5, "gemm_o": 34.3, "gemm_gate_up": 205.2, "gemm_down": 106.4, "gemm_head": 1051.0}
+NCU_GEMM_SOURCE_HASH = "aa7411522fee822a"
 NCU_GEMM_WORKLOAD = "c2"
 
 
@@ -356,8 +356,8 @@ def run_ours(args):
                                   "ms_per_forward": ms_fwd, "bytes_per_forward": fwd_bytes}
     if hbm_bound and w.name == NCU_GEMM_WORKLOAD and gemm_source_hash() == NCU_GEMM_SOURCE_HASH and n_gemm > 0:
         roofline["traffic"] = 1e6 * sum(NCU_GEMM_TRAFFIC_MB[k] * prof[k]["launches"] for k in NCU_GEMM_TRAFFIC_MB) / n_gemm
-        roofline["traffic_source"] = "ncu, profiles/gemm_tc_kernel_c2_rows32.md (bytes per launch, averaged over the launch mix)"
-    roofline.update({"kernel": "gemm_tc_kernel (all matmul launches of the decode loop)", "peak_source": f"of {peaks['source']}",
+        roofline["traffic_source"] = "ncu, profiles/matmul_kernels_c2_rows32.md (bytes per launch, averaged over the launch mix)"
+    roofline.update({"kernel": "gemm_strip_kernel, gemm_ck_kernel, gemm_tc_kernel (all matmul launches of the decode loop)", "peak_source": f"of {peaks['source']}",
                      "launches": n_gemm, "avg_launch_us": 1e3 * tot_ms / max(n_gemm, 1),
                      "algorithmic_bytes_per_launch": tot_bytes / max(n_gemm, 1)})
     per_class = {}
