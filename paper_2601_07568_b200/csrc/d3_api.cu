@@ -393,8 +393,10 @@ int launch_ck(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc:
 
 int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
                   int c_hint, const QkvExtra* qx, int w_tiled) {
-  const int T = (N + 127) / 128, KC = (K + 63) / 64;
-  const int a_rows = ((M + 31) / 32) * 32;  // 32 or 64
+  // up to 64 rows: one row tile with an X box of 32 or 64 rows; up to 256 rows: row tiles of 128
+  const int a_rows = M <= 64 ? ((M + 31) / 32) * 32 : 128;
+  const int m_tiles = (M + 127) / 128;
+  const int T = m_tiles * ((N + 127) / 128), KC = (K + 63) / 64;
   if (epi != EPI_F32 && epi != EPI_T && epi != EPI_RESID) return fail(c, D3_ERR_UNSUPPORTED, "the cluster K-split kernel has elementwise epilogues only");
   // Cluster launches of this kernel get one CTA per SM, whatever its shared memory.  The kernel is
   // paced by its single-thread pipeline loops (a fixed time per K slab), so what counts is the number
@@ -420,17 +422,18 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
       cs.n_clusters = by_waves ? T : n_res;
     }
   }
-  // ring + receive buffer stay near 100 KB, so that a CTA of the next kernel fits beside this one
+  // skinny: ring + receive buffer stay near 100 KB, so that a CTA of the next kernel fits beside this
+  // one; with 128-row tiles (32 KB stages, up to 64 KB of partials to receive) one CTA per SM
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + 128 * 128;
   const size_t recv_bytes = tc::gemm_ck_recv_bytes(a_rows, cs.C);
-  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 100) * 1024;
+  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : (a_rows <= 64 ? 100 : 200)) * 1024;
   int stages = static_cast<int>((budget > recv_bytes ? budget - recv_bytes : 0) / stage_bytes);
   stages = std::max(2, std::min(stages, 16));
   const size_t smem = tc::gemm_ck_smem_bytes(a_rows, stages, cs.C);
   tc::GemmParams p{};
   p.M = M; p.N = N; p.K = K;
   p.a_rows = a_rows;
-  p.m_tiles = 1; p.n_tiles = T; p.k_chunks = KC;
+  p.m_tiles = m_tiles; p.n_tiles = (N + 127) / 128; p.k_chunks = KC;
   p.total_units = static_cast<long long>(T) * KC;
   p.stages = stages;
   p.error_word = c->error_word;
@@ -449,7 +452,7 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   if (w_tiled) {
     if ((reinterpret_cast<uintptr_t>(W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
     p.w_packed = static_cast<const bf16*>(W);
-    p.w_blocks = static_cast<long long>(T) * KC;
+    p.w_blocks = static_cast<long long>((N + 127) / 128) * KC;
     tw = tx;
   } else {
     TRY(get_tmap(c, W, N, K, 128, &tw));
@@ -551,12 +554,14 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   // distributed shared memory beat the L2 reduction of the unit-range kernel (measured at 32 rows on
   // the 8B shapes: 13 vs 16 us and 23 vs 25 us); cluster launches of this kernel get one CTA per SM
   // only, so the cluster size is chosen for a single wave (run_linear_ck).
-  if (M <= 64 && !c->tune_no_cluster) {
-    const int T = (N + 127) / 128, KC = (K + 63) / 64;
+  if (M <= 256 && !c->tune_no_cluster) {
+    const int T = ((M + 127) / 128) * ((N + 127) / 128), KC = (K + 63) / 64;
     const bool elementwise = epi == EPI_F32 || epi == EPI_T || epi == EPI_RESID;
     if (elementwise && ctas_hint >= 1 && ctas_hint <= 8) return run_linear_ck(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
-    // few enough tiles that every tile gets a cluster of at least two resident CTAs
-    if (elementwise && ctas_hint == 0 && T * 2 <= c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 0, qx, w_tiled);
+    // few enough tiles that every tile gets a cluster of at least two resident CTAs.  By itself only
+    // up to 64 rows: with 128-row tiles (measured at 128 and 256 rows on the 7B/8B shapes) the best
+    // cluster size is only level with the unit-range kernel at 256 rows and the model below misjudges it.
+    if (elementwise && ctas_hint == 0 && M <= 64 && T * 2 <= c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 0, qx, w_tiled);
   }
   if (ctas_hint < 0) {  // a strip width asked for by name
     const int S = -ctas_hint;

@@ -719,8 +719,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 }
 
 // ----------------------------------------------------------------------------- cluster K-split kernel
-// Skinny matmuls (up to 64 rows, 128-column tiles) with an elementwise epilogue (fp32, bf16 or
-// residual output).  The grid is made of clusters of C CTAs (C = 1..8).  A cluster owns whole output
+// Matmuls of up to 256 rows (one or two row tiles of a_rows <= 128 rows, 128-column tiles) with an
+// elementwise epilogue (fp32, bf16 or residual output).  The grid is made of clusters of C CTAs (C = 1..8).  A cluster owns whole output
 // tiles; inside it every CTA takes one C-th of the K range of each tile, so all C partial
 // accumulators of a tile are complete at about the same time.  They meet in distributed shared
 // memory: a tile is cut into units of 16 rows x 32 columns, unit u belongs to CTA u mod C, and every
@@ -766,7 +766,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   const int C = cs.C;
   const int rank = static_cast<int>(cluster_ctarank());
   const int cluster = blockIdx.x / C;
-  const int T = p.n_tiles;  // one row tile: tiles = column tiles
+  const int T = p.m_tiles * p.n_tiles;  // tile t: row tile t % m_tiles, column tile t / m_tiles (the row tiles of a
+                                        // column tile run side by side and share its weights through L2)
   const int KC = p.k_chunks;
   const int t0 = static_cast<int>(static_cast<long long>(T) * cluster / cs.n_clusters);
   const int t1 = static_cast<int>(static_cast<long long>(T) * (cluster + 1) / cs.n_clusters);
@@ -819,11 +820,12 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         else tma_load_2d(dst, &tmap_w, &full_bar[s], kc * BLOCK_K, n_tile * BLOCK_N);
       };
       const int pre = static_cast<int>(n_total < stages ? n_total : stages);
+      const int MTL = p.m_tiles;
       {
         int n_tile = t0, k = 0;
         advance(n_tile, k, pi);
         for (int i = pi; i < pre; i += 2) {  // weights first: they do not depend on the kernels before this one
-          load_w(i, n_tile, kc0 + k);
+          load_w(i, n_tile / MTL, kc0 + k);
           advance(n_tile, k, 2);
         }
       }
@@ -831,7 +833,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       int n_tile = t0, k = 0;
       advance(n_tile, k, pi);
       for (int i = pi; i < pre; i += 2) {
-        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], (kc0 + k) * BLOCK_K, 0);
+        tma_load_2d(smem_a + static_cast<size_t>(i) * a_stage_bytes, &tmap_x, &full_bar[i], (kc0 + k) * BLOCK_K, (n_tile % MTL) * BLOCK_M);
         advance(n_tile, k, 2);
       }
       long long i = pre;
@@ -840,8 +842,8 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       uint32_t ph = (static_cast<uint32_t>(i / stages) & 1u) ^ 1u;  // parity to wait for on the empty barrier
       for (; i < n_total; i += 2) {
         if (!mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
-        load_w(s, n_tile, kc0 + k);
-        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], (kc0 + k) * BLOCK_K, 0);
+        load_w(s, n_tile / MTL, kc0 + k);
+        tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], (kc0 + k) * BLOCK_K, (n_tile % MTL) * BLOCK_M);
         advance(n_tile, k, 2);
         s += 2;
         if (s >= stages) { s -= stages; ph ^= 1u; }
@@ -894,13 +896,14 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
     int seg = 0;
     for (int t = t0; t < t1; ++t, ++seg) {
       const int buf = seg & 1;
-      const int n0 = t * BLOCK_N;
+      const int n0 = (t / p.m_tiles) * BLOCK_N;
+      const int m0 = (t % p.m_tiles) * BLOCK_M;  // first row of this row tile
       // the residual values this thread will update (first unit): in flight while the MMAs still run
       float4 y_pre = make_float4(0.f, 0.f, 0.f, 0.f);
       bool y_pre_ok = false;
       if constexpr (EPI == EPI_RESID) {
         if (rank < n_units) {
-          const int c = rank / RS, m = (rank % RS) * 16 + e_row, n = n0 + c * 32 + e_j * 4;
+          const int c = rank / RS, m = m0 + (rank % RS) * 16 + e_row, n = n0 + c * 32 + e_j * 4;
           if (m < p.M && n + 4 <= p.N && (p.ep.ldy & 3) == 0) {
             y_pre = *reinterpret_cast<const float4*>(static_cast<const float*>(p.ep.y) + static_cast<size_t>(m) * p.ep.ldy + n);
             y_pre_ok = true;
@@ -909,7 +912,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       }
       float rs = 1.f;  // row factor (folded RMSNorm) of this thread's row of its first unit; others are fetched later
       if (EPI != EPI_RESID && p.ep.ssq_in != nullptr && rank < n_units) {
-        const int m = (rank % RS) * 16 + e_row;
+        const int m = m0 + (rank % RS) * 16 + e_row;
         if (m < p.M) rs = row_rstd(p.ep, m);
       }
       bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
@@ -944,7 +947,7 @@ gemm_ck_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         if (!ok) { alive = false; break; }
         for (int slot = 0, u = rank; u < n_units; ++slot, u += C) {
           const int c = u / RS;
-          const int m = (u % RS) * 16 + e_row, n = n0 + c * 32 + e_j * 4;
+          const int m = m0 + (u % RS) * 16 + e_row, n = n0 + c * 32 + e_j * 4;
           float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
           const float4* src = reinterpret_cast<const float4*>(recv) + (static_cast<size_t>(slot) * C * 16 + e_row) * 8 + e_j;
           for (int s2 = 0; s2 < C; ++s2) {
