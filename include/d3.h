@@ -80,7 +80,12 @@ typedef struct d3_config {
 /* All pointers [host] or all [device] (see d3_load_weights).  Per-layer arrays have n_layers
  * entries.  Norm gains may be NULL (= all ones).  Shapes: tok_emb, lm_head [vocab, d_model];
  * wq [n_q_heads*d_head, d_model]; wk, wv [n_kv_heads*d_head, d_model]; wo [d_model,
- * n_q_heads*d_head]; w_gate, w_up [d_ffn, d_model]; w_down [d_model, d_ffn]; gains [d_model]. */
+ * n_q_heads*d_head]; w_gate, w_up [d_ffn, d_model]; w_down [d_model, d_ffn]; gains [d_model].
+ * On the bfloat16 tensor-core path the gains of each RMSNorm (Sec. 3.1: the backbone is a standard
+ * pre-norm transformer) are multiplied into the columns of the matrix that follows it when the
+ * weights are loaded (one extra bfloat16 rounding of those weights), and the row factor
+ * rsqrt(mean(x^2) + eps) is applied to the matmul's fp32 accumulator: same function, no separate
+ * normalisation kernels (D3_PROF_RMSNORM then stays empty). */
 typedef struct d3_weights {
   const void *tok_emb, *lm_head, *final_norm;
   const void *const *attn_norm, *const *wq, *const *wk, *const *wv, *const *wo;

@@ -377,5 +377,8 @@ def weights_from_numpy(shape, weights: Dict[str, object], pin: bool = False) -> 
             return torch.from_numpy(a.view(np.int16)).view(torch.bfloat16)
         return torch.from_numpy(a)
 
-    return {"tok_emb": t(weights["tok_emb"]), "lm_head": t(weights["lm_head"]),
-            "layers": [{k: t(v) for k, v in weights["layers"][l].items()} for l in range(shape.n_layers)]}
+    out = {"tok_emb": t(weights["tok_emb"]), "lm_head": t(weights["lm_head"]),
+           "layers": [{k: t(v) for k, v in weights["layers"][l].items()} for l in range(shape.n_layers)]}
+    if weights.get("final_norm") is not None:
+        out["final_norm"] = t(weights["final_norm"])
+    return out

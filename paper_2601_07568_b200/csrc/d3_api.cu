@@ -1015,8 +1015,12 @@ namespace {
 int finish_matrix(d3_ctx* c, void* rm, void* dst, size_t n, size_t k, const float* fold_gain = nullptr) {
   if (!c->w_tiled) return D3_OK;
   if (fold_gain != nullptr && c->fold_norm) {  // the norm in front of this matmul becomes a row factor: its gains go into the columns
-    const size_t total = n * k;
-    scale_columns_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, c->stream>>>(static_cast<bf16*>(rm), fold_gain, total, static_cast<int>(k));
+    // rows go in grid.y, chunked to the 65535 limit
+    for (size_t r0 = 0; r0 < n; r0 += 65535) {
+      const unsigned rows = static_cast<unsigned>(std::min<size_t>(65535, n - r0));
+      scale_columns_kernel<<<dim3(static_cast<unsigned>((k + 255) / 256), rows), 256, 0, c->stream>>>(
+          static_cast<bf16*>(rm) + r0 * k, fold_gain, static_cast<int>(k));
+    }
     TRY(check_launch(c, "scale_columns_kernel"));
   }
   dim3 grid(static_cast<unsigned>((k + 63) / 64), static_cast<unsigned>((n + 127) / 128));

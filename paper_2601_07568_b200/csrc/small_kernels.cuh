@@ -65,9 +65,12 @@ __global__ void row_prep_kernel(const float* __restrict__ x, __nv_bfloat16* __re
 
 // w[n, k] *= gain[k] (rounded to bf16 once): the gains of the RMSNorm in front of a matmul, moved
 // into its weight columns when the weights are loaded.
-__global__ void scale_columns_kernel(__nv_bfloat16* __restrict__ w, const float* __restrict__ gain, size_t total, int k) {
-  const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i < total) w[i] = __float2bfloat16_rn(__bfloat162float(w[i]) * gain[i % k]);
+// grid (ceil(k / 256), rows): one thread per element, the column index needs no division.
+__global__ void scale_columns_kernel(__nv_bfloat16* __restrict__ w, const float* __restrict__ gain, int k) {
+  const int col = blockIdx.x * blockDim.x + threadIdx.x;
+  if (col >= k) return;
+  __nv_bfloat16* e = w + static_cast<size_t>(blockIdx.y) * k + col;
+  *e = __float2bfloat16_rn(__bfloat162float(*e) * gain[col]);
 }
 
 // ----------------------------------------------------------------------------- RMSNorm

@@ -213,6 +213,21 @@ def test_small_bf16_ragged_batch_step_locked(d_head, hq, hkv, impl):
         assert st.tokens_committed == 3 * 64
 
 
+def test_small_bf16_model_width_not_a_multiple_of_the_tiles():
+    """d_model = 200: ragged K slab (200 = 3 x 64 + 8), ragged 128-column output tile, a last chunk of
+    8 columns in the sums of squares of the folded RMSNorm, ragged vocabulary."""
+    shape = si.scaled_shape(si.LLADA8B, name="ragged-200", n_layers=2, d_model=200, n_q_heads=2, n_kv_heads=1,
+                            d_ffn=320, vocab=777, d_head=128)
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("ragged-200", shape, 2, [19, 50], 32, 32, 0.9, 5)
+    model = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
+    exact = o.model_from_shape(shape, W, np.float32)
+    with Ctx(shape, W, block=32, max_batch=2, max_seq=wl.max_seq) as ctx:
+        rep, _ = step_locked(ctx, model, ids, lens, 32, 32, 0.9, logit_tol=3e-2, exact_model=exact)
+        assert rep["max_logit_err"] <= 3e-2 and rep["self_diff"] == 0 and rep["unexplained"] == 0
+        assert ctx.error_word() == 0
+
+
 def test_padded_batch_equals_single_sequences():
     """Batch elements never interact: a padded batch gives each sequence what it gets alone, and
     permuting the batch permutes the outputs.  Bit-exact equality is not required of the CUDA path:
@@ -239,6 +254,55 @@ def test_padded_batch_equals_single_sequences():
             ctx.prefill(ids[b:b + 1, :lens[b]], lens[b:b + 1])
             single = ctx.logits(blk[:1])[0]
             assert np.max(np.abs(single - batch[b])) <= tol * np.max(np.abs(batch[b]))
+
+
+@pytest.mark.parametrize("dtype,impl", [("f32", 0), ("bf16", 0), ("bf16", 1)])
+def test_norm_gains(dtype, impl):
+    """RMSNorm gains that are not all ones (the synthetic workloads leave them at one): attention, FFN
+    and final norm.  fp32 and the bf16 SIMT path normalise in a kernel of their own, the bf16
+    tensor-core path folds the gains into the weight columns and the row factor into the matmul
+    epilogues; all three must reproduce the oracle's logits."""
+    if dtype == "f32":
+        shape = si.TINY
+        tol = 1e-4
+    else:
+        shape = small_bf16(128, 4, 2, "gains-bf16")
+        tol = 3e-2
+    W = si.gen_weights(shape)
+    rng = np.random.default_rng(5)
+
+    def gain():
+        g = (0.5 + rng.random(shape.d_model)).astype(np.float32)
+        return si.bf16_bits_to_f32(si.f32_to_bf16_bits(g)) if dtype == "bf16" else g
+
+    gains = {"final_norm": gain()}
+    for l in range(shape.n_layers):
+        gains[("attn_norm", l)] = gain()
+        gains[("ffn_norm", l)] = gain()
+    # library side: gains in the context dtype next to the other tensors
+    enc = (lambda g: si.f32_to_bf16_bits(g)) if dtype == "bf16" else (lambda g: g)
+    Wg = {"tok_emb": W["tok_emb"], "lm_head": W["lm_head"], "final_norm": enc(gains["final_norm"]),
+          "layers": {l: dict(W["layers"][l], attn_norm=enc(gains[("attn_norm", l)]), ffn_norm=enc(gains[("ffn_norm", l)]))
+                     for l in range(shape.n_layers)}}
+    model = o.OracleModel(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
+                          n_kv_heads=shape.n_kv_heads, d_head=shape.d_head, d_ffn=shape.d_ffn, vocab=shape.vocab,
+                          mask_id=shape.mask_id, weights=W, rope_theta=shape.rope_theta, rms_eps=shape.rms_eps,
+                          logit_scale=shape.logit_scale, dtype=np.float64, gains=gains)
+    plain = o.model_from_shape(shape, W, np.float64)
+    wl, ids, lens = si.small_workload("gains", shape, 1, [21], 32, 16 if dtype == "f32" else 32, 0.9, 3)
+    B = wl.block
+    blk = np.full((1, B), shape.mask_id, dtype=np.int32)
+    blk[0, 2] = 11
+    with Ctx(shape, Wg, block=B, max_batch=1, max_seq=wl.max_seq, gemm_impl=impl) as ctx:
+        ctx.prefill(ids, lens)
+        got = ctx.logits(blk)[0]
+        assert ctx.error_word() == 0
+    ref = model.denoise_forward(model.prefill(ids[0, :lens[0]]), blk[0])[0]
+    ref_plain = plain.denoise_forward(plain.prefill(ids[0, :lens[0]]), blk[0])[0]
+    scale = np.max(np.abs(ref))
+    assert np.max(np.abs(got - ref)) <= tol * scale
+    # the gains matter: without them the logits are somewhere else entirely
+    assert np.max(np.abs(ref_plain - ref)) > 10 * tol * scale
 
 
 def test_column_strip_schedule_in_the_forward():
