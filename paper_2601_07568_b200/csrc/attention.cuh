@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(THREADS) attn_simt_kernel(const T* __restrict_
       float s = 0.f;
 #pragma unroll 8
       for (int d = 0; d < DH; ++d) s = fmaf(Qs[r][d], Ks[lane][d], s);
-      if (j0 + lane >= kv_len) s = -INFINITY;
+      if (j0 + lane >= row_kv_limit(rm, b, r0 + r, kv_len)) s = -INFINITY;  // keys of later segments stay unseen
       float mx = s;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -245,6 +245,8 @@ __global__ void __launch_bounds__(NW * KQ * 32) attn_tc_kernel(const __grid_cons
     for (int e = 0; e < 4; ++e) o_acc[n][e] = 0.f;
   float m_lo = -INFINITY, m_hi = -INFINITY, l_lo = 0.f, l_hi = 0.f;
 
+  // the 16 rows of a row group lie in one segment (segments are multiples of 16 rows): one key limit per warp
+  const int kv_lim = row_kv_limit(p.rm, b, (qt * BM + warp * 16) % rps, kv_len);
   // ldmatrix lane roles: lanes 0-7 address matrix 0, 8-15 matrix 1, 16-23 matrix 2, 24-31 matrix 3
   const int lm_row = lane & 7, lm_mat = lane >> 3;
   bool alive = true;
@@ -280,7 +282,7 @@ __global__ void __launch_bounds__(NW * KQ * 32) attn_tc_kernel(const __grid_cons
 #pragma unroll
     for (int n = 0; n < KPW / 8; ++n) {
       const int key = j0 + kq * KPW + n * 8 + t4 * 2;
-      const bool v0 = key < kv_len, v1 = key + 1 < kv_len;
+      const bool v0 = key < kv_lim, v1 = key + 1 < kv_lim;
       sc[n][0] = v0 ? sc[n][0] * p.scale_log2 : -INFINITY;
       sc[n][1] = v1 ? sc[n][1] * p.scale_log2 : -INFINITY;
       sc[n][2] = v0 ? sc[n][2] * p.scale_log2 : -INFINITY;

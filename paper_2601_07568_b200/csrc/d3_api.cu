@@ -87,6 +87,7 @@ struct d3_ctx {
   int tune_attn_div = 0;  // experiment: key tiles per attention split
   int tune_pair = -1;     // -1: by row count; 0 / 1: one / two row tiles per matmul unit
   int tune_no_rr = 0;     // 1: wide matmuls on contiguous unit ranges
+  bool gen_fuse = true;   // d3_generate fuses finalize forwards with the next block's first step while the forward stays skinny
   int tune_strip = 0;     // skinny matmuls as column strips: 0 when it pays, 1 never, 2 with one CTA per SM, 3 whenever possible
   int tune_no_cluster = 0;  // 1: skinny matmuls on the unit-range kernel (L2 reduction) instead of clusters
   int tune_wide_tiles = -1;  // -1: by row count; 0 / 1: force 128- / 256-column tiles
@@ -237,6 +238,10 @@ int get_tmap(d3_ctx* c, const void* ptr, int rows, int cols, int box_rows, const
   *out = &ins.first->second;
   return D3_OK;
 }
+
+// Up to this many rows a decode forward is bound by weight streaming, so twice the rows cost the same:
+// d3_generate then fuses a block's finalize forward with the next block's first denoise step.
+constexpr long long FUSE_MAX_ROWS = 64;
 
 // ---- matmul dispatch
 struct QkvExtra {
@@ -735,13 +740,14 @@ int run_stats_merge(d3_ctx* c, int M, int n_tiles, float* conf, float* ent, int*
 
 // The transformer stack over M rows laid out as bs x rows_per_seq (row map already on the device).
 //   head: 0 = none, 1 = fused statistics into ctx conf/ent/argmax, 2 = fp32 logits into `logits`.
-int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float* logits) {
+//   seg: rows per segment when a sequence's rows are consecutive blocks that must not see later ones (0: one segment).
+int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float* logits, int seg = 0) {
   const d3_config& g = c->cfg;
   const int M = bs * rows_per_seq;
   if (M == 0) return D3_OK;
   if (M > c->max_rows) return fail(c, D3_ERR_SHAPE, "forward over more rows than the workspaces hold");
   const int d = g.d_model, nq = g.n_q_heads * g.d_head, nkv = g.n_kv_heads * g.d_head, f = g.d_ffn;
-  RowMap rm{c->pos_base, c->n_valid, c->kv_len, rows_per_seq, bs};
+  RowMap rm{c->pos_base, c->n_valid, c->kv_len, rows_per_seq, bs, seg};
   c->last_rows = M;
 
   {
@@ -887,6 +893,9 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
                nkv = static_cast<size_t>(g.n_kv_heads) * g.d_head, f = g.d_ffn;
   long long pre_rows = g.max_prefill_rows > 0 ? g.max_prefill_rows : static_cast<long long>(g.max_batch) * g.max_seq;
   long long dec_rows = static_cast<long long>(g.max_batch) * g.block;
+  // d3_generate may run the finalize forward of a block together with the first step of the next one
+  // (2 * block rows per sequence) while that still is a skinny forward: room for it
+  if (2 * dec_rows <= FUSE_MAX_ROWS) dec_rows *= 2;
   c->max_rows = static_cast<int>(std::max(pre_rows, dec_rows));
   const size_t R = c->max_rows;
 #define A_(ptr, bytes)                                                         \
@@ -940,6 +949,8 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   c->gen.prefix_len = c->prefix_len;
   A_(c->gen.ids, sizeof(int) * dec_rows);
   A_(c->gen.mask, sizeof(uint8_t) * dec_rows);
+  A_(c->gen.prev, sizeof(int) * dec_rows);
+  A_(c->gen.fwd_ids, sizeof(int) * 2 * static_cast<size_t>(g.max_batch) * g.block);
   A_(c->gen.counters, sizeof(long long) * 8);
   if (cudaMallocHost(reinterpret_cast<void**>(&c->host_counters), sizeof(long long) * 8) != cudaSuccess)
     return bail(D3_ERR_OOM);
@@ -1185,17 +1196,20 @@ extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t 
   gen_init_kernel<<<bs, 32, 0, c->stream>>>(g, bs, B, c->cfg.mask_id);
   LAUNCHED(c, "gen_init_kernel");
   const long long max_iter = static_cast<long long>(n_blocks) * (B + 1) + 1;
+  const int fuse = (c->gen_fuse && 2ll * bs * B <= FUSE_MAX_ROWS && 2ll * c->cfg.max_batch * B <= FUSE_MAX_ROWS) ? 1 : 0;
   long long steps = 0;
+  int R = B;  // rows per sequence of the next forward: 2B while some sequence runs a fused finalize + first step
   for (long long it = 0; it < max_iter; ++it) {
-    gen_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(g, bs, B, c->pos_base, c->n_valid, c->kv_len);
+    gen_rowmap_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, R, c->cfg.mask_id, c->pos_base, c->n_valid, c->kv_len);
     LAUNCHED(c, "gen_rowmap_kernel");
-    TRY(forward(c, g.ids, bs, B, 1, nullptr));
-    gen_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, n_blocks, gen_len, threshold, c->cfg.decide_mode, c->cfg.mask_id);
+    TRY(forward(c, g.fwd_ids, bs, R, 1, nullptr, R > B ? B : 0));
+    gen_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, R, n_blocks, gen_len, threshold, c->cfg.decide_mode, c->cfg.mask_id, fuse);
     LAUNCHED(c, "gen_advance_kernel");
     ++steps;
-    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 5, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 6, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     if (c->host_counters[4] <= 0) break;
+    R = c->host_counters[5] > 0 ? 2 * B : B;
   }
   if (host_stats) {
     std::memset(host_stats, 0, sizeof(*host_stats));
@@ -1340,7 +1354,7 @@ extern "C" int d3_op_attention(d3_ctx* c, const void* q, int32_t layer, int32_t 
   // all rows live, positions irrelevant here
   decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(kv_len, bs, rows, c->pos_base, c->n_valid, c->kv_len);
   LAUNCHED(c, "decode_rowmap_kernel");
-  RowMap rm{c->pos_base, c->n_valid, kv_len, rows, bs};
+  RowMap rm{c->pos_base, c->n_valid, kv_len, rows, bs, 0};
   return run_attention(c, q, layer, out, rm);
 }
 
@@ -1384,7 +1398,9 @@ extern "C" int d3_get_error_word(d3_ctx* c, uint32_t* word) {
   return D3_OK;
 }
 extern "C" int d3_set_matmul_tuning(d3_ctx* c, int32_t ring_kb, int32_t ctas_per_sm) {
-  if (!c || ring_kb < 0 || (ring_kb & 0xffff) > 200 || ctas_per_sm < 0 || ctas_per_sm > 3) return D3_ERR_INVALID_ARG;
+  if (!c || ring_kb < 0 || (ring_kb & 0xffff) > 200 || ctas_per_sm < 0 || (ctas_per_sm & 0xff) > 3 || ctas_per_sm > 0x1ff) return D3_ERR_INVALID_ARG;
+  c->gen_fuse = ((ctas_per_sm >> 8) & 1) == 0;  // bit 8 of ctas_per_sm: d3_generate finalizes every block in a forward of its own
+  ctas_per_sm &= 0xff;
   c->tune_producers = (ring_kb >> 16) & 0xf;  // experiments: bits 16-19 of ring_kb = producer warps, 20-21 = tile width + 1
   c->tune_wide_tiles = ((ring_kb >> 20) & 3) - 1;
   c->tune_attn_div = (ring_kb >> 22) & 7;

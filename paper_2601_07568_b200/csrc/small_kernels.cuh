@@ -9,13 +9,22 @@ namespace d3 {
 // Per-sequence row map of one forward: row m belongs to sequence b = m / rows_per_seq at offset
 // r = m % rows_per_seq; it is live when r < n_valid[b] and sits at absolute position pos_base[b] + r;
 // its attention reads cache slots [0, kv_len[b]).
+// `seg` > 0 cuts the rows of a sequence into segments of `seg` rows (consecutive blocks in one
+// forward): row r then sees slots [0, pos_base[b] + (r / seg + 1) * seg) only - the prefix, the earlier
+// segments and its own, never a later one.  seg = 0: every row sees [0, kv_len[b]).
 struct RowMap {
   const int* pos_base;
   const int* n_valid;
   const int* kv_len;
   int rows_per_seq;
   int bs;
+  int seg;
 };
+__device__ __forceinline__ int row_kv_limit(const RowMap& rm, int b, int r, int kv_len) {
+  if (rm.seg <= 0) return kv_len;
+  const int lim = rm.pos_base[b] + (r / rm.seg + 1) * rm.seg;
+  return lim < kv_len ? lim : kv_len;
+}
 
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
@@ -312,41 +321,58 @@ __global__ void unmask_kernel(const float* __restrict__ conf, const float* __res
 }
 
 // ----------------------------------------------------------------------------- generate bookkeeping
-enum : int { SEQ_DENOISE = 0, SEQ_FINALIZE = 1, SEQ_DONE = 2 };
+// A sequence denoises its current block until no mask is left, then the block needs one more forward
+// on its final tokens so that the cached K/V are theirs (finalize).  That forward is independent of
+// the first denoise step of the next block except that the latter reads the former's K/V, which the
+// same forward writes before its attention runs: with `fuse` the two run as one forward of 2B rows
+// (segment 0 = the finished block, segment 1 = the new, fully masked block; segment 0 never sees
+// segment 1).  The last block of a request, and every block when fuse is off, is finalized alone.
+enum : int { SEQ_DENOISE = 0, SEQ_FINALIZE = 1, SEQ_DONE = 2, SEQ_FUSED = 3 };
 struct GenState {
   int* mode;        // [bs] SEQ_*
-  int* block_idx;   // [bs]
+  int* block_idx;   // [bs] block being denoised
   int* step;        // [bs] denoise steps taken in the current block
-  int* prefix_len;  // [bs]
+  int* prefix_len;  // [bs] cached prefix: prompt + finalized blocks
   int* ids;         // [bs, B] current block
   uint8_t* mask;    // [bs, B]
+  int* prev;        // [bs, B] finished block waiting for its finalize forward (SEQ_FUSED)
+  int* fwd_ids;     // [bs, 2B] ids of the next forward, rows_per_seq = B or 2B
   int* out_ids;     // [bs, gen_len]
   int* commit_step; // [bs, gen_len] or null
-  long long* counters;  // [0] denoise fwd, [1] finalize fwd, [2] tokens, [3] forced, [4] seqs not done
+  long long* counters;  // [0] denoise fwd, [1] finalize fwd, [2] tokens, [3] forced, [4] seqs not done, [5] seqs in SEQ_FUSED
 };
 
-// Row map of the next decode forward from the generate state (one thread per sequence).
-__global__ void gen_rowmap_kernel(GenState g, int bs, int B, int* pos_base, int* n_valid, int* kv_len) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= bs) return;
-  const bool live = g.mode[b] != SEQ_DONE;
-  pos_base[b] = g.prefix_len[b];
-  n_valid[b] = live ? B : 0;
-  kv_len[b] = live ? g.prefix_len[b] + B : 0;
+// Row map and input ids of the next decode forward (rows_per_seq = R, B or 2B) from the generate
+// state.  One block per sequence.
+__global__ void gen_rowmap_kernel(GenState g, int bs, int B, int R, int mask_id, int* pos_base, int* n_valid, int* kv_len) {
+  const int b = blockIdx.x;
+  const int mode = g.mode[b];
+  const int rows = mode == SEQ_DONE ? 0 : (mode == SEQ_FUSED ? 2 * B : B);
+  if (threadIdx.x == 0) {
+    pos_base[b] = g.prefix_len[b];
+    n_valid[b] = rows;
+    kv_len[b] = rows > 0 ? g.prefix_len[b] + rows : 0;
+  }
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    int id = mask_id;
+    if (mode == SEQ_FUSED) id = r < B ? g.prev[b * B + r] : g.ids[b * B + r - B];
+    else if (r < B) id = g.ids[b * B + r];
+    g.fwd_ids[b * R + r] = id;
+  }
 }
 
-// After a forward: sequences that ran a finalize forward append their block and start the next one;
-// sequences that ran a denoise forward take the unmask decision.  One warp per sequence.
+// After a forward of R rows per sequence: finalize bookkeeping and / or the unmask decision.  One warp
+// per sequence.
 __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, const float* __restrict__ ent,
-                                   const int* __restrict__ argmax, int bs, int B, int n_blocks, int gen_len, float tau,
-                                   int decide_mode, int mask_id) {
+                                   const int* __restrict__ argmax, int bs, int B, int R, int n_blocks, int gen_len,
+                                   float tau, int decide_mode, int mask_id, int fuse) {
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31;
   const int mode = g.mode[b];
   if (mode == SEQ_DONE) return;
   int* ids = g.ids + b * B;
   uint8_t* mask = g.mask + b * B;
-  if (mode == SEQ_FINALIZE) {
+  if (mode == SEQ_FINALIZE) {  // the block in `ids` is final and now cached: append it, next block or done
     const int j = g.block_idx[b];
     for (int r = lane; r < B; r += 32) {
       g.out_ids[static_cast<size_t>(b) * gen_len + j * B + r] = ids[r];
@@ -368,16 +394,45 @@ __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, c
     }
     return;
   }
+  int stat_row0 = b * R;  // rows of the block that was denoised in this forward
+  if (mode == SEQ_FUSED) {  // segment 0 finalized the block in `prev`: append it; segment 1 was a first denoise step
+    const int j = g.block_idx[b] - 1;
+    for (int r = lane; r < B; r += 32) g.out_ids[static_cast<size_t>(b) * gen_len + j * B + r] = g.prev[b * B + r];
+    if (lane == 0) {
+      g.prefix_len[b] += B;
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[1]), 1ull);
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[5]), static_cast<unsigned long long>(-1ll));
+    }
+    stat_row0 += B;
+  }
   const int step = g.step[b] + 1;
   int* cs = g.commit_step ? g.commit_step + static_cast<size_t>(b) * gen_len + g.block_idx[b] * B : nullptr;
-  UnmaskOut r = unmask_block(conf + b * B, ent + b * B, argmax + b * B, ids, mask, B, tau, decide_mode, nullptr,
-                             nullptr, cs, step);
+  UnmaskOut r = unmask_block(conf + stat_row0, ent + stat_row0, argmax + stat_row0, ids, mask, B, tau, decide_mode,
+                             nullptr, nullptr, cs, step);
+  __syncwarp();
+  const bool complete = r.remaining == 0;
+  const bool to_fused = complete && fuse && g.block_idx[b] + 1 < n_blocks;
+  if (to_fused) {  // hand the finished block to the next forward's segment 0 and open the next block
+    for (int q = lane; q < B; q += 32) {
+      g.prev[b * B + q] = ids[q];
+      ids[q] = mask_id;
+      mask[q] = 1;
+    }
+  }
+  __syncwarp();
   if (lane == 0) {
-    g.step[b] = step;
     atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[0]), 1ull);
     atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[2]), static_cast<unsigned long long>(r.committed));
     atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[3]), static_cast<unsigned long long>(r.forced));
-    if (r.remaining == 0) g.mode[b] = SEQ_FINALIZE;
+    if (to_fused) {
+      g.mode[b] = SEQ_FUSED;
+      g.block_idx[b] += 1;
+      g.step[b] = 0;
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[5]), 1ull);
+    } else {
+      g.step[b] = step;
+      g.mode[b] = complete ? SEQ_FINALIZE : SEQ_DENOISE;
+    }
   }
 }
 
@@ -392,7 +447,7 @@ __global__ void gen_init_kernel(GenState g, int bs, int B, int mask_id) {
     g.block_idx[b] = 0;
     g.step[b] = 0;
     if (b == 0) {
-      g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = 0;
+      g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = g.counters[5] = 0;
       g.counters[4] = bs;
     }
   }
