@@ -23,6 +23,12 @@ What the paper fixes (cited per function) and what it leaves open
   KV-cache paragraph: a short delay before caching).
 * Unmasking exactly one token per step is the teacher-trajectory mode
   (Sec. 3.1; Appendix, pseudo-trajectory extraction).
+* Decoding halts as soon as the end-of-sequence token has been generated
+  (Sec. 3.2, "Early Stopping on EOS Token"): the generated tokens are checked
+  after every decoding step.  Reading taken here: the sequence stops after the
+  step that commits the EOS id anywhere in the current block; positions that
+  are still masked (in this block and all later ones) are returned as the
+  mask id, and the unfinished block gets no finalize forward.
 
 Readings taken where the paper is silent are listed in the repository's
 design notes; in short: block-causal visibility between segments (prompt =
@@ -308,16 +314,20 @@ class OracleModel:
                         [np.concatenate([a, b], axis=0) for a, b in zip(state.v, vs)])
 
     def generate(self, prompt: np.ndarray, gen_len: int, block: int, tau: float,
-                 mode: int = MODE_CONFIDENCE, record: bool = False) -> Dict[str, object]:
+                 mode: int = MODE_CONFIDENCE, record: bool = False,
+                 eos_id: Optional[int] = None) -> Dict[str, object]:
         """Block-by-block threshold decoding of one sequence.
 
         Returns tokens [gen_len], the step index (within its block, from 1) at which each
-        position was committed, forward counts, and optionally a per-step trace."""
+        position was committed, forward counts, and optionally a per-step trace.  With
+        ``eos_id`` decoding halts after the step that commits that id (Sec. 3.2, early
+        stopping on EOS); undecoded positions stay ``mask_id``."""
         assert gen_len % block == 0
         state = self.prefill(prompt)
         out = np.full(gen_len, self.mask_id, dtype=np.int32)
         commit_step = np.zeros(gen_len, dtype=np.int32)
         n_denoise = n_finalize = 0
+        stopped = False
         trace: List[Dict[str, object]] = []
         for j in range(gen_len // block):
             ids = np.full(block, self.mask_id, dtype=np.int32)
@@ -334,10 +344,17 @@ class OracleModel:
                     trace.append(dict(block=j, step=step, prefix_len=state.prefix_len, ids_in=ids_in,
                                       mask_in=mask_in, conf=conf, tok=tok, ent=ent, commit=commit,
                                       ids_out=ids.copy(), mask_out=mask.copy()))
+                if eos_id is not None and np.any(ids[commit] == eos_id):
+                    stopped = True
+                    break
+            if stopped:
+                out[j * block:(j + 1) * block] = np.where(mask, self.mask_id, ids)
+                break
             state = self.finalize_block(state, ids)
             n_finalize += 1
             out[j * block:(j + 1) * block] = ids
         res = dict(tokens=out, commit_step=commit_step, n_denoise=n_denoise, n_finalize=n_finalize,
+                   stopped_early=stopped,
                    tpf_denoise=gen_len / max(n_denoise, 1),
                    tpf_all=gen_len / max(n_denoise + n_finalize, 1), state=state)
         if record:

@@ -284,3 +284,43 @@ def test_mirror_mode_stays_close_to_exact():
     la = a.denoise_forward(a.prefill(ids[:12]), ids[12:])[0]
     lb = b.denoise_forward(b.prefill(ids[:12]), ids[12:])[0]
     assert np.max(np.abs(la - lb)) < 3e-2 * np.max(np.abs(la))
+
+
+def test_eos_early_stop_is_a_prefix_of_the_run_without_it():
+    """Early stopping on EOS (Sec. 3.2): with the EOS id set to a token that the free run first commits
+    at step k of block j, decoding makes exactly the same commits up to and including that step, then
+    stops: no later forward, every undecoded position still the mask id, j finalize forwards."""
+    w = si.WORKLOADS["c1"]
+    W = si.gen_weights(w.model)
+    ids, lens = si.gen_prompts(w)
+    model = o.model_from_shape(w.model, W, np.float64)
+    prompt = ids[0, :lens[0]]
+    free = model.generate(prompt, w.gen_len, w.block, 0.3, record=True)
+    assert not free["stopped_early"] and free["n_finalize"] == w.gen_len // w.block
+    trace = free["trace"]
+    # the last step (not the very first) that commits a token no earlier step has committed
+    seen = set()
+    pick = None
+    for n, t in enumerate(trace):
+        toks = [int(x) for x in t["ids_out"][t["commit"]]]
+        fresh = [x for x in toks if x not in seen]
+        if n >= 1 and fresh:
+            pick = (n, fresh[0])
+        seen.update(toks)
+    assert pick is not None and trace[pick[0]]["block"] >= 1
+    n_stop, eos = pick
+    got = model.generate(prompt, w.gen_len, w.block, 0.3, eos_id=eos)
+    t = trace[n_stop]
+    assert got["stopped_early"]
+    assert got["n_denoise"] == n_stop + 1 and got["n_finalize"] == t["block"]
+    want = np.full(w.gen_len, w.model.mask_id, dtype=np.int32)
+    B = w.block
+    want[:t["block"] * B] = free["tokens"][:t["block"] * B]
+    want[t["block"] * B:(t["block"] + 1) * B] = np.where(t["mask_out"], w.model.mask_id, t["ids_out"])
+    assert np.array_equal(got["tokens"], want)
+    assert np.any(got["tokens"] == eos) and np.any(got["tokens"] == w.model.mask_id)
+    assert got["n_denoise"] < free["n_denoise"]
+    # an id that never comes up changes nothing
+    never = next(x for x in range(w.model.vocab) if x not in seen and x != w.model.mask_id)
+    same = model.generate(prompt, w.gen_len, w.block, 0.3, eos_id=never)
+    assert not same["stopped_early"] and np.array_equal(same["tokens"], free["tokens"])
