@@ -149,6 +149,15 @@ int d3_commit_block(d3_ctx *ctx, const int32_t *block_ids, int32_t bs);
 int d3_generate(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32_t *out_ids,
                 int32_t *commit_step, d3_stats *host_stats);
 
+/* Early stopping on the end-of-sequence token (Sec. 3.2, "Early Stopping on EOS Token"): with an id set,
+ * d3_generate stops a sequence after the denoise step that commits that id anywhere in its current
+ * block.  The block goes out as it stands, undecoded positions (there and in all later blocks) read
+ * mask_id, the unfinished block is not added to the cache, and tokens_committed counts what was
+ * decoded.  eos_id < 0 switches it off (the default).  INVALID_ARG for ids outside the vocabulary or
+ * equal to mask_id.  d3_early_stops: sequences of the latest d3_generate call that stopped this way. */
+int d3_set_eos(d3_ctx *ctx, int32_t eos_id);
+int64_t d3_early_stops(d3_ctx *ctx);
+
 /* Statistics of the latest denoise forward: conf, entropy [device][bs*B] float, argmax
  * [device][bs*B] int32 (any may be NULL). */
 int d3_get_step_stats(d3_ctx *ctx, float *conf, float *entropy, int32_t *argmax, int32_t bs);

@@ -87,6 +87,8 @@ struct d3_ctx {
   int tune_attn_div = 0;  // experiment: key tiles per attention split
   int tune_pair = -1;     // -1: by row count; 0 / 1: one / two row tiles per matmul unit
   int tune_no_rr = 0;     // 1: wide matmuls on contiguous unit ranges
+  int eos_id = -1;        // d3_generate stops a sequence once this id has been committed (< 0: never)
+  long long last_early_stops = 0;
   bool gen_fuse = true;   // d3_generate fuses finalize forwards with the next block's first step while the forward stays skinny
   int tune_strip = 0;     // skinny matmuls as column strips: 0 when it pays, 1 never, 2 with one CTA per SM, 3 whenever possible
   int tune_no_cluster = 0;  // 1: skinny matmuls on the unit-range kernel (L2 reduction) instead of clusters
@@ -1193,7 +1195,7 @@ extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t 
   GenState g = c->gen;
   g.out_ids = out_ids;
   g.commit_step = commit_step;
-  gen_init_kernel<<<bs, 32, 0, c->stream>>>(g, bs, B, c->cfg.mask_id);
+  gen_init_kernel<<<bs, 32, 0, c->stream>>>(g, bs, B, c->cfg.mask_id, gen_len);
   LAUNCHED(c, "gen_init_kernel");
   const long long max_iter = static_cast<long long>(n_blocks) * (B + 1) + 1;
   const int fuse = (c->gen_fuse && 2ll * bs * B <= FUSE_MAX_ROWS && 2ll * c->cfg.max_batch * B <= FUSE_MAX_ROWS) ? 1 : 0;
@@ -1203,14 +1205,15 @@ extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t 
     gen_rowmap_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, R, c->cfg.mask_id, c->pos_base, c->n_valid, c->kv_len);
     LAUNCHED(c, "gen_rowmap_kernel");
     TRY(forward(c, g.fwd_ids, bs, R, 1, nullptr, R > B ? B : 0));
-    gen_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, R, n_blocks, gen_len, threshold, c->cfg.decide_mode, c->cfg.mask_id, fuse);
+    gen_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, R, n_blocks, gen_len, threshold, c->cfg.decide_mode, c->cfg.mask_id, fuse, c->eos_id);
     LAUNCHED(c, "gen_advance_kernel");
     ++steps;
-    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 6, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 7, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     if (c->host_counters[4] <= 0) break;
     R = c->host_counters[5] > 0 ? 2 * B : B;
   }
+  c->last_early_stops = c->host_counters[6];
   if (host_stats) {
     std::memset(host_stats, 0, sizeof(*host_stats));
     host_stats->denoise_forwards = c->host_counters[0];
@@ -1223,6 +1226,14 @@ extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t 
   if (c->host_counters[4] > 0) return fail(c, D3_ERR_STATE, "generate loop did not finish within its step bound");
   return check_device_error(c);
 }
+
+extern "C" int d3_set_eos(d3_ctx* c, int32_t eos_id) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (eos_id >= c->cfg.vocab || eos_id == c->cfg.mask_id) return fail(c, D3_ERR_INVALID_ARG, "eos id outside the vocabulary or equal to the mask id");
+  c->eos_id = eos_id < 0 ? -1 : eos_id;
+  return D3_OK;
+}
+extern "C" int64_t d3_early_stops(d3_ctx* c) { return c ? c->last_early_stops : 0; }
 
 extern "C" int d3_get_step_stats(d3_ctx* c, float* conf, float* entropy, int32_t* argmax, int32_t bs) {
   if (!c || bs <= 0 || bs > c->cfg.max_batch) return D3_ERR_INVALID_ARG;

@@ -339,7 +339,8 @@ struct GenState {
   int* fwd_ids;     // [bs, 2B] ids of the next forward, rows_per_seq = B or 2B
   int* out_ids;     // [bs, gen_len]
   int* commit_step; // [bs, gen_len] or null
-  long long* counters;  // [0] denoise fwd, [1] finalize fwd, [2] tokens, [3] forced, [4] seqs not done, [5] seqs in SEQ_FUSED
+  long long* counters;  // [0] denoise fwd, [1] finalize fwd, [2] tokens, [3] forced, [4] seqs not done, [5] seqs in SEQ_FUSED,
+                        // [6] sequences stopped early on the end-of-sequence id
 };
 
 // Row map and input ids of the next decode forward (rows_per_seq = R, B or 2B) from the generate
@@ -365,7 +366,7 @@ __global__ void gen_rowmap_kernel(GenState g, int bs, int B, int R, int mask_id,
 // per sequence.
 __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, const float* __restrict__ ent,
                                    const int* __restrict__ argmax, int bs, int B, int R, int n_blocks, int gen_len,
-                                   float tau, int decide_mode, int mask_id, int fuse) {
+                                   float tau, int decide_mode, int mask_id, int fuse, int eos_id) {
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31;
   const int mode = g.mode[b];
@@ -407,9 +408,38 @@ __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, c
   }
   const int step = g.step[b] + 1;
   int* cs = g.commit_step ? g.commit_step + static_cast<size_t>(b) * gen_len + g.block_idx[b] * B : nullptr;
+  // positions masked before the decision: those that are not afterwards were committed in this step
+  bool was_masked[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) was_masked[q] = lane + 32 * q < B && mask[lane + 32 * q] != 0;
   UnmaskOut r = unmask_block(conf + stat_row0, ent + stat_row0, argmax + stat_row0, ids, mask, B, tau, decide_mode,
                              nullptr, nullptr, cs, step);
   __syncwarp();
+  // early stop: the end-of-sequence id was committed in this step.  The sequence is done; its current
+  // block goes out as it is (mask id where nothing was decided), later blocks stay mask ids, and the
+  // unfinished block is not cached.
+  bool hit = false;
+  if (eos_id >= 0) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const int pos = lane + 32 * q;
+      if (was_masked[q] && mask[pos] == 0 && ids[pos] == eos_id) hit = true;
+    }
+  }
+  if (__any_sync(0xffffffffu, hit)) {
+    const int j = g.block_idx[b];
+    for (int q = lane; q < B; q += 32) g.out_ids[static_cast<size_t>(b) * gen_len + j * B + q] = mask[q] ? mask_id : ids[q];
+    if (lane == 0) {
+      g.step[b] = step;
+      g.mode[b] = SEQ_DONE;
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[0]), 1ull);
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[2]), static_cast<unsigned long long>(r.committed));
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[3]), static_cast<unsigned long long>(r.forced));
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[4]), static_cast<unsigned long long>(-1ll));
+      atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[6]), 1ull);
+    }
+    return;
+  }
   const bool complete = r.remaining == 0;
   const bool to_fused = complete && fuse && g.block_idx[b] + 1 < n_blocks;
   if (to_fused) {  // hand the finished block to the next forward's segment 0 and open the next block
@@ -436,18 +466,20 @@ __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, c
   }
 }
 
-__global__ void gen_init_kernel(GenState g, int bs, int B, int mask_id) {
+__global__ void gen_init_kernel(GenState g, int bs, int B, int mask_id, int gen_len) {
   const int b = blockIdx.x;
   for (int r = threadIdx.x; r < B; r += blockDim.x) {
     g.ids[b * B + r] = mask_id;
     g.mask[b * B + r] = 1;
   }
+  // what is never decoded (early stop) reads as the mask id
+  for (int r = threadIdx.x; r < gen_len; r += blockDim.x) g.out_ids[static_cast<size_t>(b) * gen_len + r] = mask_id;
   if (threadIdx.x == 0) {
     g.mode[b] = SEQ_DENOISE;
     g.block_idx[b] = 0;
     g.step[b] = 0;
     if (b == 0) {
-      g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = g.counters[5] = 0;
+      g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = g.counters[5] = g.counters[6] = 0;
       g.counters[4] = bs;
     }
   }

@@ -218,6 +218,70 @@ def test_generate_fused_finalize_bf16_tensor_core():
     assert same_ref or near_tie
 
 
+def test_generate_stops_on_eos_like_the_oracle():
+    """Early stopping on EOS (Sec. 3.2): a batch of three fp32 sequences, the EOS id chosen as a token
+    that one of them commits midway.  Sequences that commit it stop after that step, the others run to
+    the end; tokens, commit steps and per-sequence forward counts equal the oracle's, bit for bit."""
+    shape = si.TINY
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("eos", shape, 3, [32, 11, 20], 64, 16, 0.3, 41)
+    model = o.model_from_shape(shape, W, np.float64)
+    free = [model.generate(ids[b, :lens[b]], 64, 16, 0.3, record=True) for b in range(3)]
+    # the token sequence 0 commits last for the first time, at a step that is not its first
+    seen, eos = set(), None
+    for n, t in enumerate(free[0]["trace"]):
+        toks = [int(x) for x in t["ids_out"][t["commit"]]]
+        fresh = [x for x in toks if x not in seen]
+        if n >= 1 and fresh:
+            eos = fresh[0]
+        seen.update(toks)
+    assert eos is not None
+    ref = [model.generate(ids[b, :lens[b]], 64, 16, 0.3, eos_id=eos) for b in range(3)]
+    assert ref[0]["stopped_early"]
+    with Ctx(shape, W, block=16, max_batch=3, max_seq=wl.max_seq) as ctx:
+        d3.d3_set_eos(ctx.ctx, eos)
+        ctx.prefill(ids, lens)
+        tok, cs, st = ctx.generate(3, 64, 0.3)
+        for b in range(3):
+            assert np.array_equal(tok[b], ref[b]["tokens"]), b
+            assert np.array_equal(cs[b], ref[b]["commit_step"]), b
+        assert st.denoise_forwards == sum(r["n_denoise"] for r in ref)
+        assert st.finalize_forwards == sum(r["n_finalize"] for r in ref)
+        assert st.tokens_committed == sum(int((r["tokens"] != shape.mask_id).sum()) for r in ref)
+        assert d3.d3_early_stops(ctx.ctx) == sum(int(r["stopped_early"]) for r in ref) >= 1
+        # switched off again: the free run
+        d3.d3_set_eos(ctx.ctx, -1)
+        ctx.prefill(ids, lens)
+        tok2, _, st2 = ctx.generate(3, 64, 0.3)
+        for b in range(3):
+            assert np.array_equal(tok2[b], free[b]["tokens"]), b
+        assert d3.d3_early_stops(ctx.ctx) == 0 and st2.tokens_committed == 3 * 64
+        with pytest.raises(d3.D3Error):
+            d3.d3_set_eos(ctx.ctx, shape.mask_id)
+        assert ctx.error_word() == 0
+
+
+def test_generate_stops_on_eos_at_batch_one_with_fused_finalize(c1):
+    """The same at batch 1, where finalize forwards ride along with the next block's first step: the
+    stop may fall into such a fused step."""
+    w, model, ids, lens, ctx = c1
+    free = model.generate(ids[0, :lens[0]], w.gen_len, w.block, 0.3, record=True)
+    for t in free["trace"]:
+        if t["block"] >= 1 and t["step"] == 1:  # a first step of a later block: runs fused on the GPU
+            eos = int(t["ids_out"][t["commit"]][0])
+            break
+    ref = model.generate(ids[0, :lens[0]], w.gen_len, w.block, 0.3, eos_id=eos)
+    d3.d3_set_eos(ctx.ctx, eos)
+    try:
+        ctx.prefill(ids, lens)
+        tok, cs, st = ctx.generate(1, w.gen_len, 0.3)
+    finally:
+        d3.d3_set_eos(ctx.ctx, -1)
+    assert np.array_equal(tok[0], ref["tokens"]) and np.array_equal(cs[0], ref["commit_step"])
+    assert st.denoise_forwards == ref["n_denoise"] and st.finalize_forwards == ref["n_finalize"]
+    assert d3.d3_early_stops(ctx.ctx) == int(ref["stopped_early"])
+
+
 def test_c1_entropy_mode():
     w = si.WORKLOADS["c1"]
     W = si.gen_weights(w.model)
