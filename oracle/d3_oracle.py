@@ -23,6 +23,20 @@ What the paper fixes (cited per function) and what it leaves open
   KV-cache paragraph: a short delay before caching).
 * Unmasking exactly one token per step is the teacher-trajectory mode
   (Sec. 3.1; Appendix, pseudo-trajectory extraction).
+* Multi-block decoding (Sec. 3.2, "Entropy-Based Multi-Block Parallel
+  Decoding"): the current and future blocks are decoded in one forward pass.  A
+  new block is created (Activated) when its predecessor is 10 % complete and
+  decodes only tokens that clear the threshold; when the predecessor is 95 %
+  complete it is Fully-Activated and decodes at least one token per forward; a
+  block whose tokens are all unmasked goes through one more forward
+  (Completed but Stabilizing) before its key/value states are stored
+  (Completed).  Readings taken here: blocks in flight see the cache, earlier
+  blocks in flight and themselves, never later ones (the same block-causal
+  visibility as everywhere else, so a stabilizing forward shared with other
+  blocks equals one of its own); states are read from the masks as they stand
+  before a forward; completion is compared in integers (100 u >= 10 B, 100 u >=
+  95 B for u unmasked of B tokens); the number of blocks in flight is bounded
+  by a parameter; blocks enter the cache in order, one stabilizing round each.
 * Decoding halts as soon as the end-of-sequence token has been generated
   (Sec. 3.2, "Early Stopping on EOS Token"): the generated tokens are checked
   after every decoding step.  Reading taken here: the sequence stops after the
@@ -357,6 +371,84 @@ class OracleModel:
                    stopped_early=stopped,
                    tpf_denoise=gen_len / max(n_denoise, 1),
                    tpf_all=gen_len / max(n_denoise + n_finalize, 1), state=state)
+        if record:
+            res["trace"] = trace
+        return res
+
+    def generate_multiblock(self, prompt: np.ndarray, gen_len: int, block: int, tau: float,
+                            mode: int = MODE_ENTROPY, max_active: int = 2, record: bool = False
+                            ) -> Dict[str, object]:
+        """Multi-block decoding of one sequence (Sec. 3.2, multi-block decoding strategy).
+
+        Every round is one forward over the blocks in flight (oldest first), each seeing the
+        cache, the earlier blocks in flight as they stand (masked rows included) and itself.
+        Returns tokens [gen_len], the round (from 1) in which each position was committed, the
+        number of rounds, the rows each round covered, and optionally a per-round trace."""
+        assert gen_len % block == 0 and max_active >= 1
+        n_blocks = gen_len // block
+        state = self.prefill(prompt)
+        out = np.full(gen_len, self.mask_id, dtype=np.int32)
+        commit_round = np.zeros(gen_len, dtype=np.int32)
+        lo = 0                                   # first block in flight
+        win_ids: List[np.ndarray] = [np.full(block, self.mask_id, dtype=np.int32)]
+        win_mask: List[np.ndarray] = [np.ones(block, dtype=bool)]
+        rounds = 0
+        rows: List[int] = []
+        trace: List[Dict[str, object]] = []
+        while win_ids:
+            rounds += 1
+            assert rounds <= n_blocks * (block + 1) + 1, "every round must make progress"
+            n_win = len(win_ids)
+            rows.append(n_win * block)
+            # states as the masks stand before the forward
+            unmasked = [int(block - m.sum()) for m in win_mask]
+            complete_before = [u == block for u in unmasked]
+            fully = [True if w == 0 else 100 * unmasked[w - 1] >= 95 * block for w in range(n_win)]
+            ids_in = [a.copy() for a in win_ids]
+            mask_in = [a.copy() for a in win_mask]
+            # the forward: block w sees the cache and blocks 0..w-1 of the window
+            tmp = state
+            stats = []
+            for w in range(n_win):
+                _, conf, tok, ent = self.denoise_forward(tmp, win_ids[w])
+                stats.append((conf, tok, ent))
+                if w + 1 < n_win:
+                    tmp = self.finalize_block(tmp, win_ids[w])
+            # decisions
+            commits = []
+            for w in range(n_win):
+                conf, tok, ent = stats[w]
+                m = win_mask[w]
+                if complete_before[w]:
+                    commit = np.zeros(block, dtype=bool)
+                elif fully[w]:
+                    commit = decide(conf, ent, m, tau, mode)
+                else:  # Activated: only what clears the threshold
+                    commit = m & ((conf > tau) if mode == MODE_CONFIDENCE else (ent < tau))
+                win_ids[w] = win_ids[w].copy()
+                win_ids[w][commit] = tok[commit]
+                win_mask[w] = m & ~commit
+                commit_round[(lo + w) * block:(lo + w + 1) * block][commit] = rounds
+                commits.append(commit)
+            if record:
+                trace.append(dict(round=rounds, lo=lo, n_win=n_win, fully=list(fully), ids_in=ids_in, mask_in=mask_in,
+                                  complete_before=list(complete_before), stats=stats, commits=commits,
+                                  ids_out=[a.copy() for a in win_ids], mask_out=[a.copy() for a in win_mask]))
+            # blocks that were complete before this forward have had their stabilizing round: the
+            # oldest ones enter the cache, in order
+            while win_ids and complete_before[0]:
+                state = self.finalize_block(state, win_ids[0])
+                out[lo * block:(lo + 1) * block] = win_ids[0]
+                win_ids.pop(0); win_mask.pop(0); complete_before.pop(0)
+                lo += 1
+            # a new block: when the newest one is 10 % complete (or nothing is in flight)
+            nxt = lo + len(win_ids)
+            if nxt < n_blocks and len(win_ids) < max_active:
+                if not win_ids or 100 * int(block - win_mask[-1].sum()) >= 10 * block:
+                    win_ids.append(np.full(block, self.mask_id, dtype=np.int32))
+                    win_mask.append(np.ones(block, dtype=bool))
+        res = dict(tokens=out, commit_round=commit_round, rounds=rounds, rows=rows, state=state,
+                   tokens_per_round=gen_len / max(rounds, 1))
         if record:
             res["trace"] = trace
         return res

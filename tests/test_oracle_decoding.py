@@ -324,3 +324,85 @@ def test_eos_early_stop_is_a_prefix_of_the_run_without_it():
     never = next(x for x in range(w.model.vocab) if x not in seen and x != w.model.mask_id)
     same = model.generate(prompt, w.gen_len, w.block, 0.3, eos_id=never)
     assert not same["stopped_early"] and np.array_equal(same["tokens"], free["tokens"])
+
+
+# ----------------------------------------------------------------------------- multi-block decoding
+def _c1_model():
+    w = si.WORKLOADS["c1"]
+    W = si.gen_weights(w.model)
+    ids, lens = si.gen_prompts(w)
+    return w, o.model_from_shape(w.model, W, np.float64), ids[0, :lens[0]]
+
+
+@pytest.mark.parametrize("tau,mode", [(0.9, o.MODE_CONFIDENCE), (0.3, o.MODE_CONFIDENCE), (2.42, o.MODE_ENTROPY)])
+def test_multiblock_with_one_block_in_flight_is_single_block_decoding(tau, mode):
+    """Multi-block decoding (Sec. 3.2) bounded to one block in flight has nothing to run in parallel: the
+    same tokens in the same order as block-by-block decoding, one round per denoise or finalize forward."""
+    w, model, prompt = _c1_model()
+    one = model.generate(prompt, w.gen_len, w.block, tau, mode, record=True)
+    mb = model.generate_multiblock(prompt, w.gen_len, w.block, tau, mode, max_active=1)
+    assert np.array_equal(mb["tokens"], one["tokens"])
+    assert mb["rounds"] == one["n_denoise"] + one["n_finalize"]
+    assert all(r == w.block for r in mb["rows"])
+    # commit order: rounds of the multi-block run count the finalize forwards of earlier blocks too
+    B = w.block
+    for j in range(w.gen_len // B):
+        steps = one["commit_step"][j * B:(j + 1) * B]
+        rounds = mb["commit_round"][j * B:(j + 1) * B]
+        assert np.array_equal(rounds - rounds.min(), steps - steps.min())
+    for a, b in zip(mb["state"].k, one["state"].k):
+        assert np.array_equal(a, b)
+
+
+@pytest.mark.parametrize("tau,mode,max_active", [(0.3, o.MODE_CONFIDENCE, 2), (2.42, o.MODE_ENTROPY, 3), (0.9, o.MODE_CONFIDENCE, 4)])
+def test_multiblock_rounds_follow_the_state_rules_and_the_joint_forward_is_block_causal(tau, mode, max_active):
+    """Each round against what the paper fixes: a block is created only once its predecessor is 10 %
+    complete, an Activated block (predecessor below 95 %) commits nothing but what clears the threshold,
+    a Fully-Activated one at least one token, a complete block commits nothing and enters the cache
+    after one more forward, in order.  And the statistics a block in flight gets are those of a
+    forward without any cache over prompt + earlier blocks (as they stand) + the block, under
+    segment visibility: evaluating the blocks in flight one after the other is the joint forward."""
+    w, model, prompt = _c1_model()
+    B, n_blocks = w.block, w.gen_len // w.block
+    res = model.generate_multiblock(prompt, w.gen_len, B, tau, mode, max_active=max_active, record=True)
+    tr = res["trace"]
+    assert res["rounds"] == len(tr) and np.all(res["commit_round"] >= 1) and not np.any(res["tokens"] == w.model.mask_id)
+    single = model.generate(prompt, w.gen_len, B, tau, mode)
+    assert res["rounds"] <= single["n_denoise"] + single["n_finalize"]
+    cached: list = []
+    checked_joint = 0
+    for n, t in enumerate(tr):
+        assert 1 <= t["n_win"] <= max_active and res["rows"][n] == t["n_win"] * B
+        assert t["lo"] == len(cached)
+        for k in range(t["n_win"]):
+            m_in, commit = t["mask_in"][k], t["commits"][k]
+            conf, tok, ent = t["stats"][k]
+            unm_prev = B if k == 0 else int(B - t["mask_in"][k - 1].sum())
+            fully = k == 0 or 100 * unm_prev >= 95 * B
+            assert fully == t["fully"][k]
+            clears = m_in & ((conf > tau) if mode == o.MODE_CONFIDENCE else (ent < tau))
+            if not m_in.any():
+                assert not commit.any() and t["complete_before"][k]
+            elif fully:
+                assert commit.sum() >= 1 and np.array_equal(commit | clears, commit) and (commit & ~m_in).sum() == 0
+                assert (commit & ~clears).sum() <= 1
+            else:
+                assert np.array_equal(commit, clears)
+            if t["n_win"] >= 2 and k >= 1 and checked_joint < 3:
+                lg, c2, t2, e2 = model.brute_force_block(prompt, cached + [t["ids_in"][q] for q in range(k)], t["ids_in"][k])
+                assert np.allclose(c2, conf, rtol=1e-9, atol=1e-12) and np.array_equal(t2, tok)
+                checked_joint += 1
+        # a block appears only when its predecessor is 10 % complete (or nothing was in flight)
+        if n + 1 < len(tr):
+            nxt = tr[n + 1]
+            popped = nxt["lo"] - t["lo"]
+            for q in range(popped):
+                assert t["complete_before"][q]
+                cached.append(t["ids_out"][q])
+            if nxt["n_win"] > t["n_win"] - popped:
+                assert nxt["n_win"] == t["n_win"] - popped + 1
+                if t["n_win"] - popped > 0:
+                    assert 100 * int(B - t["mask_out"][-1].sum()) >= 10 * B
+                assert nxt["mask_in"][-1].all()
+    assert checked_joint >= 1
+    assert np.array_equal(np.concatenate(cached + [x for x in tr[-1]["ids_out"]])[:w.gen_len], res["tokens"])
