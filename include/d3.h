@@ -149,6 +149,23 @@ int d3_commit_block(d3_ctx *ctx, const int32_t *block_ids, int32_t bs);
 int d3_generate(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32_t *out_ids,
                 int32_t *commit_step, d3_stats *host_stats);
 
+/* Multi-block decoding after d3_prefill (Sec. 3.2, "Entropy-Based Multi-Block Parallel Decoding"): up to
+ * max_active (1..8) consecutive blocks of a sequence are in flight; every round is one forward over
+ * all of them (a block sees the cache, the earlier blocks in flight and itself) followed by the
+ * decisions.  A block is opened, fully masked, once the newest block in flight is 10 % unmasked; it
+ * commits only what clears the threshold (config decide_mode: confidence > threshold, or entropy <
+ * threshold) while its predecessor is less than 95 % unmasked, and at least one token per round
+ * afterwards; a block without masks takes part in one more round before its K/V count as cached
+ * (blocks enter the cache in order).  States are read from the masks as they stand before a round.
+ * max_active = 1 is block-by-block decoding with every finalize forward on its own.
+ * out_ids [device][bs, gen_len]; commit_round (may be NULL) [device][bs, gen_len]: 1-based round in
+ * which each position was committed.  host_stats (may be NULL): steps = rounds, denoise_forwards =
+ * (sequence, block) decisions taken, finalize_forwards = blocks stored in the cache.  Waits for the
+ * stream.  Errors: SHAPE when gen_len is not a multiple of B, prefix + gen_len > max_seq, or
+ * bs * max_active * B rows exceed the workspaces sized by max_batch. */
+int d3_generate_multiblock(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32_t max_active,
+                           int32_t *out_ids, int32_t *commit_round, d3_stats *host_stats);
+
 /* Early stopping on the end-of-sequence token (Sec. 3.2, "Early Stopping on EOS Token"): with an id set,
  * d3_generate stops a sequence after the denoise step that commits that id anywhere in its current
  * block.  The block goes out as it stands, undecoded positions (there and in all later blocks) read

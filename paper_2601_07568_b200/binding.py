@@ -27,7 +27,7 @@ EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
     "d3_get_state", "d3_set_state", "d3_op_linear", "d3_packed_weight_elems", "d3_pack_weight", "d3_op_linear_packed", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_device_bytes",
+    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_generate_multiblock", "d3_device_bytes",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
 
@@ -181,6 +181,17 @@ def d3_generate(ctx, gen_len: int, threshold: float, out_ids: torch.Tensor,
                                   _ptr(_dev(out_ids, torch.int32)),
                                   _ptr(_dev(commit_step, torch.int32)) if commit_step is not None else C.c_void_p(0),
                                   C.byref(st)))
+    return st
+
+
+def d3_generate_multiblock(ctx, gen_len: int, threshold: float, out_ids: torch.Tensor, max_active: int,
+                           commit_round: Optional[torch.Tensor] = None) -> d3_stats:
+    st = d3_stats()
+    bs = out_ids.shape[0]
+    _check(ctx, lib().d3_generate_multiblock(ctx, C.c_int32(gen_len), C.c_float(threshold), C.c_int32(bs),
+                                             C.c_int32(max_active), _ptr(_dev(out_ids, torch.int32)),
+                                             _ptr(_dev(commit_round, torch.int32)) if commit_round is not None else C.c_void_p(0),
+                                             C.byref(st)))
     return st
 
 

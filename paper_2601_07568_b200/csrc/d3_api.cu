@@ -70,6 +70,8 @@ struct d3_ctx {
   int n_tile_count = 0;
   // generate state
   GenState gen{};
+  MbState mb{};           // multi-block decoding state (d3_generate_multiblock)
+  int stat_rows = 0;      // rows the statistics buffers hold
   long long* host_counters = nullptr;  // pinned
   // taps
   int tap_layer = -1;
@@ -952,6 +954,14 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   A_(c->gen.ids, sizeof(int) * dec_rows);
   A_(c->gen.mask, sizeof(uint8_t) * dec_rows);
   A_(c->gen.prev, sizeof(int) * dec_rows);
+  c->stat_rows = static_cast<int>(dec_rows);
+  c->mb.prefix_len = c->prefix_len;
+  c->mb.counters = nullptr;  // shares gen.counters (set below)
+  A_(c->mb.lo, sizeof(int) * g.max_batch);
+  A_(c->mb.n_win, sizeof(int) * g.max_batch);
+  A_(c->mb.ids, sizeof(int) * static_cast<size_t>(g.max_batch) * MB_MAX_WINDOW * g.block);
+  A_(c->mb.mask, sizeof(uint8_t) * static_cast<size_t>(g.max_batch) * MB_MAX_WINDOW * g.block);
+  A_(c->mb.fwd_ids, sizeof(int) * static_cast<size_t>(g.max_batch) * MB_MAX_WINDOW * g.block);
   A_(c->gen.fwd_ids, sizeof(int) * 2 * static_cast<size_t>(g.max_batch) * g.block);
   A_(c->gen.counters, sizeof(long long) * 8);
   if (cudaMallocHost(reinterpret_cast<void**>(&c->host_counters), sizeof(long long) * 8) != cudaSuccess)
@@ -1224,6 +1234,61 @@ extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t 
     host_stats->kernel_launches = c->launches - launches0;
   }
   if (c->host_counters[4] > 0) return fail(c, D3_ERR_STATE, "generate loop did not finish within its step bound");
+  return check_device_error(c);
+}
+
+extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshold, int32_t bs, int32_t max_active,
+                                      int32_t* out_ids, int32_t* commit_round, d3_stats* host_stats) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!out_ids || bs <= 0 || gen_len <= 0 || std::isnan(threshold) || max_active < 1 || max_active > MB_MAX_WINDOW)
+    return fail(c, D3_ERR_INVALID_ARG, "bad generate_multiblock arguments");
+  if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_generate_multiblock before d3_prefill");
+  const int B = c->cfg.block;
+  if (bs > c->cfg.max_batch || gen_len % B != 0) return fail(c, D3_ERR_SHAPE, "bs > max_batch or gen_len not a multiple of the block size");
+  if (static_cast<long long>(bs) * max_active * B > std::min<long long>(c->stat_rows, c->max_rows))
+    return fail(c, D3_ERR_SHAPE, "bs * max_active * block rows exceed the workspaces (raise max_batch at d3_create)");
+  {
+    std::vector<int> pl(bs);
+    CUDA_TRY(c, cudaMemcpyAsync(pl.data(), c->prefix_len, sizeof(int) * bs, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    for (int b = 0; b < bs; ++b)
+      if (pl[b] + gen_len > c->cfg.max_seq) return fail(c, D3_ERR_SHAPE, "prefix + gen_len exceeds max_seq");
+  }
+  const int n_blocks = gen_len / B;
+  const int W = MB_MAX_WINDOW;
+  const int64_t launches0 = c->launches;
+  MbState g = c->mb;
+  g.counters = c->gen.counters;
+  g.out_ids = out_ids;
+  g.commit_round = commit_round;
+  mb_init_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, W, c->cfg.mask_id, gen_len);
+  LAUNCHED(c, "mb_init_kernel");
+  const long long max_iter = static_cast<long long>(n_blocks) * (B + 1) + 1;
+  long long rounds = 0;
+  int R = B;
+  for (long long it = 0; it < max_iter; ++it) {
+    mb_rowmap_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, W, R, c->cfg.mask_id, c->pos_base, c->n_valid, c->kv_len);
+    LAUNCHED(c, "mb_rowmap_kernel");
+    TRY(forward(c, g.fwd_ids, bs, R, 1, nullptr, B));
+    ++rounds;
+    mb_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, W, R, n_blocks, gen_len, threshold,
+                                                c->cfg.decide_mode, c->cfg.mask_id, max_active, static_cast<int>(rounds));
+    LAUNCHED(c, "mb_advance_kernel");
+    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 7, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+    if (c->host_counters[4] <= 0) break;
+    R = static_cast<int>(std::max<long long>(1, c->host_counters[5])) * B;
+  }
+  if (host_stats) {
+    std::memset(host_stats, 0, sizeof(*host_stats));
+    host_stats->denoise_forwards = c->host_counters[0];
+    host_stats->finalize_forwards = c->host_counters[1];
+    host_stats->tokens_committed = c->host_counters[2];
+    host_stats->forced_commits = c->host_counters[3];
+    host_stats->steps = rounds;
+    host_stats->kernel_launches = c->launches - launches0;
+  }
+  if (c->host_counters[4] > 0) return fail(c, D3_ERR_STATE, "multi-block loop did not finish within its round bound");
   return check_device_error(c);
 }
 

@@ -261,7 +261,7 @@ struct UnmaskOut {
 };
 __device__ __forceinline__ UnmaskOut unmask_block(const float* conf, const float* ent, const int* argmax, int* ids,
                                                   uint8_t* mask, int B, float tau, int mode, int* out_pos,
-                                                  int* out_ids, int* commit_step, int step) {
+                                                  int* out_ids, int* commit_step, int step, bool force = true) {
   const int lane = threadIdx.x & 31;
   // pass 1: best masked position
   float best = -INFINITY;
@@ -291,8 +291,8 @@ __device__ __forceinline__ UnmaskOut unmask_block(const float* conf, const float
     const int r = r0 + lane;
     bool masked = (r < B) && mask[r];
     bool clears = masked && ((mode == 0) ? (conf[r] > tau) : (ent[r] < tau));
-    bool commit = clears || (masked && r == best_r);
-    if (masked && r == best_r && !clears) res.forced = 1;
+    bool commit = clears || (force && masked && r == best_r);  // without `force`: only what clears the threshold
+    if (force && masked && r == best_r && !clears) res.forced = 1;
     unsigned bal = __ballot_sync(0xffffffffu, commit);
     if (commit) {
       int slot = base + __popc(bal & ((1u << lane) - 1u));
@@ -482,6 +482,152 @@ __global__ void gen_init_kernel(GenState g, int bs, int B, int mask_id, int gen_
       g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = g.counters[5] = g.counters[6] = 0;
       g.counters[4] = bs;
     }
+  }
+}
+
+// ----------------------------------------------------------------------------- multi-block decoding
+// Several consecutive blocks of a sequence are in flight at once (Sec. 3.2, multi-block decoding): a
+// window of up to `max_active` blocks starting at the first block that is not in the cache yet.  One
+// round = one forward over the windows' rows (segment-limited attention: a block sees the cache,
+// the earlier blocks of the window and itself) + this bookkeeping.
+struct MbState {
+  int* lo;          // [bs] first block in flight
+  int* n_win;       // [bs] blocks in flight (0: the sequence is done)
+  int* prefix_len;  // [bs]
+  int* ids;         // [bs, W * B] the window's blocks, oldest first
+  uint8_t* mask;    // [bs, W * B]
+  int* fwd_ids;     // [bs, R] ids of the next forward
+  int* out_ids;     // [bs, gen_len]
+  int* commit_round;  // [bs, gen_len] or null
+  long long* counters;  // [0] block decisions taken, [1] blocks stored in the cache, [2] tokens, [3] forced commits,
+                        // [4] sequences not done, [5] largest window of the next round, [6] rows of valid work so far
+};
+constexpr int MB_MAX_WINDOW = 8;
+
+__global__ void mb_init_kernel(MbState g, int bs, int B, int W, int mask_id, int gen_len) {
+  const int b = blockIdx.x;
+  for (int r = threadIdx.x; r < W * B; r += blockDim.x) {
+    g.ids[b * W * B + r] = mask_id;
+    g.mask[b * W * B + r] = 1;
+  }
+  for (int r = threadIdx.x; r < gen_len; r += blockDim.x) g.out_ids[static_cast<size_t>(b) * gen_len + r] = mask_id;
+  if (threadIdx.x == 0) {
+    g.lo[b] = 0;
+    g.n_win[b] = 1;
+    if (b == 0) {
+      for (int i = 0; i < 8; ++i) g.counters[i] = 0;
+      g.counters[4] = bs;
+      g.counters[5] = 1;
+    }
+  }
+}
+
+// Row map and input ids of the next round (rows_per_seq = R >= the largest window).  One block per sequence.
+__global__ void mb_rowmap_kernel(MbState g, int bs, int B, int W, int R, int mask_id, int* pos_base, int* n_valid, int* kv_len) {
+  const int b = blockIdx.x;
+  const int rows = g.n_win[b] * B;
+  if (threadIdx.x == 0) {
+    pos_base[b] = g.prefix_len[b];
+    n_valid[b] = rows;
+    kv_len[b] = rows > 0 ? g.prefix_len[b] + rows : 0;
+    if (b == 0) g.counters[5] = 0;  // the next round's largest window is gathered by mb_advance_kernel
+  }
+  for (int r = threadIdx.x; r < R; r += blockDim.x) g.fwd_ids[b * R + r] = r < rows ? g.ids[b * W * B + r] : mask_id;
+}
+
+// After the forward of a round.  States are read from the masks as they stood before the forward:
+// a block without masks has just had its stabilizing forward; a block whose predecessor in the
+// window is at least 95 % unmasked (or that is the oldest) is Fully-Activated and commits at least
+// one token; the others are Activated and commit only what clears the threshold.  Then the leading
+// complete blocks enter the cache, and a new block is opened once the newest one is 10 % unmasked.
+// One warp per sequence.
+__global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, const float* __restrict__ ent,
+                                  const int* __restrict__ argmax, int bs, int B, int W, int R, int n_blocks, int gen_len,
+                                  float tau, int decide_mode, int mask_id, int max_active, int round) {
+  const int b = blockIdx.x;
+  const int lane = threadIdx.x & 31;
+  int n = g.n_win[b];
+  if (n == 0) return;
+  int* ids = g.ids + b * W * B;
+  uint8_t* mask = g.mask + b * W * B;
+  const int lo = g.lo[b];
+  int unmasked[MB_MAX_WINDOW];
+#pragma unroll
+  for (int w = 0; w < MB_MAX_WINDOW; ++w) {
+    unmasked[w] = 0;
+    if (w < n) {
+      int cnt = 0;
+      for (int r0 = 0; r0 < B; r0 += 32) {
+        const int r = r0 + lane;
+        cnt += __popc(__ballot_sync(0xffffffffu, r < B && mask[w * B + r] == 0));
+      }
+      unmasked[w] = cnt;
+    }
+  }
+  long long committed = 0, forced = 0, decisions = 0;
+#pragma unroll
+  for (int w = 0; w < MB_MAX_WINDOW; ++w) {
+    if (w < n && unmasked[w] < B) {
+      const bool fully = w == 0 || 100 * unmasked[w - 1] >= 95 * B;
+      const int row0 = b * R + w * B;
+      int* cr = g.commit_round ? g.commit_round + static_cast<size_t>(b) * gen_len + (lo + w) * B : nullptr;
+      UnmaskOut r = unmask_block(conf + row0, ent + row0, argmax + row0, ids + w * B, mask + w * B, B, tau, decide_mode,
+                                 nullptr, nullptr, cr, round, fully);
+      committed += r.committed;
+      forced += r.forced;
+      decisions += 1;
+    }
+  }
+  __syncwarp();
+  // leading blocks that were complete before this forward: out and into the cache
+  int k = 0;
+  while (k < n && unmasked[k] == B) ++k;
+  for (int q = 0; q < k; ++q)
+    for (int r = lane; r < B; r += 32) g.out_ids[static_cast<size_t>(b) * gen_len + (lo + q) * B + r] = ids[q * B + r];
+  if (k > 0) {
+    const int left = (n - k) * B;
+    for (int r0 = 0; r0 < left; r0 += 32) {  // move the rest of the window down: read, then write
+      const int r = r0 + lane;
+      int v = 0;
+      uint8_t m = 0;
+      if (r < left) { v = ids[k * B + r]; m = mask[k * B + r]; }
+      __syncwarp();
+      if (r < left) { ids[r] = v; mask[r] = m; }
+      __syncwarp();
+    }
+    n -= k;
+  }
+  // a new block once the newest one in flight is 10 % unmasked, or when nothing is in flight
+  const int nxt = lo + k + n;
+  if (nxt < n_blocks && n < max_active) {
+    bool open = n == 0;
+    if (!open) {
+      int cnt = 0;
+      for (int r0 = 0; r0 < B; r0 += 32) {
+        const int r = r0 + lane;
+        cnt += __popc(__ballot_sync(0xffffffffu, r < B && mask[(n - 1) * B + r] == 0));
+      }
+      open = 100 * cnt >= 10 * B;
+    }
+    if (open) {
+      for (int r = lane; r < B; r += 32) {
+        ids[n * B + r] = mask_id;
+        mask[n * B + r] = 1;
+      }
+      ++n;
+    }
+  }
+  __syncwarp();
+  if (lane == 0) {
+    g.lo[b] = lo + k;
+    g.n_win[b] = n;
+    g.prefix_len[b] += k * B;
+    atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[0]), static_cast<unsigned long long>(decisions));
+    atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[1]), static_cast<unsigned long long>(k));
+    atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[2]), static_cast<unsigned long long>(committed));
+    atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[3]), static_cast<unsigned long long>(forced));
+    if (n == 0) atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[4]), static_cast<unsigned long long>(-1ll));
+    atomicMax(reinterpret_cast<unsigned long long*>(&g.counters[5]), static_cast<unsigned long long>(n));
   }
 }
 

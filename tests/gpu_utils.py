@@ -71,6 +71,12 @@ class Ctx:
         st = d3.d3_generate(self.ctx, gen_len, tau, out, cs)
         return out.cpu().numpy(), cs.cpu().numpy(), st
 
+    def generate_multiblock(self, bs: int, gen_len: int, tau: float, max_active: int):
+        out = torch.full((bs, gen_len), -1, dtype=torch.int32, device=DEV)
+        cr = torch.zeros((bs, gen_len), dtype=torch.int32, device=DEV)
+        st = d3.d3_generate_multiblock(self.ctx, gen_len, tau, out, max_active, cr)
+        return out.cpu().numpy(), cr.cpu().numpy(), st
+
     def set_prefix(self, lens):
         d3.d3_set_state(self.ctx, torch.tensor(lens, dtype=torch.int32, device=DEV))
 

@@ -282,6 +282,68 @@ def test_generate_stops_on_eos_at_batch_one_with_fused_finalize(c1):
     assert d3.d3_early_stops(ctx.ctx) == int(ref["stopped_early"])
 
 
+@pytest.mark.parametrize("tau,mode", [(0.3, 0), (0.9, 0), (2.42, 1)])
+def test_multiblock_decoding_fp32_equals_the_oracle(tau, mode):
+    """Multi-block decoding (Sec. 3.2) on the fp32 path, three ragged sequences, 1, 2 and 4 blocks in
+    flight: tokens, the round of every commit, rounds, decisions and cached blocks equal the oracle's."""
+    shape = si.TINY
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("mb", shape, 3, [32, 9, 21], 64, 16, tau, 77)
+    model = o.model_from_shape(shape, W, np.float64)
+    # max_batch sizes the workspaces: 3 sequences x 4 blocks x 16 rows
+    with Ctx(shape, W, block=16, max_batch=12, max_seq=wl.max_seq, decide_mode=mode) as ctx:
+        for max_active in (1, 2, 4):
+            ref = [model.generate_multiblock(ids[b, :lens[b]], 64, 16, tau, mode, max_active=max_active, record=True)
+                   for b in range(3)]
+            ctx.prefill(ids, lens)
+            tok, cr, st = ctx.generate_multiblock(3, 64, tau, max_active)
+            for b in range(3):
+                assert np.array_equal(tok[b], ref[b]["tokens"]), (max_active, b)
+                assert np.array_equal(cr[b], ref[b]["commit_round"]), (max_active, b)
+            assert st.steps == max(r["rounds"] for r in ref)
+            assert st.tokens_committed == 3 * 64
+            assert st.finalize_forwards == 3 * 4
+            decisions = sum(sum(1 for k in range(t["n_win"]) if t["mask_in"][k].any()) for r in ref for t in r["trace"])
+            assert st.denoise_forwards == decisions
+            assert np.array_equal(ctx.get_prefix(3), lens + 64)
+            assert ctx.error_word() == 0
+        # one block in flight = block-by-block decoding
+        ctx.prefill(ids, lens)
+        tok1, _, _ = ctx.generate_multiblock(3, 64, tau, 1)
+        d3.d3_set_matmul_tuning(ctx.ctx, 0, 0x100)
+        ctx.prefill(ids, lens)
+        tok0, _, _ = ctx.generate(3, 64, tau)
+        d3.d3_set_matmul_tuning(ctx.ctx, 0, 0)
+        assert np.array_equal(tok1, tok0)
+        # too many rows for the workspaces, bad window
+        with pytest.raises(d3.D3Error):
+            ctx.generate_multiblock(4, 64, tau, 8)
+        with pytest.raises(d3.D3Error):
+            ctx.generate_multiblock(1, 64, tau, 0)
+
+
+def test_multiblock_decoding_bf16_tensor_core():
+    """The same through the tensor-core kernels at batch 1 (forwards of 32 to 128 rows, up to four
+    segments): against the oracle with mirrored bf16 roundings; ids may differ only where the oracle
+    sees a near-tie (|confidence - threshold| < 1e-3)."""
+    shape = small_bf16(128, 4, 2, "mb-bf16")
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("mb-bf16", shape, 1, [37], 128, 32, 0.9, 29)
+    model = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
+    with Ctx(shape, W, block=32, max_batch=4, max_seq=wl.max_seq) as ctx:
+        for max_active in (2, 4):
+            ref = model.generate_multiblock(ids[0, :lens[0]], 128, 32, 0.9, 0, max_active=max_active, record=True)
+            ctx.prefill(ids, lens)
+            tok, cr, st = ctx.generate_multiblock(1, 128, 0.9, max_active)
+            assert st.tokens_committed == 128 and ctx.error_word() == 0
+            near_tie = any(bool(np.any(np.abs(t["stats"][k][0][t["mask_in"][k]] - 0.9) < 1e-3))
+                           for t in ref["trace"] for k in range(t["n_win"]))
+            same = np.array_equal(tok[0], ref["tokens"]) and np.array_equal(cr[0], ref["commit_round"])
+            print("multi-block bf16, max_active", max_active, "equal to oracle:", same, "near-tie:", near_tie,
+                  "rounds", st.steps, ref["rounds"])
+            assert same or near_tie
+
+
 def test_c1_entropy_mode():
     w = si.WORKLOADS["c1"]
     W = si.gen_weights(w.model)
