@@ -44,6 +44,10 @@ def gemm_source_hash() -> str:
     return h.hexdigest()[:16]
 
 
+def tokens_of(w) -> int:
+    return w.batch * w.gen_len
+
+
 METRIC = "decoded tokens/s"
 UNIT = "tokens/s"
 
@@ -310,6 +314,19 @@ def run_ours(args):
     clock_info = clocks.stop()
     ms_e2e, _ = timed(step_e2e, args.steps)
 
+    # the paper's multi-block decoding (two blocks in flight) on the same request, beside the headline
+    # number, where the workspaces sized by the workload's batch hold two blocks per sequence
+    multiblock = None
+    if 2 * w.batch * w.block <= 64:
+        def step_multiblock():
+            d3.d3_prefill(ctx, ids_dev, lens_dev)
+            return d3.d3_generate_multiblock(ctx, w.gen_len, w.threshold, out_dev, 2)
+        step_multiblock()
+        ms_mb, st_mb = timed(step_multiblock, args.steps)
+        multiblock = {"max_active": 2, "value": whole_job_tokens_per_s(world, tokens_of(w), args.steps, ms_mb), "unit": UNIT,
+                      "rounds_per_request": int(st_mb.steps), "tokens_per_round": tokens_of(w) / max(int(st_mb.steps), 1),
+                      "ms_per_round": ms_mb / args.steps / max(int(st_mb.steps), 1)}
+
     # per-class kernel times of the decode loop (one request, events around every launch)
     d3.d3_prefill(ctx, ids_dev, lens_dev)
     torch.cuda.synchronize()
@@ -382,7 +399,7 @@ def run_ours(args):
                    "tokens_per_forward_incl_finalize": tokens / max(st.denoise_forwards + st.finalize_forwards, 1),
                    "ms_per_forward": (ms_step - ms_prefill) / max(forwards, 1), "prefill_ms": ms_prefill,
                    "forced_commits": int(st.forced_commits)},
-        "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
+        "multiblock": multiblock, "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
         "device_bytes": d3.d3_device_bytes(ctx),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
