@@ -145,7 +145,11 @@ int d3_commit_block(d3_ctx *ctx, const int32_t *block_ids, int32_t bs);
  * while others still denoise).  out_ids [device][bs, gen_len]; commit_step (may be NULL)
  * [device][bs, gen_len]: 1-based step within its block at which each position was committed;
  * host_stats [host] may be NULL.  Waits for the stream.  Errors: SHAPE when gen_len is not a
- * multiple of B or prefix + gen_len > max_seq. */
+ * multiple of B or prefix + gen_len > max_seq.
+ * While 2 * bs * B <= 64 rows (and the context was created with 2 * max_batch * B <= 64), the finalize
+ * forward of a block and the first denoise step of the next block run as one forward of 2B rows per
+ * sequence, the finished block unable to see the new one: same results as separate forwards (bit for
+ * bit on the fp32 path), one batched forward less per block. */
 int d3_generate(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32_t *out_ids,
                 int32_t *commit_step, d3_stats *host_stats);
 
@@ -278,7 +282,9 @@ int d3_set_overlap(d3_ctx *ctx, int on);
  * scheduling variants for sweeps and tests: 16-19 producer warps, 20-21 tile width + 1, 22-24 divisor
  * of the attention key splits, 25 no cluster K-split, 26-27 row-tile pairs + 1, 28 no round-robin
  * tiles, 29-30 column strips for skinny matmuls (0 when they pay, 1 never, 2 with one CTA per SM,
- * 3 wherever the shape allows).  Results do not change beyond the order of fp32 partial sums. */
+ * 3 wherever the shape allows).  Bit 8 of ctas_per_sm: d3_generate finalizes every block in a forward of
+ * its own instead of fusing that forward with the next block's first step (see d3_generate).  Results
+ * do not change beyond the order of fp32 partial sums. */
 int d3_set_matmul_tuning(d3_ctx *ctx, int32_t ring_kb, int32_t ctas_per_sm);
 
 /* Per-class kernel timing for measurement runs.  While enabled, every launch of the forward pass is
