@@ -422,7 +422,9 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
     const int n_res = std::max(1, std::min(slots / C, T));
     const long long cost_res = static_cast<long long>((T + n_res - 1) / n_res) * slabs * 16;
     const long long waves = (static_cast<long long>(T) * C + slots - 1) / slots;
-    const long long cost_waves = slabs * (4 + 3 * (waves - 1)) * 4;  // slabs * (1 + 0.75 (waves - 1)) * 16
+    // (with 128-row tiles the 200 KB of shared memory really leave one CTA per SM: whole waves)
+    const long long cost_waves = a_rows <= 64 ? slabs * (4 + 3 * (waves - 1)) * 4  // slabs * (1 + 0.75 (waves - 1)) * 16
+                                              : slabs * waves * 16;
     const bool by_waves = cost_waves < cost_res;
     const long long cost = (by_waves ? cost_waves : cost_res) + C;  // ties: smaller clusters
     if (best < 0 || cost < best) {
@@ -478,9 +480,10 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
 // narrowest strip (a multiple of 16 columns that divides N) whose CTAs are all resident at once.
 // Returns 0 when no strip width qualifies.
 int strip_width(const d3_ctx* c, int M, int N, int w_tiled) {
-  if (!w_tiled || M > 64 || c->tune_strip == 1) return 0;
+  if (!w_tiled || M > 128 || c->tune_strip == 1) return 0;
   const int a_rows = ((M + 31) / 32) * 32;
-  const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : (c->tune_strip == 2 ? 1 : 2);
+  // above 64 rows a stage is 24-48 KB: one CTA per SM with all of shared memory as its ring
+  const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : ((c->tune_strip == 2 || a_rows > 64) ? 1 : 2);
   const int slots = c->n_sms * per_sm;
   if (c->tune_strip == 3) {  // tests: the narrowest strip the shape allows, whatever it costs
     for (int S = 16; S <= 256; S += 16)
@@ -520,7 +523,7 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   p.a_rows = a_rows;
   p.m_tiles = 1; p.n_tiles = N / S; p.k_chunks = KC;
   p.total_units = static_cast<long long>(p.n_tiles) * KC;
-  const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : (c->tune_strip == 2 ? 1 : 2);
+  const int per_sm = c->tune_ctas_per_sm > 0 ? c->tune_ctas_per_sm : ((c->tune_strip == 2 || a_rows > 64) ? 1 : 2);
   const size_t ring = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 200 / per_sm) * 1024;
   const size_t stage_bytes = static_cast<size_t>(a_rows + S) * 128;
   p.stages = std::max(2, std::min<int>(std::min<int>(static_cast<int>(ring / stage_bytes), KC), 32));
@@ -568,14 +571,14 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
     const bool elementwise = epi == EPI_F32 || epi == EPI_T || epi == EPI_RESID;
     if (elementwise && ctas_hint >= 1 && ctas_hint <= 8) return run_linear_ck(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
     // few enough tiles that every tile gets a cluster of at least two resident CTAs.  By itself only
-    // up to 64 rows: with 128-row tiles (measured at 128 and 256 rows on the 7B/8B shapes) the best
-    // cluster size is only level with the unit-range kernel at 256 rows and the model below misjudges it.
-    if (elementwise && ctas_hint == 0 && M <= 64 && T * 2 <= c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 0, qx, w_tiled);
+    // up to 128 rows (one row tile): at 256 rows the best cluster size is only level with the
+    // unit-range kernel (measured on the 7B/8B shapes).
+    if (elementwise && ctas_hint == 0 && M <= 128 && T * 2 <= c->n_sms && KC >= 16) return run_linear_ck(c, X, W, M, N, K, epi, ep, 0, qx, w_tiled);
   }
   if (ctas_hint < 0) {  // a strip width asked for by name
     const int S = -ctas_hint;
-    if (!w_tiled || M > 64 || epi == EPI_STATS || S % 16 != 0 || S > 256 || N % S != 0)
-      return fail(c, D3_ERR_UNSUPPORTED, "column strips need tiled weights, at most 64 rows and a width that is a multiple of 16, at most 256, and divides n");
+    if (!w_tiled || M > 128 || epi == EPI_STATS || S % 16 != 0 || S > 256 || N % S != 0)
+      return fail(c, D3_ERR_UNSUPPORTED, "column strips need tiled weights, at most 128 rows and a width that is a multiple of 16, at most 256, and divides n");
     return run_linear_strip(c, X, W, M, N, K, epi, ep, S, qx);
   }
   if (ctas_hint == 0 && epi != EPI_STATS) {
@@ -900,6 +903,9 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   // d3_generate may run the finalize forward of a block together with the first step of the next one
   // (2 * block rows per sequence) while that still is a skinny forward: room for it
   if (2 * dec_rows <= FUSE_MAX_ROWS) dec_rows *= 2;
+  // and for a few blocks in flight per sequence (d3_generate_multiblock) while the forward stays
+  // on the skinny kernels (128 rows)
+  dec_rows = std::max<long long>(dec_rows, 128);
   c->max_rows = static_cast<int>(std::max(pre_rows, dec_rows));
   const size_t R = c->max_rows;
 #define A_(ptr, bytes)                                                         \

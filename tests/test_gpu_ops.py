@@ -103,7 +103,8 @@ def test_linear_bf16_packed_weights(ctx_bf16, m, n, k, splits):
 
 
 @pytest.mark.parametrize("m,n,k,widths", [(32, 2400, 256, [16, 48, 80, 96, 240]), (64, 2400, 200, [48, 160]),
-                                          (7, 4736, 1024, [32, 128]), (1, 512, 4096, [16, 256])])
+                                          (7, 4736, 1024, [32, 128]), (1, 512, 4096, [16, 256]),
+                                          (100, 2400, 256, [48, 240]), (128, 4736, 512, [128, 64])])
 def test_linear_bf16_column_strips(ctx_bf16, m, n, k, widths):
     """The column-strip kernel (one CTA per strip of S columns, whole K range) against the fp64 product:
     strips that start and end inside the 128-row weight blocks, span three blocks, end in half a
