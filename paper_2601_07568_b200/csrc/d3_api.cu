@@ -364,7 +364,7 @@ int run_linear_tc_bn(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   return dispatch_tc<BLOCK_N, MT>(c, epi, tx, tw, p, static_cast<int>(n_ctas), smem);
 }
 
-// Skinny matmuls (up to 64 rows): clusters of C CTAs own whole 128-column tiles and split K among
+// Skinny matmuls (up to 128 rows by default, 256 on request): clusters of C CTAs own whole 128-column tiles and split K among
 // their CTAs; the partial sums meet in distributed shared memory (gemm_ck_kernel).  C and the number
 // of clusters are chosen so that the longest CTA has the fewest (tile, K slab) units.
 template <int EPI>
