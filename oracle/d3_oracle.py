@@ -43,6 +43,18 @@ What the paper fixes (cited per function) and what it leaves open
   step that commits the EOS id anywhere in the current block; positions that
   are still masked (in this block and all later ones) are returned as the
   mask id, and the unfinished block gets no finalize forward.
+* KV-refresh (Sec. 3.2, "KV-Cache and KV-Refresh Mechanism"; abstract: all
+  previously cached states are recomputed periodically) and the cache delay
+  (Appendix, inference settings: 1-2 iterations).  Readings taken here: a
+  refresh is one forward over the tokens of the stored prefix (prompt and
+  stored blocks) in which every position sees every other one, and it
+  replaces the stored K and V; blocks in flight take no part and the next
+  forwards read the refreshed cache.  Block-by-block decoding refreshes each
+  time the number of stored blocks reaches a multiple of the period while
+  blocks remain; multi-block decoding refreshes after every period-th round
+  while blocks are in flight.  The cache delay is the number of stabilizing
+  rounds (forwards in which the block was already complete) before a block's
+  K and V are stored.
 
 Readings taken where the paper is silent are listed in the repository's
 design notes; in short: block-causal visibility between segments (prompt =
@@ -180,16 +192,18 @@ def decide(conf: np.ndarray, ent: np.ndarray, mask: np.ndarray, tau: float, mode
 # ----------------------------------------------------------------------------- model
 @dataclass
 class SeqState:
-    """Per-sequence cache: post-RoPE K and V of the committed prefix, per layer [L, hkv, dh]."""
+    """Per-sequence cache: post-RoPE K and V of the committed prefix, per layer [L, hkv, dh],
+    and the token ids of that prefix (needed to recompute the cache, see ``refresh``)."""
     k: List[np.ndarray]
     v: List[np.ndarray]
+    ids: np.ndarray = field(default_factory=lambda: np.zeros(0, dtype=np.int32))
 
     @property
     def prefix_len(self) -> int:
         return int(self.k[0].shape[0])
 
     def copy(self) -> "SeqState":
-        return SeqState([a.copy() for a in self.k], [a.copy() for a in self.v])
+        return SeqState([a.copy() for a in self.k], [a.copy() for a in self.v], self.ids.copy())
 
 
 class OracleModel:
@@ -296,7 +310,14 @@ class OracleModel:
         if prompt.shape[0] == 0:
             return self.empty_state()
         _, ks, vs = self.forward_rows(prompt, np.arange(prompt.shape[0]), None)
-        return SeqState(ks, vs)
+        return SeqState(ks, vs, prompt.astype(np.int32))
+
+    def refresh(self, state: SeqState) -> SeqState:
+        """KV-refresh (Sec. 3.2, KV-cache and KV-refresh mechanism): all previously cached
+        states are recomputed by a full forward pass.  Reading taken here: one forward over
+        the tokens of the whole stored prefix (prompt and stored blocks), every position
+        seeing every other one, replaces the stored K and V; blocks in flight take no part."""
+        return self.prefill(state.ids)
 
     def denoise_forward(self, state: SeqState, block_ids: np.ndarray):
         """One forward of the block's rows (masked rows hold mask_id) against the prefix cache.
@@ -325,19 +346,23 @@ class OracleModel:
         pos = state.prefix_len + np.arange(B)
         _, ks, vs = self.forward_rows(np.asarray(block_ids), pos, state)
         return SeqState([np.concatenate([a, b], axis=0) for a, b in zip(state.k, ks)],
-                        [np.concatenate([a, b], axis=0) for a, b in zip(state.v, vs)])
+                        [np.concatenate([a, b], axis=0) for a, b in zip(state.v, vs)],
+                        np.concatenate([state.ids, np.asarray(block_ids, dtype=np.int32)]))
 
     def generate(self, prompt: np.ndarray, gen_len: int, block: int, tau: float,
                  mode: int = MODE_CONFIDENCE, record: bool = False,
-                 eos_id: Optional[int] = None) -> Dict[str, object]:
+                 eos_id: Optional[int] = None, refresh_every: int = 0) -> Dict[str, object]:
         """Block-by-block threshold decoding of one sequence.
 
         Returns tokens [gen_len], the step index (within its block, from 1) at which each
         position was committed, forward counts, and optionally a per-step trace.  With
         ``eos_id`` decoding halts after the step that commits that id (Sec. 3.2, early
-        stopping on EOS); undecoded positions stay ``mask_id``."""
+        stopping on EOS); undecoded positions stay ``mask_id``.  With ``refresh_every`` = r > 0
+        the cache is refreshed (``refresh``) each time the number of stored blocks reaches a
+        multiple of r while blocks remain to be decoded (periodic KV-refresh, Sec. 3.2)."""
         assert gen_len % block == 0
         state = self.prefill(prompt)
+        n_refresh = 0
         out = np.full(gen_len, self.mask_id, dtype=np.int32)
         commit_step = np.zeros(gen_len, dtype=np.int32)
         n_denoise = n_finalize = 0
@@ -367,8 +392,11 @@ class OracleModel:
             state = self.finalize_block(state, ids)
             n_finalize += 1
             out[j * block:(j + 1) * block] = ids
+            if refresh_every > 0 and (j + 1) % refresh_every == 0 and j + 1 < gen_len // block:
+                state = self.refresh(state)
+                n_refresh += 1
         res = dict(tokens=out, commit_step=commit_step, n_denoise=n_denoise, n_finalize=n_finalize,
-                   stopped_early=stopped,
+                   stopped_early=stopped, n_refresh=n_refresh,
                    tpf_denoise=gen_len / max(n_denoise, 1),
                    tpf_all=gen_len / max(n_denoise + n_finalize, 1), state=state)
         if record:
@@ -376,15 +404,18 @@ class OracleModel:
         return res
 
     def generate_multiblock(self, prompt: np.ndarray, gen_len: int, block: int, tau: float,
-                            mode: int = MODE_ENTROPY, max_active: int = 2, record: bool = False
-                            ) -> Dict[str, object]:
+                            mode: int = MODE_ENTROPY, max_active: int = 2, record: bool = False,
+                            cache_delay: int = 1, refresh_every: int = 0) -> Dict[str, object]:
         """Multi-block decoding of one sequence (Sec. 3.2, multi-block decoding strategy).
 
         Every round is one forward over the blocks in flight (oldest first), each seeing the
         cache, the earlier blocks in flight as they stand (masked rows included) and itself.
         Returns tokens [gen_len], the round (from 1) in which each position was committed, the
-        number of rounds, the rows each round covered, and optionally a per-round trace."""
-        assert gen_len % block == 0 and max_active >= 1
+        number of rounds, the rows each round covered, and optionally a per-round trace.
+        ``cache_delay``: stabilizing rounds a complete block goes through before its K/V are
+        stored (1 or 2 in the paper's settings).  ``refresh_every`` = r > 0: after every r-th
+        round the stored cache is refreshed (``refresh``) while blocks are still in flight."""
+        assert gen_len % block == 0 and max_active >= 1 and cache_delay >= 1
         n_blocks = gen_len // block
         state = self.prefill(prompt)
         out = np.full(gen_len, self.mask_id, dtype=np.int32)
@@ -392,12 +423,14 @@ class OracleModel:
         lo = 0                                   # first block in flight
         win_ids: List[np.ndarray] = [np.full(block, self.mask_id, dtype=np.int32)]
         win_mask: List[np.ndarray] = [np.ones(block, dtype=bool)]
+        win_stab: List[int] = [0]                # stabilizing forwards each block in flight has had
         rounds = 0
+        n_refresh = 0
         rows: List[int] = []
         trace: List[Dict[str, object]] = []
         while win_ids:
             rounds += 1
-            assert rounds <= n_blocks * (block + 1) + 1, "every round must make progress"
+            assert rounds <= n_blocks * (block + cache_delay) + 1, "every round must make progress"
             n_win = len(win_ids)
             rows.append(n_win * block)
             # states as the masks stand before the forward
@@ -434,12 +467,15 @@ class OracleModel:
                 trace.append(dict(round=rounds, lo=lo, n_win=n_win, fully=list(fully), ids_in=ids_in, mask_in=mask_in,
                                   complete_before=list(complete_before), stats=stats, commits=commits,
                                   ids_out=[a.copy() for a in win_ids], mask_out=[a.copy() for a in win_mask]))
-            # blocks that were complete before this forward have had their stabilizing round: the
-            # oldest ones enter the cache, in order
-            while win_ids and complete_before[0]:
+            # blocks that were complete before this forward have had a stabilizing round: the
+            # oldest ones enter the cache, in order, once they have had cache_delay of them
+            for w in range(n_win):
+                if complete_before[w]:
+                    win_stab[w] += 1
+            while win_ids and win_stab[0] >= cache_delay:
                 state = self.finalize_block(state, win_ids[0])
                 out[lo * block:(lo + 1) * block] = win_ids[0]
-                win_ids.pop(0); win_mask.pop(0); complete_before.pop(0)
+                win_ids.pop(0); win_mask.pop(0); win_stab.pop(0)
                 lo += 1
             # a new block: when the newest one is 10 % complete (or nothing is in flight)
             nxt = lo + len(win_ids)
@@ -447,7 +483,12 @@ class OracleModel:
                 if not win_ids or 100 * int(block - win_mask[-1].sum()) >= 10 * block:
                     win_ids.append(np.full(block, self.mask_id, dtype=np.int32))
                     win_mask.append(np.ones(block, dtype=bool))
+                    win_stab.append(0)
+            if refresh_every > 0 and rounds % refresh_every == 0 and win_ids and state.prefix_len > 0:
+                state = self.refresh(state)
+                n_refresh += 1
         res = dict(tokens=out, commit_round=commit_round, rounds=rounds, rows=rows, state=state,
+                   n_refresh=n_refresh,
                    tokens_per_round=gen_len / max(rounds, 1))
         if record:
             res["trace"] = trace
