@@ -263,8 +263,9 @@ def run_ours(args):
     t0 = time.time()
     W = si.gen_weights(shape)
     t_gen = time.time() - t0
+    # workspace rows: the prompt forward, and the KV-refresh forward over prompt + generated blocks
     cfg = d3.make_config(shape, block=w.block, max_batch=w.batch, max_seq=w.max_seq,
-                         max_prefill_rows=w.batch * w.prompt_max)
+                         max_prefill_rows=w.batch * w.max_seq)
     ctx = d3.d3_create(cfg)
     d3.d3_load_weights(ctx, d3.weights_from_numpy(shape, W), shape.n_layers)
     del W
@@ -327,6 +328,23 @@ def run_ours(args):
         multiblock = {"max_active": mb_window, "value": whole_job_tokens_per_s(world, tokens_of(w), args.steps, ms_mb), "unit": UNIT,
                       "rounds_per_request": int(st_mb.steps), "tokens_per_round": tokens_of(w) / max(int(st_mb.steps), 1),
                       "ms_per_round": ms_mb / args.steps / max(int(st_mb.steps), 1)}
+
+    # KV-refresh: one forward over the whole stored prefix (prompt + generated blocks) of every sequence,
+    # timed alone after a request, and the request decoded with a refresh after every fourth block
+    ms_refresh, _ = timed(lambda: d3.d3_refresh_cache(ctx, w.batch), 3)
+    ms_refresh /= 3
+    refresh_rows = int(w.batch * (int(lens_np.max()) + w.gen_len))
+    d3.d3_set_cache_policy(ctx, 1, 4)
+    step_resident()
+    ms_rf, st_rf = timed(step_resident, args.steps)
+    n_refresh = d3.d3_refresh_count(ctx)
+    d3.d3_set_cache_policy(ctx, 1, 0)
+    kv_refresh = {"rows": refresh_rows, "ms": ms_refresh,
+                  # matmul flops of the layers (no LM head in a refresh forward; attention not counted)
+                  "tflops": shape.n_layers * sum(v for k, v in gemm_flops(shape, refresh_rows).items() if k != "gemm_head")
+                  / (ms_refresh * 1e-3) / 1e12,
+                  "decode_refresh_every_4_blocks": {"value": whole_job_tokens_per_s(world, tokens_of(w), args.steps, ms_rf), "unit": UNIT,
+                                                    "refreshes_per_request": int(n_refresh)}}
 
     # per-class kernel times of the decode loop (one request, events around every launch)
     d3.d3_prefill(ctx, ids_dev, lens_dev)
@@ -400,7 +418,7 @@ def run_ours(args):
                    "tokens_per_forward_incl_finalize": tokens / max(st.denoise_forwards + st.finalize_forwards, 1),
                    "ms_per_forward": (ms_step - ms_prefill) / max(forwards, 1), "prefill_ms": ms_prefill,
                    "forced_commits": int(st.forced_commits)},
-        "multiblock": multiblock, "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
+        "multiblock": multiblock, "kv_refresh": kv_refresh, "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
         "device_bytes": d3.d3_device_bytes(ctx),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

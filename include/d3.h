@@ -159,8 +159,8 @@ int d3_generate(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32
  * decisions.  A block is opened, fully masked, once the newest block in flight is 10 % unmasked; it
  * commits only what clears the threshold (config decide_mode: confidence > threshold, or entropy <
  * threshold) while its predecessor is less than 95 % unmasked, and at least one token per round
- * afterwards; a block without masks takes part in one more round before its K/V count as cached
- * (blocks enter the cache in order).  States are read from the masks as they stand before a round.
+ * afterwards; a block without masks takes part in one more round (cache_delay of them, see
+ * d3_set_cache_policy) before its K/V count as cached (blocks enter the cache in order).  States are read from the masks as they stand before a round.
  * max_active = 1 is block-by-block decoding with every finalize forward on its own.
  * out_ids [device][bs, gen_len]; commit_round (may be NULL) [device][bs, gen_len]: 1-based round in
  * which each position was committed.  host_stats (may be NULL): steps = rounds, denoise_forwards =
@@ -178,6 +178,26 @@ int d3_generate_multiblock(d3_ctx *ctx, int32_t gen_len, float threshold, int32_
  * equal to mask_id.  d3_early_stops: sequences of the latest d3_generate call that stopped this way. */
 int d3_set_eos(d3_ctx *ctx, int32_t eos_id);
 int64_t d3_early_stops(d3_ctx *ctx);
+
+/* KV-refresh (Sec. 3.2, "KV-Cache and KV-Refresh Mechanism": previously cached states are recomputed
+ * by full forward passes).  One forward over the tokens of the stored prefix of each of the bs
+ * sequences (the prompt and every block stored since, as recorded by d3_prefill, d3_commit_block and
+ * the generate loops), every position seeing the whole stored prefix; the K/V of positions
+ * [0, prefix) are overwritten in place, prefix lengths stay.  Needs bs * (longest stored prefix) rows
+ * of workspace (max_prefill_rows at d3_create), else SHAPE.  Waits for the stream once (prefix
+ * lengths are read on the host).  After d3_set_state has moved a prefix past what was recorded the
+ * recorded ids no longer describe the cache: the caller's business. */
+int d3_refresh_cache(d3_ctx *ctx, int32_t bs);
+
+/* Cache policy of the generate loops.  cache_delay (1..16, default 1; the paper's settings: 1-2):
+ * rounds of d3_generate_multiblock a complete block takes part in before its K/V count as stored.
+ * refresh_every (default 0 = never): d3_generate refreshes a sequence's cache each time the number of
+ * its stored blocks reaches a multiple of refresh_every while blocks remain to be decoded (the
+ * finalize forward is then never fused with the next block's first step); d3_generate_multiblock
+ * refreshes the sequences that are still decoding after every refresh_every-th round.
+ * d3_refresh_count: (sequence, refresh) pairs of the latest generate call. */
+int d3_set_cache_policy(d3_ctx *ctx, int32_t cache_delay, int32_t refresh_every);
+int64_t d3_refresh_count(d3_ctx *ctx);
 
 /* Statistics of the latest denoise forward: conf, entropy [device][bs*B] float, argmax
  * [device][bs*B] int32 (any may be NULL). */

@@ -27,7 +27,7 @@ EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
     "d3_get_state", "d3_set_state", "d3_op_linear", "d3_packed_weight_elems", "d3_pack_weight", "d3_op_linear_packed", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_generate_multiblock", "d3_device_bytes",
+    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_generate_multiblock", "d3_refresh_cache", "d3_set_cache_policy", "d3_refresh_count", "d3_device_bytes",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
 
@@ -79,6 +79,8 @@ def lib() -> C.CDLL:
         L.d3_launch_count_of.argtypes = [C.c_void_p, C.c_char_p]
         L.d3_early_stops.restype = C.c_int64
         L.d3_early_stops.argtypes = [C.c_void_p]
+        L.d3_refresh_count.restype = C.c_int64
+        L.d3_refresh_count.argtypes = [C.c_void_p]
         L.d3_device_bytes.restype = C.c_int64
         L.d3_device_bytes.argtypes = [C.c_void_p]
         L.d3_destroy.restype = None
@@ -354,6 +356,18 @@ def d3_set_eos(ctx, eos_id: int) -> None:
 
 def d3_early_stops(ctx) -> int:
     return int(lib().d3_early_stops(ctx))
+
+
+def d3_refresh_cache(ctx, bs: int) -> None:
+    _check(ctx, lib().d3_refresh_cache(ctx, C.c_int32(bs)))
+
+
+def d3_set_cache_policy(ctx, cache_delay: int = 1, refresh_every: int = 0) -> None:
+    _check(ctx, lib().d3_set_cache_policy(ctx, C.c_int32(cache_delay), C.c_int32(refresh_every)))
+
+
+def d3_refresh_count(ctx) -> int:
+    return int(lib().d3_refresh_count(ctx))
 
 
 def d3_device_bytes(ctx) -> int:

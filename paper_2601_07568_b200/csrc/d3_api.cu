@@ -91,6 +91,11 @@ struct d3_ctx {
   int tune_no_rr = 0;     // 1: wide matmuls on contiguous unit ranges
   int eos_id = -1;        // d3_generate stops a sequence once this id has been committed (< 0: never)
   long long last_early_stops = 0;
+  int* hist_ids = nullptr;     // [max_batch, max_seq] ids of the stored prefix of every sequence
+  int* refresh_ids = nullptr;  // [max_rows] input ids of a KV-refresh forward
+  int cache_delay = 1;         // multi-block decoding: stabilizing rounds before a complete block is stored
+  int refresh_every = 0;       // periodic KV-refresh in the generate loops (0: never)
+  long long last_refreshes = 0;
   bool gen_fuse = true;   // d3_generate fuses finalize forwards with the next block's first step while the forward stays skinny
   int tune_strip = 0;     // skinny matmuls as column strips: 0 when it pays, 1 never, 2 with one CTA per SM, 3 whenever possible
   int tune_no_cluster = 0;  // 1: skinny matmuls on the unit-range kernel (L2 reduction) instead of clusters
@@ -970,6 +975,12 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   A_(c->mb.fwd_ids, sizeof(int) * static_cast<size_t>(g.max_batch) * MB_MAX_WINDOW * g.block);
   A_(c->gen.fwd_ids, sizeof(int) * 2 * static_cast<size_t>(g.max_batch) * g.block);
   A_(c->gen.counters, sizeof(long long) * 8);
+  A_(c->hist_ids, sizeof(int) * static_cast<size_t>(g.max_batch) * g.max_seq);
+  A_(c->refresh_ids, sizeof(int) * R);
+  A_(c->gen.refresh_flag, sizeof(int) * g.max_batch);
+  A_(c->mb.stab, sizeof(int) * static_cast<size_t>(g.max_batch) * MB_MAX_WINDOW);
+  c->gen.hist = c->hist_ids;
+  c->mb.hist = c->hist_ids;
   if (cudaMallocHost(reinterpret_cast<void**>(&c->host_counters), sizeof(long long) * 8) != cudaSuccess)
     return bail(D3_ERR_OOM);
   c->tap_rows = static_cast<int>(dec_rows);
@@ -1158,9 +1169,48 @@ extern "C" int d3_prefill(d3_ctx* c, const int32_t* prompt_ids, const int32_t* p
   prefill_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(prompt_lens, bs, p_max, c->prefix_len, c->pos_base, c->n_valid, c->kv_len);
   LAUNCHED(c, "prefill_rowmap_kernel");
   TRY(forward(c, prompt_ids, bs, p_max, 0, nullptr));
+  if (p_max > 0) {
+    hist_store_kernel<<<bs, 128, 0, c->stream>>>(prompt_ids, p_max, c->prefix_len, 0, nullptr, c->hist_ids, c->cfg.max_seq);
+    LAUNCHED(c, "hist_store_kernel");
+  }
   c->prefilled = true;
   return D3_OK;
 }
+
+// One forward over the stored prefixes (flags null: every sequence; else the flagged ones, and only
+// sequences with active[b] > 0 when that is given); their K/V are overwritten in place.
+static int refresh_forward(d3_ctx* c, int bs, int* flags, const int* active, long long* pending) {
+  std::vector<int> pl(bs);
+  CUDA_TRY(c, cudaMemcpyAsync(pl.data(), c->prefix_len, sizeof(int) * bs, cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  int p_max = 0;
+  for (int b = 0; b < bs; ++b) p_max = std::max(p_max, pl[b]);
+  if (p_max > c->cfg.max_seq || static_cast<long long>(bs) * p_max > c->max_rows)
+    return fail(c, D3_ERR_SHAPE, "KV-refresh: bs * longest stored prefix exceeds the workspaces (raise max_prefill_rows at d3_create)");
+  if (p_max == 0) return D3_OK;
+  refresh_rowmap_kernel<<<bs, 128, 0, c->stream>>>(c->hist_ids, c->cfg.max_seq, c->prefix_len, flags, active, p_max, 0, c->refresh_ids,
+                                                   c->pos_base, c->n_valid, c->kv_len, pending);
+  LAUNCHED(c, "refresh_rowmap_kernel");
+  TRY(forward(c, c->refresh_ids, bs, p_max, 0, nullptr));
+  return D3_OK;
+}
+
+extern "C" int d3_refresh_cache(d3_ctx* c, int32_t bs) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (bs <= 0) return fail(c, D3_ERR_INVALID_ARG, "bad refresh_cache arguments");
+  if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_refresh_cache before d3_prefill");
+  if (bs > c->cfg.max_batch) return fail(c, D3_ERR_SHAPE, "bs > max_batch");
+  return refresh_forward(c, bs, nullptr, nullptr, nullptr);
+}
+
+extern "C" int d3_set_cache_policy(d3_ctx* c, int32_t cache_delay, int32_t refresh_every) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (cache_delay < 1 || cache_delay > 16 || refresh_every < 0) return fail(c, D3_ERR_INVALID_ARG, "cache_delay must be 1..16 and refresh_every >= 0");
+  c->cache_delay = cache_delay;
+  c->refresh_every = refresh_every;
+  return D3_OK;
+}
+extern "C" int64_t d3_refresh_count(d3_ctx* c) { return c ? c->last_refreshes : 0; }
 
 extern "C" int d3_denoise_step(d3_ctx* c, int32_t* block_ids, uint8_t* mask, float threshold, int32_t bs,
                                int32_t* out_pos, int32_t* out_ids, int32_t* out_count) {
@@ -1187,6 +1237,8 @@ extern "C" int d3_commit_block(d3_ctx* c, const int32_t* block_ids, int32_t bs) 
   decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B, c->pos_base, c->n_valid, c->kv_len);
   LAUNCHED(c, "decode_rowmap_kernel");
   TRY(forward(c, block_ids, bs, B, 0, nullptr));
+  hist_store_kernel<<<bs, 128, 0, c->stream>>>(block_ids, B, nullptr, B, c->prefix_len, c->hist_ids, c->cfg.max_seq);
+  LAUNCHED(c, "hist_store_kernel");
   add_prefix_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B);
   LAUNCHED(c, "add_prefix_kernel");
   return D3_OK;
@@ -1214,19 +1266,26 @@ extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t 
   gen_init_kernel<<<bs, 32, 0, c->stream>>>(g, bs, B, c->cfg.mask_id, gen_len);
   LAUNCHED(c, "gen_init_kernel");
   const long long max_iter = static_cast<long long>(n_blocks) * (B + 1) + 1;
-  const int fuse = (c->gen_fuse && 2ll * bs * B <= FUSE_MAX_ROWS && 2ll * c->cfg.max_batch * B <= FUSE_MAX_ROWS) ? 1 : 0;
+  // (a refresh falls between a block's finalize forward and the next block's first step: no fusing then)
+  const int fuse = (c->gen_fuse && c->refresh_every == 0 && 2ll * bs * B <= FUSE_MAX_ROWS && 2ll * c->cfg.max_batch * B <= FUSE_MAX_ROWS) ? 1 : 0;
   long long steps = 0;
+  c->last_refreshes = 0;
   int R = B;  // rows per sequence of the next forward: 2B while some sequence runs a fused finalize + first step
   for (long long it = 0; it < max_iter; ++it) {
     gen_rowmap_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, R, c->cfg.mask_id, c->pos_base, c->n_valid, c->kv_len);
     LAUNCHED(c, "gen_rowmap_kernel");
     TRY(forward(c, g.fwd_ids, bs, R, 1, nullptr, R > B ? B : 0));
-    gen_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, R, n_blocks, gen_len, threshold, c->cfg.decide_mode, c->cfg.mask_id, fuse, c->eos_id);
+    gen_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, R, n_blocks, gen_len, threshold, c->cfg.decide_mode, c->cfg.mask_id, fuse, c->eos_id,
+                                                 c->cfg.max_seq, c->refresh_every);
     LAUNCHED(c, "gen_advance_kernel");
     ++steps;
-    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 7, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 8, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     if (c->host_counters[4] <= 0) break;
+    if (c->host_counters[7] > 0) {  // some sequences stored a block that completes a refresh period
+      c->last_refreshes += c->host_counters[7];
+      TRY(refresh_forward(c, bs, g.refresh_flag, nullptr, g.counters + 7));
+    }
     R = c->host_counters[5] > 0 ? 2 * B : B;
   }
   c->last_early_stops = c->host_counters[6];
@@ -1269,8 +1328,9 @@ extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshol
   g.commit_round = commit_round;
   mb_init_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, W, c->cfg.mask_id, gen_len);
   LAUNCHED(c, "mb_init_kernel");
-  const long long max_iter = static_cast<long long>(n_blocks) * (B + 1) + 1;
+  const long long max_iter = static_cast<long long>(n_blocks) * (B + c->cache_delay) + 1;
   long long rounds = 0;
+  c->last_refreshes = 0;
   int R = B;
   for (long long it = 0; it < max_iter; ++it) {
     mb_rowmap_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, W, R, c->cfg.mask_id, c->pos_base, c->n_valid, c->kv_len);
@@ -1278,11 +1338,16 @@ extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshol
     TRY(forward(c, g.fwd_ids, bs, R, 1, nullptr, B));
     ++rounds;
     mb_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, W, R, n_blocks, gen_len, threshold,
-                                                c->cfg.decide_mode, c->cfg.mask_id, max_active, static_cast<int>(rounds));
+                                                c->cfg.decide_mode, c->cfg.mask_id, max_active, static_cast<int>(rounds), c->cache_delay,
+                                                c->cfg.max_seq);
     LAUNCHED(c, "mb_advance_kernel");
     CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 7, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     if (c->host_counters[4] <= 0) break;
+    if (c->refresh_every > 0 && rounds % c->refresh_every == 0) {  // periodic KV-refresh of the sequences still decoding
+      c->last_refreshes += c->host_counters[4];
+      TRY(refresh_forward(c, bs, nullptr, g.n_win, nullptr));
+    }
     R = static_cast<int>(std::max<long long>(1, c->host_counters[5])) * B;
   }
   if (host_stats) {

@@ -340,7 +340,9 @@ struct GenState {
   int* out_ids;     // [bs, gen_len]
   int* commit_step; // [bs, gen_len] or null
   long long* counters;  // [0] denoise fwd, [1] finalize fwd, [2] tokens, [3] forced, [4] seqs not done, [5] seqs in SEQ_FUSED,
-                        // [6] sequences stopped early on the end-of-sequence id
+                        // [6] sequences stopped early on the end-of-sequence id, [7] sequences waiting for a KV-refresh
+  int* hist;            // [bs, max_seq] ids of the stored prefix (prompt and stored blocks)
+  int* refresh_flag;    // [bs] 1: the stored prefix of this sequence is to be recomputed before the next forward
 };
 
 // Row map and input ids of the next decode forward (rows_per_seq = R, B or 2B) from the generate
@@ -366,17 +368,21 @@ __global__ void gen_rowmap_kernel(GenState g, int bs, int B, int R, int mask_id,
 // per sequence.
 __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, const float* __restrict__ ent,
                                    const int* __restrict__ argmax, int bs, int B, int R, int n_blocks, int gen_len,
-                                   float tau, int decide_mode, int mask_id, int fuse, int eos_id) {
+                                   float tau, int decide_mode, int mask_id, int fuse, int eos_id, int max_seq,
+                                   int refresh_every) {
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31;
   const int mode = g.mode[b];
   if (mode == SEQ_DONE) return;
   int* ids = g.ids + b * B;
   uint8_t* mask = g.mask + b * B;
+  const int pl = g.prefix_len[b];  // before this kernel moves it
+  __syncwarp();
   if (mode == SEQ_FINALIZE) {  // the block in `ids` is final and now cached: append it, next block or done
     const int j = g.block_idx[b];
     for (int r = lane; r < B; r += 32) {
       g.out_ids[static_cast<size_t>(b) * gen_len + j * B + r] = ids[r];
+      g.hist[static_cast<size_t>(b) * max_seq + pl + r] = ids[r];
       ids[r] = mask_id;
       mask[r] = 1;
     }
@@ -391,6 +397,11 @@ __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, c
         atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[4]), static_cast<unsigned long long>(-1ll));
       } else {
         g.mode[b] = SEQ_DENOISE;
+        // periodic KV-refresh: the stored block count reached a multiple of the period
+        if (refresh_every > 0 && (j + 1) % refresh_every == 0) {
+          g.refresh_flag[b] = 1;
+          atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[7]), 1ull);
+        }
       }
     }
     return;
@@ -398,7 +409,10 @@ __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, c
   int stat_row0 = b * R;  // rows of the block that was denoised in this forward
   if (mode == SEQ_FUSED) {  // segment 0 finalized the block in `prev`: append it; segment 1 was a first denoise step
     const int j = g.block_idx[b] - 1;
-    for (int r = lane; r < B; r += 32) g.out_ids[static_cast<size_t>(b) * gen_len + j * B + r] = g.prev[b * B + r];
+    for (int r = lane; r < B; r += 32) {
+      g.out_ids[static_cast<size_t>(b) * gen_len + j * B + r] = g.prev[b * B + r];
+      g.hist[static_cast<size_t>(b) * max_seq + pl + r] = g.prev[b * B + r];
+    }
     if (lane == 0) {
       g.prefix_len[b] += B;
       atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[1]), 1ull);
@@ -478,8 +492,9 @@ __global__ void gen_init_kernel(GenState g, int bs, int B, int mask_id, int gen_
     g.mode[b] = SEQ_DENOISE;
     g.block_idx[b] = 0;
     g.step[b] = 0;
+    g.refresh_flag[b] = 0;
     if (b == 0) {
-      g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = g.counters[5] = g.counters[6] = 0;
+      g.counters[0] = g.counters[1] = g.counters[2] = g.counters[3] = g.counters[5] = g.counters[6] = g.counters[7] = 0;
       g.counters[4] = bs;
     }
   }
@@ -501,6 +516,8 @@ struct MbState {
   int* commit_round;  // [bs, gen_len] or null
   long long* counters;  // [0] block decisions taken, [1] blocks stored in the cache, [2] tokens, [3] forced commits,
                         // [4] sequences not done, [5] largest window of the next round, [6] rows of valid work so far
+  int* stab;            // [bs, W] stabilizing forwards each block in flight has had
+  int* hist;            // [bs, max_seq] ids of the stored prefix
 };
 constexpr int MB_MAX_WINDOW = 8;
 
@@ -511,6 +528,7 @@ __global__ void mb_init_kernel(MbState g, int bs, int B, int W, int mask_id, int
     g.mask[b * W * B + r] = 1;
   }
   for (int r = threadIdx.x; r < gen_len; r += blockDim.x) g.out_ids[static_cast<size_t>(b) * gen_len + r] = mask_id;
+  if (threadIdx.x < W) g.stab[b * W + threadIdx.x] = 0;
   if (threadIdx.x == 0) {
     g.lo[b] = 0;
     g.n_win[b] = 1;
@@ -536,14 +554,16 @@ __global__ void mb_rowmap_kernel(MbState g, int bs, int B, int W, int R, int mas
 }
 
 // After the forward of a round.  States are read from the masks as they stood before the forward:
-// a block without masks has just had its stabilizing forward; a block whose predecessor in the
+// a block without masks has just had a stabilizing forward (it is stored after `cache_delay` of
+// them); a block whose predecessor in the
 // window is at least 95 % unmasked (or that is the oldest) is Fully-Activated and commits at least
 // one token; the others are Activated and commit only what clears the threshold.  Then the leading
 // complete blocks enter the cache, and a new block is opened once the newest one is 10 % unmasked.
 // One warp per sequence.
 __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, const float* __restrict__ ent,
                                   const int* __restrict__ argmax, int bs, int B, int W, int R, int n_blocks, int gen_len,
-                                  float tau, int decide_mode, int mask_id, int max_active, int round) {
+                                  float tau, int decide_mode, int mask_id, int max_active, int round, int cache_delay,
+                                  int max_seq) {
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31;
   int n = g.n_win[b];
@@ -551,7 +571,11 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
   int* ids = g.ids + b * W * B;
   uint8_t* mask = g.mask + b * W * B;
   const int lo = g.lo[b];
-  int unmasked[MB_MAX_WINDOW];
+  const int pl = g.prefix_len[b];
+  int unmasked[MB_MAX_WINDOW], stab[MB_MAX_WINDOW];
+#pragma unroll
+  for (int w = 0; w < MB_MAX_WINDOW; ++w) stab[w] = w < n ? g.stab[b * W + w] : 0;
+  __syncwarp();
 #pragma unroll
   for (int w = 0; w < MB_MAX_WINDOW; ++w) {
     unmasked[w] = 0;
@@ -579,11 +603,21 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
     }
   }
   __syncwarp();
-  // leading blocks that were complete before this forward: out and into the cache
+  // blocks that were complete before this forward have had one more stabilizing round; the leading
+  // ones that have had cache_delay of them go out and into the cache
+#pragma unroll
+  for (int w = 0; w < MB_MAX_WINDOW; ++w)
+    if (w < n && unmasked[w] == B) stab[w] += 1;
   int k = 0;
-  while (k < n && unmasked[k] == B) ++k;
+#pragma unroll
+  for (int w = 0; w < MB_MAX_WINDOW; ++w)
+    if (w == k && w < n && stab[w] >= cache_delay) ++k;
   for (int q = 0; q < k; ++q)
-    for (int r = lane; r < B; r += 32) g.out_ids[static_cast<size_t>(b) * gen_len + (lo + q) * B + r] = ids[q * B + r];
+    for (int r = lane; r < B; r += 32) {
+      g.out_ids[static_cast<size_t>(b) * gen_len + (lo + q) * B + r] = ids[q * B + r];
+      g.hist[static_cast<size_t>(b) * max_seq + pl + q * B + r] = ids[q * B + r];
+    }
+  __syncwarp();
   if (k > 0) {
     const int left = (n - k) * B;
     for (int r0 = 0; r0 < left; r0 += 32) {  // move the rest of the window down: read, then write
@@ -594,6 +628,14 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
       __syncwarp();
       if (r < left) { ids[r] = v; mask[r] = m; }
       __syncwarp();
+    }
+#pragma unroll
+    for (int w = 0; w < MB_MAX_WINDOW; ++w) {  // k is not a compile-time constant: select instead of indexing
+      int v = 0;
+#pragma unroll
+      for (int u = 0; u < MB_MAX_WINDOW; ++u)
+        if (u == w + k) v = stab[u];
+      stab[w] = v;
     }
     n -= k;
   }
@@ -614,11 +656,17 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
         ids[n * B + r] = mask_id;
         mask[n * B + r] = 1;
       }
+#pragma unroll
+      for (int w = 0; w < MB_MAX_WINDOW; ++w)
+        if (w == n) stab[w] = 0;
       ++n;
     }
   }
   __syncwarp();
   if (lane == 0) {
+#pragma unroll
+    for (int w = 0; w < MB_MAX_WINDOW; ++w)
+      if (w < W) g.stab[b * W + w] = w < n ? stab[w] : 0;
     g.lo[b] = lo + k;
     g.n_win[b] = n;
     g.prefix_len[b] += k * B;
@@ -629,6 +677,41 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
     if (n == 0) atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[4]), static_cast<unsigned long long>(-1ll));
     atomicMax(reinterpret_cast<unsigned long long*>(&g.counters[5]), static_cast<unsigned long long>(n));
   }
+}
+
+// The ids of the stored prefix are kept per sequence (prompt at prefill, every block when it is
+// stored), so that the cache can be recomputed from them (KV-refresh, Sec. 3.2).
+// hist[b, off_b + r] = src[b * src_stride + r] for r < count_b; off = 0 when `off` is null,
+// count = fixed_count when `count` is null.  One block per sequence.
+__global__ void hist_store_kernel(const int* __restrict__ src, int src_stride, const int* __restrict__ count, int fixed_count,
+                                  const int* __restrict__ off, int* __restrict__ hist, int max_seq) {
+  const int b = blockIdx.x;
+  int n = count ? count[b] : fixed_count;
+  const int o = off ? off[b] : 0;
+  n = n < 0 ? 0 : (n > src_stride ? src_stride : n);
+  if (o + n > max_seq) n = max_seq - o;
+  for (int r = threadIdx.x; r < n; r += blockDim.x) hist[static_cast<size_t>(b) * max_seq + o + r] = src[static_cast<size_t>(b) * src_stride + r];
+}
+// Row map and input ids of a KV-refresh forward over the stored prefixes: rows_per_seq = p_max, rows
+// [0, prefix_len_b) of a sequence that takes part (flag null or set; flags are cleared here) are valid
+// and sit at positions 0.., the rest is padding.  prefix_len is left alone.  One block per sequence.
+__global__ void refresh_rowmap_kernel(const int* __restrict__ hist, int max_seq, const int* __restrict__ prefix_len,
+                                      int* flag, const int* __restrict__ active, int p_max, int pad_id, int* __restrict__ dst_ids,
+                                      int* pos_base, int* n_valid, int* kv_len, long long* pending) {
+  const int b = blockIdx.x;
+  const bool take = (flag == nullptr || flag[b] != 0) && (active == nullptr || active[b] > 0);
+  int len = take ? prefix_len[b] : 0;
+  len = len > p_max ? p_max : len;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    pos_base[b] = 0;
+    n_valid[b] = len;
+    kv_len[b] = len;
+    if (flag) flag[b] = 0;
+    if (pending && b == 0) *pending = 0;
+  }
+  for (int r = threadIdx.x; r < p_max; r += blockDim.x)
+    dst_ids[static_cast<size_t>(b) * p_max + r] = r < len ? hist[static_cast<size_t>(b) * max_seq + r] : pad_id;
 }
 
 // Row maps for the explicit API.

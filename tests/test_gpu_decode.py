@@ -19,7 +19,7 @@ EPS = 1e-3
 
 
 def step_locked(ctx: Ctx, model: o.OracleModel, prompts, lens, gen_len, block, tau, mode=0, logit_tol=None,
-                exact_model=None):
+                exact_model=None, refresh_every=0):
     """Follow the oracle's trajectory: before every GPU step inject the oracle's (ids, mask), compare the
     statistics and the commit set, and finalize each block with the oracle's final ids.
 
@@ -32,11 +32,13 @@ def step_locked(ctx: Ctx, model: o.OracleModel, prompts, lens, gen_len, block, t
     two best masked positions for the forced commit, or the top-2 probability gap for the id -- is below
     1e-3), ``rounding`` (the margin is below twice the largest statistic error observed over the run,
     i.e. the two sides disagree by less than their own numerical difference), or ``unexplained``.
-    The decision kernel itself is checked bit-exactly on the GPU's own statistics (``self_diff``)."""
+    The decision kernel itself is checked bit-exactly on the GPU's own statistics (``self_diff``).
+    With ``refresh_every`` both sides refresh the cache after every that many stored blocks."""
     exact_model = exact_model or model
     bs = len(lens)
     ctx.prefill(prompts, lens)
-    traces = [model.generate(prompts[b, :lens[b]], gen_len, block, tau, mode, record=True) for b in range(bs)]
+    traces = [model.generate(prompts[b, :lens[b]], gen_len, block, tau, mode, record=True, refresh_every=refresh_every)
+              for b in range(bs)]
     report = dict(steps=0, positions=0, excused=0, rounding=0, unexplained=0, self_diff=0, max_stat_err=0.0,
                   max_logit_err=0.0)
     n_blocks = gen_len // block
@@ -52,7 +54,7 @@ def step_locked(ctx: Ctx, model: o.OracleModel, prompts, lens, gen_len, block, t
                 lg = ctx.logits(ids)
                 for b in range(bs):
                     ref = exact_model.denoise_forward(
-                        _state_at(exact_model, traces[b], prompts[b, :lens[b]], j, block), ids[b])[0]
+                        _state_at(exact_model, traces[b], prompts[b, :lens[b]], j, block, refresh_every), ids[b])[0]
                     err = np.max(np.abs(lg[b] - ref)) / np.max(np.abs(ref))
                     report["max_logit_err"] = max(report["max_logit_err"], float(err))
             got = ctx.step(ids, mask, tau)
@@ -89,12 +91,14 @@ def step_locked(ctx: Ctx, model: o.OracleModel, prompts, lens, gen_len, block, t
                 both = have & want
                 tok_diff = np.flatnonzero(both & (got["ids"][b] != t["tok"]))
                 if len(tok_diff):
-                    ref_lg = model.denoise_forward(_state_at(model, traces[b], prompts[b, :lens[b]], j, block),
+                    ref_lg = model.denoise_forward(_state_at(model, traces[b], prompts[b, :lens[b]], j, block, refresh_every),
                                                    t["ids_in"])[0]
                     gap = top2_gap(ref_lg, model.mask_id)
                     margins.extend(float(gap[r]) for r in tok_diff)
         final = np.stack([traces[b]["tokens"][j * block:(j + 1) * block] for b in range(bs)]).astype(np.int32)
         ctx.commit(final)
+        if refresh_every > 0 and (j + 1) % refresh_every == 0 and j + 1 < n_blocks:
+            d3.d3_refresh_cache(ctx.ctx, bs)
     assert ctx.error_word() == 0
     noise = 2 * report["max_stat_err"] + 1e-6
     for m in margins:
@@ -105,13 +109,15 @@ def step_locked(ctx: Ctx, model: o.OracleModel, prompts, lens, gen_len, block, t
 _STATE_CACHE = {}
 
 
-def _state_at(model, trace, prompt, j, block):
+def _state_at(model, trace, prompt, j, block, refresh_every=0):
     """Oracle cache state at the start of block j (recomputed; small models only)."""
-    key = (id(model), id(trace), j)
+    key = (id(model), id(trace), j, refresh_every)
     if key not in _STATE_CACHE:
         st = model.prefill(prompt)
         for jj in range(j):
             st = model.finalize_block(st, trace["tokens"][jj * block:(jj + 1) * block])
+            if refresh_every > 0 and (jj + 1) % refresh_every == 0:
+                st = model.refresh(st)
         _STATE_CACHE[key] = st
     return _STATE_CACHE[key]
 

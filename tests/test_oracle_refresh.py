@@ -8,7 +8,7 @@ import pytest
 
 from oracle import d3_oracle as o
 from paper_2601_07568_b200 import synth_inputs as si
-from tests.test_oracle_decoding import micro_model
+from test_oracle_decoding import micro_model
 
 
 def _c1_model():
