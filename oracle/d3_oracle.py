@@ -56,6 +56,16 @@ What the paper fixes (cited per function) and what it leaves open
   rounds (forwards in which the block was already complete) before a block's
   K and V are stored.
 
+* Pseudo-trajectory (Sec. 3.1): the teacher unmasks exactly one token per
+  step and decodes past EOS to the full length; only the order is kept.  The
+  noisy sequence keeps y_i up to the window start s and wherever trajectory
+  state T_{s+ceil(kt)} is unmasked, and masks everything after the window
+  and wherever that state is masked.  Readings: the extraction run is
+  ``generate`` at threshold 1 (no probability exceeds 1, so every step commits
+  only the forced, most confident token) without EOS stop; in the overlap of
+  the equation's cases i <= s wins, then i > s+k, then the trajectory; the
+  tokens y must not contain the mask id.
+
 Readings taken where the paper is silent are listed in the repository's
 design notes; in short: block-causal visibility between segments (prompt =
 segment 0, generation block j = segment j), which makes the prefix cache
@@ -530,6 +540,64 @@ class OracleModel:
             state = self.finalize_block(state, ids)
             tokens[j * block:(j + 1) * block] = ids
         return tokens, np.asarray(order, dtype=np.int32)
+
+
+# ----------------------------------------------------------------------------- pseudo-trajectory
+def trajectory_rank(commit_step: np.ndarray, block: int) -> np.ndarray:
+    """Decoding step (1-based, counted over the whole response) at which each position was unmasked,
+    from the per-block step indices ``generate`` records: blocks are decoded one after the other,
+    so a block's steps follow all steps of the blocks before it (Sec. 3.1: the recorded decoding
+    trajectory T_1..T_n; with exactly one token per step the ranks are a permutation of 1..n)."""
+    commit_step = np.asarray(commit_step)
+    n = commit_step.shape[0]
+    assert n % block == 0
+    rank = np.zeros(n, dtype=np.int64)
+    done = 0
+    for j in range(n // block):
+        cs = commit_step[j * block:(j + 1) * block]
+        rank[j * block:(j + 1) * block] = done + cs
+        done += int(cs.max())
+    return rank
+
+
+def trajectory_states(y: np.ndarray, rank: np.ndarray, mask_id: int) -> np.ndarray:
+    """The trajectory written out: row j (0..n_steps) is the response after j decoding steps, the
+    positions unmasked so far holding y's tokens and the rest ``mask_id`` (Sec. 3.1, T_j)."""
+    y = np.asarray(y)
+    n_steps = int(np.max(rank)) if len(rank) else 0
+    T = np.full((n_steps + 1, len(y)), mask_id, dtype=np.int64)
+    for j in range(n_steps + 1):
+        for i in range(len(y)):
+            if rank[i] <= j:
+                T[j, i] = y[i]
+    return T
+
+
+def ceil_ratio(k: int, t_num: int, t_den: int) -> int:
+    """ceil(k * t) for the mask ratio t = t_num / t_den in integers."""
+    assert t_den > 0 and 0 <= t_num <= t_den and k >= 0
+    return -((-k * t_num) // t_den)
+
+
+def noisy_sequence(y: np.ndarray, rank: np.ndarray, s: int, k: int, m: int, mask_id: int) -> np.ndarray:
+    """The noisy training sequence of Sec. 3.1 (the displayed equation): with positions counted
+    from 1, window w = {s, .., s+k} and m = ceil(k t), position i keeps y_i if i <= s or it is
+    unmasked in trajectory state T_{s+m}, and is the mask token if i > s+k or it is still masked
+    in T_{s+m}.  Reading taken where the two cases overlap: i <= s keeps the token, i > s+k is
+    masked, and only in between does the trajectory decide.  A step index beyond the recorded
+    trajectory means its last state."""
+    y = np.asarray(y)
+    T = trajectory_states(y, rank, mask_id)
+    step = min(s + m, T.shape[0] - 1)
+    out = np.empty(len(y), dtype=np.int64)
+    for i in range(1, len(y) + 1):
+        if i <= s:
+            out[i - 1] = y[i - 1]
+        elif i > s + k:
+            out[i - 1] = mask_id
+        else:
+            out[i - 1] = y[i - 1] if T[step, i - 1] != mask_id else mask_id
+    return out
 
 
 def model_from_shape(shape, weights: Dict[str, object], dtype=np.float64, mirror_bf16: bool = False
