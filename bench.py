@@ -346,6 +346,32 @@ def run_ours(args):
                   "decode_refresh_every_4_blocks": {"value": whole_job_tokens_per_s(world, tokens_of(w), args.steps, ms_rf), "unit": UNIT,
                                                     "refreshes_per_request": int(n_refresh)}}
 
+    # pseudo-trajectory extraction (threshold 1: one token per forward, full length) on the same request,
+    # and the noisy-sequence builder on a training-sized batch of responses
+    cs_dev = torch.zeros((w.batch, w.gen_len), dtype=torch.int32, device=dev)
+    def step_extract():
+        d3.d3_prefill(ctx, ids_dev, lens_dev)
+        return d3.d3_generate(ctx, w.gen_len, 1.0, out_dev, cs_dev)
+    ms_ex, st_ex = timed(step_extract, 1)
+    rank_dev = torch.zeros_like(cs_dev)
+    d3.d3_trajectory_rank(ctx, cs_dev, rank_dev)
+    nb, nn = 16384, w.gen_len
+    gnr = torch.Generator(device=dev).manual_seed(7)
+    y_big = torch.randint(0, shape.vocab - 2, (nb, nn), dtype=torch.int32, device=dev, generator=gnr)
+    rank_big = rank_dev[:1].expand(nb, nn).contiguous()
+    s_big = torch.randint(0, nn // 2, (nb,), dtype=torch.int32, device=dev, generator=gnr)
+    k_big = torch.full((nb,), w.block, dtype=torch.int32, device=dev)
+    m_big = torch.randint(0, w.block + 1, (nb,), dtype=torch.int32, device=dev, generator=gnr)
+    noisy = torch.empty_like(y_big)
+    d3.d3_noisy_sequence(ctx, y_big, rank_big, s_big, k_big, m_big, noisy)
+    ms_ns, _ = timed(lambda: d3.d3_noisy_sequence(ctx, y_big, rank_big, s_big, k_big, m_big, noisy), 20)
+    ms_ns /= 20
+    trajectory = {"extraction": {"value": whole_job_tokens_per_s(world, tokens_of(w), 1, ms_ex), "unit": UNIT,
+                                 "forwards_per_request": int(st_ex.denoise_forwards + st_ex.finalize_forwards) // max(w.batch, 1)},
+                  "noisy_sequence": {"sequences": nb, "tokens_each": nn, "us_per_launch": ms_ns * 1e3,
+                                     "GB/s": 3 * nb * nn * 4 / (ms_ns * 1e-3) / 1e9}}
+    del y_big, rank_big, noisy
+
     # per-class kernel times of the decode loop (one request, events around every launch)
     d3.d3_prefill(ctx, ids_dev, lens_dev)
     torch.cuda.synchronize()
@@ -418,7 +444,7 @@ def run_ours(args):
                    "tokens_per_forward_incl_finalize": tokens / max(st.denoise_forwards + st.finalize_forwards, 1),
                    "ms_per_forward": (ms_step - ms_prefill) / max(forwards, 1), "prefill_ms": ms_prefill,
                    "forced_commits": int(st.forced_commits)},
-        "multiblock": multiblock, "kv_refresh": kv_refresh, "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
+        "multiblock": multiblock, "kv_refresh": kv_refresh, "trajectory": trajectory, "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
         "device_bytes": d3.d3_device_bytes(ctx),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -179,6 +179,23 @@ int d3_generate_multiblock(d3_ctx *ctx, int32_t gen_len, float threshold, int32_
 int d3_set_eos(d3_ctx *ctx, int32_t eos_id);
 int64_t d3_early_stops(d3_ctx *ctx);
 
+/* Pseudo-trajectory extraction (Sec. 3.1): a d3_generate run with threshold 1 and no end-of-sequence
+ * id unmasks exactly one token per step (no probability exceeds 1, so only the forced commit of the
+ * most confident position happens) and decodes the full length; its commit_step output is the
+ * trajectory.  d3_trajectory_rank turns commit_step [device][bs, gen_len] (step within the block) into
+ * rank [device][bs, gen_len]: the step, counted from 1 over the whole response, at which each position
+ * was unmasked (a block's steps follow those of all earlier blocks; positions committed in the same
+ * step share a rank).  Asynchronous on the context's stream.  SHAPE when gen_len is not a multiple of B. */
+int d3_trajectory_rank(d3_ctx *ctx, const int32_t *commit_step, int32_t bs, int32_t gen_len, int32_t *rank);
+
+/* The noisy training sequence of Sec. 3.1 (displayed equation) for bs responses of n tokens: with
+ * positions counted from 1, window start s[b], window length k[b] and m[b] = ceil(k t) for mask ratio
+ * t (computed by the caller in integers), out[b, i] = y[b, i] if i <= s, mask_id if i > s + k, and in
+ * between y[b, i] if rank[b, i] <= s + m (unmasked in trajectory state T_{s+m}), else mask_id.
+ * y, rank, out [device][bs, n]; s, k, m [device][bs].  Asynchronous on the context's stream. */
+int d3_noisy_sequence(d3_ctx *ctx, const int32_t *y, const int32_t *rank, const int32_t *s, const int32_t *k,
+                      const int32_t *m, int32_t bs, int32_t n, int32_t *out);
+
 /* KV-refresh (Sec. 3.2, "KV-Cache and KV-Refresh Mechanism": previously cached states are recomputed
  * by full forward passes).  One forward over the tokens of the stored prefix of each of the bs
  * sequences (the prompt and every block stored since, as recorded by d3_prefill, d3_commit_block and

@@ -1363,6 +1363,24 @@ extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshol
   return check_device_error(c);
 }
 
+extern "C" int d3_trajectory_rank(d3_ctx* c, const int32_t* commit_step, int32_t bs, int32_t gen_len, int32_t* rank) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!commit_step || !rank || bs <= 0 || gen_len <= 0) return fail(c, D3_ERR_INVALID_ARG, "bad trajectory_rank arguments");
+  if (gen_len % c->cfg.block != 0) return fail(c, D3_ERR_SHAPE, "gen_len not a multiple of the block size");
+  trajectory_rank_kernel<<<bs, 32, 0, c->stream>>>(commit_step, gen_len, c->cfg.block, rank);
+  LAUNCHED(c, "trajectory_rank_kernel");
+  return D3_OK;
+}
+extern "C" int d3_noisy_sequence(d3_ctx* c, const int32_t* y, const int32_t* rank, const int32_t* s, const int32_t* k,
+                                 const int32_t* m, int32_t bs, int32_t n, int32_t* out) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!y || !rank || !s || !k || !m || !out || bs <= 0 || n <= 0) return fail(c, D3_ERR_INVALID_ARG, "bad noisy_sequence arguments");
+  if (bs > 65535) return fail(c, D3_ERR_SHAPE, "more than 65535 sequences in one call");
+  noisy_sequence_kernel<<<dim3((n + 255) / 256, bs), 256, 0, c->stream>>>(y, rank, s, k, m, n, c->cfg.mask_id, out);
+  LAUNCHED(c, "noisy_sequence_kernel");
+  return D3_OK;
+}
+
 extern "C" int d3_set_eos(d3_ctx* c, int32_t eos_id) {
   if (!c) return D3_ERR_INVALID_ARG;
   if (eos_id >= c->cfg.vocab || eos_id == c->cfg.mask_id) return fail(c, D3_ERR_INVALID_ARG, "eos id outside the vocabulary or equal to the mask id");

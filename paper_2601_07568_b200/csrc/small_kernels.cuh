@@ -714,6 +714,50 @@ __global__ void refresh_rowmap_kernel(const int* __restrict__ hist, int max_seq,
     dst_ids[static_cast<size_t>(b) * p_max + r] = r < len ? hist[static_cast<size_t>(b) * max_seq + r] : pad_id;
 }
 
+// ----------------------------------------------------------------------------- pseudo-trajectory (Sec. 3.1)
+// rank[b, i] = decoding step, counted from 1 over the whole response, at which position i was
+// unmasked, from the per-block step indices the generate loop records: a block's steps follow all
+// steps of the blocks before it.  One warp per sequence; blocks are walked in order.
+__global__ void trajectory_rank_kernel(const int* __restrict__ commit_step, int gen_len, int B, int* __restrict__ rank) {
+  const int b = blockIdx.x, lane = threadIdx.x & 31;
+  const int* cs = commit_step + static_cast<size_t>(b) * gen_len;
+  int* out = rank + static_cast<size_t>(b) * gen_len;
+  int done = 0;
+  for (int j0 = 0; j0 < gen_len; j0 += B) {
+    int mx = 0;
+    for (int r = lane; r < B; r += 32) {
+      const int v = cs[j0 + r];
+      out[j0 + r] = done + v;
+      mx = v > mx ? v : mx;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      const int other = __shfl_xor_sync(0xffffffffu, mx, o);
+      mx = other > mx ? other : mx;
+    }
+    done += mx;
+  }
+}
+// The noisy sequence of Sec. 3.1 for a batch: with positions counted from 1, window start s, window
+// length k and m = ceil(k t), position i keeps y_i if i <= s, is the mask id if i > s + k, and in
+// between keeps y_i iff the trajectory had unmasked it by step s + m (rank <= s + m).
+// grid (ceil(n / 256), bs).
+__global__ void noisy_sequence_kernel(const int* __restrict__ y, const int* __restrict__ rank, const int* __restrict__ s_arr,
+                                      const int* __restrict__ k_arr, const int* __restrict__ m_arr, int n, int mask_id,
+                                      int* __restrict__ out) {
+  const int b = blockIdx.y;
+  const int i0 = blockIdx.x * blockDim.x + threadIdx.x;  // position - 1
+  if (i0 >= n) return;
+  const int s = s_arr[b], k = k_arr[b], m = m_arr[b];
+  const size_t at = static_cast<size_t>(b) * n + i0;
+  const int i = i0 + 1;
+  int v;
+  if (i <= s) v = y[at];
+  else if (i > s + k) v = mask_id;
+  else v = rank[at] <= s + m ? y[at] : mask_id;
+  out[at] = v;
+}
+
 // Row maps for the explicit API.
 __global__ void decode_rowmap_kernel(const int* prefix_len, int bs, int B, int* pos_base, int* n_valid, int* kv_len) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
