@@ -66,6 +66,15 @@ What the paper fixes (cited per function) and what it leaves open
   the equation's cases i <= s wins, then i > s+k, then the trajectory; the
   tokens y must not contain the mask id.
 
+* Temperature (Appendix, inference settings: 0.0 or 0.1).  Readings: at
+  temperature T > 0 a row's token is drawn from softmax(l / T) by the
+  Gumbel-max rule, arg max_v (l_v + T g_v) compared in float32, with the mask
+  token excluded; the confidence that meets the threshold is softmax(l) of the
+  drawn token and the entropy is that of softmax(l); the noise comes from
+  Philox-4x32-10 keyed by the seed with counter (v // 4, absolute position,
+  step within the block, sequence index), uniform = top 23 bits centred in
+  their bucket, g = -ln(-ln u) in float32.
+
 Readings taken where the paper is silent are listed in the repository's
 design notes; in short: block-causal visibility between segments (prompt =
 segment 0, generation block j = segment j), which makes the prefix cache
@@ -174,6 +183,69 @@ def softmax_stats(logits: np.ndarray, mask_id: int) -> Tuple[np.ndarray, np.ndar
         plogp = np.where(p > 0.0, p * np.log(p), 0.0)
     ent = -np.sum(plogp, axis=-1)
     return p, conf, tok, ent
+
+
+# ----------------------------------------------------------------------------- sampling noise
+def philox4x32_10(counter: np.ndarray, key: Tuple[int, int]) -> np.ndarray:
+    """Philox-4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw: "Parallel random numbers: as easy as
+    1, 2, 3", SC'11): counter [..., 4] uint32, key two 32-bit words; returns [..., 4] uint32.
+    One round: (hi0, lo0) = M0 * c0, (hi1, lo1) = M1 * c2 as 64-bit products;
+    c <- (hi1 ^ c1 ^ k0, lo1, hi0 ^ c3 ^ k1, lo0); the key is bumped by the Weyl constants
+    between rounds."""
+    M0, M1 = np.uint64(0xD2511F53), np.uint64(0xCD9E8D57)
+    W0, W1 = 0x9E3779B9, 0xBB67AE85
+    c = np.asarray(counter, dtype=np.uint64) & np.uint64(0xFFFFFFFF)
+    c0, c1, c2, c3 = c[..., 0], c[..., 1], c[..., 2], c[..., 3]
+    k0, k1 = int(key[0]) & 0xFFFFFFFF, int(key[1]) & 0xFFFFFFFF
+    lo32, sh = np.uint64(0xFFFFFFFF), np.uint64(32)
+    for r in range(10):
+        p0, p1 = M0 * c0, M1 * c2
+        hi0, lo0, hi1, lo1 = p0 >> sh, p0 & lo32, p1 >> sh, p1 & lo32
+        c0, c1, c2, c3 = hi1 ^ c1 ^ np.uint64(k0), lo1, hi0 ^ c3 ^ np.uint64(k1), lo0
+        k0, k1 = (k0 + W0) & 0xFFFFFFFF, (k1 + W1) & 0xFFFFFFFF
+    return np.stack([c0, c1, c2, c3], axis=-1).astype(np.uint32)
+
+
+def uniform_from_bits(x: np.ndarray) -> np.ndarray:
+    """float32 in (0, 1) from a 32-bit word: the top 23 bits, centred in their bucket (k + 1/2 with
+    k < 2^23 is exact in float32, so neither end point is reached)."""
+    return ((np.asarray(x, dtype=np.uint32) >> np.uint32(9)).astype(np.float32) + np.float32(0.5)) * np.float32(2.0 ** -23)
+
+
+def gumbel_noise(seed: int, seq: int, positions: np.ndarray, step: int, vocab: int) -> np.ndarray:
+    """Standard Gumbel noise g = -ln(-ln u) (float32) for every (row, vocabulary index): one
+    Philox call per four consecutive vocabulary indices with counter (v // 4, absolute position of
+    the row, decoding step within the block, sequence index) and key = the two halves of the
+    seed; index v takes output word v % 4."""
+    positions = np.asarray(positions, dtype=np.uint32)
+    nq = (vocab + 3) // 4
+    ctr = np.zeros((len(positions), nq, 4), dtype=np.uint32)
+    ctr[..., 0] = np.arange(nq, dtype=np.uint32)[None, :]
+    ctr[..., 1] = positions[:, None]
+    ctr[..., 2] = np.uint32(step)
+    ctr[..., 3] = np.uint32(seq)
+    bits = philox4x32_10(ctr, (seed & 0xFFFFFFFF, (seed >> 32) & 0xFFFFFFFF)).reshape(len(positions), nq * 4)[:, :vocab]
+    u = uniform_from_bits(bits)
+    return -np.log(-np.log(u))  # float32 throughout
+
+
+def sample_stats(logits: np.ndarray, mask_id: int, temperature: float, noise: np.ndarray
+                 ) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Temperature sampling by the Gumbel-max rule (Appendix, inference settings: temperature 0
+    or 0.1): the token of a row is arg max_v (l_v + T g_v), which is a draw from
+    softmax(l / T); the mask token is excluded.  The comparison is made in float32 (the
+    precision the logits exist in on the device).  Confidence is the model's probability of
+    the drawn token, softmax(l)[token]; the entropy is that of softmax(l), as without
+    sampling.  Returns (conf, tok, entropy)."""
+    _, _, _, ent = softmax_stats(logits, mask_id)
+    l = np.array(logits, dtype=np.float64, copy=True)
+    l[:, mask_id] = -np.inf
+    p = softmax_rows(l)
+    pert = l.astype(np.float32) + np.float32(temperature) * np.asarray(noise, dtype=np.float32)
+    pert[:, mask_id] = -np.inf
+    tok = np.argmax(pert, axis=-1).astype(np.int32)
+    conf = p[np.arange(p.shape[0]), tok]
+    return conf, tok, ent
 
 
 def decide(conf: np.ndarray, ent: np.ndarray, mask: np.ndarray, tau: float, mode: int = MODE_CONFIDENCE
@@ -329,22 +401,28 @@ class OracleModel:
         seeing every other one, replaces the stored K and V; blocks in flight take no part."""
         return self.prefill(state.ids)
 
-    def denoise_forward(self, state: SeqState, block_ids: np.ndarray):
+    def denoise_forward(self, state: SeqState, block_ids: np.ndarray, sampler: Optional[Dict[str, object]] = None):
         """One forward of the block's rows (masked rows hold mask_id) against the prefix cache.
-        Returns (logits [B, V], conf, tok, entropy)."""
+        Returns (logits [B, V], conf, tok, entropy).  ``sampler`` = dict(temperature, seed, seq,
+        step) draws the tokens at that temperature (``sample_stats``) instead of taking the
+        arg max."""
         B = len(block_ids)
         pos = state.prefix_len + np.arange(B)
         x, _, _ = self.forward_rows(np.asarray(block_ids), pos, state)
         lg = self.logits(x)
-        _, conf, tok, ent = softmax_stats(lg, self.mask_id)
+        if sampler is not None and sampler["temperature"] > 0:
+            noise = gumbel_noise(sampler["seed"], sampler["seq"], pos, sampler["step"], self.vocab)
+            conf, tok, ent = sample_stats(lg, self.mask_id, sampler["temperature"], noise)
+        else:
+            _, conf, tok, ent = softmax_stats(lg, self.mask_id)
         return lg, conf, tok, ent
 
     def denoise_step(self, state: SeqState, block_ids: np.ndarray, mask: np.ndarray, tau: float,
-                     mode: int = MODE_CONFIDENCE):
+                     mode: int = MODE_CONFIDENCE, sampler: Optional[Dict[str, object]] = None):
         """Forward + decision.  Returns (new_ids, new_mask, commit[bool B], conf, tok, entropy)."""
         block_ids = np.array(block_ids, dtype=np.int32, copy=True)
         mask = np.array(mask, dtype=bool, copy=True)
-        _, conf, tok, ent = self.denoise_forward(state, block_ids)
+        _, conf, tok, ent = self.denoise_forward(state, block_ids, sampler)
         commit = decide(conf, ent, mask, tau, mode)
         block_ids[commit] = tok[commit]
         mask[commit] = False
@@ -361,7 +439,8 @@ class OracleModel:
 
     def generate(self, prompt: np.ndarray, gen_len: int, block: int, tau: float,
                  mode: int = MODE_CONFIDENCE, record: bool = False,
-                 eos_id: Optional[int] = None, refresh_every: int = 0) -> Dict[str, object]:
+                 eos_id: Optional[int] = None, refresh_every: int = 0,
+                 temperature: float = 0.0, seed: int = 0, seq: int = 0) -> Dict[str, object]:
         """Block-by-block threshold decoding of one sequence.
 
         Returns tokens [gen_len], the step index (within its block, from 1) at which each
@@ -369,7 +448,9 @@ class OracleModel:
         ``eos_id`` decoding halts after the step that commits that id (Sec. 3.2, early
         stopping on EOS); undecoded positions stay ``mask_id``.  With ``refresh_every`` = r > 0
         the cache is refreshed (``refresh``) each time the number of stored blocks reaches a
-        multiple of r while blocks remain to be decoded (periodic KV-refresh, Sec. 3.2)."""
+        multiple of r while blocks remain to be decoded (periodic KV-refresh, Sec. 3.2).
+        ``temperature`` > 0 samples the tokens (``sample_stats``); the noise of a forward is
+        keyed by (seed; sequence index ``seq``, absolute position, step within the block)."""
         assert gen_len % block == 0
         state = self.prefill(prompt)
         n_refresh = 0
@@ -386,7 +467,8 @@ class OracleModel:
                 step += 1
                 assert step <= block, "each step must remove at least one mask"
                 ids_in, mask_in = ids.copy(), mask.copy()
-                ids, mask, commit, conf, tok, ent = self.denoise_step(state, ids, mask, tau, mode)
+                sampler = dict(temperature=temperature, seed=seed, seq=seq, step=step) if temperature > 0 else None
+                ids, mask, commit, conf, tok, ent = self.denoise_step(state, ids, mask, tau, mode, sampler)
                 n_denoise += 1
                 commit_step[j * block:(j + 1) * block][commit] = step
                 if record:
