@@ -346,6 +346,15 @@ def run_ours(args):
                   "decode_refresh_every_4_blocks": {"value": whole_job_tokens_per_s(world, tokens_of(w), args.steps, ms_rf), "unit": UNIT,
                                                     "refreshes_per_request": int(n_refresh)}}
 
+    # temperature sampling (Gumbel-max in the LM-head epilogue) on the same request
+    d3.d3_set_sampling(ctx, 0.1, 20260107)
+    step_resident()
+    ms_sm, st_sm = timed(step_resident, args.steps)
+    d3.d3_set_sampling(ctx, 0.0, 0)
+    sampling = {"temperature": 0.1, "value": whole_job_tokens_per_s(world, tokens_of(w), args.steps, ms_sm), "unit": UNIT,
+                "forwards_per_request": int(st_sm.steps),
+                "ms_per_forward": ms_sm / args.steps / max(int(st_sm.steps), 1)}
+
     # pseudo-trajectory extraction (threshold 1: one token per forward, full length) on the same request,
     # and the noisy-sequence builder on a training-sized batch of responses
     cs_dev = torch.zeros((w.batch, w.gen_len), dtype=torch.int32, device=dev)
@@ -444,7 +453,7 @@ def run_ours(args):
                    "tokens_per_forward_incl_finalize": tokens / max(st.denoise_forwards + st.finalize_forwards, 1),
                    "ms_per_forward": (ms_step - ms_prefill) / max(forwards, 1), "prefill_ms": ms_prefill,
                    "forced_commits": int(st.forced_commits)},
-        "multiblock": multiblock, "kv_refresh": kv_refresh, "trajectory": trajectory, "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
+        "multiblock": multiblock, "kv_refresh": kv_refresh, "trajectory": trajectory, "sampling": sampling, "kernels": per_class, "device_error_word": err_word, "weight_gen_s": round(t_gen, 1),
         "device_bytes": d3.d3_device_bytes(ctx),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

@@ -179,6 +179,19 @@ int d3_generate_multiblock(d3_ctx *ctx, int32_t gen_len, float threshold, int32_
 int d3_set_eos(d3_ctx *ctx, int32_t eos_id);
 int64_t d3_early_stops(d3_ctx *ctx);
 
+/* Temperature sampling (Appendix, inference settings: temperature 0.0 or 0.1).  With temperature T > 0
+ * the token of a row is drawn from softmax(l / T) by the Gumbel-max rule: the index of the largest
+ * l_v + T * g_v over the vocabulary without the mask token (float32, product and sum rounded
+ * separately, lowest index on ties), computed in the LM-head epilogue, logits never stored.  The
+ * confidence compared with the threshold is softmax(l) of the drawn token, the entropy that of
+ * softmax(l).  Noise: g = -ln(-ln u), u = (top 23 bits of a word + 1/2) * 2^-23; the word for
+ * vocabulary index v is word v % 4 of Philox-4x32-10 with counter (v / 4, absolute position of the
+ * row, step, sequence index in the batch) and key (low, high half of seed).  step: in d3_generate
+ * the 1-based denoise step within the sequence's current block; in d3_denoise_step the number of
+ * such calls since the last d3_prefill / d3_commit_block.  T = 0 (default) is greedy decoding.
+ * d3_generate_multiblock returns UNSUPPORTED while T > 0.  INVALID_ARG for negative or non-finite T. */
+int d3_set_sampling(d3_ctx *ctx, float temperature, uint64_t seed);
+
 /* Pseudo-trajectory extraction (Sec. 3.1): a d3_generate run with threshold 1 and no end-of-sequence
  * id unmasks exactly one token per step (no probability exceeds 1, so only the forced commit of the
  * most confident position happens) and decodes the full length; its commit_step output is the

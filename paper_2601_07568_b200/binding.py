@@ -27,7 +27,7 @@ EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
     "d3_get_state", "d3_set_state", "d3_op_linear", "d3_packed_weight_elems", "d3_pack_weight", "d3_op_linear_packed", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_generate_multiblock", "d3_refresh_cache", "d3_set_cache_policy", "d3_refresh_count", "d3_trajectory_rank", "d3_noisy_sequence", "d3_device_bytes",
+    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_generate_multiblock", "d3_refresh_cache", "d3_set_cache_policy", "d3_refresh_count", "d3_trajectory_rank", "d3_noisy_sequence", "d3_set_sampling", "d3_device_bytes",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
 
@@ -370,6 +370,10 @@ def d3_noisy_sequence(ctx, y: torch.Tensor, rank: torch.Tensor, s: torch.Tensor,
     _check(ctx, lib().d3_noisy_sequence(ctx, _ptr(_dev(y, torch.int32)), _ptr(_dev(rank, torch.int32)),
                                         _ptr(_dev(s, torch.int32)), _ptr(_dev(k, torch.int32)), _ptr(_dev(m, torch.int32)),
                                         C.c_int32(bs), C.c_int32(n), _ptr(_dev(out, torch.int32))))
+
+
+def d3_set_sampling(ctx, temperature: float = 0.0, seed: int = 0) -> None:
+    _check(ctx, lib().d3_set_sampling(ctx, C.c_float(temperature), C.c_uint64(seed)))
 
 
 def d3_refresh_cache(ctx, bs: int) -> None:

@@ -40,6 +40,17 @@ struct EpiParams {
   const float* ssq_in = nullptr; // any epilogue but EPI_RESID: chunk sums of the operand rows
   int ssq_chunks = 0;
   float inv_k = 0.f, rms_eps = 0.f;
+  // EPI_STATS with temperature sampling (sample_part != nullptr): per (row, 128-column tile) also the
+  // largest perturbed logit l + temperature * g (g standard Gumbel noise), the index attaining it
+  // (lowest on ties) and the unperturbed logit there.  The noise of row m is keyed by
+  // (seed; sequence m / rows_per_seq, position pos_base[sequence] + m % rows_per_seq, step).
+  float4* sample_part = nullptr;  // [m][n_tiles]: (perturbed max, logit at it, index bits, unused)
+  float temperature = 0.f;
+  uint32_t seed_lo = 0, seed_hi = 0;
+  const int* pos_base = nullptr;    // [sequences]
+  int rows_per_seq = 1;
+  const int* draw_step = nullptr;   // [sequences] step counter of each sequence (null: draw_step_add alone)
+  int draw_step_add = 0;
 };
 
 // Row factor of a matmul whose operand rows were left un-normalised; chunk sums added in index
@@ -60,6 +71,53 @@ __device__ __forceinline__ float row_rstd(const EpiParams& ep, int m) {
   }
   for (; i < ep.ssq_chunks; ++i) tot += __ldcg(r + i);
   return rsqrtf(tot * ep.inv_k + ep.rms_eps);
+}
+
+// Philox-4x32 with 10 rounds (Salmon et al., SC'11): a counter-based generator, four 32-bit words
+// per call, no state.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint32_t k0, uint32_t k1) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k0, lo1, hi0 ^ c.w ^ k1, lo0);
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  return c;
+}
+// Standard Gumbel noise from a 32-bit word: u = (top 23 bits + 1/2) * 2^-23 in (0, 1), g = -ln(-ln u).
+__device__ __forceinline__ float gumbel_from_bits(uint32_t x) {
+  const float u = (static_cast<float>(x >> 9) + 0.5f) * 1.1920928955078125e-07f;
+  return -logf(-logf(u));
+}
+// Sampling nonce of matmul row m: counter words 1..3 = (position, step, sequence).
+struct SampleRow {
+  uint32_t pos, step, seq;
+};
+__device__ __forceinline__ SampleRow sample_row(const EpiParams& ep, int m) {
+  const int b = m / ep.rows_per_seq;
+  SampleRow r;
+  r.seq = static_cast<uint32_t>(b);
+  r.pos = static_cast<uint32_t>((ep.pos_base ? ep.pos_base[b] : 0) + m % ep.rows_per_seq);
+  r.step = static_cast<uint32_t>((ep.draw_step ? ep.draw_step[b] : 0) + ep.draw_step_add);
+  return r;
+}
+// Running maximum of the perturbed logits: pm = max, la = logit at it, pa = lowest index attaining it.
+struct SampleStat {
+  float pm, la;
+  int pa;
+};
+__device__ __forceinline__ SampleStat sample_empty() { return SampleStat{-INFINITY, 0.f, 0x7fffffff}; }
+__device__ __forceinline__ void sample_add(SampleStat& st, float pert, float l, int idx) {
+  if (pert > st.pm || (pert == st.pm && idx < st.pa)) {
+    st.pm = pert;
+    st.la = l;
+    st.pa = idx;
+  }
+}
+__device__ __forceinline__ SampleStat sample_merge(const SampleStat& a, const SampleStat& b) {
+  return (b.pm > a.pm || (b.pm == a.pm && b.pa < a.pa)) ? b : a;
 }
 
 template <typename T> struct TypeOps;

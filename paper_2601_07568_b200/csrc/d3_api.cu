@@ -91,6 +91,12 @@ struct d3_ctx {
   int tune_no_rr = 0;     // 1: wide matmuls on contiguous unit ranges
   int eos_id = -1;        // d3_generate stops a sequence once this id has been committed (< 0: never)
   long long last_early_stops = 0;
+  float4* sample_part = nullptr;  // per (row, tile) sampling partials (temperature > 0)
+  float temperature = 0.f;        // 0: greedy
+  unsigned long long seed = 0;
+  const int* draw_step = nullptr; // device step counters of the sequences for the next forward's noise (null: draw_step_add alone)
+  int draw_step_add = 1;
+  int explicit_step = 0;          // d3_denoise_step calls since the last prefill / commit
   int* hist_ids = nullptr;     // [max_batch, max_seq] ids of the stored prefix of every sequence
   int* refresh_ids = nullptr;  // [max_rows] input ids of a KV-refresh forward
   int cache_delay = 1;         // multi-block decoding: stabilizing rounds before a complete block is stored
@@ -743,8 +749,14 @@ int run_rmsnorm(d3_ctx* c, const float* x, const float* gain, void* xn, int M) {
   return D3_OK;
 }
 
-int run_stats_merge(d3_ctx* c, int M, int n_tiles, float* conf, float* ent, int* argmax) {
+int run_stats_merge(d3_ctx* c, int M, int n_tiles, float* conf, float* ent, int* argmax, bool sampled = false) {
   ProfScope ps(c, D3_PROF_OTHER);
+  if (sampled) {
+    CUDA_TRY(c, launch_pdl(c, stats_merge_sample_kernel, dim3((M + 3) / 4), dim3(128), 0, static_cast<const float4*>(c->stat_part),
+                           static_cast<const float4*>(c->sample_part), n_tiles, M, conf, ent, argmax));
+    LAUNCHED(c, "stats_merge_sample_kernel");
+    return D3_OK;
+  }
   CUDA_TRY(c, launch_pdl(c, stats_merge_kernel, dim3((M + 3) / 4), dim3(128), 0, static_cast<const float4*>(c->stat_part), n_tiles, M, conf, ent, argmax));
   LAUNCHED(c, "stats_merge_kernel");
   return D3_OK;
@@ -836,9 +848,20 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     const int n_tiles = (g.vocab + 127) / 128;
     EpiParams ep;
     ep.scale = g.logit_scale; ep.mask_id = g.mask_id; ep.stat_part = c->stat_part; ep.n_tiles = n_tiles;
+    const bool sampled = c->temperature > 0.f;
+    if (sampled) {  // temperature sampling: Gumbel noise keyed by (seed; sequence, position, step)
+      ep.sample_part = c->sample_part;
+      ep.temperature = c->temperature;
+      ep.seed_lo = static_cast<uint32_t>(c->seed & 0xffffffffull);
+      ep.seed_hi = static_cast<uint32_t>(c->seed >> 32);
+      ep.pos_base = c->pos_base;
+      ep.rows_per_seq = rows_per_seq;
+      ep.draw_step = c->draw_step;
+      ep.draw_step_add = c->draw_step_add;
+    }
     after_norm(ep);
     TRY(run_linear(c, normed, c->lm_head, M, g.vocab, d, EPI_STATS, ep, 0, nullptr, D3_PROF_GEMM_HEAD, c->w_tiled));
-    TRY(run_stats_merge(c, M, n_tiles, c->conf, c->ent, c->argmax));
+    TRY(run_stats_merge(c, M, n_tiles, c->conf, c->ent, c->argmax, sampled));
   } else {
     EpiParams ep;
     ep.y = logits; ep.ldy = g.vocab; ep.scale = g.logit_scale;
@@ -934,6 +957,7 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   A_(c->h, c->esz * R * f);
   const size_t n_tiles = (g.vocab + 127) / 128;
   A_(c->stat_part, sizeof(float4) * static_cast<size_t>(dec_rows) * n_tiles);
+  A_(c->sample_part, sizeof(float4) * static_cast<size_t>(dec_rows) * n_tiles);
   A_(c->conf, sizeof(float) * dec_rows);
   A_(c->ent, sizeof(float) * dec_rows);
   A_(c->argmax, sizeof(int) * dec_rows);
@@ -1174,6 +1198,7 @@ extern "C" int d3_prefill(d3_ctx* c, const int32_t* prompt_ids, const int32_t* p
     LAUNCHED(c, "hist_store_kernel");
   }
   c->prefilled = true;
+  c->explicit_step = 0;
   return D3_OK;
 }
 
@@ -1222,6 +1247,8 @@ extern "C" int d3_denoise_step(d3_ctx* c, int32_t* block_ids, uint8_t* mask, flo
   const int B = c->cfg.block;
   decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B, c->pos_base, c->n_valid, c->kv_len);
   LAUNCHED(c, "decode_rowmap_kernel");
+  c->draw_step = nullptr;  // sampling noise of the explicit calls: steps counted since the last prefill / commit
+  c->draw_step_add = ++c->explicit_step;
   TRY(forward(c, block_ids, bs, B, 1, nullptr));
   unmask_kernel<<<bs, 32, 0, c->stream>>>(c->conf, c->ent, c->argmax, block_ids, mask, B, threshold, c->cfg.decide_mode, out_pos, out_ids, out_count);
   LAUNCHED(c, "unmask_kernel");
@@ -1241,6 +1268,7 @@ extern "C" int d3_commit_block(d3_ctx* c, const int32_t* block_ids, int32_t bs) 
   LAUNCHED(c, "hist_store_kernel");
   add_prefix_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, B);
   LAUNCHED(c, "add_prefix_kernel");
+  c->explicit_step = 0;
   return D3_OK;
 }
 
@@ -1270,6 +1298,8 @@ extern "C" int d3_generate(d3_ctx* c, int32_t gen_len, float threshold, int32_t 
   const int fuse = (c->gen_fuse && c->refresh_every == 0 && 2ll * bs * B <= FUSE_MAX_ROWS && 2ll * c->cfg.max_batch * B <= FUSE_MAX_ROWS) ? 1 : 0;
   long long steps = 0;
   c->last_refreshes = 0;
+  c->draw_step = g.step;  // sampling noise: each sequence's step within its block (the counter is bumped after the forward)
+  c->draw_step_add = 1;
   int R = B;  // rows per sequence of the next forward: 2B while some sequence runs a fused finalize + first step
   for (long long it = 0; it < max_iter; ++it) {
     gen_rowmap_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, R, c->cfg.mask_id, c->pos_base, c->n_valid, c->kv_len);
@@ -1308,6 +1338,7 @@ extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshol
   if (!out_ids || bs <= 0 || gen_len <= 0 || std::isnan(threshold) || max_active < 1 || max_active > MB_MAX_WINDOW)
     return fail(c, D3_ERR_INVALID_ARG, "bad generate_multiblock arguments");
   if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_generate_multiblock before d3_prefill");
+  if (c->temperature > 0.f) return fail(c, D3_ERR_UNSUPPORTED, "temperature sampling is not available in multi-block decoding");
   const int B = c->cfg.block;
   if (bs > c->cfg.max_batch || gen_len % B != 0) return fail(c, D3_ERR_SHAPE, "bs > max_batch or gen_len not a multiple of the block size");
   if (static_cast<long long>(bs) * max_active * B > std::min<long long>(c->stat_rows, c->max_rows))
@@ -1378,6 +1409,14 @@ extern "C" int d3_noisy_sequence(d3_ctx* c, const int32_t* y, const int32_t* ran
   if (bs > 65535) return fail(c, D3_ERR_SHAPE, "more than 65535 sequences in one call");
   noisy_sequence_kernel<<<dim3((n + 255) / 256, bs), 256, 0, c->stream>>>(y, rank, s, k, m, n, c->cfg.mask_id, out);
   LAUNCHED(c, "noisy_sequence_kernel");
+  return D3_OK;
+}
+
+extern "C" int d3_set_sampling(d3_ctx* c, float temperature, uint64_t seed) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!(temperature >= 0.f) || !std::isfinite(temperature)) return fail(c, D3_ERR_INVALID_ARG, "temperature must be finite and >= 0");
+  c->temperature = temperature;
+  c->seed = seed;
   return D3_OK;
 }
 

@@ -98,6 +98,29 @@ __global__ void __launch_bounds__(THREADS) gemm_simt_kernel(const T* __restrict_
       if (lane == 0 && m < M)
         ep.stat_part[static_cast<size_t>(m) * ep.n_tiles + blockIdx.x] =
             make_float4(st.m, st.z, st.s, __int_as_float(st.a));
+      if (ep.sample_part != nullptr && m < M) {  // temperature sampling: largest l + T * g of the tile
+        SampleStat sp = sample_empty();
+        const SampleRow sr = sample_row(ep, m);
+        for (int c = lane; c < BN; c += 32) {
+          const int n = n0 + c;
+          if (n < N && n != ep.mask_id) {
+            const uint4 bits = philox4x32_10(make_uint4(static_cast<uint32_t>(n >> 2), sr.pos, sr.step, sr.seq), ep.seed_lo, ep.seed_hi);
+            const uint32_t w = (n & 3) == 0 ? bits.x : (n & 3) == 1 ? bits.y : (n & 3) == 2 ? bits.z : bits.w;
+            const float l = Cs[r][c] * ep.scale;
+            sample_add(sp, __fadd_rn(l, __fmul_rn(ep.temperature, gumbel_from_bits(w))), l, n);
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+          SampleStat other;
+          other.pm = __shfl_xor_sync(0xffffffffu, sp.pm, o);
+          other.la = __shfl_xor_sync(0xffffffffu, sp.la, o);
+          other.pa = __shfl_xor_sync(0xffffffffu, sp.pa, o);
+          sp = sample_merge(sp, other);
+        }
+        if (lane == 0)
+          ep.sample_part[static_cast<size_t>(m) * ep.n_tiles + blockIdx.x] = make_float4(sp.pm, sp.la, __int_as_float(sp.pa), 0.f);
+      }
     }
   }
 }

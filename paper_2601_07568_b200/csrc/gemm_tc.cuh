@@ -284,6 +284,31 @@ __device__ __forceinline__ void run_epilogue(const Source& src, const GemmParams
       int t = (n0 + g) / 128;
       if (live && t < p.ep.n_tiles)
         p.ep.stat_part[static_cast<size_t>(m) * p.ep.n_tiles + t] = make_float4(st.m, st.z, st.s, __int_as_float(st.a));
+      if (p.ep.sample_part != nullptr) {
+        // temperature sampling: a second pass over the tile for the largest l + T * g; one Philox
+        // call per four consecutive columns (the chunks start at multiples of 32)
+        SampleStat sp = sample_empty();
+        const SampleRow sr = live ? sample_row(p.ep, m) : SampleRow{0u, 0u, 0u};
+        for (int c = 0; c < 128; c += 32) {
+          if (n0 + g + c >= N) break;
+          float v[32];
+          src.load(g + c, v);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            const int nq = n0 + g + c + 4 * q;
+            const uint4 bits = philox4x32_10(make_uint4(static_cast<uint32_t>(nq >> 2), sr.pos, sr.step, sr.seq), p.ep.seed_lo, p.ep.seed_hi);
+            const uint32_t w[4] = {bits.x, bits.y, bits.z, bits.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int n = nq + j;
+              const float l = v[4 * q + j] * (p.ep.scale * rs);
+              if (n < N && n != p.ep.mask_id) sample_add(sp, __fadd_rn(l, __fmul_rn(p.ep.temperature, gumbel_from_bits(w[j]))), l, n);  // no contraction: product and sum rounded separately
+            }
+          }
+        }
+        if (live && t < p.ep.n_tiles)
+          p.ep.sample_part[static_cast<size_t>(m) * p.ep.n_tiles + t] = make_float4(sp.pm, sp.la, __int_as_float(sp.pa), 0.f);
+      }
     }
   } else if constexpr (EPI == EPI_QKV) {
     // d_head = 128.  Packed rows of W inside a q or k head: 2i = dim i, 2i+1 = dim i+64 (a RoPE pair);

@@ -223,6 +223,51 @@ __global__ void stats_merge_kernel(const float4* __restrict__ part, int n_tiles,
   }
 }
 
+// The same with temperature sampling: the token is the index of the largest perturbed logit over all
+// tiles (lowest index on ties) and the confidence its probability e^(l - m) / Z under the unperturbed
+// softmax; the entropy is unchanged.
+__global__ void stats_merge_sample_kernel(const float4* __restrict__ part, const float4* __restrict__ sample_part, int n_tiles,
+                                          int M, float* __restrict__ conf, float* __restrict__ entropy, int* __restrict__ argmax) {
+  ptx::grid_dep_wait();
+  ptx::grid_dep_launch();
+  const int m = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (m >= M) return;
+  SoftStat st = stat_empty();
+  SampleStat sp = sample_empty();
+  for (int t = lane; t < n_tiles; t += 32) {
+    const float4 v = part[static_cast<size_t>(m) * n_tiles + t];
+    st = stat_merge(st, SoftStat{v.x, v.y, v.z, __float_as_int(v.w)});
+    const float4 w = sample_part[static_cast<size_t>(m) * n_tiles + t];
+    sp = sample_merge(sp, SampleStat{w.x, w.y, __float_as_int(w.z)});
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    SoftStat other;
+    other.m = __shfl_xor_sync(0xffffffffu, st.m, o);
+    other.z = __shfl_xor_sync(0xffffffffu, st.z, o);
+    other.s = __shfl_xor_sync(0xffffffffu, st.s, o);
+    other.a = __shfl_xor_sync(0xffffffffu, st.a, o);
+    st = (lane & o) ? stat_merge(other, st) : stat_merge(st, other);
+    SampleStat so;
+    so.pm = __shfl_xor_sync(0xffffffffu, sp.pm, o);
+    so.la = __shfl_xor_sync(0xffffffffu, sp.la, o);
+    so.pa = __shfl_xor_sync(0xffffffffu, sp.pa, o);
+    sp = sample_merge(sp, so);
+  }
+  if (lane == 0) {
+    if (st.z > 0.f && sp.pa != 0x7fffffff) {
+      conf[m] = fminf(expf(sp.la - st.m) / st.z, 1.0f);
+      entropy[m] = fmaxf(logf(st.z) - st.s / st.z, 0.f);
+      argmax[m] = sp.pa;
+    } else {
+      conf[m] = 0.f;
+      entropy[m] = 0.f;
+      argmax[m] = 0;
+    }
+  }
+}
+
 // Statistics straight from fp32 logits rows (SIMT path and tests): one block per row.
 __global__ void stats_from_logits_kernel(const float* __restrict__ logits, int V, int mask_id, float4* __restrict__ part,
                                          int n_tiles) {
