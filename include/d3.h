@@ -175,7 +175,9 @@ int d3_generate_multiblock(d3_ctx *ctx, int32_t gen_len, float threshold, int32_
  * block.  The block goes out as it stands, undecoded positions (there and in all later blocks) read
  * mask_id, the unfinished block is not added to the cache, and tokens_committed counts what was
  * decoded.  eos_id < 0 switches it off (the default).  INVALID_ARG for ids outside the vocabulary or
- * equal to mask_id.  d3_early_stops: sequences of the latest d3_generate call that stopped this way. */
+ * equal to mask_id.  d3_generate_multiblock stops a sequence after the round that commits the id in any
+ * block in flight: all blocks in flight go out as they stand and none of them is added to the cache.
+ * d3_early_stops: sequences of the latest generate call that stopped this way. */
 int d3_set_eos(d3_ctx *ctx, int32_t eos_id);
 int64_t d3_early_stops(d3_ctx *ctx);
 
@@ -189,7 +191,7 @@ int64_t d3_early_stops(d3_ctx *ctx);
  * row, step, sequence index in the batch) and key (low, high half of seed).  step: in d3_generate
  * the 1-based denoise step within the sequence's current block; in d3_denoise_step the number of
  * such calls since the last d3_prefill / d3_commit_block.  T = 0 (default) is greedy decoding.
- * d3_generate_multiblock returns UNSUPPORTED while T > 0.  INVALID_ARG for negative or non-finite T. */
+ * In d3_generate_multiblock the step is the round.  INVALID_ARG for negative or non-finite T. */
 int d3_set_sampling(d3_ctx *ctx, float temperature, uint64_t seed);
 
 /* Pseudo-trajectory extraction (Sec. 3.1): a d3_generate run with threshold 1 and no end-of-sequence

@@ -497,7 +497,8 @@ class OracleModel:
 
     def generate_multiblock(self, prompt: np.ndarray, gen_len: int, block: int, tau: float,
                             mode: int = MODE_ENTROPY, max_active: int = 2, record: bool = False,
-                            cache_delay: int = 1, refresh_every: int = 0) -> Dict[str, object]:
+                            cache_delay: int = 1, refresh_every: int = 0, eos_id: Optional[int] = None,
+                            temperature: float = 0.0, seed: int = 0, seq: int = 0) -> Dict[str, object]:
         """Multi-block decoding of one sequence (Sec. 3.2, multi-block decoding strategy).
 
         Every round is one forward over the blocks in flight (oldest first), each seeing the
@@ -506,7 +507,11 @@ class OracleModel:
         number of rounds, the rows each round covered, and optionally a per-round trace.
         ``cache_delay``: stabilizing rounds a complete block goes through before its K/V are
         stored (1 or 2 in the paper's settings).  ``refresh_every`` = r > 0: after every r-th
-        round the stored cache is refreshed (``refresh``) while blocks are still in flight."""
+        round the stored cache is refreshed (``refresh``) while blocks are still in flight.
+        ``eos_id``: decoding halts after the round that commits that id in any block in flight;
+        the blocks in flight go out as they stand (masked positions as ``mask_id``) and are not
+        stored.  ``temperature`` > 0 samples the tokens; the noise of a round is keyed by (seed;
+        ``seq``, absolute position, round)."""
         assert gen_len % block == 0 and max_active >= 1 and cache_delay >= 1
         n_blocks = gen_len // block
         state = self.prefill(prompt)
@@ -518,6 +523,7 @@ class OracleModel:
         win_stab: List[int] = [0]                # stabilizing forwards each block in flight has had
         rounds = 0
         n_refresh = 0
+        stopped = False
         rows: List[int] = []
         trace: List[Dict[str, object]] = []
         while win_ids:
@@ -534,8 +540,9 @@ class OracleModel:
             # the forward: block w sees the cache and blocks 0..w-1 of the window
             tmp = state
             stats = []
+            sampler = dict(temperature=temperature, seed=seed, seq=seq, step=rounds) if temperature > 0 else None
             for w in range(n_win):
-                _, conf, tok, ent = self.denoise_forward(tmp, win_ids[w])
+                _, conf, tok, ent = self.denoise_forward(tmp, win_ids[w], sampler)
                 stats.append((conf, tok, ent))
                 if w + 1 < n_win:
                     tmp = self.finalize_block(tmp, win_ids[w])
@@ -559,6 +566,11 @@ class OracleModel:
                 trace.append(dict(round=rounds, lo=lo, n_win=n_win, fully=list(fully), ids_in=ids_in, mask_in=mask_in,
                                   complete_before=list(complete_before), stats=stats, commits=commits,
                                   ids_out=[a.copy() for a in win_ids], mask_out=[a.copy() for a in win_mask]))
+            if eos_id is not None and any(np.any(win_ids[w][commits[w]] == eos_id) for w in range(n_win)):
+                for w in range(n_win):   # early stop: everything in flight goes out as it stands
+                    out[(lo + w) * block:(lo + w + 1) * block] = np.where(win_mask[w], self.mask_id, win_ids[w])
+                stopped = True
+                break
             # blocks that were complete before this forward have had a stabilizing round: the
             # oldest ones enter the cache, in order, once they have had cache_delay of them
             for w in range(n_win):
@@ -580,7 +592,7 @@ class OracleModel:
                 state = self.refresh(state)
                 n_refresh += 1
         res = dict(tokens=out, commit_round=commit_round, rounds=rounds, rows=rows, state=state,
-                   n_refresh=n_refresh,
+                   n_refresh=n_refresh, stopped_early=stopped,
                    tokens_per_round=gen_len / max(rounds, 1))
         if record:
             res["trace"] = trace

@@ -1338,7 +1338,6 @@ extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshol
   if (!out_ids || bs <= 0 || gen_len <= 0 || std::isnan(threshold) || max_active < 1 || max_active > MB_MAX_WINDOW)
     return fail(c, D3_ERR_INVALID_ARG, "bad generate_multiblock arguments");
   if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_generate_multiblock before d3_prefill");
-  if (c->temperature > 0.f) return fail(c, D3_ERR_UNSUPPORTED, "temperature sampling is not available in multi-block decoding");
   const int B = c->cfg.block;
   if (bs > c->cfg.max_batch || gen_len % B != 0) return fail(c, D3_ERR_SHAPE, "bs > max_batch or gen_len not a multiple of the block size");
   if (static_cast<long long>(bs) * max_active * B > std::min<long long>(c->stat_rows, c->max_rows))
@@ -1366,13 +1365,15 @@ extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshol
   for (long long it = 0; it < max_iter; ++it) {
     mb_rowmap_kernel<<<bs, 64, 0, c->stream>>>(g, bs, B, W, R, c->cfg.mask_id, c->pos_base, c->n_valid, c->kv_len);
     LAUNCHED(c, "mb_rowmap_kernel");
+    c->draw_step = nullptr;  // sampling noise of a round: keyed by the round
+    c->draw_step_add = static_cast<int>(rounds + 1);
     TRY(forward(c, g.fwd_ids, bs, R, 1, nullptr, B));
     ++rounds;
     mb_advance_kernel<<<bs, 32, 0, c->stream>>>(g, c->conf, c->ent, c->argmax, bs, B, W, R, n_blocks, gen_len, threshold,
                                                 c->cfg.decide_mode, c->cfg.mask_id, max_active, static_cast<int>(rounds), c->cache_delay,
-                                                c->cfg.max_seq);
+                                                c->cfg.max_seq, c->eos_id);
     LAUNCHED(c, "mb_advance_kernel");
-    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 7, cudaMemcpyDeviceToHost, c->stream));
+    CUDA_TRY(c, cudaMemcpyAsync(c->host_counters, g.counters, sizeof(long long) * 8, cudaMemcpyDeviceToHost, c->stream));
     CUDA_TRY(c, cudaStreamSynchronize(c->stream));
     if (c->host_counters[4] <= 0) break;
     if (c->refresh_every > 0 && rounds % c->refresh_every == 0) {  // periodic KV-refresh of the sequences still decoding
@@ -1390,6 +1391,7 @@ extern "C" int d3_generate_multiblock(d3_ctx* c, int32_t gen_len, float threshol
     host_stats->steps = rounds;
     host_stats->kernel_launches = c->launches - launches0;
   }
+  c->last_early_stops = c->host_counters[7];
   if (c->host_counters[4] > 0) return fail(c, D3_ERR_STATE, "multi-block loop did not finish within its round bound");
   return check_device_error(c);
 }

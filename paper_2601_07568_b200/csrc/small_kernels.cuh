@@ -560,7 +560,8 @@ struct MbState {
   int* out_ids;     // [bs, gen_len]
   int* commit_round;  // [bs, gen_len] or null
   long long* counters;  // [0] block decisions taken, [1] blocks stored in the cache, [2] tokens, [3] forced commits,
-                        // [4] sequences not done, [5] largest window of the next round, [6] rows of valid work so far
+                        // [4] sequences not done, [5] largest window of the next round, [6] rows of valid work so far,
+                        // [7] sequences stopped early on the end-of-sequence id
   int* stab;            // [bs, W] stabilizing forwards each block in flight has had
   int* hist;            // [bs, max_seq] ids of the stored prefix
 };
@@ -608,7 +609,7 @@ __global__ void mb_rowmap_kernel(MbState g, int bs, int B, int W, int R, int mas
 __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, const float* __restrict__ ent,
                                   const int* __restrict__ argmax, int bs, int B, int W, int R, int n_blocks, int gen_len,
                                   float tau, int decide_mode, int mask_id, int max_active, int round, int cache_delay,
-                                  int max_seq) {
+                                  int max_seq, int eos_id) {
   const int b = blockIdx.x;
   const int lane = threadIdx.x & 31;
   int n = g.n_win[b];
@@ -633,6 +634,16 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
       unmasked[w] = cnt;
     }
   }
+  // positions masked before the decisions (bit w * 4 + q = position lane + 32 q of block w): what is
+  // unmasked afterwards was committed in this round
+  unsigned was_masked = 0;
+  if (eos_id >= 0) {
+#pragma unroll
+    for (int w = 0; w < MB_MAX_WINDOW; ++w)
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (w < n && lane + 32 * q < B && mask[w * B + lane + 32 * q] != 0) was_masked |= 1u << (w * 4 + q);
+  }
   long long committed = 0, forced = 0, decisions = 0;
 #pragma unroll
   for (int w = 0; w < MB_MAX_WINDOW; ++w) {
@@ -648,6 +659,32 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
     }
   }
   __syncwarp();
+  // early stop: the end-of-sequence id was committed in this round.  Everything in flight goes out as
+  // it stands (mask id where nothing was decided) and is not stored; the sequence is done.
+  if (eos_id >= 0) {
+    bool hit = false;
+#pragma unroll
+    for (int w = 0; w < MB_MAX_WINDOW; ++w)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int pos = w * B + lane + 32 * q;
+        if ((was_masked >> (w * 4 + q)) & 1u)
+          if (mask[pos] == 0 && ids[pos] == eos_id) hit = true;
+      }
+    if (__any_sync(0xffffffffu, hit)) {
+      for (int r = lane; r < n * B; r += 32)
+        g.out_ids[static_cast<size_t>(b) * gen_len + lo * B + r] = mask[r] ? mask_id : ids[r];
+      if (lane == 0) {
+        g.n_win[b] = 0;
+        atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[0]), static_cast<unsigned long long>(decisions));
+        atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[2]), static_cast<unsigned long long>(committed));
+        atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[3]), static_cast<unsigned long long>(forced));
+        atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[4]), static_cast<unsigned long long>(-1ll));
+        atomicAdd(reinterpret_cast<unsigned long long*>(&g.counters[7]), 1ull);
+      }
+      return;
+    }
+  }
   // blocks that were complete before this forward have had one more stabilizing round; the leading
   // ones that have had cache_delay of them go out and into the cache
 #pragma unroll

@@ -328,6 +328,40 @@ def test_multiblock_decoding_fp32_equals_the_oracle(tau, mode):
             ctx.generate_multiblock(1, 64, tau, 0)
 
 
+def test_multiblock_stops_on_eos_like_the_oracle():
+    """Early stop in multi-block decoding: fp32 batch of three, the EOS id a token that sequence 0 commits
+    in a middle round; sequences that commit it halt after that round with their blocks in flight written
+    out as they stand, the others run on.  Tokens, commit rounds and counts equal the oracle's."""
+    shape = si.TINY
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("mb-eos", shape, 3, [32, 11, 20], 64, 16, 0.3, 41)
+    model = o.model_from_shape(shape, W, np.float64)
+    free = model.generate_multiblock(ids[0, :lens[0]], 64, 16, 0.3, 0, max_active=3, record=True)
+    seen, eos = set(), None
+    for t in free["trace"]:
+        toks = [int(x) for k in range(t["n_win"]) for x in t["ids_out"][k][t["commits"][k]]]
+        fresh = [x for x in toks if x not in seen]
+        if t["round"] >= 2 and fresh and t["round"] < free["rounds"] - 1:
+            eos = fresh[0]
+        seen.update(toks)
+    assert eos is not None
+    ref = [model.generate_multiblock(ids[b, :lens[b]], 64, 16, 0.3, 0, max_active=3, eos_id=eos) for b in range(3)]
+    assert ref[0]["stopped_early"]
+    with Ctx(shape, W, block=16, max_batch=12, max_seq=wl.max_seq) as ctx:
+        d3.d3_set_eos(ctx.ctx, eos)
+        ctx.prefill(ids, lens)
+        tok, cr, st = ctx.generate_multiblock(3, 64, 0.3, 3)
+        for b in range(3):
+            assert np.array_equal(tok[b], ref[b]["tokens"]), b
+            live = ref[b]["tokens"] != shape.mask_id
+            assert np.array_equal(cr[b][live], ref[b]["commit_round"][live]), b
+        assert st.steps == max(r["rounds"] for r in ref)
+        assert st.tokens_committed == sum(int((r["tokens"] != shape.mask_id).sum()) for r in ref)
+        assert d3.d3_early_stops(ctx.ctx) == sum(int(r["stopped_early"]) for r in ref) >= 1
+        assert np.array_equal(ctx.get_prefix(3), [r["state"].prefix_len for r in ref]) and ctx.error_word() == 0
+        d3.d3_set_eos(ctx.ctx, -1)
+
+
 def test_multiblock_decoding_bf16_tensor_core():
     """The same through the tensor-core kernels at batch 1 (forwards of 32 to 128 rows, up to four
     segments): against the oracle with mirrored bf16 roundings; ids may differ only where the oracle

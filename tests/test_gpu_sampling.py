@@ -74,10 +74,25 @@ def test_generate_with_temperature_fp32_equals_the_oracle(T):
             assert np.array_equal(tok0[b], greedy[b]["tokens"])
         with pytest.raises(d3.D3Error):
             d3.d3_set_sampling(ctx.ctx, -1.0, 0)
-        d3.d3_set_sampling(ctx.ctx, 0.3, 1)
-        ctx.prefill(ids, lens)
-        with pytest.raises(d3.D3Error):
-            ctx.generate_multiblock(3, 64, 0.9, 2)
+
+
+def test_multiblock_with_temperature_fp32_equals_the_oracle():
+    """Multi-block decoding with sampling (noise keyed by the round) on a ragged fp32 batch, windows of 2
+    and 4 blocks: tokens, commit rounds and round counts equal the oracle's."""
+    shape = si.TINY
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("sample-mb", shape, 3, [32, 9, 21], 64, 16, 0.3, 77)
+    model = o.model_from_shape(shape, W, np.float64)
+    with Ctx(shape, W, block=16, max_batch=12, max_seq=wl.max_seq) as ctx:
+        for max_active, T, seed in [(2, 0.5, 99), (4, 0.2, (5 << 32) + 1)]:
+            ref = [model.generate_multiblock(ids[b, :lens[b]], 64, 16, 0.3, 0, max_active=max_active, temperature=T, seed=seed, seq=b)
+                   for b in range(3)]
+            d3.d3_set_sampling(ctx.ctx, T, seed)
+            ctx.prefill(ids, lens)
+            tok, cr, st = ctx.generate_multiblock(3, 64, 0.3, max_active)
+            exact = sum(int(np.array_equal(tok[b], ref[b]["tokens"]) and np.array_equal(cr[b], ref[b]["commit_round"])) for b in range(3))
+            print("multi-block sampling, window", max_active, "sequences bit-equal to the oracle:", exact, "of 3")
+            assert exact == 3 and st.steps == max(r["rounds"] for r in ref) and ctx.error_word() == 0
 
 
 def _check_step_against_own_logits(ctx, shape, ids, lens, B, T, seed, n_steps, tol_gap):

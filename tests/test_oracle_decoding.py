@@ -406,3 +406,57 @@ def test_multiblock_rounds_follow_the_state_rules_and_the_joint_forward_is_block
                 assert nxt["mask_in"][-1].all()
     assert checked_joint >= 1
     assert np.array_equal(np.concatenate(cached + [x for x in tr[-1]["ids_out"]])[:w.gen_len], res["tokens"])
+
+
+def test_multiblock_eos_stop_is_a_prefix_of_the_free_run_and_window_one_is_single_block():
+    """Early stop in multi-block decoding: with the EOS id set to a token first committed in round k (k > 1)
+    of the free run, the run makes the same commits up to and including round k and then halts: the
+    blocks in flight go out as they stood after that round, nothing later is decoded.  With one block in
+    flight it is the early stop of block-by-block decoding."""
+    w, model, prompt = _c1_model()
+    B = w.block
+    free = model.generate_multiblock(prompt, w.gen_len, B, 0.3, o.MODE_CONFIDENCE, max_active=3, record=True)
+    seen, pick = set(), None
+    for t in free["trace"]:
+        toks = [int(x) for k in range(t["n_win"]) for x in t["ids_out"][k][t["commits"][k]]]
+        fresh = [x for x in toks if x not in seen]
+        if t["round"] >= 2 and fresh and t["round"] < free["rounds"] - 1:
+            pick = (t, fresh[0])
+        seen.update(toks)
+    assert pick is not None
+    t, eos = pick
+    got = model.generate_multiblock(prompt, w.gen_len, B, 0.3, o.MODE_CONFIDENCE, max_active=3, eos_id=eos)
+    assert got["stopped_early"] and got["rounds"] == t["round"] < free["rounds"]
+    want = np.full(w.gen_len, w.model.mask_id, dtype=np.int32)
+    want[:t["lo"] * B] = free["tokens"][:t["lo"] * B]
+    for k in range(t["n_win"]):
+        want[(t["lo"] + k) * B:(t["lo"] + k + 1) * B] = np.where(t["mask_out"][k], w.model.mask_id, t["ids_out"][k])
+    assert np.array_equal(got["tokens"], want) and np.any(got["tokens"] == eos)
+    assert np.array_equal(got["commit_round"][got["tokens"] != w.model.mask_id] <= t["round"], np.ones(int((got["tokens"] != w.model.mask_id).sum()), bool))
+    assert got["state"].prefix_len == len(prompt) + t["lo"] * B        # nothing in flight was stored
+    # one block in flight: the same tokens as the single-block early stop
+    one = model.generate(prompt, w.gen_len, B, 0.3, eos_id=eos)
+    mb1 = model.generate_multiblock(prompt, w.gen_len, B, 0.3, o.MODE_CONFIDENCE, max_active=1, eos_id=eos)
+    assert one["stopped_early"] and mb1["stopped_early"] and np.array_equal(one["tokens"], mb1["tokens"])
+
+
+def test_multiblock_sampling_with_one_block_in_flight_draws_per_round():
+    """Sampling in multi-block decoding keys the noise by the round; the run is reproducible, depends on
+    the seed, and at temperature 0 is the greedy run."""
+    w, model, prompt = _c1_model()
+    B = w.block
+    greedy = model.generate_multiblock(prompt, w.gen_len, B, 0.9, o.MODE_CONFIDENCE, max_active=2)
+    zero = model.generate_multiblock(prompt, w.gen_len, B, 0.9, o.MODE_CONFIDENCE, max_active=2, temperature=0.0, seed=5)
+    assert np.array_equal(greedy["tokens"], zero["tokens"])
+    a = model.generate_multiblock(prompt, w.gen_len, B, 0.9, o.MODE_CONFIDENCE, max_active=2, temperature=0.6, seed=5, record=True)
+    b = model.generate_multiblock(prompt, w.gen_len, B, 0.9, o.MODE_CONFIDENCE, max_active=2, temperature=0.6, seed=5)
+    c = model.generate_multiblock(prompt, w.gen_len, B, 0.9, o.MODE_CONFIDENCE, max_active=2, temperature=0.6, seed=6)
+    assert np.array_equal(a["tokens"], b["tokens"]) and not np.array_equal(a["tokens"], c["tokens"])
+    assert not np.array_equal(a["tokens"], greedy["tokens"])
+    # the recorded tokens of a round are the Gumbel-max draws for (seed, position, round) from that round's logits
+    t = a["trace"][0]
+    st = model.prefill(prompt)
+    lg, *_ = model.denoise_forward(st, t["ids_in"][0])
+    noise = o.gumbel_noise(5, 0, len(prompt) + np.arange(B), 1, w.model.vocab)
+    _, tok, _ = o.sample_stats(lg, w.model.mask_id, 0.6, noise)
+    assert np.array_equal(tok, t["stats"][0][1])
