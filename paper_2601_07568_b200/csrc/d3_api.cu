@@ -697,11 +697,19 @@ int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMa
   const int q_tiles = (R + nw * 16 - 1) / (nw * 16);
   const int pairs = rm.bs * g.n_kv_heads;
   int splits = 1;
-  if (q_tiles <= 2) {  // decode-sized: split the keys when (sequence, kv head) pairs alone leave SMs idle
+  const int slots = 2 * c->n_sms;  // two CTAs of this kernel fit an SM
+  if (q_tiles <= 2 && pairs * q_tiles < slots) {
+    // decode-sized: (sequence, kv head) pairs alone leave SMs idle, so the keys of a query tile are split
+    // over a cluster (at most 8 CTAs, at least two key tiles each).  The split count that needs the
+    // fewest (waves of resident CTAs) x (key tiles per CTA); ties go to the smaller cluster.
     const int max_tiles = (g.max_seq + attn::KT - 1) / attn::KT;
-    splits = (2 * c->n_sms + pairs * q_tiles - 1) / (pairs * q_tiles);
-    splits = std::min(splits, std::max(1, c->tune_attn_div > 0 ? max_tiles / c->tune_attn_div : max_tiles / 2));
-    splits = std::max(1, std::min(splits, 8));  // one cluster per query tile: at most 8 CTAs
+    const int cap = std::max(1, std::min(8, c->tune_attn_div > 0 ? max_tiles / c->tune_attn_div : max_tiles / 2));
+    long long best = -1;
+    for (int s = 1; s <= cap; ++s) {
+      const long long waves = (static_cast<long long>(pairs) * q_tiles * s + slots - 1) / slots;
+      const long long cost = waves * ((max_tiles + s - 1) / s);
+      if (best < 0 || cost < best) { best = cost; splits = s; }
+    }
   }
   attn::AttnTcParams p{};
   p.q = static_cast<const bf16*>(q);

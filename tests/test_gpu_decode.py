@@ -106,20 +106,19 @@ def step_locked(ctx: Ctx, model: o.OracleModel, prompts, lens, gen_len, block, t
     return report, traces
 
 
-_STATE_CACHE = {}
-
-
 def _state_at(model, trace, prompt, j, block, refresh_every=0):
-    """Oracle cache state at the start of block j (recomputed; small models only)."""
-    key = (id(model), id(trace), j, refresh_every)
-    if key not in _STATE_CACHE:
+    """Oracle cache state at the start of block j (recomputed; small models only).  Kept inside the
+    trace it belongs to, so that nothing outlives the test that made it."""
+    cache = trace.setdefault("_states", {})
+    key = (id(model), j, refresh_every)
+    if key not in cache:
         st = model.prefill(prompt)
         for jj in range(j):
             st = model.finalize_block(st, trace["tokens"][jj * block:(jj + 1) * block])
             if refresh_every > 0 and (jj + 1) % refresh_every == 0:
                 st = model.refresh(st)
-        _STATE_CACHE[key] = st
-    return _STATE_CACHE[key]
+        cache[key] = st
+    return cache[key]
 
 
 # ----------------------------------------------------------------------------- config 1 (tiny fp32)
