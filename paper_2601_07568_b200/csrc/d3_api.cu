@@ -448,7 +448,8 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   // one; with 128-row tiles (32 KB stages, up to 64 KB of partials to receive) one CTA per SM
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + 128 * 128;
   const size_t recv_bytes = tc::gemm_ck_recv_bytes(a_rows, cs.C);
-  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : (a_rows <= 64 ? 100 : 200)) * 1024;
+  // (64-row tiles: 108 KB buy a third 24 KB stage beside the 32 KB of partials, and two CTAs still share an SM)
+  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : (a_rows <= 32 ? 100 : a_rows <= 64 ? 108 : 200)) * 1024;
   int stages = static_cast<int>((budget > recv_bytes ? budget - recv_bytes : 0) / stage_bytes);
   stages = std::max(2, std::min(stages, 16));
   const size_t smem = tc::gemm_ck_smem_bytes(a_rows, stages, cs.C);
