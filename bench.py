@@ -353,7 +353,7 @@ def run_ours(args):
     d3.d3_set_sampling(ctx, 0.0, 0)
     sampling = {"temperature": 0.1, "value": whole_job_tokens_per_s(world, tokens_of(w), args.steps, ms_sm), "unit": UNIT,
                 "forwards_per_request": int(st_sm.steps),
-                "ms_per_forward": ms_sm / args.steps / max(int(st_sm.steps), 1)}
+                "ms_per_step": ms_sm / args.steps / max(int(st_sm.steps), 1)}
 
     # pseudo-trajectory extraction (threshold 1: one token per forward, full length) on the same request,
     # and the noisy-sequence builder on a training-sized batch of responses
