@@ -184,19 +184,23 @@ __global__ void __launch_bounds__(NW * KQ * 32) attn_tc_kernel(const __grid_cons
     ptx::fence_barrier_init();
   }
   __syncthreads();
-  ptx::grid_dep_wait();  // everything below reads what earlier kernels of the stream wrote
   ptx::grid_dep_launch();
-
+  // The row map was written by a kernel that completed before this forward's first kernel started, and
+  // cache rows below pos_base are not touched by this forward: both may be read before the
+  // dependency wait.  Q and the rows the QKV kernel of this layer writes may not.
   const int n_valid = p.rm.n_valid[b];
   const int kv_len = p.rm.kv_len[b];
+  const int stable_keys = p.rm.pos_base[b];  // keys [0, pos_base) come from earlier forwards
   const int R = group * rps;
-  // rows of this tile that exist at all (uniform over the CTA)
-  if (qt * BM >= R || n_valid <= 0 || kv_len <= 0) return;
-  // a tile whose rows are all beyond n_valid has nothing to do (rows of one head are contiguous)
-  {
+  bool work = !(qt * BM >= R || n_valid <= 0 || kv_len <= 0);  // rows of this tile that exist at all (uniform over the CTA)
+  if (work) {  // a tile whose rows are all beyond n_valid has nothing to do (rows of one head are contiguous)
     bool any = false;
     for (int pr = qt * BM; pr < min(R, (qt + 1) * BM) && !any; pr += 1) any = (pr % rps) < n_valid;
-    if (!any) return;
+    work = any;
+  }
+  if (!work) {
+    ptx::grid_dep_wait();
+    return;
   }
   const int n_tiles = (kv_len + KT - 1) / KT;
   const int tps = (n_tiles + p.n_splits - 1) / p.n_splits;
@@ -215,8 +219,16 @@ __global__ void __launch_bounds__(NW * KQ * 32) attn_tc_kernel(const __grid_cons
     ptx::tma_load_2d(st + 2 * KT * 128, &tmap_kv, &full_bar[s], 0, static_cast<int>(vrow + j0));
     ptx::tma_load_2d(st + 3 * KT * 128, &tmap_kv, &full_bar[s], 64, static_cast<int>(vrow + j0));
   };
+  // first lap of the ring: tiles that lie wholly in the stable prefix are requested while the kernel
+  // before this one still runs, the others after the dependency wait
+  auto stable = [&](int i) { return (t0 + i + 1) * KT <= stable_keys; };
   if (threadIdx.x == 0)
-    for (int i = 0; i < min(n_my, TC_STAGES); ++i) issue(i);
+    for (int i = 0; i < min(n_my, TC_STAGES); ++i)
+      if (stable(i)) issue(i);
+  ptx::grid_dep_wait();  // everything below reads what earlier kernels of the stream wrote
+  if (threadIdx.x == 0)
+    for (int i = 0; i < min(n_my, TC_STAGES); ++i)
+      if (!stable(i)) issue(i);
 
   // ---- Q fragments of this warp's 16 packed rows (rows g4 and g4 + 8), straight from global memory
   const int pr_lo = qt * BM + warp * 16 + g4, pr_hi = pr_lo + 8;
