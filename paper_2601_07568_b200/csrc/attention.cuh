@@ -152,8 +152,11 @@ __device__ __forceinline__ uint32_t swz(int r, int c) { return static_cast<uint3
 // tensor-core partitions idle and walk through its tiles four times as long).  Warp w: row group
 // w % NW, key part w / NW.  Every warp keeps its own running softmax state; the key parts are
 // merged through shared memory after the last tile, then the key splits across the cluster.
+// Registers: two CTAs per SM (128 registers a thread) cost the 8-row-group variant a few hundred bytes
+// of spills and still pay (GQA decode: 38 -> 34 us per launch); the 4-row-group variant was slower that
+// way at long prefixes (102 -> 109 us) and keeps its 174 registers and one CTA per SM.
 template <int NW, int KQ>
-__global__ void __launch_bounds__(NW * KQ * 32) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_kv,
+__global__ void __launch_bounds__(NW * KQ * 32, NW == 4 ? 1 : 2) attn_tc_kernel(const __grid_constant__ CUtensorMap tmap_kv,
                                                                const AttnTcParams p) {
   constexpr int BM = NW * 16;
   constexpr int KPW = KT / KQ;  // keys per warp and tile: 64, 32 or 16

@@ -690,6 +690,20 @@ int launch_attn_tc(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
   return D3_OK;
 }
 
+// CTAs of one attention instantiation that fit an SM (registers and shared memory), asked once.
+template <int NW, int KQ>
+int attn_ctas_per_sm() {
+  static int cached = 0;
+  if (cached == 0) {
+    auto kern = attn::attn_tc_kernel<NW, KQ>;
+    cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::attn_tc_smem_bytes()));
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, NW * KQ * 32, attn::attn_tc_smem_bytes()) != cudaSuccess || n < 1) n = 1;
+    cached = n;
+  }
+  return cached;
+}
+
 int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
   const d3_config& g = c->cfg;
   const int group = g.n_q_heads / g.n_kv_heads;
@@ -698,19 +712,23 @@ int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMa
   const int q_tiles = (R + nw * 16 - 1) / (nw * 16);
   const int pairs = rm.bs * g.n_kv_heads;
   int splits = 1;
-  const int slots = 2 * c->n_sms;  // two CTAs of this kernel fit an SM
+  const int slots = c->n_sms * (nw == 2 ? attn_ctas_per_sm<2, 4>() : nw == 4 ? attn_ctas_per_sm<4, 2>() : attn_ctas_per_sm<8, 1>());
   if (q_tiles <= 2 && pairs * q_tiles < slots) {
     // decode-sized: (sequence, kv head) pairs alone leave SMs idle, so the keys of a query tile are split
-    // over a cluster (at most 8 CTAs, at least two key tiles each).  The split count that needs the
-    // fewest (waves of resident CTAs) x (key tiles per CTA); ties go to the smaller cluster.
+    // over a cluster (at most 8 CTAs, at least two key tiles each).  Cost of a split count:
+    // (waves of resident CTAs) x (key tiles per CTA).
     const int max_tiles = (g.max_seq + attn::KT - 1) / attn::KT;
     const int cap = std::max(1, std::min(8, c->tune_attn_div > 0 ? max_tiles / c->tune_attn_div : max_tiles / 2));
-    long long best = -1;
-    for (int s = 1; s <= cap; ++s) {
+    auto cost_of = [&](int s) {
       const long long waves = (static_cast<long long>(pairs) * q_tiles * s + slots - 1) / slots;
-      const long long cost = waves * ((max_tiles + s - 1) / s);
-      if (best < 0 || cost < best) { best = cost; splits = s; }
-    }
+      return waves * ((max_tiles + s - 1) / s);
+    };
+    long long best = cost_of(1);
+    for (int s = 2; s <= cap; ++s) best = std::min(best, cost_of(s));
+    // larger clusters cost more than this count sees (co-scheduling, the merge: eight splits at a
+    // 5120-key prefix took 160 us where two took 102): the smallest count within 15 % of the best
+    for (int s = 1; s <= cap; ++s)
+      if (cost_of(s) * 100 <= best * 115) { splits = s; break; }
   }
   attn::AttnTcParams p{};
   p.q = static_cast<const bf16*>(q);
