@@ -158,3 +158,67 @@ def test_c5_full_size_long_prefix(llada_weights):
 
 def test_c4_full_size_gqa():
     _check_workload("c4", layers=[0, 27], seqs=[0, 5])
+
+
+def test_c2_full_size_sampling_refresh_and_multiblock(llada_weights):
+    """The widened decoding features at the full 8B shape (batch 1, 32-row forwards, 126464-token head):
+    the tokens the sampling epilogue draws are the oracle's Gumbel-max rule applied to the device's own
+    fp32 logits of the same forward (all 988 vocabulary tiles, ragged last tile); a KV-refresh of a
+    prompt-only cache changes no bit of the next logits, and after a stored block it does; multi-block
+    decoding with four blocks in flight commits every token in fewer rounds than block-by-block
+    decoding takes forwards, reproducibly."""
+    w = si.WORKLOADS["c2"]
+    shape = w.model
+    ids, lens = si.gen_prompts(w)
+    B = w.block
+    with Ctx(shape, llada_weights, block=B, max_batch=w.batch, max_seq=w.max_seq, max_prefill_rows=w.batch * w.max_seq) as ctx:
+        # ---- sampling against the device's own logits
+        ctx.prefill(ids, lens)
+        blk = np.full((1, B), shape.mask_id, dtype=np.int32)
+        mask = np.ones((1, B), dtype=bool)
+        lg = ctx.logits(blk)[0]
+        greedy = np.argmax(np.where(np.arange(shape.vocab)[None, :] == shape.mask_id, -np.inf, lg), axis=1)
+        away = 0
+        for T, seed in [(0.1, 20260107), (4.0, (9 << 32) + 5)]:     # the paper's setting, and one that does move tokens
+            ctx.prefill(ids, lens)                                   # the step counter of the explicit calls starts again
+            d3.d3_set_sampling(ctx.ctx, T, seed)
+            got = ctx.step(blk, mask, w.threshold)
+            d3.d3_set_sampling(ctx.ctx, 0.0, 0)
+            noise = o.gumbel_noise(seed, 0, lens[0] + np.arange(B), 1, shape.vocab)
+            conf, tok, ent = o.sample_stats(lg, shape.mask_id, T, noise)
+            pert = lg.astype(np.float32) + np.float32(T) * noise
+            pert[:, shape.mask_id] = -np.inf
+            top = np.sort(pert, axis=1)[:, -2:]
+            clear = (top[:, 1] - top[:, 0]) > 1e-3       # the two paths' logits differ by their K-split order
+            assert clear.sum() >= B - 2
+            assert np.array_equal(got["tok"][0][clear], tok[clear])
+            same = got["tok"][0] == tok
+            assert np.allclose(got["conf"][0][same], conf[same], rtol=1e-3, atol=1e-7)
+            assert np.allclose(got["ent"][0], ent, rtol=1e-3, atol=1e-4)
+            away += int((tok != greedy).sum())
+            print("c2 sampling T", T, ": rows compared", int(clear.sum()), "rows drawn away from the arg max", int((tok != greedy).sum()))
+        assert away > 0
+        # ---- KV-refresh
+        ctx.prefill(ids, lens)
+        base = ctx.logits(blk)
+        d3.d3_refresh_cache(ctx.ctx, 1)
+        assert np.array_equal(ctx.logits(blk), base)
+        stored = np.random.default_rng(1).integers(0, shape.vocab - 2, size=(1, B)).astype(np.int32)
+        ctx.commit(stored)
+        before = ctx.logits(blk)
+        d3.d3_refresh_cache(ctx.ctx, 1)
+        after = ctx.logits(blk)
+        assert np.isfinite(after[:, :, :shape.mask_id]).all() and np.abs(after - before)[:, :, :shape.mask_id].max() > 0
+        assert np.array_equal(ctx.get_prefix(1), lens + B) and ctx.error_word() == 0
+        # ---- multi-block decoding, four blocks in flight (128-row rounds)
+        ctx.prefill(ids, lens)
+        tok1, _, st1 = ctx.generate(1, w.gen_len, w.threshold)
+        ctx.prefill(ids, lens)
+        mb1, cr1, sm1 = ctx.generate_multiblock(1, w.gen_len, w.threshold, 4)
+        ctx.prefill(ids, lens)
+        mb2, cr2, sm2 = ctx.generate_multiblock(1, w.gen_len, w.threshold, 4)
+        assert np.array_equal(mb1, mb2) and np.array_equal(cr1, cr2)
+        assert sm1.tokens_committed == w.gen_len and not (mb1 == shape.mask_id).any() and mb1.min() >= 0 and mb1.max() < shape.vocab
+        assert sm1.steps < st1.denoise_forwards + st1.finalize_forwards and cr1.min() >= 1 and cr1.max() <= sm1.steps
+        assert ctx.error_word() == 0
+        print("c2 multi-block: rounds", sm1.steps, "against", st1.denoise_forwards + st1.finalize_forwards, "forwards block by block")
