@@ -81,8 +81,9 @@ typedef struct d3_config {
  * entries.  Norm gains may be NULL (= all ones).  Shapes: tok_emb, lm_head [vocab, d_model];
  * wq [n_q_heads*d_head, d_model]; wk, wv [n_kv_heads*d_head, d_model]; wo [d_model,
  * n_q_heads*d_head]; w_gate, w_up [d_ffn, d_model]; w_down [d_model, d_ffn]; gains [d_model].
- * On the bfloat16 tensor-core path the gains of each RMSNorm (Sec. 3.1: the backbone is a standard
- * pre-norm transformer) are multiplied into the columns of the matrix that follows it when the
+ * On the bfloat16 tensor-core path the gains of each RMSNorm (the paper names no architecture beyond
+ * a plain Transformer backbone, appendix on foundation models; the pre-norm layout is that of the
+ * model shapes this library is configured with) are multiplied into the columns of the matrix that follows it when the
  * weights are loaded (one extra bfloat16 rounding of those weights), and the row factor
  * rsqrt(mean(x^2) + eps) is applied to the matmul's fp32 accumulator: same function, no separate
  * normalisation kernels (D3_PROF_RMSNORM then stays empty). */
@@ -170,6 +171,13 @@ int d3_generate(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32
 int d3_generate_multiblock(d3_ctx *ctx, int32_t gen_len, float threshold, int32_t bs, int32_t max_active,
                            int32_t *out_ids, int32_t *commit_round, d3_stats *host_stats);
 
+/* Commits per decision of the latest d3_generate / d3_generate_multiblock call (the distribution
+ * behind tokens per forward, the paper's efficiency measure, Sec. 2 and Sec. 4.1): hist[k], k < n, is
+ * the number of (sequence, denoise forward) decisions -- in multi-block decoding (sequence, block,
+ * round) decisions -- that committed exactly k tokens.  hist [host][n]; entries beyond the block
+ * size are 0.  Waits for the stream. */
+int d3_commit_histogram(d3_ctx *ctx, int64_t *hist, int32_t n);
+
 /* Early stopping on the end-of-sequence token (Sec. 3.2, "Early Stopping on EOS Token"): with an id set,
  * d3_generate stops a sequence after the denoise step that commits that id anywhere in its current
  * block.  The block goes out as it stands, undecoded positions (there and in all later blocks) read
@@ -241,6 +249,16 @@ int d3_get_step_stats(d3_ctx *ctx, float *conf, float *entropy, int32_t *argmax,
  * kept (layer < 0: none); d3_read_tap copies them out as fp32 [rows, d_model].  d3_read_kv copies
  * cache slots [pos0, pos0+n) of one layer and sequence as fp32 [n_kv_heads, n, d_head]. */
 int d3_forward_logits(d3_ctx *ctx, const int32_t *block_ids, int32_t bs, float *logits);
+/* One round of multi-block decoding without the decisions (Sec. 3.2, multi-block decoding): forward
+ * of n_win (1..8) consecutive blocks per sequence, window_ids [device][bs, n_win*B], placed at the
+ * sequences' prefixes; block w sees the cache, blocks 0..w-1 of the window and itself.  Writes the
+ * softmax statistics of every row, conf / entropy [device][bs*n_win*B] float and argmax
+ * [device][bs*n_win*B] int32 (any may be NULL), and leaves the rows' K/V in cache slots
+ * [prefix, prefix + n_win*B): advancing the prefix with d3_set_state by k*B afterwards stores the first
+ * k blocks exactly as d3_generate_multiblock does after a stabilizing round.  Errors: SHAPE when
+ * bs * n_win * B rows exceed the workspaces sized by max_batch, STATE before d3_prefill. */
+int d3_denoise_window(d3_ctx *ctx, const int32_t *window_ids, int32_t bs, int32_t n_win, float *conf,
+                      float *entropy, int32_t *argmax);
 int d3_set_tap(d3_ctx *ctx, int32_t layer);
 int d3_read_tap(d3_ctx *ctx, float *resid_in, float *resid_out, int32_t rows);
 int d3_read_kv(d3_ctx *ctx, int32_t layer, int32_t seq, int32_t pos0, int32_t n, float *k_out, float *v_out);
@@ -328,17 +346,6 @@ int d3_lm_head_stats_static(const void *x, const void *w, int32_t dtype, int32_t
  * identical either way. */
 int d3_set_overlap(d3_ctx *ctx, int on);
 
-/* Matmul tuning overrides for measurement sweeps: shared-memory ring per CTA in KB (0 = default:
- * about 100 KB for matmuls of up to 128 rows, 200 KB otherwise; at most 200) and CTAs per SM that the
- * (tile, K slab) units are dealt to (0 = default 1; at most 3).  Bits 16 and up of ring_kb select
- * scheduling variants for sweeps and tests: 16-19 producer warps, 20-21 tile width + 1, 22-24 divisor
- * of the attention key splits, 25 no cluster K-split, 26-27 row-tile pairs + 1, 28 no round-robin
- * tiles, 29-30 column strips for skinny matmuls (0 when they pay, 1 never, 2 with one CTA per SM,
- * 3 wherever the shape allows).  Bit 8 of ctas_per_sm: d3_generate finalizes every block in a forward of
- * its own instead of fusing that forward with the next block's first step (see d3_generate).  Results
- * do not change beyond the order of fp32 partial sums. */
-int d3_set_matmul_tuning(d3_ctx *ctx, int32_t ring_kb, int32_t ctas_per_sm);
-
 /* Per-class kernel timing for measurement runs.  While enabled, every launch of the forward pass is
  * bracketed by a CUDA event pair on the context's stream; d3_profile_read waits for the stream and
  * returns, per class, the summed elapsed milliseconds and the number of launches since enabling.
@@ -350,7 +357,9 @@ enum { D3_PROF_GEMM_QKV = 0, D3_PROF_GEMM_O = 1, D3_PROF_GEMM_GATE_UP = 2, D3_PR
 int d3_profile_enable(d3_ctx *ctx, int on);
 int d3_profile_read(d3_ctx *ctx, double *ms, int64_t *launches);
 
-/* Device error word: 0 when no bounded wait has given up and no kernel saw an invalid index.
+/* Device error word: 0 when no bounded wait has given up and no kernel saw an invalid index or
+ * statistic (bit 0: a wait gave up; 1: token id outside the vocabulary; 2: cache slot outside
+ * max_seq; 4: every masked row of a block had a NaN statistic, the lowest one was committed).
  * Synchronises the stream.  Returns D3_OK and writes the word, or D3_ERR_CUDA. */
 int d3_get_error_word(d3_ctx *ctx, uint32_t *word);
 /* Number of this library's kernels launched on the context since creation. */

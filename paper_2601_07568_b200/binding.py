@@ -27,9 +27,13 @@ EXPORTS = [
     "d3_create", "d3_destroy", "d3_load_weights", "d3_prefill", "d3_denoise_step", "d3_commit_block",
     "d3_generate", "d3_get_step_stats", "d3_forward_logits", "d3_set_tap", "d3_read_tap", "d3_read_kv",
     "d3_get_state", "d3_set_state", "d3_op_linear", "d3_packed_weight_elems", "d3_pack_weight", "d3_op_linear_packed", "d3_op_lm_head_stats", "d3_op_attention",
-    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_set_matmul_tuning", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_generate_multiblock", "d3_refresh_cache", "d3_set_cache_policy", "d3_refresh_count", "d3_trajectory_rank", "d3_noisy_sequence", "d3_set_sampling", "d3_device_bytes",
+    "d3_op_write_kv", "d3_op_unmask", "d3_lm_head_stats_static", "d3_set_overlap", "d3_profile_enable", "d3_profile_read", "d3_get_error_word", "d3_launch_count", "d3_launch_count_of", "d3_set_eos", "d3_early_stops", "d3_generate_multiblock", "d3_refresh_cache", "d3_set_cache_policy", "d3_refresh_count", "d3_trajectory_rank", "d3_noisy_sequence", "d3_set_sampling", "d3_device_bytes",
+    "d3_denoise_window", "d3_commit_histogram",
     "d3_strerror", "d3_last_error", "d3_version",
 ]
+# measurement and test switches (include/d3_debug.h)
+DEBUG_EXPORTS = ["d3_tuning_defaults", "d3_set_tuning", "d3_set_fused_finalize", "d3_debug_stall_probe",
+                 "d3_clear_error_word", "d3_status_of_error_word"]
 
 
 class d3_config(C.Structure):
@@ -207,6 +211,21 @@ def d3_forward_logits(ctx, block_ids: torch.Tensor, logits: torch.Tensor) -> Non
                                         _ptr(_dev(logits, torch.float32))))
 
 
+def d3_denoise_window(ctx, window_ids: torch.Tensor, n_win: int, conf: torch.Tensor, entropy: torch.Tensor,
+                      argmax: torch.Tensor) -> None:
+    bs = window_ids.shape[0]
+    _check(ctx, lib().d3_denoise_window(ctx, _ptr(_dev(window_ids, torch.int32)), C.c_int32(bs), C.c_int32(n_win),
+                                        _ptr(_dev(conf, torch.float32)), _ptr(_dev(entropy, torch.float32)),
+                                        _ptr(_dev(argmax, torch.int32))))
+
+
+def d3_commit_histogram(ctx, n: int):
+    """hist[k] = decisions of the latest generate call that committed exactly k tokens, k < n."""
+    h = (C.c_int64 * n)()
+    _check(ctx, lib().d3_commit_histogram(ctx, h, C.c_int32(n)))
+    return [int(v) for v in h]
+
+
 def d3_set_tap(ctx, layer: int) -> None:
     _check(ctx, lib().d3_set_tap(ctx, C.c_int32(layer)))
 
@@ -257,8 +276,23 @@ def d3_op_linear_packed(ctx, x: torch.Tensor, w_packed: torch.Tensor, y: torch.T
                                           C.c_int32(n), C.c_int32(k), C.c_int32(epilogue), C.c_int32(splits)))
 
 
+def _check_head_shapes(x, w, conf, entropy, argmax) -> None:
+    """The C ABI sees pointers only: sizes that would make a kernel read or write past a tensor are
+    refused here."""
+    if x.dim() != 2 or w.dim() != 2:
+        raise ValueError("x and w must be 2-D")
+    if w.shape[1] != x.shape[1]:
+        raise ValueError(f"w has {w.shape[1]} columns, x has {x.shape[1]}")
+    m = x.shape[0]
+    for name, t in (("conf", conf), ("entropy", entropy), ("argmax", argmax)):
+        if t.numel() < m:
+            raise ValueError(f"{name} holds {t.numel()} elements, {m} rows need as many")
+
+
 def d3_op_lm_head_stats(ctx, x: torch.Tensor, w: torch.Tensor, scale: float, mask_id: int, conf: torch.Tensor,
                         entropy: torch.Tensor, argmax: torch.Tensor) -> None:
+    _dev(x), _dev(w, x.dtype)
+    _check_head_shapes(x, w, conf, entropy, argmax)
     m, k = x.shape
     _check(ctx, lib().d3_op_lm_head_stats(ctx, _ptr(_dev(x)), _ptr(_dev(w)), C.c_int32(m), C.c_int32(w.shape[0]),
                                           C.c_int32(k), C.c_float(scale), C.c_int32(mask_id),
@@ -302,6 +336,7 @@ def d3_lm_head_stats_static(x: torch.Tensor, w: torch.Tensor, scale: float, mask
     _dev(x), _dev(w, x.dtype)
     if x.dtype not in (torch.float32, torch.bfloat16):
         raise ValueError("x and w must be float32 or bfloat16")
+    _check_head_shapes(x, w, conf, entropy, argmax)
     m, k = x.shape
     s = C.c_void_p(stream.cuda_stream if stream is not None else torch.cuda.current_stream().cuda_stream)
     rc = lib().d3_lm_head_stats_static(_ptr(x), _ptr(w), C.c_int32(D3_DTYPE_BF16 if x.dtype == torch.bfloat16 else D3_DTYPE_F32),
@@ -320,8 +355,43 @@ def d3_set_overlap(ctx, on: bool) -> None:
     _check(ctx, lib().d3_set_overlap(ctx, C.c_int(1 if on else 0)))
 
 
-def d3_set_matmul_tuning(ctx, ring_kb: int = 0, ctas_per_sm: int = 0) -> None:
-    _check(ctx, lib().d3_set_matmul_tuning(ctx, C.c_int32(ring_kb), C.c_int32(ctas_per_sm)))
+class d3_tuning(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("ring_kb", "ctas_per_sm", "producers", "tile_columns", "attn_key_tiles",
+                                          "cluster_k_split", "row_tile_pairs", "round_robin", "column_strips",
+                                          "strip_stages")]
+
+
+def d3_tuning_defaults() -> d3_tuning:
+    t = d3_tuning()
+    lib().d3_tuning_defaults(C.byref(t))
+    return t
+
+
+def d3_set_tuning(ctx, tuning: Optional[d3_tuning] = None, **fields) -> None:
+    """Scheduling overrides (include/d3_debug.h).  ``tuning`` or the defaults, with ``fields`` set by name."""
+    t = tuning if tuning is not None else d3_tuning_defaults()
+    for k, v in fields.items():
+        if not hasattr(t, k):
+            raise ValueError(f"d3_tuning has no field {k}")
+        setattr(t, k, v)
+    _check(ctx, lib().d3_set_tuning(ctx, C.byref(t)))
+
+
+def d3_set_fused_finalize(ctx, on: bool) -> None:
+    _check(ctx, lib().d3_set_fused_finalize(ctx, C.c_int(1 if on else 0)))
+
+
+def d3_debug_stall_probe(ctx, limit_us: int) -> int:
+    """Returns the status code of the probe (D3_ERR_DEVICE_TIMEOUT is the expected outcome)."""
+    return int(lib().d3_debug_stall_probe(ctx, C.c_int32(limit_us)))
+
+
+def d3_clear_error_word(ctx) -> None:
+    _check(ctx, lib().d3_clear_error_word(ctx))
+
+
+def d3_status_of_error_word(word: int) -> int:
+    return int(lib().d3_status_of_error_word(C.c_uint32(word)))
 
 
 def d3_profile_enable(ctx, on: bool) -> None:

@@ -12,6 +12,7 @@ enum : uint32_t {
   ERRW_BAD_TOKEN_ID = 1u << 1,   // a token id outside [0, vocab)
   ERRW_BAD_POSITION = 1u << 2,   // a cache slot outside [0, max_seq)
   ERRW_TMEM_ALLOC = 1u << 3,     // tensor-memory allocation returned an unexpected address
+  ERRW_BAD_STATISTIC = 1u << 4,  // every masked row of a block had an unusable (NaN) statistic: lowest row forced
 };
 
 // ---- matmul epilogues

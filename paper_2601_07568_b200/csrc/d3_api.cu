@@ -1,6 +1,7 @@
 // C ABI of the d3 library (see include/d3.h): context, weight repacking, the forward pass as a
 // sequence of kernel launches on one stream, the decision kernels and the generate loop.
 #include "../../include/d3.h"
+#include "../../include/d3_debug.h"
 
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -107,6 +108,8 @@ struct d3_ctx {
   int tune_no_cluster = 0;  // 1: skinny matmuls on the unit-range kernel (L2 reduction) instead of clusters
   int tune_wide_tiles = -1;  // -1: by row count; 0 / 1: force 128- / 256-column tiles
   int tune_ring_kb = 0, tune_ctas_per_sm = 0;  // matmul tuning overrides (0 = default)
+  int tune_strip_stages = 0;  // explicit pipeline depth of the column-strip kernel (0: from the ring size)
+  unsigned long long* commit_hist = nullptr;  // [COMMIT_HIST_BINS] commits per decision of the latest generate call
   struct ProfPair { cudaEvent_t a, b; int cls; };
   std::vector<ProfPair> prof_pool;
   size_t prof_used = 0;
@@ -539,6 +542,12 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   const size_t ring = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 200 / per_sm) * 1024;
   const size_t stage_bytes = static_cast<size_t>(a_rows + S) * 128;
   p.stages = std::max(2, std::min<int>(std::min<int>(static_cast<int>(ring / stage_bytes), KC), 32));
+  const bool explicit_stages = c->tune_strip_stages > 0;
+  if (explicit_stages) {
+    p.stages = c->tune_strip_stages;
+    if (p.stages < 2 || p.stages > 32 || p.stages > KC || static_cast<size_t>(p.stages) * stage_bytes > 200 * 1024)
+      return fail(c, D3_ERR_UNSUPPORTED, "strip_stages outside 2..min(32, K slabs) or beyond 200 KB of shared memory");
+  }
   p.error_word = c->error_word;
   p.skip_flag = c->skip_flag;
   p.w_tiled = 1;
@@ -548,7 +557,13 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   // two issue pipelines per CTA while both accumulators fit 256 tensor-memory columns; each then owns
   // the stages of its parity, so the ring has an even number of them
   p.n_producers = (S <= 128 && KC >= 4 && c->tune_producers != 1) ? 2 : 1;
-  if (p.n_producers == 2) p.stages &= ~1;
+  if (p.n_producers == 2) {
+    // every stage stays with one pipeline (stage s serves slabs s, s + stages, ...: the same parity
+    // of slab index only when the count is even).  An odd count asked for by name is refused.
+    if (explicit_stages && (p.stages & 1))
+      return fail(c, D3_ERR_UNSUPPORTED, "two issue pipelines need an even number of stages");
+    p.stages &= ~1;
+  }
   p.ep = ep;
   if (qx) {
     p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
@@ -902,8 +917,9 @@ int check_device_error(d3_ctx* c) {
   uint32_t w = 0;
   CUDA_TRY(c, cudaMemcpyAsync(&w, c->error_word, sizeof(w), cudaMemcpyDeviceToHost, c->stream));
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
-  if (w & ERRW_MBAR_TIMEOUT) return fail(c, D3_ERR_DEVICE_TIMEOUT, "a bounded device-side wait gave up");
-  if (w) return fail(c, D3_ERR_INVALID_ARG, "device error word " + std::to_string(w) + " (bad token id or position)");
+  const int rc = d3_status_of_error_word(w);
+  if (rc == D3_ERR_DEVICE_TIMEOUT) return fail(c, rc, "a bounded device-side wait gave up");
+  if (rc != D3_OK) return fail(c, rc, "device error word " + std::to_string(w) + " (bad token id, position or statistic)");
   return D3_OK;
 }
 
@@ -1026,6 +1042,11 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   A_(c->mb.fwd_ids, sizeof(int) * static_cast<size_t>(g.max_batch) * MB_MAX_WINDOW * g.block);
   A_(c->gen.fwd_ids, sizeof(int) * 2 * static_cast<size_t>(g.max_batch) * g.block);
   A_(c->gen.counters, sizeof(long long) * 8);
+  A_(c->commit_hist, sizeof(unsigned long long) * COMMIT_HIST_BINS);
+  c->gen.commit_hist = c->commit_hist;
+  c->mb.commit_hist = c->commit_hist;
+  c->gen.error_word = c->error_word;
+  c->mb.error_word = c->error_word;
   A_(c->hist_ids, sizeof(int) * static_cast<size_t>(g.max_batch) * g.max_seq);
   A_(c->refresh_ids, sizeof(int) * R);
   A_(c->gen.refresh_flag, sizeof(int) * g.max_batch);
@@ -1277,7 +1298,7 @@ extern "C" int d3_denoise_step(d3_ctx* c, int32_t* block_ids, uint8_t* mask, flo
   c->draw_step = nullptr;  // sampling noise of the explicit calls: steps counted since the last prefill / commit
   c->draw_step_add = ++c->explicit_step;
   TRY(forward(c, block_ids, bs, B, 1, nullptr));
-  unmask_kernel<<<bs, 32, 0, c->stream>>>(c->conf, c->ent, c->argmax, block_ids, mask, B, threshold, c->cfg.decide_mode, out_pos, out_ids, out_count);
+  unmask_kernel<<<bs, 32, 0, c->stream>>>(c->conf, c->ent, c->argmax, block_ids, mask, B, threshold, c->cfg.decide_mode, out_pos, out_ids, out_count, c->error_word);
   LAUNCHED(c, "unmask_kernel");
   return D3_OK;
 }
@@ -1477,6 +1498,27 @@ extern "C" int d3_forward_logits(d3_ctx* c, const int32_t* block_ids, int32_t bs
   return forward(c, block_ids, bs, B, 2, logits);
 }
 
+extern "C" int d3_denoise_window(d3_ctx* c, const int32_t* window_ids, int32_t bs, int32_t n_win, float* conf,
+                                 float* entropy, int32_t* argmax) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (!window_ids || bs <= 0 || n_win < 1 || n_win > MB_MAX_WINDOW) return fail(c, D3_ERR_INVALID_ARG, "bad denoise_window arguments");
+  if (!c->prefilled) return fail(c, D3_ERR_STATE, "d3_denoise_window before d3_prefill");
+  const int B = c->cfg.block;
+  const long long rows = static_cast<long long>(bs) * n_win * B;
+  if (bs > c->cfg.max_batch || rows > std::min<long long>(c->stat_rows, c->max_rows))
+    return fail(c, D3_ERR_SHAPE, "bs * n_win * block rows exceed the workspaces (raise max_batch at d3_create)");
+  decode_rowmap_kernel<<<(bs + 63) / 64, 64, 0, c->stream>>>(c->prefix_len, bs, n_win * B, c->pos_base, c->n_valid, c->kv_len);
+  LAUNCHED(c, "decode_rowmap_kernel");
+  c->draw_step = nullptr;
+  c->draw_step_add = ++c->explicit_step;
+  TRY(forward(c, window_ids, bs, n_win * B, 1, nullptr, B));
+  const size_t n = static_cast<size_t>(rows);
+  if (conf) CUDA_TRY(c, cudaMemcpyAsync(conf, c->conf, n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if (entropy) CUDA_TRY(c, cudaMemcpyAsync(entropy, c->ent, n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if (argmax) CUDA_TRY(c, cudaMemcpyAsync(argmax, c->argmax, n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  return D3_OK;
+}
+
 extern "C" int d3_set_tap(d3_ctx* c, int32_t layer) {
   if (!c || layer >= c->cfg.n_layers) return D3_ERR_INVALID_ARG;
   c->tap_layer = layer < 0 ? -1 : layer;
@@ -1618,7 +1660,7 @@ extern "C" int d3_op_unmask(d3_ctx* c, const float* conf, const float* entropy, 
   if (!conf || !entropy || !argmax || !block_ids || !mask || !out_pos || !out_ids || !out_count || bs <= 0 ||
       std::isnan(threshold))
     return fail(c, D3_ERR_INVALID_ARG, "bad op_unmask arguments");
-  unmask_kernel<<<bs, 32, 0, c->stream>>>(conf, entropy, argmax, block_ids, mask, c->cfg.block, threshold, c->cfg.decide_mode, out_pos, out_ids, out_count);
+  unmask_kernel<<<bs, 32, 0, c->stream>>>(conf, entropy, argmax, block_ids, mask, c->cfg.block, threshold, c->cfg.decide_mode, out_pos, out_ids, out_count, c->error_word);
   LAUNCHED(c, "unmask_kernel");
   return D3_OK;
 }
@@ -1630,19 +1672,86 @@ extern "C" int d3_get_error_word(d3_ctx* c, uint32_t* word) {
   CUDA_TRY(c, cudaStreamSynchronize(c->stream));
   return D3_OK;
 }
-extern "C" int d3_set_matmul_tuning(d3_ctx* c, int32_t ring_kb, int32_t ctas_per_sm) {
-  if (!c || ring_kb < 0 || (ring_kb & 0xffff) > 200 || ctas_per_sm < 0 || (ctas_per_sm & 0xff) > 3 || ctas_per_sm > 0x1ff) return D3_ERR_INVALID_ARG;
-  c->gen_fuse = ((ctas_per_sm >> 8) & 1) == 0;  // bit 8 of ctas_per_sm: d3_generate finalizes every block in a forward of its own
-  ctas_per_sm &= 0xff;
-  c->tune_producers = (ring_kb >> 16) & 0xf;  // experiments: bits 16-19 of ring_kb = producer warps, 20-21 = tile width + 1
-  c->tune_wide_tiles = ((ring_kb >> 20) & 3) - 1;
-  c->tune_attn_div = (ring_kb >> 22) & 7;
-  c->tune_no_cluster = (ring_kb >> 25) & 1;
-  c->tune_pair = ((ring_kb >> 26) & 3) - 1;
-  c->tune_no_rr = (ring_kb >> 28) & 1;
-  c->tune_strip = (ring_kb >> 29) & 3;
-  c->tune_ring_kb = ring_kb & 0xffff;
-  c->tune_ctas_per_sm = ctas_per_sm;
+extern "C" void d3_tuning_defaults(d3_tuning* t) {
+  if (!t) return;
+  std::memset(t, 0, sizeof(*t));
+  t->cluster_k_split = -1;
+  t->row_tile_pairs = -1;
+  t->round_robin = 1;
+}
+extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
+  if (!c || !t) return D3_ERR_INVALID_ARG;
+  if (t->ring_kb < 0 || t->ring_kb > 200 || t->ctas_per_sm < 0 || t->ctas_per_sm > 3 || t->producers < 0 || t->producers > 2 ||
+      (t->tile_columns != 0 && t->tile_columns != 128 && t->tile_columns != 256) || t->attn_key_tiles < 0 || t->attn_key_tiles > 7 ||
+      t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
+      (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
+      t->strip_stages > 32)
+    return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
+  c->tune_ring_kb = t->ring_kb;
+  c->tune_ctas_per_sm = t->ctas_per_sm;
+  c->tune_producers = t->producers;
+  c->tune_wide_tiles = t->tile_columns == 0 ? -1 : (t->tile_columns == 256 ? 1 : 0);
+  c->tune_attn_div = t->attn_key_tiles;
+  c->tune_no_cluster = t->cluster_k_split == 0 ? 1 : 0;
+  c->tune_pair = t->row_tile_pairs;
+  c->tune_no_rr = t->round_robin ? 0 : 1;
+  c->tune_strip = t->column_strips;
+  c->tune_strip_stages = t->strip_stages;
+  return D3_OK;
+}
+extern "C" int d3_set_fused_finalize(d3_ctx* c, int on) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  c->gen_fuse = on != 0;
+  return D3_OK;
+}
+extern "C" int d3_clear_error_word(d3_ctx* c) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  CUDA_TRY(c, cudaMemsetAsync(c->error_word, 0, sizeof(uint32_t), c->stream));
+  return D3_OK;
+}
+extern "C" int d3_debug_stall_probe(d3_ctx* c, int32_t limit_us) {
+  if (!c) return D3_ERR_INVALID_ARG;
+  if (limit_us < 1 || limit_us > 2000000) return fail(c, D3_ERR_INVALID_ARG, "limit_us must be 1..2000000");
+  if (!c->use_tc) return fail(c, D3_ERR_UNSUPPORTED, "the probe runs the tensor-core matmul kernel (bfloat16 contexts only)");
+  // One CTA, one 32 x 128 x 64 unit, no loads issued: the MMA-issuing thread's wait for the first
+  // stage runs out, it raises the abort flag and the error word, the epilogue warps see the flag at
+  // their next check, every role falls through to the final barrier and tensor memory is released.
+  // No copy and no MMA is in flight at any time.
+  tc::GemmParams p{};
+  p.M = 32; p.N = 128; p.K = 64;
+  p.a_rows = 32;
+  p.m_tiles = 1; p.n_tiles = 1; p.k_chunks = 1;
+  p.total_units = 1;
+  p.stages = 2;
+  p.partial = c->partial;
+  p.tile_count = c->tile_count;
+  p.error_word = c->error_word;
+  p.skip_flag = nullptr;
+  p.wait_limit_us = static_cast<uint32_t>(limit_us);
+  p.stall = 1;
+  p.n_producers = 1;
+  p.w_tiled = 1;
+  p.w_packed = static_cast<const bf16*>(c->xb);  // never read
+  p.w_blocks = 1;
+  p.ep.y = c->x;
+  p.ep.ldy = c->cfg.d_model;
+  const CUtensorMap* tx;
+  TRY(get_tmap(c, c->xb, 32, 64, 32, &tx));
+  const size_t smem = tc::gemm_tc_smem_bytes(32, 128, p.stages);
+  TRY((launch_tc<EPI_F32, 128, 1>(c, tx, tx, p, 1, smem)));
+  return check_device_error(c);
+}
+extern "C" int d3_status_of_error_word(uint32_t w) {
+  if (w & ERRW_MBAR_TIMEOUT) return D3_ERR_DEVICE_TIMEOUT;
+  if (w) return D3_ERR_INVALID_ARG;
+  return D3_OK;
+}
+extern "C" int d3_commit_histogram(d3_ctx* c, int64_t* hist, int32_t n) {
+  if (!c || !hist || n <= 0) return D3_ERR_INVALID_ARG;
+  unsigned long long h[COMMIT_HIST_BINS];
+  CUDA_TRY(c, cudaMemcpyAsync(h, c->commit_hist, sizeof(h), cudaMemcpyDeviceToHost, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));
+  for (int i = 0; i < n; ++i) hist[i] = i < COMMIT_HIST_BINS ? static_cast<int64_t>(h[i]) : 0;
   return D3_OK;
 }
 extern "C" int d3_set_overlap(d3_ctx* c, int on) {

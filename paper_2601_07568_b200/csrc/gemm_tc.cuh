@@ -48,6 +48,8 @@ struct GemmParams {
   int* tile_count;  // arrival counters [tiles], zero on entry and on exit
   uint32_t* error_word;
   const int* skip_flag;  // optional: non-zero -> the whole launch is a no-op
+  uint32_t wait_limit_us;  // unit-range kernel: limit of every wait in microseconds (0: the default of ptx::mbar_wait)
+  int stall;               // unit-range kernel, give-up path probe: the producers issue no loads at all
   int n_producers;       // 1 or 2 TMA-issuing warps
   int rr;                // 1: whole tiles dealt round-robin in a rasterised order (wide matmuls), 0: contiguous unit ranges
   int gm;                // round-robin mode: row tiles per band
@@ -440,6 +442,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, n_cta = gridDim.x;
+  const uint64_t wait_ns = p.wait_limit_us != 0 ? static_cast<uint64_t>(p.wait_limit_us) * 1000ull : WAIT_LIMIT_NS;
   const long long U = p.total_units;
   const int KC = p.k_chunks;
   // Unit range of this CTA.  Round-robin mode (wide matmuls): the CTA owns whole tiles cta, cta + n,
@@ -495,7 +498,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
   if (warp == 0 || warp == 6) {
     // ---------------- TMA producers: warp 0 alone, or warps 0 and 6 taking alternate units
     const int n_prod = p.n_producers, pi = warp == 0 ? 0 : 1;
-    if (lane == 0 && pi < n_prod) {
+    if (lane == 0 && pi < n_prod && !p.stall) {
       const uint32_t tx = a_stage_bytes + b_stage_bytes;
       const long long n_total = u1 - u0;
       // Arms the stage's barrier with the bytes that will arrive and issues the weight loads.
@@ -553,7 +556,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
       int s = static_cast<int>(i % stages);
       uint32_t ph = (static_cast<uint32_t>(i / stages) & 1u) ^ 1u;  // parity to wait for on the empty barrier
       for (; i < n_total; i += n_prod) {
-        if (!mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word)) break;
+        if (!mbar_wait(&empty_bar[s], ph, abort_flag, p.error_word, wait_ns)) break;
         if (tile != mn_of) { tile_mn(tile, m_t, n_t); mn_of = tile; }
         load_w(s, n_t, kc);
         tma_load_2d(smem_a + static_cast<size_t>(s) * a_stage_bytes, &tmap_x, &full_bar[s], kc * BLOCK_K, m_t * (MT * BLOCK_M));
@@ -583,11 +586,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
         const int n_k = static_cast<int>(left < KC - kc0 ? left : KC - kc0);
         const int buf = seg & 1;
         // the epilogue must have drained this accumulator (two segments ago)
-        if (!mbar_wait(&acc_empty[buf], (static_cast<uint32_t>(seg >> 1) & 1u) ^ 1u, abort_flag, p.error_word)) break;
+        if (!mbar_wait(&acc_empty[buf], (static_cast<uint32_t>(seg >> 1) & 1u) ^ 1u, abort_flag, p.error_word, wait_ns)) break;
         tc_fence_after();
         const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * MT * BLOCK_N);
         for (int j = 0; j < n_k; ++j) {
-          if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word)) { ok = false; break; }
+          if (!mbar_wait(&full_bar[s], ph, abort_flag, p.error_word, wait_ns)) { ok = false; break; }
           tc_fence_after();
 #pragma unroll
           for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk) {
@@ -658,7 +661,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
           }
         }
       }
-      bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word);
+      bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(seg >> 1) & 1u, abort_flag, p.error_word, wait_ns);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();

@@ -39,9 +39,10 @@ __device__ __forceinline__ uint64_t global_ns() {
   return t;
 }
 // Bounded wait.  Returns false (and raises the error word and the CTA's abort flag) when the
-// phase did not complete within WAIT_LIMIT_NS or another role already gave up.
+// phase did not complete within the limit (WAIT_LIMIT_NS unless the caller passes a shorter one) or
+// another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t* error_word) {
+                                          uint32_t* error_word, uint64_t limit_ns = WAIT_LIMIT_NS) {
   // The common case must stay a bare try_wait loop: the clock is only read after 1024 failed
   // polls (reading %globaltimer on every blocking wait costs more than the wait itself).
   uint64_t t0 = 0;
@@ -51,7 +52,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       if (*abort_flag) return false;
       const uint64_t now = global_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > WAIT_LIMIT_NS) {
+      else if (now - t0 > limit_ns) {
         *abort_flag = 1;
         atomicOr(error_word, ERRW_MBAR_TIMEOUT);
         return false;

@@ -306,7 +306,8 @@ struct UnmaskOut {
 };
 __device__ __forceinline__ UnmaskOut unmask_block(const float* conf, const float* ent, const int* argmax, int* ids,
                                                   uint8_t* mask, int B, float tau, int mode, int* out_pos,
-                                                  int* out_ids, int* commit_step, int step, bool force = true) {
+                                                  int* out_ids, int* commit_step, int step, bool force = true,
+                                                  uint32_t* error_word = nullptr) {
   const int lane = threadIdx.x & 31;
   // pass 1: best masked position
   float best = -INFINITY;
@@ -330,7 +331,19 @@ __device__ __forceinline__ UnmaskOut unmask_block(const float* conf, const float
     }
   }
   UnmaskOut res{0, 0, 0};
-  if (best_r == 0x7fffffff) return res;  // nothing masked
+  if (best_r == 0x7fffffff) {
+    // no masked row compared greater than -inf: either nothing is masked, or every masked row's
+    // statistic is unusable (NaN compares false).  The block must still lose a mask per forward
+    // (Sec. 3.2, at-least-one rule), so the lowest masked row is forced and the error word is raised.
+    int first = 0x7fffffff;
+    for (int r = lane; r < B; r += 32)
+      if (mask[r] && r < first) first = r;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) first = min(first, __shfl_xor_sync(0xffffffffu, first, o));
+    if (first == 0x7fffffff) return res;  // nothing masked
+    best_r = first;
+    if (lane == 0 && error_word != nullptr) atomicOr(error_word, ERRW_BAD_STATISTIC);
+  }
   int base = 0;
   for (int r0 = 0; r0 < B; r0 += 32) {
     const int r = r0 + lane;
@@ -358,10 +371,11 @@ __device__ __forceinline__ UnmaskOut unmask_block(const float* conf, const float
 
 __global__ void unmask_kernel(const float* __restrict__ conf, const float* __restrict__ ent,
                               const int* __restrict__ argmax, int* ids, uint8_t* mask, int B, float tau, int mode,
-                              int* out_pos, int* out_ids, int* out_count) {
+                              int* out_pos, int* out_ids, int* out_count, uint32_t* error_word) {
   const int b = blockIdx.x;
   UnmaskOut r = unmask_block(conf + b * B, ent + b * B, argmax + b * B, ids + b * B, mask + b * B, B, tau, mode,
-                             out_pos ? out_pos + b * B : nullptr, out_ids ? out_ids + b * B : nullptr, nullptr, 0);
+                             out_pos ? out_pos + b * B : nullptr, out_ids ? out_ids + b * B : nullptr, nullptr, 0, true,
+                             error_word);
   if (threadIdx.x == 0 && out_count) out_count[b] = r.committed;
 }
 
@@ -388,7 +402,10 @@ struct GenState {
                         // [6] sequences stopped early on the end-of-sequence id, [7] sequences waiting for a KV-refresh
   int* hist;            // [bs, max_seq] ids of the stored prefix (prompt and stored blocks)
   int* refresh_flag;    // [bs] 1: the stored prefix of this sequence is to be recomputed before the next forward
+  unsigned long long* commit_hist;  // [COMMIT_HIST_BINS] decisions that committed k tokens (k = bin index)
+  uint32_t* error_word;
 };
+constexpr int COMMIT_HIST_BINS = 129;  // a block has at most 128 positions
 
 // Row map and input ids of the next decode forward (rows_per_seq = R, B or 2B) from the generate
 // state.  One block per sequence.
@@ -472,8 +489,9 @@ __global__ void gen_advance_kernel(GenState g, const float* __restrict__ conf, c
 #pragma unroll
   for (int q = 0; q < 4; ++q) was_masked[q] = lane + 32 * q < B && mask[lane + 32 * q] != 0;
   UnmaskOut r = unmask_block(conf + stat_row0, ent + stat_row0, argmax + stat_row0, ids, mask, B, tau, decide_mode,
-                             nullptr, nullptr, cs, step);
+                             nullptr, nullptr, cs, step, true, g.error_word);
   __syncwarp();
+  if (lane == 0) atomicAdd(&g.commit_hist[r.committed], 1ull);
   // early stop: the end-of-sequence id was committed in this step.  The sequence is done; its current
   // block goes out as it is (mask id where nothing was decided), later blocks stay mask ids, and the
   // unfinished block is not cached.
@@ -543,6 +561,8 @@ __global__ void gen_init_kernel(GenState g, int bs, int B, int mask_id, int gen_
       g.counters[4] = bs;
     }
   }
+  if (b == 0)
+    for (int i = threadIdx.x; i < COMMIT_HIST_BINS; i += blockDim.x) g.commit_hist[i] = 0ull;
 }
 
 // ----------------------------------------------------------------------------- multi-block decoding
@@ -564,6 +584,8 @@ struct MbState {
                         // [7] sequences stopped early on the end-of-sequence id
   int* stab;            // [bs, W] stabilizing forwards each block in flight has had
   int* hist;            // [bs, max_seq] ids of the stored prefix
+  unsigned long long* commit_hist;  // [COMMIT_HIST_BINS] block decisions that committed k tokens
+  uint32_t* error_word;
 };
 constexpr int MB_MAX_WINDOW = 8;
 
@@ -584,6 +606,8 @@ __global__ void mb_init_kernel(MbState g, int bs, int B, int W, int mask_id, int
       g.counters[5] = 1;
     }
   }
+  if (b == 0)
+    for (int i = threadIdx.x; i < COMMIT_HIST_BINS; i += blockDim.x) g.commit_hist[i] = 0ull;
 }
 
 // Row map and input ids of the next round (rows_per_seq = R >= the largest window).  One block per sequence.
@@ -652,7 +676,8 @@ __global__ void mb_advance_kernel(MbState g, const float* __restrict__ conf, con
       const int row0 = b * R + w * B;
       int* cr = g.commit_round ? g.commit_round + static_cast<size_t>(b) * gen_len + (lo + w) * B : nullptr;
       UnmaskOut r = unmask_block(conf + row0, ent + row0, argmax + row0, ids + w * B, mask + w * B, B, tau, decide_mode,
-                                 nullptr, nullptr, cr, round, fully);
+                                 nullptr, nullptr, cr, round, fully, g.error_word);
+      if (lane == 0) atomicAdd(&g.commit_hist[r.committed], 1ull);
       committed += r.committed;
       forced += r.forced;
       decisions += 1;

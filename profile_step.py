@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Run a few denoise steps of one workload shape, for profilers and quick timing.
 
-  python -m paper_2601_07568_b200.profile_step --workload c2 --layers 4 --steps 3
+  python profile_step.py --workload c2 --layers 4 --steps 3
 
 The model has the workload's architecture with ``--layers`` layers (default: all) and seeded random
 weights; the prompt is the workload's.  After prefill the script runs ``--steps`` denoise steps on a
@@ -17,7 +17,7 @@ import json
 import os
 import sys
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 

@@ -10,8 +10,8 @@ from paper_2601_07568_b200 import build as d3build
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
-def declared_functions():
-    src = open(os.path.join(ROOT, "include", "d3.h")).read()
+def declared_functions(header="d3.h"):
+    src = open(os.path.join(ROOT, "include", header)).read()
     src = re.sub(r"/\*.*?\*/", "", src, flags=re.S)
     return sorted(set(re.findall(r"\b(d3_[a-z0-9_]+)\s*\(", src)))
 
@@ -26,6 +26,10 @@ def test_header_functions_are_exported_and_bound():
     assert sorted(binding.EXPORTS) == names
     unbound = [n for n in names if not hasattr(binding, n)]
     assert not unbound, unbound
+    # the measurement / test switches of include/d3_debug.h
+    dbg = [n for n in declared_functions("d3_debug.h") if n not in ("d3_tuning", "d3_ctx")]
+    assert sorted(binding.DEBUG_EXPORTS) == dbg
+    assert not [n for n in dbg if not hasattr(L, n) or not hasattr(binding, n)]
 
 
 def test_host_only_entry_points():
@@ -38,6 +42,24 @@ def test_host_only_entry_points():
     assert L.d3_create(None, None, None) == binding.D3_ERR_INVALID_ARG
     assert L.d3_prefill(None, None, None, 1, 1) == binding.D3_ERR_INVALID_ARG
     assert L.d3_generate(None, 32, ctypes.c_float(0.9), 1, None, None, None) == binding.D3_ERR_INVALID_ARG
+
+
+def test_error_word_to_status_mapping():
+    """Host side of the give-up path: the status a call returns for a device error word."""
+    assert binding.d3_status_of_error_word(0) == binding.D3_OK
+    assert binding.d3_status_of_error_word(1) == binding.D3_ERR_DEVICE_TIMEOUT
+    for other in (2, 4, 8, 16, 2 | 4):
+        assert binding.d3_status_of_error_word(other) == binding.D3_ERR_INVALID_ARG
+    # the time-out bit wins over the others
+    assert binding.d3_status_of_error_word(1 | 2 | 16) == binding.D3_ERR_DEVICE_TIMEOUT
+
+
+def test_tuning_defaults_and_ranges():
+    t = binding.d3_tuning_defaults()
+    assert (t.ring_kb, t.ctas_per_sm, t.producers, t.tile_columns, t.attn_key_tiles) == (0, 0, 0, 0, 0)
+    assert (t.cluster_k_split, t.row_tile_pairs, t.round_robin, t.column_strips, t.strip_stages) == (-1, -1, 1, 0, 0)
+    assert ctypes.sizeof(binding.d3_tuning) == 10 * 4
+    assert binding.lib().d3_set_tuning(None, ctypes.byref(t)) == binding.D3_ERR_INVALID_ARG
 
 
 def test_struct_layouts_match_header():

@@ -179,12 +179,12 @@ def test_generate_fused_finalize_equals_separate_forwards(c1):
     w, model, ids, lens, ctx = c1
     ctx.prefill(ids, lens)
     tok_f, cs_f, st_f = ctx.generate(1, w.gen_len, 0.9)
-    d3.d3_set_matmul_tuning(ctx.ctx, 0, 0x100)  # every block finalized in a forward of its own
+    d3.d3_set_fused_finalize(ctx.ctx, False)  # every block finalized in a forward of its own
     try:
         ctx.prefill(ids, lens)
         tok_s, cs_s, st_s = ctx.generate(1, w.gen_len, 0.9)
     finally:
-        d3.d3_set_matmul_tuning(ctx.ctx, 0, 0)
+        d3.d3_set_fused_finalize(ctx.ctx, True)
     assert np.array_equal(tok_f, tok_s) and np.array_equal(cs_f, cs_s)
     assert st_f.denoise_forwards == st_s.denoise_forwards and st_f.finalize_forwards == st_s.finalize_forwards
     n_blocks = w.gen_len // w.block
@@ -205,7 +205,7 @@ def test_generate_fused_finalize_bf16_tensor_core():
     with Ctx(shape, W, block=32, max_batch=1, max_seq=wl.max_seq) as ctx:
         ctx.prefill(ids, lens)
         tok_f, cs_f, st_f = ctx.generate(1, 128, 0.9)
-        d3.d3_set_matmul_tuning(ctx.ctx, 0, 0x100)
+        d3.d3_set_fused_finalize(ctx.ctx, False)
         ctx.prefill(ids, lens)
         tok_s, cs_s, st_s = ctx.generate(1, 128, 0.9)
         assert ctx.error_word() == 0
@@ -315,10 +315,10 @@ def test_multiblock_decoding_fp32_equals_the_oracle(tau, mode):
         # one block in flight = block-by-block decoding
         ctx.prefill(ids, lens)
         tok1, _, _ = ctx.generate_multiblock(3, 64, tau, 1)
-        d3.d3_set_matmul_tuning(ctx.ctx, 0, 0x100)
+        d3.d3_set_fused_finalize(ctx.ctx, False)
         ctx.prefill(ids, lens)
         tok0, _, _ = ctx.generate(3, 64, tau)
-        d3.d3_set_matmul_tuning(ctx.ctx, 0, 0)
+        d3.d3_set_fused_finalize(ctx.ctx, True)
         assert np.array_equal(tok1, tok0)
         # too many rows for the workspaces, bad window
         with pytest.raises(d3.D3Error):
@@ -535,7 +535,7 @@ def test_column_strip_schedule_in_the_forward():
         ctx.prefill(ids, lens)
         base = ctx.logits(blk)
         n0 = d3.d3_launch_count_of(ctx.ctx, "gemm_strip_kernel")
-        d3.d3_set_matmul_tuning(ctx.ctx, 3 << 29, 0)
+        d3.d3_set_tuning(ctx.ctx, column_strips=3)
         ctx.prefill(ids, lens)
         forced = ctx.logits(blk)
         assert d3.d3_launch_count_of(ctx.ctx, "gemm_strip_kernel") >= n0 + 4 * shape.n_layers
