@@ -35,6 +35,10 @@ typedef struct d3_tuning {
   int32_t strip_stages;     /* explicit pipeline depth of the column-strip kernel, 0 = from ring_kb.  With two
                                issue pipelines every stage belongs to one pipeline, which takes an even
                                count: an odd one is refused (D3_ERR_UNSUPPORTED at the launch), not rounded */
+  int32_t chain;            /* decode forwards of up to 64 rows run the matmuls between two attention kernels
+                               as one persistent launch: -1 = when the shapes allow (default), 0 never */
+  int32_t chain_clusters;   /* clusters of four CTAs the chain launches use: 0 = as many as are resident at once
+                               (default); a smaller count is taken as given, a larger one is cut to that */
 } d3_tuning;
 void d3_tuning_defaults(d3_tuning *t);
 int d3_set_tuning(d3_ctx *ctx, const d3_tuning *t);

@@ -17,6 +17,7 @@
 #include <vector>
 
 #include "attention.cuh"
+#include "chain.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
@@ -109,6 +110,11 @@ struct d3_ctx {
   int tune_wide_tiles = -1;  // -1: by row count; 0 / 1: force 128- / 256-column tiles
   int tune_ring_kb = 0, tune_ctas_per_sm = 0;  // matmul tuning overrides (0 = default)
   int tune_strip_stages = 0;  // explicit pipeline depth of the column-strip kernel (0: from the ring size)
+  int tune_chain = -1;        // skinny decode matmuls as chains (chain.cuh): -1 when the shapes allow, 0 never
+  int chain_clusters = -1;    // clusters of the chain kernel that are resident at once (-1: not asked yet)
+  int chain_qkv_ks = 2;       // K parts of the QKV matmul inside a chain
+  int tune_chain_clusters = 0;  // 0: as many clusters as fit
+  unsigned int* chain_sync = nullptr;  // [n_layers + 1][CHAIN_MAX_OPS] border counters of a forward's chain launches
   unsigned long long* commit_hist = nullptr;  // [COMMIT_HIST_BINS] commits per decision of the latest generate call
   struct ProfPair { cudaEvent_t a, b; int cls; };
   std::vector<ProfPair> prof_pool;
@@ -584,6 +590,156 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
+// ---- chained skinny matmuls (chain.cuh)
+struct ChainSpec {
+  const void* X;   // activations [M, K] bf16
+  const void* W;   // tiled weights [N, K]
+  int N, K;
+  int kind, epi;
+  int ks = tc::CHAIN_C;  // CHAIN_KSPLIT: CTAs of a cluster that share a strip (K parts): 1, 2 or 4
+  EpiParams ep;
+};
+
+// Clusters of the chain kernel that can be resident at once with `smem` bytes per CTA (asked once per size).
+int chain_max_clusters(d3_ctx* c, size_t smem) {
+  static std::map<size_t, int> cache;
+  auto it = cache.find(smem);
+  if (it != cache.end()) return it->second;
+  if (cudaFuncSetAttribute(tc::chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return 0;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(c->n_sms / tc::CHAIN_C * tc::CHAIN_C));
+  cfg.blockDim = dim3(tc::CHAIN_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cudaLaunchAttribute at[1];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = tc::CHAIN_C;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, tc::chain_kernel, &cfg) != cudaSuccess) {
+    (void)cudaGetLastError();
+    n = 0;
+  }
+  cache[smem] = n;
+  return n;
+}
+
+// Can a forward of M rows run its matmuls as chains?  (bf16 tensor-core context with the fused QKV
+// epilogue and folded norms; all CTAs of a chain must be resident at once.)
+bool chain_usable(d3_ctx* c, int M) {
+  const d3_config& g = c->cfg;
+  if (c->tune_chain == 0 || !c->use_tc || !c->fuse_qkv || !c->fold_norm || !c->w_tiled || c->prof_on) return false;
+  if (M > 64) return false;
+  const int d = g.d_model, nq = g.n_q_heads * g.d_head, nkv = g.n_kv_heads * g.d_head, f = g.d_ffn;
+  if (d % 32 != 0 || (nq + 2 * nkv) % 32 != 0 || (2 * f) % 16 != 0) return false;
+  if ((nq + 63) / 64 < tc::CHAIN_C || (f + 63) / 64 < tc::CHAIN_C || (d + 63) / 64 < tc::CHAIN_C) return false;  // every rank of a K-split gets slabs
+  return true;
+}
+
+int run_chain(d3_ctx* c, const ChainSpec* ops, int n_ops, int M, const QkvExtra* qx, unsigned int* sync) {
+  const int a_rows = M <= 32 ? 32 : 64;
+  tc::ChainParams p{};
+  p.n_ops = n_ops;
+  p.M = M;
+  p.a_rows = a_rows;
+  p.sync = sync;
+  p.error_word = c->error_word;
+  p.skip_flag = c->skip_flag;
+  // the grid: as many clusters as are resident at once with the largest ring that is worth having
+  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 200) * 1024;
+  int n_clusters = c->chain_clusters;
+  if (n_clusters < 0) {
+    n_clusters = std::min(chain_max_clusters(c, budget + 4096), c->n_sms / tc::CHAIN_C);
+    c->chain_clusters = n_clusters;
+  }
+  if (c->tune_chain_clusters > 0) n_clusters = std::min(n_clusters, c->tune_chain_clusters);
+  if (n_clusters < 8) return fail(c, D3_ERR_UNSUPPORTED, "too few clusters of the chain kernel fit the device");
+  const int n_cta = n_clusters * tc::CHAIN_C;
+  int max_strip = 0, max_ksplit = 0;
+  const void* xs[3] = {nullptr, nullptr, nullptr};
+  for (int j = 0; j < n_ops; ++j) {
+    const ChainSpec& o = ops[j];
+    tc::ChainOp& d = p.op[j];
+    d.kind = o.kind; d.epi = o.epi; d.N = o.N; d.K = o.K;
+    d.ks = o.ks;
+    if (o.kind == tc::CHAIN_KSPLIT && (o.ks != 1 && o.ks != 2 && o.ks != 4)) return fail(c, D3_ERR_INVALID_ARG, "chain K-split must be 1, 2 or 4");
+    if (o.kind == tc::CHAIN_KSPLIT && (o.K + 63) / 64 < o.ks) return fail(c, D3_ERR_UNSUPPORTED, "fewer K slabs than K parts");
+    d.w = static_cast<const bf16*>(o.W);
+    d.ep = o.ep;
+    if ((reinterpret_cast<uintptr_t>(o.W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
+    int cols;
+    if (o.kind == tc::CHAIN_STRIP) {
+      const int U = o.N / 16;
+      cols = ((U + n_cta - 1) / n_cta) * 16;
+    } else {
+      const int U = o.N / 32, G = n_clusters * (tc::CHAIN_C / o.ks);
+      cols = ((U + G - 1) / G) * 32;
+      max_ksplit = std::max(max_ksplit, cols);
+    }
+    if (cols > 256) return fail(c, D3_ERR_UNSUPPORTED, "a chain strip would be wider than 256 columns");
+    max_strip = std::max(max_strip, cols);
+    int slot = -1;
+    for (int q = 0; q < 3; ++q)
+      if (xs[q] == o.X || xs[q] == nullptr) { slot = q; break; }
+    if (slot < 0) return fail(c, D3_ERR_UNSUPPORTED, "a chain reads at most three different activation buffers");
+    xs[slot] = o.X;
+    d.x_map = slot;
+  }
+  p.w_stage_bytes = static_cast<uint32_t>(max_strip) * 128u;
+  const size_t recv = tc::chain_recv_bytes(a_rows, std::max(max_ksplit, 32));
+  const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + p.w_stage_bytes;
+  int stages = static_cast<int>((budget > recv ? budget - recv : 0) / stage_bytes);
+  stages = std::max(2, std::min(stages, 16));
+  p.stages = stages;
+  if (qx) {
+    p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
+    p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
+    p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
+    p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
+  }
+  const CUtensorMap* tm[3];
+  for (int q = 0; q < 3; ++q) {
+    const void* X = xs[q] ? xs[q] : xs[0];
+    int K = 0;
+    for (int j = 0; j < n_ops; ++j)
+      if (ops[j].X == X) K = ops[j].K;
+    TRY(get_tmap(c, X, M, K, a_rows, &tm[q]));
+  }
+  const size_t smem = tc::chain_smem_bytes(a_rows, p.w_stage_bytes, stages, std::max(max_ksplit, 32));
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(tc::chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(n_cta));
+  cfg.blockDim = dim3(tc::CHAIN_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  at[na].id = cudaLaunchAttributeClusterDimension;
+  at[na].val.clusterDim.x = tc::CHAIN_C;
+  at[na].val.clusterDim.y = 1;
+  at[na].val.clusterDim.z = 1;
+  ++na;
+  if (c->pdl && !c->prof_on) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = na;
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, tc::chain_kernel, *tm[0], *tm[1], *tm[2], p, static_cast<int>(recv)));
+  LAUNCHED(c, "chain_kernel");
+  return D3_OK;
+}
+
 // Tile width: 128 columns while weight streaming dominates, 256 when
 // it is bound by the tensor pipe (from 512 rows on: a third less operand traffic per flop).
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
@@ -839,6 +995,58 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     ep.yb = static_cast<bf16*>(c->xb); ep.ssq_out = c->ssq;
   };
 
+  if (chain_usable(c, M)) {
+    // Skinny decode forward: the matmuls between two attention kernels run as one chain launch
+    // (O-proj -> gate/up -> down -> the next layer's QKV), see chain.cuh.
+    CUDA_TRY(c, cudaMemsetAsync(c->chain_sync, 0, sizeof(unsigned int) * static_cast<size_t>(g.n_layers + 1) * tc::CHAIN_MAX_OPS, c->stream));
+    auto qkv_spec = [&](int l) {
+      ChainSpec s{};
+      s.X = c->xb; s.W = c->wqkv[l]; s.N = nq + 2 * nkv; s.K = d; s.kind = tc::CHAIN_KSPLIT; s.epi = EPI_QKV;
+      s.ks = c->chain_qkv_ks;
+      s.ep.y = c->q; s.ep.ldy = nq;
+      after_norm(s.ep);
+      return s;
+    };
+    {
+      ChainSpec first = qkv_spec(0);
+      QkvExtra qx{rm, k_plane(c, 0), v_plane(c, 0)};
+      TRY(run_chain(c, &first, 1, M, &qx, c->chain_sync));
+    }
+    for (int l = 0; l < g.n_layers; ++l) {
+      if (l == c->tap_layer && M <= c->tap_rows)  // QKV reads the residual stream, it does not change it
+        CUDA_TRY(c, cudaMemcpyAsync(c->tap_in, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
+      TRY(run_attention(c, c->q, l, c->o, rm));
+      ChainSpec ops[tc::CHAIN_MAX_OPS];
+      int n = 0;
+      {
+        ChainSpec& s = ops[n++];
+        s = ChainSpec{};
+        s.X = c->o; s.W = c->wo[l]; s.N = d; s.K = nq; s.kind = tc::CHAIN_KSPLIT; s.epi = EPI_RESID;
+        s.ep.y = c->x; s.ep.ldy = d;
+        updates_resid(s.ep);
+      }
+      {
+        ChainSpec& s = ops[n++];
+        s = ChainSpec{};
+        s.X = c->xb; s.W = c->wgu[l]; s.N = 2 * f; s.K = d; s.kind = tc::CHAIN_STRIP; s.epi = EPI_SWIGLU;
+        s.ep.y = c->h; s.ep.ldy = f;
+        after_norm(s.ep);
+      }
+      {
+        ChainSpec& s = ops[n++];
+        s = ChainSpec{};
+        s.X = c->h; s.W = c->wd[l]; s.N = d; s.K = f; s.kind = tc::CHAIN_KSPLIT; s.epi = EPI_RESID;
+        s.ep.y = c->x; s.ep.ldy = d;
+        updates_resid(s.ep);
+      }
+      const bool more = l + 1 < g.n_layers;
+      if (more) ops[n++] = qkv_spec(l + 1);
+      QkvExtra qx{rm, more ? k_plane(c, l + 1) : nullptr, more ? v_plane(c, l + 1) : nullptr};
+      TRY(run_chain(c, ops, n, M, &qx, c->chain_sync + static_cast<size_t>(l + 1) * tc::CHAIN_MAX_OPS));
+      if (l == c->tap_layer && M <= c->tap_rows)  // after down; the next layer's QKV leaves the stream as it is
+        CUDA_TRY(c, cudaMemcpyAsync(c->tap_out, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
+    }
+  } else
   for (int l = 0; l < g.n_layers; ++l) {
     if (l == c->tap_layer && M <= c->tap_rows)
       CUDA_TRY(c, cudaMemcpyAsync(c->tap_in, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
@@ -1043,6 +1251,7 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   A_(c->gen.fwd_ids, sizeof(int) * 2 * static_cast<size_t>(g.max_batch) * g.block);
   A_(c->gen.counters, sizeof(long long) * 8);
   A_(c->commit_hist, sizeof(unsigned long long) * COMMIT_HIST_BINS);
+  A_(c->chain_sync, sizeof(unsigned int) * static_cast<size_t>(g.n_layers + 1) * tc::CHAIN_MAX_OPS);
   c->gen.commit_hist = c->commit_hist;
   c->mb.commit_hist = c->commit_hist;
   c->gen.error_word = c->error_word;
@@ -1678,6 +1887,7 @@ extern "C" void d3_tuning_defaults(d3_tuning* t) {
   t->cluster_k_split = -1;
   t->row_tile_pairs = -1;
   t->round_robin = 1;
+  t->chain = -1;
 }
 extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   if (!c || !t) return D3_ERR_INVALID_ARG;
@@ -1685,7 +1895,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
       (t->tile_columns != 0 && t->tile_columns != 128 && t->tile_columns != 256) || t->attn_key_tiles < 0 || t->attn_key_tiles > 7 ||
       t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
       (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
-      t->strip_stages > 32)
+      t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0)
     return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
   c->tune_ring_kb = t->ring_kb;
   c->tune_ctas_per_sm = t->ctas_per_sm;
@@ -1697,6 +1907,8 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   c->tune_no_rr = t->round_robin ? 0 : 1;
   c->tune_strip = t->column_strips;
   c->tune_strip_stages = t->strip_stages;
+  c->tune_chain = t->chain;
+  c->tune_chain_clusters = t->chain_clusters;
   return D3_OK;
 }
 extern "C" int d3_set_fused_finalize(d3_ctx* c, int on) {

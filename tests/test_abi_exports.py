@@ -57,8 +57,8 @@ def test_error_word_to_status_mapping():
 def test_tuning_defaults_and_ranges():
     t = binding.d3_tuning_defaults()
     assert (t.ring_kb, t.ctas_per_sm, t.producers, t.tile_columns, t.attn_key_tiles) == (0, 0, 0, 0, 0)
-    assert (t.cluster_k_split, t.row_tile_pairs, t.round_robin, t.column_strips, t.strip_stages) == (-1, -1, 1, 0, 0)
-    assert ctypes.sizeof(binding.d3_tuning) == 10 * 4
+    assert (t.cluster_k_split, t.row_tile_pairs, t.round_robin, t.column_strips, t.strip_stages, t.chain) == (-1, -1, 1, 0, 0, -1)
+    assert ctypes.sizeof(binding.d3_tuning) == 12 * 4 and t.chain_clusters == 0
     assert binding.lib().d3_set_tuning(None, ctypes.byref(t)) == binding.D3_ERR_INVALID_ARG
 
 

@@ -535,7 +535,7 @@ def test_column_strip_schedule_in_the_forward():
         ctx.prefill(ids, lens)
         base = ctx.logits(blk)
         n0 = d3.d3_launch_count_of(ctx.ctx, "gemm_strip_kernel")
-        d3.d3_set_tuning(ctx.ctx, column_strips=3)
+        d3.d3_set_tuning(ctx.ctx, column_strips=3, chain=0)
         ctx.prefill(ids, lens)
         forced = ctx.logits(blk)
         assert d3.d3_launch_count_of(ctx.ctx, "gemm_strip_kernel") >= n0 + 4 * shape.n_layers
