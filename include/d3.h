@@ -353,7 +353,7 @@ int d3_set_overlap(d3_ctx *ctx, int on);
  * records per launch). */
 enum { D3_PROF_GEMM_QKV = 0, D3_PROF_GEMM_O = 1, D3_PROF_GEMM_GATE_UP = 2, D3_PROF_GEMM_DOWN = 3,
        D3_PROF_GEMM_HEAD = 4, D3_PROF_GEMM_OTHER = 5, D3_PROF_ATTENTION = 6, D3_PROF_RMSNORM = 7,
-       D3_PROF_OTHER = 8, D3_PROF_CLASSES = 9 };
+       D3_PROF_OTHER = 8, D3_PROF_CHAIN = 9 /* a decode forward's layers as one launch */, D3_PROF_CLASSES = 10 };
 int d3_profile_enable(d3_ctx *ctx, int on);
 int d3_profile_read(d3_ctx *ctx, double *ms, int64_t *launches);
 

@@ -21,7 +21,7 @@ extern "C" {
  * d3_set_tuning().  INVALID_ARG for values outside the ranges given here. */
 typedef struct d3_tuning {
   int32_t ring_kb;          /* shared-memory ring per CTA in KB, 0 = default (about 100 KB for matmuls of up
-                               to 128 rows, 200 KB otherwise); at most 200 */
+                               to 128 rows, 200 KB otherwise; the whole CTA of a chain launch, default 222); at most 224 */
   int32_t ctas_per_sm;      /* CTAs per SM the work is dealt to, 0 = default; at most 3 */
   int32_t producers;        /* copy-issuing warps (unit-range kernel) or issue pipelines (column strips):
                                0 = default, 1 or 2 */
@@ -39,6 +39,8 @@ typedef struct d3_tuning {
                                as one persistent launch: -1 = when the shapes allow (default), 0 never */
   int32_t chain_clusters;   /* clusters of four CTAs the chain launches use: 0 = as many as are resident at once
                                (default); a smaller count is taken as given, a larger one is cut to that */
+  int32_t chain_l2_ahead;   /* weight slabs the chain's L2 prefetch warp runs ahead of the ring: -1 = default
+                               (0: no prefetch; measured neutral at 12 slabs and slower beyond), at most 256 */
 } d3_tuning;
 void d3_tuning_defaults(d3_tuning *t);
 int d3_set_tuning(d3_ctx *ctx, const d3_tuning *t);

@@ -348,7 +348,7 @@ def d3_lm_head_stats_static(x: torch.Tensor, w: torch.Tensor, scale: float, mask
 
 
 PROF_CLASSES = ("gemm_qkv", "gemm_o", "gemm_gate_up", "gemm_down", "gemm_head", "gemm_other", "attention",
-                "rmsnorm", "other")
+                "rmsnorm", "other", "chain")
 
 
 def d3_set_overlap(ctx, on: bool) -> None:
@@ -358,7 +358,7 @@ def d3_set_overlap(ctx, on: bool) -> None:
 class d3_tuning(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("ring_kb", "ctas_per_sm", "producers", "tile_columns", "attn_key_tiles",
                                           "cluster_k_split", "row_tile_pairs", "round_robin", "column_strips",
-                                          "strip_stages", "chain", "chain_clusters")]
+                                          "strip_stages", "chain", "chain_clusters", "chain_l2_ahead")]
 
 
 def d3_tuning_defaults() -> d3_tuning:

@@ -114,7 +114,12 @@ struct d3_ctx {
   int chain_clusters = -1;    // clusters of the chain kernel that are resident at once (-1: not asked yet)
   int chain_qkv_ks = 2;       // K parts of the QKV matmul inside a chain
   int tune_chain_clusters = 0;  // 0: as many clusters as fit
-  unsigned int* chain_sync = nullptr;  // [n_layers + 1][CHAIN_MAX_OPS] border counters of a forward's chain launches
+  int tune_chain_l2 = -1;       // weight slabs the chain's L2 prefetch runs ahead (-1: default, 0: off)
+  unsigned int* chain_sync = nullptr;  // [operators of the program] border counters of a forward's chain launches
+  void* chain_prog = nullptr;          // the forward's operators (tc::ChainOp) on the device
+  int chain_prog_ops = 0;
+  bool chain_prog_ready = false;
+  CUtensorMap kv_tmap32{};             // the cache with boxes of 32 rows (attention inside the chain)
   unsigned long long* commit_hist = nullptr;  // [COMMIT_HIST_BINS] commits per decision of the latest generate call
   struct ProfPair { cudaEvent_t a, b; int cls; };
   std::vector<ProfPair> prof_pool;
@@ -590,22 +595,13 @@ int run_linear_strip(d3_ctx* c, const void* X, const void* W, int M, int N, int 
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
-// ---- chained skinny matmuls (chain.cuh)
-struct ChainSpec {
-  const void* X;   // activations [M, K] bf16
-  const void* W;   // tiled weights [N, K]
-  int N, K;
-  int kind, epi;
-  int ks = tc::CHAIN_C;  // CHAIN_KSPLIT: CTAs of a cluster that share a strip (K parts): 1, 2 or 4
-  EpiParams ep;
-};
-
+// ---- the decode forward as a chain (chain.cuh)
 // Clusters of the chain kernel that can be resident at once with `smem` bytes per CTA (asked once per size).
 int chain_max_clusters(d3_ctx* c, size_t smem) {
   static std::map<size_t, int> cache;
   auto it = cache.find(smem);
   if (it != cache.end()) return it->second;
-  if (cudaFuncSetAttribute(tc::chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) != cudaSuccess) {
+  if (cudaFuncSetAttribute(tc::chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024) != cudaSuccess) {
     (void)cudaGetLastError();
     return 0;
   }
@@ -629,91 +625,132 @@ int chain_max_clusters(d3_ctx* c, size_t smem) {
   return n;
 }
 
-// Can a forward of M rows run its matmuls as chains?  (bf16 tensor-core context with the fused QKV
-// epilogue and folded norms; all CTAs of a chain must be resident at once.)
-bool chain_usable(d3_ctx* c, int M) {
+constexpr int CHAIN_OPS_PER_LAYER = 5;  // QKV, attention, O-proj, gate/up, down
+
+// Can a forward of bs x rows_per_seq rows run as a chain?  (bf16 tensor-core context with the fused QKV
+// epilogue and folded norms; every (sequence, kv head) pair gets a cluster; all CTAs resident at once.)
+bool chain_usable(d3_ctx* c, int bs, int rows_per_seq, int seg) {
   const d3_config& g = c->cfg;
-  if (c->tune_chain == 0 || !c->use_tc || !c->fuse_qkv || !c->fold_norm || !c->w_tiled || c->prof_on) return false;
+  if (c->tune_chain == 0 || !c->use_tc || !c->fuse_qkv || !c->fold_norm || !c->w_tiled || !c->attn_tc) return false;
+  const int M = bs * rows_per_seq;
   if (M > 64) return false;
   const int d = g.d_model, nq = g.n_q_heads * g.d_head, nkv = g.n_kv_heads * g.d_head, f = g.d_ffn;
   if (d % 32 != 0 || (nq + 2 * nkv) % 32 != 0 || (2 * f) % 16 != 0) return false;
   if ((nq + 63) / 64 < tc::CHAIN_C || (f + 63) / 64 < tc::CHAIN_C || (d + 63) / 64 < tc::CHAIN_C) return false;  // every rank of a K-split gets slabs
+  if ((g.n_q_heads / g.n_kv_heads) * rows_per_seq > 64) return false;  // packed rows of a kv head: one attention tile
+  if (seg > 0 && seg % 16 != 0) return false;                         // a 16-row group lies in one segment
+  if (rows_per_seq % 16 != 0 && (g.n_q_heads / g.n_kv_heads) > 1) return false;
   return true;
 }
 
-int run_chain(d3_ctx* c, const ChainSpec* ops, int n_ops, int M, const QkvExtra* qx, unsigned int* sync) {
+// The program of a forward: QKV, attention, O-proj, gate/up, down per layer.  Built once (all
+// buffers belong to the context) and kept on the device.
+int chain_build_program(d3_ctx* c) {
+  const d3_config& g = c->cfg;
+  const int d = g.d_model, nq = g.n_q_heads * g.d_head, nkv = g.n_kv_heads * g.d_head, f = g.d_ffn;
+  std::vector<tc::ChainOp> prog(static_cast<size_t>(g.n_layers) * CHAIN_OPS_PER_LAYER);
+  auto after_norm = [&](EpiParams& ep) {
+    ep.ssq_in = c->ssq; ep.ssq_chunks = (d + 31) / 32; ep.inv_k = 1.0f / static_cast<float>(d); ep.rms_eps = g.rms_eps;
+  };
+  auto updates_resid = [&](EpiParams& ep) {
+    ep.yb = static_cast<bf16*>(c->xb); ep.ssq_out = c->ssq;
+  };
+  // activation tensor maps of a launch: 0 = attention output (O-proj), 1 = residual copy (QKV, gate/up), 2 = FFN hidden (down)
+  for (int l = 0; l < g.n_layers; ++l) {
+    tc::ChainOp* o = &prog[static_cast<size_t>(l) * CHAIN_OPS_PER_LAYER];
+    for (int q = 0; q < CHAIN_OPS_PER_LAYER; ++q) {
+      o[q] = tc::ChainOp{};
+      o[q].layer = l;
+      o[q].ks = tc::CHAIN_C;
+    }
+    o[0].kind = tc::CHAIN_KSPLIT; o[0].epi = EPI_QKV; o[0].ks = c->chain_qkv_ks; o[0].N = nq + 2 * nkv; o[0].K = d; o[0].x_map = 1;
+    o[0].w = static_cast<const bf16*>(c->wqkv[l]);
+    o[0].ep.y = c->q; o[0].ep.ldy = nq;
+    after_norm(o[0].ep);
+    o[1].kind = tc::CHAIN_ATTN; o[1].w = static_cast<const bf16*>(c->q); o[1].ep.y = c->o;
+    o[2].kind = tc::CHAIN_KSPLIT; o[2].epi = EPI_RESID; o[2].N = d; o[2].K = nq; o[2].x_map = 0;
+    o[2].w = static_cast<const bf16*>(c->wo[l]);
+    o[2].ep.y = c->x; o[2].ep.ldy = d;
+    updates_resid(o[2].ep);
+    o[3].kind = tc::CHAIN_STRIP; o[3].epi = EPI_SWIGLU; o[3].N = 2 * f; o[3].K = d; o[3].x_map = 1;
+    o[3].w = static_cast<const bf16*>(c->wgu[l]);
+    o[3].ep.y = c->h; o[3].ep.ldy = f;
+    after_norm(o[3].ep);
+    o[4].kind = tc::CHAIN_KSPLIT; o[4].epi = EPI_RESID; o[4].N = d; o[4].K = f; o[4].x_map = 2;
+    o[4].w = static_cast<const bf16*>(c->wd[l]);
+    o[4].ep.y = c->x; o[4].ep.ldy = d;
+    updates_resid(o[4].ep);
+  }
+  const size_t bytes = prog.size() * sizeof(tc::ChainOp);
+  if (!c->chain_prog) {
+    ALLOC(c, c->chain_prog, bytes);
+    ALLOC(c, c->chain_sync, sizeof(unsigned int) * prog.size());
+  }
+  CUDA_TRY(c, cudaMemcpyAsync(c->chain_prog, prog.data(), bytes, cudaMemcpyHostToDevice, c->stream));
+  CUDA_TRY(c, cudaStreamSynchronize(c->stream));  // `prog` is a local
+  c->chain_prog_ops = static_cast<int>(prog.size());
+  // widest strips of the program, for the stage size and the receive buffer (they depend on the cluster count only)
+  c->chain_prog_ready = true;
+  return D3_OK;
+}
+
+// Launch operators [op_begin, op_end) of the forward's program.
+int run_chain(d3_ctx* c, int op_begin, int op_end, const RowMap& rm) {
+  ProfScope ps(c, D3_PROF_CHAIN);
+  const d3_config& g = c->cfg;
+  const int M = rm.bs * rm.rows_per_seq;
   const int a_rows = M <= 32 ? 32 : 64;
-  tc::ChainParams p{};
-  p.n_ops = n_ops;
-  p.M = M;
-  p.a_rows = a_rows;
-  p.sync = sync;
-  p.error_word = c->error_word;
-  p.skip_flag = c->skip_flag;
-  // the grid: as many clusters as are resident at once with the largest ring that is worth having
-  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 200) * 1024;
+  const int d = g.d_model, nq = g.n_q_heads * g.d_head, nkv = g.n_kv_heads * g.d_head, f = g.d_ffn;
+  // the grid: as many clusters as are resident at once (every CTA waits for every other at the borders)
   int n_clusters = c->chain_clusters;
   if (n_clusters < 0) {
-    n_clusters = std::min(chain_max_clusters(c, budget + 4096), c->n_sms / tc::CHAIN_C);
+    n_clusters = std::min(chain_max_clusters(c, 224 * 1024), c->n_sms / tc::CHAIN_C);
     c->chain_clusters = n_clusters;
   }
   if (c->tune_chain_clusters > 0) n_clusters = std::min(n_clusters, c->tune_chain_clusters);
-  if (n_clusters < 8) return fail(c, D3_ERR_UNSUPPORTED, "too few clusters of the chain kernel fit the device");
+  if (n_clusters < 8 || n_clusters < rm.bs * g.n_kv_heads)
+    return fail(c, D3_ERR_UNSUPPORTED, "the chain kernel needs a resident cluster per (sequence, kv head) pair");
   const int n_cta = n_clusters * tc::CHAIN_C;
-  int max_strip = 0, max_ksplit = 0;
-  const void* xs[3] = {nullptr, nullptr, nullptr};
-  for (int j = 0; j < n_ops; ++j) {
-    const ChainSpec& o = ops[j];
-    tc::ChainOp& d = p.op[j];
-    d.kind = o.kind; d.epi = o.epi; d.N = o.N; d.K = o.K;
-    d.ks = o.ks;
-    if (o.kind == tc::CHAIN_KSPLIT && (o.ks != 1 && o.ks != 2 && o.ks != 4)) return fail(c, D3_ERR_INVALID_ARG, "chain K-split must be 1, 2 or 4");
-    if (o.kind == tc::CHAIN_KSPLIT && (o.K + 63) / 64 < o.ks) return fail(c, D3_ERR_UNSUPPORTED, "fewer K slabs than K parts");
-    d.w = static_cast<const bf16*>(o.W);
-    d.ep = o.ep;
-    if ((reinterpret_cast<uintptr_t>(o.W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
-    int cols;
-    if (o.kind == tc::CHAIN_STRIP) {
-      const int U = o.N / 16;
-      cols = ((U + n_cta - 1) / n_cta) * 16;
-    } else {
-      const int U = o.N / 32, G = n_clusters * (tc::CHAIN_C / o.ks);
-      cols = ((U + G - 1) / G) * 32;
-      max_ksplit = std::max(max_ksplit, cols);
-    }
-    if (cols > 256) return fail(c, D3_ERR_UNSUPPORTED, "a chain strip would be wider than 256 columns");
-    max_strip = std::max(max_strip, cols);
-    int slot = -1;
-    for (int q = 0; q < 3; ++q)
-      if (xs[q] == o.X || xs[q] == nullptr) { slot = q; break; }
-    if (slot < 0) return fail(c, D3_ERR_UNSUPPORTED, "a chain reads at most three different activation buffers");
-    xs[slot] = o.X;
-    d.x_map = slot;
-  }
+  auto strip_cols = [&](int N, int unit, int groups) { return ((N / unit + groups - 1) / groups) * unit; };
+  const int qkv_cols = strip_cols(nq + 2 * nkv, 32, n_clusters * (tc::CHAIN_C / c->chain_qkv_ks));
+  const int o_cols = strip_cols(d, 32, n_clusters);
+  const int gu_cols = strip_cols(2 * f, 16, n_cta);
+  const int max_strip = std::max(std::max(qkv_cols, o_cols), gu_cols);
+  if (max_strip > 256) return fail(c, D3_ERR_UNSUPPORTED, "a chain strip would be wider than 256 columns");
+  tc::ChainParams p{};
+  p.prog = static_cast<const tc::ChainOp*>(c->chain_prog);
+  p.op_begin = op_begin; p.op_end = op_end;
+  p.M = M;
+  p.a_rows = a_rows;
   p.w_stage_bytes = static_cast<uint32_t>(max_strip) * 128u;
-  const size_t recv = tc::chain_recv_bytes(a_rows, std::max(max_ksplit, 32));
+  const size_t recv = std::max(std::max<size_t>(tc::chain_recv_bytes(a_rows, std::max(qkv_cols, o_cols)), sizeof(float) * tc::CHAIN_ARECV_FLOATS),
+                               static_cast<size_t>(tc::CHAIN_ASTAGES) * tc::CHAIN_ASTAGE_BYTES);
+  p.recv_bytes = static_cast<int>(recv);
+  p.l2_ahead = c->tune_chain_l2 >= 0 ? c->tune_chain_l2 : 0;  // off by default: measured neutral at 12 slabs, slower beyond
+  const size_t budget = (c->tune_ring_kb > 0 ? c->tune_ring_kb : 222) * 1024;  // whole CTA
   const size_t stage_bytes = static_cast<size_t>(a_rows) * 128 + p.w_stage_bytes;
-  int stages = static_cast<int>((budget > recv ? budget - recv : 0) / stage_bytes);
+  const size_t fixed = tc::chain_fixed_smem_bytes(recv, 16);
+  int stages = static_cast<int>((budget > fixed ? budget - fixed : 0) / stage_bytes);
   stages = std::max(2, std::min(stages, 16));
   p.stages = stages;
-  if (qx) {
-    p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
-    p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
-    p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
-    p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
-  }
-  const CUtensorMap* tm[3];
-  for (int q = 0; q < 3; ++q) {
-    const void* X = xs[q] ? xs[q] : xs[0];
-    int K = 0;
-    for (int j = 0; j < n_ops; ++j)
-      if (ops[j].X == X) K = ops[j].K;
-    TRY(get_tmap(c, X, M, K, a_rows, &tm[q]));
-  }
-  const size_t smem = tc::chain_smem_bytes(a_rows, p.w_stage_bytes, stages, std::max(max_ksplit, 32));
+  p.sync = c->chain_sync;
+  p.error_word = c->error_word;
+  p.skip_flag = c->skip_flag;
+  p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
+  p.rm = rm;
+  p.n_q_heads = g.n_q_heads; p.n_kv_heads = g.n_kv_heads; p.max_seq = g.max_seq;
+  p.kv_base = static_cast<bf16*>(c->kv);
+  p.kv_plane_rows = static_cast<long long>(g.max_batch) * g.n_kv_heads * g.max_seq;
+  p.scale_log2 = 1.4426950408889634f / std::sqrt(static_cast<float>(g.d_head));
+  const CUtensorMap *t_o, *t_xb, *t_h;
+  TRY(get_tmap(c, c->o, M, nq, a_rows, &t_o));
+  TRY(get_tmap(c, c->xb, M, d, a_rows, &t_xb));
+  TRY(get_tmap(c, c->h, M, f, a_rows, &t_h));
+  const size_t smem = tc::chain_smem_bytes(a_rows, p.w_stage_bytes, stages, recv);
+  if (smem > 224 * 1024) return fail(c, D3_ERR_UNSUPPORTED, "the chain kernel's shared memory does not fit");
   static bool attr_set = false;
   if (!attr_set) {
-    CUDA_TRY(c, cudaFuncSetAttribute(tc::chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+    CUDA_TRY(c, cudaFuncSetAttribute(tc::chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 224 * 1024));
     attr_set = true;
   }
   cudaLaunchConfig_t cfg{};
@@ -735,7 +772,7 @@ int run_chain(d3_ctx* c, const ChainSpec* ops, int n_ops, int M, const QkvExtra*
   }
   cfg.attrs = at;
   cfg.numAttrs = na;
-  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, tc::chain_kernel, *tm[0], *tm[1], *tm[2], p, static_cast<int>(recv)));
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, tc::chain_kernel, *t_o, *t_xb, *t_h, c->kv_tmap32, p));
   LAUNCHED(c, "chain_kernel");
   return D3_OK;
 }
@@ -995,56 +1032,22 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
     ep.yb = static_cast<bf16*>(c->xb); ep.ssq_out = c->ssq;
   };
 
-  if (chain_usable(c, M)) {
-    // Skinny decode forward: the matmuls between two attention kernels run as one chain launch
-    // (O-proj -> gate/up -> down -> the next layer's QKV), see chain.cuh.
-    CUDA_TRY(c, cudaMemsetAsync(c->chain_sync, 0, sizeof(unsigned int) * static_cast<size_t>(g.n_layers + 1) * tc::CHAIN_MAX_OPS, c->stream));
-    auto qkv_spec = [&](int l) {
-      ChainSpec s{};
-      s.X = c->xb; s.W = c->wqkv[l]; s.N = nq + 2 * nkv; s.K = d; s.kind = tc::CHAIN_KSPLIT; s.epi = EPI_QKV;
-      s.ks = c->chain_qkv_ks;
-      s.ep.y = c->q; s.ep.ldy = nq;
-      after_norm(s.ep);
-      return s;
-    };
-    {
-      ChainSpec first = qkv_spec(0);
-      QkvExtra qx{rm, k_plane(c, 0), v_plane(c, 0)};
-      TRY(run_chain(c, &first, 1, M, &qx, c->chain_sync));
-    }
-    for (int l = 0; l < g.n_layers; ++l) {
-      if (l == c->tap_layer && M <= c->tap_rows)  // QKV reads the residual stream, it does not change it
-        CUDA_TRY(c, cudaMemcpyAsync(c->tap_in, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
-      TRY(run_attention(c, c->q, l, c->o, rm));
-      ChainSpec ops[tc::CHAIN_MAX_OPS];
-      int n = 0;
-      {
-        ChainSpec& s = ops[n++];
-        s = ChainSpec{};
-        s.X = c->o; s.W = c->wo[l]; s.N = d; s.K = nq; s.kind = tc::CHAIN_KSPLIT; s.epi = EPI_RESID;
-        s.ep.y = c->x; s.ep.ldy = d;
-        updates_resid(s.ep);
-      }
-      {
-        ChainSpec& s = ops[n++];
-        s = ChainSpec{};
-        s.X = c->xb; s.W = c->wgu[l]; s.N = 2 * f; s.K = d; s.kind = tc::CHAIN_STRIP; s.epi = EPI_SWIGLU;
-        s.ep.y = c->h; s.ep.ldy = f;
-        after_norm(s.ep);
-      }
-      {
-        ChainSpec& s = ops[n++];
-        s = ChainSpec{};
-        s.X = c->h; s.W = c->wd[l]; s.N = d; s.K = f; s.kind = tc::CHAIN_KSPLIT; s.epi = EPI_RESID;
-        s.ep.y = c->x; s.ep.ldy = d;
-        updates_resid(s.ep);
-      }
-      const bool more = l + 1 < g.n_layers;
-      if (more) ops[n++] = qkv_spec(l + 1);
-      QkvExtra qx{rm, more ? k_plane(c, l + 1) : nullptr, more ? v_plane(c, l + 1) : nullptr};
-      TRY(run_chain(c, ops, n, M, &qx, c->chain_sync + static_cast<size_t>(l + 1) * tc::CHAIN_MAX_OPS));
-      if (l == c->tap_layer && M <= c->tap_rows)  // after down; the next layer's QKV leaves the stream as it is
-        CUDA_TRY(c, cudaMemcpyAsync(c->tap_out, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
+  if (chain_usable(c, bs, rows_per_seq, seg)) {
+    // Skinny decode forward: all layers in one persistent launch (chain.cuh); a tapped layer cuts it.
+    if (!c->chain_prog_ready) TRY(chain_build_program(c));
+    CUDA_TRY(c, cudaMemsetAsync(c->chain_sync, 0, sizeof(unsigned int) * static_cast<size_t>(c->chain_prog_ops), c->stream));
+    const int n_ops = c->chain_prog_ops;
+    const bool tap = c->tap_layer >= 0 && c->tap_layer < g.n_layers && M <= c->tap_rows;
+    if (!tap) {
+      TRY(run_chain(c, 0, n_ops, rm));
+    } else {
+      // the residual stream enters layer L before its O-proj (QKV and attention only read it) and leaves it after down
+      const int o_in = c->tap_layer * CHAIN_OPS_PER_LAYER + 2, o_out = (c->tap_layer + 1) * CHAIN_OPS_PER_LAYER;
+      TRY(run_chain(c, 0, o_in, rm));
+      CUDA_TRY(c, cudaMemcpyAsync(c->tap_in, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
+      TRY(run_chain(c, o_in, o_out, rm));
+      CUDA_TRY(c, cudaMemcpyAsync(c->tap_out, c->x, sizeof(float) * M * d, cudaMemcpyDeviceToDevice, c->stream));
+      if (o_out < n_ops) TRY(run_chain(c, o_out, n_ops, rm));
     }
   } else
   for (int l = 0; l < g.n_layers; ++l) {
@@ -1230,6 +1233,9 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
       int rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, attn::KT, &tm);
       if (rc_ != D3_OK) return bail(rc_);
       c->kv_tmap = *tm;
+      rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, tc::CHAIN_AKT, &tm);
+      if (rc_ != D3_OK) return bail(rc_);
+      c->kv_tmap32 = *tm;
       c->attn_tc = true;
     }
   }
@@ -1251,7 +1257,6 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
   A_(c->gen.fwd_ids, sizeof(int) * 2 * static_cast<size_t>(g.max_batch) * g.block);
   A_(c->gen.counters, sizeof(long long) * 8);
   A_(c->commit_hist, sizeof(unsigned long long) * COMMIT_HIST_BINS);
-  A_(c->chain_sync, sizeof(unsigned int) * static_cast<size_t>(g.n_layers + 1) * tc::CHAIN_MAX_OPS);
   c->gen.commit_hist = c->commit_hist;
   c->mb.commit_hist = c->commit_hist;
   c->gen.error_word = c->error_word;
@@ -1888,14 +1893,15 @@ extern "C" void d3_tuning_defaults(d3_tuning* t) {
   t->row_tile_pairs = -1;
   t->round_robin = 1;
   t->chain = -1;
+  t->chain_l2_ahead = -1;
 }
 extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   if (!c || !t) return D3_ERR_INVALID_ARG;
-  if (t->ring_kb < 0 || t->ring_kb > 200 || t->ctas_per_sm < 0 || t->ctas_per_sm > 3 || t->producers < 0 || t->producers > 2 ||
+  if (t->ring_kb < 0 || t->ring_kb > 224 || t->ctas_per_sm < 0 || t->ctas_per_sm > 3 || t->producers < 0 || t->producers > 2 ||
       (t->tile_columns != 0 && t->tile_columns != 128 && t->tile_columns != 256) || t->attn_key_tiles < 0 || t->attn_key_tiles > 7 ||
       t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
       (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
-      t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0)
+      t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256)
     return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
   c->tune_ring_kb = t->ring_kb;
   c->tune_ctas_per_sm = t->ctas_per_sm;
@@ -1909,6 +1915,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   c->tune_strip_stages = t->strip_stages;
   c->tune_chain = t->chain;
   c->tune_chain_clusters = t->chain_clusters;
+  c->tune_chain_l2 = t->chain_l2_ahead;
   return D3_OK;
 }
 extern "C" int d3_set_fused_finalize(d3_ctx* c, int on) {
