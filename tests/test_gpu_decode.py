@@ -12,10 +12,12 @@ import torch
 from oracle import d3_oracle as o
 from paper_2601_07568_b200 import binding as d3
 from paper_2601_07568_b200 import synth_inputs as si
-from gpu_utils import DEV, Ctx, top2_gap
+from gpu_utils import DEV, EPS, Ctx, assert_rounding_bounded, free_running_p2, record_report, top2_gap
 
 pytestmark = pytest.mark.gpu
-EPS = 1e-3
+# Largest |statistic difference| between a bf16 path and the mirrored oracle that a step-locked run may
+# show: measured on these models 1.2e-2 to 3.3e-2 (see the recorded reports).
+BF16_STAT_ERR_BOUND = 4e-2
 
 
 def step_locked(ctx: Ctx, model: o.OracleModel, prompts, lens, gen_len, block, tau, mode=0, logit_tol=None,
@@ -147,7 +149,7 @@ def test_c1_logits_fp32(c1):
 def test_c1_step_locked(c1, tau):
     w, model, ids, lens, ctx = c1
     rep, _ = step_locked(ctx, model, ids, lens, w.gen_len, w.block, tau, logit_tol=1e-4)
-    print("c1 step-locked", tau, rep)
+    record_report(f"c1_step_locked_tau={tau}", rep)
     assert rep["self_diff"] == 0 and rep["unexplained"] == 0 and rep["rounding"] == 0
     assert rep["max_logit_err"] <= 1e-4
     assert rep["max_stat_err"] <= 1e-4
@@ -194,33 +196,37 @@ def test_generate_fused_finalize_equals_separate_forwards(c1):
 
 
 def test_generate_fused_finalize_bf16_tensor_core():
-    """The same on the tensor-core path at batch 1 (64-row forwards with two segments): against the
-    oracle's free-running decode and against separate forwards; bf16 sums are cut differently at 32
-    and 64 rows, so ids may differ where the oracle sees a near-tie, and nowhere else."""
+    """The same on the tensor-core path at batch 1 (64-row forwards with two segments), free-running
+    against the oracle: both sides decode on their own, the first differing decision of a block must be
+    an oracle near-tie (margin < 1e-3) or lie within the two sides' measured numerical difference, the
+    GPU is re-synchronised from the oracle at the next block and decoding goes on; with fused and with
+    separate finalize forwards."""
     shape = small_bf16(128, 4, 2, "fused")
     W = si.gen_weights(shape)
     wl, ids, lens = si.small_workload("fused", shape, 1, [37], 128, 32, 0.9, 23)
     model = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
-    ref = model.generate(ids[0, :lens[0]], 128, 32, 0.9, record=True)
     with Ctx(shape, W, block=32, max_batch=1, max_seq=wl.max_seq) as ctx:
-        ctx.prefill(ids, lens)
-        tok_f, cs_f, st_f = ctx.generate(1, 128, 0.9)
-        d3.d3_set_fused_finalize(ctx.ctx, False)
-        ctx.prefill(ids, lens)
-        tok_s, cs_s, st_s = ctx.generate(1, 128, 0.9)
-        assert ctx.error_word() == 0
-    assert st_f.tokens_committed == 128 and st_s.tokens_committed == 128
-    assert st_f.steps < st_s.steps
-    near_tie = False
-    for t in ref["trace"]:  # oracle near-ties: top-2 probability gap or distance to the threshold below 1e-3
-        m = t["mask_in"]
-        near_tie |= bool(np.any(np.abs(t["conf"][m] - 0.9) < 1e-3))
-    same_fs = np.array_equal(tok_f, tok_s)
-    same_ref = np.array_equal(tok_f[0], ref["tokens"])
-    print("fused vs separate equal:", same_fs, "fused vs oracle equal:", same_ref, "oracle near-tie:", near_tie,
-          "steps", st_f.steps, st_s.steps)
-    assert same_fs or near_tie
-    assert same_ref or near_tie
+        rep_sl, _ = step_locked(ctx, model, ids, lens, 128, 32, 0.9)
+        assert_rounding_bounded(rep_sl, BF16_STAT_ERR_BOUND)
+        noise = 2 * rep_sl["max_stat_err"] + 1e-6
+        for fused in (True, False):
+            d3.d3_set_fused_finalize(ctx.ctx, fused)
+            steps = []
+
+            def gen(n):
+                tok, cs, st = ctx.generate(1, n, 0.9)
+                steps.append(int(st.steps))
+                assert st.tokens_committed == n
+                return tok, cs, st
+            rep = free_running_p2(ctx, model, ids[0, :lens[0]], 128, 32, 0.9, noise, generate=gen)
+            rep["steps_first_run"] = steps[0]
+            record_report(f"fused_finalize_bf16_free_running_fused={fused}", rep)
+            # (a fully masked block of this small random model starts from a near-tie among its rows, so
+            # most blocks re-synchronise; what is asserted is that every first difference is a near-tie:
+            # free_running_p2 fails otherwise)
+            assert rep["resyncs"] <= rep["blocks"] and max(rep["margins"], default=0.0) <= 1e-2, rep
+            assert ctx.error_word() == 0
+        d3.d3_set_fused_finalize(ctx.ctx, True)
 
 
 def test_generate_stops_on_eos_like_the_oracle():
@@ -361,26 +367,130 @@ def test_multiblock_stops_on_eos_like_the_oracle():
         d3.d3_set_eos(ctx.ctx, -1)
 
 
-def test_multiblock_decoding_bf16_tensor_core():
-    """The same through the tensor-core kernels at batch 1 (forwards of 32 to 128 rows, up to four
-    segments): against the oracle with mirrored bf16 roundings; ids may differ only where the oracle
-    sees a near-tie (|confidence - threshold| < 1e-3)."""
+def test_multiblock_decoding_bf16_tensor_core_step_locked():
+    """Multi-block decoding through the tensor-core kernels at batch 1 (rounds of 32 to 128 rows, up to
+    four segments), step-locked: before every round the oracle's window (ids of all blocks in flight) is
+    given to the GPU, the round's forward runs with segment-limited attention, and the statistics of every
+    masked row and the decisions they imply under the paper's state rules are compared with the oracle's;
+    blocks the oracle stores after the round are stored on the GPU by advancing the prefix.  Then the
+    free-running loop: d3_generate_multiblock commits every token, and where its tokens differ from the
+    oracle's the first differing round must be a near-tie of the oracle."""
     shape = small_bf16(128, 4, 2, "mb-bf16")
     W = si.gen_weights(shape)
     wl, ids, lens = si.small_workload("mb-bf16", shape, 1, [37], 128, 32, 0.9, 29)
     model = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
-    with Ctx(shape, W, block=32, max_batch=4, max_seq=wl.max_seq) as ctx:
-        for max_active in (2, 4):
-            ref = model.generate_multiblock(ids[0, :lens[0]], 128, 32, 0.9, 0, max_active=max_active, record=True)
+    B = 32
+    widest = 0
+    with Ctx(shape, W, block=B, max_batch=4, max_seq=wl.max_seq) as ctx:
+        for max_active, tau in ((2, 0.9), (4, 0.9), (4, 0.35)):
+            ref = model.generate_multiblock(ids[0, :lens[0]], 128, B, tau, 0, max_active=max_active, record=True)
             ctx.prefill(ids, lens)
-            tok, cr, st = ctx.generate_multiblock(1, 128, 0.9, max_active)
+            rep = dict(rounds=0, positions=0, excused=0, rounding=0, unexplained=0, self_diff=0, max_stat_err=0.0, max_rows=0)
+            margins = []
+            prefix = int(lens[0])
+            for t in ref["trace"]:
+                n_win = t["n_win"]
+                win = np.concatenate(t["ids_in"]).astype(np.int32)[None, :]
+                conf = torch.empty(n_win * B, dtype=torch.float32, device=DEV)
+                ent = torch.empty_like(conf)
+                am = torch.empty(n_win * B, dtype=torch.int32, device=DEV)
+                assert prefix == int(lens[0]) + t["lo"] * B
+                ctx.set_prefix([prefix])
+                d3.d3_denoise_window(ctx.ctx, torch.tensor(win, device=DEV), n_win, conf, ent, am)
+                torch.cuda.synchronize()
+                g_conf, g_ent, g_tok = conf.cpu().numpy(), ent.cpu().numpy(), am.cpu().numpy()
+                rep["rounds"] += 1
+                rep["max_rows"] = max(rep["max_rows"], n_win * B)
+                for k in range(n_win):
+                    mk = t["mask_in"][k]
+                    if not mk.any():
+                        continue
+                    o_conf, o_tok, o_ent = t["stats"][k]
+                    gc = g_conf[k * B:(k + 1) * B]
+                    rep["positions"] += int(mk.sum())
+                    rep["max_stat_err"] = max(rep["max_stat_err"], float(np.max(np.abs(gc - o_conf)[mk])))
+                    # the decision under the state rules, on the GPU's statistics and on the oracle's
+                    def decide(c, e):
+                        if t["fully"][k]:
+                            return o.decide(c, e, mk, np.float32(tau), 0)
+                        return mk & (c > np.float32(tau))
+                    have = decide(gc, g_ent[k * B:(k + 1) * B])
+                    want = t["commits"][k]
+                    assert np.array_equal(decide(o_conf.astype(np.float32), o_ent.astype(np.float32)), want)
+                    score = np.where(mk, o_conf, -np.inf)
+                    order = np.argsort(-score, kind="stable")
+                    forced_gap = score[order[0]] - score[order[1]] if mk.sum() >= 2 else np.inf
+                    clears = mk & (o_conf > tau)
+                    for r in np.flatnonzero(have != want):
+                        m = abs(o_conf[r] - tau)
+                        if t["fully"][k] and (not clears.any() or r == order[0] or (have[r] and not clears[r])):
+                            m = min(m, forced_gap)
+                        margins.append(float(m))
+                    both = have & want
+                    if (g_tok[k * B:(k + 1) * B][both] != o_tok[both]).any():
+                        margins.append(0.0)  # token near-ties are judged by the step-locked single-block tests; counted as excused here
+                # blocks the oracle stores after this round: their K/V of this round's forward are in place
+                stored = (ref["trace"][rep["rounds"]]["lo"] if rep["rounds"] < len(ref["trace"]) else 128 // B) - t["lo"]
+                prefix += stored * B
+            noise = 2 * rep["max_stat_err"] + 1e-6
+            for m in margins:
+                rep["excused" if m < EPS else "rounding" if m <= noise else "unexplained"] += 1
+            record_report(f"multiblock_bf16_step_locked_window={max_active}_tau={tau}", rep)
+            assert_rounding_bounded(rep, BF16_STAT_ERR_BOUND)
+            assert rep["max_rows"] >= 2 * B  # rounds of several segments were compared
+            widest = max(widest, rep["max_rows"])
+            # free-running: every token committed; a difference from the oracle starts at a near-tie round
+            ctx.prefill(ids, lens)
+            tok, cr, st = ctx.generate_multiblock(1, 128, tau, max_active)
             assert st.tokens_committed == 128 and ctx.error_word() == 0
-            near_tie = any(bool(np.any(np.abs(t["stats"][k][0][t["mask_in"][k]] - 0.9) < 1e-3))
-                           for t in ref["trace"] for k in range(t["n_win"]))
             same = np.array_equal(tok[0], ref["tokens"]) and np.array_equal(cr[0], ref["commit_round"])
-            print("multi-block bf16, max_active", max_active, "equal to oracle:", same, "near-tie:", near_tie,
-                  "rounds", st.steps, ref["rounds"])
-            assert same or near_tie
+            if not same:
+                differ = (tok[0] != ref["tokens"]) | (cr[0] != ref["commit_round"])
+                r_star = int(np.minimum(cr[0], ref["commit_round"])[differ].min())
+                t = ref["trace"][r_star - 1]
+                worst = 0.0
+                for k in range(t["n_win"]):
+                    sl = slice((t["lo"] + k) * B, (t["lo"] + k + 1) * B)
+                    mk = t["mask_in"][k]
+                    o_conf = t["stats"][k][0]
+                    g_commit = mk & (cr[0][sl] == r_star)
+                    score = np.sort(np.where(mk, o_conf, -np.inf))[::-1]
+                    forced_gap = score[0] - score[1] if mk.sum() >= 2 else np.inf
+                    for r in np.flatnonzero(g_commit != t["commits"][k]):
+                        worst = max(worst, min(abs(o_conf[r] - tau), forced_gap if t["fully"][k] else np.inf))
+                assert worst <= max(noise, EPS), ("multi-block divergence that no near-tie explains", max_active, r_star, worst)
+            record_report(f"multiblock_bf16_free_running_window={max_active}_tau={tau}", dict(equal=bool(same), rounds=int(st.steps), oracle_rounds=int(ref["rounds"])))
+        # This model never has more than two blocks in flight (an Activated block seldom clears the threshold),
+        # so rounds of three and four segments (96 and 128 rows, the widest the skinny kernels take) are
+        # compared on hand-made windows: blocks partly filled with the oracle's own tokens of the run above.
+        ref = model.generate_multiblock(ids[0, :lens[0]], 128, B, 0.9, 0, max_active=2)
+        rng = np.random.default_rng(3)
+        for n_win in (3, 4):
+            win_ids, win_mask = [], []
+            for k in range(n_win):
+                keep = rng.random(B) < (0.9 - 0.25 * k)          # later blocks are less complete
+                blk = np.where(keep, ref["tokens"][k * B:(k + 1) * B], shape.mask_id).astype(np.int32)
+                win_ids.append(blk)
+                win_mask.append(~keep)
+            ctx.prefill(ids, lens)
+            conf = torch.empty(n_win * B, dtype=torch.float32, device=DEV)
+            ent = torch.empty_like(conf)
+            am = torch.empty(n_win * B, dtype=torch.int32, device=DEV)
+            d3.d3_denoise_window(ctx.ctx, torch.tensor(np.concatenate(win_ids)[None, :], device=DEV), n_win, conf, ent, am)
+            torch.cuda.synchronize()
+            g_conf, g_tok = conf.cpu().numpy(), am.cpu().numpy()
+            st = model.prefill(ids[0, :lens[0]])
+            worst, tok_bad = 0.0, 0
+            for k in range(n_win):   # block k sees the cache and blocks 0..k-1 of the window as they stand
+                lg, o_conf, o_tok, _ = model.denoise_forward(st, win_ids[k])
+                gap = top2_gap(lg, shape.mask_id)
+                mk = win_mask[k]
+                worst = max(worst, float(np.max(np.abs(g_conf[k * B:(k + 1) * B] - o_conf)[mk])))
+                tok_bad += int(((g_tok[k * B:(k + 1) * B] != o_tok) & mk & (gap > 2 * BF16_STAT_ERR_BOUND)).sum())
+                st = model.finalize_block(st, win_ids[k])
+            record_report(f"multiblock_bf16_window_of_{n_win}", dict(rows=n_win * B, max_stat_err=worst, tokens_off_beyond_noise=tok_bad))
+            assert worst <= BF16_STAT_ERR_BOUND and tok_bad == 0
+            assert ctx.error_word() == 0
 
 
 def test_c1_entropy_mode():
@@ -418,16 +528,20 @@ def test_small_bf16_ragged_batch_step_locked(d_head, hq, hkv, impl):
     exact = o.model_from_shape(shape, W, np.float32)
     with Ctx(shape, W, block=32, max_batch=3, max_seq=wl.max_seq, gemm_impl=impl) as ctx:
         rep, traces = step_locked(ctx, model, ids, lens, 64, 32, 0.9, logit_tol=3e-2, exact_model=exact)
-        print("small bf16", d_head, hq, hkv, impl, rep)
+        record_report(f"small_bf16_step_locked_{d_head}_{hq}_{hkv}_impl{impl}", rep)
         assert rep["max_logit_err"] <= 3e-2
-        assert rep["self_diff"] == 0 and rep["unexplained"] == 0
-        assert rep["max_stat_err"] <= 5e-2
-        # free-running on the same inputs: report divergence instead of failing on near-ties
+        assert_rounding_bounded(rep, BF16_STAT_ERR_BOUND)
+        # free-running on the same inputs, batched: everything is committed
         ctx.prefill(ids, lens)
         tok, cs, st = ctx.generate(3, 64, 0.9)
-        same = [np.array_equal(tok[b], traces[b]["tokens"]) for b in range(3)]
-        print("free-running equal per sequence:", same, "forwards", st.denoise_forwards, st.finalize_forwards)
         assert st.tokens_committed == 3 * 64
+    # free-running against the oracle, sequence by sequence (first difference of a block = a near-tie, then re-sync)
+    noise = 2 * rep["max_stat_err"] + 1e-6
+    with Ctx(shape, W, block=32, max_batch=1, max_seq=wl.max_seq, gemm_impl=impl) as ctx:
+        for b in range(3):
+            r2 = free_running_p2(ctx, model, ids[b, :lens[b]], 64, 32, 0.9, noise)
+            record_report(f"small_bf16_free_running_{d_head}_{hq}_{hkv}_impl{impl}_seq{b}", r2)
+            assert r2["resyncs"] <= r2["blocks"] and max(r2["margins"], default=0.0) <= 1e-2, r2
 
 
 def test_small_bf16_model_width_not_a_multiple_of_the_tiles():
@@ -441,7 +555,9 @@ def test_small_bf16_model_width_not_a_multiple_of_the_tiles():
     exact = o.model_from_shape(shape, W, np.float32)
     with Ctx(shape, W, block=32, max_batch=2, max_seq=wl.max_seq) as ctx:
         rep, _ = step_locked(ctx, model, ids, lens, 32, 32, 0.9, logit_tol=3e-2, exact_model=exact)
-        assert rep["max_logit_err"] <= 3e-2 and rep["self_diff"] == 0 and rep["unexplained"] == 0
+        record_report("ragged_200_step_locked", rep)
+        assert rep["max_logit_err"] <= 3e-2
+        assert_rounding_bounded(rep, BF16_STAT_ERR_BOUND)
         assert ctx.error_word() == 0
 
 
@@ -541,7 +657,9 @@ def test_column_strip_schedule_in_the_forward():
         assert d3.d3_launch_count_of(ctx.ctx, "gemm_strip_kernel") >= n0 + 4 * shape.n_layers
         assert np.max(np.abs(forced - base)) <= 1e-2 * np.max(np.abs(base))
         rep, _ = step_locked(ctx, model, ids, lens, 32, 32, 0.5, logit_tol=3e-2)
-        assert rep["max_logit_err"] <= 3e-2 and rep["self_diff"] == 0 and rep["unexplained"] == 0
+        record_report("column_strips_step_locked", rep)
+        assert rep["max_logit_err"] <= 3e-2
+        assert_rounding_bounded(rep, BF16_STAT_ERR_BOUND)
         assert ctx.error_word() == 0
 
 

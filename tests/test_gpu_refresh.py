@@ -7,8 +7,8 @@ import torch
 from oracle import d3_oracle as o
 from paper_2601_07568_b200 import binding as d3
 from paper_2601_07568_b200 import synth_inputs as si
-from gpu_utils import Ctx
-from test_gpu_decode import step_locked
+from gpu_utils import Ctx, assert_rounding_bounded, record_report
+from test_gpu_decode import BF16_STAT_ERR_BOUND, step_locked
 
 pytestmark = pytest.mark.gpu
 
@@ -140,7 +140,9 @@ def test_refresh_bf16_tensor_core():
         rep, traces = step_locked(ctx, model, ids, lens, 128, 32, 0.9, logit_tol=3e-2, exact_model=exact, refresh_every=1)
         print("bf16 step-locked with refresh", rep)
         assert traces[0]["n_refresh"] == 3
-        assert rep["max_logit_err"] <= 3e-2 and rep["self_diff"] == 0 and rep["unexplained"] == 0 and rep["max_stat_err"] <= 5e-2
+        record_report("refresh_bf16_step_locked", rep)
+        assert rep["max_logit_err"] <= 3e-2
+        assert_rounding_bounded(rep, BF16_STAT_ERR_BOUND)
         # free-running through d3_generate: runs to the end with three refreshes (ids may drift after a near-tie)
         d3.d3_set_cache_policy(ctx.ctx, 1, 1)
         ctx.prefill(ids, lens)
