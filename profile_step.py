@@ -36,6 +36,7 @@ def main() -> int:
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=1)
     ap.add_argument("--prefix", type=int, default=0, help="override the cached prefix length (0 = after prefill)")
+    ap.add_argument("--no-chain", action="store_true", help="one kernel per matmul instead of the chain launch")
     args = ap.parse_args()
 
     d3build.build()
@@ -53,6 +54,8 @@ def main() -> int:
     del W
     ids_np, lens_np = si.gen_prompts(w)
     d3.d3_prefill(ctx, torch.from_numpy(ids_np).to(dev), torch.from_numpy(lens_np).to(dev))
+    if args.no_chain:
+        d3.d3_set_tuning(ctx, chain=0)
     if args.prefix > 0:
         d3.d3_set_state(ctx, torch.full((w.batch,), args.prefix, dtype=torch.int32, device=dev))
     bs, B = w.batch, w.block
