@@ -686,3 +686,52 @@ def test_empty_prompt_and_state_errors():
         lg = torch.zeros((64, shape.vocab), dtype=torch.float32, device=DEV)
         d3.d3_forward_logits(ctx.ctx, bad, lg)
         assert ctx.error_word() & 2  # token id outside the vocabulary is reported, not dereferenced
+
+
+@pytest.mark.parametrize("hq,hkv,bs,plens", [(4, 4, 1, [45]), (4, 2, 1, [45]), (4, 4, 2, [33, 7]), (2, 1, 2, [20, 64])])
+def test_chain_launch_small_models(hq, hkv, bs, plens):
+    """Decode forwards of up to 64 rows run all layers as one chain launch (QKV, attention, O-proj, gate/up
+    and down as operators of a program).  Small bf16 models that reach its variants: 32 packed rows per kv
+    head (two key parts per attention tile) and 64 (GQA group of two: four row groups), one and two
+    sequences (ragged prompts, a cluster per (sequence, kv head) pair), strips narrower than a cluster
+    count's worth of units (idle CTAs), and 64-row forwards of two segments in d3_generate.  Checked:
+    the launch really is the chain; logits against the per-kernel path (same arithmetic, other summation
+    order) and against the oracle; the step-locked trajectory; free-running decode with re-sync."""
+    shape = small_bf16(128, hq, hkv, f"chain-{hq}-{hkv}-{bs}")
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("chain", shape, bs, plens, 64, 32, 0.9, 31)
+    model = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
+    exact = o.model_from_shape(shape, W, np.float32)
+    blk = np.full((bs, 32), shape.mask_id, dtype=np.int32)
+    with Ctx(shape, W, block=32, max_batch=bs, max_seq=wl.max_seq) as ctx:
+        ctx.prefill(ids, lens)
+        n0 = d3.d3_launch_count_of(ctx.ctx, "chain_kernel")
+        got = ctx.logits(blk)
+        assert d3.d3_launch_count_of(ctx.ctx, "chain_kernel") == n0 + 1  # one launch for all layers
+        d3.d3_set_tuning(ctx.ctx, chain=0)
+        ctx.prefill(ids, lens)
+        base = ctx.logits(blk)
+        assert d3.d3_launch_count_of(ctx.ctx, "chain_kernel") == n0 + 1
+        d3.d3_set_tuning(ctx.ctx)
+        for b in range(bs):
+            assert np.max(np.abs(got[b] - base[b])) <= 1e-2 * np.max(np.abs(base[b]))
+        rep, _ = step_locked(ctx, model, ids, lens, 64, 32, 0.9, logit_tol=3e-2, exact_model=exact)
+        record_report(f"chain_step_locked_{hq}_{hkv}_bs{bs}", rep)
+        assert rep["max_logit_err"] <= 3e-2
+        assert_rounding_bounded(rep, BF16_STAT_ERR_BOUND)
+        # a tapped layer cuts the program into three launches; the forward's result does not change
+        ctx.prefill(ids, lens)
+        d3.d3_set_tap(ctx.ctx, 1)
+        n1 = d3.d3_launch_count_of(ctx.ctx, "chain_kernel")
+        tapped = ctx.logits(blk)
+        d3.d3_set_tap(ctx.ctx, -1)
+        assert d3.d3_launch_count_of(ctx.ctx, "chain_kernel") == n1 + 3
+        assert np.array_equal(tapped, got)
+        assert ctx.error_word() == 0
+        noise = 2 * rep["max_stat_err"] + 1e-6
+    if bs == 1:
+        with Ctx(shape, W, block=32, max_batch=1, max_seq=wl.max_seq) as ctx:
+            r2 = free_running_p2(ctx, model, ids[0, :lens[0]], 64, 32, 0.9, noise)
+            record_report(f"chain_free_running_{hq}_{hkv}", r2)
+            assert r2["resyncs"] <= r2["blocks"] and max(r2["margins"], default=0.0) <= 1e-2, r2
+            assert d3.d3_launch_count_of(ctx.ctx, "chain_kernel") > 0 and ctx.error_word() == 0
