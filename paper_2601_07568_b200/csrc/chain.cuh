@@ -11,9 +11,9 @@
 //
 // Grid: clusters of CHAIN_C = 4 CTAs, one CTA per SM, all resident at once (the host sizes the grid
 // from the occupancy of clusters).  Two ways of cutting a matmul Y[M,N] = X[M,K] . W[N,K]^T:
-//   * CHAIN_STRIP (QKV, gate/up: many columns): CTA i owns the column strip of units
+//   * CHAIN_STRIP (gate/up: many columns): CTA i owns the column strip of units
 //     [U i / n, U (i+1) / n) of 16 columns over the whole K range; the accumulator goes straight from
-//     tensor memory to the epilogue (RoPE + cache write, SwiGLU).  No reduction.
+//     tensor memory to the epilogue (SwiGLU; RoPE + cache write is supported too).  No reduction.
 //   * CHAIN_KSPLIT (O-proj, down: few columns, long K; QKV: so that a CTA does not re-read all of X
 //     for a narrow strip): ks = 4 or 2 CTAs of a cluster share a strip of 32-column units and take a
 //     ks-th of K each; the partial sums meet in distributed shared memory: a strip is cut into units of
@@ -58,10 +58,10 @@ enum : int { CHAIN_STRIP = 0, CHAIN_KSPLIT = 1, CHAIN_ATTN = 2 };
 constexpr int CHAIN_AKT = 32;      // keys per attention tile
 constexpr int CHAIN_ASTAGES = 3;   // attention tile ring: 3 x 16 KB
 constexpr uint32_t CHAIN_ASTAGE_BYTES = 4u * CHAIN_AKT * 128u;  // K lo, K hi, V lo, V hi slabs of [32][64] bf16
-constexpr int CHAIN_ARECV_FLOATS = 64 * attn::PART_LD;           // an owner's attention receive area: 64 (source, row) partials
+constexpr int CHAIN_ARECV_FLOATS = 64 * attn::PART_LD;           // attention's staging: 64 (key part, row) partial rows of (O, m, l)
 
 struct ChainOp {
-  int kind;   // CHAIN_STRIP / CHAIN_KSPLIT
+  int kind;   // CHAIN_STRIP / CHAIN_KSPLIT / CHAIN_ATTN
   int epi;    // CHAIN_STRIP: EPI_QKV or EPI_SWIGLU; CHAIN_KSPLIT: EPI_RESID or EPI_QKV
   int ks;     // CHAIN_KSPLIT: CTAs of a cluster that share a column strip and split K among them (1, 2 or 4);
               // the cluster then holds 4 / ks strips side by side
