@@ -41,6 +41,8 @@ typedef struct d3_tuning {
                                (default); a smaller count is taken as given, a larger one is cut to that */
   int32_t chain_l2_ahead;   /* weight slabs the chain's L2 prefetch warp runs ahead of the ring: -1 = default
                                (0: no prefetch; measured neutral at 12 slabs and slower beyond), at most 256 */
+  int32_t weights_as_rows;  /* matmuls of 129..256 rows with at most one 128-column tile per SM run with the weights as the
+                               MMA's 128-row operand and a K-splitting cluster per tile: -1 = when the shape allows, 0 never */
 } d3_tuning;
 void d3_tuning_defaults(d3_tuning *t);
 int d3_set_tuning(d3_ctx *ctx, const d3_tuning *t);

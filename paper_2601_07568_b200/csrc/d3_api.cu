@@ -21,6 +21,7 @@
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_xt.cuh"
 #include "small_kernels.cuh"
 
 using namespace d3;
@@ -115,6 +116,7 @@ struct d3_ctx {
   int chain_qkv_ks = 2;       // K parts of the QKV matmul inside a chain
   int tune_chain_clusters = 0;  // 0: as many clusters as fit
   int tune_chain_l2 = -1;       // weight slabs the chain's L2 prefetch runs ahead (-1: default, 0: off)
+  int tune_xt = -1;             // 129..256-row matmuls with weights as the 128-row operand: -1 when the shape allows, 0 never
   unsigned int* chain_sync = nullptr;  // [operators of the program] border counters of a forward's chain launches
   void* chain_prog = nullptr;          // the forward's operators (tc::ChainOp) on the device
   int chain_prog_ops = 0;
@@ -502,6 +504,96 @@ int run_linear_ck(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
 
+// Matmuls of 129..256 rows with few column tiles: weights as the 128-row MMA operand, a cluster per
+// 128-column tile of the output splitting K (gemm_xt_kernel).  Returns D3_ERR_UNSUPPORTED (without a
+// message) when the shape does not qualify; the caller then takes the unit-range kernel.
+template <int EPI>
+int launch_xt(d3_ctx* c, const CUtensorMap* tx, const tc::GemmParams& p, const tc::XtSplit& xs, int n_ctas, size_t smem) {
+  auto kern = tc::gemm_xt_kernel<EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024));
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(static_cast<unsigned>(n_ctas));
+  cfg.blockDim = dim3(tc::XT_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (xs.C > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = static_cast<unsigned>(xs.C);
+    at[na].val.clusterDim.y = 1;
+    at[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  if (c->pdl && !c->prof_on) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = na;
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, *tx, p, xs));
+  LAUNCHED(c, "gemm_xt_kernel");
+  return D3_OK;
+}
+
+bool xt_usable(const d3_ctx* c, int M, int N, int K, int epi, int w_tiled, tc::XtSplit* xs, int* stages) {
+  if (c->tune_xt == 0 || !w_tiled || M <= 128 || M > 256 || N % 128 != 0) return false;
+  if (epi != EPI_F32 && epi != EPI_T && epi != EPI_RESID) return false;
+  const int T = N / 128, KC = (K + 63) / 64;
+  if (T > c->n_sms) return false;  // many column tiles: the unit-range kernel with row-tile pairs shares weight slabs already
+  for (int C = 8; C >= 1; C >>= 1) {
+    if (T * C > c->n_sms || KC < 4 * C) continue;
+    const int n_cols = ((M + 32 * C - 1) / (32 * C)) * (32 * C);
+    if (n_cols > 256) continue;
+    const size_t stage_bytes = 128 * 128 + static_cast<size_t>(n_cols) * 128;
+    int st = static_cast<int>((200 * 1024) / stage_bytes);
+    st = std::max(2, std::min(st, 8));
+    if (C > 1 && static_cast<size_t>(st) * stage_bytes < static_cast<size_t>(n_cols) * 512) continue;  // the staged partials live in the ring
+    xs->C = C;
+    xs->n_cols = n_cols;
+    *stages = st;
+    return true;
+  }
+  return false;
+}
+
+int run_linear_xt(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep, const QkvExtra* qx,
+                  const tc::XtSplit& xs, int stages) {
+  if ((reinterpret_cast<uintptr_t>(W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
+  tc::GemmParams p{};
+  p.M = M; p.N = N; p.K = K;
+  p.a_rows = xs.n_cols;
+  p.k_chunks = (K + 63) / 64;
+  p.stages = stages;
+  p.error_word = c->error_word;
+  p.skip_flag = c->skip_flag;
+  p.w_tiled = 1;
+  p.w_packed = static_cast<const bf16*>(W);
+  p.w_blocks = static_cast<long long>(N / 128) * p.k_chunks;
+  p.ep = ep;
+  if (qx) {
+    p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
+    p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
+    p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
+    p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
+  }
+  const CUtensorMap* tx;
+  TRY(get_tmap(c, X, M, K, xs.n_cols, &tx));
+  const size_t smem = tc::gemm_xt_smem_bytes(xs.n_cols, stages);
+  const int n_ctas = (N / 128) * xs.C;
+  switch (epi) {
+    case EPI_F32: return launch_xt<EPI_F32>(c, tx, p, xs, n_ctas, smem);
+    case EPI_T: return launch_xt<EPI_T>(c, tx, p, xs, n_ctas, smem);
+    case EPI_RESID: return launch_xt<EPI_RESID>(c, tx, p, xs, n_ctas, smem);
+  }
+  return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
+}
+
 // Skinny matmuls with many columns as column strips over the whole K range (gemm_strip_kernel): the
 // narrowest strip (a multiple of 16 columns that divides N) whose CTAs are all resident at once.
 // Returns 0 when no strip width qualifies.
@@ -805,6 +897,11 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
     const int S = strip_width(c, M, N, w_tiled);
     // a residual epilogue that also writes chunk sums of squares needs whole 32-column chunks
     if (S > 0 && !(ep.ssq_out != nullptr && S % 32 != 0)) return run_linear_strip(c, X, W, M, N, K, epi, ep, S, qx);
+  }
+  if (ctas_hint == 0) {
+    tc::XtSplit xs{};
+    int xt_stages = 0;
+    if (xt_usable(c, M, N, K, epi, w_tiled, &xs, &xt_stages)) return run_linear_xt(c, X, W, M, N, K, epi, ep, qx, xs, xt_stages);
   }
   const bool wide = c->tune_wide_tiles >= 0 ? c->tune_wide_tiles != 0 : M >= 512;
   if (wide && N >= 256) return run_linear_tc_bn<256, 1>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
@@ -1894,6 +1991,7 @@ extern "C" void d3_tuning_defaults(d3_tuning* t) {
   t->round_robin = 1;
   t->chain = -1;
   t->chain_l2_ahead = -1;
+  t->weights_as_rows = -1;
 }
 extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   if (!c || !t) return D3_ERR_INVALID_ARG;
@@ -1901,7 +1999,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
       (t->tile_columns != 0 && t->tile_columns != 128 && t->tile_columns != 256) || t->attn_key_tiles < 0 || t->attn_key_tiles > 7 ||
       t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
       (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
-      t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256)
+      t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256 || t->weights_as_rows < -1 || t->weights_as_rows > 0)
     return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
   c->tune_ring_kb = t->ring_kb;
   c->tune_ctas_per_sm = t->ctas_per_sm;
@@ -1916,6 +2014,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   c->tune_chain = t->chain;
   c->tune_chain_clusters = t->chain_clusters;
   c->tune_chain_l2 = t->chain_l2_ahead;
+  c->tune_xt = t->weights_as_rows;
   return D3_OK;
 }
 extern "C" int d3_set_fused_finalize(d3_ctx* c, int on) {
