@@ -1,0 +1,454 @@
+// Block-bidirectional attention (Sec. 3.2: every row of the block sees the whole prefix and the block itself,
+// no causal mask) with both products on the tcgen05 tensor cores and the accumulators in tensor memory.
+// bf16, d_head = 128.
+//
+// One CTA = one (sequence, kv head, query tile, key split), 192 threads:
+//   warps 0-3  softmax: thread t owns row t of the tile = tensor-memory lane t
+//   warp 4     producer: K and V tiles of 128 keys by TMA (128-byte swizzle) into a ring of four 32 KB stages
+//   warp 5     one thread issues the MMAs; the warp owns the tensor-memory allocation (all 512 columns)
+// Per key tile i:  S_i = Q K_i^T (M = 128 rows, N = 128 keys, K = d_head; Q and K are K-major operands)
+//                  P_i = exp2(S_i * scale - m_i) as bf16, written by the softmax threads to shared memory in the
+//                        K-major swizzled layout of an A operand
+//                  O_i = P_i V_i (N = d_head, K = 128 keys; V as it lies in the cache, [key][d], is an MN-major
+//                        B operand: 64 d values = one 128-byte swizzle row, 8 keys = one 1024-byte atom)
+// S and O are double-buffered in tensor memory (columns 0-255 and 256-511), P in shared memory, so the MMAs of
+// tile i + 1 run under the softmax of tile i.  O_i is a fresh product per tile; the running output row stays in the
+// softmax thread's registers (acc = acc * 2^(m_old - m_new) + O_i), which keeps the rescaling off the tensor path.
+//
+// Fewer than 128 packed rows: with R <= 64 (R <= 32) rows the tile holds 2 (4) copies of the rows, copy c in lanes
+// c * 128 / COPIES ..., and copy c scores only keys [c, c + 1) * 128 / COPIES of every tile: its P rows are zero in
+// the other key columns (zeroed once, never written).  Every copy keeps its own running maximum and sum; the copies
+// are merged through shared memory after the last tile.  That divides the exponentials per thread by COPIES, which
+// is what paces a tile once its rows fit a single warp.
+//
+// Key splits: as in attn_tc_kernel, the CTAs of one query tile form a cluster along z and merge their partials
+// through distributed shared memory.
+#pragma once
+#include "attention.cuh"
+
+namespace d3 {
+namespace attn {
+
+constexpr int TKT = 128;                       // keys per tile
+constexpr int TM_STAGES = 4;                   // ring of K / V tiles
+constexpr uint32_t TM_SLAB = 128u * 128u;      // [128 rows][64 bf16], swizzled
+constexpr uint32_t TM_TILE = 2u * TM_SLAB;     // one K or V tile: d 0-63, d 64-127
+constexpr uint32_t TM_OFF_Q = 0;
+constexpr uint32_t TM_OFF_RING = TM_TILE;
+constexpr uint32_t TM_OFF_P = TM_OFF_RING + TM_STAGES * TM_TILE;
+constexpr uint32_t TM_OFF_BAR = TM_OFF_P + 2 * TM_TILE;
+constexpr int TM_THREADS = 192;
+
+// K-major operand slab, 128-byte swizzle: rows of 128 bytes, 8-row atoms 1024 bytes apart (stride byte offset);
+// the leading byte offset is not used by this form.  Bits: start address >> 4 in [0,14), LBO >> 4 in [16,30),
+// SBO >> 4 in [32,46), descriptor version 1 in [46,48), swizzle mode 2 (128 bytes) in [61,64).
+__device__ __forceinline__ uint64_t tm_desc_k(uint32_t smem_addr) {
+  return static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4) | (1ull << 16) | (static_cast<uint64_t>(1024 >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// MN-major operand, 128-byte swizzle: 64 consecutive MN elements per 128-byte row, one row per K index, atoms of
+// 8 K indices (1024 bytes) `sbo` bytes apart, blocks of 64 MN elements `lbo` bytes apart.
+__device__ __forceinline__ uint64_t tm_desc_mn(uint32_t smem_addr, uint32_t lbo, uint32_t sbo) {
+  return static_cast<uint64_t>((smem_addr & 0x3FFFF) >> 4) | (static_cast<uint64_t>(lbo >> 4) << 16) |
+         (static_cast<uint64_t>(sbo >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// kind::f16 instruction descriptor: D fp32, A and B bf16, A K-major, B K-major or MN-major (bit 16).
+__host__ __device__ constexpr uint32_t tm_idesc(int m, int n, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
+         (static_cast<uint32_t>(m >> 4) << 24);
+}
+__device__ __forceinline__ void tm_bar_softmax() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// grid (q_tiles, bs * hkv, n_splits); COPIES in {1, 2, 4}: 128 / COPIES packed rows per query tile.
+template <int COPIES>
+__global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_constant__ CUtensorMap tmap_kv,
+                                                                  const AttnTcParams p) {
+  constexpr int RPC = 128 / COPIES;  // packed rows of the tile
+  constexpr int KPC = TKT / COPIES;  // keys of a tile that one copy scores
+  constexpr int NCH = KPC / 32;      // 32-column chunks of S per thread
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + TM_OFF_BAR);
+  uint64_t* kv_empty = kv_full + TM_STAGES;
+  uint64_t* s_full = kv_empty + TM_STAGES;  // [2] S_i complete in tensor memory
+  uint64_t* p_full = s_full + 2;            // [2] P_i in shared memory, S_i and O_(i-2) read
+  uint64_t* o_full = p_full + 2;            // [2] O_i complete in tensor memory
+  uint64_t* q_full = o_full + 2;            // Q (and the zeroed P buffers) in shared memory
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_full + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp_id = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int qt = blockIdx.x, pair = blockIdx.y, split = blockIdx.z;
+  const int b = pair / p.hkv, g = pair % p.hkv;
+  const int group = p.hq / p.hkv;
+  const int rps = p.rm.rows_per_seq;
+
+  // The row map was written before this forward's first kernel started and cache rows below pos_base are not
+  // touched by this forward: both may be read before the dependency wait.
+  const int n_valid = p.rm.n_valid[b];
+  const int kv_len = p.rm.kv_len[b];
+  const int stable_keys = p.rm.pos_base[b];
+  const int R = group * rps;
+  bool work = !(qt * RPC >= R || n_valid <= 0 || kv_len <= 0);
+  if (work) {
+    bool any = false;
+    for (int pr = qt * RPC; pr < min(R, (qt + 1) * RPC) && !any; pr += 1) any = (pr % rps) < n_valid;
+    work = any;
+  }
+  if (!work) {  // uniform over the CTA and over the cluster
+    ptx::grid_dep_launch();
+    ptx::grid_dep_wait();
+    return;
+  }
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmap_kv);
+    for (int s = 0; s < TM_STAGES; ++s) {
+      ptx::mbar_init(&kv_full[s], 1);
+      ptx::mbar_init(&kv_empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(&s_full[s], 1);
+      ptx::mbar_init(&p_full[s], 128);
+      ptx::mbar_init(&o_full[s], 1);
+    }
+    ptx::mbar_init(q_full, 128);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp_id == 5) {
+    ptx::tmem_alloc<512>(tmem_slot);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  ptx::grid_dep_launch();
+
+  const int n_tiles = (kv_len + TKT - 1) / TKT;
+  const int tps = (n_tiles + p.n_splits - 1) / p.n_splits;
+  const int t0 = split * tps, t1 = min(n_tiles, t0 + tps);
+  const int n_my = max(t1 - t0, 0);
+  const uint32_t sbase = ptx::smem_u32(smem);
+  bool alive = true;
+
+  // Order in which the MMA thread consumes the tiles: K0, K1, V0, K2, V1, ..., K(n-1), V(n-2), V(n-1).
+  // Position of K_i: 0 for i = 0, else 2 i - 1.  Position of V_i: 2 n - 1 for the last, else 2 i + 2.
+  if (warp_id == 4) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      const long long krow = p.k_row0 + (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
+      const long long vrow = p.v_row0 + (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
+      bool waited = false;
+      for (int s = 0; s < 2 * n_my; ++s) {
+        const int stage = s % TM_STAGES;
+        if (s >= TM_STAGES &&
+            !ptx::mbar_wait(&kv_empty[stage], static_cast<uint32_t>(s / TM_STAGES - 1) & 1u, abort_flag, p.error_word))
+          break;
+        bool is_k;
+        int i;
+        if (s == 0) { is_k = true; i = 0; }
+        else if (s & 1) { i = (s + 1) / 2; is_k = i < n_my; if (!is_k) i = n_my - 1; }
+        else { is_k = false; i = (s - 2) / 2; }
+        const int j0 = (t0 + i) * TKT;
+        if (!waited && j0 + TKT > stable_keys) {  // this tile holds rows the QKV kernel of this layer writes
+          ptx::grid_dep_wait();
+          waited = true;
+        }
+        uint8_t* dst = smem + TM_OFF_RING + stage * TM_TILE;
+        const int row = static_cast<int>((is_k ? krow : vrow) + j0);
+        ptx::mbar_arrive_expect_tx(&kv_full[stage], TM_TILE);
+        ptx::tma_load_2d(dst, &tmap_kv, &kv_full[stage], 0, row);
+        ptx::tma_load_2d(dst + TM_SLAB, &tmap_kv, &kv_full[stage], 64, row);
+      }
+      if (!waited) ptx::grid_dep_wait();
+    }
+  } else if (warp_id == 5) {
+    // ------------------------------------------------------------------ MMA issue
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = tm_idesc(128, TKT, false);
+      constexpr uint32_t idesc_pv = tm_idesc(128, 128, true);
+      bool ok = ptx::mbar_wait(q_full, 0, abort_flag, p.error_word);
+      ptx::tc_fence_after();
+      auto qk = [&](int i) {  // S_i into S buffer i & 1
+        const int seq = i == 0 ? 0 : 2 * i - 1;
+        const int stage = seq % TM_STAGES;
+        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(seq / TM_STAGES) & 1u, abort_flag, p.error_word)) return false;
+        ptx::tc_fence_after();
+        const uint32_t kb = sbase + TM_OFF_RING + stage * TM_TILE;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+          const uint64_t a = tm_desc_k(sbase + TM_OFF_Q + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
+          const uint64_t bd = tm_desc_k(kb + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
+          ptx::umma_bf16(tmem_base + static_cast<uint32_t>((i & 1) * TKT), a, bd, idesc_qk, kk > 0 ? 1u : 0u);
+        }
+        ptx::umma_commit(&kv_empty[stage]);
+        ptx::umma_commit(&s_full[i & 1]);
+        return true;
+      };
+      if (ok && n_my > 0) ok = qk(0);
+      if (ok && n_my > 1) ok = qk(1);
+      for (int i = 0; i < n_my && ok; ++i) {
+        ok = ptx::mbar_wait(&p_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word);
+        if (!ok) break;
+        const int seq = i == n_my - 1 ? 2 * n_my - 1 : 2 * i + 2;
+        const int stage = seq % TM_STAGES;
+        ok = ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(seq / TM_STAGES) & 1u, abort_flag, p.error_word);
+        if (!ok) break;
+        ptx::tc_fence_after();
+        const uint32_t vb = sbase + TM_OFF_RING + stage * TM_TILE;
+        const uint32_t pb = sbase + TM_OFF_P + (i & 1) * TM_TILE;
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step
+          const uint64_t a = tm_desc_k(pb + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
+          const uint64_t bd = tm_desc_mn(vb + kk * 2048, TM_SLAB, 1024);
+          ptx::umma_bf16(tmem_base + 256u + static_cast<uint32_t>((i & 1) * 128), a, bd, idesc_pv, kk > 0 ? 1u : 0u);
+        }
+        ptx::umma_commit(&kv_empty[stage]);
+        ptx::umma_commit(&o_full[i & 1]);
+        if (i + 2 < n_my) ok = qk(i + 2);
+      }
+    }
+  }
+
+  // ------------------------------------------------------------------ softmax warps
+  const int tid = threadIdx.x;             // row of the tile and tensor-memory lane (warps 0-3)
+  const int copy = (tid & 127) / RPC;      // which copy of the rows, = which part of every tile's keys
+  const int lr = (tid & 127) % RPC;
+  const int pr = qt * RPC + lr;            // packed row: head_in_group * rows_per_seq + r
+  const int r_seq = pr % rps;
+  const bool row_ok = warp_id < 4 && pr < R && r_seq < n_valid;
+  float acc[128];
+  float m_run = -INFINITY, l_run = 0.f;
+  if (warp_id < 4) {
+    ptx::grid_dep_wait();  // Q comes from the kernel before this one
+    // Q rows into the two K-major slabs (d 0-63, d 64-127); rows that do not exist are zero
+    for (int e = tid; e < 128 * 16; e += 128) {
+      const int row = e >> 4, ch = e & 15;
+      const int pr2 = qt * RPC + row % RPC;
+      const int hg = pr2 / rps, r2 = pr2 % rps;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (pr2 < R && r2 < n_valid)
+        v = *reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(b) * rps + r2) * p.hq * 128 + (g * group + hg) * 128 + ch * 8);
+      *reinterpret_cast<uint4*>(smem + TM_OFF_Q + (ch >> 3) * TM_SLAB + swz(row, ch & 7)) = v;
+    }
+    if constexpr (COPIES > 1) {  // key columns of a P row that its copy never writes
+      for (int e = tid; e < static_cast<int>(2 * TM_TILE / 16); e += 128)
+        *reinterpret_cast<uint4*>(smem + TM_OFF_P + e * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    ptx::fence_proxy_async();
+    ptx::mbar_arrive(q_full);
+
+#pragma unroll
+    for (int d = 0; d < 128; ++d) acc[d] = 0.f;
+    const int kv_lim = row_ok ? row_kv_limit(p.rm, b, r_seq, kv_len) : kv_len;
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp_id * 32) << 16);
+    float alpha_prev = 1.f;
+    auto add_o = [&](int i, float alpha) {  // acc = acc * alpha + O_i
+      if (!ptx::mbar_wait(&o_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word)) return false;
+      ptx::tc_fence_after();
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) {
+        float o[32];
+        ptx::tmem_ld_32x32(t_lane + 256u + static_cast<uint32_t>((i & 1) * 128 + c4 * 32), o);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) acc[c4 * 32 + c] = fmaf(acc[c4 * 32 + c], alpha, o[c]);
+      }
+      return true;
+    };
+    for (int i = 0; i < n_my && alive; ++i) {
+      alive = ptx::mbar_wait(&s_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word);
+      if (!alive) break;
+      ptx::tc_fence_after();
+      const int j0 = (t0 + i) * TKT + copy * KPC;  // first key this thread scores
+      const uint32_t t_s = t_lane + static_cast<uint32_t>((i & 1) * TKT + copy * KPC);
+      float s[32];
+      // ---- row maximum over the keys this row may see
+      float mx = -INFINITY;
+#pragma unroll
+      for (int ch = 0; ch < NCH; ++ch) {
+        ptx::tmem_ld_32x32(t_s + ch * 32, s);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) {
+          if (j0 + ch * 32 + c >= kv_lim) s[c] = -INFINITY;
+          mx = fmaxf(mx, s[c]);
+        }
+      }
+      const float m_new = fmaxf(m_run, mx * p.scale_log2);
+      const float base = m_new == -INFINITY ? 0.f : m_new;  // no key seen yet: exponentials against 0 give 0, not NaN
+      const float alpha = exp2f(m_run - base);
+      m_run = m_new;
+      // ---- P = exp2(S * scale - m) as bf16 into the A-operand layout; row sum in fp32
+      float sum = 0.f;
+      uint8_t* prow = smem + TM_OFF_P + (i & 1) * TM_TILE;
+#pragma unroll
+      for (int ch = 0; ch < NCH; ++ch) {
+        if constexpr (NCH > 1) {  // a single chunk is still in registers
+          ptx::tmem_ld_32x32(t_s + ch * 32, s);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (j0 + ch * 32 + c >= kv_lim) s[c] = -INFINITY;
+        }
+        uint32_t pk[16];
+#pragma unroll
+        for (int c = 0; c < 32; c += 2) {
+          const float p0 = exp2f(fmaf(s[c], p.scale_log2, -base));
+          const float p1 = exp2f(fmaf(s[c + 1], p.scale_log2, -base));
+          sum += p0 + p1;
+          pk[c >> 1] = pack_bf16(p0, p1);
+        }
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {  // four 16-byte chunks of 8 keys
+          const int kc = (copy * KPC + ch * 32) / 8 + q4;  // chunk of the tile's 16
+          *reinterpret_cast<uint4*>(prow + (kc >> 3) * TM_SLAB + swz(tid, kc & 7)) =
+              make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+        }
+      }
+      l_run = l_run * alpha + sum;
+      ptx::fence_proxy_async();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(&p_full[i & 1]);
+      // ---- the product of the tile before, which ran under the work above
+      if (i > 0) alive = add_o(i - 1, alpha_prev);
+      alpha_prev = alpha;
+    }
+    if (alive && n_my > 0) alive = add_o(n_my - 1, alpha_prev);
+  }
+
+  // ------------------------------------------------------------------ output
+  auto out_ptr = [&](int prow) -> __nv_bfloat16* {
+    const int hg = prow / rps, r = prow % rps;
+    return p.out + (static_cast<size_t>(b) * rps + r) * p.hq * 128 + (g * group + hg) * 128;
+  };
+  // Partials [COPIES][RPC][PART_LD] over the ring: every load into it has been consumed once the last O is read.
+  float* red = reinterpret_cast<float*>(smem + TM_OFF_RING);
+  if (warp_id < 4) {
+    if (COPIES == 1 && p.n_splits == 1) {
+      if (alive && row_ok) {
+        const float inv = 1.0f / l_run;
+        __nv_bfloat16* o = out_ptr(pr);
+#pragma unroll
+        for (int d = 0; d < 128; d += 8)
+          *reinterpret_cast<uint4*>(o + d) =
+              make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv), pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
+                         pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv), pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+      }
+    } else {
+      float* rr = red + static_cast<size_t>(tid) * PART_LD;  // tid = copy * RPC + lr
+#pragma unroll
+      for (int d = 0; d < 128; d += 4) *reinterpret_cast<float4*>(rr + d) = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
+      rr[128] = m_run;  // a copy or split without keys leaves m = -inf, l = 0
+      rr[129] = l_run;
+      tm_bar_softmax();
+      if constexpr (COPIES > 1) {
+        // one thread per (row, 4 output dims); everything is read before anything of copy 0 is overwritten
+        constexpr int EPT = RPC * 32 / 128;
+        float4 mg[EPT];
+        float Ms[EPT], Ls[EPT];
+#pragma unroll
+        for (int j = 0; j < EPT; ++j) {
+          const int e = tid + j * 128;
+          const int row = e >> 5, c4 = (e & 31) * 4;
+          mg[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          Ms[j] = -INFINITY;
+          Ls[j] = 0.f;
+          float mq[COPIES], lq[COPIES];
+#pragma unroll
+          for (int q2 = 0; q2 < COPIES; ++q2) {
+            const float* r = red + (static_cast<size_t>(q2) * RPC + row) * PART_LD;
+            mq[q2] = r[128];
+            lq[q2] = r[129];
+            Ms[j] = fmaxf(Ms[j], mq[q2]);
+          }
+#pragma unroll
+          for (int q2 = 0; q2 < COPIES; ++q2) {  // copies in index order: fixed order of the sums
+            if (lq[q2] != 0.f) {
+              const float w = exp2f(mq[q2] - Ms[j]);
+              const float4 v = *reinterpret_cast<const float4*>(red + (static_cast<size_t>(q2) * RPC + row) * PART_LD + c4);
+              Ls[j] += w * lq[q2];
+              mg[j].x += w * v.x; mg[j].y += w * v.y; mg[j].z += w * v.z; mg[j].w += w * v.w;
+            }
+          }
+        }
+        if (p.n_splits == 1) {
+          if (alive) {
+#pragma unroll
+            for (int j = 0; j < EPT; ++j) {
+              const int e = tid + j * 128;
+              const int row = e >> 5, c4 = (e & 31) * 4;
+              const int prow = qt * RPC + row;
+              if (prow >= R || (prow % rps) >= n_valid) continue;
+              const float inv = 1.0f / Ls[j];
+              *reinterpret_cast<uint2*>(out_ptr(prow) + c4) =
+                  make_uint2(pack_bf16(mg[j].x * inv, mg[j].y * inv), pack_bf16(mg[j].z * inv, mg[j].w * inv));
+            }
+          }
+        } else {
+          tm_bar_softmax();
+#pragma unroll
+          for (int j = 0; j < EPT; ++j) {
+            const int e = tid + j * 128;
+            const int row = e >> 5, c4 = (e & 31) * 4;
+            float* r = red + static_cast<size_t>(row) * PART_LD;
+            *reinterpret_cast<float4*>(r + c4) = mg[j];
+            if (c4 == 0) { r[128] = Ms[j]; r[129] = Ls[j]; }
+          }
+        }
+      }
+    }
+  }
+  if (p.n_splits > 1) {  // merge over the key splits: every CTA of the cluster takes a slice of the rows
+    __syncwarp();
+    ptx::cluster_sync_all();
+    if (warp_id < 4) {
+      const int S = p.n_splits;
+      const int rank = static_cast<int>(ptx::cluster_ctarank());
+      const int rpr = (RPC + S - 1) / S;
+      const int row0 = rank * rpr, row1 = min(RPC, row0 + rpr);
+      const uint32_t red_addr = ptx::smem_u32(red);
+      for (int e = tid; e < (row1 - row0) * 32; e += 128) {
+        const int row = row0 + (e >> 5), c4 = (e & 31) * 4;
+        const int prow = qt * RPC + row;
+        if (prow >= R || (prow % rps) >= n_valid) continue;
+        const uint32_t off = static_cast<uint32_t>(row * PART_LD) * 4u;
+        float ms[8], ls[8];
+        float4 vs[8];
+        float M = -INFINITY;
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {
+          if (s2 < S) {
+            const uint32_t a = ptx::map_to_cta(red_addr + off, static_cast<uint32_t>(s2));
+            ms[s2] = ptx::ld_cluster_f(a + 128 * 4);
+            ls[s2] = ptx::ld_cluster_f(a + 129 * 4);
+            vs[s2] = ptx::ld_cluster_f4(a + c4 * 4);
+            M = fmaxf(M, ms[s2]);
+          }
+        }
+        float L = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int s2 = 0; s2 < 8; ++s2) {
+          if (s2 < S && ls[s2] != 0.f) {
+            const float w = exp2f(ms[s2] - M);
+            L += w * ls[s2];
+            a0 += w * vs[s2].x; a1 += w * vs[s2].y; a2 += w * vs[s2].z; a3 += w * vs[s2].w;
+          }
+        }
+        const float inv = 1.0f / L;
+        *reinterpret_cast<uint2*>(out_ptr(prow) + c4) = make_uint2(pack_bf16(a0 * inv, a1 * inv), pack_bf16(a2 * inv, a3 * inv));
+      }
+    }
+    __syncwarp();
+    ptx::cluster_sync_all();  // no CTA may leave while a peer still reads its partial
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp_id == 5) ptx::tmem_dealloc<512>(tmem_base);
+}
+
+inline size_t attn_tmem_smem_bytes() { return 1024 + TM_OFF_BAR + (2 * TM_STAGES + 7) * 8 + 64; }
+
+}  // namespace attn
+}  // namespace d3

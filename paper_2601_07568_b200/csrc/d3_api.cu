@@ -17,6 +17,7 @@
 #include <vector>
 
 #include "attention.cuh"
+#include "attention_tmem.cuh"
 #include "chain.cuh"
 #include "common.cuh"
 #include "gemm_simt.cuh"
@@ -116,11 +117,13 @@ struct d3_ctx {
   int chain_qkv_ks = 2;       // K parts of the QKV matmul inside a chain
   int tune_chain_clusters = 0;  // 0: as many clusters as fit
   int tune_chain_l2 = -1;       // weight slabs the chain's L2 prefetch runs ahead (-1: default, 0: off)
+  int tune_attn_tmem = -1;      // tcgen05 attention: -1 where measured faster, 0 never, 1 wherever the shape allows
   int tune_xt = -1;             // 129..256-row matmuls with weights as the 128-row operand: -1 when the shape allows, 0 never
   unsigned int* chain_sync = nullptr;  // [operators of the program] border counters of a forward's chain launches
   void* chain_prog = nullptr;          // the forward's operators (tc::ChainOp) on the device
   int chain_prog_ops = 0;
   bool chain_prog_ready = false;
+  CUtensorMap kv_tmap128{};            // the cache with boxes of 128 rows (attn_tmem_kernel)
   CUtensorMap kv_tmap32{};             // the cache with boxes of 32 rows (attention inside the chain)
   unsigned long long* commit_hist = nullptr;  // [COMMIT_HIST_BINS] commits per decision of the latest generate call
   struct ProfPair { cudaEvent_t a, b; int cls; };
@@ -1009,10 +1012,88 @@ int attn_ctas_per_sm() {
   return cached;
 }
 
+// tcgen05 attention launch: copies of the rows from the packed rows per kv head, key splits so that the
+// CTAs (one per SM: the kernel takes all of tensor memory and nearly all shared memory) fill whole waves.
+template <int COPIES>
+int launch_attn_tmem(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
+  auto kern = attn::attn_tmem_kernel<COPIES>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::attn_tmem_smem_bytes())));
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(attn::TM_THREADS);
+  cfg.dynamicSmemBytes = attn::attn_tmem_smem_bytes();
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  int na = 0;
+  if (grid.z > 1) {
+    at[na].id = cudaLaunchAttributeClusterDimension;
+    at[na].val.clusterDim.x = 1;
+    at[na].val.clusterDim.y = 1;
+    at[na].val.clusterDim.z = grid.z;
+    ++na;
+  }
+  if (c->pdl && !c->prof_on) {
+    at[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[na].val.programmaticStreamSerializationAllowed = 1;
+    ++na;
+  }
+  cfg.attrs = at;
+  cfg.numAttrs = na;
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, c->kv_tmap128, p));
+  LAUNCHED(c, "attn_tmem_kernel");
+  return D3_OK;
+}
+
+int run_attention_tmem(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
+  const d3_config& g = c->cfg;
+  const int group = g.n_q_heads / g.n_kv_heads;
+  const int R = group * rm.rows_per_seq;
+  const int copies = R <= 32 ? 4 : (R <= 64 ? 2 : 1);
+  const int rpc = 128 / copies;
+  const int q_tiles = (R + rpc - 1) / rpc;
+  const int pairs = rm.bs * g.n_kv_heads;
+  const int slots = c->n_sms;
+  int splits = 1;
+  if (q_tiles <= 2 && pairs * q_tiles < slots) {
+    const int max_tiles = (g.max_seq + attn::TKT - 1) / attn::TKT;
+    const int cap = std::max(1, std::min(8, max_tiles / 2));
+    auto cost_of = [&](int s) {
+      const long long waves = (static_cast<long long>(pairs) * q_tiles * s + slots - 1) / slots;
+      return waves * ((max_tiles + s - 1) / s);
+    };
+    long long best = cost_of(1);
+    for (int s = 2; s <= cap; ++s) best = std::min(best, cost_of(s));
+    for (int s = 1; s <= cap; ++s)
+      if (cost_of(s) * 100 <= best * 115) { splits = s; break; }
+  }
+  attn::AttnTcParams p{};
+  p.q = static_cast<const bf16*>(q);
+  p.out = static_cast<bf16*>(out);
+  p.rm = rm;
+  p.hq = g.n_q_heads; p.hkv = g.n_kv_heads; p.max_seq = g.max_seq;
+  const long long plane_rows = static_cast<long long>(g.max_batch) * g.n_kv_heads * g.max_seq;
+  p.k_row0 = (static_cast<long long>(layer) * 2 + 0) * plane_rows;
+  p.v_row0 = (static_cast<long long>(layer) * 2 + 1) * plane_rows;
+  p.n_splits = splits;
+  p.scale_log2 = 1.4426950408889634f / std::sqrt(static_cast<float>(g.d_head));
+  p.error_word = c->error_word;
+  dim3 grid(q_tiles, pairs, splits);
+  switch (copies) {
+    case 4: return launch_attn_tmem<4>(c, p, grid);
+    case 2: return launch_attn_tmem<2>(c, p, grid);
+    default: return launch_attn_tmem<1>(c, p, grid);
+  }
+}
+
 int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
   const d3_config& g = c->cfg;
   const int group = g.n_q_heads / g.n_kv_heads;
   const int R = group * rm.rows_per_seq;
+  if (c->tune_attn_tmem == 1) return run_attention_tmem(c, q, layer, out, rm);
   const int nw = R <= 32 ? 2 : (R <= 64 ? 4 : 8);
   const int q_tiles = (R + nw * 16 - 1) / (nw * 16);
   const int pairs = rm.bs * g.n_kv_heads;
@@ -1333,6 +1414,9 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
       rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, tc::CHAIN_AKT, &tm);
       if (rc_ != D3_OK) return bail(rc_);
       c->kv_tmap32 = *tm;
+      rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, attn::TKT, &tm);
+      if (rc_ != D3_OK) return bail(rc_);
+      c->kv_tmap128 = *tm;
       c->attn_tc = true;
     }
   }
@@ -1992,6 +2076,7 @@ extern "C" void d3_tuning_defaults(d3_tuning* t) {
   t->chain = -1;
   t->chain_l2_ahead = -1;
   t->weights_as_rows = -1;
+  t->attention_tmem = -1;
 }
 extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   if (!c || !t) return D3_ERR_INVALID_ARG;
@@ -1999,7 +2084,8 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
       (t->tile_columns != 0 && t->tile_columns != 128 && t->tile_columns != 256) || t->attn_key_tiles < 0 || t->attn_key_tiles > 7 ||
       t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
       (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
-      t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256 || t->weights_as_rows < -1 || t->weights_as_rows > 0)
+      t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256 || t->weights_as_rows < -1 || t->weights_as_rows > 0 ||
+      t->attention_tmem < -1 || t->attention_tmem > 1)
     return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
   c->tune_ring_kb = t->ring_kb;
   c->tune_ctas_per_sm = t->ctas_per_sm;
@@ -2015,6 +2101,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   c->tune_chain_clusters = t->chain_clusters;
   c->tune_chain_l2 = t->chain_l2_ahead;
   c->tune_xt = t->weights_as_rows;
+  c->tune_attn_tmem = t->attention_tmem;
   return D3_OK;
 }
 extern "C" int d3_set_fused_finalize(d3_ctx* c, int on) {
