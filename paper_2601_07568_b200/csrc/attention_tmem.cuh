@@ -11,9 +11,11 @@
 //                        K-major swizzled layout of an A operand
 //                  O_i = P_i V_i (N = d_head, K = 128 keys; V as it lies in the cache, [key][d], is an MN-major
 //                        B operand: 64 d values = one 128-byte swizzle row, 8 keys = one 1024-byte atom)
-// S and O are double-buffered in tensor memory (columns 0-255 and 256-511), P in shared memory, so the MMAs of
-// tile i + 1 run under the softmax of tile i.  O_i is a fresh product per tile; the running output row stays in the
-// softmax thread's registers (acc = acc * 2^(m_old - m_new) + O_i), which keeps the rescaling off the tensor path.
+// S is double-buffered in tensor memory (columns 0-255) and P in shared memory, so the first product of tile i + 1
+// runs under the softmax of tile i; O (columns 256-383) accumulates over all tiles inside the MMA.  The
+// exponentials are taken against a reference m that follows the row maximum lazily: it moves only when a tile's
+// maximum exceeds it by more than 2^8, and only then are the row sum and the O row (tcgen05.ld, scale, tcgen05.st)
+// rescaled.  P <= 2^8 is exact enough in bf16, the sums are fp32, and the quotient O / l does not depend on m.
 //
 // Fewer than 128 packed rows: with R <= 64 (R <= 32) rows the tile holds 2 (4) copies of the rows, copy c in lanes
 // c * 128 / COPIES ..., and copy c scores only keys [c, c + 1) * 128 / COPIES of every tile: its P rows are zero in
@@ -38,6 +40,7 @@ constexpr uint32_t TM_OFF_RING = TM_TILE;
 constexpr uint32_t TM_OFF_P = TM_OFF_RING + TM_STAGES * TM_TILE;
 constexpr uint32_t TM_OFF_BAR = TM_OFF_P + 2 * TM_TILE;
 constexpr int TM_THREADS = 192;
+constexpr float TM_SLACK_LOG2 = 8.f;        // how far a tile's maximum may exceed the reference before it moves
 
 // K-major operand slab, 128-byte swizzle: rows of 128 bytes, 8-row atoms 1024 bytes apart (stride byte offset);
 // the leading byte offset is not used by this form.  Bits: start address >> 4 in [0,14), LBO >> 4 in [16,30),
@@ -72,7 +75,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   uint64_t* kv_empty = kv_full + TM_STAGES;
   uint64_t* s_full = kv_empty + TM_STAGES;  // [2] S_i complete in tensor memory
   uint64_t* p_full = s_full + 2;            // [2] P_i in shared memory, S_i and O_(i-2) read
-  uint64_t* o_full = p_full + 2;            // [2] O_i complete in tensor memory
+  uint64_t* o_full = p_full + 2;            // [2] second product of tile i complete (O updated, P_i and V_i read)
   uint64_t* q_full = o_full + 2;            // Q (and the zeroed P buffers) in shared memory
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -202,7 +205,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
         for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step
           const uint64_t a = tm_desc_k(pb + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
           const uint64_t bd = tm_desc_mn(vb + kk * 2048, TM_SLAB, 1024);
-          ptx::umma_bf16(tmem_base + 256u + static_cast<uint32_t>((i & 1) * 128), a, bd, idesc_pv, kk > 0 ? 1u : 0u);
+          ptx::umma_bf16(tmem_base + 256u, a, bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         }
         ptx::umma_commit(&kv_empty[stage]);
         ptx::umma_commit(&o_full[i & 1]);
@@ -219,6 +222,9 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   const int r_seq = pr % rps;
   const bool row_ok = warp_id < 4 && pr < R && r_seq < n_valid;
   float acc[128];
+  // m_run is the reference the exponentials are taken against, not the running maximum: it moves only when a
+  // tile's maximum exceeds it by more than 2^TM_SLACK_LOG2, so P stays below that bound (exact in bf16's range, the
+  // sums in fp32) and O in tensor memory has to be rescaled only then: in practice at most once or twice per row.
   float m_run = -INFINITY, l_run = 0.f;
   if (warp_id < 4) {
     ptx::grid_dep_wait();  // Q comes from the kernel before this one
@@ -239,64 +245,66 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
     ptx::fence_proxy_async();
     ptx::mbar_arrive(q_full);
 
-#pragma unroll
-    for (int d = 0; d < 128; ++d) acc[d] = 0.f;
     const int kv_lim = row_ok ? row_kv_limit(p.rm, b, r_seq, kv_len) : kv_len;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp_id * 32) << 16);
-    float alpha_prev = 1.f;
-    auto add_o = [&](int i, float alpha) {  // acc = acc * alpha + O_i
-      if (!ptx::mbar_wait(&o_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word)) return false;
-      ptx::tc_fence_after();
-#pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
-        float o[32];
-        ptx::tmem_ld_32x32(t_lane + 256u + static_cast<uint32_t>((i & 1) * 128 + c4 * 32), o);
-        ptx::tmem_ld_wait();
-#pragma unroll
-        for (int c = 0; c < 32; ++c) acc[c4 * 32 + c] = fmaf(acc[c4 * 32 + c], alpha, o[c]);
-      }
-      return true;
-    };
+    const uint32_t t_o = t_lane + 256u;
     for (int i = 0; i < n_my && alive; ++i) {
       alive = ptx::mbar_wait(&s_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word);
       if (!alive) break;
       ptx::tc_fence_after();
       const int j0 = (t0 + i) * TKT + copy * KPC;  // first key this thread scores
       const uint32_t t_s = t_lane + static_cast<uint32_t>((i & 1) * TKT + copy * KPC);
-      float s[32];
-      // ---- row maximum over the keys this row may see
+      float s[NCH][32];
+#pragma unroll
+      for (int ch = 0; ch < NCH; ++ch) ptx::tmem_ld_32x32(t_s + ch * 32, s[ch]);
+      ptx::tmem_ld_wait();
       float mx = -INFINITY;
 #pragma unroll
-      for (int ch = 0; ch < NCH; ++ch) {
-        ptx::tmem_ld_32x32(t_s + ch * 32, s);
-        ptx::tmem_ld_wait();
+      for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
         for (int c = 0; c < 32; ++c) {
-          if (j0 + ch * 32 + c >= kv_lim) s[c] = -INFINITY;
-          mx = fmaxf(mx, s[c]);
+          if (j0 + ch * 32 + c >= kv_lim) s[ch][c] = -INFINITY;  // keys this row may not see
+          mx = fmaxf(mx, s[ch][c]);
         }
+      mx *= p.scale_log2;
+      const bool move = mx > m_run + TM_SLACK_LOG2;  // also the first tile with a visible key (m_run = -inf)
+      const bool resc = move && m_run != -INFINITY;  // there is something to rescale
+      if (i > 0 && __any_sync(0xffffffffu, resc)) {
+        // O holds the sum over the tiles before this one: all of those products must have landed
+        alive = ptx::mbar_wait(&o_full[(i - 1) & 1], static_cast<uint32_t>((i - 1) >> 1) & 1u, abort_flag, p.error_word);
+        if (!alive) break;
+        ptx::tc_fence_after();
+        const float f = resc ? exp2f(m_run - mx) : 1.f;
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          float o[32];
+          ptx::tmem_ld_32x32(t_o + c4 * 32, o);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] *= f;
+          ptx::tmem_st_32x32(t_o + c4 * 32, o);
+        }
+        ptx::tmem_st_wait();
       }
-      const float m_new = fmaxf(m_run, mx * p.scale_log2);
-      const float base = m_new == -INFINITY ? 0.f : m_new;  // no key seen yet: exponentials against 0 give 0, not NaN
-      const float alpha = exp2f(m_run - base);
-      m_run = m_new;
+      if (move) {
+        if (resc) l_run *= exp2f(m_run - mx);
+        m_run = mx;
+      }
+      const float base = m_run == -INFINITY ? 0.f : m_run;  // no key seen yet: exponentials against 0 give 0, not NaN
+      if (i >= 2) {  // the P buffer of tile i - 2 must have been read by its product
+        alive = ptx::mbar_wait(&o_full[i & 1], static_cast<uint32_t>((i - 2) >> 1) & 1u, abort_flag, p.error_word);
+        if (!alive) break;
+      }
       // ---- P = exp2(S * scale - m) as bf16 into the A-operand layout; row sum in fp32
       float sum = 0.f;
       uint8_t* prow = smem + TM_OFF_P + (i & 1) * TM_TILE;
 #pragma unroll
       for (int ch = 0; ch < NCH; ++ch) {
-        if constexpr (NCH > 1) {  // a single chunk is still in registers
-          ptx::tmem_ld_32x32(t_s + ch * 32, s);
-          ptx::tmem_ld_wait();
-#pragma unroll
-          for (int c = 0; c < 32; ++c)
-            if (j0 + ch * 32 + c >= kv_lim) s[c] = -INFINITY;
-        }
         uint32_t pk[16];
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
-          const float p0 = exp2f(fmaf(s[c], p.scale_log2, -base));
-          const float p1 = exp2f(fmaf(s[c + 1], p.scale_log2, -base));
+          const float p0 = exp2f(fmaf(s[ch][c], p.scale_log2, -base));
+          const float p1 = exp2f(fmaf(s[ch][c + 1], p.scale_log2, -base));
           sum += p0 + p1;
           pk[c >> 1] = pack_bf16(p0, p1);
         }
@@ -307,15 +315,24 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
               make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
         }
       }
-      l_run = l_run * alpha + sum;
+      l_run += sum;
       ptx::fence_proxy_async();
       ptx::tc_fence_before();
       ptx::mbar_arrive(&p_full[i & 1]);
-      // ---- the product of the tile before, which ran under the work above
-      if (i > 0) alive = add_o(i - 1, alpha_prev);
-      alpha_prev = alpha;
     }
-    if (alive && n_my > 0) alive = add_o(n_my - 1, alpha_prev);
+    // ---- the row of O, once every product has landed
+    if (alive && n_my > 0) {
+      alive = ptx::mbar_wait(&o_full[(n_my - 1) & 1], static_cast<uint32_t>((n_my - 1) >> 1) & 1u, abort_flag, p.error_word);
+      ptx::tc_fence_after();
+    }
+    if (alive && n_my > 0) {
+#pragma unroll
+      for (int c4 = 0; c4 < 4; ++c4) ptx::tmem_ld_32x32(t_o + c4 * 32, *reinterpret_cast<float(*)[32]>(acc + c4 * 32));
+      ptx::tmem_ld_wait();
+    } else {
+#pragma unroll
+      for (int d = 0; d < 128; ++d) acc[d] = 0.f;
+    }
   }
 
   // ------------------------------------------------------------------ output

@@ -271,7 +271,7 @@ def test_lm_head_stats_special_rows(ctx_f32):
     assert c[1] > 1 - 1e-6 and e[1] < 1e-5 and a[1] == 123
 
 
-def _attention_case(ctx, shape, bf16, bs, rows, kv_lens, seed):
+def _attention_case(ctx, shape, bf16, bs, rows, kv_lens, seed, ramp=0.0):
     rng = np.random.default_rng(seed)
     hq, hkv, dh = shape.n_q_heads, shape.n_kv_heads, shape.d_head
     rnd = (lambda s: rand_bf16(rng, s)) if bf16 else (
@@ -281,6 +281,10 @@ def _attention_case(ctx, shape, bf16, bs, rows, kv_lens, seed):
     for b in range(bs):
         L = kv_lens[b]
         kt, k = rnd((hkv, L, dh))
+        if ramp:  # keys grow along the sequence: the running maximum of a row keeps rising from tile to tile
+            grow = (1.0 + ramp * np.arange(L))[None, :, None]
+            kt = (kt.float() * torch.from_numpy(grow).float()).to(torch.bfloat16)
+            k = kt.float().numpy().astype(np.float64)
         vt, v = rnd((hkv, L, dh))
         d3.d3_op_write_kv(ctx.ctx, 0, b, 0, kt.float().to(DEV).contiguous(), vt.float().to(DEV).contiguous())
         qb = q[b * rows:(b + 1) * rows].reshape(rows, hq, dh)
@@ -331,6 +335,8 @@ def test_attention_bf16_tensor_memory(shape, rows, kv_lens):
         _attention_case(ctx, shape, True, 3, rows, kv_lens, rows + sum(kv_lens))
         _attention_case(ctx, shape, True, 3, rows, kv_lens, rows + sum(kv_lens))
         assert d3.d3_launch_count_of(ctx.ctx, "attn_tmem_kernel") == 2
+        # row maxima that rise by far more than 2^8 over the tiles: the reference moves and O is rescaled in place
+        _attention_case(ctx, shape, True, 3, rows, kv_lens, 7 + rows + sum(kv_lens), ramp=0.05)
 
 
 @pytest.mark.parametrize("rows,kv_lens", [(16, [48, 17]), (5, [5, 200])])
