@@ -1,27 +1,32 @@
 // Block-bidirectional attention (Sec. 3.2: every row of the block sees the whole prefix and the block itself,
-// no causal mask) with both products on the tcgen05 tensor cores and the accumulators in tensor memory.
+// no causal mask) with both products on the tcgen05 tensor cores and S, P, O and Q in tensor memory.
 // bf16, d_head = 128.
 //
 // One CTA = one (sequence, kv head, query tile, key split), 192 threads:
 //   warps 0-3  softmax: thread t owns row t of the tile = tensor-memory lane t
-//   warp 4     producer: K and V tiles of 128 keys by TMA (128-byte swizzle) into a ring of four 32 KB stages
+//   warp 4     producer: K and V tiles of 128 keys by TMA (128-byte swizzle) into a ring of six 32 KB stages
 //   warp 5     one thread issues the MMAs; the warp owns the tensor-memory allocation (all 512 columns)
-// Per key tile i:  S_i = Q K_i^T (M = 128 rows, N = 128 keys, K = d_head; Q and K are K-major operands)
-//                  P_i = exp2(S_i * scale - m_i) as bf16, written by the softmax threads to shared memory in the
-//                        K-major swizzled layout of an A operand
-//                  O_i = P_i V_i (N = d_head, K = 128 keys; V as it lies in the cache, [key][d], is an MN-major
-//                        B operand: 64 d values = one 128-byte swizzle row, 8 keys = one 1024-byte atom)
-// S is double-buffered in tensor memory (columns 0-255) and P in shared memory, so the first product of tile i + 1
-// runs under the softmax of tile i; O (columns 256-383) accumulates over all tiles inside the MMA.  The
-// exponentials are taken against a reference m that follows the row maximum lazily: it moves only when a tile's
-// maximum exceeds it by more than 2^8, and only then are the row sum and the O row (tcgen05.ld, scale, tcgen05.st)
-// rescaled.  P <= 2^8 is exact enough in bf16, the sums are fp32, and the quotient O / l does not depend on m.
+// Per key tile i:  S_i = Q K_i^T   M = 128 rows, N = 128 keys, K = d_head; Q is the A operand from tensor memory
+//                                  (64 columns: two bf16 per column), K_i a K-major B operand in shared memory
+//                  P_i = exp2(S_i * scale - m) as bf16, stored by the softmax threads over the first 64 columns
+//                        of S_i's own buffer (every thread has read its row of S_i before it writes there)
+//                  O  += P_i V_i   N = d_head, K = 128 keys; P_i is the A operand from tensor memory; V as it lies
+//                                  in the cache, [key][d], is an MN-major B operand: 64 d values = one 128-byte
+//                                  swizzle row, 8 keys = one 1024-byte atom
+// With both A operands in tensor memory an MMA step reads 4 KB of shared memory instead of 8 (the shared-memory
+// port, 128 bytes a clock, is what paces a 128 x 128 x 16 step with two shared-memory operands), and shared
+// memory holds nothing but K and V tiles in flight.
+// S is double-buffered (columns 0-255), so the first product of tile i + 1 runs under the softmax of tile i; O
+// (columns 256-383) accumulates over all tiles inside the MMA.  The exponentials are taken against a reference m
+// that follows the row maximum lazily: it moves only when a tile's maximum exceeds it by more than 2^8, and only
+// then are the row sum and the O row (tcgen05.ld, scale, tcgen05.st) rescaled.  P <= 2^8 is exact enough in bf16,
+// the sums are fp32, and the quotient O / l does not depend on m.
 //
 // Fewer than 128 packed rows: with R <= 64 (R <= 32) rows the tile holds 2 (4) copies of the rows, copy c in lanes
 // c * 128 / COPIES ..., and copy c scores only keys [c, c + 1) * 128 / COPIES of every tile: its P rows are zero in
-// the other key columns (zeroed once, never written).  Every copy keeps its own running maximum and sum; the copies
-// are merged through shared memory after the last tile.  That divides the exponentials per thread by COPIES, which
-// is what paces a tile once its rows fit a single warp.
+// the other key columns.  Every copy keeps its own reference and sum; the copies are merged through shared memory
+// after the last tile.  That divides the exponentials per thread by COPIES, which is what paces a tile once its
+// rows fit a single warp.
 //
 // Key splits: as in attn_tc_kernel, the CTAs of one query tile form a cluster along z and merge their partials
 // through distributed shared memory.
@@ -32,15 +37,14 @@ namespace d3 {
 namespace attn {
 
 constexpr int TKT = 128;                       // keys per tile
-constexpr int TM_STAGES = 4;                   // ring of K / V tiles
+constexpr int TM_STAGES = 6;                   // ring of K / V tiles
 constexpr uint32_t TM_SLAB = 128u * 128u;      // [128 rows][64 bf16], swizzled
 constexpr uint32_t TM_TILE = 2u * TM_SLAB;     // one K or V tile: d 0-63, d 64-127
-constexpr uint32_t TM_OFF_Q = 0;
-constexpr uint32_t TM_OFF_RING = TM_TILE;
-constexpr uint32_t TM_OFF_P = TM_OFF_RING + TM_STAGES * TM_TILE;
-constexpr uint32_t TM_OFF_BAR = TM_OFF_P + 2 * TM_TILE;
+constexpr uint32_t TM_OFF_RING = 0;
+constexpr uint32_t TM_OFF_BAR = TM_OFF_RING + TM_STAGES * TM_TILE;
 constexpr int TM_THREADS = 192;
-constexpr float TM_SLACK_LOG2 = 8.f;        // how far a tile's maximum may exceed the reference before it moves
+constexpr float TM_SLACK_LOG2 = 8.f;           // how far a tile's maximum may exceed the reference before it moves
+constexpr uint32_t TM_COL_S = 0, TM_COL_O = 256, TM_COL_Q = 384;  // tensor-memory columns
 
 // K-major operand slab, 128-byte swizzle: rows of 128 bytes, 8-row atoms 1024 bytes apart (stride byte offset);
 // the leading byte offset is not used by this form.  Bits: start address >> 4 in [0,14), LBO >> 4 in [16,30),
@@ -74,9 +78,9 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + TM_OFF_BAR);
   uint64_t* kv_empty = kv_full + TM_STAGES;
   uint64_t* s_full = kv_empty + TM_STAGES;  // [2] S_i complete in tensor memory
-  uint64_t* p_full = s_full + 2;            // [2] P_i in shared memory, S_i and O_(i-2) read
+  uint64_t* p_full = s_full + 2;            // [2] P_i in tensor memory (over S_i), O rescaled where it had to be
   uint64_t* o_full = p_full + 2;            // [2] second product of tile i complete (O updated, P_i and V_i read)
-  uint64_t* q_full = o_full + 2;            // Q (and the zeroed P buffers) in shared memory
+  uint64_t* q_full = o_full + 2;            // Q in tensor memory
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -180,10 +184,10 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
         ptx::tc_fence_after();
         const uint32_t kb = sbase + TM_OFF_RING + stage * TM_TILE;
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {
-          const uint64_t a = tm_desc_k(sbase + TM_OFF_Q + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
+        for (int kk = 0; kk < 8; ++kk) {  // 16 values of d_head per step = 8 columns of Q
           const uint64_t bd = tm_desc_k(kb + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
-          ptx::umma_bf16(tmem_base + static_cast<uint32_t>((i & 1) * TKT), a, bd, idesc_qk, kk > 0 ? 1u : 0u);
+          ptx::umma_bf16_ts(tmem_base + TM_COL_S + static_cast<uint32_t>((i & 1) * TKT), tmem_base + TM_COL_Q + kk * 8, bd,
+                            idesc_qk, kk > 0 ? 1u : 0u);
         }
         ptx::umma_commit(&kv_empty[stage]);
         ptx::umma_commit(&s_full[i & 1]);
@@ -200,16 +204,15 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
         if (!ok) break;
         ptx::tc_fence_after();
         const uint32_t vb = sbase + TM_OFF_RING + stage * TM_TILE;
-        const uint32_t pb = sbase + TM_OFF_P + (i & 1) * TM_TILE;
+        const uint32_t pcol = tmem_base + TM_COL_S + static_cast<uint32_t>((i & 1) * TKT);  // P_i lies over S_i
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step
-          const uint64_t a = tm_desc_k(pb + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
+        for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step = 8 columns of P
           const uint64_t bd = tm_desc_mn(vb + kk * 2048, TM_SLAB, 1024);
-          ptx::umma_bf16(tmem_base + 256u, a, bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+          ptx::umma_bf16_ts(tmem_base + TM_COL_O, pcol + kk * 8, bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         }
         ptx::umma_commit(&kv_empty[stage]);
         ptx::umma_commit(&o_full[i & 1]);
-        if (i + 2 < n_my) ok = qk(i + 2);
+        if (i + 2 < n_my) ok = qk(i + 2);  // overwrites S_i / P_i: issued after the product that reads P_i
       }
     }
   }
@@ -222,51 +225,50 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   const int r_seq = pr % rps;
   const bool row_ok = warp_id < 4 && pr < R && r_seq < n_valid;
   float acc[128];
-  // m_run is the reference the exponentials are taken against, not the running maximum: it moves only when a
-  // tile's maximum exceeds it by more than 2^TM_SLACK_LOG2, so P stays below that bound (exact in bf16's range, the
-  // sums in fp32) and O in tensor memory has to be rescaled only then: in practice at most once or twice per row.
+  // m_run is the reference the exponentials are taken against, not the running maximum (see the head of the file)
   float m_run = -INFINITY, l_run = 0.f;
   if (warp_id < 4) {
-    ptx::grid_dep_wait();  // Q comes from the kernel before this one
-    // Q rows into the two K-major slabs (d 0-63, d 64-127); rows that do not exist are zero
-    for (int e = tid; e < 128 * 16; e += 128) {
-      const int row = e >> 4, ch = e & 15;
-      const int pr2 = qt * RPC + row % RPC;
-      const int hg = pr2 / rps, r2 = pr2 % rps;
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (pr2 < R && r2 < n_valid)
-        v = *reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(b) * rps + r2) * p.hq * 128 + (g * group + hg) * 128 + ch * 8);
-      *reinterpret_cast<uint4*>(smem + TM_OFF_Q + (ch >> 3) * TM_SLAB + swz(row, ch & 7)) = v;
-    }
-    if constexpr (COPIES > 1) {  // key columns of a P row that its copy never writes
-      for (int e = tid; e < static_cast<int>(2 * TM_TILE / 16); e += 128)
-        *reinterpret_cast<uint4*>(smem + TM_OFF_P + e * 16) = make_uint4(0u, 0u, 0u, 0u);
-    }
-    ptx::fence_proxy_async();
-    ptx::mbar_arrive(q_full);
-
-    const int kv_lim = row_ok ? row_kv_limit(p.rm, b, r_seq, kv_len) : kv_len;
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp_id * 32) << 16);
-    const uint32_t t_o = t_lane + 256u;
+    const uint32_t t_o = t_lane + TM_COL_O;
+    ptx::grid_dep_wait();  // Q comes from the kernel before this one
+    {  // this thread's row of Q into its lane: 128 bf16 = 64 columns; a row that does not exist is zero
+      const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(b) * rps + r_seq) * p.hq * 128 +
+                                                        (g * group + pr / rps) * 128);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        uint4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = row_ok ? src[h * 8 + j] : make_uint4(0u, 0u, 0u, 0u);
+        ptx::tmem_st_32x32(t_lane + TM_COL_Q + h * 32, *reinterpret_cast<const float(*)[32]>(v));
+      }
+      ptx::tmem_st_wait();
+      ptx::tc_fence_before();
+      ptx::mbar_arrive(q_full);
+    }
+    const int kv_lim = row_ok ? row_kv_limit(p.rm, b, r_seq, kv_len) : kv_len;
     for (int i = 0; i < n_my && alive; ++i) {
       alive = ptx::mbar_wait(&s_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word);
       if (!alive) break;
       ptx::tc_fence_after();
       const int j0 = (t0 + i) * TKT + copy * KPC;  // first key this thread scores
-      const uint32_t t_s = t_lane + static_cast<uint32_t>((i & 1) * TKT + copy * KPC);
+      const uint32_t t_s = t_lane + TM_COL_S + static_cast<uint32_t>((i & 1) * TKT);
       float s[NCH][32];
 #pragma unroll
-      for (int ch = 0; ch < NCH; ++ch) ptx::tmem_ld_32x32(t_s + ch * 32, s[ch]);
+      for (int ch = 0; ch < NCH; ++ch) ptx::tmem_ld_32x32(t_s + copy * KPC + ch * 32, s[ch]);
       ptx::tmem_ld_wait();
-      float mx = -INFINITY;
+      if (!__all_sync(0xffffffffu, j0 + KPC <= kv_lim)) {  // a tile that reaches beyond what some row may see
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+          for (int c = 0; c < 32; ++c)
+            if (j0 + ch * 32 + c >= kv_lim) s[ch][c] = -INFINITY;
+      }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of KPC maxima
 #pragma unroll
       for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          if (j0 + ch * 32 + c >= kv_lim) s[ch][c] = -INFINITY;  // keys this row may not see
-          mx = fmaxf(mx, s[ch][c]);
-        }
-      mx *= p.scale_log2;
+        for (int c = 0; c < 32; ++c) mx4[c & 3] = fmaxf(mx4[c & 3], s[ch][c]);
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
       const bool move = mx > m_run + TM_SLACK_LOG2;  // also the first tile with a visible key (m_run = -inf)
       const bool resc = move && m_run != -INFINITY;  // there is something to rescale
       if (i > 0 && __any_sync(0xffffffffu, resc)) {
@@ -284,39 +286,37 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
           for (int c = 0; c < 32; ++c) o[c] *= f;
           ptx::tmem_st_32x32(t_o + c4 * 32, o);
         }
-        ptx::tmem_st_wait();
       }
       if (move) {
         if (resc) l_run *= exp2f(m_run - mx);
         m_run = mx;
       }
-      const float base = m_run == -INFINITY ? 0.f : m_run;  // no key seen yet: exponentials against 0 give 0, not NaN
-      if (i >= 2) {  // the P buffer of tile i - 2 must have been read by its product
-        alive = ptx::mbar_wait(&o_full[i & 1], static_cast<uint32_t>((i - 2) >> 1) & 1u, abort_flag, p.error_word);
-        if (!alive) break;
-      }
-      // ---- P = exp2(S * scale - m) as bf16 into the A-operand layout; row sum in fp32
-      float sum = 0.f;
-      uint8_t* prow = smem + TM_OFF_P + (i & 1) * TM_TILE;
+      const float nbase = m_run == -INFINITY ? 0.f : -m_run;  // no key seen yet: exponentials against 0 give 0, not NaN
+      // ---- P = exp2(S * scale - m) as bf16, two keys per column, over the first 64 columns of S_i
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      uint32_t pk[NCH][16];
 #pragma unroll
-      for (int ch = 0; ch < NCH; ++ch) {
-        uint32_t pk[16];
+      for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
         for (int c = 0; c < 32; c += 2) {
-          const float p0 = exp2f(fmaf(s[ch][c], p.scale_log2, -base));
-          const float p1 = exp2f(fmaf(s[ch][c + 1], p.scale_log2, -base));
-          sum += p0 + p1;
-          pk[c >> 1] = pack_bf16(p0, p1);
+          const float p0 = ptx::ex2_approx(fmaf(s[ch][c], p.scale_log2, nbase));
+          const float p1 = ptx::ex2_approx(fmaf(s[ch][c + 1], p.scale_log2, nbase));
+          sum4[(c >> 1) & 3] += p0 + p1;
+          pk[ch][c >> 1] = pack_bf16(p0, p1);
         }
+      l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
 #pragma unroll
-        for (int q4 = 0; q4 < 4; ++q4) {  // four 16-byte chunks of 8 keys
-          const int kc = (copy * KPC + ch * 32) / 8 + q4;  // chunk of the tile's 16
-          *reinterpret_cast<uint4*>(prow + (kc >> 3) * TM_SLAB + swz(tid, kc & 7)) =
-              make_uint4(pk[q4 * 4], pk[q4 * 4 + 1], pk[q4 * 4 + 2], pk[q4 * 4 + 3]);
+      for (int h = 0; h < 2; ++h) {  // columns 32 h .. 32 h + 31 of P: this copy's keys, zeros for the others'
+        uint32_t v[32];
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          if constexpr (COPIES == 1) v[j] = pk[h * 2 + (j >> 4)][j & 15];
+          else if constexpr (COPIES == 2) v[j] = copy == h ? pk[j >> 4][j & 15] : 0u;
+          else v[j] = ((copy >> 1) == h && (copy & 1) == (j >> 4)) ? pk[0][j & 15] : 0u;
         }
+        ptx::tmem_st_32x32(t_s + h * 32, *reinterpret_cast<const float(*)[32]>(v));
       }
-      l_run += sum;
-      ptx::fence_proxy_async();
+      ptx::tmem_st_wait();
       ptx::tc_fence_before();
       ptx::mbar_arrive(&p_full[i & 1]);
     }
@@ -466,6 +466,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
 }
 
 inline size_t attn_tmem_smem_bytes() { return 1024 + TM_OFF_BAR + (2 * TM_STAGES + 7) * 8 + 64; }
+static_assert(TM_STAGES * TM_TILE >= 128 * PART_LD * 4, "the partials of the copies overlay the ring");
 
 }  // namespace attn
 }  // namespace d3
