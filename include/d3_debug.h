@@ -45,7 +45,8 @@ typedef struct d3_tuning {
                                MMA's 128-row operand and a K-splitting cluster per tile: -1 = when the shape allows, 0 never */
   int32_t attention_tmem;   /* attention with both products on tcgen05 MMAs and the accumulators in tensor memory
                                (attn_tmem_kernel) instead of mma.sync (attn_tc_kernel): -1 = where measured faster
-                               (default), 0 never, 1 wherever the shape allows (bf16, d_head 128) */
+                               (default), 0 never, 1 wherever the shape allows (bf16, d_head 128), 64 or 128 = the same with
+                               that many keys per tile (two CTAs per SM / one) instead of the launcher's choice */
 } d3_tuning;
 void d3_tuning_defaults(d3_tuning *t);
 int d3_set_tuning(d3_ctx *ctx, const d3_tuning *t);

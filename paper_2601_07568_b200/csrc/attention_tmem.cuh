@@ -4,29 +4,28 @@
 //
 // One CTA = one (sequence, kv head, query tile, key split), 192 threads:
 //   warps 0-3  softmax: thread t owns row t of the tile = tensor-memory lane t
-//   warp 4     producer: K and V tiles of 128 keys by TMA (128-byte swizzle) into a ring of six 32 KB stages
-//   warp 5     one thread issues the MMAs; the warp owns the tensor-memory allocation (all 512 columns)
-// Per key tile i:  S_i = Q K_i^T   M = 128 rows, N = 128 keys, K = d_head; Q is the A operand from tensor memory
+//   warp 4     producer: K and V tiles of KT keys by TMA (128-byte swizzle) into a ring of six stages
+//   warp 5     one thread issues the MMAs; the warp owns the tensor-memory allocation
+// Per key tile i:  S_i = Q K_i^T   M = 128 rows, N = KT keys, K = d_head; Q is the A operand from tensor memory
 //                                  (64 columns: two bf16 per column), K_i a K-major B operand in shared memory
-//                  P_i = exp2(S_i * scale - m) as bf16, stored by the softmax threads over the first 64 columns
+//                  P_i = exp2(S_i * scale - m) as bf16, stored by the softmax threads over the first KT / 2 columns
 //                        of S_i's own buffer (every thread has read its row of S_i before it writes there)
-//                  O  += P_i V_i   N = d_head, K = 128 keys; P_i is the A operand from tensor memory; V as it lies
+//                  O  += P_i V_i   N = d_head, K = KT keys; P_i is the A operand from tensor memory; V as it lies
 //                                  in the cache, [key][d], is an MN-major B operand: 64 d values = one 128-byte
 //                                  swizzle row, 8 keys = one 1024-byte atom
 // With both A operands in tensor memory an MMA step reads 4 KB of shared memory instead of 8 (the shared-memory
 // port, 128 bytes a clock, is what paces a 128 x 128 x 16 step with two shared-memory operands), and shared
 // memory holds nothing but K and V tiles in flight.
-// S is double-buffered (columns 0-255), so the first product of tile i + 1 runs under the softmax of tile i; O
-// (columns 256-383) accumulates over all tiles inside the MMA.  The exponentials are taken against a reference m
+// With two S buffers the first product of tile i + 1 runs under the softmax of tile i.  O accumulates over all tiles inside the MMA.  The exponentials are taken against a reference m
 // that follows the row maximum lazily: it moves only when a tile's maximum exceeds it by more than 2^8, and only
 // then are the row sum and the O row (tcgen05.ld, scale, tcgen05.st) rescaled.  P <= 2^8 is exact enough in bf16,
 // the sums are fp32, and the quotient O / l does not depend on m.
 //
-// Fewer than 128 packed rows: with R <= 64 (R <= 32) rows the tile holds 2 (4) copies of the rows, copy c in lanes
-// c * 128 / COPIES ..., and copy c scores only keys [c, c + 1) * 128 / COPIES of every tile: its P rows are zero in
-// the other key columns.  Every copy keeps its own reference and sum; the copies are merged through shared memory
-// after the last tile.  That divides the exponentials per thread by COPIES, which is what paces a tile once its
-// rows fit a single warp.
+// Fewer than 128 packed rows leave lanes (and whole warps, which then skip the softmax) idle; the MMAs do not care.
+//
+// Two shapes of the same code:  <128 keys per tile, 2 S buffers>: 448 columns of tensor memory, 192 KB of K/V in
+// flight, one CTA per SM, for long key ranges;  <64, 1>: 256 columns, 96 KB, two CTAs per SM, whose start-up, serial
+// tile loop and output overlap each other: for short key ranges, where a CTA lives for a few tiles only.
 //
 // Key splits: as in attn_tc_kernel, the CTAs of one query tile form a cluster along z and merge their partials
 // through distributed shared memory.
@@ -36,15 +35,9 @@
 namespace d3 {
 namespace attn {
 
-constexpr int TKT = 128;                       // keys per tile
 constexpr int TM_STAGES = 6;                   // ring of K / V tiles
-constexpr uint32_t TM_SLAB = 128u * 128u;      // [128 rows][64 bf16], swizzled
-constexpr uint32_t TM_TILE = 2u * TM_SLAB;     // one K or V tile: d 0-63, d 64-127
-constexpr uint32_t TM_OFF_RING = 0;
-constexpr uint32_t TM_OFF_BAR = TM_OFF_RING + TM_STAGES * TM_TILE;
 constexpr int TM_THREADS = 192;
 constexpr float TM_SLACK_LOG2 = 8.f;           // how far a tile's maximum may exceed the reference before it moves
-constexpr uint32_t TM_COL_S = 0, TM_COL_O = 256, TM_COL_Q = 384;  // tensor-memory columns
 
 // K-major operand slab, 128-byte swizzle: rows of 128 bytes, 8-row atoms 1024 bytes apart (stride byte offset);
 // the leading byte offset is not used by this form.  Bits: start address >> 4 in [0,14), LBO >> 4 in [16,30),
@@ -64,23 +57,33 @@ __host__ __device__ constexpr uint32_t tm_idesc(int m, int n, bool b_mn) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (b_mn ? (1u << 16) : 0u) | (static_cast<uint32_t>(n >> 3) << 17) |
          (static_cast<uint32_t>(m >> 4) << 24);
 }
-__device__ __forceinline__ void tm_bar_softmax() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
-// grid (q_tiles, bs * hkv, n_splits); COPIES in {1, 2, 4}: 128 / COPIES packed rows per query tile.
-template <int COPIES>
-__global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_constant__ CUtensorMap tmap_kv,
-                                                                  const AttnTcParams p) {
-  constexpr int RPC = 128 / COPIES;  // packed rows of the tile
-  constexpr int KPC = TKT / COPIES;  // keys of a tile that one copy scores
-  constexpr int NCH = KPC / 32;      // 32-column chunks of S per thread
+
+template <int KT, int SBUF>
+struct TmLayout {
+  static constexpr uint32_t SLAB = static_cast<uint32_t>(KT) * 128u;  // [KT keys][64 bf16], swizzled
+  static constexpr uint32_t TILE = 2u * SLAB;                         // one K or V tile: d 0-63, d 64-127
+  static constexpr uint32_t OFF_BAR = TM_STAGES * TILE;
+  static constexpr uint32_t COL_S = 0, COL_O = SBUF * KT, COL_Q = COL_O + 128;  // tensor-memory columns
+  static constexpr uint32_t COLS = COL_Q + 64 <= 256 ? 256 : 512;               // allocation: a power of two
+  static constexpr size_t smem_bytes() { return 1024 + OFF_BAR + (2 * TM_STAGES + 2 * SBUF + 4) * 8 + 64; }
+};
+
+// grid (q_tiles, bs * hkv, n_splits); 128 packed rows per query tile.
+template <int KT, int SBUF>
+__global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel(const __grid_constant__ CUtensorMap tmap_kv,
+                                                                                 const AttnTcParams p) {
+  using L = TmLayout<KT, SBUF>;
+  constexpr int NCH = KT / 32;  // 32-column chunks of S per thread
+  constexpr int BM = 128;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + TM_OFF_BAR);
+  uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* kv_empty = kv_full + TM_STAGES;
-  uint64_t* s_full = kv_empty + TM_STAGES;  // [2] S_i complete in tensor memory
-  uint64_t* p_full = s_full + 2;            // [2] P_i in tensor memory (over S_i), O rescaled where it had to be
-  uint64_t* o_full = p_full + 2;            // [2] second product of tile i complete (O updated, P_i and V_i read)
-  uint64_t* q_full = o_full + 2;            // Q in tensor memory
+  uint64_t* s_full = kv_empty + TM_STAGES;  // [SBUF] S_i complete in tensor memory
+  uint64_t* p_full = s_full + SBUF;         // [SBUF] P_i in tensor memory (over S_i), O rescaled where it had to be
+  uint64_t* o_full = p_full + SBUF;         // second product of tile i complete (O updated, P_i and V_i read)
+  uint64_t* q_full = o_full + 1;            // Q in tensor memory
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(q_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -96,10 +99,10 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   const int kv_len = p.rm.kv_len[b];
   const int stable_keys = p.rm.pos_base[b];
   const int R = group * rps;
-  bool work = !(qt * RPC >= R || n_valid <= 0 || kv_len <= 0);
+  bool work = !(qt * BM >= R || n_valid <= 0 || kv_len <= 0);
   if (work) {
     bool any = false;
-    for (int pr = qt * RPC; pr < min(R, (qt + 1) * RPC) && !any; pr += 1) any = (pr % rps) < n_valid;
+    for (int pr = qt * BM; pr < min(R, (qt + 1) * BM) && !any; pr += 1) any = (pr % rps) < n_valid;
     work = any;
   }
   if (!work) {  // uniform over the CTA and over the cluster
@@ -113,17 +116,17 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
       ptx::mbar_init(&kv_full[s], 1);
       ptx::mbar_init(&kv_empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) {
+    for (int s = 0; s < SBUF; ++s) {
       ptx::mbar_init(&s_full[s], 1);
       ptx::mbar_init(&p_full[s], 128);
-      ptx::mbar_init(&o_full[s], 1);
     }
+    ptx::mbar_init(o_full, 1);
     ptx::mbar_init(q_full, 128);
     *abort_flag = 0;
     ptx::fence_barrier_init();
   }
   if (warp_id == 5) {
-    ptx::tmem_alloc<512>(tmem_slot);
+    ptx::tmem_alloc<L::COLS>(tmem_slot);
     ptx::tmem_relinquish();
   }
   ptx::tc_fence_before();
@@ -132,96 +135,99 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   const uint32_t tmem_base = *tmem_slot;
   ptx::grid_dep_launch();
 
-  const int n_tiles = (kv_len + TKT - 1) / TKT;
+  const int n_tiles = (kv_len + KT - 1) / KT;
   const int tps = (n_tiles + p.n_splits - 1) / p.n_splits;
   const int t0 = split * tps, t1 = min(n_tiles, t0 + tps);
   const int n_my = max(t1 - t0, 0);
   const uint32_t sbase = ptx::smem_u32(smem);
   bool alive = true;
 
-  // Order in which the MMA thread consumes the tiles: K0, K1, V0, K2, V1, ..., K(n-1), V(n-2), V(n-1).
-  // Position of K_i: 0 for i = 0, else 2 i - 1.  Position of V_i: 2 n - 1 for the last, else 2 i + 2.
+  // Producer and MMA thread walk the tiles in the same order: K_0 .. K_(SBUF-1), then V_j, K_(j+SBUF) for every j.
   if (warp_id == 4) {
     // ------------------------------------------------------------------ producer
     if (lane == 0) {
       const long long krow = p.k_row0 + (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
       const long long vrow = p.v_row0 + (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
-      bool waited = false;
-      for (int s = 0; s < 2 * n_my; ++s) {
+      bool waited = false, ok = true;
+      int s = 0;  // position in the ring
+      auto load = [&](bool is_k, int i) {
         const int stage = s % TM_STAGES;
         if (s >= TM_STAGES &&
             !ptx::mbar_wait(&kv_empty[stage], static_cast<uint32_t>(s / TM_STAGES - 1) & 1u, abort_flag, p.error_word))
-          break;
-        bool is_k;
-        int i;
-        if (s == 0) { is_k = true; i = 0; }
-        else if (s & 1) { i = (s + 1) / 2; is_k = i < n_my; if (!is_k) i = n_my - 1; }
-        else { is_k = false; i = (s - 2) / 2; }
-        const int j0 = (t0 + i) * TKT;
-        if (!waited && j0 + TKT > stable_keys) {  // this tile holds rows the QKV kernel of this layer writes
+          return false;
+        const int j0 = (t0 + i) * KT;
+        if (!waited && j0 + KT > stable_keys) {  // this tile holds rows the QKV kernel of this layer writes
           ptx::grid_dep_wait();
           waited = true;
         }
-        uint8_t* dst = smem + TM_OFF_RING + stage * TM_TILE;
+        uint8_t* dst = smem + stage * L::TILE;
         const int row = static_cast<int>((is_k ? krow : vrow) + j0);
-        ptx::mbar_arrive_expect_tx(&kv_full[stage], TM_TILE);
+        ptx::mbar_arrive_expect_tx(&kv_full[stage], L::TILE);
         ptx::tma_load_2d(dst, &tmap_kv, &kv_full[stage], 0, row);
-        ptx::tma_load_2d(dst + TM_SLAB, &tmap_kv, &kv_full[stage], 64, row);
+        ptx::tma_load_2d(dst + L::SLAB, &tmap_kv, &kv_full[stage], 64, row);
+        ++s;
+        return true;
+      };
+      for (int i = 0; i < min(SBUF, n_my) && ok; ++i) ok = load(true, i);
+      for (int j = 0; j < n_my && ok; ++j) {
+        ok = load(false, j);
+        if (ok && j + SBUF < n_my) ok = load(true, j + SBUF);
       }
       if (!waited) ptx::grid_dep_wait();
     }
   } else if (warp_id == 5) {
     // ------------------------------------------------------------------ MMA issue
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = tm_idesc(128, TKT, false);
+      constexpr uint32_t idesc_qk = tm_idesc(128, KT, false);
       constexpr uint32_t idesc_pv = tm_idesc(128, 128, true);
       bool ok = ptx::mbar_wait(q_full, 0, abort_flag, p.error_word);
       ptx::tc_fence_after();
-      auto qk = [&](int i) {  // S_i into S buffer i & 1
-        const int seq = i == 0 ? 0 : 2 * i - 1;
-        const int stage = seq % TM_STAGES;
-        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(seq / TM_STAGES) & 1u, abort_flag, p.error_word)) return false;
+      int s = 0;  // position in the ring
+      auto stage_ready = [&](uint32_t& addr) {
+        const int stage = s % TM_STAGES;
+        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(s / TM_STAGES) & 1u, abort_flag, p.error_word)) return -1;
         ptx::tc_fence_after();
-        const uint32_t kb = sbase + TM_OFF_RING + stage * TM_TILE;
+        addr = sbase + stage * L::TILE;
+        ++s;
+        return stage;
+      };
+      auto qk = [&](int i) {  // S_i into S buffer i % SBUF
+        uint32_t kb;
+        const int stage = stage_ready(kb);
+        if (stage < 0) return false;
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {  // 16 values of d_head per step = 8 columns of Q
-          const uint64_t bd = tm_desc_k(kb + (kk >> 2) * TM_SLAB) + static_cast<uint64_t>(2 * (kk & 3));
-          ptx::umma_bf16_ts(tmem_base + TM_COL_S + static_cast<uint32_t>((i & 1) * TKT), tmem_base + TM_COL_Q + kk * 8, bd,
+          const uint64_t bd = tm_desc_k(kb + (kk >> 2) * L::SLAB) + static_cast<uint64_t>(2 * (kk & 3));
+          ptx::umma_bf16_ts(tmem_base + L::COL_S + static_cast<uint32_t>((i % SBUF) * KT), tmem_base + L::COL_Q + kk * 8, bd,
                             idesc_qk, kk > 0 ? 1u : 0u);
         }
         ptx::umma_commit(&kv_empty[stage]);
-        ptx::umma_commit(&s_full[i & 1]);
+        ptx::umma_commit(&s_full[i % SBUF]);
         return true;
       };
-      if (ok && n_my > 0) ok = qk(0);
-      if (ok && n_my > 1) ok = qk(1);
+      for (int i = 0; i < min(SBUF, n_my) && ok; ++i) ok = qk(i);
       for (int i = 0; i < n_my && ok; ++i) {
-        ok = ptx::mbar_wait(&p_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word);
+        ok = ptx::mbar_wait(&p_full[i % SBUF], static_cast<uint32_t>(i / SBUF) & 1u, abort_flag, p.error_word);
         if (!ok) break;
-        const int seq = i == n_my - 1 ? 2 * n_my - 1 : 2 * i + 2;
-        const int stage = seq % TM_STAGES;
-        ok = ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(seq / TM_STAGES) & 1u, abort_flag, p.error_word);
-        if (!ok) break;
-        ptx::tc_fence_after();
-        const uint32_t vb = sbase + TM_OFF_RING + stage * TM_TILE;
-        const uint32_t pcol = tmem_base + TM_COL_S + static_cast<uint32_t>((i & 1) * TKT);  // P_i lies over S_i
+        uint32_t vb;
+        const int stage = stage_ready(vb);
+        if (stage < 0) break;
+        const uint32_t pcol = tmem_base + L::COL_S + static_cast<uint32_t>((i % SBUF) * KT);  // P_i lies over S_i
 #pragma unroll
-        for (int kk = 0; kk < 8; ++kk) {  // 16 keys per step = 8 columns of P
-          const uint64_t bd = tm_desc_mn(vb + kk * 2048, TM_SLAB, 1024);
-          ptx::umma_bf16_ts(tmem_base + TM_COL_O, pcol + kk * 8, bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
+        for (int kk = 0; kk < KT / 16; ++kk) {  // 16 keys per step = 8 columns of P
+          const uint64_t bd = tm_desc_mn(vb + kk * 2048, L::SLAB, 1024);
+          ptx::umma_bf16_ts(tmem_base + L::COL_O, pcol + kk * 8, bd, idesc_pv, (i > 0 || kk > 0) ? 1u : 0u);
         }
         ptx::umma_commit(&kv_empty[stage]);
-        ptx::umma_commit(&o_full[i & 1]);
-        if (i + 2 < n_my) ok = qk(i + 2);  // overwrites S_i / P_i: issued after the product that reads P_i
+        ptx::umma_commit(o_full);
+        if (i + SBUF < n_my) ok = qk(i + SBUF);  // overwrites S_i / P_i: issued after the product that reads P_i
       }
     }
   }
 
   // ------------------------------------------------------------------ softmax warps
-  const int tid = threadIdx.x;             // row of the tile and tensor-memory lane (warps 0-3)
-  const int copy = (tid & 127) / RPC;      // which copy of the rows, = which part of every tile's keys
-  const int lr = (tid & 127) % RPC;
-  const int pr = qt * RPC + lr;            // packed row: head_in_group * rows_per_seq + r
+  const int tid = threadIdx.x;   // row of the tile and tensor-memory lane (warps 0-3)
+  const int pr = qt * BM + tid;  // packed row: head_in_group * rows_per_seq + r
   const int r_seq = pr % rps;
   const bool row_ok = warp_id < 4 && pr < R && r_seq < n_valid;
   float acc[128];
@@ -229,7 +235,8 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   float m_run = -INFINITY, l_run = 0.f;
   if (warp_id < 4) {
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp_id * 32) << 16);
-    const uint32_t t_o = t_lane + TM_COL_O;
+    const uint32_t t_o = t_lane + L::COL_O;
+    const bool warp_rows = __any_sync(0xffffffffu, row_ok);  // a warp without rows only keeps the barriers going
     ptx::grid_dep_wait();  // Q comes from the kernel before this one
     {  // this thread's row of Q into its lane: 128 bf16 = 64 columns; a row that does not exist is zero
       const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(b) * rps + r_seq) * p.hq * 128 +
@@ -239,7 +246,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
         uint4 v[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) v[j] = row_ok ? src[h * 8 + j] : make_uint4(0u, 0u, 0u, 0u);
-        ptx::tmem_st_32x32(t_lane + TM_COL_Q + h * 32, *reinterpret_cast<const float(*)[32]>(v));
+        ptx::tmem_st_32x32(t_lane + L::COL_Q + h * 32, *reinterpret_cast<const float(*)[32]>(v));
       }
       ptx::tmem_st_wait();
       ptx::tc_fence_before();
@@ -247,23 +254,31 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
     }
     const int kv_lim = row_ok ? row_kv_limit(p.rm, b, r_seq, kv_len) : kv_len;
     for (int i = 0; i < n_my && alive; ++i) {
-      alive = ptx::mbar_wait(&s_full[i & 1], static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.error_word);
+      alive = ptx::mbar_wait(&s_full[i % SBUF], static_cast<uint32_t>(i / SBUF) & 1u, abort_flag, p.error_word);
       if (!alive) break;
+      // Every thread watches every phase of o_full in order (a parity wait cannot tell a phase from the one two
+      // before it): the product of tile i - 1 was issued a whole tile ago, so this wait is over before it starts.
+      auto seen_o = [&]() { return i == 0 || ptx::mbar_wait(o_full, static_cast<uint32_t>(i - 1) & 1u, abort_flag, p.error_word); };
+      if (!warp_rows) {  // whatever these lanes of S hold is multiplied into rows nobody reads
+        alive = seen_o();
+        ptx::mbar_arrive(&p_full[i % SBUF]);
+        continue;
+      }
       ptx::tc_fence_after();
-      const int j0 = (t0 + i) * TKT + copy * KPC;  // first key this thread scores
-      const uint32_t t_s = t_lane + TM_COL_S + static_cast<uint32_t>((i & 1) * TKT);
+      const int j0 = (t0 + i) * KT;
+      const uint32_t t_s = t_lane + L::COL_S + static_cast<uint32_t>((i % SBUF) * KT);
       float s[NCH][32];
 #pragma unroll
-      for (int ch = 0; ch < NCH; ++ch) ptx::tmem_ld_32x32(t_s + copy * KPC + ch * 32, s[ch]);
+      for (int ch = 0; ch < NCH; ++ch) ptx::tmem_ld_32x32(t_s + ch * 32, s[ch]);
       ptx::tmem_ld_wait();
-      if (!__all_sync(0xffffffffu, j0 + KPC <= kv_lim)) {  // a tile that reaches beyond what some row may see
+      if (!__all_sync(0xffffffffu, j0 + KT <= kv_lim)) {  // a tile that reaches beyond what some row may see
 #pragma unroll
         for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
           for (int c = 0; c < 32; ++c)
             if (j0 + ch * 32 + c >= kv_lim) s[ch][c] = -INFINITY;
       }
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of KPC maxima
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};  // four chains instead of one of KT maxima
 #pragma unroll
       for (int ch = 0; ch < NCH; ++ch)
 #pragma unroll
@@ -273,7 +288,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
       const bool resc = move && m_run != -INFINITY;  // there is something to rescale
       if (i > 0 && __any_sync(0xffffffffu, resc)) {
         // O holds the sum over the tiles before this one: all of those products must have landed
-        alive = ptx::mbar_wait(&o_full[(i - 1) & 1], static_cast<uint32_t>((i - 1) >> 1) & 1u, abort_flag, p.error_word);
+        alive = ptx::mbar_wait(o_full, static_cast<uint32_t>(i - 1) & 1u, abort_flag, p.error_word);
         if (!alive) break;
         ptx::tc_fence_after();
         const float f = resc ? exp2f(m_run - mx) : 1.f;
@@ -292,40 +307,32 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
         m_run = mx;
       }
       const float nbase = m_run == -INFINITY ? 0.f : -m_run;  // no key seen yet: exponentials against 0 give 0, not NaN
-      // ---- P = exp2(S * scale - m) as bf16, two keys per column, over the first 64 columns of S_i
+      // ---- P = exp2(S * scale - m) as bf16, two keys per column, over the first KT / 2 columns of S_i
       float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t pk[NCH][16];
 #pragma unroll
-      for (int ch = 0; ch < NCH; ++ch)
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) {
-          const float p0 = ptx::ex2_approx(fmaf(s[ch][c], p.scale_log2, nbase));
-          const float p1 = ptx::ex2_approx(fmaf(s[ch][c + 1], p.scale_log2, nbase));
-          sum4[(c >> 1) & 3] += p0 + p1;
-          pk[ch][c >> 1] = pack_bf16(p0, p1);
-        }
-      l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-#pragma unroll
-      for (int h = 0; h < 2; ++h) {  // columns 32 h .. 32 h + 31 of P: this copy's keys, zeros for the others'
+      for (int h = 0; h < NCH / 2; ++h) {  // 64 keys = 32 columns of P per store
         uint32_t v[32];
 #pragma unroll
         for (int j = 0; j < 32; ++j) {
-          if constexpr (COPIES == 1) v[j] = pk[h * 2 + (j >> 4)][j & 15];
-          else if constexpr (COPIES == 2) v[j] = copy == h ? pk[j >> 4][j & 15] : 0u;
-          else v[j] = ((copy >> 1) == h && (copy & 1) == (j >> 4)) ? pk[0][j & 15] : 0u;
+          const float p0 = ptx::ex2_approx(fmaf(s[h * 2 + (j >> 4)][(j & 15) * 2], p.scale_log2, nbase));
+          const float p1 = ptx::ex2_approx(fmaf(s[h * 2 + (j >> 4)][(j & 15) * 2 + 1], p.scale_log2, nbase));
+          sum4[j & 3] += p0 + p1;
+          v[j] = pack_bf16(p0, p1);
         }
         ptx::tmem_st_32x32(t_s + h * 32, *reinterpret_cast<const float(*)[32]>(v));
       }
+      l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      alive = seen_o();
       ptx::tmem_st_wait();
       ptx::tc_fence_before();
-      ptx::mbar_arrive(&p_full[i & 1]);
+      ptx::mbar_arrive(&p_full[i % SBUF]);
     }
     // ---- the row of O, once every product has landed
     if (alive && n_my > 0) {
-      alive = ptx::mbar_wait(&o_full[(n_my - 1) & 1], static_cast<uint32_t>((n_my - 1) >> 1) & 1u, abort_flag, p.error_word);
+      alive = ptx::mbar_wait(o_full, static_cast<uint32_t>(n_my - 1) & 1u, abort_flag, p.error_word);
       ptx::tc_fence_after();
     }
-    if (alive && n_my > 0) {
+    if (alive && n_my > 0 && warp_rows) {
 #pragma unroll
       for (int c4 = 0; c4 < 4; ++c4) ptx::tmem_ld_32x32(t_o + c4 * 32, *reinterpret_cast<float(*)[32]>(acc + c4 * 32));
       ptx::tmem_ld_wait();
@@ -340,95 +347,38 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
     const int hg = prow / rps, r = prow % rps;
     return p.out + (static_cast<size_t>(b) * rps + r) * p.hq * 128 + (g * group + hg) * 128;
   };
-  // Partials [COPIES][RPC][PART_LD] over the ring: every load into it has been consumed once the last O is read.
-  float* red = reinterpret_cast<float*>(smem + TM_OFF_RING);
-  if (warp_id < 4) {
-    if (COPIES == 1 && p.n_splits == 1) {
-      if (alive && row_ok) {
-        const float inv = 1.0f / l_run;
-        __nv_bfloat16* o = out_ptr(pr);
+  if (p.n_splits == 1) {
+    if (alive && row_ok) {
+      const float inv = 1.0f / l_run;
+      __nv_bfloat16* o = out_ptr(pr);
 #pragma unroll
-        for (int d = 0; d < 128; d += 8)
-          *reinterpret_cast<uint4*>(o + d) =
-              make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv), pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
-                         pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv), pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
-      }
-    } else {
-      float* rr = red + static_cast<size_t>(tid) * PART_LD;  // tid = copy * RPC + lr
+      for (int d = 0; d < 128; d += 8)
+        *reinterpret_cast<uint4*>(o + d) =
+            make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv), pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
+                       pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv), pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+    }
+  } else {
+    // Partials [128][PART_LD] over the ring (every load into it has been consumed once the last O is read), merged
+    // over the key splits: every CTA of the cluster takes a slice of the rows.
+    float* red = reinterpret_cast<float*>(smem);
+    if (warp_id < 4) {
+      float* rr = red + static_cast<size_t>(tid) * PART_LD;
 #pragma unroll
       for (int d = 0; d < 128; d += 4) *reinterpret_cast<float4*>(rr + d) = make_float4(acc[d], acc[d + 1], acc[d + 2], acc[d + 3]);
-      rr[128] = m_run;  // a copy or split without keys leaves m = -inf, l = 0
+      rr[128] = m_run;  // a split without keys leaves m = -inf, l = 0
       rr[129] = l_run;
-      tm_bar_softmax();
-      if constexpr (COPIES > 1) {
-        // one thread per (row, 4 output dims); everything is read before anything of copy 0 is overwritten
-        constexpr int EPT = RPC * 32 / 128;
-        float4 mg[EPT];
-        float Ms[EPT], Ls[EPT];
-#pragma unroll
-        for (int j = 0; j < EPT; ++j) {
-          const int e = tid + j * 128;
-          const int row = e >> 5, c4 = (e & 31) * 4;
-          mg[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-          Ms[j] = -INFINITY;
-          Ls[j] = 0.f;
-          float mq[COPIES], lq[COPIES];
-#pragma unroll
-          for (int q2 = 0; q2 < COPIES; ++q2) {
-            const float* r = red + (static_cast<size_t>(q2) * RPC + row) * PART_LD;
-            mq[q2] = r[128];
-            lq[q2] = r[129];
-            Ms[j] = fmaxf(Ms[j], mq[q2]);
-          }
-#pragma unroll
-          for (int q2 = 0; q2 < COPIES; ++q2) {  // copies in index order: fixed order of the sums
-            if (lq[q2] != 0.f) {
-              const float w = exp2f(mq[q2] - Ms[j]);
-              const float4 v = *reinterpret_cast<const float4*>(red + (static_cast<size_t>(q2) * RPC + row) * PART_LD + c4);
-              Ls[j] += w * lq[q2];
-              mg[j].x += w * v.x; mg[j].y += w * v.y; mg[j].z += w * v.z; mg[j].w += w * v.w;
-            }
-          }
-        }
-        if (p.n_splits == 1) {
-          if (alive) {
-#pragma unroll
-            for (int j = 0; j < EPT; ++j) {
-              const int e = tid + j * 128;
-              const int row = e >> 5, c4 = (e & 31) * 4;
-              const int prow = qt * RPC + row;
-              if (prow >= R || (prow % rps) >= n_valid) continue;
-              const float inv = 1.0f / Ls[j];
-              *reinterpret_cast<uint2*>(out_ptr(prow) + c4) =
-                  make_uint2(pack_bf16(mg[j].x * inv, mg[j].y * inv), pack_bf16(mg[j].z * inv, mg[j].w * inv));
-            }
-          }
-        } else {
-          tm_bar_softmax();
-#pragma unroll
-          for (int j = 0; j < EPT; ++j) {
-            const int e = tid + j * 128;
-            const int row = e >> 5, c4 = (e & 31) * 4;
-            float* r = red + static_cast<size_t>(row) * PART_LD;
-            *reinterpret_cast<float4*>(r + c4) = mg[j];
-            if (c4 == 0) { r[128] = Ms[j]; r[129] = Ls[j]; }
-          }
-        }
-      }
     }
-  }
-  if (p.n_splits > 1) {  // merge over the key splits: every CTA of the cluster takes a slice of the rows
     __syncwarp();
     ptx::cluster_sync_all();
     if (warp_id < 4) {
       const int S = p.n_splits;
       const int rank = static_cast<int>(ptx::cluster_ctarank());
-      const int rpr = (RPC + S - 1) / S;
-      const int row0 = rank * rpr, row1 = min(RPC, row0 + rpr);
+      const int rpr = (BM + S - 1) / S;
+      const int row0 = rank * rpr, row1 = min(BM, row0 + rpr);
       const uint32_t red_addr = ptx::smem_u32(red);
       for (int e = tid; e < (row1 - row0) * 32; e += 128) {
         const int row = row0 + (e >> 5), c4 = (e & 31) * 4;
-        const int prow = qt * RPC + row;
+        const int prow = qt * BM + row;
         if (prow >= R || (prow % rps) >= n_valid) continue;
         const uint32_t off = static_cast<uint32_t>(row * PART_LD) * 4u;
         float ms[8], ls[8];
@@ -444,16 +394,16 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
             M = fmaxf(M, ms[s2]);
           }
         }
-        float L = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        float Lsum = 0.f, a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-        for (int s2 = 0; s2 < 8; ++s2) {
+        for (int s2 = 0; s2 < 8; ++s2) {  // splits in index order: fixed order of the sums
           if (s2 < S && ls[s2] != 0.f) {
             const float w = exp2f(ms[s2] - M);
-            L += w * ls[s2];
+            Lsum += w * ls[s2];
             a0 += w * vs[s2].x; a1 += w * vs[s2].y; a2 += w * vs[s2].z; a3 += w * vs[s2].w;
           }
         }
-        const float inv = 1.0f / L;
+        const float inv = 1.0f / Lsum;
         *reinterpret_cast<uint2*>(out_ptr(prow) + c4) = make_uint2(pack_bf16(a0 * inv, a1 * inv), pack_bf16(a2 * inv, a3 * inv));
       }
     }
@@ -462,11 +412,10 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_kernel(const __grid_c
   }
   ptx::tc_fence_before();
   __syncthreads();
-  if (warp_id == 5) ptx::tmem_dealloc<512>(tmem_base);
+  if (warp_id == 5) ptx::tmem_dealloc<L::COLS>(tmem_base);
 }
 
-inline size_t attn_tmem_smem_bytes() { return 1024 + TM_OFF_BAR + (2 * TM_STAGES + 7) * 8 + 64; }
-static_assert(TM_STAGES * TM_TILE >= 128 * PART_LD * 4, "the partials of the copies overlay the ring");
+static_assert(TmLayout<64, 1>::OFF_BAR >= 128 * PART_LD * 4, "the partials of the key splits overlay the ring");
 
 }  // namespace attn
 }  // namespace d3

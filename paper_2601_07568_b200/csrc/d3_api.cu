@@ -117,6 +117,7 @@ struct d3_ctx {
   int chain_qkv_ks = 2;       // K parts of the QKV matmul inside a chain
   int tune_chain_clusters = 0;  // 0: as many clusters as fit
   int tune_chain_l2 = -1;       // weight slabs the chain's L2 prefetch runs ahead (-1: default, 0: off)
+  int tune_attn_shape = 0;      // experiment: keys per tile of the tcgen05 attention (0 = by rule, 64, 128)
   int tune_attn_tmem = -1;      // tcgen05 attention: -1 where measured faster, 0 never, 1 wherever the shape allows
   int tune_xt = -1;             // 129..256-row matmuls with weights as the 128-row operand: -1 when the shape allows, 0 never
   unsigned int* chain_sync = nullptr;  // [operators of the program] border counters of a forward's chain launches
@@ -1012,20 +1013,21 @@ int attn_ctas_per_sm() {
   return cached;
 }
 
-// tcgen05 attention launch: copies of the rows from the packed rows per kv head, key splits so that the
-// CTAs (one per SM: the kernel takes all of tensor memory and nearly all shared memory) fill whole waves.
-template <int COPIES>
+// tcgen05 attention launch.  Two shapes: 128-key tiles, one CTA per SM (long key ranges), and 64-key tiles, two CTAs
+// per SM (a CTA that lives for a few tiles only: start-up and output of one overlap the tile loop of the other).
+template <int KT, int SBUF>
 int launch_attn_tmem(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
-  auto kern = attn::attn_tmem_kernel<COPIES>;
+  auto kern = attn::attn_tmem_kernel<KT, SBUF>;
+  const size_t smem = attn::TmLayout<KT, SBUF>::smem_bytes();
   static bool attr_set = false;
   if (!attr_set) {
-    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::attn_tmem_smem_bytes())));
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
     attr_set = true;
   }
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = grid;
   cfg.blockDim = dim3(attn::TM_THREADS);
-  cfg.dynamicSmemBytes = attn::attn_tmem_smem_bytes();
+  cfg.dynamicSmemBytes = smem;
   cfg.stream = c->stream;
   cudaLaunchAttribute at[2];
   int na = 0;
@@ -1043,7 +1045,7 @@ int launch_attn_tmem(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
   }
   cfg.attrs = at;
   cfg.numAttrs = na;
-  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, c->kv_tmap128, p));
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, KT == 64 ? c->kv_tmap : c->kv_tmap128, p));
   LAUNCHED(c, "attn_tmem_kernel");
   return D3_OK;
 }
@@ -1052,14 +1054,18 @@ int run_attention_tmem(d3_ctx* c, const void* q, int layer, void* out, const Row
   const d3_config& g = c->cfg;
   const int group = g.n_q_heads / g.n_kv_heads;
   const int R = group * rm.rows_per_seq;
-  const int copies = R <= 32 ? 4 : (R <= 64 ? 2 : 1);
-  const int rpc = 128 / copies;
-  const int q_tiles = (R + rpc - 1) / rpc;
+  const int q_tiles = (R + 127) / 128;
   const int pairs = rm.bs * g.n_kv_heads;
-  const int slots = c->n_sms;
+  // short key ranges (at most 8 tiles of 128 keys per CTA) and enough CTAs to fill two per SM: the small shape
+  bool small = g.max_seq <= 1024 && pairs * q_tiles >= 2 * c->n_sms;
+  if (c->tune_attn_shape > 0) small = c->tune_attn_shape == 64;
+  const int kt = small ? 64 : 128;
+  const int slots = c->n_sms * (small ? 2 : 1);
   int splits = 1;
   if (q_tiles <= 2 && pairs * q_tiles < slots) {
-    const int max_tiles = (g.max_seq + attn::TKT - 1) / attn::TKT;
+    // decode-sized: (sequence, kv head) pairs alone leave SMs idle, so the keys of a query tile are split over a
+    // cluster (at most 8 CTAs, at least two key tiles each).  Cost of a split count: waves x key tiles per CTA.
+    const int max_tiles = (g.max_seq + kt - 1) / kt;
     const int cap = std::max(1, std::min(8, max_tiles / 2));
     auto cost_of = [&](int s) {
       const long long waves = (static_cast<long long>(pairs) * q_tiles * s + slots - 1) / slots;
@@ -1082,11 +1088,7 @@ int run_attention_tmem(d3_ctx* c, const void* q, int layer, void* out, const Row
   p.scale_log2 = 1.4426950408889634f / std::sqrt(static_cast<float>(g.d_head));
   p.error_word = c->error_word;
   dim3 grid(q_tiles, pairs, splits);
-  switch (copies) {
-    case 4: return launch_attn_tmem<4>(c, p, grid);
-    case 2: return launch_attn_tmem<2>(c, p, grid);
-    default: return launch_attn_tmem<1>(c, p, grid);
-  }
+  return small ? launch_attn_tmem<64, 1>(c, p, grid) : launch_attn_tmem<128, 2>(c, p, grid);
 }
 
 int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
@@ -1414,7 +1416,7 @@ extern "C" int d3_create(const d3_config* cfg, void* cuda_stream, d3_ctx** out) 
       rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, tc::CHAIN_AKT, &tm);
       if (rc_ != D3_OK) return bail(rc_);
       c->kv_tmap32 = *tm;
-      rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, attn::TKT, &tm);
+      rc_ = get_tmap(c, c->kv, static_cast<int>(kv_rows), 128, 128, &tm);
       if (rc_ != D3_OK) return bail(rc_);
       c->kv_tmap128 = *tm;
       c->attn_tc = true;
@@ -2085,7 +2087,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
       t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
       (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
       t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256 || t->weights_as_rows < -1 || t->weights_as_rows > 0 ||
-      t->attention_tmem < -1 || t->attention_tmem > 1)
+      (t->attention_tmem < -1 || t->attention_tmem > 1) && t->attention_tmem != 64 && t->attention_tmem != 128)
     return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
   c->tune_ring_kb = t->ring_kb;
   c->tune_ctas_per_sm = t->ctas_per_sm;
@@ -2101,7 +2103,8 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   c->tune_chain_clusters = t->chain_clusters;
   c->tune_chain_l2 = t->chain_l2_ahead;
   c->tune_xt = t->weights_as_rows;
-  c->tune_attn_tmem = t->attention_tmem;
+  c->tune_attn_tmem = t->attention_tmem > 1 ? 1 : t->attention_tmem;
+  c->tune_attn_shape = t->attention_tmem > 1 ? t->attention_tmem : 0;
   return D3_OK;
 }
 extern "C" int d3_set_fused_finalize(d3_ctx* c, int on) {

@@ -326,12 +326,13 @@ def test_attention_bf16_tensor_core(shape, rows, kv_lens):
 @pytest.mark.parametrize("rows,kv_lens", [(32, [64, 33, 1]), (32, [600, 65, 257]), (64, [640, 63, 128]),
                                           (7, [40, 300, 5]), (100, [100, 37, 129]), (300, [300, 5, 64]),
                                           (32, [128, 256, 384]), (40, [129, 127, 640])])
-def test_attention_bf16_tensor_memory(shape, rows, kv_lens):
-    """The same cases on the tcgen05 kernel (S and O in tensor memory, V as an MN-major operand): 32 rows of
-    one head run as four copies of the tile that split every key tile, 64 rows as two, group 7 as whole
-    128-row tiles; one to five key tiles, ragged last tiles, key splits over a cluster."""
+@pytest.mark.parametrize("keys_per_tile", [64, 128])
+def test_attention_bf16_tensor_memory(shape, rows, kv_lens, keys_per_tile):
+    """The same cases on the tcgen05 kernel (S, P, O and Q in tensor memory, V as an MN-major operand), in both
+    shapes (64-key tiles with one S buffer, 128-key tiles with two): whole and partly filled 128-row tiles, one to
+    ten key tiles, ragged last tiles, key splits over a cluster."""
     with Ctx(shape, None, block=32, max_batch=3, max_seq=640, max_prefill_rows=3 * 300) as ctx:
-        d3.d3_set_tuning(ctx.ctx, attention_tmem=1)
+        d3.d3_set_tuning(ctx.ctx, attention_tmem=keys_per_tile)
         _attention_case(ctx, shape, True, 3, rows, kv_lens, rows + sum(kv_lens))
         _attention_case(ctx, shape, True, 3, rows, kv_lens, rows + sum(kv_lens))
         assert d3.d3_launch_count_of(ctx.ctx, "attn_tmem_kernel") == 2
