@@ -23,9 +23,10 @@
 //
 // Fewer than 128 packed rows leave lanes (and whole warps, which then skip the softmax) idle; the MMAs do not care.
 //
-// Two shapes of the same code:  <128 keys per tile, 2 S buffers>: 448 columns of tensor memory, 192 KB of K/V in
-// flight, one CTA per SM, for long key ranges;  <64, 1>: 256 columns, 96 KB, two CTAs per SM, whose start-up, serial
-// tile loop and output overlap each other: for short key ranges, where a CTA lives for a few tiles only.
+// Two shapes of the same code:  <128 keys per tile>: 448 columns of tensor memory, 192 KB of K/V in flight, one CTA
+// per SM, for long key ranges;  <64>: 256 columns (Q stays in shared memory and the first product takes both
+// operands from there), 64 KB in flight, two CTAs per SM, whose start-up and output overlap the other's tile loop:
+// for short key ranges, where a CTA lives for a few tiles only.
 //
 // Key splits: as in attn_tc_kernel, the CTAs of one query tile form a cluster along z and merge their partials
 // through distributed shared memory.
@@ -35,7 +36,6 @@
 namespace d3 {
 namespace attn {
 
-constexpr int TM_STAGES = 6;                   // ring of K / V tiles
 constexpr int TM_THREADS = 192;
 constexpr float TM_SLACK_LOG2 = 8.f;           // how far a tile's maximum may exceed the reference before it moves
 
@@ -63,10 +63,16 @@ template <int KT, int SBUF>
 struct TmLayout {
   static constexpr uint32_t SLAB = static_cast<uint32_t>(KT) * 128u;  // [KT keys][64 bf16], swizzled
   static constexpr uint32_t TILE = 2u * SLAB;                         // one K or V tile: d 0-63, d 64-127
-  static constexpr uint32_t OFF_BAR = TM_STAGES * TILE;
+  // The small shape keeps Q in shared memory (two K-major slabs of [128 rows][64 bf16]): S twice, O and Q together
+  // do not fit the 256 columns that let two CTAs share an SM's tensor memory.
+  static constexpr bool Q_SMEM = KT == 64;
+  static constexpr int STAGES = Q_SMEM ? 4 : 6;                       // ring of K / V tiles
+  static constexpr uint32_t Q_SLAB = 128u * 128u;
+  static constexpr uint32_t OFF_RING = Q_SMEM ? 2u * Q_SLAB : 0u;
+  static constexpr uint32_t OFF_BAR = OFF_RING + STAGES * TILE;
   static constexpr uint32_t COL_S = 0, COL_O = SBUF * KT, COL_Q = COL_O + 128;  // tensor-memory columns
-  static constexpr uint32_t COLS = COL_Q + 64 <= 256 ? 256 : 512;               // allocation: a power of two
-  static constexpr size_t smem_bytes() { return 1024 + OFF_BAR + (2 * TM_STAGES + 2 * SBUF + 4) * 8 + 64; }
+  static constexpr uint32_t COLS = (Q_SMEM ? COL_Q : COL_Q + 64) <= 256 ? 256 : 512;  // allocation: a power of two
+  static constexpr size_t smem_bytes() { return 1024 + OFF_BAR + (2 * STAGES + 2 * SBUF + 4) * 8 + 64; }
 };
 
 // grid (q_tiles, bs * hkv, n_splits); 128 packed rows per query tile.
@@ -79,8 +85,8 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
-  uint64_t* kv_empty = kv_full + TM_STAGES;
-  uint64_t* s_full = kv_empty + TM_STAGES;  // [SBUF] S_i complete in tensor memory
+  uint64_t* kv_empty = kv_full + L::STAGES;
+  uint64_t* s_full = kv_empty + L::STAGES;  // [SBUF] S_i complete in tensor memory
   uint64_t* p_full = s_full + SBUF;         // [SBUF] P_i in tensor memory (over S_i), O rescaled where it had to be
   uint64_t* o_full = p_full + SBUF;         // second product of tile i complete (O updated, P_i and V_i read)
   uint64_t* q_full = o_full + 1;            // Q in tensor memory
@@ -112,7 +118,7 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
   }
   if (threadIdx.x == 0) {
     ptx::prefetch_tensormap(&tmap_kv);
-    for (int s = 0; s < TM_STAGES; ++s) {
+    for (int s = 0; s < L::STAGES; ++s) {
       ptx::mbar_init(&kv_full[s], 1);
       ptx::mbar_init(&kv_empty[s], 1);
     }
@@ -151,16 +157,16 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
       bool waited = false, ok = true;
       int s = 0;  // position in the ring
       auto load = [&](bool is_k, int i) {
-        const int stage = s % TM_STAGES;
-        if (s >= TM_STAGES &&
-            !ptx::mbar_wait(&kv_empty[stage], static_cast<uint32_t>(s / TM_STAGES - 1) & 1u, abort_flag, p.error_word))
+        const int stage = s % L::STAGES;
+        if (s >= L::STAGES &&
+            !ptx::mbar_wait(&kv_empty[stage], static_cast<uint32_t>(s / L::STAGES - 1) & 1u, abort_flag, p.error_word))
           return false;
         const int j0 = (t0 + i) * KT;
         if (!waited && j0 + KT > stable_keys) {  // this tile holds rows the QKV kernel of this layer writes
           ptx::grid_dep_wait();
           waited = true;
         }
-        uint8_t* dst = smem + stage * L::TILE;
+        uint8_t* dst = smem + L::OFF_RING + stage * L::TILE;
         const int row = static_cast<int>((is_k ? krow : vrow) + j0);
         ptx::mbar_arrive_expect_tx(&kv_full[stage], L::TILE);
         ptx::tma_load_2d(dst, &tmap_kv, &kv_full[stage], 0, row);
@@ -184,10 +190,10 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
       ptx::tc_fence_after();
       int s = 0;  // position in the ring
       auto stage_ready = [&](uint32_t& addr) {
-        const int stage = s % TM_STAGES;
-        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(s / TM_STAGES) & 1u, abort_flag, p.error_word)) return -1;
+        const int stage = s % L::STAGES;
+        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(s / L::STAGES) & 1u, abort_flag, p.error_word)) return -1;
         ptx::tc_fence_after();
-        addr = sbase + stage * L::TILE;
+        addr = sbase + L::OFF_RING + stage * L::TILE;
         ++s;
         return stage;
       };
@@ -198,8 +204,11 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk) {  // 16 values of d_head per step = 8 columns of Q
           const uint64_t bd = tm_desc_k(kb + (kk >> 2) * L::SLAB) + static_cast<uint64_t>(2 * (kk & 3));
-          ptx::umma_bf16_ts(tmem_base + L::COL_S + static_cast<uint32_t>((i % SBUF) * KT), tmem_base + L::COL_Q + kk * 8, bd,
-                            idesc_qk, kk > 0 ? 1u : 0u);
+          const uint32_t sd = tmem_base + L::COL_S + static_cast<uint32_t>((i % SBUF) * KT);
+          if constexpr (L::Q_SMEM)
+            ptx::umma_bf16(sd, tm_desc_k(sbase + (kk >> 2) * L::Q_SLAB) + static_cast<uint64_t>(2 * (kk & 3)), bd, idesc_qk, kk > 0 ? 1u : 0u);
+          else
+            ptx::umma_bf16_ts(sd, tmem_base + L::COL_Q + kk * 8, bd, idesc_qk, kk > 0 ? 1u : 0u);
         }
         ptx::umma_commit(&kv_empty[stage]);
         ptx::umma_commit(&s_full[i % SBUF]);
@@ -238,18 +247,29 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
     const uint32_t t_o = t_lane + L::COL_O;
     const bool warp_rows = __any_sync(0xffffffffu, row_ok);  // a warp without rows only keeps the barriers going
     ptx::grid_dep_wait();  // Q comes from the kernel before this one
-    {  // this thread's row of Q into its lane: 128 bf16 = 64 columns; a row that does not exist is zero
+    {  // this thread's row of Q into its lane (128 bf16 = 64 columns) or its shared-memory row; a row that does not exist is zero
       const uint4* src = reinterpret_cast<const uint4*>(p.q + (static_cast<size_t>(b) * rps + r_seq) * p.hq * 128 +
                                                         (g * group + pr / rps) * 128);
+      if constexpr (L::Q_SMEM) {
+        // rows of a warp without any stay as they are: nobody reads what comes of them; a CTA without tiles needs no
+        // Q, and its warps write their partials over this memory without waiting for each other
+        if (warp_rows && n_my > 0) {
 #pragma unroll
-      for (int h = 0; h < 2; ++h) {
-        uint4 v[8];
+          for (int ch = 0; ch < 16; ++ch)
+            *reinterpret_cast<uint4*>(smem + (ch >> 3) * L::Q_SLAB + swz(tid, ch & 7)) = row_ok ? src[ch] : make_uint4(0u, 0u, 0u, 0u);
+          ptx::fence_proxy_async();
+        }
+      } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = row_ok ? src[h * 8 + j] : make_uint4(0u, 0u, 0u, 0u);
-        ptx::tmem_st_32x32(t_lane + L::COL_Q + h * 32, *reinterpret_cast<const float(*)[32]>(v));
+        for (int h = 0; h < 2; ++h) {
+          uint4 v[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) v[j] = row_ok ? src[h * 8 + j] : make_uint4(0u, 0u, 0u, 0u);
+          ptx::tmem_st_32x32(t_lane + L::COL_Q + h * 32, *reinterpret_cast<const float(*)[32]>(v));
+        }
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before();
       }
-      ptx::tmem_st_wait();
-      ptx::tc_fence_before();
       ptx::mbar_arrive(q_full);
     }
     const int kv_lim = row_ok ? row_kv_limit(p.rm, b, r_seq, kv_len) : kv_len;
@@ -415,7 +435,7 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
   if (warp_id == 5) ptx::tmem_dealloc<L::COLS>(tmem_base);
 }
 
-static_assert(TmLayout<64, 1>::OFF_BAR >= 128 * PART_LD * 4, "the partials of the key splits overlay the ring");
+static_assert(TmLayout<64, 2>::OFF_BAR >= 128 * PART_LD * 4, "the partials of the key splits overlay Q and the ring");
 
 }  // namespace attn
 }  // namespace d3

@@ -1088,14 +1088,18 @@ int run_attention_tmem(d3_ctx* c, const void* q, int layer, void* out, const Row
   p.scale_log2 = 1.4426950408889634f / std::sqrt(static_cast<float>(g.d_head));
   p.error_word = c->error_word;
   dim3 grid(q_tiles, pairs, splits);
-  return small ? launch_attn_tmem<64, 1>(c, p, grid) : launch_attn_tmem<128, 2>(c, p, grid);
+  return small ? launch_attn_tmem<64, 2>(c, p, grid) : launch_attn_tmem<128, 2>(c, p, grid);
 }
 
 int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
   const d3_config& g = c->cfg;
   const int group = g.n_q_heads / g.n_kv_heads;
   const int R = group * rm.rows_per_seq;
-  if (c->tune_attn_tmem == 1) return run_attention_tmem(c, q, layer, out, rm);
+  // From 64 packed rows per kv head on (long blocks, fused finalize, grouped query heads, prefill) the tcgen05 kernel
+  // is the faster one (measured: 60-70 against 84-110 us per layer at 64 rows x 4200-5100 keys, 27 against 33-37 at
+  // 224 rows x 550-1000 keys, a third of the time on 4096-row prompts); at 32 rows the two are level on batches and
+  // the mma.sync kernel, with its cheaper start, is ahead on a single sequence (15 against 19 us).
+  if (c->tune_attn_tmem == 1 || (c->tune_attn_tmem < 0 && R >= 64)) return run_attention_tmem(c, q, layer, out, rm);
   const int nw = R <= 32 ? 2 : (R <= 64 ? 4 : 8);
   const int q_tiles = (R + nw * 16 - 1) / (nw * 16);
   const int pairs = rm.bs * g.n_kv_heads;
