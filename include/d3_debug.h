@@ -47,6 +47,8 @@ typedef struct d3_tuning {
                                (attn_tmem_kernel) instead of mma.sync (attn_tc_kernel): -1 = where measured faster
                                (default), 0 never, 1 wherever the shape allows (bf16, d_head 128), 64 or 128 = the same with
                                that many keys per tile (two CTAs per SM / one) instead of the launcher's choice */
+  int32_t cta_pairs;        /* matmuls of at least 512 rows on tiled weights run 256 x 256 tiles on pairs of CTAs that share
+                               one MMA (cta_group::2, gemm_pair_kernel): -1 = when the shape allows (default), 0 never */
 } d3_tuning;
 void d3_tuning_defaults(d3_tuning *t);
 int d3_set_tuning(d3_ctx *ctx, const d3_tuning *t);

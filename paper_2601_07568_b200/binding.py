@@ -358,7 +358,7 @@ def d3_set_overlap(ctx, on: bool) -> None:
 class d3_tuning(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("ring_kb", "ctas_per_sm", "producers", "tile_columns", "attn_key_tiles",
                                           "cluster_k_split", "row_tile_pairs", "round_robin", "column_strips",
-                                          "strip_stages", "chain", "chain_clusters", "chain_l2_ahead", "weights_as_rows", "attention_tmem")]
+                                          "strip_stages", "chain", "chain_clusters", "chain_l2_ahead", "weights_as_rows", "attention_tmem", "cta_pairs")]
 
 
 def d3_tuning_defaults() -> d3_tuning:

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libd3.so")
 SOURCES = ["d3_api.cu"]
-HEADERS = ["common.cuh", "ptx_sm100.cuh", "gemm_tc.cuh", "gemm_xt.cuh", "chain.cuh", "gemm_simt.cuh", "attention.cuh", "attention_tmem.cuh", "small_kernels.cuh"]
+HEADERS = ["common.cuh", "ptx_sm100.cuh", "gemm_tc.cuh", "gemm_xt.cuh", "gemm_pair.cuh", "chain.cuh", "gemm_simt.cuh", "attention.cuh", "attention_tmem.cuh", "small_kernels.cuh"]
 
 
 def _nvcc() -> str:

@@ -22,6 +22,7 @@
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "gemm_pair.cuh"
 #include "gemm_xt.cuh"
 #include "small_kernels.cuh"
 
@@ -119,6 +120,8 @@ struct d3_ctx {
   int tune_chain_l2 = -1;       // weight slabs the chain's L2 prefetch runs ahead (-1: default, 0: off)
   int tune_attn_shape = 0;      // experiment: keys per tile of the tcgen05 attention (0 = by rule, 64, 128)
   int tune_attn_tmem = -1;      // tcgen05 attention: -1 where measured faster, 0 never, 1 wherever the shape allows
+  int tune_cta_pairs = -1;      // wide matmuls on CTA pairs (cta_group::2): -1 when the shape allows, 0 never
+  int pair_clusters = 0;        // CTA pairs of gemm_pair_kernel resident at once (asked once)
   int tune_xt = -1;             // 129..256-row matmuls with weights as the 128-row operand: -1 when the shape allows, 0 never
   unsigned int* chain_sync = nullptr;  // [operators of the program] border counters of a forward's chain launches
   void* chain_prog = nullptr;          // the forward's operators (tc::ChainOp) on the device
@@ -875,6 +878,83 @@ int run_chain(d3_ctx* c, int op_begin, int op_end, const RowMap& rm) {
 
 // Tile width: 128 columns while weight streaming dominates, 256 when
 // it is bound by the tensor pipe (from 512 rows on: a third less operand traffic per flop).
+// Wide matmuls on CTA pairs (gemm_pair.cuh): 256 x 256 tiles, one cluster of two CTAs per tile at a time.
+template <int EPI>
+int launch_pair(d3_ctx* c, const CUtensorMap* tx, const tc::GemmParams& p, int tiles) {
+  auto kern = tc::gemm_pair_kernel<EPI>;
+  const size_t smem = tc::gemm_pair_smem_bytes();
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    attr_set = true;
+  }
+  cudaLaunchConfig_t cfg{};
+  cfg.blockDim = dim3(tc::PAIR_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute at[2];
+  at[0].id = cudaLaunchAttributeClusterDimension;
+  at[0].val.clusterDim.x = 2;
+  at[0].val.clusterDim.y = 1;
+  at[0].val.clusterDim.z = 1;
+  cfg.attrs = at;
+  cfg.numAttrs = 1;
+  if (c->pair_clusters == 0) {  // pairs that are resident at once (a pair sits on the two SMs of one TPC)
+    cfg.gridDim = dim3(static_cast<unsigned>(c->n_sms & ~1));
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) {
+      (void)cudaGetLastError();
+      n = 1;
+    }
+    c->pair_clusters = std::min(n, c->n_sms / 2);
+  }
+  cfg.gridDim = dim3(static_cast<unsigned>(2 * std::min(c->pair_clusters, tiles)));
+  if (c->pdl && !c->prof_on) {
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
+  }
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, *tx, p));
+  LAUNCHED(c, "gemm_pair_kernel");
+  return D3_OK;
+}
+
+bool pair_usable(const d3_ctx* c, int M, int N, int K, int epi, int w_tiled) {
+  return c->tune_cta_pairs != 0 && w_tiled && M >= 512 && N % 256 == 0 && K % 64 == 0 && epi != EPI_STATS;
+}
+
+int run_linear_pair(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep, const QkvExtra* qx) {
+  tc::GemmParams p{};
+  p.M = M; p.N = N; p.K = K;
+  p.a_rows = 128;
+  p.k_chunks = K / 64;
+  p.m_tiles = (M + 255) / 256; p.n_tiles = N / 256;
+  p.error_word = c->error_word;
+  p.skip_flag = c->skip_flag;
+  p.w_tiled = 1;
+  if ((reinterpret_cast<uintptr_t>(W) & 15) != 0) return fail(c, D3_ERR_UNSUPPORTED, "tiled weights must be 16-byte aligned");
+  p.w_packed = static_cast<const bf16*>(W);
+  p.w_blocks = static_cast<long long>(N / 128) * p.k_chunks;
+  p.ep = ep;
+  if (qx) {
+    p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
+    p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
+    p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
+    p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
+  }
+  const CUtensorMap* tx;
+  TRY(get_tmap(c, X, M, K, 128, &tx));
+  const int tiles = p.m_tiles * p.n_tiles;
+  switch (epi) {
+    case EPI_F32: return launch_pair<EPI_F32>(c, tx, p, tiles);
+    case EPI_T: return launch_pair<EPI_T>(c, tx, p, tiles);
+    case EPI_RESID: return launch_pair<EPI_RESID>(c, tx, p, tiles);
+    case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(c, tx, p, tiles);
+    case EPI_QKV: return launch_pair<EPI_QKV>(c, tx, p, tiles);
+  }
+  return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
+}
+
 int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep,
                   int ctas_hint, const QkvExtra* qx, int w_tiled) {
   // `ctas_hint` 1..8 on a skinny matmul forces the cluster size; larger hints ask for the unit-range kernel
@@ -907,6 +987,7 @@ int run_linear_tc(d3_ctx* c, const void* X, const void* W, int M, int N, int K, 
     int xt_stages = 0;
     if (xt_usable(c, M, N, K, epi, w_tiled, &xs, &xt_stages)) return run_linear_xt(c, X, W, M, N, K, epi, ep, qx, xs, xt_stages);
   }
+  if (ctas_hint == 0 && c->tune_wide_tiles < 0 && pair_usable(c, M, N, K, epi, w_tiled)) return run_linear_pair(c, X, W, M, N, K, epi, ep, qx);
   const bool wide = c->tune_wide_tiles >= 0 ? c->tune_wide_tiles != 0 : M >= 512;
   if (wide && N >= 256) return run_linear_tc_bn<256, 1>(c, X, W, M, N, K, epi, ep, ctas_hint, qx, w_tiled);
   // 129..511 rows: two row tiles per unit share each weight slab
@@ -2083,6 +2164,7 @@ extern "C" void d3_tuning_defaults(d3_tuning* t) {
   t->chain_l2_ahead = -1;
   t->weights_as_rows = -1;
   t->attention_tmem = -1;
+  t->cta_pairs = -1;
 }
 extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   if (!c || !t) return D3_ERR_INVALID_ARG;
@@ -2091,7 +2173,8 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
       t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
       (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
       t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256 || t->weights_as_rows < -1 || t->weights_as_rows > 0 ||
-      (t->attention_tmem < -1 || t->attention_tmem > 1) && t->attention_tmem != 64 && t->attention_tmem != 128)
+      ((t->attention_tmem < -1 || t->attention_tmem > 1) && t->attention_tmem != 64 && t->attention_tmem != 128) ||
+      t->cta_pairs < -1 || t->cta_pairs > 0)
     return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
   c->tune_ring_kb = t->ring_kb;
   c->tune_ctas_per_sm = t->ctas_per_sm;
@@ -2109,6 +2192,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
   c->tune_xt = t->weights_as_rows;
   c->tune_attn_tmem = t->attention_tmem > 1 ? 1 : t->attention_tmem;
   c->tune_attn_shape = t->attention_tmem > 1 ? t->attention_tmem : 0;
+  c->tune_cta_pairs = t->cta_pairs;
   return D3_OK;
 }
 extern "C" int d3_set_fused_finalize(d3_ctx* c, int on) {

@@ -1,0 +1,185 @@
+// Wide matmuls (Y = X W^T with at least 512 rows) on CTA pairs: a cluster of two CTAs owns a 256 x 256 tile of Y and
+// one tcgen05.mma.cta_group::2 of M = 256 computes it.  Each CTA stages its own 128 rows of X (TMA) and its own
+// 128 of the tile's 256 weight rows (one pre-swizzled 16 KB block, bulk copy) per 64-wide K slab: 32 KB of shared
+// memory traffic per CTA and slab where a lone CTA with a 128 x 256 tile moves 48 KB for the same arithmetic.  The
+// L2-to-shared-memory path is what paces those tiles, so the pair form gains what it saves there.
+//
+// Per CTA, 192 threads: warp 0 producer (one thread), warp 1 the MMA thread in the leader (rank 0) and a relay
+// thread in the peer, warps 2-5 epilogue (one row = one tensor-memory lane per thread).
+// Hand-over per ring stage s:
+//   producer (both CTAs)  waits empty[s], expects 32 KB on its own full[s], issues its two copies
+//   relay (peer)          waits the peer's full[s], then arrives (release, cluster scope) on the leader's peer_full[s]
+//   MMA thread (leader)   waits full[s] and peer_full[s], issues four MMAs (K = 16 each) that read both CTAs' stages,
+//                         commits to empty[s] of both CTAs (tcgen05.commit with a CTA mask)
+// Accumulators: two of 256 columns per CTA (all 512 columns, allocated pair-wide), so that the epilogue of a tile
+// runs under the MMAs of the next one; the last commit of a tile goes to acc_full[buf] of both CTAs, and every
+// epilogue warp of both CTAs arrives on the leader's acc_empty[buf] when it has read its lanes.
+// Tiles are dealt round-robin to the pairs, row tiles fastest, so the pairs of a moment share weight blocks and the
+// rows of X through L2.  Epilogues are those of gemm_tc.cuh (run_epilogue on 256 columns).
+#pragma once
+#include "gemm_tc.cuh"
+
+namespace d3 {
+namespace tc {
+
+constexpr int PAIR_THREADS = 192;
+constexpr int PAIR_STAGES = 6;
+constexpr uint32_t PAIR_A_BYTES = 128u * 128u;  // [128 rows][64 bf16]
+constexpr uint32_t PAIR_B_BYTES = 128u * 128u;  // one weight block
+constexpr uint32_t PAIR_STAGE_BYTES = PAIR_A_BYTES + PAIR_B_BYTES;
+
+// kind::f16 instruction descriptor of the pair MMA: D fp32, A and B bf16 K-major, N >> 3 in [17,23), M >> 4 in [24,29).
+constexpr uint32_t PAIR_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(256 >> 3) << 17) |
+                                (static_cast<uint32_t>(256 >> 4) << 24);
+
+inline size_t gemm_pair_smem_bytes() { return 1024 + PAIR_STAGES * PAIR_STAGE_BYTES + (3 * PAIR_STAGES + 4) * 8 + 64; }
+
+// grid = 2 x pairs, cluster (2, 1, 1).  p: M, N (multiple of 256), K (multiple of 64), k_chunks, w_packed (tiled
+// weights), ep and, for EPI_QKV, the RoPE and cache fields.  tmap_x: X as [M, K] with boxes of 128 rows.
+template <int EPI>
+__global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
+  if (p.skip_flag != nullptr && *p.skip_flag != 0) return;  // uniform over the grid
+  grid_dep_launch();
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + PAIR_STAGES * PAIR_STAGE_BYTES);
+  uint64_t* empty_bar = full_bar + PAIR_STAGES;
+  uint64_t* peer_full = empty_bar + PAIR_STAGES;  // used in the leader only
+  uint64_t* acc_full = peer_full + PAIR_STAGES;   // [2]
+  uint64_t* acc_empty = acc_full + 2;             // [2], used in the leader only
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int m_tiles = (p.M + 255) / 256, n_tiles = p.N / 256;
+  const int tiles = m_tiles * n_tiles;
+  const int my_tiles = pair < tiles ? (tiles - pair + n_pairs - 1) / n_pairs : 0;
+  const int KC = p.k_chunks;
+
+  if (threadIdx.x == 0) {
+    prefetch_tensormap(&tmap_x);
+    for (int s = 0; s < PAIR_STAGES; ++s) {
+      mbar_init(&full_bar[s], 1);
+      mbar_init(&empty_bar[s], 1);
+      mbar_init(&peer_full[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&acc_full[b], 1);
+      mbar_init(&acc_empty[b], 8);  // four epilogue warps of each CTA
+    }
+    *abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair<512>(tmem_slot);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  cluster_sync_all();  // barriers of both CTAs exist before either signals the other
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      grid_dep_wait();  // X comes from the kernel before this one
+      int it = 0;
+      bool ok = true;
+      for (int t = 0; t < my_tiles && ok; ++t) {
+        const int q = pair + t * n_pairs;
+        const int m_t = q % m_tiles, n_t = q / m_tiles;
+        const int row0 = m_t * 256 + static_cast<int>(rank) * 128;
+        const __nv_bfloat16* wblk = p.w_packed + (static_cast<size_t>(n_t * 2 + static_cast<int>(rank)) * KC) * (128 * 64);
+        for (int kc = 0; kc < KC; ++kc, ++it) {
+          const int s = it % PAIR_STAGES;
+          if (it >= PAIR_STAGES && !mbar_wait(&empty_bar[s], static_cast<uint32_t>(it / PAIR_STAGES - 1) & 1u, abort_flag, p.error_word)) {
+            ok = false;
+            break;
+          }
+          uint8_t* st = smem + s * PAIR_STAGE_BYTES;
+          mbar_arrive_expect_tx(&full_bar[s], PAIR_STAGE_BYTES);
+          tma_load_2d(st, &tmap_x, &full_bar[s], kc * 64, row0);
+          bulk_load_1d(st + PAIR_A_BYTES, wblk + static_cast<size_t>(kc) * (128 * 64), PAIR_B_BYTES, &full_bar[s]);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      if (rank != 0) {
+        // -------------------------------------------------------------- relay (peer): its stage has landed
+        int it = 0;
+        bool ok = true;
+        for (int t = 0; t < my_tiles && ok; ++t)
+          for (int kc = 0; kc < KC; ++kc, ++it) {
+            const int s = it % PAIR_STAGES;
+            if (!mbar_wait(&full_bar[s], static_cast<uint32_t>(it / PAIR_STAGES) & 1u, abort_flag, p.error_word)) {
+              ok = false;
+              break;
+            }
+            mbar_arrive_remote(&peer_full[s], 0);
+          }
+      } else {
+        // -------------------------------------------------------------- MMA issue (leader)
+        const uint32_t sb = smem_u32(smem);
+        int it = 0;
+        bool ok = true;
+        for (int t = 0; t < my_tiles && ok; ++t) {
+          const int buf = t & 1;
+          if (t >= 2) ok = mbar_wait_cluster(&acc_empty[buf], static_cast<uint32_t>((t >> 1) - 1) & 1u, abort_flag, p.error_word);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * 256);
+          for (int kc = 0; kc < KC; ++kc, ++it) {
+            const int s = it % PAIR_STAGES;
+            const uint32_t ph = static_cast<uint32_t>(it / PAIR_STAGES) & 1u;
+            ok = mbar_wait(&full_bar[s], ph, abort_flag, p.error_word) && mbar_wait_cluster(&peer_full[s], ph, abort_flag, p.error_word);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t adesc = make_smem_desc(sb + s * PAIR_STAGE_BYTES);
+            const uint64_t bdesc = make_smem_desc(sb + s * PAIR_STAGE_BYTES + PAIR_A_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < BLOCK_K / UMMA_K; ++kk)
+              umma_bf16_pair(tmem_d, adesc + static_cast<uint64_t>(2 * kk), bdesc + static_cast<uint64_t>(2 * kk), PAIR_IDESC,
+                             (kc > 0 || kk > 0) ? 1u : 0u);
+            umma_commit_pair(&empty_bar[s], 3);
+          }
+          if (ok) umma_commit_pair(&acc_full[buf], 3);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps: lane group = warp % 4
+    grid_dep_wait();  // residual rows, positions and row sums come from earlier kernels
+    const int lg = warp & 3;
+    const int row = lg * 32 + lane;
+    for (int t = 0; t < my_tiles; ++t) {
+      const int q = pair + t * n_pairs;
+      const int m_t = q % m_tiles, n_t = q / m_tiles;
+      const int m = m_t * 256 + static_cast<int>(rank) * 128 + row;
+      const int buf = t & 1;
+      float rs = 1.f;  // folded RMSNorm: the row's factor, fetched while the MMAs still run
+      if (p.ep.ssq_in != nullptr && m < p.M) rs = row_rstd(p.ep, m);
+      bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(t >> 1) & 1u, abort_flag, p.error_word);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const bool warp_live = m_t * 256 + static_cast<int>(rank) * 128 + lg * 32 < p.M;  // warp-uniform
+      TmemSource tsrc{tmem_base + static_cast<uint32_t>(buf * 256) + (static_cast<uint32_t>(lg * 32) << 16)};
+      if (warp_live) run_epilogue<EPI, 256>(tsrc, p, m, n_t * 256, m < p.M, 0, 1, -1, rs);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_remote(&acc_empty[buf], 0);
+    }
+  }
+  // Neither CTA may leave (its shared memory is an operand of the leader's MMAs, its barriers a target of the
+  // leader's commits) nor give back tensor memory before both are through.
+  __syncwarp();
+  tc_fence_before();
+  cluster_sync_all();
+  if (warp == 1) tmem_dealloc_pair<512>(tmem_base);
+}
+
+}  // namespace tc
+}  // namespace d3

@@ -58,7 +58,7 @@ def test_tuning_defaults_and_ranges():
     t = binding.d3_tuning_defaults()
     assert (t.ring_kb, t.ctas_per_sm, t.producers, t.tile_columns, t.attn_key_tiles) == (0, 0, 0, 0, 0)
     assert (t.cluster_k_split, t.row_tile_pairs, t.round_robin, t.column_strips, t.strip_stages, t.chain) == (-1, -1, 1, 0, 0, -1)
-    assert ctypes.sizeof(binding.d3_tuning) == 15 * 4 and t.attention_tmem == -1 and t.chain_clusters == 0 and t.chain_l2_ahead == -1 and t.weights_as_rows == -1
+    assert ctypes.sizeof(binding.d3_tuning) == 16 * 4 and t.attention_tmem == -1 and t.cta_pairs == -1 and t.chain_clusters == 0 and t.chain_l2_ahead == -1 and t.weights_as_rows == -1
     assert binding.lib().d3_set_tuning(None, ctypes.byref(t)) == binding.D3_ERR_INVALID_ARG
 
 

@@ -141,6 +141,49 @@ def test_linear_bf16_weights_as_rows(ctx_bf16, m, n, k, cluster):
     assert ctx_bf16.error_word() == 0
 
 
+@pytest.mark.parametrize("m,n,k", [(512, 256, 64), (1024, 512, 512), (640, 768, 1024), (1000, 256, 4096), (2048, 4096, 1024),
+                                   (513, 12288, 256)])
+def test_linear_bf16_cta_pairs(ctx_bf16, m, n, k):
+    """Matmuls of at least 512 rows on tiled weights: 256 x 256 tiles, each computed by one MMA of 256 rows that a
+    pair of CTAs shares (each stages its own 128 rows of X and 128 of the tile's weight rows).  Row counts that end
+    inside the leader's half, inside the peer's half and on a tile border; one K slab and many; more tiles than
+    pairs (two accumulators in turn) and fewer; fp32, residual, bf16 and SwiGLU epilogues against the fp64 product,
+    and the same through single CTAs."""
+    rng = np.random.default_rng(m + n + k)
+    xt, x = rand_bf16(rng, (m, k))
+    wt, w = rand_bf16(rng, (n, k), 0.05)
+    ref = x @ w.T
+    tol = 2e-5 * np.sqrt(k) * np.abs(ref).max() + 1e-6
+    xd, wd = xt.to(DEV), wt.to(DEV)
+    packed = torch.full((d3.d3_packed_weight_elems(n, k),), 3.0, dtype=torch.bfloat16, device=DEV)
+    d3.d3_pack_weight(ctx_bf16.ctx, wd, packed)
+    n0 = d3.d3_launch_count_of(ctx_bf16.ctx, "gemm_pair_kernel")
+    y = torch.full((m, n), 7.0, dtype=torch.float32, device=DEV)
+    d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, y, n, 0, 0)
+    assert np.max(np.abs(y.cpu().numpy() - ref)) <= tol
+    y0 = rng.standard_normal((m, n)).astype(np.float32)
+    yr = torch.from_numpy(y0).to(DEV)
+    d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, yr, n, 2, 0)
+    assert np.max(np.abs(yr.cpu().numpy() - (ref + y0))) <= tol + 1e-6
+    yb = torch.zeros((m, n), dtype=torch.bfloat16, device=DEV)
+    d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, yb, n, 1, 0)
+    assert np.max(np.abs(yb.float().cpu().numpy() - ref)) <= tol + 2 ** -8 * np.abs(ref).max()
+    h = torch.zeros((m, n // 2), dtype=torch.bfloat16, device=DEV)
+    d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, h, n, 3, 0)
+    want = swiglu_ref(ref, n)
+    assert np.max(np.abs(h.float().cpu().numpy() - want)) <= 2 ** -7 * np.abs(want).max() + tol
+    assert d3.d3_launch_count_of(ctx_bf16.ctx, "gemm_pair_kernel") == n0 + 4
+    # the same through single CTAs (switch off): same products up to the order of the fp32 sums
+    d3.d3_set_tuning(ctx_bf16.ctx, cta_pairs=0)
+    y2 = torch.full((m, n), 7.0, dtype=torch.float32, device=DEV)
+    d3.d3_op_linear_packed(ctx_bf16.ctx, xd, packed, y2, n, 0, 0)
+    d3.d3_set_tuning(ctx_bf16.ctx)
+    assert d3.d3_launch_count_of(ctx_bf16.ctx, "gemm_pair_kernel") == n0 + 4
+    assert np.max(np.abs(y2.cpu().numpy() - ref)) <= tol
+    assert np.max(np.abs(y.cpu().numpy() - y2.cpu().numpy())) <= tol
+    assert ctx_bf16.error_word() == 0
+
+
 @pytest.mark.parametrize("m,n,k,widths", [(32, 2400, 256, [16, 48, 80, 96, 240]), (64, 2400, 200, [48, 160]),
                                           (7, 4736, 1024, [32, 128]), (1, 512, 4096, [16, 256]),
                                           (100, 2400, 256, [48, 240]), (128, 4736, 512, [128, 64])])
