@@ -251,8 +251,9 @@ EncodeTiledFn get_encode_fn() {
 }
 
 // bf16 row-major [rows, cols] matrix, box = [box_rows, 64 columns], 128-byte swizzle, zero fill.
-int get_tmap(d3_ctx* c, const void* ptr, int rows, int cols, int box_rows, const CUtensorMap** out) {
-  auto key = std::make_tuple(ptr, rows, cols, box_rows);
+// `swizzle` false: rows of the box land one after the other as they are (a block that is stored pre-swizzled).
+int get_tmap(d3_ctx* c, const void* ptr, int rows, int cols, int box_rows, const CUtensorMap** out, bool swizzle = true) {
+  auto key = std::make_tuple(ptr, rows, cols, swizzle ? box_rows : -box_rows);
   auto it = c->tmaps.find(key);
   if (it != c->tmaps.end()) {
     *out = &it->second;
@@ -268,7 +269,7 @@ int get_tmap(d3_ctx* c, const void* ptr, int rows, int cols, int box_rows, const
   cuuint32_t box[2] = {64, static_cast<cuuint32_t>(box_rows)};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), gdim, gstr, box, estr,
-                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) return fail(c, D3_ERR_CUDA, "cuTensorMapEncodeTiled failed with " + std::to_string(r));
   if (c->tmaps.size() > 4096) c->tmaps.clear();
@@ -880,7 +881,7 @@ int run_chain(d3_ctx* c, int op_begin, int op_end, const RowMap& rm) {
 // it is bound by the tensor pipe (from 512 rows on: a third less operand traffic per flop).
 // Wide matmuls on CTA pairs (gemm_pair.cuh): 256 x 256 tiles, one cluster of two CTAs per tile at a time.
 template <int EPI>
-int launch_pair(d3_ctx* c, const CUtensorMap* tx, const tc::GemmParams& p, int tiles) {
+int launch_pair(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const tc::GemmParams& p, int tiles) {
   auto kern = tc::gemm_pair_kernel<EPI>;
   const size_t smem = tc::gemm_pair_smem_bytes();
   static bool attr_set = false;
@@ -914,13 +915,14 @@ int launch_pair(d3_ctx* c, const CUtensorMap* tx, const tc::GemmParams& p, int t
     at[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.numAttrs = 2;
   }
-  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, *tx, p));
+  CUDA_TRY(c, cudaLaunchKernelEx(&cfg, kern, *tx, *tw, p));
   LAUNCHED(c, "gemm_pair_kernel");
   return D3_OK;
 }
 
 bool pair_usable(const d3_ctx* c, int M, int N, int K, int epi, int w_tiled) {
-  return c->tune_cta_pairs != 0 && w_tiled && M >= 512 && N % 256 == 0 && K % 64 == 0 && epi != EPI_STATS;
+  return c->tune_cta_pairs != 0 && w_tiled && M >= 512 && N % 256 == 0 && K % 64 == 0 && epi != EPI_STATS &&
+         static_cast<long long>(N / 128) * (K / 64) * 128 < (1ll << 31);
 }
 
 int run_linear_pair(d3_ctx* c, const void* X, const void* W, int M, int N, int K, int epi, const EpiParams& ep, const QkvExtra* qx) {
@@ -942,15 +944,16 @@ int run_linear_pair(d3_ctx* c, const void* X, const void* W, int M, int N, int K
     p.n_q_heads = c->cfg.n_q_heads; p.n_kv_heads = c->cfg.n_kv_heads; p.max_seq = c->cfg.max_seq;
     p.k_cache = static_cast<bf16*>(qx->k_cache); p.v_cache = static_cast<bf16*>(qx->v_cache);
   }
-  const CUtensorMap* tx;
+  const CUtensorMap *tx, *tw;
   TRY(get_tmap(c, X, M, K, 128, &tx));
+  TRY(get_tmap(c, W, static_cast<int>(p.w_blocks) * 128, 64, 128, &tw, false));
   const int tiles = p.m_tiles * p.n_tiles;
   switch (epi) {
-    case EPI_F32: return launch_pair<EPI_F32>(c, tx, p, tiles);
-    case EPI_T: return launch_pair<EPI_T>(c, tx, p, tiles);
-    case EPI_RESID: return launch_pair<EPI_RESID>(c, tx, p, tiles);
-    case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(c, tx, p, tiles);
-    case EPI_QKV: return launch_pair<EPI_QKV>(c, tx, p, tiles);
+    case EPI_F32: return launch_pair<EPI_F32>(c, tx, tw, p, tiles);
+    case EPI_T: return launch_pair<EPI_T>(c, tx, tw, p, tiles);
+    case EPI_RESID: return launch_pair<EPI_RESID>(c, tx, tw, p, tiles);
+    case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(c, tx, tw, p, tiles);
+    case EPI_QKV: return launch_pair<EPI_QKV>(c, tx, tw, p, tiles);
   }
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }

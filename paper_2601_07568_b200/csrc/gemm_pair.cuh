@@ -1,21 +1,27 @@
 // Wide matmuls (Y = X W^T with at least 512 rows) on CTA pairs: a cluster of two CTAs owns a 256 x 256 tile of Y and
 // one tcgen05.mma.cta_group::2 of M = 256 computes it.  Each CTA stages its own 128 rows of X (TMA) and its own
-// 128 of the tile's 256 weight rows (one pre-swizzled 16 KB block, bulk copy) per 64-wide K slab: 32 KB of shared
+// 128 of the tile's 256 weight rows (one pre-swizzled 16 KB block) per 64-wide K slab, both by TMA: 32 KB of shared
 // memory traffic per CTA and slab where a lone CTA with a 128 x 256 tile moves 48 KB for the same arithmetic.  The
 // L2-to-shared-memory path is what paces those tiles, so the pair form gains what it saves there.
 //
-// Per CTA, 192 threads: warp 0 producer (one thread), warp 1 the MMA thread in the leader (rank 0) and a relay
-// thread in the peer, warps 2-5 epilogue (one row = one tensor-memory lane per thread).
+// Per CTA, 192 threads: warp 0 producer (one thread), warp 1 the MMA thread (in the leader, rank 0, only), warps 2-5
+// epilogue (one row = one tensor-memory lane per thread).
 // Hand-over per ring stage s:
-//   producer (both CTAs)  waits empty[s], expects 32 KB on its own full[s], issues its two copies
-//   relay (peer)          waits the peer's full[s], then arrives (release, cluster scope) on the leader's peer_full[s]
-//   MMA thread (leader)   waits full[s] and peer_full[s], issues four MMAs (K = 16 each) that read both CTAs' stages,
-//                         commits to empty[s] of both CTAs (tcgen05.commit with a CTA mask)
+//   producer (both CTAs)  waits its empty[s] and issues its two tile loads (cta_group::2 form: the bytes land in
+//                         its own shared memory and are counted on the LEADER's full[s]); the leader's producer
+//                         first expects the 64 KB of both CTAs there
+//   MMA thread (leader)   waits full[s], issues four MMAs (K = 16 each) that read both CTAs' stages, commits to
+//                         empty[s] of both CTAs (tcgen05.commit with a CTA mask)
+// (A first form, in which the peer's loads were counted on its own barrier and a relay thread passed each stage on
+// to the leader with a remote arrive, ran at half the speed of the single-CTA kernel: the extra hop per stage is
+// longer than the six stages cover.)  The weights, pre-swizzled 128 x 64 blocks stored one after the other, are read
+// through a tensor map over [blocks * 128 rows][64] without swizzle, which copies a block verbatim.
 // Accumulators: two of 256 columns per CTA (all 512 columns, allocated pair-wide), so that the epilogue of a tile
 // runs under the MMAs of the next one; the last commit of a tile goes to acc_full[buf] of both CTAs, and every
 // epilogue warp of both CTAs arrives on the leader's acc_empty[buf] when it has read its lanes.
-// Tiles are dealt round-robin to the pairs, row tiles fastest, so the pairs of a moment share weight blocks and the
-// rows of X through L2.  Epilogues are those of gemm_tc.cuh (run_epilogue on 256 columns).
+// Tiles are dealt round-robin to the pairs in bands of eight row tiles (2048 rows), row tiles fastest inside a band:
+// the pairs of a moment share a few weight blocks, and a band's rows of X stay in L2 while all column tiles pass
+// (with row tiles fastest over all of a 16384-row X, every column tile streamed X from HBM again: 17 % slower).  Epilogues are those of gemm_tc.cuh (run_epilogue on 256 columns).
 #pragma once
 #include "gemm_tc.cuh"
 
@@ -24,6 +30,7 @@ namespace tc {
 
 constexpr int PAIR_THREADS = 192;
 constexpr int PAIR_STAGES = 6;
+constexpr int PAIR_BAND = 8;  // row tiles per band of the tile order
 constexpr uint32_t PAIR_A_BYTES = 128u * 128u;  // [128 rows][64 bf16]
 constexpr uint32_t PAIR_B_BYTES = 128u * 128u;  // one weight block
 constexpr uint32_t PAIR_STAGE_BYTES = PAIR_A_BYTES + PAIR_B_BYTES;
@@ -32,20 +39,29 @@ constexpr uint32_t PAIR_STAGE_BYTES = PAIR_A_BYTES + PAIR_B_BYTES;
 constexpr uint32_t PAIR_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(256 >> 3) << 17) |
                                 (static_cast<uint32_t>(256 >> 4) << 24);
 
-inline size_t gemm_pair_smem_bytes() { return 1024 + PAIR_STAGES * PAIR_STAGE_BYTES + (3 * PAIR_STAGES + 4) * 8 + 64; }
+__device__ __forceinline__ void pair_tile_mn(int q, int m_tiles, int n_tiles, int& m_t, int& n_t) {
+  const int band_sz = PAIR_BAND * n_tiles;
+  const int band = q / band_sz, r = q - band * band_sz;
+  const int rows_here = min(PAIR_BAND, m_tiles - band * PAIR_BAND);
+  n_t = r / rows_here;
+  m_t = band * PAIR_BAND + r % rows_here;
+}
+
+inline size_t gemm_pair_smem_bytes() { return 1024 + PAIR_STAGES * PAIR_STAGE_BYTES + (2 * PAIR_STAGES + 4) * 8 + 64; }
 
 // grid = 2 x pairs, cluster (2, 1, 1).  p: M, N (multiple of 256), K (multiple of 64), k_chunks, w_packed (tiled
-// weights), ep and, for EPI_QKV, the RoPE and cache fields.  tmap_x: X as [M, K] with boxes of 128 rows.
+// weights), ep and, for EPI_QKV, the RoPE and cache fields.  tmap_x: X as [M, K] with boxes of 128 rows (128-byte
+// swizzle); tmap_w: the weight blocks as [N / 128 * k_chunks * 128, 64] with boxes of 128 rows, no swizzle.
 template <int EPI>
-__global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const GemmParams p) {
+__global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x,
+                                                                    const __grid_constant__ CUtensorMap tmap_w, const GemmParams p) {
   if (p.skip_flag != nullptr && *p.skip_flag != 0) return;  // uniform over the grid
   grid_dep_launch();
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + PAIR_STAGES * PAIR_STAGE_BYTES);
   uint64_t* empty_bar = full_bar + PAIR_STAGES;
-  uint64_t* peer_full = empty_bar + PAIR_STAGES;  // used in the leader only
-  uint64_t* acc_full = peer_full + PAIR_STAGES;   // [2]
+  uint64_t* acc_full = empty_bar + PAIR_STAGES;   // [2]
   uint64_t* acc_empty = acc_full + 2;             // [2], used in the leader only
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -60,10 +76,10 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmap_x);
+    prefetch_tensormap(&tmap_w);
     for (int s = 0; s < PAIR_STAGES; ++s) {
       mbar_init(&full_bar[s], 1);
       mbar_init(&empty_bar[s], 1);
-      mbar_init(&peer_full[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&acc_full[b], 1);
@@ -89,9 +105,10 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
       bool ok = true;
       for (int t = 0; t < my_tiles && ok; ++t) {
         const int q = pair + t * n_pairs;
-        const int m_t = q % m_tiles, n_t = q / m_tiles;
+        int m_t, n_t;
+        pair_tile_mn(q, m_tiles, n_tiles, m_t, n_t);
         const int row0 = m_t * 256 + static_cast<int>(rank) * 128;
-        const __nv_bfloat16* wblk = p.w_packed + (static_cast<size_t>(n_t * 2 + static_cast<int>(rank)) * KC) * (128 * 64);
+        const int wrow0 = (n_t * 2 + static_cast<int>(rank)) * KC * 128;  // first row of this CTA's first weight block
         for (int kc = 0; kc < KC; ++kc, ++it) {
           const int s = it % PAIR_STAGES;
           if (it >= PAIR_STAGES && !mbar_wait(&empty_bar[s], static_cast<uint32_t>(it / PAIR_STAGES - 1) & 1u, abort_flag, p.error_word)) {
@@ -99,28 +116,16 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
             break;
           }
           uint8_t* st = smem + s * PAIR_STAGE_BYTES;
-          mbar_arrive_expect_tx(&full_bar[s], PAIR_STAGE_BYTES);
-          tma_load_2d(st, &tmap_x, &full_bar[s], kc * 64, row0);
-          bulk_load_1d(st + PAIR_A_BYTES, wblk + static_cast<size_t>(kc) * (128 * 64), PAIR_B_BYTES, &full_bar[s]);
+          if (rank == 0) mbar_arrive_expect_tx(&full_bar[s], 2 * PAIR_STAGE_BYTES);
+          const uint32_t lead_full = map_to_cta(smem_u32(&full_bar[s]), 0);
+          tma_load_2d_pair(st, &tmap_x, lead_full, kc * 64, row0);
+          tma_load_2d_pair(st + PAIR_A_BYTES, &tmap_w, lead_full, 0, wrow0 + kc * 128);
         }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      if (rank != 0) {
-        // -------------------------------------------------------------- relay (peer): its stage has landed
-        int it = 0;
-        bool ok = true;
-        for (int t = 0; t < my_tiles && ok; ++t)
-          for (int kc = 0; kc < KC; ++kc, ++it) {
-            const int s = it % PAIR_STAGES;
-            if (!mbar_wait(&full_bar[s], static_cast<uint32_t>(it / PAIR_STAGES) & 1u, abort_flag, p.error_word)) {
-              ok = false;
-              break;
-            }
-            mbar_arrive_remote(&peer_full[s], 0);
-          }
-      } else {
+      if (rank == 0) {
         // -------------------------------------------------------------- MMA issue (leader)
         const uint32_t sb = smem_u32(smem);
         int it = 0;
@@ -134,7 +139,7 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
           for (int kc = 0; kc < KC; ++kc, ++it) {
             const int s = it % PAIR_STAGES;
             const uint32_t ph = static_cast<uint32_t>(it / PAIR_STAGES) & 1u;
-            ok = mbar_wait(&full_bar[s], ph, abort_flag, p.error_word) && mbar_wait_cluster(&peer_full[s], ph, abort_flag, p.error_word);
+            ok = mbar_wait_cluster(&full_bar[s], ph, abort_flag, p.error_word);
             if (!ok) break;
             tc_fence_after();
             const uint64_t adesc = make_smem_desc(sb + s * PAIR_STAGE_BYTES);
@@ -156,7 +161,8 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
     const int row = lg * 32 + lane;
     for (int t = 0; t < my_tiles; ++t) {
       const int q = pair + t * n_pairs;
-      const int m_t = q % m_tiles, n_t = q / m_tiles;
+      int m_t, n_t;
+      pair_tile_mn(q, m_tiles, n_tiles, m_t, n_t);
       const int m = m_t * 256 + static_cast<int>(rank) * 128 + row;
       const int buf = t & 1;
       float rs = 1.f;  // folded RMSNorm: the row's factor, fetched while the MMAs still run

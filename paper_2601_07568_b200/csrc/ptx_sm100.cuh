@@ -275,6 +275,16 @@ __device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, 
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(z)
       : "memory");
 }
+// Tile load of a CTA pair: the bytes land in this CTA's shared memory and are counted on the mbarrier at
+// `bar_cluster_addr`, a shared::cluster address that may lie in the pair's other CTA (the leader's full barrier,
+// which then needs no word from the peer before it issues an MMA that reads both CTAs' tiles).
+__device__ __forceinline__ void tma_load_2d_pair(void* smem_dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(reinterpret_cast<uint64_t>(map)), "r"(bar_cluster_addr), "r"(c0), "r"(c1)
+      : "memory");
+}
 // Arrive, once all MMAs issued so far by this thread have completed, on the barrier at this shared-memory offset
 // in every CTA of `cta_mask` (bit r = rank r of the cluster).
 __device__ __forceinline__ void umma_commit_pair(uint64_t* bar, uint16_t cta_mask) {
