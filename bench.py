@@ -354,7 +354,7 @@ def measure_batched(name, W, dev, local, world, dist, peaks, steps):
                    "ms_per_forward": ms_fwd, "prefill_ms": ms_prefill},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
-                     "kernel": "gemm_tc_kernel (all matmul launches of the decode loop, CUDA events around every launch, launched serialized)",
+                     "kernel": "gemm_pair_kernel and, for the LM head, gemm_tc_kernel (all matmul launches of the decode loop, CUDA events around every launch, launched serialized)",
                      "peak_source": f"of {peaks['source']} (sustained)", "launches": n_gemm, "avg_launch_us": 1e3 * tot_ms / max(n_gemm, 1),
                      "flops_per_launch": tot_flops / max(n_gemm, 1),
                      "step_effective": {"TFLOP/s": fwd_flops / (ms_fwd / 1e3) / 1e12,
@@ -542,7 +542,7 @@ def run_ours(args):
         tot_ms, n_dom = chain["ms"], chain["launches"]
         traffic_kernel = "chain_kernel"
     else:
-        dominant = "gemm_strip_kernel, gemm_ck_kernel, gemm_tc_kernel (all matmul launches of the decode loop)"
+        dominant = "gemm_strip_kernel, gemm_ck_kernel, gemm_xt_kernel, gemm_tc_kernel, gemm_pair_kernel (all matmul launches of the decode loop)"
         tot_bytes = sum(gb[k] * prof[k]["launches"] for k in gb)
         tot_flops = sum(gf[k] * prof[k]["launches"] for k in gf)
         tot_ms = sum(prof[k]["ms"] for k in gb)
