@@ -46,7 +46,9 @@ typedef struct d3_tuning {
   int32_t attention_tmem;   /* attention with both products on tcgen05 MMAs and the accumulators in tensor memory
                                (attn_tmem_kernel) instead of mma.sync (attn_tc_kernel): -1 = where measured faster
                                (default), 0 never, 1 wherever the shape allows (bf16, d_head 128), 64 or 128 = the same with
-                               that many keys per tile (two CTAs per SM / one) instead of the launcher's choice */
+                               that many keys per tile (two CTAs per SM / one) instead of the launcher's choice, 2 = the persistent
+                               form (one CTA per SM streams through its (sequence, kv head) pairs) wherever all packed rows
+                               of a pair fit one 128-row tile, whatever the number of pairs */
   int32_t cta_pairs;        /* matmuls of at least 512 rows on tiled weights run 256 x 256 tiles on pairs of CTAs that share
                                one MMA (cta_group::2, gemm_pair_kernel): -1 = when the shape allows (default), 0 never */
 } d3_tuning;

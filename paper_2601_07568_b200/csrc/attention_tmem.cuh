@@ -437,5 +437,336 @@ __global__ void __launch_bounds__(TM_THREADS, KT == 64 ? 2 : 1) attn_tmem_kernel
 
 static_assert(TmLayout<64, 2>::OFF_BAR >= 128 * PART_LD * 4, "the partials of the key splits overlay Q and the ring");
 
+
+// ----------------------------------------------------------------------------- persistent form
+// The same tile pipeline for decode-sized batches: all packed rows of a (sequence, kv head) pair fit one 128-row
+// tile, a pair's keys take a few tiles only, and there are several pairs per SM.  A CTA per pair pays its fixed cost
+// (tensor-memory allocation, Q, first loads, pipeline fill, output: about 7 us against 1.1 us per 64-key tile) once
+// per pair, which at 32 rows x 350 keys is most of its life.  Here one CTA per SM walks through its pairs (pair
+// blockIdx.x, blockIdx.x + gridDim.x, ...) and treats their key tiles as one stream: the producer runs ahead across
+// pair borders (K/V ring, and the next pair's Q by TMA into the second Q buffer), the MMA thread issues the first
+// products of the next pair while the softmax threads read out O of the pair before, and nothing is set up twice.
+// 128-key tiles, two S buffers, Q in shared memory (two buffers of two K-major slabs), four ring stages.
+struct TmStream {
+  static constexpr int KT = 128, STAGES = 4;
+  static constexpr uint32_t SLAB = 128u * 128u, TILE = 2u * SLAB;
+  static constexpr uint32_t OFF_Q = 0, OFF_RING = 2u * TILE, OFF_BAR = OFF_RING + STAGES * TILE;
+  static constexpr uint32_t COL_S = 0, COL_O = 256;
+  static constexpr size_t smem_bytes() { return 1024 + OFF_BAR + (2 * STAGES + 9) * 8 + 64; }
+};
+
+// Position in the stream of key tiles of this CTA's pairs: pairs without live rows or keys are passed over.
+struct TmCursor {
+  int w;    // pair index (sequence * hkv + kv head); >= pairs: the stream has ended
+  int j;    // tile of the pair
+  int n_t;  // tiles of the pair
+  int qi;   // ordinal of the pair among those this CTA works on
+  int g;    // ordinal of the tile in the stream
+};
+__device__ __forceinline__ int tm_pair_tiles(const AttnTcParams& p, int w) {
+  const int b = w / p.hkv;
+  const int kv = p.rm.kv_len[b];
+  return (p.rm.n_valid[b] > 0 && kv > 0) ? (kv + TmStream::KT - 1) / TmStream::KT : 0;
+}
+__device__ __forceinline__ void tm_cursor_seek(const AttnTcParams& p, int pairs, TmCursor& c) {  // to the first pair with tiles, from c.w on
+  while (c.w < pairs && (c.n_t = tm_pair_tiles(p, c.w)) == 0) c.w += gridDim.x;
+  c.j = 0;
+}
+__device__ __forceinline__ void tm_cursor_next(const AttnTcParams& p, int pairs, TmCursor& c) {
+  ++c.g;
+  if (++c.j < c.n_t) return;
+  c.w += gridDim.x;
+  ++c.qi;
+  tm_cursor_seek(p, pairs, c);
+}
+
+// grid (min(SMs, pairs)); needs group * rows_per_seq <= 128.  tmap_q: Q as [bs * rows_per_seq, hq * 128] with boxes of
+// rows_per_seq rows x 64 columns (128-byte swizzle).
+__global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const __grid_constant__ CUtensorMap tmap_kv,
+                                                                         const __grid_constant__ CUtensorMap tmap_q,
+                                                                         const AttnTcParams p) {
+  using L = TmStream;
+  constexpr int KT = L::KT, NCH = KT / 32;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  uint64_t* kv_empty = kv_full + L::STAGES;
+  uint64_t* s_full = kv_empty + L::STAGES;  // [2]
+  uint64_t* p_full = s_full + 2;            // [2]
+  uint64_t* q_full = p_full + 2;            // [2] Q of a pair in its buffer
+  uint64_t* q_empty = q_full + 2;           // [2] the pair's last first product has read it
+  uint64_t* o_full = q_empty + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp_id = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group = p.hq / p.hkv;
+  const int rps = p.rm.rows_per_seq;
+  const int R = group * rps;
+  const int pairs = p.rm.bs * p.hkv;
+
+  if (threadIdx.x == 0) {
+    ptx::prefetch_tensormap(&tmap_kv);
+    ptx::prefetch_tensormap(&tmap_q);
+    for (int s = 0; s < L::STAGES; ++s) {
+      ptx::mbar_init(&kv_full[s], 1);
+      ptx::mbar_init(&kv_empty[s], 1);
+    }
+    for (int s = 0; s < 2; ++s) {
+      ptx::mbar_init(&s_full[s], 1);
+      ptx::mbar_init(&p_full[s], 128);
+      ptx::mbar_init(&q_full[s], 1);
+      ptx::mbar_init(&q_empty[s], 1);
+    }
+    ptx::mbar_init(o_full, 1);
+    *abort_flag = 0;
+    ptx::fence_barrier_init();
+  }
+  if (warp_id == 5) {
+    ptx::tmem_alloc<512>(tmem_slot);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  ptx::grid_dep_launch();
+  const uint32_t sbase = ptx::smem_u32(smem);
+
+  // The row map was written before this forward's first kernel started and cache rows below pos_base are not
+  // touched by this forward: both may be read before the dependency wait.
+  TmCursor c0{static_cast<int>(blockIdx.x), 0, 0, 0, 0};
+  tm_cursor_seek(p, pairs, c0);
+
+  // Producer and MMA thread walk the stream in the same order: K(0), K(1), then V(g), K(g + 2) for every tile g.
+  if (warp_id == 4) {
+    // ------------------------------------------------------------------ producer
+    if (lane == 0) {
+      bool waited = false, ok = true;
+      int s = 0;  // position in the ring
+      auto load = [&](bool is_k, const TmCursor& c) {
+        const int stage = s % L::STAGES;
+        if (s >= L::STAGES &&
+            !ptx::mbar_wait(&kv_empty[stage], static_cast<uint32_t>(s / L::STAGES - 1) & 1u, abort_flag, p.error_word))
+          return false;
+        const int b = c.w / p.hkv, g = c.w % p.hkv;
+        const int j0 = c.j * KT;
+        if (!waited && j0 + KT > p.rm.pos_base[b]) {  // this tile holds rows the QKV kernel of this layer writes
+          ptx::grid_dep_wait();
+          waited = true;
+        }
+        uint8_t* dst = smem + L::OFF_RING + stage * L::TILE;
+        const long long plane = (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
+        const int row = static_cast<int>((is_k ? p.k_row0 : p.v_row0) + plane + j0);
+        ptx::mbar_arrive_expect_tx(&kv_full[stage], L::TILE);
+        ptx::tma_load_2d(dst, &tmap_kv, &kv_full[stage], 0, row);
+        ptx::tma_load_2d(dst + L::SLAB, &tmap_kv, &kv_full[stage], 64, row);
+        ++s;
+        if (is_k && c.j == 0) {  // the pair's Q follows its first K tile
+          if (!waited) {
+            ptx::grid_dep_wait();
+            waited = true;
+          }
+          const int qb = c.qi & 1;
+          if (c.qi >= 2 && !ptx::mbar_wait(&q_empty[qb], static_cast<uint32_t>((c.qi >> 1) - 1) & 1u, abort_flag, p.error_word))
+            return false;
+          uint8_t* qd = smem + L::OFF_Q + qb * L::TILE;
+          ptx::mbar_arrive_expect_tx(&q_full[qb], static_cast<uint32_t>(R) * 256u);
+          for (int hg = 0; hg < group; ++hg)
+            for (int h = 0; h < 2; ++h)
+              ptx::tma_load_2d(qd + h * L::SLAB + hg * rps * 128, &tmap_q, &q_full[qb], (g * group + hg) * 128 + h * 64, b * rps);
+        }
+        return true;
+      };
+      TmCursor ck = c0, cv = c0;
+      for (int i = 0; i < 2 && ok && ck.w < pairs; ++i) {
+        ok = load(true, ck);
+        tm_cursor_next(p, pairs, ck);
+      }
+      while (ok && cv.w < pairs) {
+        ok = load(false, cv);
+        tm_cursor_next(p, pairs, cv);
+        if (ok && ck.w < pairs) {
+          ok = load(true, ck);
+          tm_cursor_next(p, pairs, ck);
+        }
+      }
+      if (!waited) ptx::grid_dep_wait();
+    }
+  } else if (warp_id == 5) {
+    // ------------------------------------------------------------------ MMA issue
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = tm_idesc(128, KT, false);
+      constexpr uint32_t idesc_pv = tm_idesc(128, 128, true);
+      bool ok = true;
+      int s = 0;
+      auto stage_ready = [&](uint32_t& addr) {
+        const int stage = s % L::STAGES;
+        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(s / L::STAGES) & 1u, abort_flag, p.error_word)) return -1;
+        addr = sbase + L::OFF_RING + stage * L::TILE;
+        ++s;
+        return stage;
+      };
+      auto qk = [&](const TmCursor& c) {  // S of tile c.g into S buffer c.g & 1
+        uint32_t kb;
+        const int stage = stage_ready(kb);
+        if (stage < 0) return false;
+        const int qb = c.qi & 1;
+        if (c.j == 0 && !ptx::mbar_wait(&q_full[qb], static_cast<uint32_t>(c.qi >> 1) & 1u, abort_flag, p.error_word)) return false;
+        ptx::tc_fence_after();
+        const uint32_t qa = sbase + L::OFF_Q + qb * L::TILE;
+        const uint32_t sd = tmem_base + L::COL_S + static_cast<uint32_t>((c.g & 1) * KT);
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk)
+          ptx::umma_bf16(sd, tm_desc_k(qa + (kk >> 2) * L::SLAB) + static_cast<uint64_t>(2 * (kk & 3)),
+                         tm_desc_k(kb + (kk >> 2) * L::SLAB) + static_cast<uint64_t>(2 * (kk & 3)), idesc_qk, kk > 0 ? 1u : 0u);
+        ptx::umma_commit(&kv_empty[stage]);
+        ptx::umma_commit(&s_full[c.g & 1]);
+        if (c.j == c.n_t - 1) ptx::umma_commit(&q_empty[qb]);
+        return true;
+      };
+      TmCursor ck = c0, cv = c0;
+      for (int i = 0; i < 2 && ok && ck.w < pairs; ++i) {
+        ok = qk(ck);
+        tm_cursor_next(p, pairs, ck);
+      }
+      while (ok && cv.w < pairs) {
+        ok = ptx::mbar_wait(&p_full[cv.g & 1], static_cast<uint32_t>(cv.g >> 1) & 1u, abort_flag, p.error_word);
+        if (!ok) break;
+        uint32_t vb;
+        const int stage = stage_ready(vb);
+        if (stage < 0) break;
+        ptx::tc_fence_after();
+        const uint32_t pcol = tmem_base + L::COL_S + static_cast<uint32_t>((cv.g & 1) * KT);  // P lies over its S
+#pragma unroll
+        for (int kk = 0; kk < KT / 16; ++kk)
+          ptx::umma_bf16_ts(tmem_base + L::COL_O, pcol + kk * 8, tm_desc_mn(vb + kk * 2048, L::SLAB, 1024), idesc_pv,
+                            (cv.j > 0 || kk > 0) ? 1u : 0u);
+        ptx::umma_commit(&kv_empty[stage]);
+        ptx::umma_commit(o_full);
+        tm_cursor_next(p, pairs, cv);
+        if (ck.w < pairs) {  // overwrites the S / P buffer of the tile just multiplied: issued after that product
+          ok = qk(ck);
+          tm_cursor_next(p, pairs, ck);
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ softmax warps
+    const int tid = threadIdx.x;  // row of the tile, tensor-memory lane, packed row head_in_group * rows_per_seq + r
+    const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(warp_id * 32) << 16);
+    const uint32_t t_o = t_lane + L::COL_O;
+    const int r_seq = tid % rps, hg = tid / rps;
+    bool alive = true;
+    ptx::grid_dep_wait();
+    for (TmCursor c = c0; c.w < pairs && alive;) {
+      const int b = c.w / p.hkv, g = c.w % p.hkv;
+      const int n_valid = p.rm.n_valid[b], kv_len = p.rm.kv_len[b];
+      const bool row_ok = tid < R && r_seq < n_valid;
+      const bool warp_rows = __any_sync(0xffffffffu, row_ok);
+      const int kv_lim = row_ok ? row_kv_limit(p.rm, b, r_seq, kv_len) : kv_len;
+      const int n_t = c.n_t;
+      float m_run = -INFINITY, l_run = 0.f;  // m_run: the reference of the exponentials (see the head of the file)
+      for (int j = 0; j < n_t && alive; ++j, tm_cursor_next(p, pairs, c)) {
+        const int gt = c.g;
+        alive = ptx::mbar_wait(&s_full[gt & 1], static_cast<uint32_t>(gt >> 1) & 1u, abort_flag, p.error_word);
+        if (!alive) break;
+        // every thread watches every phase of o_full in order (a parity wait cannot tell a phase from the one two before)
+        auto seen_o = [&]() { return gt == 0 || ptx::mbar_wait(o_full, static_cast<uint32_t>(gt - 1) & 1u, abort_flag, p.error_word); };
+        if (!warp_rows) {
+          alive = seen_o();
+          ptx::mbar_arrive(&p_full[gt & 1]);
+          continue;
+        }
+        ptx::tc_fence_after();
+        const int j0 = j * KT;
+        const uint32_t t_s = t_lane + L::COL_S + static_cast<uint32_t>((gt & 1) * KT);
+        float s[NCH][32];
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch) ptx::tmem_ld_32x32(t_s + ch * 32, s[ch]);
+        ptx::tmem_ld_wait();
+        if (!__all_sync(0xffffffffu, j0 + KT <= kv_lim)) {
+#pragma unroll
+          for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+            for (int cc = 0; cc < 32; ++cc)
+              if (j0 + ch * 32 + cc >= kv_lim) s[ch][cc] = -INFINITY;
+        }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+        for (int ch = 0; ch < NCH; ++ch)
+#pragma unroll
+          for (int cc = 0; cc < 32; ++cc) mx4[cc & 3] = fmaxf(mx4[cc & 3], s[ch][cc]);
+        const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.scale_log2;
+        const bool move = mx > m_run + TM_SLACK_LOG2;
+        const bool resc = move && m_run != -INFINITY;
+        if (j > 0 && __any_sync(0xffffffffu, resc)) {
+          alive = seen_o();  // O holds the sum over the pair's tiles before this one
+          if (!alive) break;
+          ptx::tc_fence_after();
+          const float f = resc ? exp2f(m_run - mx) : 1.f;
+#pragma unroll
+          for (int c4 = 0; c4 < 4; ++c4) {
+            float o[32];
+            ptx::tmem_ld_32x32(t_o + c4 * 32, o);
+            ptx::tmem_ld_wait();
+#pragma unroll
+            for (int cc = 0; cc < 32; ++cc) o[cc] *= f;
+            ptx::tmem_st_32x32(t_o + c4 * 32, o);
+          }
+        }
+        if (move) {
+          if (resc) l_run *= exp2f(m_run - mx);
+          m_run = mx;
+        }
+        const float nbase = m_run == -INFINITY ? 0.f : -m_run;
+        float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int h = 0; h < NCH / 2; ++h) {
+          uint32_t v[32];
+#pragma unroll
+          for (int jj = 0; jj < 32; ++jj) {
+            const float p0 = ptx::ex2_approx(fmaf(s[h * 2 + (jj >> 4)][(jj & 15) * 2], p.scale_log2, nbase));
+            const float p1 = ptx::ex2_approx(fmaf(s[h * 2 + (jj >> 4)][(jj & 15) * 2 + 1], p.scale_log2, nbase));
+            sum4[jj & 3] += p0 + p1;
+            v[jj] = pack_bf16(p0, p1);
+          }
+          ptx::tmem_st_32x32(t_s + h * 32, *reinterpret_cast<const float(*)[32]>(v));
+        }
+        l_run += (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+        alive = seen_o();
+        ptx::tmem_st_wait();
+        ptx::tc_fence_before();
+        ptx::mbar_arrive(&p_full[gt & 1]);
+      }
+      if (!alive) break;
+      // ---- the pair's rows of O (c now stands on the first tile of the next pair: the last tile was c.g - 1)
+      alive = ptx::mbar_wait(o_full, static_cast<uint32_t>(c.g - 1) & 1u, abort_flag, p.error_word);
+      if (!alive) break;
+      if (warp_rows) {
+        ptx::tc_fence_after();
+        float acc[128];
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) ptx::tmem_ld_32x32(t_o + c4 * 32, *reinterpret_cast<float(*)[32]>(acc + c4 * 32));
+        ptx::tmem_ld_wait();
+        ptx::tc_fence_before();  // the next pair's first P (and with it the product that overwrites O) comes after this
+        if (row_ok) {
+          const float inv = 1.0f / l_run;
+          __nv_bfloat16* o = p.out + (static_cast<size_t>(b) * rps + r_seq) * p.hq * 128 + (g * group + hg) * 128;
+#pragma unroll
+          for (int d = 0; d < 128; d += 8)
+            *reinterpret_cast<uint4*>(o + d) =
+                make_uint4(pack_bf16(acc[d] * inv, acc[d + 1] * inv), pack_bf16(acc[d + 2] * inv, acc[d + 3] * inv),
+                           pack_bf16(acc[d + 4] * inv, acc[d + 5] * inv), pack_bf16(acc[d + 6] * inv, acc[d + 7] * inv));
+        }
+      }
+    }
+  }
+  __syncwarp();
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp_id == 5) ptx::tmem_dealloc<512>(tmem_base);
+}
+
 }  // namespace attn
 }  // namespace d3

@@ -1134,6 +1134,41 @@ int launch_attn_tmem(d3_ctx* c, const attn::AttnTcParams& p, dim3 grid) {
   return D3_OK;
 }
 
+// Decode-sized batches with several (sequence, kv head) pairs per SM: one persistent CTA per SM streams through its pairs.
+bool attn_stream_usable(const d3_ctx* c, const RowMap& rm) {
+  const d3_config& g = c->cfg;
+  const int R = (g.n_q_heads / g.n_kv_heads) * rm.rows_per_seq;
+  return R <= 128 && rm.rows_per_seq % 8 == 0 && rm.rows_per_seq <= 256 &&
+         static_cast<long long>(rm.bs) * rm.rows_per_seq < (1ll << 31);
+}
+int run_attention_tmem_stream(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
+  const d3_config& g = c->cfg;
+  auto kern = attn::attn_tmem_stream_kernel;
+  const size_t smem = attn::TmStream::smem_bytes();
+  static bool attr_set = false;
+  if (!attr_set) {
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    attr_set = true;
+  }
+  attn::AttnTcParams p{};
+  p.q = static_cast<const bf16*>(q);
+  p.out = static_cast<bf16*>(out);
+  p.rm = rm;
+  p.hq = g.n_q_heads; p.hkv = g.n_kv_heads; p.max_seq = g.max_seq;
+  const long long plane_rows = static_cast<long long>(g.max_batch) * g.n_kv_heads * g.max_seq;
+  p.k_row0 = (static_cast<long long>(layer) * 2 + 0) * plane_rows;
+  p.v_row0 = (static_cast<long long>(layer) * 2 + 1) * plane_rows;
+  p.n_splits = 1;
+  p.scale_log2 = 1.4426950408889634f / std::sqrt(static_cast<float>(g.d_head));
+  p.error_word = c->error_word;
+  const CUtensorMap* tq;
+  TRY(get_tmap(c, q, rm.bs * rm.rows_per_seq, g.n_q_heads * 128, rm.rows_per_seq, &tq));
+  const int pairs = rm.bs * g.n_kv_heads;
+  CUDA_TRY(c, launch_pdl(c, kern, dim3(static_cast<unsigned>(std::min(c->n_sms, pairs))), dim3(attn::TM_THREADS), smem, c->kv_tmap128, *tq, p));
+  LAUNCHED(c, "attn_tmem_stream_kernel");
+  return D3_OK;
+}
+
 int run_attention_tmem(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
   const d3_config& g = c->cfg;
   const int group = g.n_q_heads / g.n_kv_heads;
@@ -1183,6 +1218,9 @@ int run_attention_tc(d3_ctx* c, const void* q, int layer, void* out, const RowMa
   // is the faster one (measured: 60-70 against 84-110 us per layer at 64 rows x 4200-5100 keys, 27 against 33-37 at
   // 224 rows x 550-1000 keys, a third of the time on 4096-row prompts); at 32 rows the two are level on batches and
   // the mma.sync kernel, with its cheaper start, is ahead on a single sequence (15 against 19 us).
+  if (c->tune_attn_shape == 2 ? attn_stream_usable(c, rm)
+                              : (c->tune_attn_tmem < 0 && attn_stream_usable(c, rm) && rm.bs * g.n_kv_heads >= 2 * c->n_sms))
+    return run_attention_tmem_stream(c, q, layer, out, rm);
   if (c->tune_attn_tmem == 1 || (c->tune_attn_tmem < 0 && R >= 64)) return run_attention_tmem(c, q, layer, out, rm);
   const int nw = R <= 32 ? 2 : (R <= 64 ? 4 : 8);
   const int q_tiles = (R + nw * 16 - 1) / (nw * 16);
@@ -2176,7 +2214,7 @@ extern "C" int d3_set_tuning(d3_ctx* c, const d3_tuning* t) {
       t->cluster_k_split < -1 || t->cluster_k_split > 0 || t->row_tile_pairs < -1 || t->row_tile_pairs > 1 ||
       (t->round_robin != 0 && t->round_robin != 1) || t->column_strips < 0 || t->column_strips > 3 || t->strip_stages < 0 ||
       t->strip_stages > 32 || t->chain < -1 || t->chain > 0 || t->chain_clusters < 0 || t->chain_l2_ahead < -1 || t->chain_l2_ahead > 256 || t->weights_as_rows < -1 || t->weights_as_rows > 0 ||
-      ((t->attention_tmem < -1 || t->attention_tmem > 1) && t->attention_tmem != 64 && t->attention_tmem != 128) ||
+      ((t->attention_tmem < -1 || t->attention_tmem > 2) && t->attention_tmem != 64 && t->attention_tmem != 128) ||
       t->cta_pairs < -1 || t->cta_pairs > 0)
     return fail(c, D3_ERR_INVALID_ARG, "d3_set_tuning: a field is outside its range");
   c->tune_ring_kb = t->ring_kb;

@@ -383,6 +383,30 @@ def test_attention_bf16_tensor_memory(shape, rows, kv_lens, keys_per_tile):
         _attention_case(ctx, shape, True, 3, rows, kv_lens, 7 + rows + sum(kv_lens), ramp=0.05)
 
 
+ATT_GQA2 = si.scaled_shape(si.QWEN7B, name="att-gqa2", n_layers=1, d_model=256, n_q_heads=4, n_kv_heads=2,
+                           d_ffn=256, vocab=1000, d_head=128)
+
+
+@pytest.mark.parametrize("shape,rows,bs", [(ATT_MHA, 32, 64), (ATT_MHA, 64, 50), (ATT_GQA2, 32, 90), (ATT_GQA2, 64, 3),
+                                           (ATT_MHA, 8, 120), (ATT_MHA, 128, 70)], ids=["mha32", "mha64", "gqa2x32", "gqa2x64", "mha8", "mha128"])
+def test_attention_bf16_tensor_memory_persistent(shape, rows, bs):
+    """The persistent form: one CTA per SM walks through its (sequence, kv head) pairs and treats their key tiles as
+    one stream.  More pairs than SMs (CTAs with one, two and three pairs) and fewer, ragged key ranges from 1 key to
+    5 tiles, one or two query heads per kv head, part-filled and full 128-row tiles; then the row maxima that keep
+    rising."""
+    rng = np.random.default_rng(rows + bs)
+    kv_lens = [int(v) for v in rng.integers(1, 640, size=bs)]
+    kv_lens[1] = 640
+    kv_lens[2] = 128
+    kv_lens[5 % bs] = 1
+    with Ctx(shape, None, block=32, max_batch=bs, max_seq=640, max_prefill_rows=bs * rows) as ctx:
+        d3.d3_set_tuning(ctx.ctx, attention_tmem=2)
+        _attention_case(ctx, shape, True, bs, rows, kv_lens, rows + bs)
+        _attention_case(ctx, shape, True, bs, rows, kv_lens, rows + bs)
+        assert d3.d3_launch_count_of(ctx.ctx, "attn_tmem_stream_kernel") == 2
+        _attention_case(ctx, shape, True, bs, rows, kv_lens, 7 + rows + bs, ramp=0.05)
+
+
 @pytest.mark.parametrize("rows,kv_lens", [(16, [48, 17]), (5, [5, 200])])
 def test_attention_fp32(ctx_f32, rows, kv_lens):
     _attention_case(ctx_f32, F32_SHAPE, False, 2, rows, kv_lens, rows)
