@@ -446,13 +446,19 @@ static_assert(TmLayout<64, 2>::OFF_BAR >= 128 * PART_LD * 4, "the partials of th
 // blockIdx.x, blockIdx.x + gridDim.x, ...) and treats their key tiles as one stream: the producer runs ahead across
 // pair borders (K/V ring, and the next pair's Q by TMA into the second Q buffer), the MMA thread issues the first
 // products of the next pair while the softmax threads read out O of the pair before, and nothing is set up twice.
-// 128-key tiles, two S buffers, Q in shared memory (two buffers of two K-major slabs), four ring stages.
+// 128-key tiles, two S buffers, Q in shared memory (two buffers of two K-major slabs), five ring stages.
+// Shared memory: two Q buffers of two whole 128-row slabs each (64 KB), five 32 KB ring stages, the barriers.
+// (Q buffers cut down to the rows a pair has, so that the 128-row A operand reads on into the other buffer and the
+// ring, made room for a sixth stage and cost 10 % of the kernel's speed; a fifth stage over four gained nothing.)
 struct TmStream {
-  static constexpr int KT = 128, STAGES = 4;
+  static constexpr int KT = 128, MAX_STAGES = 5;
   static constexpr uint32_t SLAB = 128u * 128u, TILE = 2u * SLAB;
-  static constexpr uint32_t OFF_Q = 0, OFF_RING = 2u * TILE, OFF_BAR = OFF_RING + STAGES * TILE;
   static constexpr uint32_t COL_S = 0, COL_O = 256;
-  static constexpr size_t smem_bytes() { return 1024 + OFF_BAR + (2 * STAGES + 9) * 8 + 64; }
+  static __host__ __device__ uint32_t q_slab(int) { return SLAB; }
+  static __host__ __device__ uint32_t off_ring(int R) { return 4u * q_slab(R); }
+  static __host__ __device__ int stages(int) { return MAX_STAGES; }
+  static __host__ __device__ uint32_t off_bar(int R) { return off_ring(R) + static_cast<uint32_t>(stages(R)) * TILE; }
+  static size_t smem_bytes(int R) { return 1024 + off_bar(R) + (2 * MAX_STAGES + 9) * 8 + 64; }
 };
 
 // Position in the stream of key tiles of this CTA's pairs: pairs without live rows or keys are passed over.
@@ -489,9 +495,16 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const _
   constexpr int KT = L::KT, NCH = KT / 32;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
-  uint64_t* kv_empty = kv_full + L::STAGES;
-  uint64_t* s_full = kv_empty + L::STAGES;  // [2]
+  const int warp_id = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int group = p.hq / p.hkv;
+  const int rps = p.rm.rows_per_seq;
+  const int R = group * rps;
+  const int pairs = p.rm.bs * p.hkv;
+  const int n_stages = L::stages(R);
+  const uint32_t q_slab = L::q_slab(R), off_ring = L::off_ring(R);
+  uint64_t* kv_full = reinterpret_cast<uint64_t*>(smem + L::off_bar(R));
+  uint64_t* kv_empty = kv_full + L::MAX_STAGES;
+  uint64_t* s_full = kv_empty + L::MAX_STAGES;  // [2]
   uint64_t* p_full = s_full + 2;            // [2]
   uint64_t* q_full = p_full + 2;            // [2] Q of a pair in its buffer
   uint64_t* q_empty = q_full + 2;           // [2] the pair's last first product has read it
@@ -499,16 +512,11 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const _
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(o_full + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-  const int warp_id = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int group = p.hq / p.hkv;
-  const int rps = p.rm.rows_per_seq;
-  const int R = group * rps;
-  const int pairs = p.rm.bs * p.hkv;
 
   if (threadIdx.x == 0) {
     ptx::prefetch_tensormap(&tmap_kv);
     ptx::prefetch_tensormap(&tmap_q);
-    for (int s = 0; s < L::STAGES; ++s) {
+    for (int s = 0; s < n_stages; ++s) {
       ptx::mbar_init(&kv_full[s], 1);
       ptx::mbar_init(&kv_empty[s], 1);
     }
@@ -545,9 +553,9 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const _
       bool waited = false, ok = true;
       int s = 0;  // position in the ring
       auto load = [&](bool is_k, const TmCursor& c) {
-        const int stage = s % L::STAGES;
-        if (s >= L::STAGES &&
-            !ptx::mbar_wait(&kv_empty[stage], static_cast<uint32_t>(s / L::STAGES - 1) & 1u, abort_flag, p.error_word))
+        const int stage = s % n_stages;
+        if (s >= n_stages &&
+            !ptx::mbar_wait(&kv_empty[stage], static_cast<uint32_t>(s / n_stages - 1) & 1u, abort_flag, p.error_word))
           return false;
         const int b = c.w / p.hkv, g = c.w % p.hkv;
         const int j0 = c.j * KT;
@@ -555,7 +563,7 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const _
           ptx::grid_dep_wait();
           waited = true;
         }
-        uint8_t* dst = smem + L::OFF_RING + stage * L::TILE;
+        uint8_t* dst = smem + off_ring + stage * L::TILE;
         const long long plane = (static_cast<long long>(b) * p.hkv + g) * p.max_seq;
         const int row = static_cast<int>((is_k ? p.k_row0 : p.v_row0) + plane + j0);
         ptx::mbar_arrive_expect_tx(&kv_full[stage], L::TILE);
@@ -570,11 +578,11 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const _
           const int qb = c.qi & 1;
           if (c.qi >= 2 && !ptx::mbar_wait(&q_empty[qb], static_cast<uint32_t>((c.qi >> 1) - 1) & 1u, abort_flag, p.error_word))
             return false;
-          uint8_t* qd = smem + L::OFF_Q + qb * L::TILE;
+          uint8_t* qd = smem + qb * 2 * q_slab;
           ptx::mbar_arrive_expect_tx(&q_full[qb], static_cast<uint32_t>(R) * 256u);
           for (int hg = 0; hg < group; ++hg)
             for (int h = 0; h < 2; ++h)
-              ptx::tma_load_2d(qd + h * L::SLAB + hg * rps * 128, &tmap_q, &q_full[qb], (g * group + hg) * 128 + h * 64, b * rps);
+              ptx::tma_load_2d(qd + h * q_slab + hg * rps * 128, &tmap_q, &q_full[qb], (g * group + hg) * 128 + h * 64, b * rps);
         }
         return true;
       };
@@ -601,9 +609,9 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const _
       bool ok = true;
       int s = 0;
       auto stage_ready = [&](uint32_t& addr) {
-        const int stage = s % L::STAGES;
-        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(s / L::STAGES) & 1u, abort_flag, p.error_word)) return -1;
-        addr = sbase + L::OFF_RING + stage * L::TILE;
+        const int stage = s % n_stages;
+        if (!ptx::mbar_wait(&kv_full[stage], static_cast<uint32_t>(s / n_stages) & 1u, abort_flag, p.error_word)) return -1;
+        addr = sbase + off_ring + stage * L::TILE;
         ++s;
         return stage;
       };
@@ -614,11 +622,11 @@ __global__ void __launch_bounds__(TM_THREADS, 1) attn_tmem_stream_kernel(const _
         const int qb = c.qi & 1;
         if (c.j == 0 && !ptx::mbar_wait(&q_full[qb], static_cast<uint32_t>(c.qi >> 1) & 1u, abort_flag, p.error_word)) return false;
         ptx::tc_fence_after();
-        const uint32_t qa = sbase + L::OFF_Q + qb * L::TILE;
+        const uint32_t qa = sbase + qb * 2 * q_slab;
         const uint32_t sd = tmem_base + L::COL_S + static_cast<uint32_t>((c.g & 1) * KT);
 #pragma unroll
         for (int kk = 0; kk < 8; ++kk)
-          ptx::umma_bf16(sd, tm_desc_k(qa + (kk >> 2) * L::SLAB) + static_cast<uint64_t>(2 * (kk & 3)),
+          ptx::umma_bf16(sd, tm_desc_k(qa + (kk >> 2) * q_slab) + static_cast<uint64_t>(2 * (kk & 3)),
                          tm_desc_k(kb + (kk >> 2) * L::SLAB) + static_cast<uint64_t>(2 * (kk & 3)), idesc_qk, kk > 0 ? 1u : 0u);
         ptx::umma_commit(&kv_empty[stage]);
         ptx::umma_commit(&s_full[c.g & 1]);

@@ -1144,10 +1144,10 @@ bool attn_stream_usable(const d3_ctx* c, const RowMap& rm) {
 int run_attention_tmem_stream(d3_ctx* c, const void* q, int layer, void* out, const RowMap& rm) {
   const d3_config& g = c->cfg;
   auto kern = attn::attn_tmem_stream_kernel;
-  const size_t smem = attn::TmStream::smem_bytes();
+  const size_t smem = attn::TmStream::smem_bytes((g.n_q_heads / g.n_kv_heads) * rm.rows_per_seq);
   static bool attr_set = false;
   if (!attr_set) {
-    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    CUDA_TRY(c, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(attn::TmStream::smem_bytes(64))));
     attr_set = true;
   }
   attn::AttnTcParams p{};
