@@ -447,6 +447,12 @@ static_assert(TmLayout<64, 2>::OFF_BAR >= 128 * PART_LD * 4, "the partials of th
 // pair borders (K/V ring, and the next pair's Q by TMA into the second Q buffer), the MMA thread issues the first
 // products of the next pair while the softmax threads read out O of the pair before, and nothing is set up twice.
 // 128-key tiles, two S buffers, Q in shared memory (two buffers of two K-major slabs), five ring stages.
+// (A tile row is a tensor-memory lane and a lane quadrant belongs to one scheduler partition, so 32 live rows use a
+// quarter of the SM's exponential rate: about 2200 clocks per 128-key tile on the one warp, against 2750 for the
+// tile's 64 KB at an SM's share of HBM.  A form with 2 or 4 copies of the rows in the tile, each copy taking a part
+// of every tile's keys, with one reference per row agreed through shared memory and the copies' parts of O added
+// there after the pair's last tile, was built and passed the same tests, but was slower (77-79 and 98-103 us per
+// layer against 72-73 and 92-93): a barrier per tile and eight per pair cost more than the exponentials saved.)
 // Shared memory: two Q buffers of two whole 128-row slabs each (64 KB), five 32 KB ring stages, the barriers.
 // (Q buffers cut down to the rows a pair has, so that the 128-row A operand reads on into the other buffer and the
 // ring, made room for a sixth stage and cost 10 % of the kernel's speed; a fifth stage over four gained nothing.)
