@@ -49,7 +49,7 @@ typedef struct d3_tuning {
                                that many keys per tile (two CTAs per SM / one) instead of the launcher's choice, 2 = the persistent
                                form (one CTA per SM streams through its (sequence, kv head) pairs) wherever all packed rows
                                of a pair fit one 128-row tile, whatever the number of pairs */
-  int32_t cta_pairs;        /* matmuls of at least 512 rows on tiled weights run 256 x 256 tiles on pairs of CTAs that share
+  int32_t cta_pairs;        /* matmuls of more than 128 rows on tiled weights run 256 x 256 tiles on pairs of CTAs that share
                                one MMA (cta_group::2, gemm_pair_kernel): -1 = when the shape allows (default), 0 never */
 } d3_tuning;
 void d3_tuning_defaults(d3_tuning *t);

@@ -1,4 +1,4 @@
-// Wide matmuls (Y = X W^T with at least 512 rows) on CTA pairs: a cluster of two CTAs owns a 256 x 256 tile of Y and
+// Matmuls Y = X W^T of more than 128 rows on CTA pairs: a cluster of two CTAs owns a 256 x 256 tile of Y and
 // one tcgen05.mma.cta_group::2 of M = 256 computes it.  Each CTA stages its own 128 rows of X (TMA) and its own
 // 128 of the tile's 256 weight rows (one pre-swizzled 16 KB block) per 64-wide K slab, both by TMA: 32 KB of shared
 // memory traffic per CTA and slab where a lone CTA with a 128 x 256 tile moves 48 KB for the same arithmetic.  The

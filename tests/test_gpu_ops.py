@@ -142,9 +142,10 @@ def test_linear_bf16_weights_as_rows(ctx_bf16, m, n, k, cluster):
 
 
 @pytest.mark.parametrize("m,n,k", [(512, 256, 64), (1024, 512, 512), (640, 768, 1024), (1000, 256, 4096), (2048, 4096, 1024),
-                                   (513, 12288, 256)])
+                                   (513, 12288, 256), (256, 19200, 128), (130, 19200, 64)])
 def test_linear_bf16_cta_pairs(ctx_bf16, m, n, k):
-    """Matmuls of at least 512 rows on tiled weights: 256 x 256 tiles, each computed by one MMA of 256 rows that a
+    """Matmuls of more than 128 rows on tiled weights (the 130- and 256-row cases have more column tiles than the
+    weights-as-rows kernel takes): 256 x 256 tiles, each computed by one MMA of 256 rows that a
     pair of CTAs shares (each stages its own 128 rows of X and 128 of the tile's weight rows).  Row counts that end
     inside the leader's half, inside the peer's half and on a tile border; one K slab and many; more tiles than
     pairs (two accumulators in turn) and fewer; fp32, residual, bf16 and SwiGLU epilogues against the fp64 product,
