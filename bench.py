@@ -354,7 +354,7 @@ def measure_batched(name, W, dev, local, world, dist, peaks, steps):
                    "ms_per_forward": ms_fwd, "prefill_ms": ms_prefill},
         "roofline": {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                      "frac": achieved / peaks["bf16_tflops_sustained"], "traffic": None,
-                     "kernel": "gemm_pair_kernel and, for the LM head, gemm_tc_kernel (all matmul launches of the decode loop, CUDA events around every launch, launched serialized)",
+                     "kernel": "gemm_pair_kernel (all matmul launches of the decode loop, LM head included; CUDA events around every launch, launched serialized)",
                      "peak_source": f"of {peaks['source']} (sustained)", "launches": n_gemm, "avg_launch_us": 1e3 * tot_ms / max(n_gemm, 1),
                      "flops_per_launch": tot_flops / max(n_gemm, 1),
                      "step_effective": {"TFLOP/s": fwd_flops / (ms_fwd / 1e3) / 1e12,

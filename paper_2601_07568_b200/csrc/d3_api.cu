@@ -923,7 +923,7 @@ int launch_pair(d3_ctx* c, const CUtensorMap* tx, const CUtensorMap* tw, const t
 bool pair_usable(const d3_ctx* c, int M, int N, int K, int epi, int w_tiled) {
   // from 129 rows on: at 129..256 rows a pair's tile holds all rows, so every weight block is staged once (measured
   // at 256 rows: QKV 58 -> 41 us and gate/up 77 -> 60 us per launch on the 8B shape, gate/up 69 -> 58 on the 7B one)
-  return c->tune_cta_pairs != 0 && w_tiled && M > 128 && N % 256 == 0 && K % 64 == 0 && epi != EPI_STATS &&
+  return c->tune_cta_pairs != 0 && w_tiled && M > 128 && N % 256 == 0 && K % 64 == 0 &&
          static_cast<long long>(N / 128) * (K / 64) * 128 < (1ll << 31);
 }
 
@@ -956,6 +956,7 @@ int run_linear_pair(d3_ctx* c, const void* X, const void* W, int M, int N, int K
     case EPI_RESID: return launch_pair<EPI_RESID>(c, tx, tw, p, tiles);
     case EPI_SWIGLU: return launch_pair<EPI_SWIGLU>(c, tx, tw, p, tiles);
     case EPI_QKV: return launch_pair<EPI_QKV>(c, tx, tw, p, tiles);
+    case EPI_STATS: return launch_pair<EPI_STATS>(c, tx, tw, p, tiles);
   }
   return fail(c, D3_ERR_INVALID_ARG, "unknown epilogue");
 }
