@@ -544,6 +544,29 @@ def test_small_bf16_ragged_batch_step_locked(d_head, hq, hkv, impl):
             assert r2["resyncs"] <= r2["blocks"] and max(r2["margins"], default=0.0) <= 1e-2, r2
 
 
+def test_small_bf16_batch_on_cta_pairs_step_locked():
+    """Six sequences x 32 rows = 192 rows per decode forward, 768 padded rows in the prefill, and a vocabulary and
+    widths that are multiples of 256: QKV (RoPE + cache write), gate/up (SwiGLU) and the LM head (fused statistics)
+    run on CTA pairs, attention of the prefill on the tensor-memory kernel.  Step-locked against the oracle."""
+    shape = si.scaled_shape(si.LLADA8B, name="small-pairs", n_layers=3, d_model=256, n_q_heads=4, n_kv_heads=2,
+                            d_ffn=640, vocab=1024, d_head=128)
+    W = si.gen_weights(shape)
+    wl, ids, lens = si.small_workload("small-pairs", shape, 6, [40, 7, 97, 64, 33, 128], 64, 32, 0.9, 78)
+    model = o.model_from_shape(shape, W, np.float32, mirror_bf16=True)
+    exact = o.model_from_shape(shape, W, np.float32)
+    with Ctx(shape, W, block=32, max_batch=6, max_seq=wl.max_seq) as ctx:
+        rep, traces = step_locked(ctx, model, ids, lens, 64, 32, 0.9, logit_tol=3e-2, exact_model=exact)
+        record_report("small_bf16_step_locked_on_cta_pairs", rep)
+        assert rep["max_logit_err"] <= 3e-2
+        assert_rounding_bounded(rep, BF16_STAT_ERR_BOUND)
+        assert d3.d3_launch_count_of(ctx.ctx, "gemm_pair_kernel") > 0
+        assert d3.d3_launch_count_of(ctx.ctx, "attn_tmem_kernel") > 0
+        ctx.prefill(ids, lens)
+        tok, cs, st = ctx.generate(6, 64, 0.9)
+        assert st.tokens_committed == 6 * 64
+        assert ctx.error_word() == 0
+
+
 def test_small_bf16_model_width_not_a_multiple_of_the_tiles():
     """d_model = 200: ragged K slab (200 = 3 x 64 + 8), ragged 128-column output tile, a last chunk of
     8 columns in the sums of squares of the folded RMSNorm, ragged vocabulary."""
