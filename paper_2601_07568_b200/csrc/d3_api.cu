@@ -120,6 +120,8 @@ struct d3_ctx {
   int tune_chain_l2 = -1;       // weight slabs the chain's L2 prefetch runs ahead (-1: default, 0: off)
   int tune_attn_shape = 0;      // experiment: keys per tile of the tcgen05 attention (0 = by rule, 64, 128)
   int tune_attn_tmem = -1;      // tcgen05 attention: -1 where measured faster, 0 never, 1 wherever the shape allows
+  const int* live_n_valid = nullptr;  // set for the span of a forward whose sequences have rows_per_seq % 256 == 0 rows
+  int live_rps = 0, live_rows = 0;    // (padded prompts): the pair kernel passes over row tiles without a live row
   int tune_cta_pairs = -1;      // wide matmuls on CTA pairs (cta_group::2): -1 when the shape allows, 0 never
   int pair_clusters = 0;        // CTA pairs of gemm_pair_kernel resident at once (asked once)
   int tune_xt = -1;             // 129..256-row matmuls with weights as the 128-row operand: -1 when the shape allows, 0 never
@@ -940,6 +942,10 @@ int run_linear_pair(d3_ctx* c, const void* X, const void* W, int M, int N, int K
   p.w_packed = static_cast<const bf16*>(W);
   p.w_blocks = static_cast<long long>(N / 128) * p.k_chunks;
   p.ep = ep;
+  if (c->live_n_valid != nullptr && M == c->live_rows) {
+    p.live_n_valid = c->live_n_valid;
+    p.live_rps = c->live_rps;
+  }
   if (qx) {
     p.rope_cos = c->rope_cos; p.rope_sin = c->rope_sin;
     p.pos_base = qx->rm.pos_base; p.n_valid = qx->rm.n_valid; p.rows_per_seq = qx->rm.rows_per_seq;
@@ -1317,6 +1323,15 @@ int forward(d3_ctx* c, const int* ids, int bs, int rows_per_seq, int head, float
   const int d = g.d_model, nq = g.n_q_heads * g.d_head, nkv = g.n_kv_heads * g.d_head, f = g.d_ffn;
   RowMap rm{c->pos_base, c->n_valid, c->kv_len, rows_per_seq, bs, seg};
   c->last_rows = M;
+  // Padded prompts: the matmuls on CTA pairs pass over 256-row tiles that hold no live row of their sequence (rows
+  // beyond n_valid are computed by nobody's reader: attention, the cache write and the decisions skip them already).
+  struct LiveRows {
+    d3_ctx* c;
+    LiveRows(d3_ctx* c_, const int* n_valid, int rps, int rows) : c(c_) {
+      if (rps % 256 == 0) { c->live_n_valid = n_valid; c->live_rps = rps; c->live_rows = rows; }
+    }
+    ~LiveRows() { c->live_n_valid = nullptr; c->live_rps = 0; c->live_rows = 0; }
+  } live_rows(c, c->n_valid, rows_per_seq, M);
 
   {
     ProfScope ps(c, D3_PROF_OTHER);

@@ -73,6 +73,13 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
   const int tiles = m_tiles * n_tiles;
   const int my_tiles = pair < tiles ? (tiles - pair + n_pairs - 1) / n_pairs : 0;
   const int KC = p.k_chunks;
+  // A row tile that lies wholly in the unused tail of a sequence's rows (padded prompts) is passed over by all three
+  // roles alike.  (The row map was written before the forward's first kernel started: readable before the dependency wait.)
+  auto tile_dead = [&](int m_t) {
+    if (p.live_n_valid == nullptr) return false;
+    const int row0 = m_t * 256;
+    return row0 % p.live_rps >= p.live_n_valid[row0 / p.live_rps];
+  };
 
   if (threadIdx.x == 0) {
     prefetch_tensormap(&tmap_x);
@@ -107,6 +114,7 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
         const int q = pair + t * n_pairs;
         int m_t, n_t;
         pair_tile_mn(q, m_tiles, n_tiles, m_t, n_t);
+        if (tile_dead(m_t)) continue;
         const int row0 = m_t * 256 + static_cast<int>(rank) * 128;
         const int wrow0 = (n_t * 2 + static_cast<int>(rank)) * KC * 128;  // first row of this CTA's first weight block
         for (int kc = 0; kc < KC; ++kc, ++it) {
@@ -130,9 +138,13 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
         const uint32_t sb = smem_u32(smem);
         int it = 0;
         bool ok = true;
+        int n_done = 0;  // tiles computed so far: accumulator buffer and barrier phases
         for (int t = 0; t < my_tiles && ok; ++t) {
-          const int buf = t & 1;
-          if (t >= 2) ok = mbar_wait_cluster(&acc_empty[buf], static_cast<uint32_t>((t >> 1) - 1) & 1u, abort_flag, p.error_word);
+          int m_t, n_t;
+          pair_tile_mn(pair + t * n_pairs, m_tiles, n_tiles, m_t, n_t);
+          if (tile_dead(m_t)) continue;
+          const int buf = n_done & 1;
+          if (n_done >= 2) ok = mbar_wait_cluster(&acc_empty[buf], static_cast<uint32_t>((n_done >> 1) - 1) & 1u, abort_flag, p.error_word);
           if (!ok) break;
           tc_fence_after();
           const uint32_t tmem_d = tmem_base + static_cast<uint32_t>(buf * 256);
@@ -151,6 +163,7 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
             umma_commit_pair(&empty_bar[s], 3);
           }
           if (ok) umma_commit_pair(&acc_full[buf], 3);
+          ++n_done;
         }
       }
     }
@@ -159,15 +172,17 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
     grid_dep_wait();  // residual rows, positions and row sums come from earlier kernels
     const int lg = warp & 3;
     const int row = lg * 32 + lane;
+    int n_done = 0;
     for (int t = 0; t < my_tiles; ++t) {
       const int q = pair + t * n_pairs;
       int m_t, n_t;
       pair_tile_mn(q, m_tiles, n_tiles, m_t, n_t);
+      if (tile_dead(m_t)) continue;
       const int m = m_t * 256 + static_cast<int>(rank) * 128 + row;
-      const int buf = t & 1;
+      const int buf = n_done & 1;
       float rs = 1.f;  // folded RMSNorm: the row's factor, fetched while the MMAs still run
       if (p.ep.ssq_in != nullptr && m < p.M) rs = row_rstd(p.ep, m);
-      bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(t >> 1) & 1u, abort_flag, p.error_word);
+      bool ok = mbar_wait(&acc_full[buf], static_cast<uint32_t>(n_done >> 1) & 1u, abort_flag, p.error_word);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -177,6 +192,7 @@ __global__ void __launch_bounds__(PAIR_THREADS, 1) gemm_pair_kernel(const __grid
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_remote(&acc_empty[buf], 0);
+      ++n_done;
     }
   }
   // Neither CTA may leave (its shared memory is an operand of the leader's MMAs, its barriers a target of the

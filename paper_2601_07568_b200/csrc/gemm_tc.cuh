@@ -57,6 +57,10 @@ struct GemmParams {
   long long w_blocks;             // number of 128 x 64 blocks in w_packed
   int w_tiled;           // 0: W row-major [N, K]; 1: W stored as contiguous [128 x 64] blocks, block (n_tile, kc) at
                          // row (n_tile * k_chunks + kc) * 128 of a [rows, 64] array (see pack_tiled_kernel)
+  // pair kernel, optional: rows are laid out as sequences of live_rps rows (a multiple of 256) of which the first
+  // live_n_valid[sequence] are in use; a 256-row tile without a live row is not computed
+  const int* live_n_valid;
+  int live_rps;
   EpiParams ep;
   // EPI_QKV only
   const float* rope_cos;  // [max_seq][64]
